@@ -1,0 +1,419 @@
+#!/usr/bin/env python
+"""Benchmark of the mixed-batch multi-LoRA layer on B200.
+
+A "step" is one pass of the whole hot path - shrink, fused base GEMM + LoRA expand with
+activation save, then the LoRA backward (V, dB, dA, dX) - over one synthetic mixed batch, for
+every projection of the workload.  The default workload is the Llama-3-8B-shaped decoder-layer
+projection set (q, k, v, o, gate, up, down; 32 adapters of rank 16; 4096 rows of which 1024 are
+decode rows and 2048 fine-tuning rows).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3|cfg2|cfg5] [--impl reference]
+
+Prints ONE JSON line.  With N > 1 (under torchrun) every rank runs the same workload on its own
+GPU (rows are independent, the path needs no collective): weak scaling, value = all ranks' tokens
+divided by the slowest rank's time.  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2607_28848_b200 import synth  # noqa: E402
+
+METRIC = "mixed-batch multi-LoRA layer tokens/s (fwd + LoRA bwd)"
+UNIT = "tokens/s"
+
+
+# ---------------------------------------------------------------------------------------------
+# workloads and their algorithmic work
+# ---------------------------------------------------------------------------------------------
+def get_workloads(name: str, seed: int = 0):
+    if name == "cfg3":
+        return synth.cfg3_layer_set(seed), "cfg3: Llama-3-8B decoder-layer projection set (q,k,v,o,gate,up,down), " \
+                                           "bf16, 32 adapters r=16, 4096 mixed rows (1024 prefill in 12 segments, " \
+                                           "1024 decode, 4x512 fine-tune)"
+    if name == "cfg2":
+        return [synth.cfg2_single_projection(seed)], "cfg2: 4096x4096 projection, bf16, 16 adapters r=16, 1600 rows"
+    if name == "cfg5":
+        return [synth.cfg5_decode_heavy(seed)], "cfg5: 5120x13824 up projection, bf16, 128 adapters r=32, " \
+                                                "512 decode rows + one 2048-row fine-tune segment"
+    raise SystemExit(f"unknown workload {name}")
+
+
+def flops(w) -> dict:
+    """Algorithmic FLOPs: no credit for padded tiles or recomputation."""
+    T, Tf, di, do, r = w.n_rows, w.ft_rows, w.d_in, w.d_out, w.rank
+    return {
+        "fwd": 2.0 * T * di * do + 2.0 * T * r * (di + do),
+        "bwd": 2.0 * Tf * di * do + 2.0 * Tf * r * (2 * do + 2 * di),
+        "gemm_fwd": 2.0 * T * do * (di + r),          # base product + expand, one kernel
+        "gemm_bwd": 2.0 * Tf * di * (do + r),         # dY W^T + V A, one kernel
+    }
+
+
+def algorithmic_bytes(w) -> dict:
+    """Each tensor once (bytes), per kernel class."""
+    T, Tf, di, do, r, e = w.n_rows, w.ft_rows, w.d_in, w.d_out, w.rank, w.elem_bytes
+    seg = w.segments
+    used = len(set(seg[seg[:, 2] >= 0, 2].tolist())) if len(seg) else 0
+    fta = len(set(seg[seg[:, 3] != 0, 2].tolist())) if len(seg) else 0
+    return {
+        "shrink_fwd": e * T * di + e * used * r * di + 4 * T * r + e * Tf * di + 4 * Tf * r,   # + save copies
+        "shrink_bwd": e * Tf * do + e * fta * r * do + 4 * Tf * r,
+        "grad_dB": e * Tf * do + 4 * Tf * r + 4 * fta * r * do,
+        "grad_dA": e * Tf * di + 4 * Tf * r + 4 * fta * r * di,
+        "gemm_fwd": e * (T * di + di * do + T * do + used * r * do) + 4 * T * r,
+        "gemm_bwd": e * (Tf * do + di * do + Tf * di + fta * r * di) + 4 * Tf * r,
+    }
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.NamedTemporaryFile(prefix="clocks_", suffix=".csv", delete=False).name
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(gpu_index), f"--query-gpu=timestamp,{self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-f", self.path], stdout=subprocess.DEVNULL, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+        self.t0 = self.t1 = None
+
+    def mark_start(self):
+        self.t0 = time.time()
+
+    def mark_stop(self):
+        self.t1 = time.time()
+
+    def finish(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = []
+        try:
+            import datetime
+            with open(self.path) as fh:
+                for ln in fh:
+                    f = [x.strip() for x in ln.split(",")]
+                    if len(f) < 8:
+                        continue
+                    try:
+                        ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                        rows.append((ts, float(f[1]), float(f[2]), float(f[3]), f[4:8]))
+                    except ValueError:
+                        continue
+            os.unlink(self.path)
+        except OSError:
+            pass
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        inside = [r for r in rows if self.t0 is not None and self.t0 <= r[0] <= self.t1] or rows
+        sm = float(np.median([r[1] for r in inside]))
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({names[i] for r in inside for i in range(4) if r[4][i].lower().startswith("active")})
+        return {"sm_mhz": sm, "sm_max_mhz": rows[0][2], "reasons": reasons, "samples": len(inside),
+                "power_w_max": max(r[3] for r in inside)}
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ---------------------------------------------------------------------------------------------
+def oracle_pass(w, t):
+    from oracle import mlora_oracle as orc
+    f = orc.forward_blocked(t["X"], t["W"], t["A_all"], t["B_all"], t["scale"], w.segments)
+    orc.backward_blocked(t["dY"], t["W"], t["A_all"], t["B_all"], t["scale"], w.segments, f["x_save"], f["u_save"],
+                         n_rows=w.n_rows)
+
+
+def host_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def cpu_baseline(workloads, sample_names) -> dict:
+    """Times the oracle as it stands on a bounded sample and scales by algorithmic FLOPs."""
+    total = sum(flops(w)["fwd"] + flops(w)["bwd"] for w in workloads)
+    sample = [w for w in workloads if w.name.split("_", 1)[1] in sample_names] or workloads[:1]
+    sflops, secs = 0.0, 0.0
+    for w in sample:
+        t = synth.make_tensors(w)
+        t0 = time.perf_counter()
+        oracle_pass(w, t)
+        secs += time.perf_counter() - t0
+        sflops += flops(w)["fwd"] + flops(w)["bwd"]
+    est = secs * total / sflops
+    return {"value": workloads[0].n_rows / est, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+            "sample": f"fp64 numpy oracle, forward+backward of projection(s) {[w.name for w in sample]} "
+                      f"({sflops / 1e9:.0f} of {total / 1e9:.0f} GFLOP) in {secs:.1f} s, scaled to the whole step by FLOPs"}
+
+
+def run_reference(args, workloads, label):
+    """The reference arm: the CPU oracle timed on the host cores, one bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    total = sum(flops(w)["fwd"] + flops(w)["bwd"] for w in workloads)
+    w = min(workloads, key=lambda x: flops(x)["fwd"] + flops(x)["bwd"])
+    t = synth.make_tensors(w)
+    for _ in range(args.warmup):
+        oracle_pass(w, t)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_pass(w, t)
+    secs = (time.perf_counter() - t0) / max(args.steps, 1)
+    sf = flops(w)["fwd"] + flops(w)["bwd"]
+    est = secs * total / sf
+    value = workloads[0].n_rows / est
+    sample = (f"each step = fp64 numpy oracle forward+backward of {w.name} ({sf / 1e9:.0f} of {total / 1e9:.0f} GFLOP "
+              f"per full step), scaled to the whole step by FLOPs")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": label},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": host_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+# GPU arm
+# ---------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="cfg3")
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    workloads, label = get_workloads(args.workload, args.seed + rank)
+    if args.impl == "reference":
+        run_reference(args, workloads, label)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2607_28848_b200 import binding as mb
+    from paper_2607_28848_b200.runner import LayerRun, Session
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the layer has no CPU fallback")
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    sess = Session(local_rank)
+    peaks = load_peaks()
+
+    runs = []
+    for w in workloads:
+        t = synth.make_tensors(w)
+        runs.append(LayerRun(sess, w.dtype, t, w.segments, w.n_rows))
+        del t
+    resident = sum(w.d_in * w.d_out * w.elem_bytes + w.n_rows * (w.d_in + w.d_out) * w.elem_bytes for w in workloads)
+
+    def step():
+        for r in runs:
+            r.forward()
+            r.backward()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    if sess.ctx and mb.mlora_poll_status(sess.ctx) != mb.MLORA_OK:
+        raise SystemExit("device status word reports a timed-out wait")
+
+    launches_per_step_probe = mb.mlora_launch_count(sess.ctx)
+    step()
+    launches_per_step = mb.mlora_launch_count(sess.ctx) - launches_per_step_probe
+    mb.mlora_profile_enable(sess.ctx, launches_per_step * args.steps)
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    if sampler:
+        sampler.mark_start()
+    l0 = mb.mlora_launch_count(sess.ctx)
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    barrier()
+    if sampler:
+        sampler.mark_stop()
+    gpu_launches = mb.mlora_launch_count(sess.ctx) - l0
+    ms_total = ev0.elapsed_time(ev1)
+    if world > 1:
+        tt = torch.tensor([ms_total], device=sess.device)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+    clocks = sampler.finish() if sampler else None
+    kinds, kms = mb.mlora_profile_collect(sess.ctx)
+    mb.mlora_profile_enable(sess.ctx, 0)
+
+    ms_per_step = ms_total / args.steps
+    T = workloads[0].n_rows
+    value = world * T / (ms_per_step * 1e-3)
+    tot_flops = sum(flops(w)["fwd"] + flops(w)["bwd"] for w in workloads)
+
+    # ---- per-kernel accounting (CUDA events recorded by the library around each launch) ----
+    per_kind = {}
+    for k, name in enumerate(mb.PROFILE_KINDS):
+        sel = kms[kinds == k]
+        if len(sel):
+            per_kind[name] = {"launches_per_step": len(sel) / args.steps, "ms_per_step": float(sel.sum() / args.steps)}
+    gemm_fwd_flops = sum(flops(w)["gemm_fwd"] for w in workloads)
+    gemm_bwd_flops = sum(flops(w)["gemm_bwd"] for w in workloads)
+    ab = [algorithmic_bytes(w) for w in workloads]
+    kernels = {}
+    if "gemm_fwd" in per_kind:
+        kernels["gemm_fwd"] = {**per_kind["gemm_fwd"], "tflops": gemm_fwd_flops / per_kind["gemm_fwd"]["ms_per_step"] / 1e9}
+    if "gemm_bwd" in per_kind:
+        kernels["gemm_bwd"] = {**per_kind["gemm_bwd"], "tflops": gemm_bwd_flops / per_kind["gemm_bwd"]["ms_per_step"] / 1e9}
+    if "shrink" in per_kind:
+        b = sum(a["shrink_fwd"] + a["shrink_bwd"] for a in ab)
+        kernels["shrink"] = {**per_kind["shrink"], "gbs": b / per_kind["shrink"]["ms_per_step"] / 1e6}
+    if "grad" in per_kind:
+        b = sum(a["grad_dA"] + a["grad_dB"] for a in ab)
+        kernels["grad"] = {**per_kind["grad"], "gbs": b / per_kind["grad"]["ms_per_step"] / 1e6}
+    roofline = None
+    if "gemm_fwd" in kernels:
+        n_launch = per_kind["gemm_fwd"]["launches_per_step"]
+        achieved = kernels["gemm_fwd"]["tflops"]
+        peak = peaks["bf16_tflops_sustained"]
+        roofline = {"kernel": "gemm_lora_kernel (forward: base GEMM + LoRA expand)", "bound": "tensor",
+                    "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                    "peak_source": f"{peaks['source']} sustained bf16 ({peak}); burst {peaks['bf16_tflops']}",
+                    "frac_of_burst": achieved / peaks["bf16_tflops"],
+                    "flops_per_launch": gemm_fwd_flops / n_launch,
+                    "avg_launch_ms": per_kind["gemm_fwd"]["ms_per_step"] / n_launch,
+                    "traffic": None}
+        prof = os.path.join(ROOT, "profiles", "traffic.json")
+        if os.path.exists(prof):
+            try:
+                with open(prof) as fh:
+                    roofline["traffic"] = json.load(fh).get(args.workload, {}).get("gemm_fwd_bytes_per_launch")
+            except Exception:
+                pass
+
+    # ---- end to end through the public API with host buffers ----
+    e2e = None
+    if rank == 0 or world > 1:
+        hx = [r.X.cpu().pin_memory() for r in runs]
+        hdy = [r.dY.cpu().pin_memory() for r in runs]
+        hy = [torch.empty_like(r.Y, device="cpu").pin_memory() for r in runs]
+        hda = [torch.empty_like(r.dA, device="cpu").pin_memory() for r in runs]
+        hdb = [torch.empty_like(r.dB, device="cpu").pin_memory() for r in runs]
+        hdx = [torch.empty_like(r.dX, device="cpu").pin_memory() for r in runs]
+        h2d = sum(t.numel() * t.element_size() for t in hx + hdy)
+        d2h = sum(t.numel() * t.element_size() for t in hy + hda + hdb + hdx)
+
+        def e2e_step():
+            for i, r in enumerate(runs):
+                r.X.copy_(hx[i], non_blocking=True)
+                r.dY.copy_(hdy[i], non_blocking=True)
+                r.forward()
+                r.backward()
+                hy[i].copy_(r.Y, non_blocking=True)
+                hda[i].copy_(r.dA, non_blocking=True)
+                hdb[i].copy_(r.dB, non_blocking=True)
+                hdx[i].copy_(r.dX, non_blocking=True)
+
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        ms_e2e = e0.elapsed_time(e1)
+        if world > 1:
+            tt = torch.tensor([ms_e2e], device=sess.device)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ms_e2e = float(tt.item())
+        e2e = {"value": world * T * args.e2e_steps / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.e2e_steps, "steps": args.e2e_steps}
+
+    status = mb.mlora_poll_status(sess.ctx)
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": label, "rows_per_step": T, "ft_rows_per_step": workloads[0].ft_rows,
+                   "l2_policy": f"inputs larger than L2: one step touches {resident / 1e6:.0f} MB of weights and "
+                                f"activations, so nothing survives in the 126 MB L2 from step to step",
+                   "parallelism": "replicas (rows are independent; no collective)" if world > 1 else "single GPU"},
+        "tflops": tot_flops / (ms_per_step * 1e-3) / 1e12 * 1.0,
+        "roofline_whole_step": {"t_roof_ms": tot_flops / (peaks["bf16_tflops"] * 1e12) * 1e3,
+                                "frac_of_burst_peak": tot_flops / (peaks["bf16_tflops"] * 1e12) * 1e3 / ms_per_step,
+                                "frac_of_sustained_peak": tot_flops / (peaks["bf16_tflops_sustained"] * 1e12) * 1e3 / ms_per_step},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches), "device_status": int(status),
+        "roofline": roofline, "kernels": kernels,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        names = {"cfg3": ["k", "q"], "cfg2": ["proj4096"], "cfg5": ["mixed"]}[args.workload]
+        line["cpu_baseline"] = cpu_baseline(workloads, names)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,190 @@
+/*
+ * mlora.h - C ABI of the mixed-batch multi-LoRA linear layer for NVIDIA B200 (sm_100a).
+ *
+ * One call runs inference rows (prefill and decode tokens) and LoRA fine-tuning rows
+ * through ONE pass over a frozen base weight, every row applying the low-rank adapter it
+ * is bound to; fine-tuning rows additionally leave behind the activations their backward
+ * needs.  A second call computes the LoRA gradients (and the input gradient) for those rows.
+ *
+ * Row-vector convention.  For a row x bound to adapter a:
+ *        y = x W + s_a (x A_a^T) B_a
+ * with W [d_in, d_out], A_a [rank, d_in], B_a [rank, d_out], s_a = alpha_a / rank.
+ * (Paper, Section 2.2: frozen W plus a trainable rank-r product, W_eff = W + B A; its A is
+ * A_a, its B is B_a transposed.  The scaling s comes from Section 5, "Fine-tuning
+ * Workload": r = 16, alpha = 32.)
+ *
+ * General rules
+ *  - Every pointer named "device" is a CUDA device pointer on the context's device; every
+ *    other pointer is a host pointer.  All device buffers are BORROWED: the library never
+ *    frees them and does not touch them after the work queued on the stream has finished.
+ *  - Matrices are row-major; leading dimensions (ld*) are in ELEMENTS.
+ *  - Calls return an mlora_status_t.  Argument errors are found on the host before
+ *    anything is launched.  mlora_mixed_forward / mlora_backward are asynchronous on the
+ *    given stream, allocate nothing and never synchronise.
+ *  - There is no CPU fallback: without an sm_100 device mlora_create fails with
+ *    MLORA_ERR_ARCH and no compute entry point can be used.
+ *  - The library never aborts the process and throws nothing across this boundary.
+ */
+#ifndef MLORA_H_
+#define MLORA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mlora_ctx mlora_ctx;     /* per-device state: workspace, status word        */
+typedef struct mlora_plan mlora_plan;   /* a validated segment table and its device tables */
+
+/* One contiguous run of rows bound to one adapter (paper, Section 2.2 "multi-LoRA batching":
+ * adapter-bound requests share one base pass; Section 3.2 "Mixed forward batch": a
+ * fine-tuning sample is one more prefill-like entry routed to its adapter).
+ * adapter_id = -1 means "base weight only"; is_finetune != 0 marks rows whose activations
+ * are saved and which take part in the backward. */
+typedef struct {
+  int32_t row_start;
+  int32_t row_len;
+  int32_t adapter_id;
+  int32_t is_finetune;
+} mlora_segment_t;
+
+typedef enum { MLORA_F32 = 0, MLORA_BF16 = 1 } mlora_dtype_t;
+
+typedef enum {
+  MLORA_OK = 0,
+  MLORA_ERR_INVALID_ARG = 1,     /* null pointer, negative size, bad enum                       */
+  MLORA_ERR_SEGMENT_RANGE = 2,   /* a segment leaves [0, n_rows) or has negative length         */
+  MLORA_ERR_SEGMENT_OVERLAP = 3, /* two segments share a row                                    */
+  MLORA_ERR_ADAPTER_ID = 4,      /* adapter id outside [-1, n_adapters), or fine-tune with -1   */
+  MLORA_ERR_SAVE_CAPACITY = 5,   /* fine-tune rows do not fit the activation buffer             */
+  MLORA_ERR_UNSUPPORTED = 6,     /* shape / rank / alignment outside what the kernels handle    */
+  MLORA_ERR_ARCH = 7,            /* no CUDA device of compute capability 10.x                   */
+  MLORA_ERR_CUDA = 8,            /* a CUDA runtime or driver call failed                        */
+  MLORA_ERR_DEVICE_TIMEOUT = 9   /* a bounded wait inside a kernel ran out (see poll_status)    */
+} mlora_status_t;
+
+/* One projection.  dtype is the storage type of X, W, A, B, Y, dY, dX and x_save.
+ *   MLORA_BF16: tensor-core path; needs d_in, d_out multiples of 64, rank in {8,16,32,64,128},
+ *               ldw a multiple of 8 and every base pointer 16-byte aligned.
+ *   MLORA_F32 : plain fp32 path (small layers, correctness work); rank <= 128. */
+typedef struct {
+  int32_t d_in, d_out, rank, n_adapters;
+  int32_t dtype;          /* mlora_dtype_t */
+  const void* W;          /* device [d_in, d_out], row stride ldw; frozen                    */
+  int64_t ldw;
+  const void* A_all;      /* device [n_adapters, rank, d_in], dense                           */
+  const void* B_all;      /* device [n_adapters, rank, d_out], dense                          */
+  const float* scale;     /* device [n_adapters] fp32, s_a = alpha_a / rank                   */
+} mlora_layer_t;
+
+/* ---- context ---------------------------------------------------------------------------*/
+
+/* Creates the per-device state on CUDA device `device`.  Fails with MLORA_ERR_ARCH when the
+ * device is not compute capability 10.x, MLORA_ERR_CUDA when the runtime cannot be used. */
+mlora_status_t mlora_create(mlora_ctx** ctx, int device);
+void mlora_destroy(mlora_ctx* ctx);
+
+/* ---- plan: segment table -> validated routing ------------------------------------------*/
+
+/* Validates `segs` (host array of n_segs entries) for a batch of n_rows rows and n_adapters
+ * adapters, and derives: the adapter of every row, the save offset of every fine-tuning
+ * segment (exclusive prefix sum of the fine-tuning lengths in TABLE ORDER; paper, Section
+ * 3.2: captured activations are appended to a buffer the backward consumes), the gradient
+ * slots (one per distinct fine-tuning adapter, in order of first appearance) and the tile
+ * schedules of the kernels.  Segments may come in any order; zero-length segments are legal;
+ * rows covered by no segment use the base weight only.
+ * With ctx == NULL the plan is host-only (for inspection; it cannot be executed).  With a
+ * context the tables are uploaded and the context's workspace is grown if needed, so this
+ * call may allocate device memory and synchronise; the compute calls never do.
+ * Errors: MLORA_ERR_SEGMENT_RANGE, MLORA_ERR_SEGMENT_OVERLAP, MLORA_ERR_ADAPTER_ID,
+ * MLORA_ERR_INVALID_ARG, MLORA_ERR_CUDA. */
+mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, int32_t n_segs,
+                                 int32_t n_rows, int32_t n_adapters, mlora_plan** plan);
+void mlora_plan_destroy(mlora_plan* plan);
+
+int32_t mlora_plan_rows(const mlora_plan* plan);        /* n_rows                              */
+int32_t mlora_plan_ft_rows(const mlora_plan* plan);     /* total fine-tuning rows, T_ft        */
+/* Writes up to `cap` adapter ids, slot g -> adapter id, and returns the number of slots. */
+int32_t mlora_plan_ft_adapters(const mlora_plan* plan, int32_t* ids, int32_t cap);
+/* Inspection: out[k] = save offset of segment k, or -1 when it is not a fine-tuning segment
+ * (n_segs entries); row_adapter[t] = adapter of row t or -1 (n_rows entries). Either may be NULL. */
+mlora_status_t mlora_plan_describe(const mlora_plan* plan, int32_t* seg_save_offset, int32_t* row_adapter);
+
+/* ---- forward ---------------------------------------------------------------------------*/
+
+/* Y[t,:] = X[t,:] W + s_a (X[t,:] A_a^T) B_a for every row t (a = adapter of t; base only when
+ * a = -1), inference and fine-tuning rows in the same pass (paper, Section 2.2 multi-LoRA
+ * batching; Section 3.2 "Mixed forward batch").  For fine-tuning rows only, the row of X and the
+ * UNSCALED rank-r product u = x A_a^T are written to the caller's activation buffer at row
+ *        save_row_base + save_offset(segment) + i          (i = row index inside the segment)
+ * (paper, Section 3.2: activation capture for fine-tuning rows; intermediates may be cached to
+ * avoid recomputation).  Inference rows save nothing.
+ *   X       device [n_rows, d_in], row stride ldx          (read)
+ *   Y       device [n_rows, d_out], row stride ldy         (written once, every row)
+ *   x_save  device [save_capacity_rows, d_in] dense, layer dtype; NULL skips the copy of X
+ *   u_save  device [save_capacity_rows, rank] dense fp32; required when the plan has
+ *           fine-tuning rows
+ * save_row_base + T_ft > save_capacity_rows -> MLORA_ERR_SAVE_CAPACITY (nothing launched).
+ * Other errors: MLORA_ERR_INVALID_ARG, MLORA_ERR_ADAPTER_ID (plan built for more adapters than
+ * the layer has), MLORA_ERR_UNSUPPORTED, MLORA_ERR_CUDA. */
+mlora_status_t mlora_mixed_forward(mlora_ctx* ctx, const mlora_layer_t* layer, const mlora_plan* plan,
+                                   const void* X, int64_t ldx, void* Y, int64_t ldy,
+                                   void* x_save, float* u_save,
+                                   int64_t save_row_base, int64_t save_capacity_rows,
+                                   void* cuda_stream);
+
+/* ---- backward --------------------------------------------------------------------------*/
+
+/* LoRA backward for the plan's fine-tuning rows (paper, Section 3.2 "Backward subprocess":
+ * LoRA gradients are computed from the saved activations; the formulas are the chain rule of
+ * the forward).  All row-indexed buffers are in SAVE ORDER: row m is the m-th fine-tuning row
+ * (the pointers address the first row this plan saved, i.e. the caller adds save_row_base).
+ *        V    = s_a dY B_a^T                           [T_ft, rank]  (internal)
+ *        dB_g (+)= sum over rows of slot g  s_a u^T dY [rank, d_out]
+ *        dA_g (+)= sum over rows of slot g  V^T x      [rank, d_in]
+ *        dX   = dY W^T + V A_a                         [T_ft, d_in]
+ *   dY_ft   device [T_ft, d_out], row stride lddy, layer dtype      (read)
+ *   x_save  device [T_ft, d_in] dense, layer dtype                  (read)
+ *   u_save  device [T_ft, rank] dense fp32                          (read)
+ *   dA      device [n_slots, rank, d_in]  fp32, dense (same orientation as A_all)
+ *   dB      device [n_slots, rank, d_out] fp32, dense (same orientation as B_all)
+ *   dX_ft   device [T_ft, d_in], row stride lddx, layer dtype; NULL skips dX
+ *   accumulate  0: dA, dB are overwritten;  nonzero: the new gradients are added to them
+ * Slot g belongs to adapter mlora_plan_ft_adapters()[g]; several fine-tuning segments on one
+ * adapter add into one slot.  A plan without fine-tuning rows makes this a no-op. */
+mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* layer, const mlora_plan* plan,
+                              const void* dY_ft, int64_t lddy,
+                              const void* x_save, const float* u_save,
+                              float* dA, float* dB, void* dX_ft, int64_t lddx,
+                              int32_t accumulate, void* cuda_stream);
+
+/* ---- status / diagnostics --------------------------------------------------------------*/
+
+/* Synchronises the stream and returns the device status word: MLORA_OK, or
+ * MLORA_ERR_DEVICE_TIMEOUT when a bounded wait inside a kernel gave up (the kernel then
+ * released its resources and returned; its outputs are invalid).  Clears the word. */
+mlora_status_t mlora_poll_status(mlora_ctx* ctx, void* cuda_stream);
+const char* mlora_status_string(mlora_status_t s);
+
+/* Number of kernels the library has launched on this context since it was created. */
+int64_t mlora_launch_count(const mlora_ctx* ctx);
+
+/* Per-kernel timing.  mlora_profile_enable(ctx, n) with n > 0 creates n CUDA event pairs (this
+ * allocates; call it outside any timed or captured region) and makes every later kernel launch
+ * of this context record one pair around itself on the launching stream, until the pairs run
+ * out; n = 0 switches recording off and frees the events.  mlora_profile_collect synchronises
+ * the device, writes for each recorded launch its kind (0 shrink, 1 forward GEMM, 2 input-gradient
+ * GEMM, 3 gradient kernel, 4 CUDA-core kernels) and its duration in milliseconds into the host
+ * arrays (up to cap entries), forgets the records and returns how many there were. */
+mlora_status_t mlora_profile_enable(mlora_ctx* ctx, int32_t max_records);
+int32_t mlora_profile_collect(mlora_ctx* ctx, int32_t* kinds, float* ms, int32_t cap);
+
+/* Selects the base-product kernel for MLORA_BF16 layers: 0 = tcgen05 tensor-core kernel
+ * (default), 1 = the plain CUDA-core kernel (a slow cross-check used by the tests). */
+mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MLORA_H_ */

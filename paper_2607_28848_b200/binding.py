@@ -1,0 +1,238 @@
+"""ctypes binding of libmlora.so: the same names as the C ABI (include/mlora.h), plus thin
+object wrappers that only marshal arguments (torch tensors -> device pointers, leading
+dimensions, the current CUDA stream).  Every step of the layer runs inside the library's
+kernels; nothing here computes, and there is no fallback: if the library cannot be loaded, or
+no sm_100 device is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG_DIR, "libmlora.so")
+
+MLORA_F32, MLORA_BF16 = 0, 1
+(MLORA_OK, MLORA_ERR_INVALID_ARG, MLORA_ERR_SEGMENT_RANGE, MLORA_ERR_SEGMENT_OVERLAP, MLORA_ERR_ADAPTER_ID,
+ MLORA_ERR_SAVE_CAPACITY, MLORA_ERR_UNSUPPORTED, MLORA_ERR_ARCH, MLORA_ERR_CUDA, MLORA_ERR_DEVICE_TIMEOUT) = range(10)
+
+EXPORTS = (
+    "mlora_create", "mlora_destroy", "mlora_plan_create", "mlora_plan_destroy", "mlora_plan_rows",
+    "mlora_plan_ft_rows", "mlora_plan_ft_adapters", "mlora_plan_describe", "mlora_mixed_forward",
+    "mlora_backward", "mlora_poll_status", "mlora_status_string", "mlora_launch_count", "mlora_set_gemm_path",
+    "mlora_profile_enable", "mlora_profile_collect",
+)
+
+
+class mlora_segment_t(ctypes.Structure):
+    _fields_ = [("row_start", ctypes.c_int32), ("row_len", ctypes.c_int32),
+                ("adapter_id", ctypes.c_int32), ("is_finetune", ctypes.c_int32)]
+
+
+class mlora_layer_t(ctypes.Structure):
+    _fields_ = [("d_in", ctypes.c_int32), ("d_out", ctypes.c_int32), ("rank", ctypes.c_int32),
+                ("n_adapters", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("W", ctypes.c_void_p), ("ldw", ctypes.c_int64),
+                ("A_all", ctypes.c_void_p), ("B_all", ctypes.c_void_p), ("scale", ctypes.c_void_p)]
+
+
+class MloraError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+_lib = None
+
+
+def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
+    """Load libmlora.so (building it with nvcc first when it is missing or stale)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if build_if_missing:
+        from . import build as _build
+        if _build.is_stale():
+            _build.build()
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_28848_b200.build`")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    P = ctypes.POINTER
+    lib.mlora_create.argtypes = [P(vp), ctypes.c_int]
+    lib.mlora_create.restype = ctypes.c_int
+    lib.mlora_destroy.argtypes = [vp]
+    lib.mlora_destroy.restype = None
+    lib.mlora_plan_create.argtypes = [vp, P(mlora_segment_t), i32, i32, i32, P(vp)]
+    lib.mlora_plan_create.restype = ctypes.c_int
+    lib.mlora_plan_destroy.argtypes = [vp]
+    lib.mlora_plan_destroy.restype = None
+    lib.mlora_plan_rows.argtypes = [vp]
+    lib.mlora_plan_rows.restype = i32
+    lib.mlora_plan_ft_rows.argtypes = [vp]
+    lib.mlora_plan_ft_rows.restype = i32
+    lib.mlora_plan_ft_adapters.argtypes = [vp, P(i32), i32]
+    lib.mlora_plan_ft_adapters.restype = i32
+    lib.mlora_plan_describe.argtypes = [vp, P(i32), P(i32)]
+    lib.mlora_plan_describe.restype = ctypes.c_int
+    lib.mlora_mixed_forward.argtypes = [vp, P(mlora_layer_t), vp, vp, i64, vp, i64, vp, vp, i64, i64, vp]
+    lib.mlora_mixed_forward.restype = ctypes.c_int
+    lib.mlora_backward.argtypes = [vp, P(mlora_layer_t), vp, vp, i64, vp, vp, vp, vp, vp, i64, i32, vp]
+    lib.mlora_backward.restype = ctypes.c_int
+    lib.mlora_poll_status.argtypes = [vp, vp]
+    lib.mlora_poll_status.restype = ctypes.c_int
+    lib.mlora_status_string.argtypes = [ctypes.c_int]
+    lib.mlora_status_string.restype = ctypes.c_char_p
+    lib.mlora_launch_count.argtypes = [vp]
+    lib.mlora_launch_count.restype = i64
+    lib.mlora_set_gemm_path.argtypes = [vp, i32]
+    lib.mlora_set_gemm_path.restype = ctypes.c_int
+    lib.mlora_profile_enable.argtypes = [vp, i32]
+    lib.mlora_profile_enable.restype = ctypes.c_int
+    lib.mlora_profile_collect.argtypes = [vp, P(i32), P(ctypes.c_float), i32]
+    lib.mlora_profile_collect.restype = i32
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().mlora_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != MLORA_OK:
+        raise MloraError(status, where)
+
+
+def _segments_ctypes(segments) -> "ctypes.Array":
+    seg = np.ascontiguousarray(np.asarray(segments, dtype=np.int32).reshape(-1, 4))
+    arr = (mlora_segment_t * max(len(seg), 1))()
+    for i, (a, b, c, d) in enumerate(seg.tolist()):
+        arr[i] = mlora_segment_t(a, b, c, d)
+    return arr, len(seg)
+
+
+# --------------------------------------------------------------------------------------------
+# same-name functions (raise MloraError on a non-zero status)
+# --------------------------------------------------------------------------------------------
+def mlora_create(device: int = 0) -> ctypes.c_void_p:
+    h = ctypes.c_void_p()
+    _check(load_library().mlora_create(ctypes.byref(h), int(device)), "mlora_create")
+    return h
+
+
+def mlora_destroy(ctx) -> None:
+    load_library().mlora_destroy(ctx)
+
+
+def mlora_plan_create(ctx, segments, n_rows: int, n_adapters: int) -> ctypes.c_void_p:
+    arr, n = _segments_ctypes(segments)
+    h = ctypes.c_void_p()
+    _check(load_library().mlora_plan_create(ctx, arr, n, int(n_rows), int(n_adapters), ctypes.byref(h)),
+           "mlora_plan_create")
+    return h
+
+
+def mlora_plan_destroy(plan) -> None:
+    load_library().mlora_plan_destroy(plan)
+
+
+def mlora_plan_rows(plan) -> int:
+    return int(load_library().mlora_plan_rows(plan))
+
+
+def mlora_plan_ft_rows(plan) -> int:
+    return int(load_library().mlora_plan_ft_rows(plan))
+
+
+def mlora_plan_ft_adapters(plan) -> List[int]:
+    lib = load_library()
+    n = lib.mlora_plan_ft_adapters(plan, None, 0)
+    buf = (ctypes.c_int32 * max(n, 1))()
+    lib.mlora_plan_ft_adapters(plan, buf, n)
+    return [int(buf[i]) for i in range(n)]
+
+
+def mlora_plan_describe(plan, n_segs: int):
+    lib = load_library()
+    n_rows = lib.mlora_plan_rows(plan)
+    so = (ctypes.c_int32 * max(n_segs, 1))()
+    ra = (ctypes.c_int32 * max(n_rows, 1))()
+    _check(lib.mlora_plan_describe(plan, so, ra), "mlora_plan_describe")
+    return np.asarray(so[:n_segs], dtype=np.int32), np.asarray(ra[:n_rows], dtype=np.int32)
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else int(t.data_ptr())
+
+
+def _stream_ptr(stream=None) -> int:
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def make_layer(W, A_all, B_all, scale) -> mlora_layer_t:
+    """Describe a projection from torch CUDA tensors (W [d_in,d_out], A_all [n,r,d_in], B_all [n,r,d_out])."""
+    import torch
+    assert W.is_cuda and A_all.is_cuda and B_all.is_cuda and scale.is_cuda
+    assert A_all.is_contiguous() and B_all.is_contiguous() and scale.dtype == torch.float32
+    assert W.dtype == A_all.dtype == B_all.dtype and W.stride(1) == 1
+    dt = {torch.float32: MLORA_F32, torch.bfloat16: MLORA_BF16}[W.dtype]
+    n, r, d_in = A_all.shape
+    d_out = B_all.shape[2]
+    assert W.shape == (d_in, d_out) and B_all.shape[:2] == (n, r) and scale.numel() == n
+    return mlora_layer_t(d_in, d_out, r, n, dt, _ptr(W), W.stride(0), _ptr(A_all), _ptr(B_all), _ptr(scale))
+
+
+def mlora_mixed_forward(ctx, layer: mlora_layer_t, plan, X, Y, x_save, u_save, save_row_base: int = 0,
+                        save_capacity_rows: Optional[int] = None, stream=None) -> None:
+    """Queue the forward on the current (or given) stream.  X, Y, x_save, u_save are torch CUDA tensors."""
+    if save_capacity_rows is None:
+        save_capacity_rows = 0 if u_save is None else int(u_save.shape[0])
+    st = load_library().mlora_mixed_forward(
+        ctx, ctypes.byref(layer), plan, _ptr(X), X.stride(0) if X is not None else 0,
+        _ptr(Y), Y.stride(0) if Y is not None else 0, _ptr(x_save), _ptr(u_save),
+        int(save_row_base), int(save_capacity_rows), _stream_ptr(stream))
+    _check(st, "mlora_mixed_forward")
+
+
+def mlora_backward(ctx, layer: mlora_layer_t, plan, dY, x_save, u_save, dA, dB, dX, accumulate: bool = False,
+                   stream=None) -> None:
+    """Queue the LoRA backward; all row-indexed tensors start at the first row this plan saved."""
+    st = load_library().mlora_backward(
+        ctx, ctypes.byref(layer), plan, _ptr(dY), dY.stride(0) if dY is not None else 0, _ptr(x_save), _ptr(u_save),
+        _ptr(dA), _ptr(dB), _ptr(dX), dX.stride(0) if dX is not None else 0, int(bool(accumulate)),
+        _stream_ptr(stream))
+    _check(st, "mlora_backward")
+
+
+def mlora_poll_status(ctx, stream=None) -> int:
+    return int(load_library().mlora_poll_status(ctx, _stream_ptr(stream)))
+
+
+def mlora_launch_count(ctx) -> int:
+    return int(load_library().mlora_launch_count(ctx))
+
+
+def mlora_set_gemm_path(ctx, path: int) -> None:
+    _check(load_library().mlora_set_gemm_path(ctx, int(path)), "mlora_set_gemm_path")
+
+
+PROFILE_KINDS = ("shrink", "gemm_fwd", "gemm_bwd", "grad", "simt")
+
+
+def mlora_profile_enable(ctx, max_records: int) -> None:
+    _check(load_library().mlora_profile_enable(ctx, int(max_records)), "mlora_profile_enable")
+
+
+def mlora_profile_collect(ctx, cap: int = 1 << 16):
+    """Returns (kinds, ms) numpy arrays of the launches recorded since the last collect."""
+    kinds = (ctypes.c_int32 * cap)()
+    ms = (ctypes.c_float * cap)()
+    n = load_library().mlora_profile_collect(ctx, kinds, ms, cap)
+    n = min(n, cap)
+    return np.asarray(kinds[:n], dtype=np.int32), np.asarray(ms[:n], dtype=np.float64)

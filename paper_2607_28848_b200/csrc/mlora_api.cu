@@ -1,0 +1,536 @@
+// C ABI of the mixed-batch multi-LoRA layer: context, plan upload, argument checks, tensor-map
+// encoding and kernel dispatch.  See include/mlora.h for the contract of every entry point.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "mlora.h"
+#include "plan.h"
+#include "gemm_tcgen05.cuh"
+#include "simt.cuh"
+#include "skinny.cuh"
+
+using namespace mlora;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct mlora_ctx {
+  int device = 0;
+  int sm_count = 0;
+  int32_t* status_dev = nullptr;     // device status word
+  float* ws_p = nullptr;             // [ws_rows, kMaxRank] rank-r intermediate of the running call
+  int64_t ws_rows = 0;
+  int64_t launches = 0;
+  int32_t gemm_path = 0;
+  EncodeTiledFn encode = nullptr;
+  // optional per-launch timing
+  std::vector<cudaEvent_t> ev_start, ev_stop;
+  std::vector<int32_t> ev_kind;
+  int32_t ev_used = 0;
+};
+
+enum { KIND_SHRINK = 0, KIND_GEMM_FWD = 1, KIND_GEMM_BWD = 2, KIND_GRAD = 3, KIND_SIMT = 4 };
+
+// Device copy of one RowSpace.
+struct DevRowSpace {
+  const int32_t* row_adapter = nullptr;
+  const int32_t* row_save = nullptr;
+  const int32_t* row_grp = nullptr;
+  const int32_t* tile_grp_off = nullptr;
+  const int32_t* grp_adapter = nullptr;
+  const int32_t* item_row0 = nullptr;
+  const int32_t* item_nrows = nullptr;
+  const int32_t* item_adapter = nullptr;
+  const int32_t* item_save0 = nullptr;
+};
+
+struct mlora_plan {
+  HostPlan h;
+  mlora_ctx* ctx = nullptr;
+  int32_t* blob = nullptr;           // all device tables in one allocation
+  DevRowSpace fwd, bwd;
+  const int32_t* slot_chunk_off = nullptr;
+  const int32_t* chunk_row0 = nullptr;
+  const int32_t* chunk_nrows = nullptr;
+  const int32_t* slot_adapter = nullptr;
+};
+
+namespace {
+
+struct BlobBuilder {
+  std::vector<int32_t> data;
+  size_t add(const std::vector<int32_t>& v) {
+    const size_t off = data.size();
+    data.insert(data.end(), v.begin(), v.end());
+    while (data.size() % 4) data.push_back(0);      // keep every table 16-byte aligned
+    if (v.empty()) { data.insert(data.end(), 4, 0); }
+    return off;
+  }
+};
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+mlora_status_t make_tmap_bf16(const mlora_ctx* ctx, CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer,
+                              uint64_t row_stride_elems, uint32_t box_inner, uint32_t box_outer) {
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {row_stride_elems * 2};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = ctx->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MLORA_OK : MLORA_ERR_CUDA;
+}
+
+bool rank_ok_bf16(int r) { return r == 8 || r == 16 || r == 32 || r == 64 || r == 128; }
+
+mlora_status_t check_layer(const mlora_layer_t* L) {
+  if (!L || !L->W || !L->A_all || !L->B_all || !L->scale) return MLORA_ERR_INVALID_ARG;
+  if (L->d_in <= 0 || L->d_out <= 0 || L->rank <= 0 || L->n_adapters <= 0) return MLORA_ERR_INVALID_ARG;
+  if (L->dtype != MLORA_F32 && L->dtype != MLORA_BF16) return MLORA_ERR_INVALID_ARG;
+  if (L->ldw < L->d_out) return MLORA_ERR_INVALID_ARG;
+  if (L->rank > kMaxRank) return MLORA_ERR_UNSUPPORTED;
+  if (L->dtype == MLORA_BF16) {
+    if (!rank_ok_bf16(L->rank) || L->d_in % 64 || L->d_out % 64 || L->ldw % 8) return MLORA_ERR_UNSUPPORTED;
+    if (!aligned16(L->W) || !aligned16(L->A_all) || !aligned16(L->B_all)) return MLORA_ERR_UNSUPPORTED;
+  }
+  return MLORA_OK;
+}
+
+// Brackets one kernel launch: optional event pair, launch counter, launch-error check.
+struct LaunchScope {
+  mlora_ctx* ctx; cudaStream_t st; int slot;
+  LaunchScope(mlora_ctx* c, cudaStream_t s, int kind) : ctx(c), st(s), slot(-1) {
+    if (c->ev_used < (int32_t)c->ev_start.size()) {
+      slot = c->ev_used++;
+      c->ev_kind[slot] = kind;
+      cudaEventRecord(c->ev_start[slot], st);
+    }
+  }
+  mlora_status_t done() {
+    if (slot >= 0) cudaEventRecord(ctx->ev_stop[slot], st);
+    ctx->launches++;
+    return cudaGetLastError() == cudaSuccess ? MLORA_OK : MLORA_ERR_CUDA;
+  }
+};
+
+// ---- bf16 launches ------------------------------------------------------------------------
+template <int RB>
+void launch_shrink_rb(const ShrinkArgs& a, int n_items, cudaStream_t st) {
+  shrink_kernel<RB><<<n_items, SHRINK_THREADS, 0, st>>>(a);
+}
+mlora_status_t launch_shrink(mlora_ctx* ctx, int R, const ShrinkArgs& a, int n_items, cudaStream_t st) {
+  if (n_items <= 0) return MLORA_OK;
+  LaunchScope scope(ctx, st, KIND_SHRINK);
+  switch (R) {
+    case 8: launch_shrink_rb<1>(a, n_items, st); break;
+    case 16: launch_shrink_rb<2>(a, n_items, st); break;
+    case 32: launch_shrink_rb<4>(a, n_items, st); break;
+    case 64: launch_shrink_rb<8>(a, n_items, st); break;
+    case 128: launch_shrink_rb<16>(a, n_items, st); break;
+    default: return MLORA_ERR_UNSUPPORTED;
+  }
+  return scope.done();
+}
+
+mlora_status_t launch_grad(mlora_ctx* ctx, const GradArgs& a, int n_slots, cudaStream_t st) {
+  if (n_slots <= 0) return MLORA_OK;
+  LaunchScope scope(ctx, st, KIND_GRAD);
+  if (a.R <= 16) {
+    grad_kernel<1><<<dim3(a.D / 64, n_slots, 1), GRAD_THREADS, 0, st>>>(a);
+  } else {
+    grad_kernel<2><<<dim3(a.D / 64, n_slots, (a.R + 31) / 32), GRAD_THREADS, 0, st>>>(a);
+  }
+  return scope.done();
+}
+
+template <int R, bool W_KMAJOR>
+mlora_status_t launch_gemm_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUtensorMap& tW, const CUtensorMap& tL,
+                             const CUtensorMap& tOut, const GemmArgs& g, cudaStream_t st) {
+  static bool attr_set = false;     // per instantiation; the attribute is per function, per device context
+  auto kern = gemm_lora_kernel<R, W_KMAJOR>;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_BYTES) != cudaSuccess)
+      return MLORA_ERR_CUDA;
+    attr_set = true;
+  }
+  const int tiles = g.n_mtiles * g.n_ntiles;
+  const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+  LaunchScope scope(ctx, st, W_KMAJOR ? KIND_GEMM_BWD : KIND_GEMM_FWD);
+  kern<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(tIn, tW, tL, tOut, g);
+  return scope.done();
+}
+
+template <bool W_KMAJOR>
+mlora_status_t launch_gemm(mlora_ctx* ctx, int R, const CUtensorMap& tIn, const CUtensorMap& tW, const CUtensorMap& tL,
+                           const CUtensorMap& tOut, const GemmArgs& g, cudaStream_t st) {
+  switch (R) {
+    case 8: return launch_gemm_r<8, W_KMAJOR>(ctx, tIn, tW, tL, tOut, g, st);
+    case 16: return launch_gemm_r<16, W_KMAJOR>(ctx, tIn, tW, tL, tOut, g, st);
+    case 32: return launch_gemm_r<32, W_KMAJOR>(ctx, tIn, tW, tL, tOut, g, st);
+    case 64: return launch_gemm_r<64, W_KMAJOR>(ctx, tIn, tW, tL, tOut, g, st);
+    case 128: return launch_gemm_r<128, W_KMAJOR>(ctx, tIn, tW, tL, tOut, g, st);
+    default: return MLORA_ERR_UNSUPPORTED;
+  }
+}
+
+// Out = In Wop + (scale) P L over one row space, tensor-core path.
+template <bool W_KMAJOR>
+mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace& hs, const DevRowSpace& ds,
+                         const void* In, int64_t ld_in, void* Out, int64_t ld_out, const void* L_all,
+                         const float* P, const float* scale, int M, int N, int K, cudaStream_t st) {
+  CUtensorMap tIn, tW, tL, tOut;
+  mlora_status_t s;
+  if ((s = make_tmap_bf16(ctx, &tIn, In, K, M, ld_in, GEMM_BK, GEMM_BM)) != MLORA_OK) return s;
+  if (W_KMAJOR) {   // W [N rows, K cols] (the stored [d_in, d_out] matrix read as the transposed operand)
+    if ((s = make_tmap_bf16(ctx, &tW, L->W, K, N, L->ldw, GEMM_BK, GEMM_BN)) != MLORA_OK) return s;
+  } else {          // W [K rows, N cols]
+    if ((s = make_tmap_bf16(ctx, &tW, L->W, N, K, L->ldw, 64, GEMM_BK)) != MLORA_OK) return s;
+  }
+  const int R = L->rank;
+  if ((s = make_tmap_bf16(ctx, &tL, L_all, N, (uint64_t)L->n_adapters * R, N, 64, R < 64 ? R : 64)) != MLORA_OK) return s;
+  if ((s = make_tmap_bf16(ctx, &tOut, Out, N, M, ld_out, 64, 32)) != MLORA_OK) return s;
+  GemmArgs g;
+  g.M = M; g.N = N; g.K = K;
+  g.n_mtiles = (M + GEMM_BM - 1) / GEMM_BM;
+  g.n_ntiles = (N + GEMM_BN - 1) / GEMM_BN;
+  g.lora_enabled = hs.grp_adapter.empty() ? 0 : 1;
+  g.row_grp = ds.row_grp; g.row_adapter = ds.row_adapter;
+  g.tile_grp_off = ds.tile_grp_off; g.grp_adapter = ds.grp_adapter;
+  g.P = P; g.scale = scale; g.status = ctx->status_dev;
+  return launch_gemm<W_KMAJOR>(ctx, R, tIn, tW, tL, tOut, g, st);
+}
+
+// ---- generic (fp32 / cross-check) launches --------------------------------------------------
+template <typename T>
+mlora_status_t simt_shrink(mlora_ctx* ctx, const T* In, int64_t ld_in, int D, int R, const T* P_all,
+                           const float* scale, const DevRowSpace& ds, float* Out, T* x_save, float* u_save,
+                           int64_t save_base, int n_rows, cudaStream_t st) {
+  if (n_rows <= 0) return MLORA_OK;
+  const int64_t warps = (int64_t)n_rows * R;
+  const int blocks = (int)((warps * 32 + 255) / 256);
+  LaunchScope scope(ctx, st, KIND_SIMT);
+  simt::shrink_kernel<T><<<blocks, 256, 0, st>>>(In, ld_in, D, R, P_all, scale, ds.row_adapter, ds.row_save, Out,
+                                                 x_save, u_save, save_base, n_rows);
+  return scope.done();
+}
+
+template <typename T, bool W_KMAJOR>
+mlora_status_t simt_gemm(mlora_ctx* ctx, const T* In, int64_t ld_in, const T* W, int64_t ldw, const T* L_all,
+                         const float* P, const float* scale, const DevRowSpace& ds, T* Out, int64_t ld_out, int M,
+                         int N, int K, int R, cudaStream_t st) {
+  if (M <= 0) return MLORA_OK;
+  dim3 grid((N + 31) / 32, (M + 31) / 32), block(32, 32);
+  LaunchScope scope(ctx, st, KIND_SIMT);
+  simt::gemm_lora_kernel<T, W_KMAJOR><<<grid, block, 0, st>>>(In, ld_in, W, ldw, L_all, P, scale, ds.row_adapter, Out,
+                                                              ld_out, M, N, K, R);
+  return scope.done();
+}
+
+template <typename T>
+mlora_status_t simt_grad(mlora_ctx* ctx, const mlora_plan* p, const float* P, int R, const float* scale, const T* Q,
+                         int64_t ldq, int D, float* G, int accumulate, cudaStream_t st) {
+  const int n_slots = (int)p->h.ft_adapters.size();
+  if (n_slots <= 0) return MLORA_OK;
+  dim3 grid((D + 127) / 128, R, n_slots);
+  LaunchScope scope(ctx, st, KIND_SIMT);
+  simt::grad_kernel<T><<<grid, 128, 0, st>>>(P, R, scale, Q, ldq, D, G, p->slot_chunk_off, p->chunk_row0,
+                                             p->chunk_nrows, p->slot_adapter, accumulate);
+  return scope.done();
+}
+
+template <typename T>
+mlora_status_t forward_simt(mlora_ctx* ctx, const mlora_layer_t* L, const mlora_plan* p, const void* X, int64_t ldx,
+                            void* Y, int64_t ldy, void* x_save, float* u_save, int64_t save_base, cudaStream_t st) {
+  mlora_status_t s = simt_shrink<T>(ctx, (const T*)X, ldx, L->d_in, L->rank, (const T*)L->A_all, nullptr, p->fwd,
+                                    ctx->ws_p, (T*)x_save, u_save, save_base, p->h.n_rows, st);
+  if (s != MLORA_OK) return s;
+  return simt_gemm<T, false>(ctx, (const T*)X, ldx, (const T*)L->W, L->ldw, (const T*)L->B_all, ctx->ws_p, L->scale,
+                             p->fwd, (T*)Y, ldy, p->h.n_rows, L->d_out, L->d_in, L->rank, st);
+}
+
+template <typename T>
+mlora_status_t backward_simt(mlora_ctx* ctx, const mlora_layer_t* L, const mlora_plan* p, const void* dY, int64_t lddy,
+                             const void* x_save, const float* u_save, float* dA, float* dB, void* dX, int64_t lddx,
+                             int accumulate, cudaStream_t st) {
+  const int Tft = p->h.ft_rows;
+  mlora_status_t s = simt_shrink<T>(ctx, (const T*)dY, lddy, L->d_out, L->rank, (const T*)L->B_all, L->scale, p->bwd,
+                                    ctx->ws_p, (T*)nullptr, nullptr, 0, Tft, st);
+  if (s != MLORA_OK) return s;
+  if ((s = simt_grad<T>(ctx, p, u_save, L->rank, L->scale, (const T*)dY, lddy, L->d_out, dB, accumulate, st)) != MLORA_OK)
+    return s;
+  if ((s = simt_grad<T>(ctx, p, ctx->ws_p, L->rank, nullptr, (const T*)x_save, L->d_in, L->d_in, dA, accumulate, st)) !=
+      MLORA_OK)
+    return s;
+  if (dX)
+    s = simt_gemm<T, true>(ctx, (const T*)dY, lddy, (const T*)L->W, L->ldw, (const T*)L->A_all, ctx->ws_p, nullptr,
+                           p->bwd, (T*)dX, lddx, Tft, L->d_in, L->d_out, L->rank, st);
+  return s;
+}
+
+}  // namespace
+
+// =============================================================================================
+extern "C" {
+
+const char* mlora_status_string(mlora_status_t s) {
+  switch (s) {
+    case MLORA_OK: return "ok";
+    case MLORA_ERR_INVALID_ARG: return "invalid argument";
+    case MLORA_ERR_SEGMENT_RANGE: return "segment outside the batch rows";
+    case MLORA_ERR_SEGMENT_OVERLAP: return "segments overlap";
+    case MLORA_ERR_ADAPTER_ID: return "adapter id out of range (or fine-tuning segment without adapter)";
+    case MLORA_ERR_SAVE_CAPACITY: return "fine-tuning rows exceed the activation buffer capacity";
+    case MLORA_ERR_UNSUPPORTED: return "shape, rank or alignment not supported";
+    case MLORA_ERR_ARCH: return "no sm_100 CUDA device";
+    case MLORA_ERR_CUDA: return "CUDA call failed";
+    case MLORA_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+  }
+  return "unknown status";
+}
+
+mlora_status_t mlora_create(mlora_ctx** out, int device) {
+  if (!out) return MLORA_ERR_INVALID_ARG;
+  *out = nullptr;
+  int n = 0;
+  if (cudaGetDeviceCount(&n) != cudaSuccess || n <= 0) { cudaGetLastError(); return MLORA_ERR_ARCH; }
+  if (device < 0 || device >= n) return MLORA_ERR_INVALID_ARG;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MLORA_ERR_CUDA;
+  if (prop.major != 10) return MLORA_ERR_ARCH;
+  if (cudaSetDevice(device) != cudaSuccess) return MLORA_ERR_CUDA;
+  mlora_ctx* c = new (std::nothrow) mlora_ctx();
+  if (!c) return MLORA_ERR_INVALID_ARG;
+  c->device = device;
+  c->sm_count = prop.multiProcessorCount;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+      q != cudaDriverEntryPointSuccess || !fn) {
+    delete c;
+    return MLORA_ERR_CUDA;
+  }
+  c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if (cudaMalloc(&c->status_dev, sizeof(int32_t)) != cudaSuccess ||
+      cudaMemset(c->status_dev, 0, sizeof(int32_t)) != cudaSuccess) {
+    delete c;
+    return MLORA_ERR_CUDA;
+  }
+  *out = c;
+  return MLORA_OK;
+}
+
+mlora_status_t mlora_profile_enable(mlora_ctx* c, int32_t max_records) {
+  if (!c || max_records < 0) return MLORA_ERR_INVALID_ARG;
+  if (cudaSetDevice(c->device) != cudaSuccess) return MLORA_ERR_CUDA;
+  for (cudaEvent_t e : c->ev_start) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->ev_stop) cudaEventDestroy(e);
+  c->ev_start.clear(); c->ev_stop.clear(); c->ev_kind.clear(); c->ev_used = 0;
+  for (int32_t i = 0; i < max_records; ++i) {
+    cudaEvent_t a, b;
+    if (cudaEventCreate(&a) != cudaSuccess) return MLORA_ERR_CUDA;
+    if (cudaEventCreate(&b) != cudaSuccess) { cudaEventDestroy(a); return MLORA_ERR_CUDA; }
+    c->ev_start.push_back(a); c->ev_stop.push_back(b); c->ev_kind.push_back(0);
+  }
+  return MLORA_OK;
+}
+
+int32_t mlora_profile_collect(mlora_ctx* c, int32_t* kinds, float* ms, int32_t cap) {
+  if (!c) return 0;
+  cudaSetDevice(c->device);
+  cudaDeviceSynchronize();
+  const int32_t n = c->ev_used;
+  for (int32_t i = 0; i < n && i < cap; ++i) {
+    float t = 0.f;
+    cudaEventElapsedTime(&t, c->ev_start[i], c->ev_stop[i]);
+    if (kinds) kinds[i] = c->ev_kind[i];
+    if (ms) ms[i] = t;
+  }
+  c->ev_used = 0;
+  return n;
+}
+
+void mlora_destroy(mlora_ctx* c) {
+  if (!c) return;
+  cudaSetDevice(c->device);
+  for (cudaEvent_t e : c->ev_start) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->ev_stop) cudaEventDestroy(e);
+  cudaFree(c->status_dev);
+  cudaFree(c->ws_p);
+  delete c;
+}
+
+mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, int32_t n_segs, int32_t n_rows,
+                                 int32_t n_adapters, mlora_plan** out) {
+  if (!out) return MLORA_ERR_INVALID_ARG;
+  *out = nullptr;
+  mlora_plan* p = new (std::nothrow) mlora_plan();
+  if (!p) return MLORA_ERR_INVALID_ARG;
+  mlora_status_t s = build_plan(segs, n_segs, n_rows, n_adapters, p->h);
+  if (s != MLORA_OK) { delete p; return s; }
+  p->ctx = ctx;
+  if (ctx) {
+    if (cudaSetDevice(ctx->device) != cudaSuccess) { delete p; return MLORA_ERR_CUDA; }
+    BlobBuilder b;
+    const HostPlan& h = p->h;
+    size_t o[32]; int n = 0;
+    const RowSpace* rs[2] = {&h.fwd, &h.bwd};
+    for (int i = 0; i < 2; ++i) {
+      o[n++] = b.add(rs[i]->row_adapter); o[n++] = b.add(rs[i]->row_save); o[n++] = b.add(rs[i]->row_grp);
+      o[n++] = b.add(rs[i]->tile_grp_off); o[n++] = b.add(rs[i]->grp_adapter); o[n++] = b.add(rs[i]->item_row0);
+      o[n++] = b.add(rs[i]->item_nrows); o[n++] = b.add(rs[i]->item_adapter); o[n++] = b.add(rs[i]->item_save0);
+    }
+    o[n++] = b.add(h.slot_chunk_off); o[n++] = b.add(h.chunk_row0); o[n++] = b.add(h.chunk_nrows);
+    o[n++] = b.add(h.ft_adapters);
+    if (cudaMalloc(&p->blob, b.data.size() * sizeof(int32_t)) != cudaSuccess) { delete p; return MLORA_ERR_CUDA; }
+    if (cudaMemcpy(p->blob, b.data.data(), b.data.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
+      cudaFree(p->blob); delete p; return MLORA_ERR_CUDA;
+    }
+    DevRowSpace* ds[2] = {&p->fwd, &p->bwd};
+    n = 0;
+    for (int i = 0; i < 2; ++i) {
+      ds[i]->row_adapter = p->blob + o[n++]; ds[i]->row_save = p->blob + o[n++]; ds[i]->row_grp = p->blob + o[n++];
+      ds[i]->tile_grp_off = p->blob + o[n++]; ds[i]->grp_adapter = p->blob + o[n++]; ds[i]->item_row0 = p->blob + o[n++];
+      ds[i]->item_nrows = p->blob + o[n++]; ds[i]->item_adapter = p->blob + o[n++]; ds[i]->item_save0 = p->blob + o[n++];
+    }
+    p->bwd.row_save = nullptr;       // the compact space has no save offsets
+    p->bwd.item_save0 = nullptr;
+    p->slot_chunk_off = p->blob + o[n++]; p->chunk_row0 = p->blob + o[n++]; p->chunk_nrows = p->blob + o[n++];
+    p->slot_adapter = p->blob + o[n++];
+    if (n_rows > ctx->ws_rows) {     // grow the rank-r workspace (the only other device allocation)
+      if (cudaDeviceSynchronize() != cudaSuccess) { cudaFree(p->blob); delete p; return MLORA_ERR_CUDA; }
+      cudaFree(ctx->ws_p);
+      ctx->ws_p = nullptr; ctx->ws_rows = 0;
+      if (cudaMalloc(&ctx->ws_p, (size_t)n_rows * kMaxRank * sizeof(float)) != cudaSuccess) {
+        cudaFree(p->blob); delete p; return MLORA_ERR_CUDA;
+      }
+      ctx->ws_rows = n_rows;
+    }
+  }
+  *out = p;
+  return MLORA_OK;
+}
+
+void mlora_plan_destroy(mlora_plan* p) {
+  if (!p) return;
+  if (p->blob) { if (p->ctx) cudaSetDevice(p->ctx->device); cudaFree(p->blob); }
+  delete p;
+}
+
+int32_t mlora_plan_rows(const mlora_plan* p) { return p ? p->h.n_rows : 0; }
+int32_t mlora_plan_ft_rows(const mlora_plan* p) { return p ? p->h.ft_rows : 0; }
+int32_t mlora_plan_ft_adapters(const mlora_plan* p, int32_t* ids, int32_t cap) {
+  if (!p) return 0;
+  const int32_t n = (int32_t)p->h.ft_adapters.size();
+  for (int32_t i = 0; ids && i < n && i < cap; ++i) ids[i] = p->h.ft_adapters[i];
+  return n;
+}
+mlora_status_t mlora_plan_describe(const mlora_plan* p, int32_t* seg_save_offset, int32_t* row_adapter) {
+  if (!p) return MLORA_ERR_INVALID_ARG;
+  if (seg_save_offset) for (int32_t k = 0; k < p->h.n_segs; ++k) seg_save_offset[k] = p->h.seg_save_off[k];
+  if (row_adapter) for (int32_t t = 0; t < p->h.n_rows; ++t) row_adapter[t] = p->h.fwd.row_adapter[t];
+  return MLORA_OK;
+}
+
+mlora_status_t mlora_mixed_forward(mlora_ctx* ctx, const mlora_layer_t* L, const mlora_plan* p, const void* X,
+                                   int64_t ldx, void* Y, int64_t ldy, void* x_save, float* u_save,
+                                   int64_t save_row_base, int64_t save_capacity_rows, void* cuda_stream) {
+  if (!ctx || !p || p->ctx != ctx || !p->blob) return MLORA_ERR_INVALID_ARG;
+  mlora_status_t s = check_layer(L);
+  if (s != MLORA_OK) return s;
+  const HostPlan& h = p->h;
+  if (h.n_adapters > L->n_adapters) return MLORA_ERR_ADAPTER_ID;
+  if (h.n_rows == 0) return MLORA_OK;
+  if (!X || !Y || ldx < L->d_in || ldy < L->d_out) return MLORA_ERR_INVALID_ARG;
+  if (save_row_base < 0 || save_capacity_rows < 0) return MLORA_ERR_INVALID_ARG;
+  if (h.ft_rows > 0) {
+    if (save_row_base + h.ft_rows > save_capacity_rows) return MLORA_ERR_SAVE_CAPACITY;
+    if (!u_save) return MLORA_ERR_INVALID_ARG;
+  }
+  if (h.n_rows > ctx->ws_rows) return MLORA_ERR_INVALID_ARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (L->dtype == MLORA_F32)
+    return forward_simt<float>(ctx, L, p, X, ldx, Y, ldy, x_save, u_save, save_row_base, st);
+  if (ldx % 8 || ldy % 8 || !aligned16(X) || !aligned16(Y) || (x_save && !aligned16(x_save))) return MLORA_ERR_UNSUPPORTED;
+  if (ctx->gemm_path == 1)
+    return forward_simt<__nv_bfloat16>(ctx, L, p, X, ldx, Y, ldy, x_save, u_save, save_row_base, st);
+
+  ShrinkArgs sa;
+  sa.In = (const __nv_bfloat16*)X; sa.ld_in = ldx; sa.D = L->d_in;
+  sa.P_all = (const __nv_bfloat16*)L->A_all; sa.scale = nullptr; sa.Out = ctx->ws_p;
+  sa.item_row0 = p->fwd.item_row0; sa.item_nrows = p->fwd.item_nrows; sa.item_adapter = p->fwd.item_adapter;
+  sa.item_save0 = p->fwd.item_save0;
+  sa.x_save = (__nv_bfloat16*)x_save; sa.u_save = u_save; sa.save_base = save_row_base;
+  if ((s = launch_shrink(ctx, L->rank, sa, h.fwd.n_items(), st)) != MLORA_OK) return s;
+  return gemm_bf16<false>(ctx, L, h.fwd, p->fwd, X, ldx, Y, ldy, L->B_all, ctx->ws_p, L->scale, h.n_rows, L->d_out,
+                          L->d_in, st);
+}
+
+mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlora_plan* p, const void* dY, int64_t lddy,
+                              const void* x_save, const float* u_save, float* dA, float* dB, void* dX, int64_t lddx,
+                              int32_t accumulate, void* cuda_stream) {
+  if (!ctx || !p || p->ctx != ctx || !p->blob) return MLORA_ERR_INVALID_ARG;
+  mlora_status_t s = check_layer(L);
+  if (s != MLORA_OK) return s;
+  const HostPlan& h = p->h;
+  if (h.n_adapters > L->n_adapters) return MLORA_ERR_ADAPTER_ID;
+  if (h.ft_rows == 0) return MLORA_OK;
+  if (!dY || !x_save || !u_save || !dA || !dB || lddy < L->d_out || (dX && lddx < L->d_in)) return MLORA_ERR_INVALID_ARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (L->dtype == MLORA_F32)
+    return backward_simt<float>(ctx, L, p, dY, lddy, x_save, u_save, dA, dB, dX, lddx, accumulate, st);
+  if (lddy % 8 || (dX && lddx % 8) || !aligned16(dY) || !aligned16(x_save) || (dX && !aligned16(dX)))
+    return MLORA_ERR_UNSUPPORTED;
+  if (ctx->gemm_path == 1)
+    return backward_simt<__nv_bfloat16>(ctx, L, p, dY, lddy, x_save, u_save, dA, dB, dX, lddx, accumulate, st);
+
+  const int n_slots = (int)h.ft_adapters.size();
+  ShrinkArgs sa;                     // V = s dY B^T
+  sa.In = (const __nv_bfloat16*)dY; sa.ld_in = lddy; sa.D = L->d_out;
+  sa.P_all = (const __nv_bfloat16*)L->B_all; sa.scale = L->scale; sa.Out = ctx->ws_p;
+  sa.item_row0 = p->bwd.item_row0; sa.item_nrows = p->bwd.item_nrows; sa.item_adapter = p->bwd.item_adapter;
+  sa.item_save0 = nullptr; sa.x_save = nullptr; sa.u_save = nullptr; sa.save_base = 0;
+  if ((s = launch_shrink(ctx, L->rank, sa, h.bwd.n_items(), st)) != MLORA_OK) return s;
+
+  GradArgs ga;                       // dB = (s U)^T dY
+  ga.P = u_save; ga.R = L->rank; ga.scale = L->scale; ga.Q = (const __nv_bfloat16*)dY; ga.ldq = lddy; ga.D = L->d_out;
+  ga.G = dB; ga.slot_chunk_off = p->slot_chunk_off; ga.chunk_row0 = p->chunk_row0; ga.chunk_nrows = p->chunk_nrows;
+  ga.slot_adapter = p->slot_adapter; ga.accumulate = accumulate;
+  if ((s = launch_grad(ctx, ga, n_slots, st)) != MLORA_OK) return s;
+  ga.P = ctx->ws_p; ga.scale = nullptr; ga.Q = (const __nv_bfloat16*)x_save; ga.ldq = L->d_in; ga.D = L->d_in;
+  ga.G = dA;                         // dA = V^T X
+  if ((s = launch_grad(ctx, ga, n_slots, st)) != MLORA_OK) return s;
+  if (!dX) return MLORA_OK;
+  return gemm_bf16<true>(ctx, L, h.bwd, p->bwd, dY, lddy, dX, lddx, L->A_all, ctx->ws_p, nullptr, h.ft_rows, L->d_in,
+                         L->d_out, st);
+}
+
+mlora_status_t mlora_poll_status(mlora_ctx* ctx, void* cuda_stream) {
+  if (!ctx) return MLORA_ERR_INVALID_ARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  int32_t v = 0;
+  if (cudaMemcpyAsync(&v, ctx->status_dev, sizeof(v), cudaMemcpyDeviceToHost, st) != cudaSuccess) return MLORA_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return MLORA_ERR_CUDA;
+  if (v != 0) {
+    cudaMemsetAsync(ctx->status_dev, 0, sizeof(v), st);
+    cudaStreamSynchronize(st);
+  }
+  return (mlora_status_t)v;
+}
+
+int64_t mlora_launch_count(const mlora_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path) {
+  if (!ctx || (path != 0 && path != 1)) return MLORA_ERR_INVALID_ARG;
+  ctx->gemm_path = path;
+  return MLORA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,147 @@
+// Host-side planning for the mixed-batch multi-LoRA layer: segment table -> validated routing
+// and the work lists the kernels consume.  Pure C++ (no CUDA), so it can be exercised without a
+// GPU through the C ABI (mlora_plan_create with a null context).
+#pragma once
+
+#include <cstdint>
+#include <vector>
+
+#include "mlora.h"
+
+namespace mlora {
+
+constexpr int kTileRows = 128;     // rows per tensor-core tile (UMMA M)
+constexpr int kItemRows = 16;      // rows per skinny-kernel work item (mma.sync M)
+constexpr int kMaxRank = 128;
+
+// Tables over one row space: the batch rows (forward) or the compact fine-tuning rows (backward).
+struct RowSpace {
+  int32_t n_rows = 0;
+  std::vector<int32_t> row_adapter;    // [n_rows] adapter id or -1
+  std::vector<int32_t> row_save;       // [n_rows] save offset of the row or -1 (forward space only)
+  // Tensor-core tiles of kTileRows rows: the distinct adapters of a tile ("groups", in order of
+  // first appearance) and, per row, the index of its group inside its tile (-1: base only).
+  std::vector<int32_t> row_grp;        // [n_rows]
+  std::vector<int32_t> tile_grp_off;   // [n_tiles + 1]
+  std::vector<int32_t> grp_adapter;    // [tile_grp_off.back()]
+  // Skinny-kernel items: runs of <= kItemRows consecutive rows bound to one adapter whose save
+  // offsets (if any) are consecutive too.
+  std::vector<int32_t> item_row0, item_nrows, item_adapter, item_save0;
+  int32_t n_tiles() const { return (n_rows + kTileRows - 1) / kTileRows; }
+  int32_t n_items() const { return (int32_t)item_row0.size(); }
+};
+
+struct HostPlan {
+  int32_t n_rows = 0, n_adapters = 0, n_segs = 0;
+  int32_t ft_rows = 0;
+  std::vector<int32_t> seg_save_off;   // [n_segs] save offset or -1
+  std::vector<int32_t> ft_adapters;    // slot -> adapter id
+  RowSpace fwd;                        // batch rows
+  RowSpace bwd;                        // compact fine-tuning rows, in save order
+  // Gradient work: per slot, chunks of <= kItemRows compact rows.
+  std::vector<int32_t> slot_chunk_off; // [n_slots + 1]
+  std::vector<int32_t> chunk_row0, chunk_nrows;
+};
+
+inline void build_tiles_and_items(RowSpace& rs) {
+  const int32_t n = rs.n_rows;
+  rs.row_grp.assign(n, -1);
+  rs.tile_grp_off.assign(1, 0);
+  rs.grp_adapter.clear();
+  for (int32_t t0 = 0; t0 < n; t0 += kTileRows) {
+    const int32_t t1 = t0 + kTileRows < n ? t0 + kTileRows : n;
+    const int32_t base = (int32_t)rs.grp_adapter.size();
+    for (int32_t t = t0; t < t1; ++t) {
+      const int32_t a = rs.row_adapter[t];
+      if (a < 0) continue;
+      int32_t g = -1;
+      for (int32_t i = base; i < (int32_t)rs.grp_adapter.size(); ++i)
+        if (rs.grp_adapter[i] == a) { g = i - base; break; }
+      if (g < 0) { g = (int32_t)rs.grp_adapter.size() - base; rs.grp_adapter.push_back(a); }
+      rs.row_grp[t] = g;
+    }
+    rs.tile_grp_off.push_back((int32_t)rs.grp_adapter.size());
+  }
+  rs.item_row0.clear(); rs.item_nrows.clear(); rs.item_adapter.clear(); rs.item_save0.clear();
+  const bool has_save = !rs.row_save.empty();
+  int32_t t = 0;
+  while (t < n) {
+    const int32_t a = rs.row_adapter[t];
+    if (a < 0) { ++t; continue; }
+    const int32_t s0 = has_save ? rs.row_save[t] : -1;
+    int32_t len = 1;
+    while (t + len < n && len < kItemRows && rs.row_adapter[t + len] == a) {
+      const int32_t s = has_save ? rs.row_save[t + len] : -1;
+      if (s0 >= 0 ? (s != s0 + len) : (s >= 0)) break;
+      ++len;
+    }
+    rs.item_row0.push_back(t); rs.item_nrows.push_back(len);
+    rs.item_adapter.push_back(a); rs.item_save0.push_back(s0);
+    t += len;
+  }
+}
+
+// Validates the table and fills `p`.  Returns MLORA_OK or the error the header documents.
+inline mlora_status_t build_plan(const mlora_segment_t* segs, int32_t n_segs, int32_t n_rows,
+                                 int32_t n_adapters, HostPlan& p) {
+  if (n_segs < 0 || n_rows < 0 || n_adapters < 0 || (n_segs > 0 && segs == nullptr))
+    return MLORA_ERR_INVALID_ARG;
+  p = HostPlan();
+  p.n_rows = n_rows; p.n_adapters = n_adapters; p.n_segs = n_segs;
+  p.fwd.n_rows = n_rows;
+  p.fwd.row_adapter.assign(n_rows, -1);
+  p.fwd.row_save.assign(n_rows, -1);
+  p.seg_save_off.assign(n_segs, -1);
+  std::vector<uint8_t> taken(n_rows, 0);
+  // pass 1: ranges and adapter ids, so that the error reported does not depend on table order
+  for (int32_t k = 0; k < n_segs; ++k) {
+    const mlora_segment_t& s = segs[k];
+    if (s.row_len < 0 || s.row_start < 0 || (int64_t)s.row_start + s.row_len > n_rows)
+      return MLORA_ERR_SEGMENT_RANGE;
+    if (s.adapter_id < -1 || s.adapter_id >= n_adapters) return MLORA_ERR_ADAPTER_ID;
+    if (s.is_finetune && s.adapter_id < 0) return MLORA_ERR_ADAPTER_ID;
+  }
+  int32_t off = 0;
+  for (int32_t k = 0; k < n_segs; ++k) {
+    const mlora_segment_t& s = segs[k];
+    for (int32_t i = 0; i < s.row_len; ++i) {
+      const int32_t t = s.row_start + i;
+      if (taken[t]) return MLORA_ERR_SEGMENT_OVERLAP;
+      taken[t] = 1;
+      p.fwd.row_adapter[t] = s.adapter_id;
+      if (s.is_finetune) p.fwd.row_save[t] = off + i;
+    }
+    if (s.is_finetune) {
+      p.seg_save_off[k] = off;
+      off += s.row_len;
+      bool seen = false;
+      for (int32_t a : p.ft_adapters) seen = seen || (a == s.adapter_id);
+      if (!seen) p.ft_adapters.push_back(s.adapter_id);
+    }
+  }
+  p.ft_rows = off;
+  build_tiles_and_items(p.fwd);
+
+  // compact fine-tuning row space (save order) and the gradient chunk lists
+  p.bwd.n_rows = p.ft_rows;
+  p.bwd.row_adapter.assign(p.ft_rows, -1);
+  for (int32_t k = 0; k < n_segs; ++k) {
+    if (!segs[k].is_finetune) continue;
+    for (int32_t i = 0; i < segs[k].row_len; ++i) p.bwd.row_adapter[p.seg_save_off[k] + i] = segs[k].adapter_id;
+  }
+  build_tiles_and_items(p.bwd);
+  p.slot_chunk_off.assign(1, 0);
+  for (int32_t a : p.ft_adapters) {
+    for (int32_t k = 0; k < n_segs; ++k) {
+      if (!segs[k].is_finetune || segs[k].adapter_id != a) continue;
+      for (int32_t i = 0; i < segs[k].row_len; i += kItemRows) {
+        p.chunk_row0.push_back(p.seg_save_off[k] + i);
+        p.chunk_nrows.push_back(segs[k].row_len - i < kItemRows ? segs[k].row_len - i : kItemRows);
+      }
+    }
+    p.slot_chunk_off.push_back((int32_t)p.chunk_row0.size());
+  }
+  return MLORA_OK;
+}
+
+}  // namespace mlora

@@ -1,0 +1,334 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element.
+
+Tolerances: bf16 layers  |err| <= 2e-2 (1 + |ref|)  (bf16 storage, fp32 accumulation);
+fp32 layers |err| <= 1e-4 (1 + |ref|).  Routing and the activation-save indexing are checked
+bit for bit (saved rows of X, and the exact-integer probe where every output is an integer).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mlora_oracle as orc
+from paper_2607_28848_b200 import binding as mb
+from paper_2607_28848_b200 import synth
+from paper_2607_28848_b200.runner import LayerRun, Session
+from probes import integer_probe
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"bf16": 2e-2, "f32": 1e-4}
+
+
+@pytest.fixture(scope="module")
+def sess():
+    s = Session(0)
+    yield s
+    s.close()
+
+
+def assert_close(name, got, ref, tol):
+    got, ref = np.asarray(got, dtype=np.float64), np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape, (name, got.shape, ref.shape)
+    assert np.isfinite(got).all(), f"{name}: non-finite values"
+    excess = np.abs(got - ref) - tol * (1.0 + np.abs(ref))
+    if excess.size and excess.max() > 0:
+        i = np.unravel_index(np.argmax(excess), excess.shape)
+        raise AssertionError(f"{name}: |err| {abs(got[i] - ref[i]):.4g} at {i} (got {got[i]:.6g}, ref {ref[i]:.6g}), "
+                             f"{int((excess > 0).sum())} of {excess.size} outside tolerance {tol}")
+
+
+def run_and_check(sess, w, t, path=0, check_backward=True, tol=None, base=0, cap=None, blocked=False):
+    tol = TOL[w.dtype] if tol is None else tol
+    mb.mlora_set_gemm_path(sess.ctx, path)
+    run = LayerRun(sess, w.dtype, t, w.segments, w.n_rows, save_row_base=base, save_capacity_rows=cap, guard=True)
+    try:
+        run.forward()
+        assert run.status() == mb.MLORA_OK
+        fwd = (orc.forward_blocked if blocked else orc.forward)(t["X"], t["W"], t["A_all"], t["B_all"], t["scale"],
+                                                                 w.segments)
+        assert_close("Y", run.host(run.Y), fwd["Y"], tol)
+        n = run.ft_rows
+        assert n == fwd["ft_rows"] and run.slots == fwd["ft_adapters"]
+        if n:
+            xs = run.host(run.x_save)[base:base + n]
+            assert np.array_equal(xs, fwd["x_save"][:n]), "saved rows of X must be bit-exact copies"
+            assert_close("u_save", run.host(run.u_save)[base:base + n], fwd["u_save"][:n], min(tol, 1e-3))
+        # guard: rows of the activation buffer outside [base, base + n) are untouched
+        assert torch.isnan(run.u_save[:base]).all() and torch.isnan(run.u_save[base + n:]).all()
+        assert torch.isnan(run.x_save[:base].float()).all() and torch.isnan(run.x_save[base + n:].float()).all()
+        if check_backward and n:
+            run.backward()
+            assert run.status() == mb.MLORA_OK
+            bwd = (orc.backward_blocked if blocked else orc.backward)(
+                t["dY"], t["W"], t["A_all"], t["B_all"], t["scale"], w.segments, fwd["x_save"], fwd["u_save"],
+                n_rows=w.n_rows)
+            assert_close("dX", run.host(run.dX)[:n], bwd["dX"], tol)
+            assert_close("dA", run.host(run.dA), bwd["dA"], tol)
+            assert_close("dB", run.host(run.dB), bwd["dB"], tol)
+        return run
+    finally:
+        mb.mlora_set_gemm_path(sess.ctx, 0)
+        run.close()
+
+
+# ------------------------------------------------------------------------------------------
+def test_cfg1_tiny_fp32(sess):
+    w = synth.cfg1_tiny()
+    run_and_check(sess, w, synth.make_tensors(w))
+
+
+@pytest.mark.parametrize("path", [0, 1])
+def test_bf16_ragged_multi_tile(sess, path):
+    w = synth.random_workload(5, 256, 512, 16, 6, 389, max_seg=150)
+    run_and_check(sess, w, synth.make_tensors(w), path=path)
+
+
+def test_fp32_ragged(sess):
+    w = synth.random_workload(6, 96, 160, 12, 5, 201, dtype="f32", max_seg=60)
+    run_and_check(sess, w, synth.make_tensors(w))
+
+
+@pytest.mark.parametrize("rank", [8, 16, 32, 64, 128])
+def test_rank_sweep(sess, rank):
+    w = synth.random_workload(10 + rank, 320, 448, rank, 7, 300, max_seg=90)
+    run_and_check(sess, w, synth.make_tensors(w))
+
+
+@pytest.mark.parametrize("rank", [8, 32])
+def test_every_row_its_own_adapter(sess, rank):
+    """Decode-style tiles: up to 128 distinct adapters inside one 128-row tile."""
+    n = 150
+    ad = np.random.default_rng(1).permutation(n)
+    segs = [(i, 1, int(ad[i]), 0) for i in range(n)] + [(n, 70, 3, 1)]
+    w = synth.Workload("decode_tile", 256, 320, rank, n, "bf16", n + 70, synth.segments_array(segs))
+    run_and_check(sess, w, synth.make_tensors(w))
+
+
+@pytest.mark.parametrize("lens", [[0, 1, 127, 128, 129], [128, 128], [1], [300]])
+def test_segment_lengths_around_a_tile(sess, lens):
+    segs, row = [], 0
+    for i, ln in enumerate(lens):
+        segs.append((row, ln, i % 3, i % 2))
+        row += ln
+    w = synth.Workload("edges", 128, 256, 16, 3, "bf16", max(row, 1), synth.segments_array(segs))
+    run_and_check(sess, w, synth.make_tensors(w))
+
+
+def test_base_only_rows_and_no_finetune(sess):
+    segs = [(0, 40, -1, 0), (60, 30, 1, 0)]      # rows 40..59 and 90..99 uncovered
+    w = synth.Workload("base_only", 192, 256, 16, 2, "bf16", 100, synth.segments_array(segs))
+    t = synth.make_tensors(w)
+    run = run_and_check(sess, w, t)
+    assert run.ft_rows == 0
+    w2 = synth.Workload("no_segments", 192, 256, 16, 2, "bf16", 100, np.zeros((0, 4), np.int32))
+    run_and_check(sess, w2, synth.make_tensors(w2))
+
+
+def test_empty_batch_is_a_no_op(sess):
+    plan = mb.mlora_plan_create(sess.ctx, np.zeros((0, 4), np.int32), 0, 2)
+    w = synth.Workload("x", 64, 64, 8, 2, "bf16", 4, synth.segments_array([(0, 4, 0, 0)]))
+    run = LayerRun(sess, "bf16", synth.make_tensors(w), w.segments, 4)
+    mb.mlora_mixed_forward(sess.ctx, run.layer, plan, None, None, None, None, 0, 0)
+    mb.mlora_backward(sess.ctx, run.layer, plan, None, None, None, None, None, None)
+    assert mb.mlora_poll_status(sess.ctx) == mb.MLORA_OK
+    mb.mlora_plan_destroy(plan)
+    run.close()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_integer_probe_bit_exact(sess, dtype):
+    p = integer_probe(n_rows=333, d_in=128, d_out=192, rank=16, n_adapters=9, seed=4, dtype=dtype)
+    w = synth.Workload("probe", 128, 192, 16, 9, dtype, 333, p["segments"])
+    fwd = orc.forward(p["X"], p["W"], p["A_all"], p["B_all"], p["scale"], p["segments"])
+    run = LayerRun(sess, dtype, p, p["segments"], 333, guard=True)
+    try:
+        run.forward()
+        assert run.status() == mb.MLORA_OK
+        n = run.ft_rows
+        assert np.array_equal(run.host(run.Y), fwd["Y"])
+        assert np.array_equal(run.host(run.x_save)[:n], fwd["x_save"])
+        assert np.array_equal(run.host(run.u_save)[:n], fwd["u_save"])
+        run.backward()
+        bwd = orc.backward(p["dY"], p["W"], p["A_all"], p["B_all"], p["scale"], p["segments"], fwd["x_save"],
+                           fwd["u_save"], n_rows=333)
+        assert np.array_equal(run.host(run.dX)[:n], bwd["dX"])
+        assert np.array_equal(run.host(run.dA), bwd["dA"])
+        assert np.array_equal(run.host(run.dB), bwd["dB"])
+    finally:
+        run.close()
+
+
+def test_append_two_steps_then_one_backward(sess):
+    """Two forward steps append into one activation buffer; one backward consumes both
+    (activations accumulate until a backward batch is full)."""
+    d_in, d_out, r, n_ad = 128, 192, 16, 4
+    w1 = synth.Workload("s1", d_in, d_out, r, n_ad, "bf16", 90, synth.segments_array([(0, 50, 0, 0), (50, 40, 2, 1)]))
+    w2 = synth.Workload("s2", d_in, d_out, r, n_ad, "bf16", 70, synth.segments_array([(0, 30, 3, 1), (30, 40, 1, 0)]),
+                        tag_base=50)
+    t1, t2 = synth.make_tensors(w1), synth.make_tensors(w2)
+    t2["W"], t2["A_all"], t2["B_all"] = t1["W"], t1["A_all"], t1["B_all"]
+    cap = 70
+    r1 = LayerRun(sess, "bf16", t1, w1.segments, 90, save_row_base=0, save_capacity_rows=cap)
+    r2 = LayerRun(sess, "bf16", t2, w2.segments, 70, save_row_base=40, save_capacity_rows=cap)
+    r2.x_save, r2.u_save = r1.x_save, r1.u_save          # one shared activation buffer
+    r1.forward()
+    r2.forward()
+    # backward over all 70 saved rows: a fine-tune-only table in save order
+    segs_b = synth.segments_array([(0, 40, 2, 1), (40, 30, 3, 1)])
+    dY = np.concatenate([t1["dY"], t2["dY"]])
+    tb = dict(t1, X=np.zeros((70, d_in), np.float32), dY=dY)
+    rb = LayerRun(sess, "bf16", tb, segs_b, 70)
+    rb.x_save, rb.u_save = r1.x_save, r1.u_save
+    rb.backward()
+    assert rb.status() == mb.MLORA_OK
+    f1 = orc.forward(t1["X"], t1["W"], t1["A_all"], t1["B_all"], t1["scale"], w1.segments)
+    f2 = orc.forward(t2["X"], t1["W"], t1["A_all"], t1["B_all"], t1["scale"], w2.segments)
+    xs = np.concatenate([f1["x_save"], f2["x_save"]])
+    us = np.concatenate([f1["u_save"], f2["u_save"]])
+    assert np.array_equal(rb.host(r1.x_save)[:70], xs)
+    ref = orc.backward(dY, t1["W"], t1["A_all"], t1["B_all"], t1["scale"], segs_b, xs, us, n_rows=70)
+    assert rb.slots == ref["ft_adapters"] == [2, 3]
+    assert_close("dA", rb.host(rb.dA), ref["dA"], 2e-2)
+    assert_close("dB", rb.host(rb.dB), ref["dB"], 2e-2)
+    assert_close("dX", rb.host(rb.dX), ref["dX"], 2e-2)
+    # the buffer is full now: one more fine-tuning row must be refused before anything runs
+    with pytest.raises(mb.MloraError) as e:
+        mb.mlora_mixed_forward(sess.ctx, r2.layer, r2.plan, r2.X, r2.Y, r1.x_save, r1.u_save, 41, cap)
+    assert e.value.status == mb.MLORA_ERR_SAVE_CAPACITY
+    for r_ in (r1, r2, rb):
+        r_.close()
+
+
+def test_accumulate_and_optional_outputs(sess):
+    w = synth.random_workload(21, 128, 192, 16, 4, 260, max_seg=80, p_finetune=0.5)
+    t = synth.make_tensors(w)
+    run = LayerRun(sess, "bf16", t, w.segments, w.n_rows, save_x=True)
+    run.forward()
+    run.backward(accumulate=False)
+    dA1, dB1 = run.host(run.dA), run.host(run.dB)
+    run.backward(accumulate=True, want_dx=False)
+    assert_close("dA x2", run.host(run.dA), 2 * dA1, 1e-5)
+    assert_close("dB x2", run.host(run.dB), 2 * dB1, 1e-5)
+    # x_save = NULL skips the copy but still produces Y and u_save
+    run2 = LayerRun(sess, "bf16", t, w.segments, w.n_rows, save_x=False)
+    run2.forward()
+    assert torch.equal(run2.Y, run.Y) and torch.equal(run2.u_save, run.u_save)
+    run.close()
+    run2.close()
+
+
+def test_strided_inputs_and_outputs(sess):
+    w = synth.random_workload(22, 128, 256, 16, 3, 200, max_seg=70)
+    t = synth.make_tensors(w)
+    run = LayerRun(sess, "bf16", t, w.segments, w.n_rows)
+    big_x = torch.zeros((w.n_rows, 128 + 64), dtype=torch.bfloat16, device=sess.device)
+    big_x[:, 64:] = run.X
+    big_y = torch.full((w.n_rows, 256 + 128), 7.0, dtype=torch.bfloat16, device=sess.device)
+    run.forward()
+    y_ref = run.Y.clone()
+    run.X, run.Y = big_x[:, 64:], big_y[:, 128:]
+    run.forward()
+    assert torch.equal(run.Y, y_ref)
+    assert (big_y[:, :128] == 7.0).all()
+    run.close()
+
+
+def test_run_to_run_determinism(sess):
+    w = synth.random_workload(23, 256, 320, 32, 5, 500, max_seg=120, p_finetune=0.5)
+    t = synth.make_tensors(w)
+    run = LayerRun(sess, "bf16", t, w.segments, w.n_rows)
+    outs = []
+    for _ in range(2):
+        run.forward()
+        run.backward()
+        outs.append([x.clone() for x in (run.Y, run.u_save, run.dA, run.dB, run.dX)])
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+    run.close()
+
+
+def test_argument_errors_launch_nothing(sess):
+    w = synth.random_workload(24, 128, 128, 16, 3, 64, max_seg=20, p_finetune=0.6)
+    t = synth.make_tensors(w)
+    run = LayerRun(sess, "bf16", t, w.segments, w.n_rows)
+    before = mb.mlora_launch_count(sess.ctx)
+    with pytest.raises(mb.MloraError) as e:                     # capacity too small
+        mb.mlora_mixed_forward(sess.ctx, run.layer, run.plan, run.X, run.Y, run.x_save, run.u_save, 0, run.ft_rows - 1)
+    assert e.value.status == mb.MLORA_ERR_SAVE_CAPACITY
+    with pytest.raises(mb.MloraError) as e:                     # u_save missing
+        mb.mlora_mixed_forward(sess.ctx, run.layer, run.plan, run.X, run.Y, run.x_save, None, 0, 1000)
+    assert e.value.status == mb.MLORA_ERR_INVALID_ARG
+    few = mb.make_layer(run.W, run.A_all[:2].contiguous(), run.B_all[:2].contiguous(), run.scale[:2].contiguous())
+    with pytest.raises(mb.MloraError) as e:                     # plan built for more adapters than the layer has
+        mb.mlora_mixed_forward(sess.ctx, few, run.plan, run.X, run.Y, run.x_save, run.u_save, 0, 1000)
+    assert e.value.status == mb.MLORA_ERR_ADAPTER_ID
+    odd = mb.make_layer(run.W, run.A_all, run.B_all, run.scale)
+    odd.rank = 24
+    with pytest.raises(mb.MloraError) as e:
+        mb.mlora_mixed_forward(sess.ctx, odd, run.plan, run.X, run.Y, run.x_save, run.u_save, 0, 1000)
+    assert e.value.status == mb.MLORA_ERR_UNSUPPORTED
+    assert mb.mlora_launch_count(sess.ctx) == before
+    run.close()
+
+
+# ---- full-size configurations --------------------------------------------------------------
+def test_cfg2_full_size(sess):
+    w = synth.cfg2_single_projection()
+    run_and_check(sess, w, synth.make_tensors(w), blocked=True)
+
+
+def _sampled_check(sess, w, n_sample=24, seed=0):
+    """Full-size run in the benchmark's launch configuration; the oracle recomputes sampled rows of Y
+    and dX one by one and sampled columns of dA / dB."""
+    t = synth.make_tensors(w)
+    run = LayerRun(sess, w.dtype, t, w.segments, w.n_rows)
+    try:
+        run.forward()
+        assert run.status() == mb.MLORA_OK
+        rng = np.random.default_rng(seed)
+        rows = np.unique(np.concatenate([[0, w.n_rows - 1], rng.integers(0, w.n_rows, n_sample)]))
+        y_ref = orc.forward_rows(t["X"], t["W"], t["A_all"], t["B_all"], t["scale"], w.segments, rows)
+        assert_close("Y[sample]", run.host(run.Y[torch.from_numpy(rows).to(sess.device)]), y_ref, 2e-2)
+        _ra, ft, n, slots = orc.route(w.segments, w.n_rows, w.n_adapters)
+        if not n:
+            return
+        # saved rows: bit-exact against X for every fine-tuning row
+        src = np.concatenate([np.arange(s, s + ln) for s, ln, _a, _o in ft])
+        assert torch.equal(run.x_save[:n], run.X[torch.from_numpy(src).to(sess.device)])
+        run.backward()
+        assert run.status() == mb.MLORA_OK
+        A, B, W, sc = (t[k].astype(np.float64) for k in ("A_all", "B_all", "W", "scale"))
+        Xs = t["X"].astype(np.float64)[src]
+        dY = t["dY"].astype(np.float64)
+        m_ad = np.concatenate([np.full(ln, a) for _s, ln, a, _o in ft])
+        # V and U for all fine-tuning rows (cheap), then sampled rows / columns of the big outputs
+        V = np.stack([sc[a] * (B[a] @ dY[m]) for m, a in enumerate(m_ad)])
+        U = np.stack([A[a] @ Xs[m] for m, a in enumerate(m_ad)])
+        assert_close("u_save", run.host(run.u_save[:n]), U, 1e-3)
+        ms = np.unique(np.concatenate([[0, n - 1], rng.integers(0, n, n_sample)]))
+        dx_ref = np.stack([W @ dY[m] + V[m] @ A[m_ad[m]] for m in ms])
+        assert_close("dX[sample]", run.host(run.dX[torch.from_numpy(ms).to(sess.device)]), dx_ref, 2e-2)
+        cols_o = rng.integers(0, w.d_out, 16)
+        cols_i = rng.integers(0, w.d_in, 16)
+        dA, dB = run.host(run.dA), run.host(run.dB)
+        for g, a in enumerate(slots):
+            sel = m_ad == a
+            assert_close("dB[cols]", dB[g][:, cols_o], sc[a] * (U[sel].T @ dY[sel][:, cols_o]), 2e-2)
+            assert_close("dA[cols]", dA[g][:, cols_i], V[sel].T @ Xs[sel][:, cols_i], 2e-2)
+    finally:
+        run.close()
+
+
+@pytest.mark.parametrize("proj", ["k", "gate", "down"])
+def test_cfg3_projection_sampled(sess, proj):
+    _sampled_check(sess, synth.cfg3_layer_set(projections=[proj])[0])
+
+
+def test_cfg5_decode_heavy_sampled(sess):
+    _sampled_check(sess, synth.cfg5_decode_heavy())
+
+
+@pytest.mark.parametrize("rank,n_adapters,f,sorted_rows", [(8, 256, 0.25, True), (128, 64, 0.5, True),
+                                                           (16, 64, 0.0, False)])
+def test_cfg4_points_sampled(sess, rank, n_adapters, f, sorted_rows):
+    _sampled_check(sess, synth.cfg4_sweep_point(rank, n_adapters, f, sorted_rows=sorted_rows), n_sample=12)
