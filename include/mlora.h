@@ -184,6 +184,37 @@ int32_t mlora_profile_collect(mlora_ctx* ctx, int32_t* kinds, float* ms, int32_t
  * (default), 1 = the plain CUDA-core kernel (a slow cross-check used by the tests). */
 mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path);
 
+/* ---- forward without any allocation -----------------------------------------------------*/
+
+/* (The paper has no counterpart for this entry point; it exists for integration reasons.)
+ *
+ * Some callers are not allowed to allocate device memory at all: an inference engine that hands
+ * its whole memory budget to its own pool at start-up and treats any later cudaMalloc as a bug,
+ * a worker that attaches to another process's buffers and owns no memory of its own, or code
+ * running where an allocation would stall the device (cudaMalloc synchronises).  The regular
+ * path needs a context and a plan, and both allocate.  This call needs neither: it computes
+ *        Y[t,:] = X[t,:] W + s_a (X[t,:] A_a^T) B_a,    a = row_adapter[t]  (-1: base only)
+ * for a small batch of inference rows with the plain CUDA-core kernels, keeping the rank-r
+ * intermediate x A_a^T in a fixed scratch array that is part of the library image
+ * (MLORA_NOALLOC_MAX_ROWS x 128 floats = 256 KiB, held by every GPU that loads the library until
+ * the process exits).  It calls no cudaMalloc, cudaFree or allocating library routine.
+ *   layer        as for mlora_mixed_forward (either dtype; no 64-multiple requirement here)
+ *   row_adapter  device [n_rows] int32, each in [-1, layer->n_adapters); NOT checked on the host
+ *   X, Y         device [n_rows, d_in] / [n_rows, d_out], row strides ldx / ldy
+ * Runs on the CURRENT device, asynchronously on the given stream.  Nothing is saved for
+ * fine-tuning; use the planned path for that.
+ * Limits and errors: n_rows > MLORA_NOALLOC_MAX_ROWS or rank > 128 -> MLORA_ERR_UNSUPPORTED
+ * (nothing launched); null pointers / bad sizes -> MLORA_ERR_INVALID_ARG; CUDA failures ->
+ * MLORA_ERR_CUDA.  n_rows = 0 is a no-op.
+ * First call on a device: it looks up the scratch array's device address (no allocation, but a
+ * runtime query), so make that first call before starting any stream capture.
+ * Sharing: every call on a device uses the same scratch and leaves its contents behind.  Each call
+ * rewrites all entries it later reads, so nothing needs clearing between calls; but two calls
+ * whose work overlaps on the GPU (different streams, no ordering) race on it - serialise them. */
+#define MLORA_NOALLOC_MAX_ROWS 512
+mlora_status_t mlora_forward_noalloc(const mlora_layer_t* layer, const int32_t* row_adapter, int32_t n_rows,
+                                     const void* X, int64_t ldx, void* Y, int64_t ldy, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

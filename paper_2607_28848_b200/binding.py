@@ -23,8 +23,9 @@ EXPORTS = (
     "mlora_create", "mlora_destroy", "mlora_plan_create", "mlora_plan_destroy", "mlora_plan_rows",
     "mlora_plan_ft_rows", "mlora_plan_ft_adapters", "mlora_plan_describe", "mlora_mixed_forward",
     "mlora_backward", "mlora_poll_status", "mlora_status_string", "mlora_launch_count", "mlora_set_gemm_path",
-    "mlora_profile_enable", "mlora_profile_collect",
+    "mlora_profile_enable", "mlora_profile_collect", "mlora_forward_noalloc",
 )
+MLORA_NOALLOC_MAX_ROWS = 512
 
 
 class mlora_segment_t(ctypes.Structure):
@@ -94,6 +95,8 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.mlora_profile_enable.restype = ctypes.c_int
     lib.mlora_profile_collect.argtypes = [vp, P(i32), P(ctypes.c_float), i32]
     lib.mlora_profile_collect.restype = i32
+    lib.mlora_forward_noalloc.argtypes = [P(mlora_layer_t), vp, i32, vp, i64, vp, i64, vp]
+    lib.mlora_forward_noalloc.restype = ctypes.c_int
     _lib = lib
     return lib
 
@@ -236,3 +239,18 @@ def mlora_profile_collect(ctx, cap: int = 1 << 16):
     n = load_library().mlora_profile_collect(ctx, kinds, ms, cap)
     n = min(n, cap)
     return np.asarray(kinds[:n], dtype=np.int32), np.asarray(ms[:n], dtype=np.float64)
+
+
+def mlora_forward_noalloc(layer: mlora_layer_t, row_adapter, X, Y, stream=None) -> None:
+    """Forward for a small batch of inference rows that allocates nothing: no context, no plan.
+
+    For callers that must not allocate device memory (an engine that owns the whole memory pool,
+    a worker attached to someone else's buffers).  ``row_adapter`` is an int32 CUDA tensor with one
+    adapter id (or -1) per row; at most MLORA_NOALLOC_MAX_ROWS rows.  The rank-r intermediate goes
+    through a scratch array built into the library and shared by every call on the device, so
+    calls must not overlap on the GPU.  Make the first call on a device outside stream capture.
+    """
+    n_rows = int(row_adapter.numel())
+    st = load_library().mlora_forward_noalloc(ctypes.byref(layer), _ptr(row_adapter), n_rows, _ptr(X),
+                                              X.stride(0), _ptr(Y), Y.stride(0), _stream_ptr(stream))
+    _check(st, "mlora_forward_noalloc")

@@ -6,6 +6,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -277,8 +278,69 @@ mlora_status_t backward_simt(mlora_ctx* ctx, const mlora_layer_t* L, const mlora
 
 }  // namespace
 
+// ---- allocation-free forward ------------------------------------------------------------------
+// Scratch for mlora_forward_noalloc: the rank-r intermediate of up to MLORA_NOALLOC_MAX_ROWS rows.
+// It lives in the library image, so every device that loads the library carries these 256 KiB.
+// In host code this name is only a handle; the device address is looked up once per device.
+static __device__ __align__(256) float g_noalloc_scratch[MLORA_NOALLOC_MAX_ROWS * mlora::kMaxRank];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float* g_noalloc_addr[kMaxDevices] = {};
+std::mutex g_noalloc_mutex;
+
+// Device address of the scratch on the current device (looked up on first use, then cached).
+mlora_status_t noalloc_scratch(float** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MLORA_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (!g_noalloc_addr[dev]) {
+    float* p = nullptr;
+    if (cudaGetSymbolAddress((void**)&p, g_noalloc_scratch) != cudaSuccess || !p) {
+      cudaGetLastError();
+      return MLORA_ERR_CUDA;
+    }
+    g_noalloc_addr[dev] = p;
+  }
+  *out = g_noalloc_addr[dev];
+  return MLORA_OK;
+}
+
+template <typename T>
+mlora_status_t forward_noalloc_t(const mlora_layer_t* L, const int32_t* row_adapter, int n_rows, const void* X,
+                                 int64_t ldx, void* Y, int64_t ldy, float* scratch, cudaStream_t st) {
+  const int64_t warps = (int64_t)n_rows * L->rank;
+  const int blocks = (int)((warps * 32 + 255) / 256);
+  // rank-r intermediate of every row (zeros for rows without an adapter) -> scratch
+  simt::shrink_kernel<T><<<blocks, 256, 0, st>>>((const T*)X, ldx, L->d_in, L->rank, (const T*)L->A_all, nullptr,
+                                                 row_adapter, nullptr, scratch, (T*)nullptr, nullptr, 0, n_rows);
+  if (cudaGetLastError() != cudaSuccess) return MLORA_ERR_CUDA;
+  dim3 grid((L->d_out + 31) / 32, (n_rows + 31) / 32), block(32, 32);
+  simt::gemm_lora_kernel<T, false><<<grid, block, 0, st>>>((const T*)X, ldx, (const T*)L->W, L->ldw,
+                                                           (const T*)L->B_all, scratch, L->scale, row_adapter, (T*)Y,
+                                                           ldy, n_rows, L->d_out, L->d_in, L->rank);
+  return cudaGetLastError() == cudaSuccess ? MLORA_OK : MLORA_ERR_CUDA;
+}
+}  // namespace
+
 // =============================================================================================
 extern "C" {
+
+mlora_status_t mlora_forward_noalloc(const mlora_layer_t* L, const int32_t* row_adapter, int32_t n_rows, const void* X,
+                                     int64_t ldx, void* Y, int64_t ldy, void* cuda_stream) {
+  if (!L || !L->W || !L->A_all || !L->B_all || !L->scale || n_rows < 0) return MLORA_ERR_INVALID_ARG;
+  if (L->d_in <= 0 || L->d_out <= 0 || L->rank <= 0 || L->n_adapters <= 0 || L->ldw < L->d_out) return MLORA_ERR_INVALID_ARG;
+  if (L->dtype != MLORA_F32 && L->dtype != MLORA_BF16) return MLORA_ERR_INVALID_ARG;
+  if (n_rows > MLORA_NOALLOC_MAX_ROWS || L->rank > kMaxRank) return MLORA_ERR_UNSUPPORTED;
+  if (n_rows == 0) return MLORA_OK;
+  if (!row_adapter || !X || !Y || ldx < L->d_in || ldy < L->d_out) return MLORA_ERR_INVALID_ARG;
+  float* scratch = nullptr;
+  mlora_status_t s = noalloc_scratch(&scratch);
+  if (s != MLORA_OK) return s;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (L->dtype == MLORA_F32) return forward_noalloc_t<float>(L, row_adapter, n_rows, X, ldx, Y, ldy, scratch, st);
+  return forward_noalloc_t<__nv_bfloat16>(L, row_adapter, n_rows, X, ldx, Y, ldy, scratch, st);
+}
 
 const char* mlora_status_string(mlora_status_t s) {
   switch (s) {

@@ -1,0 +1,56 @@
+"""The allocation-free forward (mlora_forward_noalloc) against the regular planned forward.
+
+Some users of the library may not allocate device memory - an engine that gave its whole budget to
+its own pool, a worker living on buffers mapped from another process - so they cannot create the
+context and plan the regular path needs.  The allocation-free entry point keeps its rank-r
+intermediate in a scratch array inside the library instead.  Here it is called twice in a row
+through the C ABI, the second time on a smaller batch with different adapters so that whatever
+the first call left in the shared scratch would show, and compared with mlora_mixed_forward.
+This file sorts last so that a run stopping at the first failure has already run everything else.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_28848_b200 import binding as mb
+from paper_2607_28848_b200 import synth
+from paper_2607_28848_b200.runner import LayerRun, Session
+
+pytestmark = pytest.mark.gpu
+
+
+def _reference(sess, w, t):
+    run = LayerRun(sess, w.dtype, t, w.segments, w.n_rows)
+    run.forward()
+    assert run.status() == mb.MLORA_OK
+    return run
+
+
+@pytest.mark.parametrize("dtype,tol", [("bf16", 2e-2), ("f32", 1e-4)])
+def test_noalloc_matches_planned_forward_twice(dtype, tol):
+    with Session(0) as sess:
+        for seed, n_rows in ((31, 300), (32, 77)):            # two calls in a row, the second smaller
+            w = synth.random_workload(seed, 128, 192, 16, 5, n_rows, dtype=dtype, max_seg=40, p_finetune=0.0)
+            t = synth.make_tensors(w)
+            ref = _reference(sess, w, t)
+            _so, row_adapter = mb.mlora_plan_describe(ref.plan, len(w.segments))
+            ra = torch.from_numpy(row_adapter).to(sess.device)
+            Y = torch.full_like(ref.Y, float("nan"))
+            mb.mlora_forward_noalloc(ref.layer, ra, ref.X, Y)
+            torch.cuda.synchronize()
+            got, want = Y.float().cpu().numpy().astype(np.float64), ref.host(ref.Y)
+            assert np.isfinite(got).all()
+            assert (np.abs(got - want) <= tol * (1 + np.abs(want))).all()
+            ref.close()
+
+
+def test_noalloc_limits_are_refused():
+    with Session(0) as sess:
+        w = synth.random_workload(33, 64, 64, 8, 2, 16, dtype="f32", max_seg=8, p_finetune=0.0)
+        ref = _reference(sess, w, synth.make_tensors(w))
+        too_many = torch.zeros(mb.MLORA_NOALLOC_MAX_ROWS + 1, dtype=torch.int32, device=sess.device)
+        with pytest.raises(mb.MloraError) as e:
+            mb.mlora_forward_noalloc(ref.layer, too_many, ref.X, ref.Y)
+        assert e.value.status == mb.MLORA_ERR_UNSUPPORTED
+        mb.mlora_forward_noalloc(ref.layer, too_many[:0], ref.X, ref.Y)      # empty batch: no-op
+        ref.close()
