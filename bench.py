@@ -226,13 +226,18 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--e2e-steps", type=int, default=10, help="0 skips the end-to-end leg")
+    ap.add_argument("--projections", default="", help="comma list: run only these projections of the workload")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     workloads, label = get_workloads(args.workload, args.seed + rank)
+    if args.projections:
+        keep = set(args.projections.split(","))
+        workloads = [w for w in workloads if w.name.split("_", 1)[1] in keep]
+        label += f" [only {sorted(keep)}]"
     if args.impl == "reference":
         run_reference(args, workloads, label)
         return
@@ -348,7 +353,7 @@ def main():
 
     # ---- end to end through the public API with host buffers ----
     e2e = None
-    if rank == 0 or world > 1:
+    if args.e2e_steps > 0 and (rank == 0 or world > 1):
         hx = [r.X.cpu().pin_memory() for r in runs]
         hdy = [r.dY.cpu().pin_memory() for r in runs]
         hy = [torch.empty_like(r.Y, device="cpu").pin_memory() for r in runs]
@@ -408,7 +413,7 @@ def main():
         "roofline": roofline, "kernels": kernels,
     }
     if not args.no_cpu_baseline and world == 1:
-        names = {"cfg3": ["k", "q"], "cfg2": ["proj4096"], "cfg5": ["mixed"]}[args.workload]
+        names = {"cfg3": ["q", "k", "v", "o", "gate"], "cfg2": ["proj4096"], "cfg5": ["mixed"]}[args.workload]
         line["cpu_baseline"] = cpu_baseline(workloads, names)
     print(json.dumps(line), flush=True)
     if world > 1:

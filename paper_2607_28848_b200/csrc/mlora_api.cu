@@ -28,6 +28,10 @@ struct mlora_ctx {
   int32_t* status_dev = nullptr;     // device status word
   float* ws_p = nullptr;             // [ws_rows, kMaxRank] rank-r intermediate of the running call
   int64_t ws_rows = 0;
+  float* ws_partial = nullptr;       // split-K partials of the shrink kernel: [ws_partial_items, 32, kMaxRank]
+  int64_t ws_partial_items = 0;
+  int32_t* ws_counters = nullptr;    // [ws_counter_items] arrival counters, zero between launches
+  int64_t ws_counter_items = 0;
   int64_t launches = 0;
   int32_t gemm_path = 0;
   EncodeTiledFn encode = nullptr;
@@ -36,6 +40,8 @@ struct mlora_ctx {
   std::vector<int32_t> ev_kind;
   int32_t ev_used = 0;
 };
+
+constexpr int kMaxKSplit = 16;
 
 enum { KIND_SHRINK = 0, KIND_GEMM_FWD = 1, KIND_GEMM_BWD = 2, KIND_GRAD = 3, KIND_SIMT = 4 };
 
@@ -46,10 +52,10 @@ struct DevRowSpace {
   const int32_t* row_grp = nullptr;
   const int32_t* tile_grp_off = nullptr;
   const int32_t* grp_adapter = nullptr;
-  const int32_t* item_row0 = nullptr;
+  const int32_t* item_rows = nullptr;
+  const int32_t* item_start = nullptr;
   const int32_t* item_nrows = nullptr;
   const int32_t* item_adapter = nullptr;
-  const int32_t* item_save0 = nullptr;
 };
 
 struct mlora_plan {
@@ -123,19 +129,32 @@ struct LaunchScope {
 };
 
 // ---- bf16 launches ------------------------------------------------------------------------
-template <int RB>
-void launch_shrink_rb(const ShrinkArgs& a, int n_items, cudaStream_t st) {
-  shrink_kernel<RB><<<n_items, SHRINK_THREADS, 0, st>>>(a);
+template <int RB, int MT, int WARPS, int MIN_CTAS>
+void launch_shrink_rb(const ShrinkArgs& a, int n_items, int ksplit, cudaStream_t st) {
+  shrink_kernel<RB, MT, WARPS, MIN_CTAS><<<dim3(n_items, ksplit, kItemRows / (16 * MT)), WARPS * 32, 0, st>>>(a);
 }
-mlora_status_t launch_shrink(mlora_ctx* ctx, int R, const ShrinkArgs& a, int n_items, cudaStream_t st) {
+// Few items with a long contraction leave most SMs idle: split K over several CTAs per item so
+// that about three CTAs per SM are in flight, keeping at least 16 K-blocks (1024 elements) each.
+int shrink_ksplit(const mlora_ctx* ctx, int n_items, int D) {
+  const int want = (3 * ctx->sm_count + n_items - 1) / n_items;
+  const int cap = D / 64 / 16;
+  int k = want < cap ? want : cap;
+  k = k < kMaxKSplit ? k : kMaxKSplit;
+  return k < 1 ? 1 : k;
+}
+mlora_status_t launch_shrink(mlora_ctx* ctx, int R, ShrinkArgs a, int n_items, cudaStream_t st) {
   if (n_items <= 0) return MLORA_OK;
+  const int ksplit = shrink_ksplit(ctx, n_items, a.D);
+  a.partial = ctx->ws_partial;
+  a.counters = ctx->ws_counters;
+  if ((int64_t)n_items * ksplit > ctx->ws_partial_items || n_items > ctx->ws_counter_items) return MLORA_ERR_INVALID_ARG;
   LaunchScope scope(ctx, st, KIND_SHRINK);
   switch (R) {
-    case 8: launch_shrink_rb<1>(a, n_items, st); break;
-    case 16: launch_shrink_rb<2>(a, n_items, st); break;
-    case 32: launch_shrink_rb<4>(a, n_items, st); break;
-    case 64: launch_shrink_rb<8>(a, n_items, st); break;
-    case 128: launch_shrink_rb<16>(a, n_items, st); break;
+    case 8: launch_shrink_rb<1, 2, 8, 2>(a, n_items, ksplit, st); break;
+    case 16: launch_shrink_rb<2, 2, 8, 2>(a, n_items, ksplit, st); break;
+    case 32: launch_shrink_rb<4, 2, 8, 2>(a, n_items, ksplit, st); break;
+    case 64: launch_shrink_rb<8, 2, 4, 2>(a, n_items, ksplit, st); break;
+    case 128: launch_shrink_rb<16, 1, 4, 2>(a, n_items, ksplit, st); break;
     default: return MLORA_ERR_UNSUPPORTED;
   }
   return scope.done();
@@ -143,11 +162,18 @@ mlora_status_t launch_shrink(mlora_ctx* ctx, int R, const ShrinkArgs& a, int n_i
 
 mlora_status_t launch_grad(mlora_ctx* ctx, const GradArgs& a, int n_slots, cudaStream_t st) {
   if (n_slots <= 0) return MLORA_OK;
+  constexpr int smem1 = (GRAD_THREADS / 32) * 16 * 65 * 4, smem2 = 2 * smem1;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(grad_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2) != cudaSuccess)
+      return MLORA_ERR_CUDA;
+    attr_set = true;
+  }
   LaunchScope scope(ctx, st, KIND_GRAD);
   if (a.R <= 16) {
-    grad_kernel<1><<<dim3(a.D / 64, n_slots, 1), GRAD_THREADS, 0, st>>>(a);
+    grad_kernel<1><<<dim3(a.D / 64, n_slots, 1), GRAD_THREADS, smem1, st>>>(a);
   } else {
-    grad_kernel<2><<<dim3(a.D / 64, n_slots, (a.R + 31) / 32), GRAD_THREADS, 0, st>>>(a);
+    grad_kernel<2><<<dim3(a.D / 64, n_slots, (a.R + 31) / 32), GRAD_THREADS, smem2, st>>>(a);
   }
   return scope.done();
 }
@@ -426,6 +452,8 @@ void mlora_destroy(mlora_ctx* c) {
   for (cudaEvent_t e : c->ev_stop) cudaEventDestroy(e);
   cudaFree(c->status_dev);
   cudaFree(c->ws_p);
+  cudaFree(c->ws_partial);
+  cudaFree(c->ws_counters);
   delete c;
 }
 
@@ -446,8 +474,8 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
     const RowSpace* rs[2] = {&h.fwd, &h.bwd};
     for (int i = 0; i < 2; ++i) {
       o[n++] = b.add(rs[i]->row_adapter); o[n++] = b.add(rs[i]->row_save); o[n++] = b.add(rs[i]->row_grp);
-      o[n++] = b.add(rs[i]->tile_grp_off); o[n++] = b.add(rs[i]->grp_adapter); o[n++] = b.add(rs[i]->item_row0);
-      o[n++] = b.add(rs[i]->item_nrows); o[n++] = b.add(rs[i]->item_adapter); o[n++] = b.add(rs[i]->item_save0);
+      o[n++] = b.add(rs[i]->tile_grp_off); o[n++] = b.add(rs[i]->grp_adapter); o[n++] = b.add(rs[i]->item_rows);
+      o[n++] = b.add(rs[i]->item_start); o[n++] = b.add(rs[i]->item_nrows); o[n++] = b.add(rs[i]->item_adapter);
     }
     o[n++] = b.add(h.slot_chunk_off); o[n++] = b.add(h.chunk_row0); o[n++] = b.add(h.chunk_nrows);
     o[n++] = b.add(h.ft_adapters);
@@ -459,11 +487,10 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
     n = 0;
     for (int i = 0; i < 2; ++i) {
       ds[i]->row_adapter = p->blob + o[n++]; ds[i]->row_save = p->blob + o[n++]; ds[i]->row_grp = p->blob + o[n++];
-      ds[i]->tile_grp_off = p->blob + o[n++]; ds[i]->grp_adapter = p->blob + o[n++]; ds[i]->item_row0 = p->blob + o[n++];
-      ds[i]->item_nrows = p->blob + o[n++]; ds[i]->item_adapter = p->blob + o[n++]; ds[i]->item_save0 = p->blob + o[n++];
+      ds[i]->tile_grp_off = p->blob + o[n++]; ds[i]->grp_adapter = p->blob + o[n++]; ds[i]->item_rows = p->blob + o[n++];
+      ds[i]->item_start = p->blob + o[n++]; ds[i]->item_nrows = p->blob + o[n++]; ds[i]->item_adapter = p->blob + o[n++];
     }
     p->bwd.row_save = nullptr;       // the compact space has no save offsets
-    p->bwd.item_save0 = nullptr;
     p->slot_chunk_off = p->blob + o[n++]; p->chunk_row0 = p->blob + o[n++]; p->chunk_nrows = p->blob + o[n++];
     p->slot_adapter = p->blob + o[n++];
     if (n_rows > ctx->ws_rows) {     // grow the rank-r workspace (the only other device allocation)
@@ -474,6 +501,19 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
         cudaFree(p->blob); delete p; return MLORA_ERR_CUDA;
       }
       ctx->ws_rows = n_rows;
+    }
+    const int64_t items = h.fwd.n_items() > h.bwd.n_items() ? h.fwd.n_items() : h.bwd.n_items();
+    const int64_t part_items = items + 4 * ctx->sm_count;      // items * ksplit never exceeds this
+    if (part_items > ctx->ws_partial_items || items > ctx->ws_counter_items) {
+      if (cudaDeviceSynchronize() != cudaSuccess) { cudaFree(p->blob); delete p; return MLORA_ERR_CUDA; }
+      cudaFree(ctx->ws_partial); cudaFree(ctx->ws_counters);
+      ctx->ws_partial = nullptr; ctx->ws_counters = nullptr; ctx->ws_partial_items = ctx->ws_counter_items = 0;
+      if (cudaMalloc(&ctx->ws_partial, (size_t)part_items * kItemRows * kMaxRank * sizeof(float)) != cudaSuccess ||
+          cudaMalloc(&ctx->ws_counters, (size_t)(2 * items + 1) * sizeof(int32_t)) != cudaSuccess ||
+          cudaMemset(ctx->ws_counters, 0, (size_t)(2 * items + 1) * sizeof(int32_t)) != cudaSuccess) {
+        cudaFree(p->blob); delete p; return MLORA_ERR_CUDA;
+      }
+      ctx->ws_partial_items = part_items; ctx->ws_counter_items = items;
     }
   }
   *out = p;
@@ -527,8 +567,8 @@ mlora_status_t mlora_mixed_forward(mlora_ctx* ctx, const mlora_layer_t* L, const
   ShrinkArgs sa;
   sa.In = (const __nv_bfloat16*)X; sa.ld_in = ldx; sa.D = L->d_in;
   sa.P_all = (const __nv_bfloat16*)L->A_all; sa.scale = nullptr; sa.Out = ctx->ws_p;
-  sa.item_row0 = p->fwd.item_row0; sa.item_nrows = p->fwd.item_nrows; sa.item_adapter = p->fwd.item_adapter;
-  sa.item_save0 = p->fwd.item_save0;
+  sa.item_rows = p->fwd.item_rows; sa.item_start = p->fwd.item_start; sa.item_nrows = p->fwd.item_nrows;
+  sa.item_adapter = p->fwd.item_adapter; sa.row_save = p->fwd.row_save;
   sa.x_save = (__nv_bfloat16*)x_save; sa.u_save = u_save; sa.save_base = save_row_base;
   if ((s = launch_shrink(ctx, L->rank, sa, h.fwd.n_items(), st)) != MLORA_OK) return s;
   return gemm_bf16<false>(ctx, L, h.fwd, p->fwd, X, ldx, Y, ldy, L->B_all, ctx->ws_p, L->scale, h.n_rows, L->d_out,
@@ -557,8 +597,8 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   ShrinkArgs sa;                     // V = s dY B^T
   sa.In = (const __nv_bfloat16*)dY; sa.ld_in = lddy; sa.D = L->d_out;
   sa.P_all = (const __nv_bfloat16*)L->B_all; sa.scale = L->scale; sa.Out = ctx->ws_p;
-  sa.item_row0 = p->bwd.item_row0; sa.item_nrows = p->bwd.item_nrows; sa.item_adapter = p->bwd.item_adapter;
-  sa.item_save0 = nullptr; sa.x_save = nullptr; sa.u_save = nullptr; sa.save_base = 0;
+  sa.item_rows = p->bwd.item_rows; sa.item_start = p->bwd.item_start; sa.item_nrows = p->bwd.item_nrows;
+  sa.item_adapter = p->bwd.item_adapter; sa.row_save = nullptr; sa.x_save = nullptr; sa.u_save = nullptr; sa.save_base = 0;
   if ((s = launch_shrink(ctx, L->rank, sa, h.bwd.n_items(), st)) != MLORA_OK) return s;
 
   GradArgs ga;                       // dB = (s U)^T dY

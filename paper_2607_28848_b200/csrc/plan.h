@@ -11,7 +11,8 @@
 namespace mlora {
 
 constexpr int kTileRows = 128;     // rows per tensor-core tile (UMMA M)
-constexpr int kItemRows = 16;      // rows per skinny-kernel work item (mma.sync M)
+constexpr int kItemRows = 32;      // most rows in one shrink work item (two mma.sync row blocks)
+constexpr int kChunkRows = 16;     // rows per gradient chunk (one mma.sync contraction step)
 constexpr int kMaxRank = 128;
 
 // Tables over one row space: the batch rows (forward) or the compact fine-tuning rows (backward).
@@ -24,11 +25,14 @@ struct RowSpace {
   std::vector<int32_t> row_grp;        // [n_rows]
   std::vector<int32_t> tile_grp_off;   // [n_tiles + 1]
   std::vector<int32_t> grp_adapter;    // [tile_grp_off.back()]
-  // Skinny-kernel items: runs of <= kItemRows consecutive rows bound to one adapter whose save
-  // offsets (if any) are consecutive too.
-  std::vector<int32_t> item_row0, item_nrows, item_adapter, item_save0;
+  // Shrink items: the rows that have an adapter, gathered BY ADAPTER (ascending adapter id, rows
+  // ascending inside an adapter) and cut into items of <= kItemRows rows.  Rows of an item need
+  // not be adjacent in the batch: decode rows that share an adapter are processed together, so an
+  // adapter's matrix is fetched once per item instead of once per row.
+  std::vector<int32_t> item_rows;      // [rows with an adapter] row ids, grouped by adapter
+  std::vector<int32_t> item_start, item_nrows, item_adapter;
   int32_t n_tiles() const { return (n_rows + kTileRows - 1) / kTileRows; }
-  int32_t n_items() const { return (int32_t)item_row0.size(); }
+  int32_t n_items() const { return (int32_t)item_start.size(); }
 };
 
 struct HostPlan {
@@ -38,7 +42,7 @@ struct HostPlan {
   std::vector<int32_t> ft_adapters;    // slot -> adapter id
   RowSpace fwd;                        // batch rows
   RowSpace bwd;                        // compact fine-tuning rows, in save order
-  // Gradient work: per slot, chunks of <= kItemRows compact rows.
+  // Gradient work: per slot, chunks of <= kChunkRows compact rows.
   std::vector<int32_t> slot_chunk_off; // [n_slots + 1]
   std::vector<int32_t> chunk_row0, chunk_nrows;
 };
@@ -62,22 +66,23 @@ inline void build_tiles_and_items(RowSpace& rs) {
     }
     rs.tile_grp_off.push_back((int32_t)rs.grp_adapter.size());
   }
-  rs.item_row0.clear(); rs.item_nrows.clear(); rs.item_adapter.clear(); rs.item_save0.clear();
-  const bool has_save = !rs.row_save.empty();
-  int32_t t = 0;
-  while (t < n) {
-    const int32_t a = rs.row_adapter[t];
-    if (a < 0) { ++t; continue; }
-    const int32_t s0 = has_save ? rs.row_save[t] : -1;
-    int32_t len = 1;
-    while (t + len < n && len < kItemRows && rs.row_adapter[t + len] == a) {
-      const int32_t s = has_save ? rs.row_save[t + len] : -1;
-      if (s0 >= 0 ? (s != s0 + len) : (s >= 0)) break;
-      ++len;
+  rs.item_rows.clear(); rs.item_start.clear(); rs.item_nrows.clear(); rs.item_adapter.clear();
+  int32_t max_adapter = -1;
+  for (int32_t t = 0; t < n; ++t) max_adapter = rs.row_adapter[t] > max_adapter ? rs.row_adapter[t] : max_adapter;
+  std::vector<int32_t> count(max_adapter + 2, 0);
+  for (int32_t t = 0; t < n; ++t) if (rs.row_adapter[t] >= 0) count[rs.row_adapter[t] + 1]++;
+  for (int32_t a = 0; a <= max_adapter; ++a) count[a + 1] += count[a];
+  rs.item_rows.assign(max_adapter >= 0 ? count[max_adapter + 1] : 0, 0);
+  {
+    std::vector<int32_t> fill(count.begin(), count.end());
+    for (int32_t t = 0; t < n; ++t) if (rs.row_adapter[t] >= 0) rs.item_rows[fill[rs.row_adapter[t]]++] = t;
+  }
+  for (int32_t a = 0; a <= max_adapter; ++a) {
+    for (int32_t i = count[a]; i < count[a + 1]; i += kItemRows) {
+      rs.item_start.push_back(i);
+      rs.item_nrows.push_back(count[a + 1] - i < kItemRows ? count[a + 1] - i : kItemRows);
+      rs.item_adapter.push_back(a);
     }
-    rs.item_row0.push_back(t); rs.item_nrows.push_back(len);
-    rs.item_adapter.push_back(a); rs.item_save0.push_back(s0);
-    t += len;
   }
 }
 
@@ -134,9 +139,9 @@ inline mlora_status_t build_plan(const mlora_segment_t* segs, int32_t n_segs, in
   for (int32_t a : p.ft_adapters) {
     for (int32_t k = 0; k < n_segs; ++k) {
       if (!segs[k].is_finetune || segs[k].adapter_id != a) continue;
-      for (int32_t i = 0; i < segs[k].row_len; i += kItemRows) {
+      for (int32_t i = 0; i < segs[k].row_len; i += kChunkRows) {
         p.chunk_row0.push_back(p.seg_save_off[k] + i);
-        p.chunk_nrows.push_back(segs[k].row_len - i < kItemRows ? segs[k].row_len - i : kItemRows);
+        p.chunk_nrows.push_back(segs[k].row_len - i < kChunkRows ? segs[k].row_len - i : kChunkRows);
       }
     }
     p.slot_chunk_off.push_back((int32_t)p.chunk_row0.size());
