@@ -281,7 +281,6 @@ def main():
     launches_per_step_probe = mb.mlora_launch_count(sess.ctx)
     step()
     launches_per_step = mb.mlora_launch_count(sess.ctx) - launches_per_step_probe
-    mb.mlora_profile_enable(sess.ctx, launches_per_step * args.steps)
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -302,6 +301,15 @@ def main():
         tt = torch.tensor([ms_total], device=sess.device)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         ms_total = float(tt.item())
+    # Per-kernel durations: the same steps once more, now with the library recording a CUDA event
+    # pair around every launch (which also switches off the overlap of a kernel's set-up with its
+    # predecessor's tail, so each pair times one whole kernel).  Kept out of the region above so
+    # that the headline number carries no event overhead.
+    prof_steps = max(1, min(args.steps, 20))
+    mb.mlora_profile_enable(sess.ctx, launches_per_step * prof_steps)
+    for _ in range(prof_steps):
+        step()
+    barrier()
     clocks = sampler.finish() if sampler else None
     kinds, kms = mb.mlora_profile_collect(sess.ctx)
     mb.mlora_profile_enable(sess.ctx, 0)
@@ -316,7 +324,7 @@ def main():
     for k, name in enumerate(mb.PROFILE_KINDS):
         sel = kms[kinds == k]
         if len(sel):
-            per_kind[name] = {"launches_per_step": len(sel) / args.steps, "ms_per_step": float(sel.sum() / args.steps)}
+            per_kind[name] = {"launches_per_step": len(sel) / prof_steps, "ms_per_step": float(sel.sum() / prof_steps)}
     gemm_fwd_flops = sum(flops(w)["gemm_fwd"] for w in workloads)
     gemm_bwd_flops = sum(flops(w)["gemm_bwd"] for w in workloads)
     ab = [algorithmic_bytes(w) for w in workloads]

@@ -47,6 +47,8 @@ constexpr uint32_t GEMM_TMEM_COLS = 512;
 struct GemmArgs {
   int32_t M, N, K;
   int32_t n_mtiles, n_ntiles;
+  int32_t n_full;                // work units [0, n_full) are whole 128 x 256 tiles; the tiles after
+  int32_t n_units;               // them (the last, partly filled wave) are cut into two 128 x 128 halves
   int32_t lora_enabled;
   const int32_t* row_grp;        // [M] group of the row inside its 128-row tile, -1: none
   const int32_t* row_adapter;    // [M]
@@ -65,6 +67,19 @@ __device__ __forceinline__ bool gemm_wait(uint32_t bar, uint32_t parity, volatil
   *abort_flag = 1;
   atomicExch(status, (int32_t)MLORA_ERR_DEVICE_TIMEOUT);
   return false;
+}
+
+// Work unit -> (row tile, first output column, width in columns).
+__device__ __forceinline__ void gemm_unit(const GemmArgs& args, int unit, int& mt, int& n0, int& nw) {
+  int tile = unit, half = 0;
+  nw = GEMM_BN;
+  if (unit >= args.n_full) {
+    tile = args.n_full + ((unit - args.n_full) >> 1);
+    half = (unit - args.n_full) & 1;
+    nw = GEMM_BN / 2;
+  }
+  mt = tile % args.n_mtiles;
+  n0 = (tile / args.n_mtiles) * GEMM_BN + half * (GEMM_BN / 2);
 }
 
 template <int R, bool W_KMAJOR>
@@ -122,9 +137,13 @@ gemm_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_ptr_smem;
+  // set-up (barriers, tensor memory, descriptor prefetch) may overlap the predecessor's tail;
+  // its outputs (In, P) are first touched below
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();
 
   const int KB = (args.K + GEMM_BK - 1) / GEMM_BK;
-  const int n_tiles = args.n_mtiles * args.n_ntiles;
+  const int n_units = args.n_units;
 
   auto tile_groups = [&](int mt) -> int {
     return args.lora_enabled ? (args.tile_grp_off[mt + 1] - args.tile_grp_off[mt]) : 0;
@@ -135,21 +154,24 @@ gemm_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        const int mt = tile % args.n_mtiles, nt = tile / args.n_mtiles;
-        const int m0 = mt * GEMM_BM, n0 = nt * GEMM_BN;
+      for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+        int mt, n0, nw;
+        gemm_unit(args, unit, mt, n0, nw);
+        const int m0 = mt * GEMM_BM;
+        const int nbox = nw / 64;                      // 64-column boxes of the B operand
         for (int kb = 0; kb < KB; ++kb, ++it) {
           const int s = it % GEMM_STAGES;
           if (!(ok = gemm_wait(bar_empty(s), ((it / GEMM_STAGES) & 1) ^ 1, abort_flag, args.status))) break;
           const uint32_t a = sA0 + s * GEMM_STAGE_BYTES, b = a + GEMM_A_BYTES;
-          ptx::mbar_arrive_expect_tx(bar_full(s), GEMM_STAGE_BYTES);
+          ptx::mbar_arrive_expect_tx(bar_full(s), GEMM_A_BYTES + (uint32_t)nw * GEMM_BK * 2u);
           ptx::tma_load_2d(a, &tmIn, kb * GEMM_BK, m0, bar_full(s));
-          if (W_KMAJOR) {
+          // the B operand arrives in halves of 128 output columns (one TMA each)
+          if (W_KMAJOR) {                              // [N, K]: box of 128 rows x 64 k
             ptx::tma_load_2d(b, &tmW, kb * GEMM_BK, n0, bar_full(s));
-          } else {
-#pragma unroll
-            for (int nb = 0; nb < 4; ++nb)
-              ptx::tma_load_2d(b + nb * 8192, &tmW, n0 + nb * 64, kb * GEMM_BK, bar_full(s));
+            if (nw == GEMM_BN) ptx::tma_load_2d(b + 16384, &tmW, kb * GEMM_BK, n0 + 128, bar_full(s));
+          } else {                                     // [K, N] seen as (64 n, K, N / 64): box 64 x 64 k x 2
+            ptx::tma_load_3d(b, &tmW, 0, kb * GEMM_BK, n0 >> 6, bar_full(s));
+            if (nw == GEMM_BN) ptx::tma_load_3d(b + 16384, &tmW, 0, kb * GEMM_BK, (n0 >> 6) + 2, bar_full(s));
           }
         }
         if (!ok) break;
@@ -169,20 +191,19 @@ gemm_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
             int ng = G - g0 < GPC ? G - g0 : GPC;
             // a half-filled 16-deep MMA step (rank 8, odd group count) is padded with a second
             // copy of the last group: its A columns are zero, so it only has to be finite
-            const int nbox = (R == 8 && (ng & 1)) ? ng + 1 : ng;
-            ptx::mbar_arrive_expect_tx(bar_full(s), (uint32_t)nbox * R * 128u * 4u);
-            for (int i = 0; i < nbox; ++i) {
+            const int ngl = (R == 8 && (ng & 1)) ? ng + 1 : ng;
+            ptx::mbar_arrive_expect_tx(bar_full(s), (uint32_t)ngl * R * 128u * (uint32_t)nbox);
+            for (int i = 0; i < ngl; ++i) {
               const int adapter = ga[g0 + (i < ng ? i : ng - 1)];
-#pragma unroll
-              for (int nb = 0; nb < 4; ++nb)
-                ptx::tma_load_2d(b + nb * 8192 + i * R * 128, &tmL, n0 + nb * 64, adapter * R, bar_full(s));
+              // one box per 64-column block: block nb of the stage starts at nb * 8 KiB
+              for (int nb = 0; nb < nbox; ++nb)
+                ptx::tma_load_3d(b + nb * 8192 + i * R * 128, &tmL, 0, adapter * R, (n0 >> 6) + nb, bar_full(s));
             }
           } else {
             const int adapter = ga[lc >> 1];
-            ptx::mbar_arrive_expect_tx(bar_full(s), 64u * 128u * 4u);
-#pragma unroll
-            for (int nb = 0; nb < 4; ++nb)
-              ptx::tma_load_2d(b + nb * 8192, &tmL, n0 + nb * 64, adapter * R + (lc & 1) * 64, bar_full(s));
+            ptx::mbar_arrive_expect_tx(bar_full(s), 64u * 128u * (uint32_t)nbox);
+            for (int nb = 0; nb < nbox; ++nb)
+              ptx::tma_load_3d(b + nb * 8192, &tmL, 0, adapter * R + (lc & 1) * 64, (n0 >> 6) + nb, bar_full(s));
           }
         }
       }
@@ -191,12 +212,17 @@ gemm_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
   } else if (warp == 1) {
     // ============================ MMA issuer ============================
     if (lane == 0) {
-      constexpr uint32_t idesc_main = ptx::make_idesc_bf16(GEMM_BM, GEMM_BN, false, !W_KMAJOR);
-      constexpr uint32_t idesc_lora = ptx::make_idesc_bf16(GEMM_BM, GEMM_BN, false, true);
+      constexpr uint32_t idesc_main_full = ptx::make_idesc_bf16(GEMM_BM, GEMM_BN, false, !W_KMAJOR);
+      constexpr uint32_t idesc_lora_full = ptx::make_idesc_bf16(GEMM_BM, GEMM_BN, false, true);
+      constexpr uint32_t idesc_main_half = ptx::make_idesc_bf16(GEMM_BM, GEMM_BN / 2, false, !W_KMAJOR);
+      constexpr uint32_t idesc_lora_half = ptx::make_idesc_bf16(GEMM_BM, GEMM_BN / 2, false, true);
       uint32_t it = 0, lt = 0, lora_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++lt) {
-        const int mt = tile % args.n_mtiles;
+      for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x, ++lt) {
+        int mt, n0, nw;
+        gemm_unit(args, unit, mt, n0, nw);
+        const uint32_t idesc_main = nw == GEMM_BN ? idesc_main_full : idesc_main_half;
+        const uint32_t idesc_lora = nw == GEMM_BN ? idesc_lora_full : idesc_lora_half;
         const uint32_t buf = lt & 1;
         if (!(ok = gemm_wait(bar_tempty(buf), ((lt >> 1) & 1) ^ 1, abort_flag, args.status))) break;
         ptx::tc_fence_after();
@@ -250,20 +276,22 @@ gemm_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
     const uint32_t stage0 = sEpi + (uint32_t)(warp - 2) * 8192u;
     uint32_t lt = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++lt) {
-      const int mt = tile % args.n_mtiles, nt = tile / args.n_mtiles;
-      const int m0 = mt * GEMM_BM + e * 32, n0 = nt * GEMM_BN;
+    for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x, ++lt) {
+      int mt, n0, nw;
+      gemm_unit(args, unit, mt, n0, nw);
+      const int m0 = mt * GEMM_BM + e * 32;
+      const int nchunks = nw / 64;
       const uint32_t buf = lt & 1;
       if (!(ok = gemm_wait(bar_tfull(buf), (lt >> 1) & 1, abort_flag, args.status))) break;
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + buf * GEMM_BN + ((uint32_t)(e * 32) << 16);
 #pragma unroll 1
-      for (int c = 0; c < GEMM_BN / 64; ++c) {
+      for (int c = 0; c < nchunks; ++c) {
         uint32_t v0[32], v1[32];
         ptx::tmem_ld_32x32b_x32(taddr + c * 64, v0);
         ptx::tmem_ld_32x32b_x32(taddr + c * 64 + 32, v1);
         ptx::tmem_ld_wait();
-        if (c == GEMM_BN / 64 - 1) {                // accumulator fully read: hand it back
+        if (c == nchunks - 1) {                     // accumulator fully read: hand it back
           ptx::tc_fence_before();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(bar_tempty(buf));
@@ -305,8 +333,9 @@ gemm_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
     const int rloc = (warp - 6) * 32 + lane;        // row inside the tile
     uint32_t it = 0, go_phase = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-      const int mt = tile % args.n_mtiles;
+    for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+      int mt, n0, nw;
+      gemm_unit(args, unit, mt, n0, nw);
       const int G = tile_groups(mt);
       const int LC = (G * R + 63) / 64;
       it += KB;

@@ -8,6 +8,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "mlora.h"
@@ -34,6 +35,7 @@ struct mlora_ctx {
   int64_t ws_counter_items = 0;
   int64_t launches = 0;
   int32_t gemm_path = 0;
+  int32_t shrink_path = 0;           // 0: streaming kernel for rank <= 32; 1: per-item kernel for every rank
   EncodeTiledFn encode = nullptr;
   // optional per-launch timing
   std::vector<cudaEvent_t> ev_start, ev_stop;
@@ -53,6 +55,7 @@ struct DevRowSpace {
   const int32_t* tile_grp_off = nullptr;
   const int32_t* grp_adapter = nullptr;
   const int32_t* item_rows = nullptr;
+  const int32_t* item_save = nullptr;
   const int32_t* item_start = nullptr;
   const int32_t* item_nrows = nullptr;
   const int32_t* item_adapter = nullptr;
@@ -96,6 +99,21 @@ mlora_status_t make_tmap_bf16(const mlora_ctx* ctx, CUtensorMap* m, const void* 
   return r == CUDA_SUCCESS ? MLORA_OK : MLORA_ERR_CUDA;
 }
 
+// [rows, cols] (cols contiguous, a multiple of 64) seen as (64, rows, cols / 64): a box of
+// 64 x box_rows x box_blocks lands in shared memory as box_blocks consecutive [box_rows][64]
+// blocks, the MN-major operand layout of the tensor-core kernel.
+mlora_status_t make_tmap_bf16_blocked(const mlora_ctx* ctx, CUtensorMap* m, const void* base, uint64_t rows,
+                                      uint64_t cols, uint64_t row_stride_elems, uint32_t box_rows, uint32_t box_blocks) {
+  cuuint64_t dims[3] = {64, rows, cols / 64};
+  cuuint64_t strides[2] = {row_stride_elems * 2, 128};
+  cuuint32_t box[3] = {64, box_rows, box_blocks};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = ctx->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MLORA_OK : MLORA_ERR_CUDA;
+}
+
 bool rank_ok_bf16(int r) { return r == 8 || r == 16 || r == 32 || r == 64 || r == 128; }
 
 mlora_status_t check_layer(const mlora_layer_t* L) {
@@ -128,10 +146,26 @@ struct LaunchScope {
   }
 };
 
+// Launch with programmatic stream serialization: the kernel may start its set-up while the
+// previous kernel of the stream drains; it calls griddepcontrol.wait before touching data.
+// Switched off while per-launch events are being recorded, so that those time whole kernels.
+template <typename... KArgs, typename... Args>
+void launch_pdl(bool overlap, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = overlap ? 1 : 0;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
 // ---- bf16 launches ------------------------------------------------------------------------
 template <int RB, int MT, int WARPS, int MIN_CTAS>
-void launch_shrink_rb(const ShrinkArgs& a, int n_items, int ksplit, cudaStream_t st) {
-  shrink_kernel<RB, MT, WARPS, MIN_CTAS><<<dim3(n_items, ksplit, kItemRows / (16 * MT)), WARPS * 32, 0, st>>>(a);
+void launch_shrink_rb(bool overlap, const ShrinkArgs& a, int n_items, int ksplit, cudaStream_t st) {
+  launch_pdl(overlap, shrink_kernel<RB, MT, WARPS, MIN_CTAS>, dim3(n_items, ksplit, kItemRows / (16 * MT)),
+             dim3(WARPS * 32), 0, st, a);
 }
 // Few items with a long contraction leave most SMs idle: split K over several CTAs per item so
 // that about three CTAs per SM are in flight, keeping at least 16 K-blocks (1024 elements) each.
@@ -142,19 +176,51 @@ int shrink_ksplit(const mlora_ctx* ctx, int n_items, int D) {
   k = k < kMaxKSplit ? k : kMaxKSplit;
   return k < 1 ? 1 : k;
 }
+template <int RB, int STAGES>
+mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, cudaStream_t st) {
+  constexpr int R = RB * 8;
+  constexpr size_t smem = (size_t)STAGES * (32 + R) * STREAM_PITCH + (size_t)(RB >= 4 ? 4 : 8) * 32 * (R + 1) * 4;
+  static bool attr_set = false;
+  auto kern = shrink_stream_kernel<RB, STAGES>;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return MLORA_ERR_CUDA;
+    attr_set = true;
+  }
+  StreamArgs sa;
+  sa.s = a;
+  sa.s.partial = ctx->ws_partial;
+  sa.s.counters = ctx->ws_counters;
+  sa.n_items = n_items;
+  sa.chunks_per_item = (a.D / 64 + STREAM_CHUNK - 1) / STREAM_CHUNK;
+  sa.n_units = n_items * sa.chunks_per_item;
+  int grid = sa.n_units < ctx->sm_count ? sa.n_units : ctx->sm_count;
+  sa.units_per_cta = (sa.n_units + grid - 1) / grid;
+  grid = (sa.n_units + sa.units_per_cta - 1) / sa.units_per_cta;
+  if (2 * (int64_t)grid > ctx->ws_partial_items || n_items > ctx->ws_counter_items) return MLORA_ERR_INVALID_ARG;
+  LaunchScope scope(ctx, st, KIND_SHRINK);
+  sa.status = ctx->status_dev;
+  launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(STREAM_THREADS), smem, st, sa);
+  return scope.done();
+}
+
 mlora_status_t launch_shrink(mlora_ctx* ctx, int R, ShrinkArgs a, int n_items, cudaStream_t st) {
   if (n_items <= 0) return MLORA_OK;
+  if (ctx->shrink_path == 0) {
+    if (R == 8) return launch_shrink_stream<1, 4>(ctx, a, n_items, st);
+    if (R == 16) return launch_shrink_stream<2, 4>(ctx, a, n_items, st);
+    if (R == 32) return launch_shrink_stream<4, 3>(ctx, a, n_items, st);
+  }
   const int ksplit = shrink_ksplit(ctx, n_items, a.D);
   a.partial = ctx->ws_partial;
   a.counters = ctx->ws_counters;
   if ((int64_t)n_items * ksplit > ctx->ws_partial_items || n_items > ctx->ws_counter_items) return MLORA_ERR_INVALID_ARG;
   LaunchScope scope(ctx, st, KIND_SHRINK);
   switch (R) {
-    case 8: launch_shrink_rb<1, 2, 8, 2>(a, n_items, ksplit, st); break;
-    case 16: launch_shrink_rb<2, 2, 8, 2>(a, n_items, ksplit, st); break;
-    case 32: launch_shrink_rb<4, 2, 8, 2>(a, n_items, ksplit, st); break;
-    case 64: launch_shrink_rb<8, 2, 4, 2>(a, n_items, ksplit, st); break;
-    case 128: launch_shrink_rb<16, 1, 4, 2>(a, n_items, ksplit, st); break;
+    case 8: launch_shrink_rb<1, 2, 8, 2>(scope.slot < 0, a, n_items, ksplit, st); break;
+    case 16: launch_shrink_rb<2, 2, 8, 2>(scope.slot < 0, a, n_items, ksplit, st); break;
+    case 32: launch_shrink_rb<4, 2, 8, 2>(scope.slot < 0, a, n_items, ksplit, st); break;
+    case 64: launch_shrink_rb<8, 2, 4, 2>(scope.slot < 0, a, n_items, ksplit, st); break;
+    case 128: launch_shrink_rb<16, 1, 4, 2>(scope.slot < 0, a, n_items, ksplit, st); break;
     default: return MLORA_ERR_UNSUPPORTED;
   }
   return scope.done();
@@ -171,9 +237,9 @@ mlora_status_t launch_grad(mlora_ctx* ctx, const GradArgs& a, int n_slots, cudaS
   }
   LaunchScope scope(ctx, st, KIND_GRAD);
   if (a.R <= 16) {
-    grad_kernel<1><<<dim3(a.D / 64, n_slots, 1), GRAD_THREADS, smem1, st>>>(a);
+    launch_pdl(scope.slot < 0, grad_kernel<1>, dim3(a.D / 64, n_slots, 1), dim3(GRAD_THREADS), smem1, st, a);
   } else {
-    grad_kernel<2><<<dim3(a.D / 64, n_slots, (a.R + 31) / 32), GRAD_THREADS, smem2, st>>>(a);
+    launch_pdl(scope.slot < 0, grad_kernel<2>, dim3(a.D / 64, n_slots, (a.R + 31) / 32), dim3(GRAD_THREADS), smem2, st, a);
   }
   return scope.done();
 }
@@ -188,10 +254,9 @@ mlora_status_t launch_gemm_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUten
       return MLORA_ERR_CUDA;
     attr_set = true;
   }
-  const int tiles = g.n_mtiles * g.n_ntiles;
-  const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+  const int grid = g.n_units < ctx->sm_count ? g.n_units : ctx->sm_count;
   LaunchScope scope(ctx, st, W_KMAJOR ? KIND_GEMM_BWD : KIND_GEMM_FWD);
-  kern<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(tIn, tW, tL, tOut, g);
+  launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(GEMM_THREADS), GEMM_SMEM_BYTES, st, tIn, tW, tL, tOut, g);
   return scope.done();
 }
 
@@ -217,17 +282,28 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
   mlora_status_t s;
   if ((s = make_tmap_bf16(ctx, &tIn, In, K, M, ld_in, GEMM_BK, GEMM_BM)) != MLORA_OK) return s;
   if (W_KMAJOR) {   // W [N rows, K cols] (the stored [d_in, d_out] matrix read as the transposed operand)
-    if ((s = make_tmap_bf16(ctx, &tW, L->W, K, N, L->ldw, GEMM_BK, GEMM_BN)) != MLORA_OK) return s;
+    if ((s = make_tmap_bf16(ctx, &tW, L->W, K, N, L->ldw, GEMM_BK, GEMM_BN / 2)) != MLORA_OK) return s;
   } else {          // W [K rows, N cols]
-    if ((s = make_tmap_bf16(ctx, &tW, L->W, N, K, L->ldw, 64, GEMM_BK)) != MLORA_OK) return s;
+    if ((s = make_tmap_bf16_blocked(ctx, &tW, L->W, K, N, L->ldw, GEMM_BK, 2)) != MLORA_OK) return s;
   }
   const int R = L->rank;
-  if ((s = make_tmap_bf16(ctx, &tL, L_all, N, (uint64_t)L->n_adapters * R, N, 64, R < 64 ? R : 64)) != MLORA_OK) return s;
+  if ((s = make_tmap_bf16_blocked(ctx, &tL, L_all, (uint64_t)L->n_adapters * R, N, N, R < 64 ? R : 64, 1)) != MLORA_OK)
+    return s;
   if ((s = make_tmap_bf16(ctx, &tOut, Out, N, M, ld_out, 64, 32)) != MLORA_OK) return s;
   GemmArgs g;
   g.M = M; g.N = N; g.K = K;
   g.n_mtiles = (M + GEMM_BM - 1) / GEMM_BM;
   g.n_ntiles = (N + GEMM_BN - 1) / GEMM_BN;
+  // The last wave of tiles usually fills only part of the SMs; when it fills at most half, its
+  // tiles are cut into two 128 x 128 halves so that it takes half as long.
+  {
+    const int tiles = g.n_mtiles * g.n_ntiles;
+    const int sms = ctx->sm_count;
+    const int rem = tiles % sms;
+    const bool split = tiles > sms && rem > 0 && 2 * rem <= sms;
+    g.n_full = split ? tiles - rem : tiles;
+    g.n_units = split ? tiles + rem : tiles;
+  }
   g.lora_enabled = hs.grp_adapter.empty() ? 0 : 1;
   g.row_grp = ds.row_grp; g.row_adapter = ds.row_adapter;
   g.tile_grp_off = ds.tile_grp_off; g.grp_adapter = ds.grp_adapter;
@@ -470,12 +546,12 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
     if (cudaSetDevice(ctx->device) != cudaSuccess) { delete p; return MLORA_ERR_CUDA; }
     BlobBuilder b;
     const HostPlan& h = p->h;
-    size_t o[32]; int n = 0;
+    size_t o[40]; int n = 0;
     const RowSpace* rs[2] = {&h.fwd, &h.bwd};
     for (int i = 0; i < 2; ++i) {
       o[n++] = b.add(rs[i]->row_adapter); o[n++] = b.add(rs[i]->row_save); o[n++] = b.add(rs[i]->row_grp);
       o[n++] = b.add(rs[i]->tile_grp_off); o[n++] = b.add(rs[i]->grp_adapter); o[n++] = b.add(rs[i]->item_rows);
-      o[n++] = b.add(rs[i]->item_start); o[n++] = b.add(rs[i]->item_nrows); o[n++] = b.add(rs[i]->item_adapter);
+      o[n++] = b.add(rs[i]->item_save); o[n++] = b.add(rs[i]->item_start); o[n++] = b.add(rs[i]->item_nrows); o[n++] = b.add(rs[i]->item_adapter);
     }
     o[n++] = b.add(h.slot_chunk_off); o[n++] = b.add(h.chunk_row0); o[n++] = b.add(h.chunk_nrows);
     o[n++] = b.add(h.ft_adapters);
@@ -488,7 +564,7 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
     for (int i = 0; i < 2; ++i) {
       ds[i]->row_adapter = p->blob + o[n++]; ds[i]->row_save = p->blob + o[n++]; ds[i]->row_grp = p->blob + o[n++];
       ds[i]->tile_grp_off = p->blob + o[n++]; ds[i]->grp_adapter = p->blob + o[n++]; ds[i]->item_rows = p->blob + o[n++];
-      ds[i]->item_start = p->blob + o[n++]; ds[i]->item_nrows = p->blob + o[n++]; ds[i]->item_adapter = p->blob + o[n++];
+      ds[i]->item_save = p->blob + o[n++]; ds[i]->item_start = p->blob + o[n++]; ds[i]->item_nrows = p->blob + o[n++]; ds[i]->item_adapter = p->blob + o[n++];
     }
     p->bwd.row_save = nullptr;       // the compact space has no save offsets
     p->slot_chunk_off = p->blob + o[n++]; p->chunk_row0 = p->blob + o[n++]; p->chunk_nrows = p->blob + o[n++];
@@ -568,7 +644,7 @@ mlora_status_t mlora_mixed_forward(mlora_ctx* ctx, const mlora_layer_t* L, const
   sa.In = (const __nv_bfloat16*)X; sa.ld_in = ldx; sa.D = L->d_in;
   sa.P_all = (const __nv_bfloat16*)L->A_all; sa.scale = nullptr; sa.Out = ctx->ws_p;
   sa.item_rows = p->fwd.item_rows; sa.item_start = p->fwd.item_start; sa.item_nrows = p->fwd.item_nrows;
-  sa.item_adapter = p->fwd.item_adapter; sa.row_save = p->fwd.row_save;
+  sa.item_adapter = p->fwd.item_adapter; sa.item_save = p->fwd.item_save;
   sa.x_save = (__nv_bfloat16*)x_save; sa.u_save = u_save; sa.save_base = save_row_base;
   if ((s = launch_shrink(ctx, L->rank, sa, h.fwd.n_items(), st)) != MLORA_OK) return s;
   return gemm_bf16<false>(ctx, L, h.fwd, p->fwd, X, ldx, Y, ldy, L->B_all, ctx->ws_p, L->scale, h.n_rows, L->d_out,
@@ -598,7 +674,7 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   sa.In = (const __nv_bfloat16*)dY; sa.ld_in = lddy; sa.D = L->d_out;
   sa.P_all = (const __nv_bfloat16*)L->B_all; sa.scale = L->scale; sa.Out = ctx->ws_p;
   sa.item_rows = p->bwd.item_rows; sa.item_start = p->bwd.item_start; sa.item_nrows = p->bwd.item_nrows;
-  sa.item_adapter = p->bwd.item_adapter; sa.row_save = nullptr; sa.x_save = nullptr; sa.u_save = nullptr; sa.save_base = 0;
+  sa.item_adapter = p->bwd.item_adapter; sa.item_save = nullptr; sa.x_save = nullptr; sa.u_save = nullptr; sa.save_base = 0;
   if ((s = launch_shrink(ctx, L->rank, sa, h.bwd.n_items(), st)) != MLORA_OK) return s;
 
   GradArgs ga;                       // dB = (s U)^T dY
@@ -630,8 +706,9 @@ mlora_status_t mlora_poll_status(mlora_ctx* ctx, void* cuda_stream) {
 int64_t mlora_launch_count(const mlora_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path) {
-  if (!ctx || (path != 0 && path != 1)) return MLORA_ERR_INVALID_ARG;
-  ctx->gemm_path = path;
+  if (!ctx || path < 0 || path > 2) return MLORA_ERR_INVALID_ARG;
+  ctx->gemm_path = path == 1 ? 1 : 0;
+  ctx->shrink_path = path == 2 ? 1 : 0;
   return MLORA_OK;
 }
 

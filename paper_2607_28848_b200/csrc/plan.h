@@ -30,6 +30,7 @@ struct RowSpace {
   // not be adjacent in the batch: decode rows that share an adapter are processed together, so an
   // adapter's matrix is fetched once per item instead of once per row.
   std::vector<int32_t> item_rows;      // [rows with an adapter] row ids, grouped by adapter
+  std::vector<int32_t> item_save;      // parallel to item_rows: save offset of that row or -1
   std::vector<int32_t> item_start, item_nrows, item_adapter;
   int32_t n_tiles() const { return (n_rows + kTileRows - 1) / kTileRows; }
   int32_t n_items() const { return (int32_t)item_start.size(); }
@@ -77,6 +78,9 @@ inline void build_tiles_and_items(RowSpace& rs) {
     std::vector<int32_t> fill(count.begin(), count.end());
     for (int32_t t = 0; t < n; ++t) if (rs.row_adapter[t] >= 0) rs.item_rows[fill[rs.row_adapter[t]]++] = t;
   }
+  rs.item_save.assign(rs.item_rows.size(), -1);
+  if (!rs.row_save.empty())
+    for (size_t i = 0; i < rs.item_rows.size(); ++i) rs.item_save[i] = rs.row_save[rs.item_rows[i]];
   for (int32_t a = 0; a <= max_adapter; ++a) {
     for (int32_t i = count[a]; i < count[a + 1]; i += kItemRows) {
       rs.item_start.push_back(i);

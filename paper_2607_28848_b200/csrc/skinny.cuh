@@ -28,7 +28,7 @@ struct ShrinkArgs {
   const int32_t* item_start;   // first entry of the item in item_rows
   const int32_t* item_nrows;
   const int32_t* item_adapter;
-  const int32_t* row_save;     // nullable: [rows] save offset of a row or -1
+  const int32_t* item_save;    // nullable: parallel to item_rows, save offset of the row or -1
   __nv_bfloat16* x_save;       // nullable, [cap, D] dense
   float* u_save;               // nullable, [cap, R] dense
   int64_t save_base;
@@ -61,6 +61,7 @@ shrink_kernel(const ShrinkArgs a) {
   const int item = blockIdx.x * gridDim.z + blockIdx.z;          // index of this row block in the scratch
   const int adapter = a.item_adapter[blockIdx.x];
   const int32_t* rows = a.item_rows + a.item_start[blockIdx.x] + roff;
+  const int32_t* saves = a.item_save ? a.item_save + a.item_start[blockIdx.x] + roff : nullptr;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, c = lane & 3;
@@ -74,11 +75,14 @@ shrink_kernel(const ShrinkArgs a) {
     if (rl < nrows) {
       const int row = rows[rl];
       xp[j] = a.In + (size_t)row * a.ld_in + 16 * c;
-      const int sv = (a.row_save && a.x_save) ? a.row_save[row] : -1;
+      const int sv = (saves && a.x_save) ? saves[rl] : -1;
       if (sv >= 0) sp[j] = a.x_save + (size_t)(a.save_base + sv) * a.D + 16 * c;
     }
   }
   const __nv_bfloat16* p0 = a.P_all + ((size_t)adapter * R + g) * a.D + 16 * c;
+  // everything above read only the plan's tables; from here on the predecessor's data is touched
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();
 
   float acc[MT][RB][4];
 #pragma unroll
@@ -172,12 +176,279 @@ shrink_kernel(const ShrinkArgs a) {
     }
     const int row = rows[r];
     a.Out[(size_t)row * R + q] = u * sc;
-    if (a.u_save && a.row_save) {
-      const int sv = a.row_save[row];
+    if (a.u_save && saves) {
+      const int sv = saves[r];
       if (sv >= 0) a.u_save[(size_t)(a.save_base + sv) * R + q] = u;
     }
   }
   if (ksplit > 1 && threadIdx.x == 0) a.counters[item] = 0;     // ready for the next launch
+}
+
+// ---------------------------------------------------------------------------------------------
+// Streaming shrink for ranks up to 32: a persistent grid (one CTA per SM) walks the flattened list
+// of work units (item, chunk of 8 K-blocks = 512 elements) in equal contiguous ranges, so every SM
+// streams the same number of bytes in one wave.  A producer warp moves each unit into a
+// STAGES-deep shared-memory ring with bulk asynchronous copies (one 1 KiB copy per row of the
+// item and per row of the adapter, completion counted on an mbarrier), which keeps ~150 KB per SM
+// in flight at almost no instruction cost.  Eight consumer warps each take one K-block of the
+// unit: fragments come out of shared memory with conflict-free 16-byte loads (row pitch 1040 B),
+// feed mma.sync, and the rows of In are stored on to x_save for fine-tuning rows.  Accumulators
+// persist across the chunks of an item and are flushed when the item ends.  An item whose chunks
+// were shared by several CTAs is finished by whichever of them arrives last, adding the partials
+// in CTA order (a fixed order).  Every mbarrier wait is bounded.
+constexpr int STREAM_WARPS = 8;      // consumer warps; warp 8 is the producer
+constexpr int STREAM_THREADS = (STREAM_WARPS + 1) * 32;
+constexpr int STREAM_CHUNK = 8;      // K-blocks (of 64) per unit: one per consumer warp
+constexpr uint32_t STREAM_PITCH = 1040;   // bytes between rows of a stage (1 KiB + 16: no bank conflicts)
+constexpr uint32_t STREAM_SPIN_LIMIT = 1u << 22;
+
+struct StreamArgs {
+  ShrinkArgs s;
+  int32_t n_items;
+  int32_t chunks_per_item;   // ceil(D / 512)
+  int32_t n_units;           // n_items * chunks_per_item
+  int32_t units_per_cta;     // ceil(n_units / gridDim.x)
+  int32_t* status;           // device status word
+};
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ bool stream_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  for (uint32_t i = 0; i < STREAM_SPIN_LIMIT; ++i) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((i & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  atomicExch(status, (int32_t)MLORA_ERR_DEVICE_TIMEOUT);
+  return false;
+}
+
+template <int RB, int STAGES>
+__global__ void __launch_bounds__(STREAM_THREADS, 1)
+shrink_stream_kernel(const StreamArgs sa) {
+  constexpr int R = RB * 8;
+  constexpr int ROWS = 32 + R;                            // rows of a stage: the item's, then the adapter's
+  constexpr uint32_t STAGE_BYTES = ROWS * STREAM_PITCH;
+  constexpr int RW = RB >= 4 ? 4 : 8;                     // reduction buffers (rank 32: two rounds of 4 warps)
+  extern __shared__ __align__(128) uint8_t stream_smem[];
+  float (*red)[32][R + 1] = reinterpret_cast<float (*)[32][R + 1]>(stream_smem + STAGES * STAGE_BYTES);
+  __shared__ __align__(8) uint64_t bars[2 * STAGES];     // full[STAGES] | empty[STAGES]
+  __shared__ int is_last;
+  __shared__ int abort_word;
+  volatile int* abort_flag = &abort_word;
+  const ShrinkArgs& a = sa.s;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int cta = blockIdx.x;
+  const int u_begin = cta * sa.units_per_cta;
+  const int u_end = min(u_begin + sa.units_per_cta, sa.n_units);
+  const int KC = sa.chunks_per_item;
+  const int nkb = a.D / 64;
+  const uint32_t ring = ptx::smem_u32(stream_smem);
+  const uint32_t bar0 = ptx::smem_u32(bars);
+  auto bar_full = [&](int st) { return bar0 + 8u * st; };
+  auto bar_empty = [&](int st) { return bar0 + 8u * (STAGES + st); };
+
+  if (threadIdx.x == 0) {
+    for (int st = 0; st < STAGES; ++st) {
+      ptx::mbar_init(bar_full(st), 1);
+      ptx::mbar_init(bar_empty(st), STREAM_WARPS);
+    }
+    abort_word = 0;
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
+
+  if (warp == STREAM_WARPS) {
+    // ======================= producer =======================
+    int item = u_begin / KC, kc = u_begin % KC;
+    int cur = -1, nrows = 0;
+    const __nv_bfloat16* src0 = nullptr;     // lane l moves stage row l ...
+    const __nv_bfloat16* src1 = nullptr;     // ... and stage row l + 32 (adapter row l), if l < R
+    auto set_item = [&](int it) {
+      cur = it;
+      nrows = a.item_nrows[it];
+      src0 = lane < nrows ? a.In + (size_t)a.item_rows[a.item_start[it] + lane] * a.ld_in : nullptr;
+      src1 = lane < R ? a.P_all + ((size_t)a.item_adapter[it] * R + lane) * a.D : nullptr;
+    };
+    if (u_begin < u_end) set_item(item);
+    ptx::grid_dependency_wait();             // only plan tables were read so far
+    ptx::grid_launch_dependents();
+    bool ok = true;
+    for (int u = u_begin; u < u_end && ok; ++u) {
+      const int i = u - u_begin, st = i % STAGES;
+      if (item != cur) set_item(item);
+      if (lane == 0) ok = stream_wait(bar_empty(st), ((i / STAGES) & 1) ^ 1, abort_flag, sa.status);
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+      const int k0 = kc * (STREAM_CHUNK * 64);
+      const uint32_t bytes = (uint32_t)min(STREAM_CHUNK * 64, a.D - k0) * 2u;
+      if (lane == 0) ptx::mbar_arrive_expect_tx(bar_full(st), (uint32_t)(nrows + R) * bytes);
+      __syncwarp();
+      const uint32_t dst = ring + (uint32_t)st * STAGE_BYTES;
+      if (src0) bulk_load(dst + (uint32_t)lane * STREAM_PITCH, src0 + k0, bytes, bar_full(st));
+      if (src1) bulk_load(dst + (uint32_t)(32 + lane) * STREAM_PITCH, src1 + k0, bytes, bar_full(st));
+      if (++kc == KC) { kc = 0; ++item; }
+    }
+  } else {
+    // ======================= consumers =======================
+    const int g = lane >> 2, c = lane & 3;
+    float acc[2][RB][4];
+#pragma unroll
+    for (int m = 0; m < 2; ++m)
+#pragma unroll
+      for (int i = 0; i < RB; ++i) acc[m][i][0] = acc[m][i][1] = acc[m][i][2] = acc[m][i][3] = 0.f;
+
+    int item = u_begin / KC, kc = u_begin % KC;
+    int cur_item = -1, cur_nrows = 0, cur_adapter = 0;
+    const int32_t* cur_rows = nullptr;
+    const int32_t* cur_saves = nullptr;
+    __nv_bfloat16* sp[4] = {nullptr, nullptr, nullptr, nullptr};
+    // byte offset of this thread's pieces inside a stage row: K-block `warp`, elements 16c .. 16c+15
+    const uint32_t piece = (uint32_t)warp * 128u + (uint32_t)c * 32u;
+    ptx::grid_dependency_wait();
+    bool ok = true;
+
+    for (int u = u_begin; u < u_end; ++u) {
+      const int i = u - u_begin, st = i % STAGES;
+      if (item != cur_item) {
+        cur_item = item;
+        cur_nrows = a.item_nrows[item];
+        cur_adapter = a.item_adapter[item];
+        cur_rows = a.item_rows + a.item_start[item];
+        cur_saves = a.item_save ? a.item_save + a.item_start[item] : nullptr;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int rl = g + 8 * j;
+          const int sv = (cur_saves && a.x_save && rl < cur_nrows) ? cur_saves[rl] : -1;
+          sp[j] = sv >= 0 ? a.x_save + (size_t)(a.save_base + sv) * a.D + 16 * c : nullptr;
+        }
+      }
+      ok = stream_wait(bar_full(st), (i / STAGES) & 1, abort_flag, sa.status);
+      if (!ok) break;
+      const int kb = kc * STREAM_CHUNK + warp;
+      if (kb < nkb) {
+        const uint32_t src = ring + (uint32_t)st * STAGE_BYTES + piece;
+        uint4 x[4][2];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t ra = src + (uint32_t)(g + 8 * j) * STREAM_PITCH;
+          x[j][0] = lds_v4(ra);
+          x[j][1] = lds_v4(ra + 16);
+        }
+        uint4 p[RB][2];
+#pragma unroll
+        for (int n = 0; n < RB; ++n) {
+          const uint32_t rp = src + (uint32_t)(32 + 8 * n + g) * STREAM_PITCH;
+          p[n][0] = lds_v4(rp);
+          p[n][1] = lds_v4(rp + 16);
+        }
+        // rows past the item's end were not copied: their stale bytes only reach accumulator rows
+        // that are never written out, but keep them out of the MMA anyway
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (g + 8 * j >= cur_nrows) { x[j][0] = make_uint4(0, 0, 0, 0); x[j][1] = make_uint4(0, 0, 0, 0); }
+#pragma unroll
+        for (int n = 0; n < RB; ++n) {
+          const uint32_t rp[8] = {p[n][0].x, p[n][0].y, p[n][0].z, p[n][0].w, p[n][1].x, p[n][1].y, p[n][1].z, p[n][1].w};
+#pragma unroll
+          for (int m = 0; m < 2; ++m) {
+            const uint4 &l0 = x[2 * m][0], &l1 = x[2 * m][1], &h0 = x[2 * m + 1][0], &h1 = x[2 * m + 1][1];
+            const uint32_t ra[8] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w};
+            const uint32_t rb[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
+#pragma unroll
+            for (int s = 0; s < 4; ++s)
+              ptx::mma_bf16_16816(acc[m][n], ra[2 * s], rb[2 * s], ra[2 * s + 1], rb[2 * s + 1], rp[2 * s], rp[2 * s + 1]);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar_empty(st));      // the stage's bytes are in registers now
+        const int ko = kb * 64;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (sp[j]) {     // activation save: the rows of In pass through here exactly once
+            *reinterpret_cast<uint4*>(sp[j] + ko) = x[j][0];
+            *reinterpret_cast<uint4*>(sp[j] + ko + 8) = x[j][1];
+          }
+      } else {
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar_empty(st));
+      }
+
+      // ---- flush when the item (or this CTA's range) ends ----
+      const bool item_ends = (kc == KC - 1) || (u == u_end - 1);
+      const int this_item = item;
+      if (++kc == KC) { kc = 0; ++item; }
+      if (!item_ends) continue;
+#pragma unroll
+      for (int round = 0; round < STREAM_WARPS / RW; ++round) {
+        if (warp / RW == round) {
+          float (*mine)[R + 1] = red[warp % RW];
+#pragma unroll
+          for (int m = 0; m < 2; ++m)
+#pragma unroll
+            for (int n = 0; n < RB; ++n) {
+              float* r0 = &mine[m * 16 + g][n * 8 + 2 * c];
+              float* r1 = &mine[m * 16 + g + 8][n * 8 + 2 * c];
+              if (round == 0) { r0[0] = acc[m][n][0]; r0[1] = acc[m][n][1]; r1[0] = acc[m][n][2]; r1[1] = acc[m][n][3]; }
+              else { r0[0] += acc[m][n][0]; r0[1] += acc[m][n][1]; r1[0] += acc[m][n][2]; r1[1] += acc[m][n][3]; }
+              acc[m][n][0] = acc[m][n][1] = acc[m][n][2] = acc[m][n][3] = 0.f;
+            }
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");    // consumers only
+      }
+      const int c0 = (this_item * KC) / sa.units_per_cta, c1 = (this_item * KC + KC - 1) / sa.units_per_cta;
+      bool finish = true;                // does this CTA write the item's final result?
+      if (c0 != c1) {
+        const int slot = (this_item == (cta * sa.units_per_cta) / KC) ? 0 : 1;
+        float* mine = a.partial + ((size_t)cta * 2 + slot) * (32 * R);
+        for (int idx = threadIdx.x; idx < cur_nrows * R; idx += STREAM_WARPS * 32) {
+          const int r = idx / R, q = idx % R;
+          float v = 0.f;
+#pragma unroll
+          for (int w = 0; w < RW; ++w) v += red[w][r][q];
+          mine[idx] = v;
+        }
+        __threadfence();
+        asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");
+        if (threadIdx.x == 0) is_last = (atomicAdd(a.counters + this_item, 1) == c1 - c0);
+        asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");
+        finish = is_last != 0;
+        if (finish) __threadfence();
+      }
+      if (finish) {
+        const float sc = a.scale ? a.scale[cur_adapter] : 1.0f;
+        for (int idx = threadIdx.x; idx < cur_nrows * R; idx += STREAM_WARPS * 32) {
+          const int r = idx / R, q = idx % R;
+          float v = 0.f;
+          if (c0 != c1) {
+            for (int cc = c0; cc <= c1; ++cc) {        // fixed order: by CTA index
+              const int slot = (this_item == (cc * sa.units_per_cta) / KC) ? 0 : 1;
+              v += __ldcg(a.partial + ((size_t)cc * 2 + slot) * (32 * R) + idx);
+            }
+          } else {
+#pragma unroll
+            for (int w = 0; w < RW; ++w) v += red[w][r][q];
+          }
+          const int row = cur_rows[r];
+          a.Out[(size_t)row * R + q] = v * sc;
+          if (a.u_save && cur_saves) {
+            const int sv = cur_saves[r];
+            if (sv >= 0) a.u_save[(size_t)(a.save_base + sv) * R + q] = v;
+          }
+        }
+        if (c0 != c1 && threadIdx.x == 0) a.counters[this_item] = 0;    // ready for the next launch
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");      // red[] is reused by the next item
+    }
+  }
 }
 
 struct GradArgs {
@@ -210,7 +481,7 @@ grad_kernel(const GradArgs a) {
   const int qbase = blockIdx.z * MB * 16;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, c = lane & 3;
-  const float sc = a.scale ? a.scale[a.slot_adapter[slot]] : 1.0f;
+  const int slot_ad = a.slot_adapter[slot];
   const int R = a.R;
 
   float acc[MB][8][4];
@@ -220,6 +491,9 @@ grad_kernel(const GradArgs a) {
     for (int n = 0; n < 8; ++n) acc[m][n][0] = acc[m][n][1] = acc[m][n][2] = acc[m][n][3] = 0.f;
 
   const int ch0 = a.slot_chunk_off[slot], ch1 = a.slot_chunk_off[slot + 1];
+  ptx::grid_dependency_wait();       // only plan tables were read so far
+  ptx::grid_launch_dependents();
+  const float sc = a.scale ? a.scale[slot_ad] : 1.0f;
   const uint4 zero4 = make_uint4(0, 0, 0, 0);
   const int tr[4] = {2 * c, 2 * c + 1, 2 * c + 8, 2 * c + 9};
   // Two-deep register pipeline: the loads of chunk i+1 (4 rows of Q, 8 values of P per rank

@@ -77,7 +77,7 @@ def test_cfg1_tiny_fp32(sess):
     run_and_check(sess, w, synth.make_tensors(w))
 
 
-@pytest.mark.parametrize("path", [0, 1])
+@pytest.mark.parametrize("path", [0, 1, 2])
 def test_bf16_ragged_multi_tile(sess, path):
     w = synth.random_workload(5, 256, 512, 16, 6, 389, max_seg=150)
     run_and_check(sess, w, synth.make_tensors(w), path=path)
