@@ -180,10 +180,10 @@ int64_t mlora_launch_count(const mlora_ctx* ctx);
 mlora_status_t mlora_profile_enable(mlora_ctx* ctx, int32_t max_records);
 int32_t mlora_profile_collect(mlora_ctx* ctx, int32_t* kinds, float* ms, int32_t cap);
 
-/* Selects kernel variants for MLORA_BF16 layers: 0 = defaults (tcgen05 tensor-core GEMM, streaming
- * shrink kernel for rank <= 32); 1 = the plain CUDA-core kernels for every step (a slow
+/* Selects kernel variants for MLORA_BF16 layers: 0 = defaults (two-SM tcgen05 tensor-core GEMM,
+ * streaming shrink kernel for rank <= 32); 1 = the plain CUDA-core kernels for every step (a slow
  * cross-check used by the tests); 2 = defaults, but the per-item shrink kernel for every rank
- * (the variant ranks 64 and 128 always use). */
+ * (the variant ranks 64 and 128 always use); 3 = defaults, but the one-SM tensor-core GEMM. */
 mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path);
 
 /* ---- forward without any allocation -----------------------------------------------------*/

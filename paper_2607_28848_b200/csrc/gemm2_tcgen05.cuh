@@ -1,0 +1,422 @@
+// Two-SM variant of the fused GEMM + LoRA-expand kernel (see gemm_tcgen05.cuh for the operator).
+//
+// Two CTAs of a cluster (a pair of SMs) share one 256 x 256 output tile with tcgen05.mma
+// cta_group::2: CTA r of the pair owns rows [128 r, 128 r + 128) of the tile (its A operand and
+// its accumulator, 128 lanes x 256 columns of its own tensor memory) and supplies columns
+// [128 r, 128 r + 128) of the B operand; the tensor cores of both SMs read both halves of B.
+// Per output element this moves a third less data from L2 into shared memory than two
+// independent 128 x 256 tiles, which is what bounds the one-SM kernel.  No load is multicast:
+// every CTA fetches exactly the bytes that land in its own shared memory.
+//
+// Synchronisation across the pair (rank 0 = leader, the only issuer of MMAs):
+//   full[s]       in the leader: leader's producer arrives with the byte count of BOTH CTAs;
+//                 both CTAs' TMA loads complete on it (cta_group::2 loads may signal the peer).
+//   empty[s]      in each CTA: tcgen05.commit multicast to both (releases both producers).
+//   lora_go[s]    in each CTA: producer -> its own operand builders (slot is free).
+//   lora_full[s]  in the leader: 8 arrivals = 4 builder warps x 2 CTAs.
+//   tmem_full[b]  in each CTA: tcgen05.commit multicast (wakes both epilogues).
+//   tmem_empty[b] in the leader: 8 arrivals = 4 epilogue warps x 2 CTAs.
+// Every wait is bounded; the pair leaves through a cluster barrier before tensor memory is freed,
+// so neither CTA exits while the other may still touch its shared memory.
+#pragma once
+
+#include <cuda.h>
+
+#include "gemm_tcgen05.cuh"
+#include "ptx.cuh"
+
+namespace mlora {
+
+constexpr int GEMM2_BM = 256;                 // rows of a pair tile (128 per CTA)
+constexpr int GEMM2_BN = 256;
+constexpr int GEMM2_STAGES = 6;
+constexpr uint32_t GEMM2_A_BYTES = 128 * GEMM_BK * 2;               // 16 KiB: this CTA's rows
+constexpr uint32_t GEMM2_B_BYTES = 128 * GEMM_BK * 2;               // 16 KiB: this CTA's half of B
+constexpr uint32_t GEMM2_STAGE_BYTES = GEMM2_A_BYTES + GEMM2_B_BYTES;
+constexpr uint32_t GEMM2_SMEM_BYTES = GEMM2_STAGES * GEMM2_STAGE_BYTES + GEMM_EPI_BYTES + 512 + 1024;
+
+namespace ptx {
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Arrive on an mbarrier given by a shared::cluster address (possibly in the peer CTA).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred P;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 P, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Tiled loads of a CTA pair: data lands in the executing CTA, completion is counted on `bar`,
+// a shared::cluster address that may name the peer's barrier.
+__device__ __forceinline__ void tma2_load_2d(uint32_t dst, const void* tmap, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma2_load_3d(uint32_t dst, const void* tmap, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tmem2_alloc(uint32_t smem_result, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem2_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem2_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma2_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on the barrier at this shared-memory offset in BOTH CTAs of the pair once every
+// tcgen05 operation issued so far by this thread is done.
+__device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
+  asm volatile(
+      "{\n\t.reg .b16 m;\n\tmov.b16 m, 3;\n\t"
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n\t}\n"
+      ::"r"(bar) : "memory");
+}
+
+}  // namespace ptx
+
+__device__ __forceinline__ bool gemm2_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  for (uint32_t i = 0; i < GEMM_SPIN_LIMIT; ++i) {
+    if (ptx::mbar_try_wait_cluster(bar, parity)) return true;
+    if ((i & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  atomicExch(status, (int32_t)MLORA_ERR_DEVICE_TIMEOUT);
+  return false;
+}
+
+// args: n_mtiles counts 256-row pair tiles, n_ntiles 256-column tiles, n_units = their product;
+// row_grp / tile_grp_off / grp_adapter are the tables for 256-row tiles.
+template <int R, bool W_KMAJOR>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ CUtensorMap tmW,
+                  const __grid_constant__ CUtensorMap tmL, const __grid_constant__ CUtensorMap tmOut,
+                  const GemmArgs args) {
+  static_assert(R == 8 || R == 16 || R == 32 || R == 64 || R == 128, "rank");
+  constexpr int GPC = R <= 64 ? 64 / R : 1;          // groups per 64-wide low-rank block
+  constexpr int S = GEMM2_STAGES;
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+
+  const uint32_t sA0 = smem_base;
+  const uint32_t sEpi = smem_base + S * GEMM2_STAGE_BYTES;
+  const uint32_t sBar = sEpi + GEMM_EPI_BYTES;
+  // barriers: full[S] | empty[S] | lora_full[S] | lora_go[S] | tmem_full[2] | tmem_empty[2]
+  auto bar_full = [&](int s) { return sBar + 8u * s; };
+  auto bar_empty = [&](int s) { return sBar + 8u * (S + s); };
+  auto bar_lora = [&](int s) { return sBar + 8u * (2 * S + s); };
+  auto bar_go = [&](int s) { return sBar + 8u * (3 * S + s); };
+  auto bar_tfull = [&](int b) { return sBar + 8u * (4 * S + b); };
+  auto bar_tempty = [&](int b) { return sBar + 8u * (4 * S + 2 + b); };
+  const uint32_t sMisc = sBar + 8u * (4 * S + 4);
+  uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(smem_gen + (sMisc - smem_base));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + (sMisc - smem_base) + 8);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = ptx::cluster_ctarank();     // 0: leader
+  const bool leader = rank == 0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      ptx::mbar_init(bar_full(s), 1);
+      ptx::mbar_init(bar_empty(s), 1);
+      ptx::mbar_init(bar_lora(s), 8);
+      ptx::mbar_init(bar_go(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(bar_tfull(b), 1);
+      ptx::mbar_init(bar_tempty(b), 8);
+    }
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmIn);
+    ptx::prefetch_tmap(&tmW);
+    ptx::prefetch_tmap(&tmL);
+    ptx::prefetch_tmap(&tmOut);
+  }
+  if (warp == 1) {                                   // the same warp in both CTAs
+    ptx::tmem2_alloc(ptx::smem_u32(tmem_ptr_smem), GEMM_TMEM_COLS);
+    ptx::tmem2_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync_all();                           // the peer's barriers exist from here on
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_ptr_smem;
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();
+
+  const int KB = (args.K + GEMM_BK - 1) / GEMM_BK;
+  const int n_units = args.n_units;
+  const int n_pairs = gridDim.x >> 1;
+  const int pair = blockIdx.x >> 1;
+
+  auto tile_groups = [&](int mt) -> int {
+    return args.lora_enabled ? (args.tile_grp_off[mt + 1] - args.tile_grp_off[mt]) : 0;
+  };
+
+  if (warp == 0) {
+    // ============================ TMA producer (both CTAs) ============================
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int unit = pair; unit < n_units && ok; unit += n_pairs) {
+        const int mt = unit % args.n_mtiles, nt = unit / args.n_mtiles;
+        const int m0 = mt * GEMM2_BM + (int)rank * 128;
+        const int nh = nt * GEMM2_BN + (int)rank * 128;     // this CTA's half of the B columns
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % S;
+          if (!(ok = gemm2_wait(bar_empty(s), ((it / S) & 1) ^ 1, abort_flag, args.status))) break;
+          const uint32_t a = sA0 + s * GEMM2_STAGE_BYTES, b = a + GEMM2_A_BYTES;
+          const uint32_t full = ptx::map_to_cta(bar_full(s), 0);
+          if (leader) ptx::mbar_arrive_expect_tx(bar_full(s), 2 * GEMM2_STAGE_BYTES);
+          ptx::tma2_load_2d(a, &tmIn, kb * GEMM_BK, m0, full);
+          if (W_KMAJOR) ptx::tma2_load_2d(b, &tmW, kb * GEMM_BK, nh, full);          // [N, K]: 128 rows x 64 k
+          else          ptx::tma2_load_3d(b, &tmW, 0, kb * GEMM_BK, nh >> 6, full);  // (64 n, K, N/64): 64 x 64 k x 2
+        }
+        if (!ok) break;
+        const int G = tile_groups(mt);
+        const int LC = (G * R + 63) / 64;
+        const int32_t* ga = args.grp_adapter + (args.lora_enabled ? args.tile_grp_off[mt] : 0);
+        for (int lc = 0; lc < LC; ++lc, ++it) {
+          const int s = it % S;
+          if (!(ok = gemm2_wait(bar_empty(s), ((it / S) & 1) ^ 1, abort_flag, args.status))) break;
+          ptx::mbar_arrive(bar_go(s));               // hand the free slot to this CTA's builders
+          const uint32_t b = sA0 + s * GEMM2_STAGE_BYTES + GEMM2_A_BYTES;
+          const uint32_t full = ptx::map_to_cta(bar_full(s), 0);
+          if (R <= 64) {
+            const int g0 = lc * GPC;
+            const int ng = G - g0 < GPC ? G - g0 : GPC;
+            const int ngl = (R == 8 && (ng & 1)) ? ng + 1 : ng;   // rank 8: pad a half-filled MMA step
+            if (leader) ptx::mbar_arrive_expect_tx(bar_full(s), 2u * (uint32_t)ngl * R * 128u * 2u);
+            for (int i = 0; i < ngl; ++i) {
+              const int adapter = ga[g0 + (i < ng ? i : ng - 1)];
+#pragma unroll
+              for (int nb = 0; nb < 2; ++nb)
+                ptx::tma2_load_3d(b + nb * 8192 + i * R * 128, &tmL, 0, adapter * R, (nh >> 6) + nb, full);
+            }
+          } else {
+            const int adapter = ga[lc >> 1];
+            if (leader) ptx::mbar_arrive_expect_tx(bar_full(s), 2u * 64u * 128u * 2u);
+#pragma unroll
+            for (int nb = 0; nb < 2; ++nb)
+              ptx::tma2_load_3d(b + nb * 8192, &tmL, 0, adapter * R + (lc & 1) * 64, (nh >> 6) + nb, full);
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ============================ MMA issuer (leader only) ============================
+    if (leader && lane == 0) {
+      constexpr uint32_t idesc_main = ptx::make_idesc_bf16(GEMM2_BM, GEMM2_BN, false, !W_KMAJOR);
+      constexpr uint32_t idesc_lora = ptx::make_idesc_bf16(GEMM2_BM, GEMM2_BN, false, true);
+      uint32_t it = 0, lt = 0, lora_phase = 0;
+      bool ok = true;
+      for (int unit = pair; unit < n_units && ok; unit += n_pairs, ++lt) {
+        const int mt = unit % args.n_mtiles;
+        const uint32_t buf = lt & 1;
+        if (!(ok = gemm2_wait(bar_tempty(buf), ((lt >> 1) & 1) ^ 1, abort_flag, args.status))) break;
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * GEMM2_BN;
+        uint32_t acc = 0;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % S;
+          if (!(ok = gemm2_wait(bar_full(s), (it / S) & 1, abort_flag, args.status))) break;
+          ptx::tc_fence_after();
+          const uint32_t a = sA0 + s * GEMM2_STAGE_BYTES, b = a + GEMM2_A_BYTES;
+          const uint64_t adesc = ptx::make_smem_desc(a, 16, 1024);
+          const uint64_t bdesc = W_KMAJOR ? ptx::make_smem_desc(b, 16, 1024) : ptx::make_smem_desc(b, 8192, 1024);
+#pragma unroll
+          for (int ks = 0; ks < GEMM_BK / 16; ++ks) {
+            ptx::umma2_f16(d_tmem, adesc + (uint64_t)(ks * 2), bdesc + (uint64_t)(W_KMAJOR ? ks * 2 : ks * 128),
+                           idesc_main, acc);
+            acc = 1;
+          }
+          ptx::umma2_commit_both(bar_empty(s));
+        }
+        if (!ok) break;
+        const int G = tile_groups(mt);
+        const int LC = (G * R + 63) / 64;
+        for (int lc = 0; lc < LC; ++lc, ++it) {
+          const int s = it % S;
+          if (!(ok = gemm2_wait(bar_full(s), (it / S) & 1, abort_flag, args.status))) break;
+          if (!(ok = gemm2_wait(bar_lora(s), (lora_phase >> s) & 1, abort_flag, args.status))) break;
+          lora_phase ^= 1u << s;
+          ptx::tc_fence_after();
+          const uint32_t a = sA0 + s * GEMM2_STAGE_BYTES, b = a + GEMM2_A_BYTES;
+          const uint64_t adesc = ptx::make_smem_desc(a, 16, 1024);
+          const uint64_t bdesc = ptx::make_smem_desc(b, 8192, 1024);
+          int ksteps = (G * R - lc * 64 + 15) / 16;
+          ksteps = ksteps < 4 ? ksteps : 4;
+          for (int ks = 0; ks < ksteps; ++ks) {
+            ptx::umma2_f16(d_tmem, adesc + (uint64_t)(ks * 2), bdesc + (uint64_t)(ks * 128), idesc_lora, acc);
+            acc = 1;
+          }
+          ptx::umma2_commit_both(bar_empty(s));
+        }
+        if (!ok) break;
+        ptx::umma2_commit_both(bar_tfull(buf));
+      }
+    }
+    __syncwarp();
+  } else if (warp < 6) {
+    // ============================ epilogue (both CTAs, own rows) ============================
+    const int e = warp & 3;
+    const uint32_t stage0 = sEpi + (uint32_t)(warp - 2) * 8192u;
+    uint32_t lt = 0;
+    bool ok = true;
+    for (int unit = pair; unit < n_units && ok; unit += n_pairs, ++lt) {
+      const int mt = unit % args.n_mtiles, nt = unit / args.n_mtiles;
+      const int m0 = mt * GEMM2_BM + (int)rank * 128 + e * 32, n0 = nt * GEMM2_BN;
+      const uint32_t buf = lt & 1;
+      if (!(ok = gemm2_wait(bar_tfull(buf), (lt >> 1) & 1, abort_flag, args.status))) break;
+      ptx::tc_fence_after();
+      const uint32_t taddr = tmem_base + buf * GEMM2_BN + ((uint32_t)(e * 32) << 16);
+#pragma unroll 1
+      for (int c = 0; c < GEMM2_BN / 64; ++c) {
+        uint32_t v0[32], v1[32];
+        ptx::tmem_ld_32x32b_x32(taddr + c * 64, v0);
+        ptx::tmem_ld_32x32b_x32(taddr + c * 64 + 32, v1);
+        ptx::tmem_ld_wait();
+        if (c == GEMM2_BN / 64 - 1) {               // accumulator fully read: tell the leader
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_tempty(buf), 0));
+        }
+        const uint32_t sb = stage0 + (uint32_t)(c & 1) * 4096u;
+        if (lane == 0) ptx::tma_store_wait_read<1>();
+        __syncwarp();
+        const uint32_t rowaddr = sb + (uint32_t)lane * 128u;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t p0 = ptx::pack_bf16(__uint_as_float(v0[8 * j + 0]), __uint_as_float(v0[8 * j + 1]));
+          const uint32_t p1 = ptx::pack_bf16(__uint_as_float(v0[8 * j + 2]), __uint_as_float(v0[8 * j + 3]));
+          const uint32_t p2 = ptx::pack_bf16(__uint_as_float(v0[8 * j + 4]), __uint_as_float(v0[8 * j + 5]));
+          const uint32_t p3 = ptx::pack_bf16(__uint_as_float(v0[8 * j + 6]), __uint_as_float(v0[8 * j + 7]));
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(rowaddr + (uint32_t)((j ^ (lane & 7)) << 4)),
+                       "r"(p0), "r"(p1), "r"(p2), "r"(p3) : "memory");
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t p0 = ptx::pack_bf16(__uint_as_float(v1[8 * j + 0]), __uint_as_float(v1[8 * j + 1]));
+          const uint32_t p1 = ptx::pack_bf16(__uint_as_float(v1[8 * j + 2]), __uint_as_float(v1[8 * j + 3]));
+          const uint32_t p2 = ptx::pack_bf16(__uint_as_float(v1[8 * j + 4]), __uint_as_float(v1[8 * j + 5]));
+          const uint32_t p3 = ptx::pack_bf16(__uint_as_float(v1[8 * j + 6]), __uint_as_float(v1[8 * j + 7]));
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(rowaddr + (uint32_t)(((4 + j) ^ (lane & 7)) << 4)),
+                       "r"(p0), "r"(p1), "r"(p2), "r"(p3) : "memory");
+        }
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0 && m0 < args.M && n0 + c * 64 < args.N) {
+          ptx::tma_store_2d(&tmOut, sb, n0 + c * 64, m0);
+          ptx::tma_store_commit();
+        }
+      }
+    }
+    if (lane == 0) ptx::tma_store_wait<0>();
+    __syncwarp();
+  } else {
+    // ============================ low-rank operand builder (both CTAs, own rows) ============================
+    const int rloc = (warp - 6) * 32 + lane;        // row inside this CTA's half of the pair tile
+    uint32_t it = 0, go_phase = 0;
+    bool ok = true;
+    for (int unit = pair; unit < n_units && ok; unit += n_pairs) {
+      const int mt = unit % args.n_mtiles;
+      const int G = tile_groups(mt);
+      const int LC = (G * R + 63) / 64;
+      it += KB;
+      if (LC == 0) continue;
+      const int row = mt * GEMM2_BM + (int)rank * 128 + rloc;
+      const int grp = row < args.M ? args.row_grp[row] : -1;
+      uint32_t ub[R / 2];
+      if (grp >= 0) {
+        const float sc = args.scale ? args.scale[args.row_adapter[row]] : 1.0f;
+        const float4* src = reinterpret_cast<const float4*>(args.P + (size_t)row * R);
+#pragma unroll
+        for (int i = 0; i < R / 4; ++i) {
+          const float4 f = src[i];
+          ub[2 * i] = ptx::pack_bf16(f.x * sc, f.y * sc);
+          ub[2 * i + 1] = ptx::pack_bf16(f.z * sc, f.w * sc);
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < R / 2; ++i) ub[i] = 0;
+      }
+      for (int lc = 0; lc < LC; ++lc, ++it) {
+        const int s = it % S;
+        if (!(ok = gemm_wait(bar_go(s), (go_phase >> s) & 1, abort_flag, args.status))) break;
+        go_phase ^= 1u << s;
+        const uint32_t rowaddr = sA0 + s * GEMM2_STAGE_BYTES + (uint32_t)rloc * 128u;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          uint32_t w0 = 0, w1 = 0, w2 = 0, w3 = 0;
+          if constexpr (R <= 64) {
+            const int gg = lc * GPC + (c * 8) / R;
+            constexpr int rr = R;
+            const int o = ((c * 8) % rr) / 2;
+            if (grp == gg) { w0 = ub[o]; w1 = ub[o + 1]; w2 = ub[o + 2]; w3 = ub[o + 3]; }
+          } else {
+            if (grp == (lc >> 1)) {
+              if (lc & 1) { w0 = ub[R / 4 + c * 4]; w1 = ub[R / 4 + c * 4 + 1]; w2 = ub[R / 4 + c * 4 + 2]; w3 = ub[R / 4 + c * 4 + 3]; }
+              else        { w0 = ub[c * 4]; w1 = ub[c * 4 + 1]; w2 = ub[c * 4 + 2]; w3 = ub[c * 4 + 3]; }
+            }
+          }
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(rowaddr + (uint32_t)((c ^ (rloc & 7)) << 4)),
+                       "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+        }
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_lora(s), 0));
+      }
+    }
+  }
+
+  // ============================ common exit ============================
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync_all();          // the peer is done with this CTA's shared memory and barriers
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem2_dealloc(tmem_base, GEMM_TMEM_COLS);
+  }
+}
+
+}  // namespace mlora

@@ -14,6 +14,7 @@
 #include "mlora.h"
 #include "plan.h"
 #include "gemm_tcgen05.cuh"
+#include "gemm2_tcgen05.cuh"
 #include "simt.cuh"
 #include "skinny.cuh"
 
@@ -36,6 +37,7 @@ struct mlora_ctx {
   int64_t launches = 0;
   int32_t gemm_path = 0;
   int32_t shrink_path = 0;           // 0: streaming kernel for rank <= 32; 1: per-item kernel for every rank
+  int32_t gemm_pairs = 1;            // 1: two-SM (CTA pair) tensor-core kernel; 0: one-SM kernel
   EncodeTiledFn encode = nullptr;
   // optional per-launch timing
   std::vector<cudaEvent_t> ev_start, ev_stop;
@@ -54,6 +56,9 @@ struct DevRowSpace {
   const int32_t* row_grp = nullptr;
   const int32_t* tile_grp_off = nullptr;
   const int32_t* grp_adapter = nullptr;
+  const int32_t* row_grp2 = nullptr;
+  const int32_t* tile2_grp_off = nullptr;
+  const int32_t* grp2_adapter = nullptr;
   const int32_t* item_rows = nullptr;
   const int32_t* item_save = nullptr;
   const int32_t* item_start = nullptr;
@@ -161,6 +166,21 @@ void launch_pdl(bool overlap, void (*kern)(KArgs...), dim3 grid, dim3 block, siz
   cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 
+// Same, for a kernel whose CTAs come in clusters of two.
+template <typename... KArgs, typename... Args>
+void launch_pdl_pairs(bool overlap, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                      Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = overlap ? 1 : 0;
+  at[1].id = cudaLaunchAttributeClusterDimension;
+  at[1].val.clusterDim.x = 2; at[1].val.clusterDim.y = 1; at[1].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 2;
+  cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
 // ---- bf16 launches ------------------------------------------------------------------------
 template <int RB, int MT, int WARPS, int MIN_CTAS>
 void launch_shrink_rb(bool overlap, const ShrinkArgs& a, int n_items, int ksplit, cudaStream_t st) {
@@ -260,6 +280,44 @@ mlora_status_t launch_gemm_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUten
   return scope.done();
 }
 
+// Two-SM kernel: grid = 2 x (number of CTA pairs that can be resident at once).
+template <int R, bool W_KMAJOR>
+mlora_status_t launch_gemm2_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUtensorMap& tW, const CUtensorMap& tL,
+                              const CUtensorMap& tOut, const GemmArgs& g, cudaStream_t st) {
+  static int max_pairs = 0;         // per instantiation
+  auto kern = gemm2_lora_kernel<R, W_KMAJOR>;
+  if (max_pairs == 0) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM2_SMEM_BYTES) != cudaSuccess)
+      return MLORA_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * ctx->sm_count); cfg.blockDim = dim3(GEMM_THREADS); cfg.dynamicSmemBytes = GEMM2_SMEM_BYTES;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) { cudaGetLastError(); return MLORA_ERR_CUDA; }
+    max_pairs = n;
+  }
+  const int pairs = g.n_units < max_pairs ? g.n_units : max_pairs;
+  LaunchScope scope(ctx, st, W_KMAJOR ? KIND_GEMM_BWD : KIND_GEMM_FWD);
+  launch_pdl_pairs(scope.slot < 0, kern, dim3(2 * pairs), dim3(GEMM_THREADS), GEMM2_SMEM_BYTES, st, tIn, tW, tL, tOut, g);
+  return scope.done();
+}
+
+template <bool W_KMAJOR>
+mlora_status_t launch_gemm2(mlora_ctx* ctx, int R, const CUtensorMap& tIn, const CUtensorMap& tW, const CUtensorMap& tL,
+                            const CUtensorMap& tOut, const GemmArgs& g, cudaStream_t st) {
+  switch (R) {
+    case 8: return launch_gemm2_r<8, W_KMAJOR>(ctx, tIn, tW, tL, tOut, g, st);
+    case 16: return launch_gemm2_r<16, W_KMAJOR>(ctx, tIn, tW, tL, tOut, g, st);
+    case 32: return launch_gemm2_r<32, W_KMAJOR>(ctx, tIn, tW, tL, tOut, g, st);
+    case 64: return launch_gemm2_r<64, W_KMAJOR>(ctx, tIn, tW, tL, tOut, g, st);
+    case 128: return launch_gemm2_r<128, W_KMAJOR>(ctx, tIn, tW, tL, tOut, g, st);
+    default: return MLORA_ERR_UNSUPPORTED;
+  }
+}
+
 template <bool W_KMAJOR>
 mlora_status_t launch_gemm(mlora_ctx* ctx, int R, const CUtensorMap& tIn, const CUtensorMap& tW, const CUtensorMap& tL,
                            const CUtensorMap& tOut, const GemmArgs& g, cudaStream_t st) {
@@ -292,6 +350,16 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
   if ((s = make_tmap_bf16(ctx, &tOut, Out, N, M, ld_out, 64, 32)) != MLORA_OK) return s;
   GemmArgs g;
   g.M = M; g.N = N; g.K = K;
+  if (ctx->gemm_pairs) {            // two-SM kernel: 256-row tiles and their group tables
+    g.n_mtiles = (M + GEMM2_BM - 1) / GEMM2_BM;
+    g.n_ntiles = (N + GEMM2_BN - 1) / GEMM2_BN;
+    g.n_full = g.n_units = g.n_mtiles * g.n_ntiles;
+    g.lora_enabled = hs.grp2_adapter.empty() ? 0 : 1;
+    g.row_grp = ds.row_grp2; g.row_adapter = ds.row_adapter;
+    g.tile_grp_off = ds.tile2_grp_off; g.grp_adapter = ds.grp2_adapter;
+    g.P = P; g.scale = scale; g.status = ctx->status_dev;
+    return launch_gemm2<W_KMAJOR>(ctx, R, tIn, tW, tL, tOut, g, st);
+  }
   g.n_mtiles = (M + GEMM_BM - 1) / GEMM_BM;
   g.n_ntiles = (N + GEMM_BN - 1) / GEMM_BN;
   // The last wave of tiles usually fills only part of the SMs; when it fills at most half, its
@@ -546,11 +614,12 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
     if (cudaSetDevice(ctx->device) != cudaSuccess) { delete p; return MLORA_ERR_CUDA; }
     BlobBuilder b;
     const HostPlan& h = p->h;
-    size_t o[40]; int n = 0;
+    size_t o[48]; int n = 0;
     const RowSpace* rs[2] = {&h.fwd, &h.bwd};
     for (int i = 0; i < 2; ++i) {
       o[n++] = b.add(rs[i]->row_adapter); o[n++] = b.add(rs[i]->row_save); o[n++] = b.add(rs[i]->row_grp);
       o[n++] = b.add(rs[i]->tile_grp_off); o[n++] = b.add(rs[i]->grp_adapter); o[n++] = b.add(rs[i]->item_rows);
+      o[n++] = b.add(rs[i]->row_grp2); o[n++] = b.add(rs[i]->tile2_grp_off); o[n++] = b.add(rs[i]->grp2_adapter);
       o[n++] = b.add(rs[i]->item_save); o[n++] = b.add(rs[i]->item_start); o[n++] = b.add(rs[i]->item_nrows); o[n++] = b.add(rs[i]->item_adapter);
     }
     o[n++] = b.add(h.slot_chunk_off); o[n++] = b.add(h.chunk_row0); o[n++] = b.add(h.chunk_nrows);
@@ -564,6 +633,7 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
     for (int i = 0; i < 2; ++i) {
       ds[i]->row_adapter = p->blob + o[n++]; ds[i]->row_save = p->blob + o[n++]; ds[i]->row_grp = p->blob + o[n++];
       ds[i]->tile_grp_off = p->blob + o[n++]; ds[i]->grp_adapter = p->blob + o[n++]; ds[i]->item_rows = p->blob + o[n++];
+      ds[i]->row_grp2 = p->blob + o[n++]; ds[i]->tile2_grp_off = p->blob + o[n++]; ds[i]->grp2_adapter = p->blob + o[n++];
       ds[i]->item_save = p->blob + o[n++]; ds[i]->item_start = p->blob + o[n++]; ds[i]->item_nrows = p->blob + o[n++]; ds[i]->item_adapter = p->blob + o[n++];
     }
     p->bwd.row_save = nullptr;       // the compact space has no save offsets
@@ -706,9 +776,10 @@ mlora_status_t mlora_poll_status(mlora_ctx* ctx, void* cuda_stream) {
 int64_t mlora_launch_count(const mlora_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path) {
-  if (!ctx || path < 0 || path > 2) return MLORA_ERR_INVALID_ARG;
+  if (!ctx || path < 0 || path > 3) return MLORA_ERR_INVALID_ARG;
   ctx->gemm_path = path == 1 ? 1 : 0;
   ctx->shrink_path = path == 2 ? 1 : 0;
+  ctx->gemm_pairs = path == 3 ? 0 : 1;
   return MLORA_OK;
 }
 

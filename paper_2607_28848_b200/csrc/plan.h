@@ -10,7 +10,8 @@
 
 namespace mlora {
 
-constexpr int kTileRows = 128;     // rows per tensor-core tile (UMMA M)
+constexpr int kTileRows = 128;     // rows per tensor-core tile of the one-SM kernel (UMMA M = 128)
+constexpr int kPairTileRows = 256; // rows per tile of the two-SM kernel (a CTA pair, UMMA M = 256)
 constexpr int kItemRows = 32;      // most rows in one shrink work item (two mma.sync row blocks)
 constexpr int kChunkRows = 16;     // rows per gradient chunk (one mma.sync contraction step)
 constexpr int kMaxRank = 128;
@@ -25,6 +26,8 @@ struct RowSpace {
   std::vector<int32_t> row_grp;        // [n_rows]
   std::vector<int32_t> tile_grp_off;   // [n_tiles + 1]
   std::vector<int32_t> grp_adapter;    // [tile_grp_off.back()]
+  // the same three tables for tiles of kPairTileRows rows
+  std::vector<int32_t> row_grp2, tile2_grp_off, grp2_adapter;
   // Shrink items: the rows that have an adapter, gathered BY ADAPTER (ascending adapter id, rows
   // ascending inside an adapter) and cut into items of <= kItemRows rows.  Rows of an item need
   // not be adjacent in the batch: decode rows that share an adapter are processed together, so an
@@ -48,25 +51,33 @@ struct HostPlan {
   std::vector<int32_t> chunk_row0, chunk_nrows;
 };
 
-inline void build_tiles_and_items(RowSpace& rs) {
-  const int32_t n = rs.n_rows;
-  rs.row_grp.assign(n, -1);
-  rs.tile_grp_off.assign(1, 0);
-  rs.grp_adapter.clear();
-  for (int32_t t0 = 0; t0 < n; t0 += kTileRows) {
-    const int32_t t1 = t0 + kTileRows < n ? t0 + kTileRows : n;
-    const int32_t base = (int32_t)rs.grp_adapter.size();
+inline void build_tile_groups(const std::vector<int32_t>& row_adapter, int32_t tile_rows,
+                              std::vector<int32_t>& row_grp, std::vector<int32_t>& tile_grp_off,
+                              std::vector<int32_t>& grp_adapter) {
+  const int32_t n = (int32_t)row_adapter.size();
+  row_grp.assign(n, -1);
+  tile_grp_off.assign(1, 0);
+  grp_adapter.clear();
+  for (int32_t t0 = 0; t0 < n; t0 += tile_rows) {
+    const int32_t t1 = t0 + tile_rows < n ? t0 + tile_rows : n;
+    const int32_t base = (int32_t)grp_adapter.size();
     for (int32_t t = t0; t < t1; ++t) {
-      const int32_t a = rs.row_adapter[t];
+      const int32_t a = row_adapter[t];
       if (a < 0) continue;
       int32_t g = -1;
-      for (int32_t i = base; i < (int32_t)rs.grp_adapter.size(); ++i)
-        if (rs.grp_adapter[i] == a) { g = i - base; break; }
-      if (g < 0) { g = (int32_t)rs.grp_adapter.size() - base; rs.grp_adapter.push_back(a); }
-      rs.row_grp[t] = g;
+      for (int32_t i = base; i < (int32_t)grp_adapter.size(); ++i)
+        if (grp_adapter[i] == a) { g = i - base; break; }
+      if (g < 0) { g = (int32_t)grp_adapter.size() - base; grp_adapter.push_back(a); }
+      row_grp[t] = g;
     }
-    rs.tile_grp_off.push_back((int32_t)rs.grp_adapter.size());
+    tile_grp_off.push_back((int32_t)grp_adapter.size());
   }
+}
+
+inline void build_tiles_and_items(RowSpace& rs) {
+  const int32_t n = rs.n_rows;
+  build_tile_groups(rs.row_adapter, kTileRows, rs.row_grp, rs.tile_grp_off, rs.grp_adapter);
+  build_tile_groups(rs.row_adapter, kPairTileRows, rs.row_grp2, rs.tile2_grp_off, rs.grp2_adapter);
   rs.item_rows.clear(); rs.item_start.clear(); rs.item_nrows.clear(); rs.item_adapter.clear();
   int32_t max_adapter = -1;
   for (int32_t t = 0; t < n; ++t) max_adapter = rs.row_adapter[t] > max_adapter ? rs.row_adapter[t] : max_adapter;

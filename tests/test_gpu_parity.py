@@ -77,7 +77,7 @@ def test_cfg1_tiny_fp32(sess):
     run_and_check(sess, w, synth.make_tensors(w))
 
 
-@pytest.mark.parametrize("path", [0, 1, 2])
+@pytest.mark.parametrize("path", [0, 1, 2, 3])
 def test_bf16_ragged_multi_tile(sess, path):
     w = synth.random_workload(5, 256, 512, 16, 6, 389, max_seg=150)
     run_and_check(sess, w, synth.make_tensors(w), path=path)
@@ -92,6 +92,13 @@ def test_fp32_ragged(sess):
 def test_rank_sweep(sess, rank):
     w = synth.random_workload(10 + rank, 320, 448, rank, 7, 300, max_seg=90)
     run_and_check(sess, w, synth.make_tensors(w))
+
+
+@pytest.mark.parametrize("rank", [8, 128])
+def test_one_sm_gemm_kernel(sess, rank):
+    """The one-SM tensor-core kernel (kernel variant 3) on ranks at both ends."""
+    w = synth.random_workload(40 + rank, 320, 448, rank, 7, 300, max_seg=90)
+    run_and_check(sess, w, synth.make_tensors(w), path=3)
 
 
 @pytest.mark.parametrize("rank", [8, 32])
