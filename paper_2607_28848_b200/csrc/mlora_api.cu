@@ -64,6 +64,7 @@ struct DevRowSpace {
   const int32_t* item_start = nullptr;
   const int32_t* item_nrows = nullptr;
   const int32_t* item_adapter = nullptr;
+  const int32_t* item_contig = nullptr;
 };
 
 struct mlora_plan {
@@ -93,13 +94,13 @@ struct BlobBuilder {
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 mlora_status_t make_tmap_bf16(const mlora_ctx* ctx, CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer,
-                              uint64_t row_stride_elems, uint32_t box_inner, uint32_t box_outer) {
+                              uint64_t row_stride_elems, uint32_t box_inner, uint32_t box_outer, bool swizzle = true) {
   cuuint64_t dims[2] = {inner, outer};
   cuuint64_t strides[1] = {row_stride_elems * 2};
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = ctx->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? MLORA_OK : MLORA_ERR_CUDA;
 }
@@ -196,12 +197,19 @@ int shrink_ksplit(const mlora_ctx* ctx, int n_items, int D) {
   k = k < kMaxKSplit ? k : kMaxKSplit;
   return k < 1 ? 1 : k;
 }
-template <int RB, int STAGES>
-mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, cudaStream_t st) {
+template <int RB, int STAGES, int CHUNK>
+mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, const int32_t* item_contig, int n_rows,
+                                    int n_adapters, cudaStream_t st) {
   constexpr int R = RB * 8;
-  constexpr size_t smem = (size_t)STAGES * (32 + R) * STREAM_PITCH + (size_t)(RB >= 4 ? 4 : 8) * 32 * (R + 1) * 4;
+  constexpr size_t xrow = 32 * (CHUNK * 128 + 16), xtile = (size_t)(CHUNK / 4) * 32 * 512;
+  constexpr size_t xbytes = ((xrow > xtile ? xrow : xtile) + 127) / 128 * 128;
+  constexpr size_t smem = (size_t)STAGES * (xbytes + (size_t)(CHUNK / 4) * R * 512) + (size_t)(RB >= 4 ? 4 : 8) * 32 * (R + 1) * 4;
+  CUtensorMap tIn, tP;
+  mlora_status_t ms;
+  if ((ms = make_tmap_bf16(ctx, &tIn, a.In, a.D, n_rows, a.ld_in, 256, 32, false)) != MLORA_OK) return ms;
+  if ((ms = make_tmap_bf16(ctx, &tP, a.P_all, a.D, (uint64_t)n_adapters * R, a.D, 256, R, false)) != MLORA_OK) return ms;
   static bool attr_set = false;
-  auto kern = shrink_stream_kernel<RB, STAGES>;
+  auto kern = shrink_stream_kernel<RB, STAGES, CHUNK>;
   if (!attr_set) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return MLORA_ERR_CUDA;
     attr_set = true;
@@ -211,7 +219,7 @@ mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, c
   sa.s.partial = ctx->ws_partial;
   sa.s.counters = ctx->ws_counters;
   sa.n_items = n_items;
-  sa.chunks_per_item = (a.D / 64 + STREAM_CHUNK - 1) / STREAM_CHUNK;
+  sa.chunks_per_item = (a.D / 64 + CHUNK - 1) / CHUNK;
   sa.n_units = n_items * sa.chunks_per_item;
   int grid = sa.n_units < ctx->sm_count ? sa.n_units : ctx->sm_count;
   sa.units_per_cta = (sa.n_units + grid - 1) / grid;
@@ -219,16 +227,18 @@ mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, c
   if (2 * (int64_t)grid > ctx->ws_partial_items || n_items > ctx->ws_counter_items) return MLORA_ERR_INVALID_ARG;
   LaunchScope scope(ctx, st, KIND_SHRINK);
   sa.status = ctx->status_dev;
-  launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(STREAM_THREADS), smem, st, sa);
+  sa.item_contig = item_contig;
+  launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(STREAM_THREADS), smem, st, tIn, tP, sa);
   return scope.done();
 }
 
-mlora_status_t launch_shrink(mlora_ctx* ctx, int R, ShrinkArgs a, int n_items, cudaStream_t st) {
+mlora_status_t launch_shrink(mlora_ctx* ctx, int R, ShrinkArgs a, int n_items, const int32_t* item_contig, int n_rows,
+                             int n_adapters, cudaStream_t st) {
   if (n_items <= 0) return MLORA_OK;
   if (ctx->shrink_path == 0) {
-    if (R == 8) return launch_shrink_stream<1, 4>(ctx, a, n_items, st);
-    if (R == 16) return launch_shrink_stream<2, 4>(ctx, a, n_items, st);
-    if (R == 32) return launch_shrink_stream<4, 3>(ctx, a, n_items, st);
+    if (R == 8) return launch_shrink_stream<1, 2, 16>(ctx, a, n_items, item_contig, n_rows, n_adapters, st);
+    if (R == 16) return launch_shrink_stream<2, 2, 16>(ctx, a, n_items, item_contig, n_rows, n_adapters, st);
+    if (R == 32) return launch_shrink_stream<4, 3, 8>(ctx, a, n_items, item_contig, n_rows, n_adapters, st);
   }
   const int ksplit = shrink_ksplit(ctx, n_items, a.D);
   a.partial = ctx->ws_partial;
@@ -614,13 +624,13 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
     if (cudaSetDevice(ctx->device) != cudaSuccess) { delete p; return MLORA_ERR_CUDA; }
     BlobBuilder b;
     const HostPlan& h = p->h;
-    size_t o[48]; int n = 0;
+    size_t o[56]; int n = 0;
     const RowSpace* rs[2] = {&h.fwd, &h.bwd};
     for (int i = 0; i < 2; ++i) {
       o[n++] = b.add(rs[i]->row_adapter); o[n++] = b.add(rs[i]->row_save); o[n++] = b.add(rs[i]->row_grp);
       o[n++] = b.add(rs[i]->tile_grp_off); o[n++] = b.add(rs[i]->grp_adapter); o[n++] = b.add(rs[i]->item_rows);
       o[n++] = b.add(rs[i]->row_grp2); o[n++] = b.add(rs[i]->tile2_grp_off); o[n++] = b.add(rs[i]->grp2_adapter);
-      o[n++] = b.add(rs[i]->item_save); o[n++] = b.add(rs[i]->item_start); o[n++] = b.add(rs[i]->item_nrows); o[n++] = b.add(rs[i]->item_adapter);
+      o[n++] = b.add(rs[i]->item_save); o[n++] = b.add(rs[i]->item_start); o[n++] = b.add(rs[i]->item_contig); o[n++] = b.add(rs[i]->item_nrows); o[n++] = b.add(rs[i]->item_adapter);
     }
     o[n++] = b.add(h.slot_chunk_off); o[n++] = b.add(h.chunk_row0); o[n++] = b.add(h.chunk_nrows);
     o[n++] = b.add(h.ft_adapters);
@@ -634,7 +644,7 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
       ds[i]->row_adapter = p->blob + o[n++]; ds[i]->row_save = p->blob + o[n++]; ds[i]->row_grp = p->blob + o[n++];
       ds[i]->tile_grp_off = p->blob + o[n++]; ds[i]->grp_adapter = p->blob + o[n++]; ds[i]->item_rows = p->blob + o[n++];
       ds[i]->row_grp2 = p->blob + o[n++]; ds[i]->tile2_grp_off = p->blob + o[n++]; ds[i]->grp2_adapter = p->blob + o[n++];
-      ds[i]->item_save = p->blob + o[n++]; ds[i]->item_start = p->blob + o[n++]; ds[i]->item_nrows = p->blob + o[n++]; ds[i]->item_adapter = p->blob + o[n++];
+      ds[i]->item_save = p->blob + o[n++]; ds[i]->item_start = p->blob + o[n++]; ds[i]->item_contig = p->blob + o[n++]; ds[i]->item_nrows = p->blob + o[n++]; ds[i]->item_adapter = p->blob + o[n++];
     }
     p->bwd.row_save = nullptr;       // the compact space has no save offsets
     p->slot_chunk_off = p->blob + o[n++]; p->chunk_row0 = p->blob + o[n++]; p->chunk_nrows = p->blob + o[n++];
@@ -716,7 +726,8 @@ mlora_status_t mlora_mixed_forward(mlora_ctx* ctx, const mlora_layer_t* L, const
   sa.item_rows = p->fwd.item_rows; sa.item_start = p->fwd.item_start; sa.item_nrows = p->fwd.item_nrows;
   sa.item_adapter = p->fwd.item_adapter; sa.item_save = p->fwd.item_save;
   sa.x_save = (__nv_bfloat16*)x_save; sa.u_save = u_save; sa.save_base = save_row_base;
-  if ((s = launch_shrink(ctx, L->rank, sa, h.fwd.n_items(), st)) != MLORA_OK) return s;
+  if ((s = launch_shrink(ctx, L->rank, sa, h.fwd.n_items(), p->fwd.item_contig, h.n_rows, L->n_adapters, st)) != MLORA_OK)
+    return s;
   return gemm_bf16<false>(ctx, L, h.fwd, p->fwd, X, ldx, Y, ldy, L->B_all, ctx->ws_p, L->scale, h.n_rows, L->d_out,
                           L->d_in, st);
 }
@@ -745,7 +756,8 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   sa.P_all = (const __nv_bfloat16*)L->B_all; sa.scale = L->scale; sa.Out = ctx->ws_p;
   sa.item_rows = p->bwd.item_rows; sa.item_start = p->bwd.item_start; sa.item_nrows = p->bwd.item_nrows;
   sa.item_adapter = p->bwd.item_adapter; sa.item_save = nullptr; sa.x_save = nullptr; sa.u_save = nullptr; sa.save_base = 0;
-  if ((s = launch_shrink(ctx, L->rank, sa, h.bwd.n_items(), st)) != MLORA_OK) return s;
+  if ((s = launch_shrink(ctx, L->rank, sa, h.bwd.n_items(), p->bwd.item_contig, h.ft_rows, L->n_adapters, st)) != MLORA_OK)
+    return s;
 
   GradArgs ga;                       // dB = (s U)^T dY
   ga.P = u_save; ga.R = L->rank; ga.scale = L->scale; ga.Q = (const __nv_bfloat16*)dY; ga.ldq = lddy; ga.D = L->d_out;

@@ -35,6 +35,7 @@ struct RowSpace {
   std::vector<int32_t> item_rows;      // [rows with an adapter] row ids, grouped by adapter
   std::vector<int32_t> item_save;      // parallel to item_rows: save offset of that row or -1
   std::vector<int32_t> item_start, item_nrows, item_adapter;
+  std::vector<int32_t> item_contig;    // 1: the item's rows are consecutive rows of the batch
   int32_t n_tiles() const { return (n_rows + kTileRows - 1) / kTileRows; }
   int32_t n_items() const { return (int32_t)item_start.size(); }
 };
@@ -78,7 +79,7 @@ inline void build_tiles_and_items(RowSpace& rs) {
   const int32_t n = rs.n_rows;
   build_tile_groups(rs.row_adapter, kTileRows, rs.row_grp, rs.tile_grp_off, rs.grp_adapter);
   build_tile_groups(rs.row_adapter, kPairTileRows, rs.row_grp2, rs.tile2_grp_off, rs.grp2_adapter);
-  rs.item_rows.clear(); rs.item_start.clear(); rs.item_nrows.clear(); rs.item_adapter.clear();
+  rs.item_rows.clear(); rs.item_start.clear(); rs.item_nrows.clear(); rs.item_adapter.clear(); rs.item_contig.clear();
   int32_t max_adapter = -1;
   for (int32_t t = 0; t < n; ++t) max_adapter = rs.row_adapter[t] > max_adapter ? rs.row_adapter[t] : max_adapter;
   std::vector<int32_t> count(max_adapter + 2, 0);
@@ -99,6 +100,10 @@ inline void build_tiles_and_items(RowSpace& rs) {
       rs.item_adapter.push_back(a);
     }
   }
+  rs.item_contig.assign(rs.item_start.size(), 1);
+  for (size_t it = 0; it < rs.item_start.size(); ++it)
+    for (int32_t i = 1; i < rs.item_nrows[it]; ++i)
+      if (rs.item_rows[rs.item_start[it] + i] != rs.item_rows[rs.item_start[it]] + i) { rs.item_contig[it] = 0; break; }
 }
 
 // Validates the table and fills `p`.  Returns MLORA_OK or the error the header documents.

@@ -188,27 +188,31 @@ shrink_kernel(const ShrinkArgs a) {
 // Streaming shrink for ranks up to 32: a persistent grid (one CTA per SM) walks the flattened list
 // of work units (item, chunk of 8 K-blocks = 512 elements) in equal contiguous ranges, so every SM
 // streams the same number of bytes in one wave.  A producer warp moves each unit into a
-// STAGES-deep shared-memory ring with bulk asynchronous copies (one 1 KiB copy per row of the
-// item and per row of the adapter, completion counted on an mbarrier), which keeps ~150 KB per SM
-// in flight at almost no instruction cost.  Eight consumer warps each take one K-block of the
-// unit: fragments come out of shared memory with conflict-free 16-byte loads (row pitch 1040 B),
-// feed mma.sync, and the rows of In are stored on to x_save for fine-tuning rows.  Accumulators
+// STAGES-deep shared-memory ring, completion counted on an mbarrier: tensor-map tiles of
+// 256 elements x 32 rows (16 KiB per instruction) for the adapter rows and for items whose rows
+// are adjacent in memory (prefill and fine-tune segments), one bulk copy per row only for items
+// gathered from scattered rows (decode rows) - the copy engine's cost is per instruction, not per
+// byte.  Eight consumer warps share the K-blocks of the unit: fragments come out of shared memory
+// with 16-byte loads, feed mma.sync, and the rows of In are stored on to x_save for fine-tuning
+// rows.  Accumulators
 // persist across the chunks of an item and are flushed when the item ends.  An item whose chunks
 // were shared by several CTAs is finished by whichever of them arrives last, adding the partials
 // in CTA order (a fixed order).  Every mbarrier wait is bounded.
 constexpr int STREAM_WARPS = 8;      // consumer warps; warp 8 is the producer
 constexpr int STREAM_THREADS = (STREAM_WARPS + 1) * 32;
-constexpr int STREAM_CHUNK = 8;      // K-blocks (of 64) per unit: one per consumer warp
-constexpr uint32_t STREAM_PITCH = 1040;   // bytes between rows of a stage (1 KiB + 16: no bank conflicts)
+// A unit covers CHUNK K-blocks of 64 (a template parameter: 8 or 16).  Tile layout of a stage:
+// CHUNK / 4 boxes of [rows][256 elements]; row-copy layout (gathered items): rows CHUNK * 128 + 16
+// bytes apart, so that fragment loads hit distinct banks.
 constexpr uint32_t STREAM_SPIN_LIMIT = 1u << 22;
 
 struct StreamArgs {
   ShrinkArgs s;
   int32_t n_items;
-  int32_t chunks_per_item;   // ceil(D / 512)
+  int32_t chunks_per_item;   // ceil(D / (64 CHUNK))
   int32_t n_units;           // n_items * chunks_per_item
   int32_t units_per_cta;     // ceil(n_units / gridDim.x)
   int32_t* status;           // device status word
+  const int32_t* item_contig;  // [n_items] 1: the item's rows are consecutive rows of In
 };
 
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -230,12 +234,18 @@ __device__ __forceinline__ bool stream_wait(uint32_t bar, uint32_t parity, volat
   return false;
 }
 
-template <int RB, int STAGES>
+template <int RB, int STAGES, int CHUNK>
 __global__ void __launch_bounds__(STREAM_THREADS, 1)
-shrink_stream_kernel(const StreamArgs sa) {
+shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ CUtensorMap tmP,
+                     const StreamArgs sa) {
   constexpr int R = RB * 8;
-  constexpr int ROWS = 32 + R;                            // rows of a stage: the item's, then the adapter's
-  constexpr uint32_t STAGE_BYTES = ROWS * STREAM_PITCH;
+  constexpr int NBOX = CHUNK / 4;                          // 256-element boxes per unit
+  constexpr uint32_t STREAM_PITCH = CHUNK * 128 + 16;     // row-copy layout
+  constexpr uint32_t XBOX_BYTES = 32 * 512;               // tile layout: [32 rows][256 elements]
+  constexpr uint32_t X_BYTES = ((32 * STREAM_PITCH > NBOX * XBOX_BYTES ? 32 * STREAM_PITCH : NBOX * XBOX_BYTES) + 127) / 128 * 128;
+  constexpr uint32_t PBOX_BYTES = R * 512;                // adapter rows: [R rows][256 elements] per box
+  constexpr uint32_t STAGE_BYTES = X_BYTES + NBOX * PBOX_BYTES;
+  static_assert(CHUNK % STREAM_WARPS == 0, "each consumer warp takes CHUNK / 8 K-blocks of a unit");
   constexpr int RW = RB >= 4 ? 4 : 8;                     // reduction buffers (rank 32: two rounds of 4 warps)
   extern __shared__ __align__(128) uint8_t stream_smem[];
   float (*red)[32][R + 1] = reinterpret_cast<float (*)[32][R + 1]>(stream_smem + STAGES * STAGE_BYTES);
@@ -269,16 +279,20 @@ shrink_stream_kernel(const StreamArgs sa) {
   if (warp == STREAM_WARPS) {
     // ======================= producer =======================
     int item = u_begin / KC, kc = u_begin % KC;
-    int cur = -1, nrows = 0;
-    const __nv_bfloat16* src0 = nullptr;     // lane l moves stage row l ...
-    const __nv_bfloat16* src1 = nullptr;     // ... and stage row l + 32 (adapter row l), if l < R
+    int cur = -1, nrows = 0, contig = 0, row0 = 0, prow0 = 0;
+    const __nv_bfloat16* src0 = nullptr;     // gathered items: lane l copies the item's row l
     auto set_item = [&](int it) {
       cur = it;
       nrows = a.item_nrows[it];
-      src0 = lane < nrows ? a.In + (size_t)a.item_rows[a.item_start[it] + lane] * a.ld_in : nullptr;
-      src1 = lane < R ? a.P_all + ((size_t)a.item_adapter[it] * R + lane) * a.D : nullptr;
+      contig = sa.item_contig[it];
+      const int32_t* rows = a.item_rows + a.item_start[it];
+      row0 = rows[0];
+      src0 = (!contig && lane < nrows) ? a.In + (size_t)rows[lane] * a.ld_in : nullptr;
+      prow0 = a.item_adapter[it] * R;
     };
     if (u_begin < u_end) set_item(item);
+    ptx::prefetch_tmap(&tmIn);
+    ptx::prefetch_tmap(&tmP);
     ptx::grid_dependency_wait();             // only plan tables were read so far
     ptx::grid_launch_dependents();
     bool ok = true;
@@ -288,13 +302,21 @@ shrink_stream_kernel(const StreamArgs sa) {
       if (lane == 0) ok = stream_wait(bar_empty(st), ((i / STAGES) & 1) ^ 1, abort_flag, sa.status);
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
-      const int k0 = kc * (STREAM_CHUNK * 64);
-      const uint32_t bytes = (uint32_t)min(STREAM_CHUNK * 64, a.D - k0) * 2u;
-      if (lane == 0) ptx::mbar_arrive_expect_tx(bar_full(st), (uint32_t)(nrows + R) * bytes);
+      const int k0 = kc * (CHUNK * 64);
+      const uint32_t row_bytes = (uint32_t)min(CHUNK * 64, a.D - k0) * 2u;
+      const uint32_t xbytes = contig ? NBOX * XBOX_BYTES : (uint32_t)nrows * row_bytes;
+      if (lane == 0) ptx::mbar_arrive_expect_tx(bar_full(st), xbytes + NBOX * PBOX_BYTES);
       __syncwarp();
       const uint32_t dst = ring + (uint32_t)st * STAGE_BYTES;
-      if (src0) bulk_load(dst + (uint32_t)lane * STREAM_PITCH, src0 + k0, bytes, bar_full(st));
-      if (src1) bulk_load(dst + (uint32_t)(32 + lane) * STREAM_PITCH, src1 + k0, bytes, bar_full(st));
+      // lanes 0 .. NBOX-1: one adapter tile each; lanes NBOX .. 2 NBOX-1: one tile of the item's rows
+      // (tiles reaching past the tensor's edge are zero-filled and still count their full size)
+      if (lane < NBOX) ptx::tma_load_2d(dst + X_BYTES + (uint32_t)lane * PBOX_BYTES, &tmP, k0 + lane * 256, prow0, bar_full(st));
+      if (contig) {
+        if (lane >= NBOX && lane < 2 * NBOX)
+          ptx::tma_load_2d(dst + (uint32_t)(lane - NBOX) * XBOX_BYTES, &tmIn, k0 + (lane - NBOX) * 256, row0, bar_full(st));
+      } else if (src0) {
+        bulk_load(dst + (uint32_t)lane * STREAM_PITCH, src0 + k0, row_bytes, bar_full(st));
+      }
       if (++kc == KC) { kc = 0; ++item; }
     }
   } else {
@@ -307,12 +329,11 @@ shrink_stream_kernel(const StreamArgs sa) {
       for (int i = 0; i < RB; ++i) acc[m][i][0] = acc[m][i][1] = acc[m][i][2] = acc[m][i][3] = 0.f;
 
     int item = u_begin / KC, kc = u_begin % KC;
-    int cur_item = -1, cur_nrows = 0, cur_adapter = 0;
+    int cur_item = -1, cur_nrows = 0, cur_adapter = 0, cur_contig = 0;
     const int32_t* cur_rows = nullptr;
     const int32_t* cur_saves = nullptr;
     __nv_bfloat16* sp[4] = {nullptr, nullptr, nullptr, nullptr};
-    // byte offset of this thread's pieces inside a stage row: K-block `warp`, elements 16c .. 16c+15
-    const uint32_t piece = (uint32_t)warp * 128u + (uint32_t)c * 32u;
+    // this thread's pieces of a K-block: elements 16c .. 16c+15 of the block
     ptx::grid_dependency_wait();
     bool ok = true;
 
@@ -322,6 +343,7 @@ shrink_stream_kernel(const StreamArgs sa) {
         cur_item = item;
         cur_nrows = a.item_nrows[item];
         cur_adapter = a.item_adapter[item];
+        cur_contig = sa.item_contig[item];
         cur_rows = a.item_rows + a.item_start[item];
         cur_saves = a.item_save ? a.item_save + a.item_start[item] : nullptr;
 #pragma unroll
@@ -333,25 +355,33 @@ shrink_stream_kernel(const StreamArgs sa) {
       }
       ok = stream_wait(bar_full(st), (i / STAGES) & 1, abort_flag, sa.status);
       if (!ok) break;
-      const int kb = kc * STREAM_CHUNK + warp;
-      if (kb < nkb) {
-        const uint32_t src = ring + (uint32_t)st * STAGE_BYTES + piece;
+#pragma unroll
+      for (int kk = 0; kk < CHUNK / STREAM_WARPS; ++kk) {
+        const int kb = kc * CHUNK + kk * STREAM_WARPS + warp;
+        if (kb >= nkb) continue;
+        const int kbl = kk * STREAM_WARPS + warp;            // K-block inside the unit
+        const uint32_t stage = ring + (uint32_t)st * STAGE_BYTES;
+        const uint32_t in_box = (uint32_t)(kbl & 3) * 128u + (uint32_t)c * 32u;
+        // rows of In: tile layout [box][row][512 B] or row-copy layout [row][pitch]
+        const uint32_t xsrc = cur_contig ? stage + (uint32_t)(kbl >> 2) * XBOX_BYTES + in_box
+                                         : stage + (uint32_t)kbl * 128u + (uint32_t)c * 32u;
+        const uint32_t xpitch = cur_contig ? 512u : STREAM_PITCH;
         uint4 x[4][2];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const uint32_t ra = src + (uint32_t)(g + 8 * j) * STREAM_PITCH;
+          const uint32_t ra = xsrc + (uint32_t)(g + 8 * j) * xpitch;
           x[j][0] = lds_v4(ra);
           x[j][1] = lds_v4(ra + 16);
         }
+        const uint32_t psrc = stage + X_BYTES + (uint32_t)(kbl >> 2) * PBOX_BYTES + in_box;
         uint4 p[RB][2];
 #pragma unroll
         for (int n = 0; n < RB; ++n) {
-          const uint32_t rp = src + (uint32_t)(32 + 8 * n + g) * STREAM_PITCH;
+          const uint32_t rp = psrc + (uint32_t)(8 * n + g) * 512u;
           p[n][0] = lds_v4(rp);
           p[n][1] = lds_v4(rp + 16);
         }
-        // rows past the item's end were not copied: their stale bytes only reach accumulator rows
-        // that are never written out, but keep them out of the MMA anyway
+        // rows past the item's end were not copied: keep their stale bytes out of the MMA
 #pragma unroll
         for (int j = 0; j < 4; ++j)
           if (g + 8 * j >= cur_nrows) { x[j][0] = make_uint4(0, 0, 0, 0); x[j][1] = make_uint4(0, 0, 0, 0); }
@@ -368,8 +398,6 @@ shrink_stream_kernel(const StreamArgs sa) {
               ptx::mma_bf16_16816(acc[m][n], ra[2 * s], rb[2 * s], ra[2 * s + 1], rb[2 * s + 1], rp[2 * s], rp[2 * s + 1]);
           }
         }
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(bar_empty(st));      // the stage's bytes are in registers now
         const int ko = kb * 64;
 #pragma unroll
         for (int j = 0; j < 4; ++j)
@@ -377,10 +405,9 @@ shrink_stream_kernel(const StreamArgs sa) {
             *reinterpret_cast<uint4*>(sp[j] + ko) = x[j][0];
             *reinterpret_cast<uint4*>(sp[j] + ko + 8) = x[j][1];
           }
-      } else {
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(bar_empty(st));
       }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar_empty(st));        // the stage's bytes are in registers now
 
       // ---- flush when the item (or this CTA's range) ends ----
       const bool item_ends = (kc == KC - 1) || (u == u_end - 1);
