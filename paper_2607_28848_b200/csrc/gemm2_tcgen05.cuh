@@ -33,7 +33,7 @@ constexpr int GEMM2_STAGES = 6;
 constexpr uint32_t GEMM2_A_BYTES = 128 * GEMM_BK * 2;               // 16 KiB: this CTA's rows
 constexpr uint32_t GEMM2_B_BYTES = 128 * GEMM_BK * 2;               // 16 KiB: this CTA's half of B
 constexpr uint32_t GEMM2_STAGE_BYTES = GEMM2_A_BYTES + GEMM2_B_BYTES;
-constexpr uint32_t GEMM2_SMEM_BYTES = GEMM2_STAGES * GEMM2_STAGE_BYTES + GEMM_EPI_BYTES + 512 + 1024;
+constexpr uint32_t GEMM2_SMEM_BYTES = GEMM2_STAGES * GEMM2_STAGE_BYTES + GEMM_EPI_BYTES + 512 + 1024 + 1024;
 
 namespace ptx {
 
@@ -194,51 +194,72 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
 
   if (warp == 0) {
     // ============================ TMA producer (both CTAs) ============================
-    if (lane == 0) {
-      uint32_t it = 0;
-      bool ok = true;
-      for (int unit = pair; unit < n_units && ok; unit += n_pairs) {
-        const int mt = unit % args.n_mtiles, nt = unit / args.n_mtiles;
-        const int m0 = mt * GEMM2_BM + (int)rank * 128;
-        const int nh = nt * GEMM2_BN + (int)rank * 128;     // this CTA's half of the B columns
-        for (int kb = 0; kb < KB; ++kb, ++it) {
-          const int s = it % S;
-          if (!(ok = gemm2_wait(bar_empty(s), ((it / S) & 1) ^ 1, abort_flag, args.status))) break;
-          const uint32_t a = sA0 + s * GEMM2_STAGE_BYTES, b = a + GEMM2_A_BYTES;
-          const uint32_t full = ptx::map_to_cta(bar_full(s), 0);
-          if (leader) ptx::mbar_arrive_expect_tx(bar_full(s), 2 * GEMM2_STAGE_BYTES);
-          ptx::tma2_load_2d(a, &tmIn, kb * GEMM_BK, m0, full);
-          if (W_KMAJOR) ptx::tma2_load_2d(b, &tmW, kb * GEMM_BK, nh, full);          // [N, K]: 128 rows x 64 k
-          else          ptx::tma2_load_3d(b, &tmW, 0, kb * GEMM_BK, nh >> 6, full);  // (64 n, K, N/64): 64 x 64 k x 2
-        }
-        if (!ok) break;
-        const int G = tile_groups(mt);
-        const int LC = (G * R + 63) / 64;
+    // Lane 0 waits and issues the main loads; the low-rank stages are issued by all lanes, one
+    // adapter group per lane, from a copy of the tile's adapter list in shared memory, so that
+    // the list costs one memory latency per tile rather than one per group.
+    int32_t* ga_smem = reinterpret_cast<int32_t*>(smem_gen + (sMisc - smem_base) + 64);   // 256 entries
+    uint32_t it = 0;
+    bool ok = true;
+    for (int unit = pair; unit < n_units && ok; unit += n_pairs) {
+      const int mt = unit % args.n_mtiles, nt = unit / args.n_mtiles;
+      const int m0 = mt * GEMM2_BM + (int)rank * 128;
+      const int nh = nt * GEMM2_BN + (int)rank * 128;     // this CTA's half of the B columns
+      const int G = tile_groups(mt);
+      const int LC = (G * R + 63) / 64;
+      int32_t ga_reg[8];                                  // G <= 256 adapters of the pair tile
+      {
         const int32_t* ga = args.grp_adapter + (args.lora_enabled ? args.tile_grp_off[mt] : 0);
-        for (int lc = 0; lc < LC; ++lc, ++it) {
-          const int s = it % S;
-          if (!(ok = gemm2_wait(bar_empty(s), ((it / S) & 1) ^ 1, abort_flag, args.status))) break;
-          ptx::mbar_arrive(bar_go(s));               // hand the free slot to this CTA's builders
-          const uint32_t b = sA0 + s * GEMM2_STAGE_BYTES + GEMM2_A_BYTES;
-          const uint32_t full = ptx::map_to_cta(bar_full(s), 0);
-          if (R <= 64) {
-            const int g0 = lc * GPC;
-            const int ng = G - g0 < GPC ? G - g0 : GPC;
-            const int ngl = (R == 8 && (ng & 1)) ? ng + 1 : ng;   // rank 8: pad a half-filled MMA step
-            if (leader) ptx::mbar_arrive_expect_tx(bar_full(s), 2u * (uint32_t)ngl * R * 128u * 2u);
-            for (int i = 0; i < ngl; ++i) {
-              const int adapter = ga[g0 + (i < ng ? i : ng - 1)];
 #pragma unroll
-              for (int nb = 0; nb < 2; ++nb)
-                ptx::tma2_load_3d(b + nb * 8192 + i * R * 128, &tmL, 0, adapter * R, (nh >> 6) + nb, full);
-            }
-          } else {
-            const int adapter = ga[lc >> 1];
-            if (leader) ptx::mbar_arrive_expect_tx(bar_full(s), 2u * 64u * 128u * 2u);
+        for (int j = 0; j < 8; ++j) ga_reg[j] = (lane + 32 * j < G) ? ga[lane + 32 * j] : 0;
+      }
+      for (int kb = 0; kb < KB; ++kb, ++it) {
+        const int s = it % S;
+        if (lane == 0) {
+          ok = gemm2_wait(bar_empty(s), ((it / S) & 1) ^ 1, abort_flag, args.status);
+          if (ok) {
+            const uint32_t a = sA0 + s * GEMM2_STAGE_BYTES, b = a + GEMM2_A_BYTES;
+            const uint32_t full = ptx::map_to_cta(bar_full(s), 0);
+            if (leader) ptx::mbar_arrive_expect_tx(bar_full(s), 2 * GEMM2_STAGE_BYTES);
+            ptx::tma2_load_2d(a, &tmIn, kb * GEMM_BK, m0, full);
+            if (W_KMAJOR) ptx::tma2_load_2d(b, &tmW, kb * GEMM_BK, nh, full);          // [N, K]: 128 rows x 64 k
+            else          ptx::tma2_load_3d(b, &tmW, 0, kb * GEMM_BK, nh >> 6, full);  // (64 n, K, N/64): 64 x 64 k x 2
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+      }
+      if (!ok) break;
+      if (LC > 0) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (lane + 32 * j < G) ga_smem[lane + 32 * j] = ga_reg[j];
+        __syncwarp();
+      }
+      for (int lc = 0; lc < LC; ++lc, ++it) {
+        const int s = it % S;
+        if (lane == 0) {
+          ok = gemm2_wait(bar_empty(s), ((it / S) & 1) ^ 1, abort_flag, args.status);
+          if (ok) ptx::mbar_arrive(bar_go(s));       // hand the free slot to this CTA's builders
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        const uint32_t b = sA0 + s * GEMM2_STAGE_BYTES + GEMM2_A_BYTES;
+        const uint32_t full = ptx::map_to_cta(bar_full(s), 0);
+        if (R <= 64) {
+          const int g0 = lc * GPC;
+          const int ng = G - g0 < GPC ? G - g0 : GPC;
+          const int ngl = (R == 8 && (ng & 1)) ? ng + 1 : ng;   // rank 8: pad a half-filled MMA step
+          if (leader && lane == 0) ptx::mbar_arrive_expect_tx(bar_full(s), 2u * (uint32_t)ngl * R * 128u * 2u);
+          if (lane < ngl) {
+            const int adapter = ga_smem[g0 + (lane < ng ? lane : ng - 1)];
 #pragma unroll
             for (int nb = 0; nb < 2; ++nb)
-              ptx::tma2_load_3d(b + nb * 8192, &tmL, 0, adapter * R + (lc & 1) * 64, (nh >> 6) + nb, full);
+              ptx::tma2_load_3d(b + nb * 8192 + lane * R * 128, &tmL, 0, adapter * R, (nh >> 6) + nb, full);
           }
+        } else {
+          if (leader && lane == 0) ptx::mbar_arrive_expect_tx(bar_full(s), 2u * 64u * 128u * 2u);
+          if (lane < 2)
+            ptx::tma2_load_3d(b + lane * 8192, &tmL, 0, ga_smem[lc >> 1] * R + (lc & 1) * 64, (nh >> 6) + lane, full);
         }
       }
     }
