@@ -8,12 +8,15 @@
 // independent 128 x 256 tiles, which is what bounds the one-SM kernel.  No load is multicast:
 // every CTA fetches exactly the bytes that land in its own shared memory.
 //
+// The low-rank part needs no software-built operand here: the shrink kernel has already written
+// the rows' scaled rank-R values as block-diagonal bf16 chunks of [256 rows][64] (see PbdArgs), so
+// an extra K-block is an ordinary stage - A tile from that buffer, B tile = the groups' expand
+// matrices - and the CTA has only three roles (TMA producer, MMA issuer, four epilogue warps).
+//
 // Synchronisation across the pair (rank 0 = leader, the only issuer of MMAs):
 //   full[s]       in the leader: leader's producer arrives with the byte count of BOTH CTAs;
 //                 both CTAs' TMA loads complete on it (cta_group::2 loads may signal the peer).
 //   empty[s]      in each CTA: tcgen05.commit multicast to both (releases both producers).
-//   lora_go[s]    in each CTA: producer -> its own operand builders (slot is free).
-//   lora_full[s]  in the leader: 8 arrivals = 4 builder warps x 2 CTAs.
 //   tmem_full[b]  in each CTA: tcgen05.commit multicast (wakes both epilogues).
 //   tmem_empty[b] in the leader: 8 arrivals = 4 epilogue warps x 2 CTAs.
 // Every wait is bounded; the pair leaves through a cluster barrier before tensor memory is freed,
@@ -30,6 +33,7 @@ namespace mlora {
 constexpr int GEMM2_BM = 256;                 // rows of a pair tile (128 per CTA)
 constexpr int GEMM2_BN = 256;
 constexpr int GEMM2_STAGES = 6;
+constexpr int GEMM2_THREADS = 192;          // producer warp, MMA warp, four epilogue warps
 constexpr uint32_t GEMM2_A_BYTES = 128 * GEMM_BK * 2;               // 16 KiB: this CTA's rows
 constexpr uint32_t GEMM2_B_BYTES = 128 * GEMM_BK * 2;               // 16 KiB: this CTA's half of B
 constexpr uint32_t GEMM2_STAGE_BYTES = GEMM2_A_BYTES + GEMM2_B_BYTES;
@@ -122,10 +126,10 @@ __device__ __forceinline__ bool gemm2_wait(uint32_t bar, uint32_t parity, volati
 // args: n_mtiles counts 256-row pair tiles, n_ntiles 256-column tiles, n_units = their product;
 // row_grp / tile_grp_off / grp_adapter are the tables for 256-row tiles.
 template <int R, bool W_KMAJOR>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __launch_bounds__(GEMM2_THREADS, 1)
 gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ CUtensorMap tmW,
                   const __grid_constant__ CUtensorMap tmL, const __grid_constant__ CUtensorMap tmOut,
-                  const GemmArgs args) {
+                  const __grid_constant__ CUtensorMap tmPbd, const GemmArgs args) {
   static_assert(R == 8 || R == 16 || R == 32 || R == 64 || R == 128, "rank");
   constexpr int GPC = R <= 64 ? 64 / R : 1;          // groups per 64-wide low-rank block
   constexpr int S = GEMM2_STAGES;
@@ -137,14 +141,12 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
   const uint32_t sA0 = smem_base;
   const uint32_t sEpi = smem_base + S * GEMM2_STAGE_BYTES;
   const uint32_t sBar = sEpi + GEMM_EPI_BYTES;
-  // barriers: full[S] | empty[S] | lora_full[S] | lora_go[S] | tmem_full[2] | tmem_empty[2]
+  // barriers: full[S] | empty[S] | tmem_full[2] | tmem_empty[2]
   auto bar_full = [&](int s) { return sBar + 8u * s; };
   auto bar_empty = [&](int s) { return sBar + 8u * (S + s); };
-  auto bar_lora = [&](int s) { return sBar + 8u * (2 * S + s); };
-  auto bar_go = [&](int s) { return sBar + 8u * (3 * S + s); };
-  auto bar_tfull = [&](int b) { return sBar + 8u * (4 * S + b); };
-  auto bar_tempty = [&](int b) { return sBar + 8u * (4 * S + 2 + b); };
-  const uint32_t sMisc = sBar + 8u * (4 * S + 4);
+  auto bar_tfull = [&](int b) { return sBar + 8u * (2 * S + b); };
+  auto bar_tempty = [&](int b) { return sBar + 8u * (2 * S + 2 + b); };
+  const uint32_t sMisc = sBar + 8u * (2 * S + 4);
   uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(smem_gen + (sMisc - smem_base));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + (sMisc - smem_base) + 8);
 
@@ -157,8 +159,6 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
     for (int s = 0; s < S; ++s) {
       ptx::mbar_init(bar_full(s), 1);
       ptx::mbar_init(bar_empty(s), 1);
-      ptx::mbar_init(bar_lora(s), 8);
-      ptx::mbar_init(bar_go(s), 1);
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(bar_tfull(b), 1);
@@ -170,6 +170,7 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
     ptx::prefetch_tmap(&tmW);
     ptx::prefetch_tmap(&tmL);
     ptx::prefetch_tmap(&tmOut);
+    ptx::prefetch_tmap(&tmPbd);
   }
   if (warp == 1) {                                   // the same warp in both CTAs
     ptx::tmem2_alloc(ptx::smem_u32(tmem_ptr_smem), GEMM_TMEM_COLS);
@@ -206,6 +207,7 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
       const int nh = nt * GEMM2_BN + (int)rank * 128;     // this CTA's half of the B columns
       const int G = tile_groups(mt);
       const int LC = (G * R + 63) / 64;
+      const int chunk_base = args.lora_enabled ? args.tile_grp_off[mt] : 0;   // chunk slot = 2 * this + lc
       int32_t ga_reg[8];                                  // G <= 256 adapters of the pair tile
       {
         const int32_t* ga = args.grp_adapter + (args.lora_enabled ? args.tile_grp_off[mt] : 0);
@@ -237,19 +239,18 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
       }
       for (int lc = 0; lc < LC; ++lc, ++it) {
         const int s = it % S;
-        if (lane == 0) {
-          ok = gemm2_wait(bar_empty(s), ((it / S) & 1) ^ 1, abort_flag, args.status);
-          if (ok) ptx::mbar_arrive(bar_go(s));       // hand the free slot to this CTA's builders
-        }
+        if (lane == 0) ok = gemm2_wait(bar_empty(s), ((it / S) & 1) ^ 1, abort_flag, args.status);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) break;
-        const uint32_t b = sA0 + s * GEMM2_STAGE_BYTES + GEMM2_A_BYTES;
+        const uint32_t a = sA0 + s * GEMM2_STAGE_BYTES, b = a + GEMM2_A_BYTES;
         const uint32_t full = ptx::map_to_cta(bar_full(s), 0);
+        // A operand: this CTA's 128 rows of chunk lc of the tile's block-diagonal low-rank matrix
+        if (lane == 0) ptx::tma2_load_2d(a, &tmPbd, 0, (2 * chunk_base + lc) * 256 + (int)rank * 128, full);
         if (R <= 64) {
           const int g0 = lc * GPC;
           const int ng = G - g0 < GPC ? G - g0 : GPC;
           const int ngl = (R == 8 && (ng & 1)) ? ng + 1 : ng;   // rank 8: pad a half-filled MMA step
-          if (leader && lane == 0) ptx::mbar_arrive_expect_tx(bar_full(s), 2u * (uint32_t)ngl * R * 128u * 2u);
+          if (leader && lane == 0) ptx::mbar_arrive_expect_tx(bar_full(s), 2u * (GEMM2_A_BYTES + (uint32_t)ngl * R * 128u * 2u));
           if (lane < ngl) {
             const int adapter = ga_smem[g0 + (lane < ng ? lane : ng - 1)];
 #pragma unroll
@@ -257,7 +258,7 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
               ptx::tma2_load_3d(b + nb * 8192 + lane * R * 128, &tmL, 0, adapter * R, (nh >> 6) + nb, full);
           }
         } else {
-          if (leader && lane == 0) ptx::mbar_arrive_expect_tx(bar_full(s), 2u * 64u * 128u * 2u);
+          if (leader && lane == 0) ptx::mbar_arrive_expect_tx(bar_full(s), 2u * (GEMM2_A_BYTES + 64u * 128u * 2u));
           if (lane < 2)
             ptx::tma2_load_3d(b + lane * 8192, &tmL, 0, ga_smem[lc >> 1] * R + (lc & 1) * 64, (nh >> 6) + lane, full);
         }
@@ -269,7 +270,7 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
     if (leader && lane == 0) {
       constexpr uint32_t idesc_main = ptx::make_idesc_bf16(GEMM2_BM, GEMM2_BN, false, !W_KMAJOR);
       constexpr uint32_t idesc_lora = ptx::make_idesc_bf16(GEMM2_BM, GEMM2_BN, false, true);
-      uint32_t it = 0, lt = 0, lora_phase = 0;
+      uint32_t it = 0, lt = 0;
       bool ok = true;
       for (int unit = pair; unit < n_units && ok; unit += n_pairs, ++lt) {
         const int mt = unit % args.n_mtiles;
@@ -299,8 +300,6 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
         for (int lc = 0; lc < LC; ++lc, ++it) {
           const int s = it % S;
           if (!(ok = gemm2_wait(bar_full(s), (it / S) & 1, abort_flag, args.status))) break;
-          if (!(ok = gemm2_wait(bar_lora(s), (lora_phase >> s) & 1, abort_flag, args.status))) break;
-          lora_phase ^= 1u << s;
           ptx::tc_fence_after();
           const uint32_t a = sA0 + s * GEMM2_STAGE_BYTES, b = a + GEMM2_A_BYTES;
           const uint64_t adesc = ptx::make_smem_desc(a, 16, 1024);
@@ -318,7 +317,7 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
       }
     }
     __syncwarp();
-  } else if (warp < 6) {
+  } else {
     // ============================ epilogue (both CTAs, own rows) ============================
     const int e = warp & 3;
     const uint32_t stage0 = sEpi + (uint32_t)(warp - 2) * 8192u;
@@ -374,60 +373,6 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
     }
     if (lane == 0) ptx::tma_store_wait<0>();
     __syncwarp();
-  } else {
-    // ============================ low-rank operand builder (both CTAs, own rows) ============================
-    const int rloc = (warp - 6) * 32 + lane;        // row inside this CTA's half of the pair tile
-    uint32_t it = 0, go_phase = 0;
-    bool ok = true;
-    for (int unit = pair; unit < n_units && ok; unit += n_pairs) {
-      const int mt = unit % args.n_mtiles;
-      const int G = tile_groups(mt);
-      const int LC = (G * R + 63) / 64;
-      it += KB;
-      if (LC == 0) continue;
-      const int row = mt * GEMM2_BM + (int)rank * 128 + rloc;
-      const int grp = row < args.M ? args.row_grp[row] : -1;
-      uint32_t ub[R / 2];
-      if (grp >= 0) {
-        const float sc = args.scale ? args.scale[args.row_adapter[row]] : 1.0f;
-        const float4* src = reinterpret_cast<const float4*>(args.P + (size_t)row * R);
-#pragma unroll
-        for (int i = 0; i < R / 4; ++i) {
-          const float4 f = src[i];
-          ub[2 * i] = ptx::pack_bf16(f.x * sc, f.y * sc);
-          ub[2 * i + 1] = ptx::pack_bf16(f.z * sc, f.w * sc);
-        }
-      } else {
-#pragma unroll
-        for (int i = 0; i < R / 2; ++i) ub[i] = 0;
-      }
-      for (int lc = 0; lc < LC; ++lc, ++it) {
-        const int s = it % S;
-        if (!(ok = gemm_wait(bar_go(s), (go_phase >> s) & 1, abort_flag, args.status))) break;
-        go_phase ^= 1u << s;
-        const uint32_t rowaddr = sA0 + s * GEMM2_STAGE_BYTES + (uint32_t)rloc * 128u;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          uint32_t w0 = 0, w1 = 0, w2 = 0, w3 = 0;
-          if constexpr (R <= 64) {
-            const int gg = lc * GPC + (c * 8) / R;
-            constexpr int rr = R;
-            const int o = ((c * 8) % rr) / 2;
-            if (grp == gg) { w0 = ub[o]; w1 = ub[o + 1]; w2 = ub[o + 2]; w3 = ub[o + 3]; }
-          } else {
-            if (grp == (lc >> 1)) {
-              if (lc & 1) { w0 = ub[R / 4 + c * 4]; w1 = ub[R / 4 + c * 4 + 1]; w2 = ub[R / 4 + c * 4 + 2]; w3 = ub[R / 4 + c * 4 + 3]; }
-              else        { w0 = ub[c * 4]; w1 = ub[c * 4 + 1]; w2 = ub[c * 4 + 2]; w3 = ub[c * 4 + 3]; }
-            }
-          }
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(rowaddr + (uint32_t)((c ^ (rloc & 7)) << 4)),
-                       "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
-        }
-        ptx::fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_lora(s), 0));
-      }
-    }
   }
 
   // ============================ common exit ============================

@@ -34,6 +34,8 @@ struct mlora_ctx {
   int64_t ws_partial_items = 0;
   int32_t* ws_counters = nullptr;    // [ws_counter_items] arrival counters, zero between launches
   int64_t ws_counter_items = 0;
+  __nv_bfloat16* ws_pbd = nullptr;   // block-diagonal low-rank operand: [2 * ws_pbd_groups * 256, 64] bf16
+  int64_t ws_pbd_groups = 0;
   int64_t launches = 0;
   int32_t gemm_path = 0;
   int32_t shrink_path = 0;           // 0: streaming kernel for rank <= 32; 1: per-item kernel for every rank
@@ -59,6 +61,7 @@ struct DevRowSpace {
   const int32_t* row_grp2 = nullptr;
   const int32_t* tile2_grp_off = nullptr;
   const int32_t* grp2_adapter = nullptr;
+  const int32_t* zero_rows2 = nullptr;
   const int32_t* item_rows = nullptr;
   const int32_t* item_save = nullptr;
   const int32_t* item_start = nullptr;
@@ -293,14 +296,14 @@ mlora_status_t launch_gemm_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUten
 // Two-SM kernel: grid = 2 x (number of CTA pairs that can be resident at once).
 template <int R, bool W_KMAJOR>
 mlora_status_t launch_gemm2_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUtensorMap& tW, const CUtensorMap& tL,
-                              const CUtensorMap& tOut, const GemmArgs& g, cudaStream_t st) {
+                              const CUtensorMap& tOut, const CUtensorMap& tPbd, const GemmArgs& g, cudaStream_t st) {
   static int max_pairs = 0;         // per instantiation
   auto kern = gemm2_lora_kernel<R, W_KMAJOR>;
   if (max_pairs == 0) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM2_SMEM_BYTES) != cudaSuccess)
       return MLORA_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2 * ctx->sm_count); cfg.blockDim = dim3(GEMM_THREADS); cfg.dynamicSmemBytes = GEMM2_SMEM_BYTES;
+    cfg.gridDim = dim3(2 * ctx->sm_count); cfg.blockDim = dim3(GEMM2_THREADS); cfg.dynamicSmemBytes = GEMM2_SMEM_BYTES;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
@@ -311,19 +314,19 @@ mlora_status_t launch_gemm2_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUte
   }
   const int pairs = g.n_units < max_pairs ? g.n_units : max_pairs;
   LaunchScope scope(ctx, st, W_KMAJOR ? KIND_GEMM_BWD : KIND_GEMM_FWD);
-  launch_pdl_pairs(scope.slot < 0, kern, dim3(2 * pairs), dim3(GEMM_THREADS), GEMM2_SMEM_BYTES, st, tIn, tW, tL, tOut, g);
+  launch_pdl_pairs(scope.slot < 0, kern, dim3(2 * pairs), dim3(GEMM2_THREADS), GEMM2_SMEM_BYTES, st, tIn, tW, tL, tOut, tPbd, g);
   return scope.done();
 }
 
 template <bool W_KMAJOR>
 mlora_status_t launch_gemm2(mlora_ctx* ctx, int R, const CUtensorMap& tIn, const CUtensorMap& tW, const CUtensorMap& tL,
-                            const CUtensorMap& tOut, const GemmArgs& g, cudaStream_t st) {
+                            const CUtensorMap& tOut, const CUtensorMap& tPbd, const GemmArgs& g, cudaStream_t st) {
   switch (R) {
-    case 8: return launch_gemm2_r<8, W_KMAJOR>(ctx, tIn, tW, tL, tOut, g, st);
-    case 16: return launch_gemm2_r<16, W_KMAJOR>(ctx, tIn, tW, tL, tOut, g, st);
-    case 32: return launch_gemm2_r<32, W_KMAJOR>(ctx, tIn, tW, tL, tOut, g, st);
-    case 64: return launch_gemm2_r<64, W_KMAJOR>(ctx, tIn, tW, tL, tOut, g, st);
-    case 128: return launch_gemm2_r<128, W_KMAJOR>(ctx, tIn, tW, tL, tOut, g, st);
+    case 8: return launch_gemm2_r<8, W_KMAJOR>(ctx, tIn, tW, tL, tOut, tPbd, g, st);
+    case 16: return launch_gemm2_r<16, W_KMAJOR>(ctx, tIn, tW, tL, tOut, tPbd, g, st);
+    case 32: return launch_gemm2_r<32, W_KMAJOR>(ctx, tIn, tW, tL, tOut, tPbd, g, st);
+    case 64: return launch_gemm2_r<64, W_KMAJOR>(ctx, tIn, tW, tL, tOut, tPbd, g, st);
+    case 128: return launch_gemm2_r<128, W_KMAJOR>(ctx, tIn, tW, tL, tOut, tPbd, g, st);
     default: return MLORA_ERR_UNSUPPORTED;
   }
 }
@@ -368,7 +371,11 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
     g.row_grp = ds.row_grp2; g.row_adapter = ds.row_adapter;
     g.tile_grp_off = ds.tile2_grp_off; g.grp_adapter = ds.grp2_adapter;
     g.P = P; g.scale = scale; g.status = ctx->status_dev;
-    return launch_gemm2<W_KMAJOR>(ctx, R, tIn, tW, tL, tOut, g, st);
+    CUtensorMap tPbd;
+    const uint64_t slots = g.lora_enabled ? 2 * (uint64_t)hs.grp2_adapter.size() : 1;
+    if ((s = make_tmap_bf16(ctx, &tPbd, ctx->ws_pbd ? (const void*)ctx->ws_pbd : In, 64, slots * 256, 64, 64, 128)) != MLORA_OK)
+      return s;
+    return launch_gemm2<W_KMAJOR>(ctx, R, tIn, tW, tL, tOut, tPbd, g, st);
   }
   g.n_mtiles = (M + GEMM_BM - 1) / GEMM_BM;
   g.n_ntiles = (N + GEMM_BN - 1) / GEMM_BN;
@@ -608,6 +615,7 @@ void mlora_destroy(mlora_ctx* c) {
   cudaFree(c->ws_p);
   cudaFree(c->ws_partial);
   cudaFree(c->ws_counters);
+  cudaFree(c->ws_pbd);
   delete c;
 }
 
@@ -624,12 +632,13 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
     if (cudaSetDevice(ctx->device) != cudaSuccess) { delete p; return MLORA_ERR_CUDA; }
     BlobBuilder b;
     const HostPlan& h = p->h;
-    size_t o[56]; int n = 0;
+    size_t o[64]; int n = 0;
     const RowSpace* rs[2] = {&h.fwd, &h.bwd};
     for (int i = 0; i < 2; ++i) {
       o[n++] = b.add(rs[i]->row_adapter); o[n++] = b.add(rs[i]->row_save); o[n++] = b.add(rs[i]->row_grp);
       o[n++] = b.add(rs[i]->tile_grp_off); o[n++] = b.add(rs[i]->grp_adapter); o[n++] = b.add(rs[i]->item_rows);
       o[n++] = b.add(rs[i]->row_grp2); o[n++] = b.add(rs[i]->tile2_grp_off); o[n++] = b.add(rs[i]->grp2_adapter);
+      o[n++] = b.add(rs[i]->zero_rows2);
       o[n++] = b.add(rs[i]->item_save); o[n++] = b.add(rs[i]->item_start); o[n++] = b.add(rs[i]->item_contig); o[n++] = b.add(rs[i]->item_nrows); o[n++] = b.add(rs[i]->item_adapter);
     }
     o[n++] = b.add(h.slot_chunk_off); o[n++] = b.add(h.chunk_row0); o[n++] = b.add(h.chunk_nrows);
@@ -644,6 +653,7 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
       ds[i]->row_adapter = p->blob + o[n++]; ds[i]->row_save = p->blob + o[n++]; ds[i]->row_grp = p->blob + o[n++];
       ds[i]->tile_grp_off = p->blob + o[n++]; ds[i]->grp_adapter = p->blob + o[n++]; ds[i]->item_rows = p->blob + o[n++];
       ds[i]->row_grp2 = p->blob + o[n++]; ds[i]->tile2_grp_off = p->blob + o[n++]; ds[i]->grp2_adapter = p->blob + o[n++];
+      ds[i]->zero_rows2 = p->blob + o[n++];
       ds[i]->item_save = p->blob + o[n++]; ds[i]->item_start = p->blob + o[n++]; ds[i]->item_contig = p->blob + o[n++]; ds[i]->item_nrows = p->blob + o[n++]; ds[i]->item_adapter = p->blob + o[n++];
     }
     p->bwd.row_save = nullptr;       // the compact space has no save offsets
@@ -670,6 +680,17 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
         cudaFree(p->blob); delete p; return MLORA_ERR_CUDA;
       }
       ctx->ws_partial_items = part_items; ctx->ws_counter_items = items;
+    }
+    const int64_t groups = (int64_t)(h.fwd.grp2_adapter.size() > h.bwd.grp2_adapter.size() ? h.fwd.grp2_adapter.size()
+                                                                                          : h.bwd.grp2_adapter.size());
+    if (groups > ctx->ws_pbd_groups) {   // two chunk slots of [256][64] bf16 per adapter group of a tile
+      if (cudaDeviceSynchronize() != cudaSuccess) { cudaFree(p->blob); delete p; return MLORA_ERR_CUDA; }
+      cudaFree(ctx->ws_pbd);
+      ctx->ws_pbd = nullptr; ctx->ws_pbd_groups = 0;
+      if (cudaMalloc(&ctx->ws_pbd, (size_t)groups * 2 * 256 * 64 * sizeof(__nv_bfloat16)) != cudaSuccess) {
+        cudaFree(p->blob); delete p; return MLORA_ERR_CUDA;
+      }
+      ctx->ws_pbd_groups = groups;
     }
   }
   *out = p;
@@ -725,6 +746,8 @@ mlora_status_t mlora_mixed_forward(mlora_ctx* ctx, const mlora_layer_t* L, const
   sa.P_all = (const __nv_bfloat16*)L->A_all; sa.scale = nullptr; sa.Out = ctx->ws_p;
   sa.item_rows = p->fwd.item_rows; sa.item_start = p->fwd.item_start; sa.item_nrows = p->fwd.item_nrows;
   sa.item_adapter = p->fwd.item_adapter; sa.item_save = p->fwd.item_save;
+  sa.pbd = PbdArgs{ctx->gemm_pairs ? ctx->ws_pbd : nullptr, p->fwd.row_grp2, p->fwd.tile2_grp_off, L->scale,
+                   p->fwd.zero_rows2, (int32_t)h.fwd.zero_rows2.size()};
   sa.x_save = (__nv_bfloat16*)x_save; sa.u_save = u_save; sa.save_base = save_row_base;
   if ((s = launch_shrink(ctx, L->rank, sa, h.fwd.n_items(), p->fwd.item_contig, h.n_rows, L->n_adapters, st)) != MLORA_OK)
     return s;
@@ -755,6 +778,8 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   sa.In = (const __nv_bfloat16*)dY; sa.ld_in = lddy; sa.D = L->d_out;
   sa.P_all = (const __nv_bfloat16*)L->B_all; sa.scale = L->scale; sa.Out = ctx->ws_p;
   sa.item_rows = p->bwd.item_rows; sa.item_start = p->bwd.item_start; sa.item_nrows = p->bwd.item_nrows;
+  sa.pbd = PbdArgs{(ctx->gemm_pairs && dX) ? ctx->ws_pbd : nullptr, p->bwd.row_grp2, p->bwd.tile2_grp_off, nullptr,
+                   p->bwd.zero_rows2, (int32_t)h.bwd.zero_rows2.size()};
   sa.item_adapter = p->bwd.item_adapter; sa.item_save = nullptr; sa.x_save = nullptr; sa.u_save = nullptr; sa.save_base = 0;
   if ((s = launch_shrink(ctx, L->rank, sa, h.bwd.n_items(), p->bwd.item_contig, h.ft_rows, L->n_adapters, st)) != MLORA_OK)
     return s;

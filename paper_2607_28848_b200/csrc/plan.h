@@ -28,6 +28,7 @@ struct RowSpace {
   std::vector<int32_t> grp_adapter;    // [tile_grp_off.back()]
   // the same three tables for tiles of kPairTileRows rows
   std::vector<int32_t> row_grp2, tile2_grp_off, grp2_adapter;
+  std::vector<int32_t> zero_rows2;     // rows without an adapter inside 256-row tiles that have groups
   // Shrink items: the rows that have an adapter, gathered BY ADAPTER (ascending adapter id, rows
   // ascending inside an adapter) and cut into items of <= kItemRows rows.  Rows of an item need
   // not be adjacent in the batch: decode rows that share an adapter are processed together, so an
@@ -79,6 +80,11 @@ inline void build_tiles_and_items(RowSpace& rs) {
   const int32_t n = rs.n_rows;
   build_tile_groups(rs.row_adapter, kTileRows, rs.row_grp, rs.tile_grp_off, rs.grp_adapter);
   build_tile_groups(rs.row_adapter, kPairTileRows, rs.row_grp2, rs.tile2_grp_off, rs.grp2_adapter);
+  rs.zero_rows2.clear();
+  for (int32_t t = 0; t < n; ++t) {
+    const int32_t tile = t / kPairTileRows;
+    if (rs.row_adapter[t] < 0 && rs.tile2_grp_off[tile + 1] > rs.tile2_grp_off[tile]) rs.zero_rows2.push_back(t);
+  }
   rs.item_rows.clear(); rs.item_start.clear(); rs.item_nrows.clear(); rs.item_adapter.clear(); rs.item_contig.clear();
   int32_t max_adapter = -1;
   for (int32_t t = 0; t < n; ++t) max_adapter = rs.row_adapter[t] > max_adapter ? rs.row_adapter[t] : max_adapter;

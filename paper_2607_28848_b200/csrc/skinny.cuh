@@ -17,6 +17,42 @@ namespace mlora {
 
 constexpr int GRAD_THREADS = 256;
 
+// Block-diagonal low-rank operand of the two-SM GEMM, written by the shrink kernels.  For each
+// 256-row tile with G adapter groups the rows' (scaled) rank-R values are laid out as a
+// [256, G R] matrix that is zero outside each row's own group block, cut into 64-column chunks of
+// [256 rows][64] bf16 (one chunk = the A operand of one extra K-block of the GEMM).  Chunk c of
+// tile t lives at chunk slot 2 * tile2_grp_off[t] + c (two slots per group cover rank <= 128).
+struct PbdArgs {
+  __nv_bfloat16* pbd;            // nullable: [slots * 256, 64]
+  const int32_t* row_grp2;       // [rows] group of the row inside its 256-row tile, -1: none
+  const int32_t* tile2_grp_off;  // [tiles + 1]
+  const float* scale;            // nullable: values multiplied by scale[adapter]
+  const int32_t* zero_rows;      // rows without an adapter inside tiles that have groups
+  int32_t n_zero_rows;
+};
+
+// One warp writes all chunks of one row: `vals` = the row's R fp32 values (nullptr: all zero).
+template <int R>
+__device__ __forceinline__ void pbd_write_row(const PbdArgs& pa, int row, const float* vals, float sc, int lane) {
+  const int tile = row >> 8, rl = row & 255;
+  const int goff = pa.tile2_grp_off[tile];
+  const int G = pa.tile2_grp_off[tile + 1] - goff;
+  const int LC = (G * R + 63) / 64;
+  const int g = vals ? pa.row_grp2[row] : -1;
+  for (int piece = lane; piece < LC * 8; piece += 32) {
+    const int c = piece >> 3, kcol = piece * 8;          // chunk, first low-rank column of the piece
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (g >= 0 && kcol >= g * R && kcol < (g + 1) * R) {
+      const float4 f0 = *reinterpret_cast<const float4*>(vals + (kcol - g * R));
+      const float4 f1 = *reinterpret_cast<const float4*>(vals + (kcol - g * R) + 4);
+      v.x = ptx::pack_bf16(f0.x * sc, f0.y * sc); v.y = ptx::pack_bf16(f0.z * sc, f0.w * sc);
+      v.z = ptx::pack_bf16(f1.x * sc, f1.y * sc); v.w = ptx::pack_bf16(f1.z * sc, f1.w * sc);
+    }
+    __nv_bfloat16* dst = pa.pbd + ((size_t)(2 * goff + c) * 256 + rl) * 64 + (piece & 7) * 8;
+    *reinterpret_cast<uint4*>(dst) = v;
+  }
+}
+
 struct ShrinkArgs {
   const __nv_bfloat16* In;     // [rows, D], row stride ld_in
   int64_t ld_in;
@@ -35,6 +71,7 @@ struct ShrinkArgs {
   // split of the contraction over gridDim.y CTAs per item (used when there are few items):
   float* partial;              // [n_items * gridDim.z * gridDim.y, MT * 16, R] scratch
   int32_t* counters;           // [n_items * gridDim.z], zero between launches
+  PbdArgs pbd;                 // optional block-diagonal copy of the result for the two-SM GEMM
 };
 
 // One CTA per item; its warps take the 64-wide K blocks round-robin and reduce through shared
@@ -83,6 +120,9 @@ shrink_kernel(const ShrinkArgs a) {
   // everything above read only the plan's tables; from here on the predecessor's data is touched
   ptx::grid_dependency_wait();
   ptx::grid_launch_dependents();
+  if (a.pbd.pbd && blockIdx.y == 0 && blockIdx.z == 0)         // rows nobody else owns: all-zero chunks
+    for (int i = blockIdx.x * WARPS + warp; i < a.pbd.n_zero_rows; i += gridDim.x * WARPS)
+      pbd_write_row<R>(a.pbd, a.pbd.zero_rows[i], nullptr, 0.f, lane);
 
   float acc[MT][RB][4];
 #pragma unroll
@@ -182,6 +222,13 @@ shrink_kernel(const ShrinkArgs a) {
     }
   }
   if (ksplit > 1 && threadIdx.x == 0) a.counters[item] = 0;     // ready for the next launch
+  if (a.pbd.pbd) {
+    __syncthreads();             // the rows of Out written above are read back below
+    for (int r = warp; r < nrows; r += WARPS) {
+      const int row = rows[r];
+      pbd_write_row<R>(a.pbd, row, a.Out + (size_t)row * R, a.pbd.scale ? a.pbd.scale[adapter] : 1.0f, lane);
+    }
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -336,6 +383,9 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
     // this thread's pieces of a K-block: elements 16c .. 16c+15 of the block
     ptx::grid_dependency_wait();
     bool ok = true;
+    if (a.pbd.pbd)                                            // rows nobody else owns: all-zero chunks
+      for (int i = cta * STREAM_WARPS + warp; i < a.pbd.n_zero_rows; i += gridDim.x * STREAM_WARPS)
+        pbd_write_row<R>(a.pbd, a.pbd.zero_rows[i], nullptr, 0.f, lane);
 
     for (int u = u_begin; u < u_end; ++u) {
       const int i = u - u_begin, st = i % STAGES;
@@ -472,6 +522,13 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
           }
         }
         if (c0 != c1 && threadIdx.x == 0) a.counters[this_item] = 0;    // ready for the next launch
+        if (a.pbd.pbd) {
+          asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");  // Out rows written above are read back
+          for (int r = warp; r < cur_nrows; r += STREAM_WARPS) {
+            const int row = cur_rows[r];
+            pbd_write_row<R>(a.pbd, row, a.Out + (size_t)row * R, a.pbd.scale ? a.pbd.scale[cur_adapter] : 1.0f, lane);
+          }
+        }
       }
       asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");      // red[] is reused by the next item
     }
