@@ -79,6 +79,9 @@ struct mlora_plan {
   const int32_t* chunk_row0 = nullptr;
   const int32_t* chunk_nrows = nullptr;
   const int32_t* slot_adapter = nullptr;
+  const int32_t* slot_blk_off = nullptr;
+  const int32_t* blk_row0 = nullptr;
+  const int32_t* blk_nrows = nullptr;
 };
 
 namespace {
@@ -259,8 +262,37 @@ mlora_status_t launch_shrink(mlora_ctx* ctx, int R, ShrinkArgs a, int n_items, c
   return scope.done();
 }
 
-mlora_status_t launch_grad(mlora_ctx* ctx, const GradArgs& a, int n_slots, cudaStream_t st) {
+template <int MB>
+mlora_status_t launch_grad_stream(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& a, int n_slots, int n_rows,
+                                  cudaStream_t st) {
+  constexpr size_t smem = (size_t)gstream_stages(MB) * (128 * 128 + 128 * MB * 16 * 4) + (size_t)STREAM_WARPS * MB * 16 * 65 * 4 + 1024;
+  static bool attr_set = false;
+  auto kern = grad_stream_kernel<MB>;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return MLORA_ERR_CUDA;
+    attr_set = true;
+  }
+  CUtensorMap tQ;
+  mlora_status_t ms = make_tmap_bf16(ctx, &tQ, a.Q, a.D, n_rows, a.ldq, 64, 128);
+  if (ms != MLORA_OK) return ms;
+  GradStreamArgs ga;
+  ga.g = a;
+  ga.slot_blk_off = p->slot_blk_off; ga.blk_row0 = p->blk_row0; ga.blk_nrows = p->blk_nrows;
+  ga.n_slots = n_slots; ga.n_strips = a.D / 64; ga.status = ctx->status_dev;
+  const int groups = n_slots * ga.n_strips;
+  const int grid = groups < ctx->sm_count ? groups : ctx->sm_count;
+  LaunchScope scope(ctx, st, KIND_GRAD);
+  launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(STREAM_THREADS), smem, st, tQ, ga);
+  return scope.done();
+}
+
+mlora_status_t launch_grad(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& a, int n_slots, int n_rows,
+                           cudaStream_t st) {
   if (n_slots <= 0) return MLORA_OK;
+  if (ctx->shrink_path == 0) {
+    if (a.R <= 16) return launch_grad_stream<1>(ctx, p, a, n_slots, n_rows, st);
+    if (a.R <= 32) return launch_grad_stream<2>(ctx, p, a, n_slots, n_rows, st);
+  }
   constexpr int smem1 = (GRAD_THREADS / 32) * 16 * 65 * 4, smem2 = 2 * smem1;
   static bool attr_set = false;
   if (!attr_set) {
@@ -643,6 +675,7 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
     }
     o[n++] = b.add(h.slot_chunk_off); o[n++] = b.add(h.chunk_row0); o[n++] = b.add(h.chunk_nrows);
     o[n++] = b.add(h.ft_adapters);
+    o[n++] = b.add(h.slot_blk_off); o[n++] = b.add(h.blk_row0); o[n++] = b.add(h.blk_nrows);
     if (cudaMalloc(&p->blob, b.data.size() * sizeof(int32_t)) != cudaSuccess) { delete p; return MLORA_ERR_CUDA; }
     if (cudaMemcpy(p->blob, b.data.data(), b.data.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
       cudaFree(p->blob); delete p; return MLORA_ERR_CUDA;
@@ -659,6 +692,7 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
     p->bwd.row_save = nullptr;       // the compact space has no save offsets
     p->slot_chunk_off = p->blob + o[n++]; p->chunk_row0 = p->blob + o[n++]; p->chunk_nrows = p->blob + o[n++];
     p->slot_adapter = p->blob + o[n++];
+    p->slot_blk_off = p->blob + o[n++]; p->blk_row0 = p->blob + o[n++]; p->blk_nrows = p->blob + o[n++];
     if (n_rows > ctx->ws_rows) {     // grow the rank-r workspace (the only other device allocation)
       if (cudaDeviceSynchronize() != cudaSuccess) { cudaFree(p->blob); delete p; return MLORA_ERR_CUDA; }
       cudaFree(ctx->ws_p);
@@ -788,10 +822,10 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   ga.P = u_save; ga.R = L->rank; ga.scale = L->scale; ga.Q = (const __nv_bfloat16*)dY; ga.ldq = lddy; ga.D = L->d_out;
   ga.G = dB; ga.slot_chunk_off = p->slot_chunk_off; ga.chunk_row0 = p->chunk_row0; ga.chunk_nrows = p->chunk_nrows;
   ga.slot_adapter = p->slot_adapter; ga.accumulate = accumulate;
-  if ((s = launch_grad(ctx, ga, n_slots, st)) != MLORA_OK) return s;
+  if ((s = launch_grad(ctx, p, ga, n_slots, h.ft_rows, st)) != MLORA_OK) return s;
   ga.P = ctx->ws_p; ga.scale = nullptr; ga.Q = (const __nv_bfloat16*)x_save; ga.ldq = L->d_in; ga.D = L->d_in;
   ga.G = dA;                         // dA = V^T X
-  if ((s = launch_grad(ctx, ga, n_slots, st)) != MLORA_OK) return s;
+  if ((s = launch_grad(ctx, p, ga, n_slots, h.ft_rows, st)) != MLORA_OK) return s;
   if (!dX) return MLORA_OK;
   return gemm_bf16<true>(ctx, L, h.bwd, p->bwd, dY, lddy, dX, lddx, L->A_all, ctx->ws_p, nullptr, h.ft_rows, L->d_in,
                          L->d_out, st);

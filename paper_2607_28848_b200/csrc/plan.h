@@ -51,6 +51,9 @@ struct HostPlan {
   // Gradient work: per slot, chunks of <= kChunkRows compact rows.
   std::vector<int32_t> slot_chunk_off; // [n_slots + 1]
   std::vector<int32_t> chunk_row0, chunk_nrows;
+  // The same rows as blocks of <= kTileRows consecutive compact rows (tiles of the streaming kernel).
+  std::vector<int32_t> slot_blk_off;   // [n_slots + 1]
+  std::vector<int32_t> blk_row0, blk_nrows;
 };
 
 inline void build_tile_groups(const std::vector<int32_t>& row_adapter, int32_t tile_rows,
@@ -171,6 +174,17 @@ inline mlora_status_t build_plan(const mlora_segment_t* segs, int32_t n_segs, in
       }
     }
     p.slot_chunk_off.push_back((int32_t)p.chunk_row0.size());
+  }
+  p.slot_blk_off.assign(1, 0);
+  for (int32_t a : p.ft_adapters) {
+    for (int32_t k = 0; k < n_segs; ++k) {
+      if (!segs[k].is_finetune || segs[k].adapter_id != a) continue;
+      for (int32_t i = 0; i < segs[k].row_len; i += kTileRows) {
+        p.blk_row0.push_back(p.seg_save_off[k] + i);
+        p.blk_nrows.push_back(segs[k].row_len - i < kTileRows ? segs[k].row_len - i : kTileRows);
+      }
+    }
+    p.slot_blk_off.push_back((int32_t)p.blk_row0.size());
   }
   return MLORA_OK;
 }

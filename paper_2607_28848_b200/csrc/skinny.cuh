@@ -664,4 +664,175 @@ grad_kernel(const GradArgs a) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Streaming gradient kernel for ranks up to 32.  A persistent CTA takes whole (slot, 64-column
+// strip) groups in turn; for each it streams the slot's rows as tiles of 128 rows x 64 columns
+// (one tensor-map load into 128B-swizzled shared memory) together with the matching 128 x R block
+// of P (one bulk copy) through a ring of stages, so that the bytes in flight do not depend on
+// registers.  Consumer warp w contracts rows 16w .. 16w+15 of every tile (one MMA K-step, rows as
+// the contraction index); the eight warps are added in a fixed order when the strip is done.
+__host__ __device__ constexpr int gstream_stages(int mb) { return mb == 1 ? 6 : 4; }
+
+struct GradStreamArgs {
+  GradArgs g;
+  const int32_t* slot_blk_off;
+  const int32_t* blk_row0;
+  const int32_t* blk_nrows;
+  int32_t n_slots, n_strips;
+  int32_t* status;
+};
+
+template <int MB>
+__global__ void __launch_bounds__(STREAM_THREADS, 1)
+grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const GradStreamArgs ga) {
+  constexpr int S = gstream_stages(MB);
+  constexpr int RMAX = MB * 16;
+  constexpr uint32_t Q_BYTES = 128 * 128;                 // 128 rows x 64 bf16, swizzled
+  constexpr uint32_t P_BYTES = 128 * RMAX * 4;
+  constexpr uint32_t STAGE_BYTES = Q_BYTES + P_BYTES;
+  extern __shared__ __align__(1024) uint8_t gs_smem[];
+  __shared__ __align__(8) uint64_t bars[2 * S];
+  __shared__ int abort_word;
+  volatile int* abort_flag = &abort_word;
+  const GradArgs& a = ga.g;
+  const int R = a.R;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t ring = (ptx::smem_u32(gs_smem) + 1023u) & ~1023u;      // swizzled tiles need 1 KiB alignment
+  float (*red)[MB * 16][64 + 1] = reinterpret_cast<float (*)[MB * 16][64 + 1]>(
+      gs_smem + (ring - ptx::smem_u32(gs_smem)) + S * STAGE_BYTES);
+  const uint32_t bar0 = ptx::smem_u32(bars);
+  auto bar_full = [&](int st) { return bar0 + 8u * st; };
+  auto bar_empty = [&](int st) { return bar0 + 8u * (S + st); };
+  if (threadIdx.x == 0) {
+    for (int st = 0; st < S; ++st) { ptx::mbar_init(bar_full(st), 1); ptx::mbar_init(bar_empty(st), STREAM_WARPS); }
+    abort_word = 0;
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmQ);
+  }
+  __syncthreads();
+  const int n_groups = ga.n_slots * ga.n_strips;
+
+  if (warp == STREAM_WARPS) {
+    // ======================= producer =======================
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
+    if (lane == 0) {
+      uint32_t i = 0;
+      bool ok = true;
+      for (int grp = blockIdx.x; grp < n_groups && ok; grp += gridDim.x) {
+        const int slot = grp / ga.n_strips, strip = grp % ga.n_strips;
+        for (int b = ga.slot_blk_off[slot]; b < ga.slot_blk_off[slot + 1]; ++b, ++i) {
+          const int st = i % S;
+          if (!(ok = stream_wait(bar_empty(st), ((i / S) & 1) ^ 1, abort_flag, ga.status))) break;
+          const int row0 = ga.blk_row0[b], nrows = ga.blk_nrows[b];
+          const uint32_t dst = ring + (uint32_t)st * STAGE_BYTES;
+          const uint32_t pbytes = (uint32_t)nrows * (uint32_t)R * 4u;
+          ptx::mbar_arrive_expect_tx(bar_full(st), Q_BYTES + pbytes);
+          ptx::tma_load_2d(dst, &tmQ, strip * 64, row0, bar_full(st));       // rows past the block are masked below
+          bulk_load(dst + Q_BYTES, a.P + (size_t)row0 * R, pbytes, bar_full(st));
+        }
+      }
+    }
+  } else {
+    // ======================= consumers =======================
+    const int g = lane >> 2, c = lane & 3;
+    ptx::grid_dependency_wait();
+    float acc[MB][8][4];
+    uint32_t i = 0;
+    bool ok = true;
+    for (int grp = blockIdx.x; grp < n_groups && ok; grp += gridDim.x) {
+      const int slot = grp / ga.n_strips, strip = grp % ga.n_strips;
+      const float sc = a.scale ? a.scale[a.slot_adapter[slot]] : 1.0f;
+#pragma unroll
+      for (int m = 0; m < MB; ++m)
+#pragma unroll
+        for (int n = 0; n < 8; ++n) acc[m][n][0] = acc[m][n][1] = acc[m][n][2] = acc[m][n][3] = 0.f;
+      for (int b = ga.slot_blk_off[slot]; b < ga.slot_blk_off[slot + 1]; ++b, ++i) {
+        const int st = i % S;
+        const int nrows = ga.blk_nrows[b];
+        if (!(ok = stream_wait(bar_full(st), (i / S) & 1, abort_flag, ga.status))) break;
+        const uint32_t qbase = ring + (uint32_t)st * STAGE_BYTES;
+        const uint32_t pbase = qbase + Q_BYTES;
+        if (warp * 16 < nrows) {
+          // rows of this warp's K-step: r = 16 warp + {2c, 2c+1, 2c+8, 2c+9}
+          uint4 q[4];
+          uint32_t ahi[MB][4], alo[MB][4];
+          const int tr[4] = {2 * c, 2 * c + 1, 2 * c + 8, 2 * c + 9};
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const int r = warp * 16 + tr[k];
+            // 16-byte piece g of row r sits at piece (g ^ (r & 7)) of the swizzled 128-byte row
+            q[k] = lds_v4(qbase + (uint32_t)r * 128u + (uint32_t)((g ^ (r & 7)) << 4));
+            if (r >= nrows) q[k] = make_uint4(0, 0, 0, 0);      // rows of the tile past the block's end
+          }
+#pragma unroll
+          for (int m = 0; m < MB; ++m) {
+            float pv[4][2];
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                const int r = warp * 16 + tr[k], qq = m * 16 + g + 8 * h;
+                float v = 0.f;
+                if (r < nrows && qq < R)
+                  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(pbase + (uint32_t)(r * R + qq) * 4u));
+                pv[k][h] = v * sc;
+              }
+#pragma unroll
+            for (int f = 0; f < 4; ++f) {       // a0 (q=g, rows 2c,2c+1), a1 (q=g+8, same rows), a2, a3: rows 2c+8,2c+9
+              const int h = f & 1, rp = (f >> 1) * 2;
+              const float e0 = pv[rp][h], e1 = pv[rp + 1][h];
+              const __nv_bfloat16 h0 = __float2bfloat16_rn(e0), h1 = __float2bfloat16_rn(e1);
+              ahi[m][f] = ptx::pack_bf16(e0, e1);
+              alo[m][f] = ptx::pack_bf16(e0 - __bfloat162float(h0), e1 - __bfloat162float(h1));
+            }
+          }
+          const uint32_t qr[4][4] = {{q[0].x, q[0].y, q[0].z, q[0].w}, {q[1].x, q[1].y, q[1].z, q[1].w},
+                                     {q[2].x, q[2].y, q[2].z, q[2].w}, {q[3].x, q[3].y, q[3].z, q[3].w}};
+#pragma unroll
+          for (int nb = 0; nb < 8; ++nb) {
+            const uint32_t sel = (nb & 1) ? 0x7632u : 0x5410u;
+            const uint32_t b0 = __byte_perm(qr[0][nb >> 1], qr[1][nb >> 1], sel);
+            const uint32_t b1 = __byte_perm(qr[2][nb >> 1], qr[3][nb >> 1], sel);
+#pragma unroll
+            for (int m = 0; m < MB; ++m) {
+              ptx::mma_bf16_16816(acc[m][nb], ahi[m][0], ahi[m][1], ahi[m][2], ahi[m][3], b0, b1);
+              ptx::mma_bf16_16816(acc[m][nb], alo[m][0], alo[m][1], alo[m][2], alo[m][3], b0, b1);
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar_empty(st));
+      }
+      if (!ok) break;
+      // ---- strip done: fixed-order sum over the warps, then write (or add to) the gradient ----
+      {
+        float (*mine)[64 + 1] = red[warp];
+#pragma unroll
+        for (int m = 0; m < MB; ++m)
+#pragma unroll
+          for (int nb = 0; nb < 8; ++nb) {
+            const int ca = 8 * (2 * c) + nb, cb = 8 * (2 * c + 1) + nb;
+            mine[m * 16 + g][ca] = acc[m][nb][0];
+            mine[m * 16 + g][cb] = acc[m][nb][1];
+            mine[m * 16 + g + 8][ca] = acc[m][nb][2];
+            mine[m * 16 + g + 8][cb] = acc[m][nb][3];
+          }
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");
+      for (int idx = threadIdx.x; idx < MB * 16 * 64; idx += STREAM_WARPS * 32) {
+        const int ql = idx / 64, j = idx % 64;
+        if (ql >= R) continue;
+        float v = 0.f;
+#pragma unroll
+        for (int w = 0; w < STREAM_WARPS; ++w) v += red[w][ql][j];
+        float* dst = a.G + ((size_t)slot * R + ql) * a.D + strip * 64 + j;
+        *dst = a.accumulate ? (*dst + v) : v;
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");
+    }
+  }
+}
+
 }  // namespace mlora
