@@ -344,7 +344,7 @@ def main():
         n_launch = per_kind["gemm_fwd"]["launches_per_step"]
         achieved = kernels["gemm_fwd"]["tflops"]
         peak = peaks["bf16_tflops_sustained"]
-        roofline = {"kernel": "gemm_lora_kernel (forward: base GEMM + LoRA expand)", "bound": "tensor",
+        roofline = {"kernel": "gemm2_lora_kernel<R, false> (forward: base GEMM + LoRA expand, two-SM tcgen05)", "bound": "tensor",
                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                     "peak_source": f"{peaks['source']} sustained bf16 ({peak}); burst {peaks['bf16_tflops']}",
                     "frac_of_burst": achieved / peaks["bf16_tflops"],
@@ -421,7 +421,7 @@ def main():
         "roofline": roofline, "kernels": kernels,
     }
     if not args.no_cpu_baseline and world == 1:
-        names = {"cfg3": ["q", "k", "v", "o", "gate"], "cfg2": ["proj4096"], "cfg5": ["mixed"]}[args.workload]
+        names = {"cfg3": ["q", "k", "v", "o", "gate", "up", "down"], "cfg2": ["proj4096"], "cfg5": ["mixed"]}[args.workload]
         line["cpu_baseline"] = cpu_baseline(workloads, names)
     print(json.dumps(line), flush=True)
     if world > 1:

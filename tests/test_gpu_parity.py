@@ -121,6 +121,31 @@ def test_segment_lengths_around_a_tile(sess, lens):
     run_and_check(sess, w, synth.make_tensors(w))
 
 
+@pytest.mark.parametrize("n_rows", [5, 129, 257])
+def test_small_batches(sess, n_rows):
+    """Fewer rows than one tile, and batches that leave the second CTA of a pair tile (almost) empty."""
+    segs = [(0, n_rows // 2, 1, 0), (n_rows // 2, n_rows - n_rows // 2, 0, 1)]
+    w = synth.Workload("small", 192, 320, 16, 2, "bf16", n_rows, synth.segments_array(segs))
+    run_and_check(sess, w, synth.make_tensors(w))
+
+
+def test_gathered_and_contiguous_items(sess):
+    """Rows of one adapter scattered between other rows (gathered shrink items) next to long
+    contiguous segments, with base-only rows inside tiles that have adapters."""
+    segs, row = [], 0
+    for i in range(60):                              # decode-style rows cycling over 5 adapters, some without adapter
+        segs.append((row, 1, (i % 6) - 1, 0))
+        row += 1
+    segs.append((row, 150, 2, 1)); row += 150        # fine-tune segment
+    row += 7                                         # uncovered rows
+    segs.append((row, 90, 4, 0)); row += 90
+    for i in range(40):
+        segs.append((row, 1, i % 5, 0))
+        row += 1
+    w = synth.Workload("mixed_items", 2048, 320, 16, 5, "bf16", row, synth.segments_array(segs))
+    run_and_check(sess, w, synth.make_tensors(w))
+
+
 def test_base_only_rows_and_no_finetune(sess):
     segs = [(0, 40, -1, 0), (60, 30, 1, 0)]      # rows 40..59 and 90..99 uncovered
     w = synth.Workload("base_only", 192, 256, 16, 2, "bf16", 100, synth.segments_array(segs))
