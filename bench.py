@@ -245,6 +245,7 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2607_28848_b200 import binding as mb
+    from paper_2607_28848_b200 import replicas
     from paper_2607_28848_b200.runner import LayerRun, Session
 
     if not torch.cuda.is_available():
@@ -267,8 +268,7 @@ def main():
             r.backward()
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
     warmup = max(args.warmup, 3)
@@ -296,11 +296,7 @@ def main():
     if sampler:
         sampler.mark_stop()
     gpu_launches = mb.mlora_launch_count(sess.ctx) - l0
-    ms_total = ev0.elapsed_time(ev1)
-    if world > 1:
-        tt = torch.tensor([ms_total], device=sess.device)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total = float(tt.item())
+    ms_total = replicas.max_over_ranks(ev0.elapsed_time(ev1), sess.device)     # slowest rank
     # Per-kernel durations: the same steps once more, now with the library recording a CUDA event
     # pair around every launch (which also switches off the overlap of a kernel's set-up with its
     # predecessor's tail, so each pair times one whole kernel).  Kept out of the region above so
@@ -391,11 +387,7 @@ def main():
             e2e_step()
         e1.record()
         barrier()
-        ms_e2e = e0.elapsed_time(e1)
-        if world > 1:
-            tt = torch.tensor([ms_e2e], device=sess.device)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            ms_e2e = float(tt.item())
+        ms_e2e = replicas.max_over_ranks(e0.elapsed_time(e1), sess.device)
         e2e = {"value": world * T * args.e2e_steps / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.e2e_steps, "steps": args.e2e_steps}
 
