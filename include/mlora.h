@@ -159,6 +159,37 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* layer, const 
                               float* dA, float* dB, void* dX_ft, int64_t lddx,
                               int32_t accumulate, void* cuda_stream);
 
+/* ---- optimizer step on the fine-tuned adapters ------------------------------------------*/
+
+/* AdamW hyper-parameters (paper, Section 5 "Fine-tuning Workload": AdamW, learning rate 1e-3,
+ * weight decay 0.01; betas and epsilon are not stated there, the usual 0.9 / 0.999 / 1e-8 are the
+ * documented defaults).  `step` is the 1-based index of this update (bias correction). */
+typedef struct {
+  float lr, beta1, beta2, eps, weight_decay;
+  int32_t step;
+} mlora_adamw_t;
+
+/* Applies one decoupled-weight-decay Adam update to the adapters the plan fine-tunes, consuming
+ * the gradients mlora_backward produced, and rewrites those adapters' rows of A_all and B_all in
+ * place (paper, Section 3.2 "Backward subprocess": optimizer updates are applied directly to the
+ * shared adapter weights):
+ *        w <- w - lr wd w;  m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2;
+ *        w <- w - lr (m / (1-b1^t)) / (sqrt(v / (1-b2^t)) + eps)
+ * All arithmetic is fp32 on fp32 master weights; the layer's stored weights (layer dtype) are the
+ * master weights rounded to nearest even.  One fused, vectorised pass over 30 bytes per element.
+ *   layer     A_all / B_all are WRITTEN for the plan's fine-tuning adapters (only those rows)
+ *   dA, dB    device fp32 [n_slots, rank, d_in] / [n_slots, rank, d_out]   (read)
+ *   wA, wB    device fp32 master weights, same shapes, slot-indexed        (read + written)
+ *   mA, vA, mB, vB  device fp32 first / second moments, same shapes        (read + written)
+ * Slot g belongs to adapter mlora_plan_ft_adapters()[g].  The caller initialises the master
+ * weights from the adapters once and zeroes the moments.  A plan without fine-tuning rows makes
+ * this a no-op.  Errors: MLORA_ERR_INVALID_ARG (null pointers, step < 1, betas outside [0,1)),
+ * MLORA_ERR_ADAPTER_ID, MLORA_ERR_CUDA.  Asynchronous on the stream; allocates nothing. */
+mlora_status_t mlora_adamw_update(mlora_ctx* ctx, const mlora_layer_t* layer, const mlora_plan* plan,
+                                  const float* dA, const float* dB, float* wA, float* wB,
+                                  float* mA, float* vA, float* mB, float* vB,
+                                  const mlora_adamw_t* hp, void* cuda_stream);
+
 /* ---- status / diagnostics --------------------------------------------------------------*/
 
 /* Synchronises the stream and returns the device status word: MLORA_OK, or
@@ -175,7 +206,7 @@ int64_t mlora_launch_count(const mlora_ctx* ctx);
  * of this context record one pair around itself on the launching stream, until the pairs run
  * out; n = 0 switches recording off and frees the events.  mlora_profile_collect synchronises
  * the device, writes for each recorded launch its kind (0 shrink, 1 forward GEMM, 2 input-gradient
- * GEMM, 3 gradient kernel, 4 CUDA-core kernels) and its duration in milliseconds into the host
+ * GEMM, 3 gradient kernel, 4 CUDA-core kernels, 5 optimizer update) and its duration in milliseconds into the host
  * arrays (up to cap entries), forgets the records and returns how many there were. */
 mlora_status_t mlora_profile_enable(mlora_ctx* ctx, int32_t max_records);
 int32_t mlora_profile_collect(mlora_ctx* ctx, int32_t* kinds, float* ms, int32_t cap);

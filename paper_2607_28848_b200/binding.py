@@ -23,7 +23,7 @@ EXPORTS = (
     "mlora_create", "mlora_destroy", "mlora_plan_create", "mlora_plan_destroy", "mlora_plan_rows",
     "mlora_plan_ft_rows", "mlora_plan_ft_adapters", "mlora_plan_describe", "mlora_mixed_forward",
     "mlora_backward", "mlora_poll_status", "mlora_status_string", "mlora_launch_count", "mlora_set_gemm_path",
-    "mlora_profile_enable", "mlora_profile_collect", "mlora_forward_noalloc",
+    "mlora_profile_enable", "mlora_profile_collect", "mlora_forward_noalloc", "mlora_adamw_update",
 )
 MLORA_NOALLOC_MAX_ROWS = 512
 
@@ -38,6 +38,11 @@ class mlora_layer_t(ctypes.Structure):
                 ("n_adapters", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("W", ctypes.c_void_p), ("ldw", ctypes.c_int64),
                 ("A_all", ctypes.c_void_p), ("B_all", ctypes.c_void_p), ("scale", ctypes.c_void_p)]
+
+
+class mlora_adamw_t(ctypes.Structure):
+    _fields_ = [("lr", ctypes.c_float), ("beta1", ctypes.c_float), ("beta2", ctypes.c_float),
+                ("eps", ctypes.c_float), ("weight_decay", ctypes.c_float), ("step", ctypes.c_int32)]
 
 
 class MloraError(RuntimeError):
@@ -95,6 +100,8 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.mlora_profile_enable.restype = ctypes.c_int
     lib.mlora_profile_collect.argtypes = [vp, P(i32), P(ctypes.c_float), i32]
     lib.mlora_profile_collect.restype = i32
+    lib.mlora_adamw_update.argtypes = [vp, P(mlora_layer_t), vp, vp, vp, vp, vp, vp, vp, vp, vp, P(mlora_adamw_t), vp]
+    lib.mlora_adamw_update.restype = ctypes.c_int
     lib.mlora_forward_noalloc.argtypes = [P(mlora_layer_t), vp, i32, vp, i64, vp, i64, vp]
     lib.mlora_forward_noalloc.restype = ctypes.c_int
     _lib = lib
@@ -225,7 +232,18 @@ def mlora_set_gemm_path(ctx, path: int) -> None:
     _check(load_library().mlora_set_gemm_path(ctx, int(path)), "mlora_set_gemm_path")
 
 
-PROFILE_KINDS = ("shrink", "gemm_fwd", "gemm_bwd", "grad", "simt")
+PROFILE_KINDS = ("shrink", "gemm_fwd", "gemm_bwd", "grad", "simt", "adamw")
+
+
+def mlora_adamw_update(ctx, layer: mlora_layer_t, plan, dA, dB, wA, wB, mA, vA, mB, vB, step: int, lr: float = 1e-3,
+                       beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, weight_decay: float = 0.01,
+                       stream=None) -> None:
+    """Queue one AdamW update of the plan's fine-tuning adapters (all tensors fp32 CUDA, slot-indexed)."""
+    hp = mlora_adamw_t(lr, beta1, beta2, eps, weight_decay, int(step))
+    st = load_library().mlora_adamw_update(ctx, ctypes.byref(layer), plan, _ptr(dA), _ptr(dB), _ptr(wA), _ptr(wB),
+                                           _ptr(mA), _ptr(vA), _ptr(mB), _ptr(vB), ctypes.byref(hp),
+                                           _stream_ptr(stream))
+    _check(st, "mlora_adamw_update")
 
 
 def mlora_profile_enable(ctx, max_records: int) -> None:

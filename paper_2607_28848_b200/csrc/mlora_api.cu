@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
@@ -49,7 +50,7 @@ struct mlora_ctx {
 
 constexpr int kMaxKSplit = 16;
 
-enum { KIND_SHRINK = 0, KIND_GEMM_FWD = 1, KIND_GEMM_BWD = 2, KIND_GRAD = 3, KIND_SIMT = 4 };
+enum { KIND_SHRINK = 0, KIND_GEMM_FWD = 1, KIND_GEMM_BWD = 2, KIND_GRAD = 3, KIND_SIMT = 4, KIND_ADAMW = 5 };
 
 // Device copy of one RowSpace.
 struct DevRowSpace {
@@ -829,6 +830,37 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   if (!dX) return MLORA_OK;
   return gemm_bf16<true>(ctx, L, h.bwd, p->bwd, dY, lddy, dX, lddx, L->A_all, ctx->ws_p, nullptr, h.ft_rows, L->d_in,
                          L->d_out, st);
+}
+
+mlora_status_t mlora_adamw_update(mlora_ctx* ctx, const mlora_layer_t* L, const mlora_plan* p, const float* dA,
+                                  const float* dB, float* wA, float* wB, float* mA, float* vA, float* mB, float* vB,
+                                  const mlora_adamw_t* hp, void* cuda_stream) {
+  if (!ctx || !p || p->ctx != ctx || !p->blob || !hp) return MLORA_ERR_INVALID_ARG;
+  mlora_status_t s = check_layer(L);
+  if (s != MLORA_OK) return s;
+  const HostPlan& h = p->h;
+  if (h.n_adapters > L->n_adapters) return MLORA_ERR_ADAPTER_ID;
+  if (hp->step < 1 || !(hp->beta1 >= 0.f && hp->beta1 < 1.f) || !(hp->beta2 >= 0.f && hp->beta2 < 1.f))
+    return MLORA_ERR_INVALID_ARG;
+  const int n_slots = (int)h.ft_adapters.size();
+  if (n_slots == 0) return MLORA_OK;
+  if (!dA || !dB || !wA || !wB || !mA || !vA || !mB || !vB) return MLORA_ERR_INVALID_ARG;
+  if (L->d_in % 4 || L->d_out % 4) return MLORA_ERR_UNSUPPORTED;
+  simt::AdamwArgs a;
+  a.side[0] = simt::AdamwSide{dA, wA, mA, vA, const_cast<void*>(L->A_all), L->d_in};
+  a.side[1] = simt::AdamwSide{dB, wB, mB, vB, const_cast<void*>(L->B_all), L->d_out};
+  a.slot_adapter = p->slot_adapter; a.n_slots = n_slots; a.R = L->rank;
+  a.lr = hp->lr; a.beta1 = hp->beta1; a.beta2 = hp->beta2; a.eps = hp->eps; a.wd = hp->weight_decay;
+  a.inv_bc1 = (float)(1.0 / (1.0 - pow((double)hp->beta1, (double)hp->step)));
+  a.inv_bc2 = (float)(1.0 / (1.0 - pow((double)hp->beta2, (double)hp->step)));
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const int64_t widest = (int64_t)n_slots * L->rank * (L->d_in > L->d_out ? L->d_in : L->d_out) / 4;
+  int blocks = (int)((widest + 255) / 256);
+  blocks = blocks < 4 * ctx->sm_count ? blocks : 4 * ctx->sm_count;
+  LaunchScope scope(ctx, st, KIND_ADAMW);
+  if (L->dtype == MLORA_F32) simt::adamw_kernel<float><<<dim3(blocks, 2), 256, 0, st>>>(a);
+  else simt::adamw_kernel<__nv_bfloat16><<<dim3(blocks, 2), 256, 0, st>>>(a);
+  return scope.done();
 }
 
 mlora_status_t mlora_poll_status(mlora_ctx* ctx, void* cuda_stream) {

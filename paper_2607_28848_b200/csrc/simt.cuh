@@ -102,5 +102,54 @@ __global__ void grad_kernel(const float* P, int R, const float* scale, const T* 
   *dst = accumulate ? *dst + acc : acc;
 }
 
+// One AdamW update of the adapters of the fine-tuning slots; element i of slot g, rank row q,
+// column j.  `which` = blockIdx.y: 0 -> the A matrices (width d_in), 1 -> the B matrices (d_out).
+struct AdamwSide {
+  const float* grad;   // [n_slots, R, D]
+  float* master;       // [n_slots, R, D]
+  float* m;
+  float* v;
+  void* weights;       // [n_adapters, R, D] in the layer's storage type
+  int32_t D;
+};
+struct AdamwArgs {
+  AdamwSide side[2];
+  const int32_t* slot_adapter;
+  int32_t n_slots, R;
+  float lr, beta1, beta2, eps, wd, inv_bc1, inv_bc2;   // inv_bc = 1 / (1 - beta^t)
+};
+
+template <typename T>
+__global__ void adamw_kernel(const AdamwArgs a) {
+  const AdamwSide& s = a.side[blockIdx.y];
+  const int64_t per_slot = (int64_t)a.R * s.D;
+  const int64_t total4 = (int64_t)a.n_slots * per_slot / 4;           // D is a multiple of 4
+  for (int64_t i4 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i4 < total4; i4 += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t i = i4 * 4;
+    const int slot = (int)(i / per_slot);
+    const int64_t off = i - (int64_t)slot * per_slot;
+    const float4 g = *reinterpret_cast<const float4*>(s.grad + i);
+    float4 w = *reinterpret_cast<const float4*>(s.master + i);
+    float4 m = *reinterpret_cast<const float4*>(s.m + i);
+    float4 v = *reinterpret_cast<const float4*>(s.v + i);
+    float* gw = reinterpret_cast<float*>(const_cast<float4*>(&g));
+    float *pw = reinterpret_cast<float*>(&w), *pm = reinterpret_cast<float*>(&m), *pv = reinterpret_cast<float*>(&v);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      float wk = pw[k] - a.lr * a.wd * pw[k];
+      const float mk = a.beta1 * pm[k] + (1.0f - a.beta1) * gw[k];
+      const float vk = a.beta2 * pv[k] + (1.0f - a.beta2) * gw[k] * gw[k];
+      wk -= a.lr * (mk * a.inv_bc1) / (sqrtf(vk * a.inv_bc2) + a.eps);
+      pw[k] = wk; pm[k] = mk; pv[k] = vk;
+    }
+    *reinterpret_cast<float4*>(s.master + i) = w;
+    *reinterpret_cast<float4*>(s.m + i) = m;
+    *reinterpret_cast<float4*>(s.v + i) = v;
+    T* dst = reinterpret_cast<T*>(s.weights) + (int64_t)a.slot_adapter[slot] * per_slot + off;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) st(dst + k, pw[k]);
+  }
+}
+
 }  // namespace simt
 }  // namespace mlora
