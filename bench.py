@@ -228,6 +228,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=10, help="0 skips the end-to-end leg")
     ap.add_argument("--projections", default="", help="comma list: run only these projections of the workload")
+    ap.add_argument("--with-update", action="store_true",
+                    help="also run the AdamW update of the fine-tuned adapters after each backward (not part of the "
+                         "headline step; reported under kernels.adamw)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -262,10 +265,24 @@ def main():
         del t
     resident = sum(w.d_in * w.d_out * w.elem_bytes + w.n_rows * (w.d_in + w.d_out) * w.elem_bytes for w in workloads)
 
-    def step():
+    opt = []
+    if args.with_update:
         for r in runs:
+            idx = torch.tensor(r.slots, device=sess.device)
+            wA, wB = r.A_all[idx].float().contiguous(), r.B_all[idx].float().contiguous()
+            opt.append([wA, wB] + [torch.zeros_like(x) for x in (wA, wA, wB, wB)])
+    n_updates = [0]
+
+    def step():
+        if args.with_update:
+            n_updates[0] += 1
+        for i, r in enumerate(runs):
             r.forward()
             r.backward()
+            if args.with_update:
+                wA, wB, mA, vA, mB, vB = opt[i]
+                mb.mlora_adamw_update(sess.ctx, r.layer, r.plan, r.dA, r.dB, wA, wB, mA, vA, mB, vB, n_updates[0],
+                                      lr=1e-6)
 
     def barrier():
         replicas.barrier()
@@ -335,6 +352,10 @@ def main():
     if "grad" in per_kind:
         b = sum(a["grad_dA"] + a["grad_dB"] for a in ab)
         kernels["grad"] = {**per_kind["grad"], "gbs": b / per_kind["grad"]["ms_per_step"] / 1e6}
+    if "adamw" in per_kind:
+        b = sum(30.0 * len(r.slots) * w.rank * (w.d_in + w.d_out) for r, w in zip(runs, workloads))
+        kernels["adamw"] = {**per_kind["adamw"], "gbs": b / per_kind["adamw"]["ms_per_step"] / 1e6,
+                            "note": "30 bytes per adapter element: grad, weight, two moments read; weight, moments, stored weight written"}
     roofline = None
     if "gemm_fwd" in kernels:
         n_launch = per_kind["gemm_fwd"]["launches_per_step"]
