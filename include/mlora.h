@@ -61,7 +61,8 @@ typedef enum {
   MLORA_ERR_UNSUPPORTED = 6,     /* shape / rank / alignment outside what the kernels handle    */
   MLORA_ERR_ARCH = 7,            /* no CUDA device of compute capability 10.x                   */
   MLORA_ERR_CUDA = 8,            /* a CUDA runtime or driver call failed                        */
-  MLORA_ERR_DEVICE_TIMEOUT = 9   /* a bounded wait inside a kernel ran out (see poll_status)    */
+  MLORA_ERR_DEVICE_TIMEOUT = 9,  /* a bounded wait inside a kernel ran out (see poll_status)    */
+  MLORA_CANCELLED = 10           /* the caller's cancel flag was raised; the call stopped early */
 } mlora_status_t;
 
 /* One projection.  dtype is the storage type of X, W, A, B, Y, dY, dX and x_save.
@@ -158,6 +159,21 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* layer, const 
                               const void* x_save, const float* u_save,
                               float* dA, float* dB, void* dX_ft, int64_t lddx,
                               int32_t accumulate, void* cuda_stream);
+
+/* ---- cooperative cancellation --------------------------------------------------------------*/
+
+/* Registers a HOST flag (for example a word in pinned or ordinary host memory that another
+ * thread writes) that mlora_mixed_forward, mlora_backward and mlora_adamw_update read before each
+ * kernel they launch; NULL unregisters.  When it is non-zero the call launches nothing further and
+ * returns MLORA_CANCELLED.  Kernels already queued still run to completion, so the GPU is free
+ * within one kernel's time; the outputs of the interrupted call are incomplete and the caller
+ * drops them (for a forward: do not advance save_row_base, so the partial activations are
+ * overwritten by the next step; the interrupted rows go back to the caller's pool).
+ * (Paper, Section 4 "Backward preemption" and "Fine-tuning forward interruption": a grant flag /
+ * abort signal polled at layer boundaries, discarding partial activations.  Here the boundary is
+ * finer - between the two to four kernels of one projection - and the flag is read on the host,
+ * which learns of the request before its next launch, so no kernel ever waits on it.) */
+mlora_status_t mlora_set_cancel_flag(mlora_ctx* ctx, const volatile int32_t* host_flag);
 
 /* ---- optimizer step on the fine-tuned adapters ------------------------------------------*/
 

@@ -17,13 +17,15 @@ LIB_PATH = os.path.join(_PKG_DIR, "libmlora.so")
 
 MLORA_F32, MLORA_BF16 = 0, 1
 (MLORA_OK, MLORA_ERR_INVALID_ARG, MLORA_ERR_SEGMENT_RANGE, MLORA_ERR_SEGMENT_OVERLAP, MLORA_ERR_ADAPTER_ID,
- MLORA_ERR_SAVE_CAPACITY, MLORA_ERR_UNSUPPORTED, MLORA_ERR_ARCH, MLORA_ERR_CUDA, MLORA_ERR_DEVICE_TIMEOUT) = range(10)
+ MLORA_ERR_SAVE_CAPACITY, MLORA_ERR_UNSUPPORTED, MLORA_ERR_ARCH, MLORA_ERR_CUDA, MLORA_ERR_DEVICE_TIMEOUT,
+ MLORA_CANCELLED) = range(11)
 
 EXPORTS = (
     "mlora_create", "mlora_destroy", "mlora_plan_create", "mlora_plan_destroy", "mlora_plan_rows",
     "mlora_plan_ft_rows", "mlora_plan_ft_adapters", "mlora_plan_describe", "mlora_mixed_forward",
     "mlora_backward", "mlora_poll_status", "mlora_status_string", "mlora_launch_count", "mlora_set_gemm_path",
     "mlora_profile_enable", "mlora_profile_collect", "mlora_forward_noalloc", "mlora_adamw_update",
+    "mlora_set_cancel_flag",
 )
 MLORA_NOALLOC_MAX_ROWS = 512
 
@@ -102,6 +104,8 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.mlora_profile_collect.restype = i32
     lib.mlora_adamw_update.argtypes = [vp, P(mlora_layer_t), vp, vp, vp, vp, vp, vp, vp, vp, vp, P(mlora_adamw_t), vp]
     lib.mlora_adamw_update.restype = ctypes.c_int
+    lib.mlora_set_cancel_flag.argtypes = [vp, P(i32)]
+    lib.mlora_set_cancel_flag.restype = ctypes.c_int
     lib.mlora_forward_noalloc.argtypes = [P(mlora_layer_t), vp, i32, vp, i64, vp, i64, vp]
     lib.mlora_forward_noalloc.restype = ctypes.c_int
     _lib = lib
@@ -272,3 +276,9 @@ def mlora_forward_noalloc(layer: mlora_layer_t, row_adapter, X, Y, stream=None) 
     st = load_library().mlora_forward_noalloc(ctypes.byref(layer), _ptr(row_adapter), n_rows, _ptr(X),
                                               X.stride(0), _ptr(Y), Y.stride(0), _stream_ptr(stream))
     _check(st, "mlora_forward_noalloc")
+
+
+def mlora_set_cancel_flag(ctx, flag) -> None:
+    """Register a host flag (a ctypes.c_int32 the caller keeps alive, or None) checked before every launch."""
+    ptr = None if flag is None else ctypes.pointer(flag)
+    _check(load_library().mlora_set_cancel_flag(ctx, ptr), "mlora_set_cancel_flag")

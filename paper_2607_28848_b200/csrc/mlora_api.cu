@@ -42,6 +42,7 @@ struct mlora_ctx {
   int32_t shrink_path = 0;           // 0: streaming kernel for rank <= 32; 1: per-item kernel for every rank
   int32_t gemm_pairs = 1;            // 1: two-SM (CTA pair) tensor-core kernel; 0: one-SM kernel
   EncodeTiledFn encode = nullptr;
+  const volatile int32_t* cancel = nullptr;   // caller's host flag, read before every launch
   // optional per-launch timing
   std::vector<cudaEvent_t> ev_start, ev_stop;
   std::vector<int32_t> ev_kind;
@@ -142,6 +143,8 @@ mlora_status_t check_layer(const mlora_layer_t* L) {
   return MLORA_OK;
 }
 
+inline bool cancelled(const mlora_ctx* c) { return c->cancel && *c->cancel != 0; }
+
 // Brackets one kernel launch: optional event pair, launch counter, launch-error check.
 struct LaunchScope {
   mlora_ctx* ctx; cudaStream_t st; int slot;
@@ -231,6 +234,7 @@ mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, c
   int grid = sa.n_units < ctx->sm_count ? sa.n_units : ctx->sm_count;
   sa.units_per_cta = (sa.n_units + grid - 1) / grid;
   grid = (sa.n_units + sa.units_per_cta - 1) / sa.units_per_cta;
+  if (cancelled(ctx)) return MLORA_CANCELLED;
   if (2 * (int64_t)grid > ctx->ws_partial_items || n_items > ctx->ws_counter_items) return MLORA_ERR_INVALID_ARG;
   LaunchScope scope(ctx, st, KIND_SHRINK);
   sa.status = ctx->status_dev;
@@ -247,6 +251,7 @@ mlora_status_t launch_shrink(mlora_ctx* ctx, int R, ShrinkArgs a, int n_items, c
     if (R == 16) return launch_shrink_stream<2, 2, 16>(ctx, a, n_items, item_contig, n_rows, n_adapters, st);
     if (R == 32) return launch_shrink_stream<4, 3, 8>(ctx, a, n_items, item_contig, n_rows, n_adapters, st);
   }
+  if (cancelled(ctx)) return MLORA_CANCELLED;
   const int ksplit = shrink_ksplit(ctx, n_items, a.D);
   a.partial = ctx->ws_partial;
   a.counters = ctx->ws_counters;
@@ -282,6 +287,7 @@ mlora_status_t launch_grad_stream(mlora_ctx* ctx, const mlora_plan* p, const Gra
   ga.n_slots = n_slots; ga.n_strips = a.D / 64; ga.status = ctx->status_dev;
   const int groups = n_slots * ga.n_strips;
   const int grid = groups < ctx->sm_count ? groups : ctx->sm_count;
+  if (cancelled(ctx)) return MLORA_CANCELLED;
   LaunchScope scope(ctx, st, KIND_GRAD);
   launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(STREAM_THREADS), smem, st, tQ, ga);
   return scope.done();
@@ -294,6 +300,7 @@ mlora_status_t launch_grad(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& 
     if (a.R <= 16) return launch_grad_stream<1>(ctx, p, a, n_slots, n_rows, st);
     if (a.R <= 32) return launch_grad_stream<2>(ctx, p, a, n_slots, n_rows, st);
   }
+  if (cancelled(ctx)) return MLORA_CANCELLED;
   constexpr int smem1 = (GRAD_THREADS / 32) * 16 * 65 * 4, smem2 = 2 * smem1;
   static bool attr_set = false;
   if (!attr_set) {
@@ -320,6 +327,7 @@ mlora_status_t launch_gemm_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUten
       return MLORA_ERR_CUDA;
     attr_set = true;
   }
+  if (cancelled(ctx)) return MLORA_CANCELLED;
   const int grid = g.n_units < ctx->sm_count ? g.n_units : ctx->sm_count;
   LaunchScope scope(ctx, st, W_KMAJOR ? KIND_GEMM_BWD : KIND_GEMM_FWD);
   launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(GEMM_THREADS), GEMM_SMEM_BYTES, st, tIn, tW, tL, tOut, g);
@@ -345,6 +353,7 @@ mlora_status_t launch_gemm2_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUte
     if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) { cudaGetLastError(); return MLORA_ERR_CUDA; }
     max_pairs = n;
   }
+  if (cancelled(ctx)) return MLORA_CANCELLED;
   const int pairs = g.n_units < max_pairs ? g.n_units : max_pairs;
   LaunchScope scope(ctx, st, W_KMAJOR ? KIND_GEMM_BWD : KIND_GEMM_FWD);
   launch_pdl_pairs(scope.slot < 0, kern, dim3(2 * pairs), dim3(GEMM2_THREADS), GEMM2_SMEM_BYTES, st, tIn, tW, tL, tOut, tPbd, g);
@@ -435,6 +444,7 @@ mlora_status_t simt_shrink(mlora_ctx* ctx, const T* In, int64_t ld_in, int D, in
                            const float* scale, const DevRowSpace& ds, float* Out, T* x_save, float* u_save,
                            int64_t save_base, int n_rows, cudaStream_t st) {
   if (n_rows <= 0) return MLORA_OK;
+  if (cancelled(ctx)) return MLORA_CANCELLED;
   const int64_t warps = (int64_t)n_rows * R;
   const int blocks = (int)((warps * 32 + 255) / 256);
   LaunchScope scope(ctx, st, KIND_SIMT);
@@ -448,6 +458,7 @@ mlora_status_t simt_gemm(mlora_ctx* ctx, const T* In, int64_t ld_in, const T* W,
                          const float* P, const float* scale, const DevRowSpace& ds, T* Out, int64_t ld_out, int M,
                          int N, int K, int R, cudaStream_t st) {
   if (M <= 0) return MLORA_OK;
+  if (cancelled(ctx)) return MLORA_CANCELLED;
   dim3 grid((N + 31) / 32, (M + 31) / 32), block(32, 32);
   LaunchScope scope(ctx, st, KIND_SIMT);
   simt::gemm_lora_kernel<T, W_KMAJOR><<<grid, block, 0, st>>>(In, ld_in, W, ldw, L_all, P, scale, ds.row_adapter, Out,
@@ -460,6 +471,7 @@ mlora_status_t simt_grad(mlora_ctx* ctx, const mlora_plan* p, const float* P, in
                          int64_t ldq, int D, float* G, int accumulate, cudaStream_t st) {
   const int n_slots = (int)p->h.ft_adapters.size();
   if (n_slots <= 0) return MLORA_OK;
+  if (cancelled(ctx)) return MLORA_CANCELLED;
   dim3 grid((D + 127) / 128, R, n_slots);
   LaunchScope scope(ctx, st, KIND_SIMT);
   simt::grad_kernel<T><<<grid, 128, 0, st>>>(P, R, scale, Q, ldq, D, G, p->slot_chunk_off, p->chunk_row0,
@@ -574,6 +586,7 @@ const char* mlora_status_string(mlora_status_t s) {
     case MLORA_ERR_ARCH: return "no sm_100 CUDA device";
     case MLORA_ERR_CUDA: return "CUDA call failed";
     case MLORA_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case MLORA_CANCELLED: return "cancelled by the caller's flag";
   }
   return "unknown status";
 }
@@ -853,6 +866,7 @@ mlora_status_t mlora_adamw_update(mlora_ctx* ctx, const mlora_layer_t* L, const 
   a.lr = hp->lr; a.beta1 = hp->beta1; a.beta2 = hp->beta2; a.eps = hp->eps; a.wd = hp->weight_decay;
   a.inv_bc1 = (float)(1.0 / (1.0 - pow((double)hp->beta1, (double)hp->step)));
   a.inv_bc2 = (float)(1.0 / (1.0 - pow((double)hp->beta2, (double)hp->step)));
+  if (cancelled(ctx)) return MLORA_CANCELLED;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   const int64_t widest = (int64_t)n_slots * L->rank * (L->d_in > L->d_out ? L->d_in : L->d_out) / 4;
   int blocks = (int)((widest + 255) / 256);
@@ -874,6 +888,12 @@ mlora_status_t mlora_poll_status(mlora_ctx* ctx, void* cuda_stream) {
     cudaStreamSynchronize(st);
   }
   return (mlora_status_t)v;
+}
+
+mlora_status_t mlora_set_cancel_flag(mlora_ctx* ctx, const volatile int32_t* host_flag) {
+  if (!ctx) return MLORA_ERR_INVALID_ARG;
+  ctx->cancel = host_flag;
+  return MLORA_OK;
 }
 
 int64_t mlora_launch_count(const mlora_ctx* ctx) { return ctx ? ctx->launches : 0; }

@@ -27,7 +27,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_status_strings():
-    for s in range(10):
+    for s in range(11):
         assert mb.status_string(s) and mb.status_string(s) != "unknown status"
     assert mb.status_string(99) == "unknown status"
 

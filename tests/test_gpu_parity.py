@@ -303,6 +303,38 @@ def test_argument_errors_launch_nothing(sess):
     run.close()
 
 
+def test_cancel_flag_stops_between_kernels(sess):
+    """The caller's host flag is read before every launch: once raised, a call launches nothing
+    more and reports MLORA_CANCELLED; once lowered, the same step runs normally (the interrupted
+    step is simply repeated, its partial activations overwritten)."""
+    import ctypes
+    w = synth.random_workload(25, 128, 192, 16, 3, 200, max_seg=60, p_finetune=0.5)
+    t = synth.make_tensors(w)
+    run = LayerRun(sess, "bf16", t, w.segments, w.n_rows)
+    run.forward()
+    run.backward()
+    ref = [x.clone() for x in (run.Y, run.u_save, run.dA, run.dB, run.dX)]
+    flag = ctypes.c_int32(0)
+    mb.mlora_set_cancel_flag(sess.ctx, flag)
+    try:
+        flag.value = 1
+        before = mb.mlora_launch_count(sess.ctx)
+        for call in (run.forward, run.backward):
+            with pytest.raises(mb.MloraError) as e:
+                call()
+            assert e.value.status == mb.MLORA_CANCELLED
+        assert mb.mlora_launch_count(sess.ctx) == before
+        flag.value = 0
+        run.Y.zero_()
+        run.forward()
+        run.backward()
+        for a, b in zip(ref, (run.Y, run.u_save, run.dA, run.dB, run.dX)):
+            assert torch.equal(a, b)
+    finally:
+        mb.mlora_set_cancel_flag(sess.ctx, None)
+    run.close()
+
+
 # ---- full-size configurations --------------------------------------------------------------
 def test_cfg2_full_size(sess):
     w = synth.cfg2_single_projection()
