@@ -322,6 +322,24 @@ def main():
         b = sum(30.0 * len(r.slots) * w.rank * (w.d_in + w.d_out) for r, w in zip(runs, workloads))
         kernels["adamw"] = {**per_kind["adamw"], "gbs": b / per_kind["adamw"]["ms_per_step"] / 1e6,
                             "note": "30 bytes per adapter element: grad, weight, two moments read; weight, moments, stored weight written"}
+    # per-launch view of the memory-bound kernels: which launch is which follows from the fixed order
+    # shrink(fwd), GEMM fwd, shrink(bwd), grad dB, grad dA, GEMM bwd [, update] per projection
+    per_step = len(kms) // prof_steps if prof_steps else 0
+    labels = []
+    for w, a_ in zip(workloads, ab):
+        labels += [(w.name, "shrink_fwd", a_["shrink_fwd"]), (w.name, "gemm_fwd", None), (w.name, "shrink_bwd", a_["shrink_bwd"]),
+                   (w.name, "grad_dB", a_["grad_dB"]), (w.name, "grad_dA", a_["grad_dA"]), (w.name, "gemm_bwd", None)]
+        if args.with_update:
+            labels.append((w.name, "adamw", None))
+    skinny = []
+    if per_step == len(labels) and per_step > 0:
+        mean_ms = kms[:per_step * prof_steps].reshape(prof_steps, per_step).mean(0)
+        for (proj, kern, nbytes), t in zip(labels, mean_ms):
+            if nbytes:
+                skinny.append({"launch": f"{proj}:{kern}", "mbytes": nbytes / 1e6, "us": float(t * 1e3),
+                               "gbs": nbytes / t / 1e6, "frac_hbm": nbytes / t / 1e6 / peaks["hbm_gbs"]})
+        skinny.sort(key=lambda d: -d["mbytes"])
+        kernels["skinny_largest_launches"] = skinny[:4]
     roofline = None
     if "gemm_fwd" in kernels:
         n_launch = per_kind["gemm_fwd"]["launches_per_step"]

@@ -190,6 +190,39 @@ def test_integer_probe_bit_exact(sess, dtype):
         run.close()
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_random_tables_route_bit_exactly(sess, seed):
+    """Random valid segment tables (ragged lengths, single rows, gaps, adapter -1, shuffled order,
+    several fine-tune segments per adapter) on the exact-integer probe: every output must equal the
+    oracle bit for bit, so any mis-routed row, wrong scale or mis-indexed save row shows."""
+    rng = np.random.default_rng(seed)
+    n_rows = int(rng.integers(1, 700))
+    n_adapters = int(rng.integers(1, 40))
+    rank = int(rng.choice([8, 16, 32]))
+    d_in, d_out = int(rng.choice([64, 128, 192])), int(rng.choice([64, 256, 320]))
+    p = integer_probe(n_rows=n_rows, d_in=d_in, d_out=d_out, rank=rank, n_adapters=n_adapters, seed=100 + seed,
+                      max_seg=int(rng.integers(2, 300)))
+    fwd = orc.forward(p["X"], p["W"], p["A_all"], p["B_all"], p["scale"], p["segments"])
+    run = LayerRun(sess, "bf16", p, p["segments"], n_rows, guard=True)
+    try:
+        run.forward()
+        assert run.status() == mb.MLORA_OK
+        n = run.ft_rows
+        assert n == fwd["ft_rows"] and run.slots == fwd["ft_adapters"]
+        assert np.array_equal(run.host(run.Y), fwd["Y"])
+        assert np.array_equal(run.host(run.x_save)[:n], fwd["x_save"])
+        assert np.array_equal(run.host(run.u_save)[:n], fwd["u_save"])
+        if n:
+            run.backward()
+            bwd = orc.backward(p["dY"], p["W"], p["A_all"], p["B_all"], p["scale"], p["segments"], fwd["x_save"],
+                               fwd["u_save"], n_rows=n_rows)
+            assert np.array_equal(run.host(run.dX)[:n], bwd["dX"])
+            assert np.array_equal(run.host(run.dA), bwd["dA"])
+            assert np.array_equal(run.host(run.dB), bwd["dB"])
+    finally:
+        run.close()
+
+
 def test_append_two_steps_then_one_backward(sess):
     """Two forward steps append into one activation buffer; one backward consumes both
     (activations accumulate until a backward batch is full)."""
