@@ -1,0 +1,53 @@
+"""Forward (with activation save) and backward captured in a CUDA graph and replayed.
+
+The paper's co-serving step has to run eagerly because its activation capture lives in Python
+hooks that cannot run inside a replayed graph (Section 4, "Execution-mode coefficients").  Here the
+save is part of a kernel, the calls allocate nothing and never synchronise, so a whole
+forward + backward + update can be captured once and replayed on new inputs."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_28848_b200 import binding as mb
+from paper_2607_28848_b200 import synth
+from paper_2607_28848_b200.runner import LayerRun, Session
+
+pytestmark = pytest.mark.gpu
+
+
+def test_graph_replay_matches_eager_on_new_inputs():
+    with Session(0) as sess:
+        w = synth.random_workload(61, 256, 384, 16, 5, 420, max_seg=130, p_finetune=0.4)
+        t = synth.make_tensors(w)
+        run = LayerRun(sess, "bf16", t, w.segments, w.n_rows)
+        dev = sess.device
+        stream = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(stream):
+            for _ in range(2):                      # warm-up: one-time function attributes are set here
+                run.forward()
+                run.backward()
+            stream.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                run.forward()
+                run.backward()
+            # new inputs in the same buffers
+            x2 = torch.from_numpy(synth.round_to_bf16(synth.normal(5, 1, run.X.numel()).reshape(run.X.shape))).to(dev).to(torch.bfloat16)
+            dy2 = torch.from_numpy(synth.round_to_bf16(synth.normal(5, 2, run.dY.numel()).reshape(run.dY.shape))).to(dev).to(torch.bfloat16)
+            run.X.copy_(x2)
+            run.dY.copy_(dy2)
+            for buf in (run.Y, run.x_save, run.u_save, run.dA, run.dB, run.dX):
+                buf.zero_()
+            graph.replay()
+            stream.synchronize()
+            replayed = [b.clone() for b in (run.Y, run.x_save, run.u_save, run.dA, run.dB, run.dX)]
+            for buf in (run.Y, run.x_save, run.u_save, run.dA, run.dB, run.dX):
+                buf.zero_()
+            run.forward()
+            run.backward()
+            stream.synchronize()
+        assert mb.mlora_poll_status(sess.ctx) == mb.MLORA_OK
+        for a, b in zip(replayed, (run.Y, run.x_save, run.u_save, run.dA, run.dB, run.dX)):
+            assert torch.equal(a, b)
+        assert float(run.Y.float().abs().max()) > 0
+        run.close()
