@@ -323,12 +323,12 @@ def main():
         kernels["adamw"] = {**per_kind["adamw"], "gbs": b / per_kind["adamw"]["ms_per_step"] / 1e6,
                             "note": "30 bytes per adapter element: grad, weight, two moments read; weight, moments, stored weight written"}
     # per-launch view of the memory-bound kernels: which launch is which follows from the fixed order
-    # shrink(fwd), GEMM fwd, shrink(bwd), grad dB, grad dA, GEMM bwd [, update] per projection
+    # shrink(fwd), GEMM fwd, shrink(bwd), gradients (dB and dA in one launch), GEMM bwd [, update] per projection
     per_step = len(kms) // prof_steps if prof_steps else 0
     labels = []
     for w, a_ in zip(workloads, ab):
         labels += [(w.name, "shrink_fwd", a_["shrink_fwd"]), (w.name, "gemm_fwd", None), (w.name, "shrink_bwd", a_["shrink_bwd"]),
-                   (w.name, "grad_dB", a_["grad_dB"]), (w.name, "grad_dA", a_["grad_dA"]), (w.name, "gemm_bwd", None)]
+                   (w.name, "grad_dB+dA", a_["grad_dB"] + a_["grad_dA"]), (w.name, "gemm_bwd", None)]
         if args.with_update:
             labels.append((w.name, "adamw", None))
     skinny = []

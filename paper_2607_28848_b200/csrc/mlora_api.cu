@@ -268,9 +268,10 @@ mlora_status_t launch_shrink(mlora_ctx* ctx, int R, ShrinkArgs a, int n_items, c
   return scope.done();
 }
 
+// Both gradients of a backward in one launch of the streaming kernel (dB first, then dA).
 template <int MB>
-mlora_status_t launch_grad_stream(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& a, int n_slots, int n_rows,
-                                  cudaStream_t st) {
+mlora_status_t launch_grad_stream2(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& gb, const GradArgs& ga_, int n_slots,
+                                   int n_rows, cudaStream_t st) {
   constexpr size_t smem = (size_t)gstream_stages(MB) * (128 * 128 + 128 * MB * 16 * 4) + (size_t)STREAM_WARPS * MB * 16 * 65 * 4 + 1024;
   static bool attr_set = false;
   auto kern = grad_stream_kernel<MB>;
@@ -278,28 +279,27 @@ mlora_status_t launch_grad_stream(mlora_ctx* ctx, const mlora_plan* p, const Gra
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return MLORA_ERR_CUDA;
     attr_set = true;
   }
-  CUtensorMap tQ;
-  mlora_status_t ms = make_tmap_bf16(ctx, &tQ, a.Q, a.D, n_rows, a.ldq, 64, 128);
-  if (ms != MLORA_OK) return ms;
-  GradStreamArgs ga;
-  ga.g = a;
-  ga.slot_blk_off = p->slot_blk_off; ga.blk_row0 = p->blk_row0; ga.blk_nrows = p->blk_nrows;
-  ga.n_slots = n_slots; ga.n_strips = a.D / 64; ga.status = ctx->status_dev;
-  const int groups = n_slots * ga.n_strips;
+  CUtensorMap tQ0, tQ1;
+  mlora_status_t ms;
+  if ((ms = make_tmap_bf16(ctx, &tQ0, gb.Q, gb.D, n_rows, gb.ldq, 64, 128)) != MLORA_OK) return ms;
+  if ((ms = make_tmap_bf16(ctx, &tQ1, ga_.Q, ga_.D, n_rows, ga_.ldq, 64, 128)) != MLORA_OK) return ms;
+  GradStreamArgs g;
+  g.prob[0] = GradProblem{gb.P, gb.scale, gb.G, gb.D, gb.D / 64};
+  g.prob[1] = GradProblem{ga_.P, ga_.scale, ga_.G, ga_.D, ga_.D / 64};
+  g.n_problems = 2; g.R = gb.R; g.accumulate = gb.accumulate;
+  g.slot_adapter = p->slot_adapter; g.slot_blk_off = p->slot_blk_off; g.blk_row0 = p->blk_row0; g.blk_nrows = p->blk_nrows;
+  g.n_slots = n_slots; g.status = ctx->status_dev;
+  const int groups = n_slots * (g.prob[0].n_strips + g.prob[1].n_strips);
   const int grid = groups < ctx->sm_count ? groups : ctx->sm_count;
   if (cancelled(ctx)) return MLORA_CANCELLED;
   LaunchScope scope(ctx, st, KIND_GRAD);
-  launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(STREAM_THREADS), smem, st, tQ, ga);
+  launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(STREAM_THREADS), smem, st, tQ0, tQ1, g);
   return scope.done();
 }
 
 mlora_status_t launch_grad(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& a, int n_slots, int n_rows,
                            cudaStream_t st) {
   if (n_slots <= 0) return MLORA_OK;
-  if (ctx->shrink_path == 0) {
-    if (a.R <= 16) return launch_grad_stream<1>(ctx, p, a, n_slots, n_rows, st);
-    if (a.R <= 32) return launch_grad_stream<2>(ctx, p, a, n_slots, n_rows, st);
-  }
   if (cancelled(ctx)) return MLORA_CANCELLED;
   constexpr int smem1 = (GRAD_THREADS / 32) * 16 * 65 * 4, smem2 = 2 * smem1;
   static bool attr_set = false;
@@ -836,6 +836,16 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   ga.P = u_save; ga.R = L->rank; ga.scale = L->scale; ga.Q = (const __nv_bfloat16*)dY; ga.ldq = lddy; ga.D = L->d_out;
   ga.G = dB; ga.slot_chunk_off = p->slot_chunk_off; ga.chunk_row0 = p->chunk_row0; ga.chunk_nrows = p->chunk_nrows;
   ga.slot_adapter = p->slot_adapter; ga.accumulate = accumulate;
+  GradArgs gA = ga;                  // dA = V^T X
+  gA.P = ctx->ws_p; gA.scale = nullptr; gA.Q = (const __nv_bfloat16*)x_save; gA.ldq = L->d_in; gA.D = L->d_in; gA.G = dA;
+  if (ctx->shrink_path == 0 && L->rank <= 32) {      // both gradients in one launch of the streaming kernel
+    s = L->rank <= 16 ? launch_grad_stream2<1>(ctx, p, ga, gA, n_slots, h.ft_rows, st)
+                      : launch_grad_stream2<2>(ctx, p, ga, gA, n_slots, h.ft_rows, st);
+    if (s != MLORA_OK) return s;
+    if (!dX) return MLORA_OK;
+    return gemm_bf16<true>(ctx, L, h.bwd, p->bwd, dY, lddy, dX, lddx, L->A_all, ctx->ws_p, nullptr, h.ft_rows, L->d_in,
+                           L->d_out, st);
+  }
   if ((s = launch_grad(ctx, p, ga, n_slots, h.ft_rows, st)) != MLORA_OK) return s;
   ga.P = ctx->ws_p; ga.scale = nullptr; ga.Q = (const __nv_bfloat16*)x_save; ga.ldq = L->d_in; ga.D = L->d_in;
   ga.G = dA;                         // dA = V^T X

@@ -673,18 +673,30 @@ grad_kernel(const GradArgs a) {
 // the contraction index); the eight warps are added in a fixed order when the strip is done.
 __host__ __device__ constexpr int gstream_stages(int mb) { return mb == 1 ? 6 : 4; }
 
+// One launch computes both gradients of a backward: problem 0 (dB: P = u_save scaled, Q = dY,
+// D = d_out) and problem 1 (dA: P = V, Q = x_save, D = d_in); groups of problem 0 come first.
+struct GradProblem {
+  const float* P;              // [rows, R] fp32
+  const float* scale;          // nullable
+  float* G;                    // [n_slots, R, D]
+  int32_t D, n_strips;         // D / 64
+};
 struct GradStreamArgs {
-  GradArgs g;
+  GradProblem prob[2];
+  int32_t n_problems;          // 1 or 2
+  int32_t R, accumulate;
+  const int32_t* slot_adapter;
   const int32_t* slot_blk_off;
   const int32_t* blk_row0;
   const int32_t* blk_nrows;
-  int32_t n_slots, n_strips;
+  int32_t n_slots;
   int32_t* status;
 };
 
 template <int MB>
 __global__ void __launch_bounds__(STREAM_THREADS, 1)
-grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const GradStreamArgs ga) {
+grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_constant__ CUtensorMap tmQ1,
+                   const GradStreamArgs ga) {
   constexpr int S = gstream_stages(MB);
   constexpr int RMAX = MB * 16;
   constexpr uint32_t Q_BYTES = 128 * 128;                 // 128 rows x 64 bf16, swizzled
@@ -694,8 +706,7 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const GradStreamArgs
   __shared__ __align__(8) uint64_t bars[2 * S];
   __shared__ int abort_word;
   volatile int* abort_flag = &abort_word;
-  const GradArgs& a = ga.g;
-  const int R = a.R;
+  const int R = ga.R;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t ring = (ptx::smem_u32(gs_smem) + 1023u) & ~1023u;      // swizzled tiles need 1 KiB alignment
@@ -708,10 +719,12 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const GradStreamArgs
     for (int st = 0; st < S; ++st) { ptx::mbar_init(bar_full(st), 1); ptx::mbar_init(bar_empty(st), STREAM_WARPS); }
     abort_word = 0;
     ptx::fence_barrier_init();
-    ptx::prefetch_tmap(&tmQ);
+    ptx::prefetch_tmap(&tmQ0);
+    ptx::prefetch_tmap(&tmQ1);
   }
   __syncthreads();
-  const int n_groups = ga.n_slots * ga.n_strips;
+  const int groups0 = ga.n_slots * ga.prob[0].n_strips;
+  const int n_groups = groups0 + (ga.n_problems > 1 ? ga.n_slots * ga.prob[1].n_strips : 0);
 
   if (warp == STREAM_WARPS) {
     // ======================= producer =======================
@@ -721,7 +734,11 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const GradStreamArgs
       uint32_t i = 0;
       bool ok = true;
       for (int grp = blockIdx.x; grp < n_groups && ok; grp += gridDim.x) {
-        const int slot = grp / ga.n_strips, strip = grp % ga.n_strips;
+        const int pi = grp >= groups0 ? 1 : 0;
+        const GradProblem& pr = ga.prob[pi];
+        const CUtensorMap* tmQ = pi ? &tmQ1 : &tmQ0;
+        const int gl = grp - pi * groups0;
+        const int slot = gl / pr.n_strips, strip = gl % pr.n_strips;
         for (int b = ga.slot_blk_off[slot]; b < ga.slot_blk_off[slot + 1]; ++b, ++i) {
           const int st = i % S;
           if (!(ok = stream_wait(bar_empty(st), ((i / S) & 1) ^ 1, abort_flag, ga.status))) break;
@@ -729,8 +746,8 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const GradStreamArgs
           const uint32_t dst = ring + (uint32_t)st * STAGE_BYTES;
           const uint32_t pbytes = (uint32_t)nrows * (uint32_t)R * 4u;
           ptx::mbar_arrive_expect_tx(bar_full(st), Q_BYTES + pbytes);
-          ptx::tma_load_2d(dst, &tmQ, strip * 64, row0, bar_full(st));       // rows past the block are masked below
-          bulk_load(dst + Q_BYTES, a.P + (size_t)row0 * R, pbytes, bar_full(st));
+          ptx::tma_load_2d(dst, tmQ, strip * 64, row0, bar_full(st));        // rows past the block are masked below
+          bulk_load(dst + Q_BYTES, pr.P + (size_t)row0 * R, pbytes, bar_full(st));
         }
       }
     }
@@ -742,8 +759,11 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const GradStreamArgs
     uint32_t i = 0;
     bool ok = true;
     for (int grp = blockIdx.x; grp < n_groups && ok; grp += gridDim.x) {
-      const int slot = grp / ga.n_strips, strip = grp % ga.n_strips;
-      const float sc = a.scale ? a.scale[a.slot_adapter[slot]] : 1.0f;
+      const int pi = grp >= groups0 ? 1 : 0;
+      const GradProblem& pr = ga.prob[pi];
+      const int gl = grp - pi * groups0;
+      const int slot = gl / pr.n_strips, strip = gl % pr.n_strips;
+      const float sc = pr.scale ? pr.scale[ga.slot_adapter[slot]] : 1.0f;
 #pragma unroll
       for (int m = 0; m < MB; ++m)
 #pragma unroll
@@ -827,8 +847,8 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const GradStreamArgs
         float v = 0.f;
 #pragma unroll
         for (int w = 0; w < STREAM_WARPS; ++w) v += red[w][ql][j];
-        float* dst = a.G + ((size_t)slot * R + ql) * a.D + strip * 64 + j;
-        *dst = a.accumulate ? (*dst + v) : v;
+        float* dst = pr.G + ((size_t)slot * R + ql) * pr.D + strip * 64 + j;
+        *dst = ga.accumulate ? (*dst + v) : v;
       }
       asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");
     }
