@@ -31,7 +31,7 @@ if ROOT not in sys.path:
 
 from paper_2607_28848_b200 import synth  # noqa: E402
 
-METRIC = "mixed-batch multi-LoRA layer tokens/s (fwd + LoRA bwd)"
+METRIC = "mixed-batch multi-LoRA layer tokens/s and TFLOP/s (fwd+LoRA bwd) vs BF16 roofline"
 UNIT = "tokens/s"
 
 
