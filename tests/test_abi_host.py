@@ -17,13 +17,18 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def test_library_exports_every_declared_symbol():
+    from paper_2607_28848_b200 import sched as ms
     lib = mb.load_library()
-    header = open(os.path.join(ROOT, "include", "mlora.h")).read()
-    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = set(re.findall(r"\b(mlora_[a-z_]+)\s*\(", header))
-    assert declared == set(mb.EXPORTS)
-    for name in declared:
-        assert hasattr(lib, name), name
+    bound = {"mlora.h": set(mb.EXPORTS), "mlora_sched.h": set(ms.EXPORTS)}
+    inc = os.path.join(ROOT, "include")
+    assert sorted(f for f in os.listdir(inc) if f.endswith(".h")) == sorted(bound)
+    for fname, names in bound.items():
+        header = open(os.path.join(inc, fname)).read()
+        header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+        declared = set(re.findall(r"\b(mlora_[a-z_]+)\s*\(", header))
+        assert declared == names, fname
+        for name in declared:
+            assert hasattr(lib, name), name
 
 
 def test_status_strings():
