@@ -69,7 +69,7 @@ struct DevRowSpace {
   const int32_t* item_start = nullptr;
   const int32_t* item_nrows = nullptr;
   const int32_t* item_adapter = nullptr;
-  const int32_t* item_contig = nullptr;
+  const int32_t* item_desc = nullptr;
 };
 
 struct mlora_plan {
@@ -208,16 +208,24 @@ int shrink_ksplit(const mlora_ctx* ctx, int n_items, int D) {
   return k < 1 ? 1 : k;
 }
 template <int RB, int STAGES, int CHUNK>
-mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, const int32_t* item_contig, int n_rows,
+mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, const int32_t* item_desc, int n_rows,
                                     int n_adapters, cudaStream_t st) {
   constexpr int R = RB * 8;
   constexpr size_t xrow = 32 * (CHUNK * 128 + 16), xtile = (size_t)(CHUNK / 4) * 32 * 512;
-  constexpr size_t xbytes = ((xrow > xtile ? xrow : xtile) + 127) / 128 * 128;
-  constexpr size_t smem = (size_t)STAGES * (xbytes + (size_t)(CHUNK / 4) * R * 512) + (size_t)(RB >= 4 ? 4 : 8) * 32 * (R + 1) * 4;
-  CUtensorMap tIn, tP;
+  constexpr size_t xbytes = ((xrow > xtile ? xrow : xtile) + 1023) / 1024 * 1024;
+  constexpr size_t smem = 1024 + (size_t)STAGES * (xbytes + (size_t)(CHUNK / 4) * R * 512) + (size_t)(RB >= 4 ? 4 : 8) * 32 * (R + 1) * 4;
+  CUtensorMap tIn, tP, tSave;
   mlora_status_t ms;
-  if ((ms = make_tmap_bf16(ctx, &tIn, a.In, a.D, n_rows, a.ld_in, 256, 32, false)) != MLORA_OK) return ms;
-  if ((ms = make_tmap_bf16(ctx, &tP, a.P_all, a.D, (uint64_t)n_adapters * R, a.D, 256, R, false)) != MLORA_OK) return ms;
+  // (64, rows, D / 64) views: one box = 4 K-blocks x rows x 128 bytes, 128-byte swizzle
+  if ((ms = make_tmap_bf16_blocked(ctx, &tIn, a.In, n_rows, a.D, a.ld_in, 32, 4)) != MLORA_OK) return ms;
+  if ((ms = make_tmap_bf16_blocked(ctx, &tP, a.P_all, (uint64_t)n_adapters * R, a.D, a.D, R, 4)) != MLORA_OK) return ms;
+  // full items of fine-tuning rows are saved as blocks straight from the staged tiles
+  const bool tma_save = a.x_save != nullptr && a.save_cap > 0;
+  if (tma_save) {
+    if ((ms = make_tmap_bf16_blocked(ctx, &tSave, a.x_save, (uint64_t)a.save_cap, a.D, a.D, 32, 4)) != MLORA_OK) return ms;
+  } else {
+    tSave = tIn;
+  }
   static bool attr_set = false;
   auto kern = shrink_stream_kernel<RB, STAGES, CHUNK>;
   if (!attr_set) {
@@ -229,6 +237,7 @@ mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, c
   sa.s.partial = ctx->ws_partial;
   sa.s.counters = ctx->ws_counters;
   sa.n_items = n_items;
+  sa.tma_save = tma_save ? 1 : 0;
   sa.chunks_per_item = (a.D / 64 + CHUNK - 1) / CHUNK;
   sa.n_units = n_items * sa.chunks_per_item;
   int grid = sa.n_units < ctx->sm_count ? sa.n_units : ctx->sm_count;
@@ -238,18 +247,18 @@ mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, c
   if (2 * (int64_t)grid > ctx->ws_partial_items || n_items > ctx->ws_counter_items) return MLORA_ERR_INVALID_ARG;
   LaunchScope scope(ctx, st, KIND_SHRINK);
   sa.status = ctx->status_dev;
-  sa.item_contig = item_contig;
-  launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(STREAM_THREADS), smem, st, tIn, tP, sa);
+  sa.item_desc = item_desc;
+  launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(STREAM_THREADS), smem, st, tIn, tP, tSave, sa);
   return scope.done();
 }
 
-mlora_status_t launch_shrink(mlora_ctx* ctx, int R, ShrinkArgs a, int n_items, const int32_t* item_contig, int n_rows,
+mlora_status_t launch_shrink(mlora_ctx* ctx, int R, ShrinkArgs a, int n_items, const int32_t* item_desc, int n_rows,
                              int n_adapters, cudaStream_t st) {
   if (n_items <= 0) return MLORA_OK;
   if (ctx->shrink_path == 0) {
-    if (R == 8) return launch_shrink_stream<1, 2, 16>(ctx, a, n_items, item_contig, n_rows, n_adapters, st);
-    if (R == 16) return launch_shrink_stream<2, 2, 16>(ctx, a, n_items, item_contig, n_rows, n_adapters, st);
-    if (R == 32) return launch_shrink_stream<4, 3, 8>(ctx, a, n_items, item_contig, n_rows, n_adapters, st);
+    if (R == 8) return launch_shrink_stream<1, 2, 16>(ctx, a, n_items, item_desc, n_rows, n_adapters, st);
+    if (R == 16) return launch_shrink_stream<2, 2, 16>(ctx, a, n_items, item_desc, n_rows, n_adapters, st);
+    if (R == 32) return launch_shrink_stream<4, 3, 8>(ctx, a, n_items, item_desc, n_rows, n_adapters, st);
   }
   if (cancelled(ctx)) return MLORA_CANCELLED;
   const int ksplit = shrink_ksplit(ctx, n_items, a.D);
@@ -685,7 +694,7 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
       o[n++] = b.add(rs[i]->tile_grp_off); o[n++] = b.add(rs[i]->grp_adapter); o[n++] = b.add(rs[i]->item_rows);
       o[n++] = b.add(rs[i]->row_grp2); o[n++] = b.add(rs[i]->tile2_grp_off); o[n++] = b.add(rs[i]->grp2_adapter);
       o[n++] = b.add(rs[i]->zero_rows2);
-      o[n++] = b.add(rs[i]->item_save); o[n++] = b.add(rs[i]->item_start); o[n++] = b.add(rs[i]->item_contig); o[n++] = b.add(rs[i]->item_nrows); o[n++] = b.add(rs[i]->item_adapter);
+      o[n++] = b.add(rs[i]->item_save); o[n++] = b.add(rs[i]->item_start); o[n++] = b.add(rs[i]->item_desc); o[n++] = b.add(rs[i]->item_nrows); o[n++] = b.add(rs[i]->item_adapter);
     }
     o[n++] = b.add(h.slot_chunk_off); o[n++] = b.add(h.chunk_row0); o[n++] = b.add(h.chunk_nrows);
     o[n++] = b.add(h.ft_adapters);
@@ -701,7 +710,7 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
       ds[i]->tile_grp_off = p->blob + o[n++]; ds[i]->grp_adapter = p->blob + o[n++]; ds[i]->item_rows = p->blob + o[n++];
       ds[i]->row_grp2 = p->blob + o[n++]; ds[i]->tile2_grp_off = p->blob + o[n++]; ds[i]->grp2_adapter = p->blob + o[n++];
       ds[i]->zero_rows2 = p->blob + o[n++];
-      ds[i]->item_save = p->blob + o[n++]; ds[i]->item_start = p->blob + o[n++]; ds[i]->item_contig = p->blob + o[n++]; ds[i]->item_nrows = p->blob + o[n++]; ds[i]->item_adapter = p->blob + o[n++];
+      ds[i]->item_save = p->blob + o[n++]; ds[i]->item_start = p->blob + o[n++]; ds[i]->item_desc = p->blob + o[n++]; ds[i]->item_nrows = p->blob + o[n++]; ds[i]->item_adapter = p->blob + o[n++];
     }
     p->bwd.row_save = nullptr;       // the compact space has no save offsets
     p->slot_chunk_off = p->blob + o[n++]; p->chunk_row0 = p->blob + o[n++]; p->chunk_nrows = p->blob + o[n++];
@@ -797,7 +806,8 @@ mlora_status_t mlora_mixed_forward(mlora_ctx* ctx, const mlora_layer_t* L, const
   sa.pbd = PbdArgs{ctx->gemm_pairs ? ctx->ws_pbd : nullptr, p->fwd.row_grp2, p->fwd.tile2_grp_off, L->scale,
                    p->fwd.zero_rows2, (int32_t)h.fwd.zero_rows2.size()};
   sa.x_save = (__nv_bfloat16*)x_save; sa.u_save = u_save; sa.save_base = save_row_base;
-  if ((s = launch_shrink(ctx, L->rank, sa, h.fwd.n_items(), p->fwd.item_contig, h.n_rows, L->n_adapters, st)) != MLORA_OK)
+  sa.save_cap = save_capacity_rows;
+  if ((s = launch_shrink(ctx, L->rank, sa, h.fwd.n_items(), p->fwd.item_desc, h.n_rows, L->n_adapters, st)) != MLORA_OK)
     return s;
   return gemm_bf16<false>(ctx, L, h.fwd, p->fwd, X, ldx, Y, ldy, L->B_all, ctx->ws_p, L->scale, h.n_rows, L->d_out,
                           L->d_in, st);
@@ -828,8 +838,8 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   sa.item_rows = p->bwd.item_rows; sa.item_start = p->bwd.item_start; sa.item_nrows = p->bwd.item_nrows;
   sa.pbd = PbdArgs{(ctx->gemm_pairs && dX) ? ctx->ws_pbd : nullptr, p->bwd.row_grp2, p->bwd.tile2_grp_off, nullptr,
                    p->bwd.zero_rows2, (int32_t)h.bwd.zero_rows2.size()};
-  sa.item_adapter = p->bwd.item_adapter; sa.item_save = nullptr; sa.x_save = nullptr; sa.u_save = nullptr; sa.save_base = 0;
-  if ((s = launch_shrink(ctx, L->rank, sa, h.bwd.n_items(), p->bwd.item_contig, h.ft_rows, L->n_adapters, st)) != MLORA_OK)
+  sa.item_adapter = p->bwd.item_adapter; sa.item_save = nullptr; sa.x_save = nullptr; sa.u_save = nullptr; sa.save_base = 0; sa.save_cap = 0;
+  if ((s = launch_shrink(ctx, L->rank, sa, h.bwd.n_items(), p->bwd.item_desc, h.ft_rows, L->n_adapters, st)) != MLORA_OK)
     return s;
 
   GradArgs ga;                       // dB = (s U)^T dY
@@ -915,5 +925,17 @@ mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path) {
   ctx->gemm_pairs = path == 3 ? 0 : 1;
   return MLORA_OK;
 }
+
+#ifdef MLORA_TIMELINE
+// Development aid, not part of the ABI: copies the per-CTA clock stamps of the last streaming launch.
+int mlora_debug_timeline(long long* host, int n) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+  return cudaMemcpyFromSymbol(host, mlora::g_timeline, sizeof(long long) * (size_t)n) == cudaSuccess ? 0 : -1;
+}
+int mlora_debug_timeline_reset() {
+  static long long zeros[160 * 16];
+  return cudaMemcpyToSymbol(mlora::g_timeline, zeros, sizeof(zeros)) == cudaSuccess ? 0 : -1;
+}
+#endif
 
 }  // extern "C"

@@ -13,6 +13,7 @@ namespace mlora {
 constexpr int kTileRows = 128;     // rows per tensor-core tile of the one-SM kernel (UMMA M = 128)
 constexpr int kPairTileRows = 256; // rows per tile of the two-SM kernel (a CTA pair, UMMA M = 256)
 constexpr int kItemRows = 32;      // most rows in one shrink work item (two mma.sync row blocks)
+constexpr int kItemDescInts = 8;  // ints per packed item record (RowSpace::item_desc)
 constexpr int kChunkRows = 16;     // rows per gradient chunk (one mma.sync contraction step)
 constexpr int kMaxRank = 128;
 
@@ -36,7 +37,11 @@ struct RowSpace {
   std::vector<int32_t> item_rows;      // [rows with an adapter] row ids, grouped by adapter
   std::vector<int32_t> item_save;      // parallel to item_rows: save offset of that row or -1
   std::vector<int32_t> item_start, item_nrows, item_adapter;
-  std::vector<int32_t> item_contig;    // 1: the item's rows are consecutive rows of the batch
+  // One packed record per item for the streaming kernels, kItemDescInts ints:
+  // {start, nrows, adapter, flags, first row, first save offset (-1: none), 0, 0}; flag bit 0: the
+  // item's rows are consecutive rows of the batch; bit 1: additionally the item is full
+  // (kItemRows rows) and its save offsets are consecutive, so its rows can be saved as one block.
+  std::vector<int32_t> item_desc;
   int32_t n_tiles() const { return (n_rows + kTileRows - 1) / kTileRows; }
   int32_t n_items() const { return (int32_t)item_start.size(); }
 };
@@ -88,7 +93,7 @@ inline void build_tiles_and_items(RowSpace& rs) {
     const int32_t tile = t / kPairTileRows;
     if (rs.row_adapter[t] < 0 && rs.tile2_grp_off[tile + 1] > rs.tile2_grp_off[tile]) rs.zero_rows2.push_back(t);
   }
-  rs.item_rows.clear(); rs.item_start.clear(); rs.item_nrows.clear(); rs.item_adapter.clear(); rs.item_contig.clear();
+  rs.item_rows.clear(); rs.item_start.clear(); rs.item_nrows.clear(); rs.item_adapter.clear(); rs.item_desc.clear();
   int32_t max_adapter = -1;
   for (int32_t t = 0; t < n; ++t) max_adapter = rs.row_adapter[t] > max_adapter ? rs.row_adapter[t] : max_adapter;
   std::vector<int32_t> count(max_adapter + 2, 0);
@@ -109,10 +114,19 @@ inline void build_tiles_and_items(RowSpace& rs) {
       rs.item_adapter.push_back(a);
     }
   }
-  rs.item_contig.assign(rs.item_start.size(), 1);
-  for (size_t it = 0; it < rs.item_start.size(); ++it)
-    for (int32_t i = 1; i < rs.item_nrows[it]; ++i)
-      if (rs.item_rows[rs.item_start[it] + i] != rs.item_rows[rs.item_start[it]] + i) { rs.item_contig[it] = 0; break; }
+  rs.item_desc.assign(rs.item_start.size() * kItemDescInts, 0);
+  for (size_t it = 0; it < rs.item_start.size(); ++it) {
+    const int32_t start = rs.item_start[it], nr = rs.item_nrows[it];
+    bool contig = true, block_save = nr == kItemRows && rs.item_save[start] >= 0;
+    for (int32_t i = 1; i < nr; ++i) {
+      if (rs.item_rows[start + i] != rs.item_rows[start] + i) contig = false;
+      if (rs.item_save[start + i] != rs.item_save[start] + i) block_save = false;
+    }
+    int32_t* d = &rs.item_desc[it * kItemDescInts];
+    d[0] = start; d[1] = nr; d[2] = rs.item_adapter[it];
+    d[3] = (contig ? 1 : 0) | (contig && block_save ? 2 : 0);
+    d[4] = rs.item_rows[start]; d[5] = rs.item_save[start];
+  }
 }
 
 // Validates the table and fills `p`.  Returns MLORA_OK or the error the header documents.

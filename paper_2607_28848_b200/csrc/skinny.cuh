@@ -11,6 +11,7 @@
 //  grad_kernel   : G_g[q, j] = sum_{rows t of slot g} P[t, q] * Q[t, j]   (dB = (s U)^T dY, dA = V^T X)
 #pragma once
 
+#include "plan.h"
 #include "ptx.cuh"
 
 namespace mlora {
@@ -68,6 +69,7 @@ struct ShrinkArgs {
   __nv_bfloat16* x_save;       // nullable, [cap, D] dense
   float* u_save;               // nullable, [cap, R] dense
   int64_t save_base;
+  int64_t save_cap;            // rows of x_save (extent of its tensor map)
   // split of the contraction over gridDim.y CTAs per item (used when there are few items):
   float* partial;              // [n_items * gridDim.z * gridDim.y, MT * 16, R] scratch
   int32_t* counters;           // [n_items * gridDim.z], zero between launches
@@ -252,6 +254,18 @@ constexpr int STREAM_THREADS = (STREAM_WARPS + 1) * 32;
 // bytes apart, so that fragment loads hit distinct banks.
 constexpr uint32_t STREAM_SPIN_LIMIT = 1u << 22;
 
+#ifdef MLORA_TIMELINE
+// Development aid (off in the product build): per-CTA clock stamps of the streaming kernels.
+__device__ long long g_timeline[160 * 16];
+__device__ __forceinline__ long long tl_clock() { return clock64(); }
+__device__ __forceinline__ long long tl_global() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define MLORA_TL_SET(slot, v) do { g_timeline[blockIdx.x * 16 + (slot)] = (v); } while (0)
+#define MLORA_TL_ADD(slot, v) do { g_timeline[blockIdx.x * 16 + (slot)] += (v); } while (0)
+#else
+#define MLORA_TL_SET(slot, v) do {} while (0)
+#define MLORA_TL_ADD(slot, v) do {} while (0)
+#endif
+
 struct StreamArgs {
   ShrinkArgs s;
   int32_t n_items;
@@ -259,7 +273,8 @@ struct StreamArgs {
   int32_t n_units;           // n_items * chunks_per_item
   int32_t units_per_cta;     // ceil(n_units / gridDim.x)
   int32_t* status;           // device status word
-  const int32_t* item_contig;  // [n_items] 1: the item's rows are consecutive rows of In
+  const int32_t* item_desc;    // [n_items][kItemDescInts] packed item records (see RowSpace::item_desc)
+  int32_t tma_save;            // 1: tmSave covers x_save; full contiguous fine-tuning items are saved as blocks
 };
 
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -284,19 +299,23 @@ __device__ __forceinline__ bool stream_wait(uint32_t bar, uint32_t parity, volat
 template <int RB, int STAGES, int CHUNK>
 __global__ void __launch_bounds__(STREAM_THREADS, 1)
 shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ CUtensorMap tmP,
-                     const StreamArgs sa) {
+                     const __grid_constant__ CUtensorMap tmSave, const StreamArgs sa) {
   constexpr int R = RB * 8;
   constexpr int NBOX = CHUNK / 4;                          // 256-element boxes per unit
   constexpr uint32_t STREAM_PITCH = CHUNK * 128 + 16;     // row-copy layout
-  constexpr uint32_t XBOX_BYTES = 32 * 512;               // tile layout: [32 rows][256 elements]
-  constexpr uint32_t X_BYTES = ((32 * STREAM_PITCH > NBOX * XBOX_BYTES ? 32 * STREAM_PITCH : NBOX * XBOX_BYTES) + 127) / 128 * 128;
-  constexpr uint32_t PBOX_BYTES = R * 512;                // adapter rows: [R rows][256 elements] per box
+  // tile layout of a box: [4 K-blocks][32 rows][128 B], 16-byte pieces swizzled by (row & 7)
+  // (the 128-byte swizzle of the tensor maps), so the 8 rows a warp reads at one K offset fall
+  // into 8 different bank groups
+  constexpr uint32_t XBOX_BYTES = 4 * 32 * 128;
+  constexpr uint32_t X_BYTES = ((32 * STREAM_PITCH > NBOX * XBOX_BYTES ? 32 * STREAM_PITCH : NBOX * XBOX_BYTES) + 1023) / 1024 * 1024;
+  constexpr uint32_t PBOX_BYTES = 4 * R * 128;            // adapter rows: [4 K-blocks][R rows][128 B], swizzled
   constexpr uint32_t STAGE_BYTES = X_BYTES + NBOX * PBOX_BYTES;
   static_assert(CHUNK % STREAM_WARPS == 0, "each consumer warp takes CHUNK / 8 K-blocks of a unit");
   constexpr int RW = RB >= 4 ? 4 : 8;                     // reduction buffers (rank 32: two rounds of 4 warps)
   extern __shared__ __align__(128) uint8_t stream_smem[];
-  float (*red)[32][R + 1] = reinterpret_cast<float (*)[32][R + 1]>(stream_smem + STAGES * STAGE_BYTES);
+  __shared__ __align__(16) float fin[32][R];             // an item's final rows, read back for the operand chunks
   __shared__ __align__(8) uint64_t bars[2 * STAGES];     // full[STAGES] | empty[STAGES]
+  __shared__ int stage_save[STAGES][2];                  // producer only: {first x_save row or -1, k0} of the staged unit
   __shared__ int is_last;
   __shared__ int abort_word;
   volatile int* abort_flag = &abort_word;
@@ -308,11 +327,19 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
   const int u_end = min(u_begin + sa.units_per_cta, sa.n_units);
   const int KC = sa.chunks_per_item;
   const int nkb = a.D / 64;
-  const uint32_t ring = ptx::smem_u32(stream_smem);
+  const uint32_t ring = (ptx::smem_u32(stream_smem) + 1023u) & ~1023u;   // swizzled tiles need 1 KiB alignment
   const uint32_t bar0 = ptx::smem_u32(bars);
   auto bar_full = [&](int st) { return bar0 + 8u * st; };
   auto bar_empty = [&](int st) { return bar0 + 8u * (STAGES + st); };
+  float (*red)[32][R + 1] = reinterpret_cast<float (*)[32][R + 1]>(
+      stream_smem + (ring - ptx::smem_u32(stream_smem)) + STAGES * STAGE_BYTES);
 
+#ifdef MLORA_TIMELINE
+  const long long tl0 = tl_clock();
+  const bool tl_on = threadIdx.x == 0;
+  long long tl_wait = 0, tl_flush = 0, tl_nflush = 0;
+  if (tl_on) { for (int i = 0; i < 16; ++i) MLORA_TL_SET(i, 0); MLORA_TL_SET(14, tl_global()); }
+#endif
   if (threadIdx.x == 0) {
     for (int st = 0; st < STAGES; ++st) {
       ptx::mbar_init(bar_full(st), 1);
@@ -326,46 +353,76 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
   if (warp == STREAM_WARPS) {
     // ======================= producer =======================
     int item = u_begin / KC, kc = u_begin % KC;
-    int cur = -1, nrows = 0, contig = 0, row0 = 0, prow0 = 0;
+    int cur = -1, nrows = 0, contig = 0, row0 = 0, prow0 = 0, save_row = -1;
     const __nv_bfloat16* src0 = nullptr;     // gathered items: lane l copies the item's row l
     auto set_item = [&](int it) {
       cur = it;
-      nrows = a.item_nrows[it];
-      contig = sa.item_contig[it];
-      const int32_t* rows = a.item_rows + a.item_start[it];
-      row0 = rows[0];
-      src0 = (!contig && lane < nrows) ? a.In + (size_t)rows[lane] * a.ld_in : nullptr;
-      prow0 = a.item_adapter[it] * R;
+      const int4 d0 = *reinterpret_cast<const int4*>(sa.item_desc + (size_t)it * kItemDescInts);
+      const int2 d1 = *reinterpret_cast<const int2*>(sa.item_desc + (size_t)it * kItemDescInts + 4);
+      nrows = d0.y;
+      contig = d0.w & 1;
+      row0 = d1.x;
+      save_row = (sa.tma_save && (d0.w & 2)) ? (int)a.save_base + d1.y : -1;
+      src0 = (!contig && lane < nrows) ? a.In + (size_t)a.item_rows[d0.x + lane] * a.ld_in : nullptr;
+      prow0 = d0.z * R;
+    };
+    // block save of a staged unit: the tiles of a full fine-tuning item go from shared memory to
+    // x_save as they are (one bulk tensor store per 256-element box, lanes 0 .. NBOX-1)
+    auto store_unit = [&](int j) -> bool {
+      const int sj = j % STAGES;
+      const int srow = stage_save[sj][0];
+      if (srow < 0) return true;                         // same value in every lane
+      bool got = true;
+      if (lane == 0) got = stream_wait(bar_full(sj), (j / STAGES) & 1, abort_flag, sa.status);
+      got = __shfl_sync(0xffffffffu, got ? 1 : 0, 0) != 0;
+      if (!got) return false;
+      const int k0 = stage_save[sj][1];
+      if (lane < NBOX && k0 + lane * 256 < a.D)
+        ptx::tma_store_3d(&tmSave, ring + (uint32_t)sj * STAGE_BYTES + (uint32_t)lane * XBOX_BYTES, 0, srow, (k0 >> 6) + lane * 4);
+      ptx::tma_store_commit();
+      return true;
     };
     if (u_begin < u_end) set_item(item);
     ptx::prefetch_tmap(&tmIn);
     ptx::prefetch_tmap(&tmP);
+    if (sa.tma_save) ptx::prefetch_tmap(&tmSave);
     ptx::grid_dependency_wait();             // only plan tables were read so far
     ptx::grid_launch_dependents();
     bool ok = true;
+    int stored = u_begin;                    // units [u_begin, stored) have had their block save issued
     for (int u = u_begin; u < u_end && ok; ++u) {
       const int i = u - u_begin, st = i % STAGES;
       if (item != cur) set_item(item);
       if (lane == 0) ok = stream_wait(bar_empty(st), ((i / STAGES) & 1) ^ 1, abort_flag, sa.status);
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
+      ptx::tma_store_wait_read<0>();         // the stage's previous block save has left shared memory
+      __syncwarp();
       const int k0 = kc * (CHUNK * 64);
       const uint32_t row_bytes = (uint32_t)min(CHUNK * 64, a.D - k0) * 2u;
       const uint32_t xbytes = contig ? NBOX * XBOX_BYTES : (uint32_t)nrows * row_bytes;
-      if (lane == 0) ptx::mbar_arrive_expect_tx(bar_full(st), xbytes + NBOX * PBOX_BYTES);
+      if (lane == 0) {
+        stage_save[st][0] = save_row;
+        stage_save[st][1] = k0;
+        ptx::mbar_arrive_expect_tx(bar_full(st), xbytes + NBOX * PBOX_BYTES);
+      }
       __syncwarp();
       const uint32_t dst = ring + (uint32_t)st * STAGE_BYTES;
       // lanes 0 .. NBOX-1: one adapter tile each; lanes NBOX .. 2 NBOX-1: one tile of the item's rows
       // (tiles reaching past the tensor's edge are zero-filled and still count their full size)
-      if (lane < NBOX) ptx::tma_load_2d(dst + X_BYTES + (uint32_t)lane * PBOX_BYTES, &tmP, k0 + lane * 256, prow0, bar_full(st));
+      if (lane < NBOX) ptx::tma_load_3d(dst + X_BYTES + (uint32_t)lane * PBOX_BYTES, &tmP, 0, prow0, (k0 >> 6) + lane * 4, bar_full(st));
       if (contig) {
         if (lane >= NBOX && lane < 2 * NBOX)
-          ptx::tma_load_2d(dst + (uint32_t)(lane - NBOX) * XBOX_BYTES, &tmIn, k0 + (lane - NBOX) * 256, row0, bar_full(st));
+          ptx::tma_load_3d(dst + (uint32_t)(lane - NBOX) * XBOX_BYTES, &tmIn, 0, row0, (k0 >> 6) + (lane - NBOX) * 4, bar_full(st));
       } else if (src0) {
         bulk_load(dst + (uint32_t)lane * STREAM_PITCH, src0 + k0, row_bytes, bar_full(st));
       }
       if (++kc == KC) { kc = 0; ++item; }
+      // with the next load in flight, save the oldest staged unit whose data must have been asked for
+      if (i >= STAGES - 1) { ok = store_unit(i - (STAGES - 1)); stored = u - (STAGES - 1) + 1; }
     }
+    for (int u = stored; u < u_end && ok; ++u) ok = store_unit(u - u_begin);
+    ptx::tma_store_wait<0>();                // block saves complete before the CTA ends
   } else {
     // ======================= consumers =======================
     const int g = lane >> 2, c = lane & 3;
@@ -380,56 +437,96 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
     const int32_t* cur_rows = nullptr;
     const int32_t* cur_saves = nullptr;
     __nv_bfloat16* sp[4] = {nullptr, nullptr, nullptr, nullptr};
+    // flush-time values fetched when the item starts: element idx = tid + 256 k of the item's
+    // [rows][R] result belongs to row idx / R
+    int my_row[RB], my_save[RB];
+    float my_scale = 1.0f;
     // this thread's pieces of a K-block: elements 16c .. 16c+15 of the block
+#ifdef MLORA_TIMELINE
+    if (tl_on) MLORA_TL_SET(1, tl_clock() - tl0);
+#endif
     ptx::grid_dependency_wait();
+#ifdef MLORA_TIMELINE
+    if (tl_on) MLORA_TL_SET(2, tl_clock() - tl0);
+#endif
     bool ok = true;
     if (a.pbd.pbd)                                            // rows nobody else owns: all-zero chunks
       for (int i = cta * STREAM_WARPS + warp; i < a.pbd.n_zero_rows; i += gridDim.x * STREAM_WARPS)
         pbd_write_row<R>(a.pbd, a.pbd.zero_rows[i], nullptr, 0.f, lane);
 
+#ifdef MLORA_TIMELINE
+    if (tl_on) MLORA_TL_SET(3, tl_clock() - tl0);
+#endif
     for (int u = u_begin; u < u_end; ++u) {
       const int i = u - u_begin, st = i % STAGES;
       if (item != cur_item) {
         cur_item = item;
-        cur_nrows = a.item_nrows[item];
-        cur_adapter = a.item_adapter[item];
-        cur_contig = sa.item_contig[item];
-        cur_rows = a.item_rows + a.item_start[item];
-        cur_saves = a.item_save ? a.item_save + a.item_start[item] : nullptr;
+        const int4 d0 = *reinterpret_cast<const int4*>(sa.item_desc + (size_t)item * kItemDescInts);
+        cur_nrows = d0.y;
+        cur_adapter = d0.z;
+        cur_contig = d0.w & 1;
+        const bool block_saved = sa.tma_save && (d0.w & 2);   // the producer stores this item's rows
+#ifdef MLORA_TIMELINE
+        if (tl_on) MLORA_TL_SET(11, 8 + d0.w + (block_saved ? 4 : 0) + ((cur_saves && cur_saves[0] >= 0) ? 16 : 0));
+#endif
+        cur_rows = a.item_rows + d0.x;
+        cur_saves = a.item_save ? a.item_save + d0.x : nullptr;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int rl = g + 8 * j;
-          const int sv = (cur_saves && a.x_save && rl < cur_nrows) ? cur_saves[rl] : -1;
+          const int sv = (!block_saved && cur_saves && a.x_save && rl < cur_nrows) ? cur_saves[rl] : -1;
           sp[j] = sv >= 0 ? a.x_save + (size_t)(a.save_base + sv) * a.D + 16 * c : nullptr;
         }
+#pragma unroll
+        for (int k = 0; k < RB; ++k) {
+          const int r = ((int)threadIdx.x + k * STREAM_WARPS * 32) / R;
+          my_row[k] = r < cur_nrows ? cur_rows[r] : -1;
+          my_save[k] = (r < cur_nrows && cur_saves && a.u_save) ? cur_saves[r] : -1;
+        }
+        my_scale = a.scale ? a.scale[cur_adapter] : 1.0f;
       }
+#ifdef MLORA_TIMELINE
+      const long long tw0 = tl_clock();
+#endif
       ok = stream_wait(bar_full(st), (i / STAGES) & 1, abort_flag, sa.status);
       if (!ok) break;
+#ifdef MLORA_TIMELINE
+      if (tl_on) { tl_wait += tl_clock() - tw0; if (i == 0) MLORA_TL_SET(4, tl_clock() - tl0); }
+#endif
 #pragma unroll
       for (int kk = 0; kk < CHUNK / STREAM_WARPS; ++kk) {
         const int kb = kc * CHUNK + kk * STREAM_WARPS + warp;
         if (kb >= nkb) continue;
         const int kbl = kk * STREAM_WARPS + warp;            // K-block inside the unit
         const uint32_t stage = ring + (uint32_t)st * STAGE_BYTES;
-        const uint32_t in_box = (uint32_t)(kbl & 3) * 128u + (uint32_t)c * 32u;
-        // rows of In: tile layout [box][row][512 B] or row-copy layout [row][pitch]
-        const uint32_t xsrc = cur_contig ? stage + (uint32_t)(kbl >> 2) * XBOX_BYTES + in_box
-                                         : stage + (uint32_t)kbl * 128u + (uint32_t)c * 32u;
-        const uint32_t xpitch = cur_contig ? 512u : STREAM_PITCH;
+        // this thread's two 16-byte pieces (2c, 2c+1) of a row's 128-byte K-block; in the tile
+        // layout piece i of row r sits at piece i ^ (r & 7), and r & 7 == g for every row read here
+        const uint32_t sw0 = (uint32_t)((2 * c) ^ g) << 4, sw1 = (uint32_t)((2 * c + 1) ^ g) << 4;
         uint4 x[4][2];
+        if (cur_contig) {        // tile layout [box][K-block][row][128 B]
+          const uint32_t xsrc = stage + (uint32_t)(kbl >> 2) * XBOX_BYTES + (uint32_t)(kbl & 3) * 4096u;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const uint32_t ra = xsrc + (uint32_t)(g + 8 * j) * xpitch;
-          x[j][0] = lds_v4(ra);
-          x[j][1] = lds_v4(ra + 16);
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t ra = xsrc + (uint32_t)(g + 8 * j) * 128u;
+            x[j][0] = lds_v4(ra + sw0);
+            x[j][1] = lds_v4(ra + sw1);
+          }
+        } else {                 // row-copy layout [row][pitch]
+          const uint32_t xsrc = stage + (uint32_t)kbl * 128u + (uint32_t)c * 32u;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t ra = xsrc + (uint32_t)(g + 8 * j) * STREAM_PITCH;
+            x[j][0] = lds_v4(ra);
+            x[j][1] = lds_v4(ra + 16);
+          }
         }
-        const uint32_t psrc = stage + X_BYTES + (uint32_t)(kbl >> 2) * PBOX_BYTES + in_box;
+        const uint32_t psrc = stage + X_BYTES + (uint32_t)(kbl >> 2) * PBOX_BYTES + (uint32_t)(kbl & 3) * (R * 128u);
         uint4 p[RB][2];
 #pragma unroll
         for (int n = 0; n < RB; ++n) {
-          const uint32_t rp = psrc + (uint32_t)(8 * n + g) * 512u;
-          p[n][0] = lds_v4(rp);
-          p[n][1] = lds_v4(rp + 16);
+          const uint32_t rp = psrc + (uint32_t)(8 * n + g) * 128u;
+          p[n][0] = lds_v4(rp + sw0);
+          p[n][1] = lds_v4(rp + sw1);
         }
         // rows past the item's end were not copied: keep their stale bytes out of the MMA
 #pragma unroll
@@ -444,14 +541,19 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
             const uint32_t ra[8] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w};
             const uint32_t rb[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
 #pragma unroll
-            for (int s = 0; s < 4; ++s)
+            for (int s = 0; s < 4; ++s) {
+#ifdef MLORA_EXP_NOMMA
+              acc[m][n][0] += __uint_as_float(ra[2 * s] ^ rb[2 * s] ^ ra[2 * s + 1] ^ rb[2 * s + 1] ^ rp[2 * s] ^ rp[2 * s + 1]);
+#else
               ptx::mma_bf16_16816(acc[m][n], ra[2 * s], rb[2 * s], ra[2 * s + 1], rb[2 * s + 1], rp[2 * s], rp[2 * s + 1]);
+#endif
+            }
           }
         }
         const int ko = kb * 64;
 #pragma unroll
         for (int j = 0; j < 4; ++j)
-          if (sp[j]) {     // activation save: the rows of In pass through here exactly once
+          if (sp[j]) {     // activation save of rows that are not block-saved: they pass through here exactly once
             *reinterpret_cast<uint4*>(sp[j] + ko) = x[j][0];
             *reinterpret_cast<uint4*>(sp[j] + ko + 8) = x[j][1];
           }
@@ -464,6 +566,10 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
       const int this_item = item;
       if (++kc == KC) { kc = 0; ++item; }
       if (!item_ends) continue;
+#ifdef MLORA_TIMELINE
+      const long long tf0 = tl_clock();
+      if (tl_on && u == u_end - 1) MLORA_TL_SET(5, tf0 - tl0);
+#endif
 #pragma unroll
       for (int round = 0; round < STREAM_WARPS / RW; ++round) {
         if (warp / RW == round) {
@@ -501,9 +607,11 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
         if (finish) __threadfence();
       }
       if (finish) {
-        const float sc = a.scale ? a.scale[cur_adapter] : 1.0f;
-        for (int idx = threadIdx.x; idx < cur_nrows * R; idx += STREAM_WARPS * 32) {
+#pragma unroll
+        for (int k = 0; k < RB; ++k) {
+          const int idx = (int)threadIdx.x + k * STREAM_WARPS * 32;
           const int r = idx / R, q = idx % R;
+          if (r >= cur_nrows) continue;
           float v = 0.f;
           if (c0 != c1) {
             for (int cc = c0; cc <= c1; ++cc) {        // fixed order: by CTA index
@@ -514,24 +622,26 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
 #pragma unroll
             for (int w = 0; w < RW; ++w) v += red[w][r][q];
           }
-          const int row = cur_rows[r];
-          a.Out[(size_t)row * R + q] = v * sc;
-          if (a.u_save && cur_saves) {
-            const int sv = cur_saves[r];
-            if (sv >= 0) a.u_save[(size_t)(a.save_base + sv) * R + q] = v;
-          }
+          const float vs = v * my_scale;
+          a.Out[(size_t)my_row[k] * R + q] = vs;
+          fin[r][q] = vs;
+          if (my_save[k] >= 0) a.u_save[(size_t)(a.save_base + my_save[k]) * R + q] = v;
         }
         if (c0 != c1 && threadIdx.x == 0) a.counters[this_item] = 0;    // ready for the next launch
         if (a.pbd.pbd) {
-          asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");  // Out rows written above are read back
-          for (int r = warp; r < cur_nrows; r += STREAM_WARPS) {
-            const int row = cur_rows[r];
-            pbd_write_row<R>(a.pbd, row, a.Out + (size_t)row * R, a.pbd.scale ? a.pbd.scale[cur_adapter] : 1.0f, lane);
-          }
+          asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");  // fin[] complete
+          for (int r = warp; r < cur_nrows; r += STREAM_WARPS)
+            pbd_write_row<R>(a.pbd, cur_rows[r], fin[r], a.pbd.scale ? a.pbd.scale[cur_adapter] : 1.0f, lane);
         }
       }
-      asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");      // red[] is reused by the next item
+      asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");      // red[] and fin[] are reused by the next item
+#ifdef MLORA_TIMELINE
+      if (tl_on) { tl_flush += tl_clock() - tf0; ++tl_nflush; }
+#endif
     }
+#ifdef MLORA_TIMELINE
+    if (tl_on) { MLORA_TL_SET(9, tl_clock() - tl0); MLORA_TL_SET(15, tl_global()); MLORA_TL_SET(10, u_end - u_begin); MLORA_TL_SET(8, tl_wait); MLORA_TL_SET(6, tl_flush); MLORA_TL_SET(7, tl_nflush); }
+#endif
   }
 }
 
@@ -709,6 +819,12 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
   const int R = ga.R;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#ifdef MLORA_TIMELINE
+  const long long tl0 = tl_clock();
+  const bool tl_on = threadIdx.x == 0;
+  long long tl_wait = 0, tl_flush = 0, tl_nflush = 0, tl_nstage = 0;
+  if (tl_on) { for (int i = 0; i < 16; ++i) MLORA_TL_SET(i, 0); MLORA_TL_SET(14, tl_global()); }
+#endif
   const uint32_t ring = (ptx::smem_u32(gs_smem) + 1023u) & ~1023u;      // swizzled tiles need 1 KiB alignment
   float (*red)[MB * 16][64 + 1] = reinterpret_cast<float (*)[MB * 16][64 + 1]>(
       gs_smem + (ring - ptx::smem_u32(gs_smem)) + S * STAGE_BYTES);
@@ -754,7 +870,13 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
   } else {
     // ======================= consumers =======================
     const int g = lane >> 2, c = lane & 3;
+#ifdef MLORA_TIMELINE
+    if (tl_on) MLORA_TL_SET(1, tl_clock() - tl0);
+#endif
     ptx::grid_dependency_wait();
+#ifdef MLORA_TIMELINE
+    if (tl_on) { MLORA_TL_SET(2, tl_clock() - tl0); MLORA_TL_SET(3, tl_clock() - tl0); }
+#endif
     float acc[MB][8][4];
     uint32_t i = 0;
     bool ok = true;
@@ -771,7 +893,13 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
       for (int b = ga.slot_blk_off[slot]; b < ga.slot_blk_off[slot + 1]; ++b, ++i) {
         const int st = i % S;
         const int nrows = ga.blk_nrows[b];
+#ifdef MLORA_TIMELINE
+        const long long tw0 = tl_clock();
+#endif
         if (!(ok = stream_wait(bar_full(st), (i / S) & 1, abort_flag, ga.status))) break;
+#ifdef MLORA_TIMELINE
+        if (tl_on) { tl_wait += tl_clock() - tw0; if (i == 0) MLORA_TL_SET(4, tl_clock() - tl0); ++tl_nstage; }
+#endif
         const uint32_t qbase = ring + (uint32_t)st * STAGE_BYTES;
         const uint32_t pbase = qbase + Q_BYTES;
         if (warp * 16 < nrows) {
@@ -826,6 +954,10 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
         if (lane == 0) ptx::mbar_arrive(bar_empty(st));
       }
       if (!ok) break;
+#ifdef MLORA_TIMELINE
+      const long long tf0 = tl_clock();
+      if (tl_on && grp + (int)gridDim.x >= n_groups) MLORA_TL_SET(5, tf0 - tl0);
+#endif
       // ---- strip done: fixed-order sum over the warps, then write (or add to) the gradient ----
       {
         float (*mine)[64 + 1] = red[warp];
@@ -851,7 +983,13 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
         *dst = ga.accumulate ? (*dst + v) : v;
       }
       asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");
+#ifdef MLORA_TIMELINE
+      if (tl_on) { tl_flush += tl_clock() - tf0; ++tl_nflush; }
+#endif
     }
+#ifdef MLORA_TIMELINE
+    if (tl_on) { MLORA_TL_SET(9, tl_clock() - tl0); MLORA_TL_SET(15, tl_global()); MLORA_TL_SET(10, tl_nstage); MLORA_TL_SET(8, tl_wait); MLORA_TL_SET(6, tl_flush); MLORA_TL_SET(7, tl_nflush); }
+#endif
   }
 }
 
