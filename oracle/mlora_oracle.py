@@ -27,6 +27,20 @@ What it follows
       dA_a += V^T X                   [r, d_in]
       dX = dY W^T + V A_a             [rows, d_in]
 
+Variants (Section 5, "Fine-tuning Workload": the adapter is trained with dropout 0.05; adapters of
+different ranks share one base model in Section 2.2's serving setting):
+* LoRA dropout acts on the input of the low-rank branch of the fine-tuning rows only (the usual
+  LoRA definition: y = x W + s B A dropout(x)); inference rows never see it.  The keep decision
+  of element (m, k) - m the row's place in this batch's save order, k the input column - comes
+  from a counter-based generator so that forward and backward regenerate the same mask:
+  output number c + 1 of the SplitMix64 stream started at ``seed``, c = m * 2^32 + (k >> 2);
+  its 16-bit field number k & 3 is compared with round(p * 65536); kept elements are scaled by
+  1 / (1 - p).  With the mask K (0/1) the chain rule gives U = (X * K) A^T / (1 - p),
+  dA += (V / (1 - p))^T (X * K),  dX = dY W^T + (V A) * K / (1 - p); V and dB keep their form.
+* Adapters of different ranks are stored padded to the layer's rank r with zero rows; a zero row of
+  A_a and B_a contributes nothing to Y, V, dX and gets a zero gradient, so the padded layer
+  computes exactly what the per-adapter ranks define (``forward_ragged`` states that definition).
+
 Matrix products use numpy's float64 ``@`` as a library step; there is no blocking,
 fusion or reordering beyond the definitions above.  Inputs are the stored values
 (already rounded to the storage type by the caller); nothing is rounded in between.
@@ -35,7 +49,10 @@ Parity pins (tests/test_oracle_pins.py): element-by-element brute force in pure
 Python on tiny shapes, a hand-computed worked example, the B = 0 and s-linearity
 invariants, the merged-weight identity W_eff of Section 2.2 per segment, invariance
 under table reordering / segment splitting / the is_finetune flag, and central finite
-differences for every gradient.  No function here is "parity unpinned".
+differences for every gradient; for the variants, the published SplitMix64 test vector, the
+p = 0 and keep-frequency checks, finite differences through the masked forward, and the
+zero-padding identity against per-adapter matrices of their own ranks.  No function here is
+"parity unpinned".
 """
 from __future__ import annotations
 
@@ -50,6 +67,53 @@ class SegmentError(ValueError):
 
 def _f64(x) -> np.ndarray:
     return np.asarray(x, dtype=np.float64)
+
+
+# --------------------------------------------------------------------------------------
+# LoRA dropout: counter-based keep mask
+# --------------------------------------------------------------------------------------
+_M64 = (1 << 64) - 1
+
+
+def splitmix64_output(seed: int, index: int) -> int:
+    """Output number ``index`` (1-based) of the SplitMix64 stream whose state starts at ``seed``."""
+    z = (seed + index * 0x9E3779B97F4A7C15) & _M64
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & _M64
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & _M64
+    return z ^ (z >> 31)
+
+
+def dropout_threshold(p: float) -> int:
+    return int(round(p * 65536.0))
+
+
+def dropout_keep(seed: int, n_rows: int, d_in: int, p: float) -> np.ndarray:
+    """keep[m, k] (bool) for save-order rows m < n_rows and input columns k < d_in."""
+    thr = dropout_threshold(p)
+    keep = np.ones((n_rows, d_in), dtype=bool)
+    for m in range(n_rows):
+        for k4 in range((d_in + 3) // 4):
+            z = splitmix64_output(seed, ((m << 32) | k4) + 1)
+            for j in range(4):
+                k = 4 * k4 + j
+                if k < d_in:
+                    keep[m, k] = ((z >> (16 * j)) & 0xFFFF) >= thr
+    return keep
+
+
+def dropout_keep_vectorised(seed: int, n_rows: int, d_in: int, p: float) -> np.ndarray:
+    """Same mask as :func:`dropout_keep`, the generator written with numpy uint64 arrays (for the
+    large cases, where the Python loops would take minutes); pinned against the loop version."""
+    thr = dropout_threshold(p)
+    k4 = (d_in + 3) // 4
+    with np.errstate(over="ignore"):
+        c = (np.arange(n_rows, dtype=np.uint64)[:, None] << np.uint64(32)) | np.arange(k4, dtype=np.uint64)[None, :]
+        z = np.uint64(seed) + (c + np.uint64(1)) * np.uint64(0x9E3779B97F4A7C15)
+        z = (z ^ (z >> np.uint64(30))) * np.uint64(0xBF58476D1CE4E5B9)
+        z = (z ^ (z >> np.uint64(27))) * np.uint64(0x94D049BB133111EB)
+        z = z ^ (z >> np.uint64(31))
+    fields = np.stack([(z >> np.uint64(16 * j)) & np.uint64(0xFFFF) for j in range(4)], axis=-1)
+    return (fields.reshape(n_rows, 4 * k4)[:, :d_in] >= np.uint64(thr))
 
 
 # --------------------------------------------------------------------------------------
@@ -102,7 +166,7 @@ def route(segments, n_rows: int, n_adapters: int):
 # forward
 # --------------------------------------------------------------------------------------
 def forward(X, W, A_all, B_all, scale, segments, save_row_base: int = 0,
-            save_capacity_rows: Optional[int] = None) -> Dict[str, np.ndarray]:
+            save_capacity_rows: Optional[int] = None, dropout: Optional[Tuple[float, int]] = None) -> Dict[str, np.ndarray]:
     """Y = X W + s_a (X A_a^T) B_a per row, plus the activation save for fine-tuning rows.
 
     Shapes: X [T, d_in], W [d_in, d_out], A_all [n, r, d_in], B_all [n, r, d_out],
@@ -113,6 +177,9 @@ def forward(X, W, A_all, B_all, scale, segments, save_row_base: int = 0,
     Save order (Section 3.2: activations are appended to a buffer of limited capacity that
     the backward later consumes): fine-tuning segments in table order, rows in order inside
     each; a batch that does not fit the remaining capacity is refused.
+
+    ``dropout`` = (p, seed) switches LoRA dropout on for the fine-tuning rows (see the module
+    header); row m of the mask is the row's place in this batch's save order (without the base).
     """
     X, W, A_all, B_all, scale = _f64(X), _f64(W), _f64(A_all), _f64(B_all), _f64(scale)
     T, d_in = X.shape
@@ -123,13 +190,21 @@ def forward(X, W, A_all, B_all, scale, segments, save_row_base: int = 0,
     if save_row_base < 0 or save_row_base + ft_rows > cap:
         raise SegmentError("fine-tuning rows exceed the activation buffer capacity")
 
+    save_place = np.full(T, -1, dtype=np.int64)  # place of a fine-tuning row in this batch's save order
+    for start, length, _adapter, off in ft_segments:
+        save_place[start:start + length] = off + np.arange(length)
+    keep = dropout_keep(dropout[1], ft_rows, d_in, dropout[0]) if dropout is not None else None
+
     Y = X @ W                                   # the shared base pass
     U = np.zeros((T, r))
     for t in range(T):
         a = row_adapter[t]
         if a < 0:
             continue
-        U[t] = A_all[a] @ X[t]                  # shrink:  u = x A_a^T
+        x_lora = X[t]
+        if keep is not None and save_place[t] >= 0:
+            x_lora = X[t] * keep[save_place[t]] / (1.0 - dropout[0])   # dropout on the branch input
+        U[t] = A_all[a] @ x_lora                # shrink:  u = x A_a^T
         Y[t] += scale[a] * (U[t] @ B_all[a])    # expand:  y += s u B_a
 
     x_save = np.zeros((cap, d_in))
@@ -141,6 +216,30 @@ def forward(X, W, A_all, B_all, scale, segments, save_row_base: int = 0,
             u_save[m] = U[start + i]
     return {"Y": Y, "U": U, "x_save": x_save, "u_save": u_save, "ft_rows": ft_rows,
             "ft_adapters": ft_adapters, "row_adapter": row_adapter}
+
+
+def forward_ragged(X, W, A_list, B_list, scale, segments) -> np.ndarray:
+    """Y when adapter a has its own rank: ``A_list[a]`` [r_a, d_in], ``B_list[a]`` [r_a, d_out]."""
+    X, W, scale = _f64(X), _f64(W), _f64(scale)
+    row_adapter, _, _, _ = route(segments, X.shape[0], len(A_list))
+    Y = X @ W
+    for t in range(X.shape[0]):
+        a = row_adapter[t]
+        if a >= 0:
+            Y[t] += scale[a] * ((_f64(A_list[a]) @ X[t]) @ _f64(B_list[a]))
+    return Y
+
+
+def pad_adapters(A_list, B_list, r: int):
+    """Stack per-adapter matrices of different ranks into [n, r, d] arrays with zero rows."""
+    n = len(A_list)
+    A_all = np.zeros((n, r, np.asarray(A_list[0]).shape[1]))
+    B_all = np.zeros((n, r, np.asarray(B_list[0]).shape[1]))
+    for a in range(n):
+        ra = np.asarray(A_list[a]).shape[0]
+        A_all[a, :ra] = A_list[a]
+        B_all[a, :ra] = B_list[a]
+    return A_all, B_all
 
 
 def forward_rows(X, W, A_all, B_all, scale, segments, rows: Sequence[int]) -> np.ndarray:
@@ -160,7 +259,7 @@ def forward_rows(X, W, A_all, B_all, scale, segments, rows: Sequence[int]) -> np
 # backward (fine-tuning rows only, in save-buffer order)
 # --------------------------------------------------------------------------------------
 def backward(dY, W, A_all, B_all, scale, segments, x_save, u_save, n_rows: Optional[int] = None,
-             dA_init=None, dB_init=None) -> Dict[str, np.ndarray]:
+             dA_init=None, dB_init=None, dropout: Optional[Tuple[float, int]] = None) -> Dict[str, np.ndarray]:
     """LoRA gradients and input gradient for the fine-tuning rows.
 
     ``dY`` [ft_rows, d_out], ``x_save`` [ft_rows, d_in] and ``u_save`` [ft_rows, r] are in
@@ -186,19 +285,25 @@ def backward(dY, W, A_all, B_all, scale, segments, x_save, u_save, n_rows: Optio
     dB = np.zeros((len(ft_adapters), r, d_out)) if dB_init is None else _f64(dB_init).copy()
     dX = np.zeros((ft_rows, d_in))
     V = np.zeros((ft_rows, r))
+    keep = dropout_keep(dropout[1], ft_rows, d_in, dropout[0]) if dropout is not None else None
     for _start, length, a, off in ft_segments:
         g = ft_adapters.index(a)
         s = scale[a]
         for m in range(off, off + length):
             V[m] = s * (B_all[a] @ dY[m])                  # v = s dy B_a^T
             dB[g] += s * np.outer(u_save[m], dY[m])        # dB_a += s u^T dy
-            dA[g] += np.outer(V[m], x_save[m])             # dA_a += v^T x
-            dX[m] = W @ dY[m] + V[m] @ A_all[a]            # dx = dy W^T + v A_a
+            if keep is None:
+                dA[g] += np.outer(V[m], x_save[m])         # dA_a += v^T x
+                dX[m] = W @ dY[m] + V[m] @ A_all[a]        # dx = dy W^T + v A_a
+            else:
+                k = keep[m] / (1.0 - dropout[0])
+                dA[g] += np.outer(V[m], x_save[m] * k)     # the branch saw x * k
+                dX[m] = W @ dY[m] + (V[m] @ A_all[a]) * k
     return {"dA": dA, "dB": dB, "dX": dX, "V": V, "ft_adapters": ft_adapters}
 
 
 def backward_blocked(dY, W, A_all, B_all, scale, segments, x_save, u_save,
-                     n_rows: Optional[int] = None) -> Dict[str, np.ndarray]:
+                     n_rows: Optional[int] = None, dropout: Optional[Tuple[float, int]] = None) -> Dict[str, np.ndarray]:
     """Same result as :func:`backward`, one library matrix product per segment instead of one
     row at a time (the sums over a segment's rows are exactly the matrix products
     U^T dY, V^T X, dY W^T); used where the row loop would take minutes."""
@@ -214,17 +319,20 @@ def backward_blocked(dY, W, A_all, B_all, scale, segments, x_save, u_save,
     dB = np.zeros((len(ft_adapters), r, d_out))
     dX = np.zeros((ft_rows, d_in))
     V = np.zeros((ft_rows, r))
+    k = np.ones((ft_rows, d_in))
+    if dropout is not None:
+        k = dropout_keep_vectorised(dropout[1], ft_rows, d_in, dropout[0]) / (1.0 - dropout[0])
     for _start, length, a, off in ft_segments:
         g = ft_adapters.index(a)
         sl = slice(off, off + length)
         V[sl] = scale[a] * (dY[sl] @ B_all[a].T)
         dB[g] += scale[a] * (u_save[sl].T @ dY[sl])
-        dA[g] += V[sl].T @ x_save[sl]
-        dX[sl] = dY[sl] @ W.T + V[sl] @ A_all[a]
+        dA[g] += V[sl].T @ (x_save[sl] * k[sl])
+        dX[sl] = dY[sl] @ W.T + (V[sl] @ A_all[a]) * k[sl]
     return {"dA": dA, "dB": dB, "dX": dX, "V": V, "ft_adapters": ft_adapters}
 
 
-def forward_blocked(X, W, A_all, B_all, scale, segments) -> Dict[str, np.ndarray]:
+def forward_blocked(X, W, A_all, B_all, scale, segments, dropout: Optional[Tuple[float, int]] = None) -> Dict[str, np.ndarray]:
     """Same result as :func:`forward` (without the save buffers), one library product per
     segment instead of one row at a time; used for the timed CPU baseline and large cases."""
     X, W, A_all, B_all, scale = _f64(X), _f64(W), _f64(A_all), _f64(B_all), _f64(scale)
@@ -233,12 +341,18 @@ def forward_blocked(X, W, A_all, B_all, scale, segments) -> Dict[str, np.ndarray
     _ra, ft_segments, ft_rows, ft_adapters = route(segments, T, n)
     Y = X @ W
     U = np.zeros((T, r))
+    keep = dropout_keep_vectorised(dropout[1], ft_rows, X.shape[1], dropout[0]) if dropout is not None else None
+    ft_off = {(st, ln): off for st, ln, _a, off in ft_segments}
     for seg in np.asarray(segments, dtype=np.int64).reshape(-1, 4):
-        start, length, a, _ = (int(v) for v in seg)
+        start, length, a, is_ft = (int(v) for v in seg)
         if a < 0 or length == 0:
             continue
         sl = slice(start, start + length)
-        U[sl] = X[sl] @ A_all[a].T
+        x_lora = X[sl]
+        if keep is not None and is_ft:
+            off = ft_off[(start, length)]
+            x_lora = X[sl] * keep[off:off + length] / (1.0 - dropout[0])
+        U[sl] = x_lora @ A_all[a].T
         Y[sl] += scale[a] * (U[sl] @ B_all[a])
     x_save = np.zeros((ft_rows, X.shape[1]))
     u_save = np.zeros((ft_rows, r))
