@@ -197,6 +197,9 @@ def main():
     ap.add_argument("--with-update", action="store_true",
                     help="also run the AdamW update of the fine-tuned adapters after each backward (not part of the "
                          "headline step; reported under kernels.adamw)")
+    ap.add_argument("--dropout", type=float, default=0.0,
+                    help="LoRA dropout rate on the fine-tuning rows (the paper trains with 0.05; the headline step "
+                         "runs without it); a new seed every step")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -239,10 +242,15 @@ def main():
             opt.append([wA, wB] + [torch.zeros_like(x) for x in (wA, wA, wB, wB)])
     n_updates = [0]
 
+    n_steps_run = [0]
+
     def step():
         if args.with_update:
             n_updates[0] += 1
+        n_steps_run[0] += 1
         for i, r in enumerate(runs):
+            if args.dropout > 0:
+                mb.mlora_set_dropout(sess.ctx, args.dropout, (n_steps_run[0] << 8) + i)
             r.forward()
             r.backward()
             if args.with_update:
@@ -406,7 +414,7 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": label, "rows_per_step": T, "ft_rows_per_step": workloads[0].ft_rows,
+        "config": {"workload": label + (f" + LoRA dropout {args.dropout}" if args.dropout > 0 else ""), "rows_per_step": T, "ft_rows_per_step": workloads[0].ft_rows,
                    "l2_policy": f"inputs larger than L2: one step touches {resident / 1e6:.0f} MB of weights and "
                                 f"activations, so nothing survives in the 126 MB L2 from step to step",
                    "parallelism": "replicas (rows are independent; no collective)" if world > 1 else "single GPU"},

@@ -175,6 +175,27 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* layer, const 
  * which learns of the request before its next launch, so no kernel ever waits on it.) */
 mlora_status_t mlora_set_cancel_flag(mlora_ctx* ctx, const volatile int32_t* host_flag);
 
+/* ---- LoRA dropout on the fine-tuning rows --------------------------------------------------*/
+
+/* Switches dropout of the low-rank branch's input on (0 < p < 1) or off (p == 0) for the compute
+ * calls that follow on this context.  (Paper, Section 5 "Fine-tuning Workload": the adapter is
+ * trained with dropout 0.05; reading: the usual LoRA placement y = x W + s B A dropout(x), on
+ * fine-tuning rows only - inference rows and the base product never see it.)
+ * The keep decision of element (m, k) - m the row's place in the batch's save order, counted from
+ * the first row the plan saves, k the input column - is output number c + 1 of the SplitMix64
+ * stream started at `seed`, c = m * 2^32 + (k >> 2); its 16-bit field k & 3 is compared with
+ * round(p * 65536) (ties to even), values below it are dropped; kept elements count 1 / (1 - p).
+ * Forward:  u_save and Y use the dropped input, x_save keeps the row as it is.
+ * Backward: dA = (V / (1 - p))^T (x_save * keep), dX = dY W^T + (V A) * keep / (1 - p); V and dB
+ * keep their form.  The forward and the backward of one batch must run under the same (p, seed);
+ * the caller changes the seed from step to step and from layer to layer.  A captured graph keeps
+ * the values it was captured with.
+ * Supported for fp32 layers and for bf16 layers of rank <= 32 on the default kernel path;
+ * otherwise the compute call returns MLORA_ERR_UNSUPPORTED.  With dropout on, the low-rank part
+ * of dX is added by one extra elementwise kernel after the base product.
+ * Errors: MLORA_ERR_INVALID_ARG (NULL context, p outside [0, 1)). */
+mlora_status_t mlora_set_dropout(mlora_ctx* ctx, double p, uint64_t seed);
+
 /* ---- optimizer step on the fine-tuned adapters ------------------------------------------*/
 
 /* AdamW hyper-parameters (paper, Section 5 "Fine-tuning Workload": AdamW, learning rate 1e-3,

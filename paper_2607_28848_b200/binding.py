@@ -25,7 +25,7 @@ EXPORTS = (
     "mlora_plan_ft_rows", "mlora_plan_ft_adapters", "mlora_plan_describe", "mlora_mixed_forward",
     "mlora_backward", "mlora_poll_status", "mlora_status_string", "mlora_launch_count", "mlora_set_gemm_path",
     "mlora_profile_enable", "mlora_profile_collect", "mlora_forward_noalloc", "mlora_adamw_update",
-    "mlora_set_cancel_flag",
+    "mlora_set_cancel_flag", "mlora_set_dropout",
 )
 MLORA_NOALLOC_MAX_ROWS = 512
 
@@ -106,6 +106,8 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.mlora_adamw_update.restype = ctypes.c_int
     lib.mlora_set_cancel_flag.argtypes = [vp, P(i32)]
     lib.mlora_set_cancel_flag.restype = ctypes.c_int
+    lib.mlora_set_dropout.argtypes = [vp, ctypes.c_double, ctypes.c_uint64]
+    lib.mlora_set_dropout.restype = ctypes.c_int
     lib.mlora_forward_noalloc.argtypes = [P(mlora_layer_t), vp, i32, vp, i64, vp, i64, vp]
     lib.mlora_forward_noalloc.restype = ctypes.c_int
     _lib = lib
@@ -282,3 +284,8 @@ def mlora_set_cancel_flag(ctx, flag) -> None:
     """Register a host flag (a ctypes.c_int32 the caller keeps alive, or None) checked before every launch."""
     ptr = None if flag is None else ctypes.pointer(flag)
     _check(load_library().mlora_set_cancel_flag(ctx, ptr), "mlora_set_cancel_flag")
+
+
+def mlora_set_dropout(ctx, p: float, seed: int) -> None:
+    """LoRA dropout of the fine-tuning rows' branch input for the calls that follow (p = 0: off)."""
+    _check(load_library().mlora_set_dropout(ctx, float(p), int(seed) & 0xFFFFFFFFFFFFFFFF), "mlora_set_dropout")

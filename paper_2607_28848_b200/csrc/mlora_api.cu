@@ -43,6 +43,7 @@ struct mlora_ctx {
   int32_t gemm_pairs = 1;            // 1: two-SM (CTA pair) tensor-core kernel; 0: one-SM kernel
   EncodeTiledFn encode = nullptr;
   const volatile int32_t* cancel = nullptr;   // caller's host flag, read before every launch
+  DropArgs drop = {0, 0, 1.0f};               // LoRA dropout of the fine-tuning rows (thr == 0: off)
   // optional per-launch timing
   std::vector<cudaEvent_t> ev_start, ev_stop;
   std::vector<int32_t> ev_kind;
@@ -238,6 +239,7 @@ mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, c
   sa.s.counters = ctx->ws_counters;
   sa.n_items = n_items;
   sa.tma_save = tma_save ? 1 : 0;
+  sa.drop = a.item_save ? ctx->drop : DropArgs{0, 0, 1.0f};   // only the forward's fine-tuning rows are dropped
   sa.chunks_per_item = (a.D / 64 + CHUNK - 1) / CHUNK;
   sa.n_units = n_items * sa.chunks_per_item;
   int grid = sa.n_units < ctx->sm_count ? sa.n_units : ctx->sm_count;
@@ -293,8 +295,8 @@ mlora_status_t launch_grad_stream2(mlora_ctx* ctx, const mlora_plan* p, const Gr
   if ((ms = make_tmap_bf16(ctx, &tQ0, gb.Q, gb.D, n_rows, gb.ldq, 64, 128)) != MLORA_OK) return ms;
   if ((ms = make_tmap_bf16(ctx, &tQ1, ga_.Q, ga_.D, n_rows, ga_.ldq, 64, 128)) != MLORA_OK) return ms;
   GradStreamArgs g;
-  g.prob[0] = GradProblem{gb.P, gb.scale, gb.G, gb.D, gb.D / 64};
-  g.prob[1] = GradProblem{ga_.P, ga_.scale, ga_.G, ga_.D, ga_.D / 64};
+  g.prob[0] = GradProblem{gb.P, gb.scale, gb.G, gb.D, gb.D / 64, DropArgs{0, 0, 1.0f}};
+  g.prob[1] = GradProblem{ga_.P, ga_.scale, ga_.G, ga_.D, ga_.D / 64, ctx->drop};   // dA sees the dropped branch input
   g.n_problems = 2; g.R = gb.R; g.accumulate = gb.accumulate;
   g.slot_adapter = p->slot_adapter; g.slot_blk_off = p->slot_blk_off; g.blk_row0 = p->blk_row0; g.blk_nrows = p->blk_nrows;
   g.n_slots = n_slots; g.status = ctx->status_dev;
@@ -323,6 +325,20 @@ mlora_status_t launch_grad(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& 
   } else {
     launch_pdl(scope.slot < 0, grad_kernel<2>, dim3(a.D / 64, n_slots, (a.R + 31) / 32), dim3(GRAD_THREADS), smem2, st, a);
   }
+  return scope.done();
+}
+
+// dX += keep * (V A_a) / (1 - p): the low-rank part of the input gradient under dropout, after the
+// base product has been written by the GEMM.
+mlora_status_t launch_expand_mask(mlora_ctx* ctx, const mlora_layer_t* L, const DevRowSpace& ds, void* dX, int64_t lddx,
+                                  int n_rows, cudaStream_t st) {
+  if (n_rows <= 0) return MLORA_OK;
+  if (cancelled(ctx)) return MLORA_CANCELLED;
+  ExpandMaskArgs a;
+  a.V = ctx->ws_p; a.R = L->rank; a.A_all = (const __nv_bfloat16*)L->A_all; a.row_adapter = ds.row_adapter;
+  a.dX = (__nv_bfloat16*)dX; a.lddx = lddx; a.D = L->d_in; a.n_rows = n_rows; a.drop = ctx->drop;
+  LaunchScope scope(ctx, st, KIND_SHRINK);
+  launch_pdl(scope.slot < 0, expand_mask_kernel, dim3(n_rows, (L->d_in / 8 + 127) / 128), dim3(128), 0, st, a);
   return scope.done();
 }
 
@@ -399,7 +415,7 @@ mlora_status_t launch_gemm(mlora_ctx* ctx, int R, const CUtensorMap& tIn, const 
 template <bool W_KMAJOR>
 mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace& hs, const DevRowSpace& ds,
                          const void* In, int64_t ld_in, void* Out, int64_t ld_out, const void* L_all,
-                         const float* P, const float* scale, int M, int N, int K, cudaStream_t st) {
+                         const float* P, const float* scale, int M, int N, int K, cudaStream_t st, bool lora = true) {
   CUtensorMap tIn, tW, tL, tOut;
   mlora_status_t s;
   if ((s = make_tmap_bf16(ctx, &tIn, In, K, M, ld_in, GEMM_BK, GEMM_BM)) != MLORA_OK) return s;
@@ -418,7 +434,7 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
     g.n_mtiles = (M + GEMM2_BM - 1) / GEMM2_BM;
     g.n_ntiles = (N + GEMM2_BN - 1) / GEMM2_BN;
     g.n_full = g.n_units = g.n_mtiles * g.n_ntiles;
-    g.lora_enabled = hs.grp2_adapter.empty() ? 0 : 1;
+    g.lora_enabled = (lora && !hs.grp2_adapter.empty()) ? 1 : 0;
     g.row_grp = ds.row_grp2; g.row_adapter = ds.row_adapter;
     g.tile_grp_off = ds.tile2_grp_off; g.grp_adapter = ds.grp2_adapter;
     g.P = P; g.scale = scale; g.status = ctx->status_dev;
@@ -440,7 +456,7 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
     g.n_full = split ? tiles - rem : tiles;
     g.n_units = split ? tiles + rem : tiles;
   }
-  g.lora_enabled = hs.grp_adapter.empty() ? 0 : 1;
+  g.lora_enabled = (lora && !hs.grp_adapter.empty()) ? 1 : 0;
   g.row_grp = ds.row_grp; g.row_adapter = ds.row_adapter;
   g.tile_grp_off = ds.tile_grp_off; g.grp_adapter = ds.grp_adapter;
   g.P = P; g.scale = scale; g.status = ctx->status_dev;
@@ -451,51 +467,52 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
 template <typename T>
 mlora_status_t simt_shrink(mlora_ctx* ctx, const T* In, int64_t ld_in, int D, int R, const T* P_all,
                            const float* scale, const DevRowSpace& ds, float* Out, T* x_save, float* u_save,
-                           int64_t save_base, int n_rows, cudaStream_t st) {
+                           int64_t save_base, int n_rows, const DropArgs& drop, cudaStream_t st) {
   if (n_rows <= 0) return MLORA_OK;
   if (cancelled(ctx)) return MLORA_CANCELLED;
   const int64_t warps = (int64_t)n_rows * R;
   const int blocks = (int)((warps * 32 + 255) / 256);
   LaunchScope scope(ctx, st, KIND_SIMT);
   simt::shrink_kernel<T><<<blocks, 256, 0, st>>>(In, ld_in, D, R, P_all, scale, ds.row_adapter, ds.row_save, Out,
-                                                 x_save, u_save, save_base, n_rows);
+                                                 x_save, u_save, save_base, n_rows, drop);
   return scope.done();
 }
 
 template <typename T, bool W_KMAJOR>
 mlora_status_t simt_gemm(mlora_ctx* ctx, const T* In, int64_t ld_in, const T* W, int64_t ldw, const T* L_all,
                          const float* P, const float* scale, const DevRowSpace& ds, T* Out, int64_t ld_out, int M,
-                         int N, int K, int R, cudaStream_t st) {
+                         int N, int K, int R, const DropArgs& drop, cudaStream_t st) {
   if (M <= 0) return MLORA_OK;
   if (cancelled(ctx)) return MLORA_CANCELLED;
   dim3 grid((N + 31) / 32, (M + 31) / 32), block(32, 32);
   LaunchScope scope(ctx, st, KIND_SIMT);
   simt::gemm_lora_kernel<T, W_KMAJOR><<<grid, block, 0, st>>>(In, ld_in, W, ldw, L_all, P, scale, ds.row_adapter, Out,
-                                                              ld_out, M, N, K, R);
+                                                              ld_out, M, N, K, R, drop);
   return scope.done();
 }
 
 template <typename T>
 mlora_status_t simt_grad(mlora_ctx* ctx, const mlora_plan* p, const float* P, int R, const float* scale, const T* Q,
-                         int64_t ldq, int D, float* G, int accumulate, cudaStream_t st) {
+                         int64_t ldq, int D, float* G, int accumulate, const DropArgs& drop, cudaStream_t st) {
   const int n_slots = (int)p->h.ft_adapters.size();
   if (n_slots <= 0) return MLORA_OK;
   if (cancelled(ctx)) return MLORA_CANCELLED;
   dim3 grid((D + 127) / 128, R, n_slots);
   LaunchScope scope(ctx, st, KIND_SIMT);
   simt::grad_kernel<T><<<grid, 128, 0, st>>>(P, R, scale, Q, ldq, D, G, p->slot_chunk_off, p->chunk_row0,
-                                             p->chunk_nrows, p->slot_adapter, accumulate);
+                                             p->chunk_nrows, p->slot_adapter, accumulate, drop);
   return scope.done();
 }
 
 template <typename T>
 mlora_status_t forward_simt(mlora_ctx* ctx, const mlora_layer_t* L, const mlora_plan* p, const void* X, int64_t ldx,
                             void* Y, int64_t ldy, void* x_save, float* u_save, int64_t save_base, cudaStream_t st) {
+  const DropArgs off = {0, 0, 1.0f};
   mlora_status_t s = simt_shrink<T>(ctx, (const T*)X, ldx, L->d_in, L->rank, (const T*)L->A_all, nullptr, p->fwd,
-                                    ctx->ws_p, (T*)x_save, u_save, save_base, p->h.n_rows, st);
+                                    ctx->ws_p, (T*)x_save, u_save, save_base, p->h.n_rows, ctx->drop, st);
   if (s != MLORA_OK) return s;
   return simt_gemm<T, false>(ctx, (const T*)X, ldx, (const T*)L->W, L->ldw, (const T*)L->B_all, ctx->ws_p, L->scale,
-                             p->fwd, (T*)Y, ldy, p->h.n_rows, L->d_out, L->d_in, L->rank, st);
+                             p->fwd, (T*)Y, ldy, p->h.n_rows, L->d_out, L->d_in, L->rank, off, st);
 }
 
 template <typename T>
@@ -503,17 +520,18 @@ mlora_status_t backward_simt(mlora_ctx* ctx, const mlora_layer_t* L, const mlora
                              const void* x_save, const float* u_save, float* dA, float* dB, void* dX, int64_t lddx,
                              int accumulate, cudaStream_t st) {
   const int Tft = p->h.ft_rows;
+  const DropArgs off = {0, 0, 1.0f};
   mlora_status_t s = simt_shrink<T>(ctx, (const T*)dY, lddy, L->d_out, L->rank, (const T*)L->B_all, L->scale, p->bwd,
-                                    ctx->ws_p, (T*)nullptr, nullptr, 0, Tft, st);
+                                    ctx->ws_p, (T*)nullptr, nullptr, 0, Tft, off, st);
   if (s != MLORA_OK) return s;
-  if ((s = simt_grad<T>(ctx, p, u_save, L->rank, L->scale, (const T*)dY, lddy, L->d_out, dB, accumulate, st)) != MLORA_OK)
+  if ((s = simt_grad<T>(ctx, p, u_save, L->rank, L->scale, (const T*)dY, lddy, L->d_out, dB, accumulate, off, st)) != MLORA_OK)
     return s;
-  if ((s = simt_grad<T>(ctx, p, ctx->ws_p, L->rank, nullptr, (const T*)x_save, L->d_in, L->d_in, dA, accumulate, st)) !=
-      MLORA_OK)
+  if ((s = simt_grad<T>(ctx, p, ctx->ws_p, L->rank, nullptr, (const T*)x_save, L->d_in, L->d_in, dA, accumulate, ctx->drop,
+                        st)) != MLORA_OK)
     return s;
   if (dX)
     s = simt_gemm<T, true>(ctx, (const T*)dY, lddy, (const T*)L->W, L->ldw, (const T*)L->A_all, ctx->ws_p, nullptr,
-                           p->bwd, (T*)dX, lddx, Tft, L->d_in, L->d_out, L->rank, st);
+                           p->bwd, (T*)dX, lddx, Tft, L->d_in, L->d_out, L->rank, ctx->drop, st);
   return s;
 }
 
@@ -554,12 +572,13 @@ mlora_status_t forward_noalloc_t(const mlora_layer_t* L, const int32_t* row_adap
   const int blocks = (int)((warps * 32 + 255) / 256);
   // rank-r intermediate of every row (zeros for rows without an adapter) -> scratch
   simt::shrink_kernel<T><<<blocks, 256, 0, st>>>((const T*)X, ldx, L->d_in, L->rank, (const T*)L->A_all, nullptr,
-                                                 row_adapter, nullptr, scratch, (T*)nullptr, nullptr, 0, n_rows);
+                                                 row_adapter, nullptr, scratch, (T*)nullptr, nullptr, 0, n_rows,
+                                                 DropArgs{0, 0, 1.0f});
   if (cudaGetLastError() != cudaSuccess) return MLORA_ERR_CUDA;
   dim3 grid((L->d_out + 31) / 32, (n_rows + 31) / 32), block(32, 32);
   simt::gemm_lora_kernel<T, false><<<grid, block, 0, st>>>((const T*)X, ldx, (const T*)L->W, L->ldw,
                                                            (const T*)L->B_all, scratch, L->scale, row_adapter, (T*)Y,
-                                                           ldy, n_rows, L->d_out, L->d_in, L->rank);
+                                                           ldy, n_rows, L->d_out, L->d_in, L->rank, DropArgs{0, 0, 1.0f});
   return cudaGetLastError() == cudaSuccess ? MLORA_OK : MLORA_ERR_CUDA;
 }
 }  // namespace
@@ -798,6 +817,7 @@ mlora_status_t mlora_mixed_forward(mlora_ctx* ctx, const mlora_layer_t* L, const
   if (ctx->gemm_path == 1)
     return forward_simt<__nv_bfloat16>(ctx, L, p, X, ldx, Y, ldy, x_save, u_save, save_row_base, st);
 
+  if (ctx->drop.thr != 0 && h.ft_rows > 0 && (ctx->shrink_path != 0 || L->rank > 32)) return MLORA_ERR_UNSUPPORTED;
   ShrinkArgs sa;
   sa.In = (const __nv_bfloat16*)X; sa.ld_in = ldx; sa.D = L->d_in;
   sa.P_all = (const __nv_bfloat16*)L->A_all; sa.scale = nullptr; sa.Out = ctx->ws_p;
@@ -832,11 +852,13 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
     return backward_simt<__nv_bfloat16>(ctx, L, p, dY, lddy, x_save, u_save, dA, dB, dX, lddx, accumulate, st);
 
   const int n_slots = (int)h.ft_adapters.size();
+  const bool dropping = ctx->drop.thr != 0;
+  if (dropping && (ctx->shrink_path != 0 || L->rank > 32)) return MLORA_ERR_UNSUPPORTED;
   ShrinkArgs sa;                     // V = s dY B^T
   sa.In = (const __nv_bfloat16*)dY; sa.ld_in = lddy; sa.D = L->d_out;
   sa.P_all = (const __nv_bfloat16*)L->B_all; sa.scale = L->scale; sa.Out = ctx->ws_p;
   sa.item_rows = p->bwd.item_rows; sa.item_start = p->bwd.item_start; sa.item_nrows = p->bwd.item_nrows;
-  sa.pbd = PbdArgs{(ctx->gemm_pairs && dX) ? ctx->ws_pbd : nullptr, p->bwd.row_grp2, p->bwd.tile2_grp_off, nullptr,
+  sa.pbd = PbdArgs{(ctx->gemm_pairs && dX && !dropping) ? ctx->ws_pbd : nullptr, p->bwd.row_grp2, p->bwd.tile2_grp_off, nullptr,
                    p->bwd.zero_rows2, (int32_t)h.bwd.zero_rows2.size()};
   sa.item_adapter = p->bwd.item_adapter; sa.item_save = nullptr; sa.x_save = nullptr; sa.u_save = nullptr; sa.save_base = 0; sa.save_cap = 0;
   if ((s = launch_shrink(ctx, L->rank, sa, h.bwd.n_items(), p->bwd.item_desc, h.ft_rows, L->n_adapters, st)) != MLORA_OK)
@@ -853,6 +875,12 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
                       : launch_grad_stream2<2>(ctx, p, ga, gA, n_slots, h.ft_rows, st);
     if (s != MLORA_OK) return s;
     if (!dX) return MLORA_OK;
+    if (dropping) {   // the mask acts on the low-rank term per element: base product first, then the masked expand
+      if ((s = gemm_bf16<true>(ctx, L, h.bwd, p->bwd, dY, lddy, dX, lddx, L->A_all, ctx->ws_p, nullptr, h.ft_rows,
+                               L->d_in, L->d_out, st, false)) != MLORA_OK)
+        return s;
+      return launch_expand_mask(ctx, L, p->bwd, dX, lddx, h.ft_rows, st);
+    }
     return gemm_bf16<true>(ctx, L, h.bwd, p->bwd, dY, lddy, dX, lddx, L->A_all, ctx->ws_p, nullptr, h.ft_rows, L->d_in,
                            L->d_out, st);
   }
@@ -913,6 +941,14 @@ mlora_status_t mlora_poll_status(mlora_ctx* ctx, void* cuda_stream) {
 mlora_status_t mlora_set_cancel_flag(mlora_ctx* ctx, const volatile int32_t* host_flag) {
   if (!ctx) return MLORA_ERR_INVALID_ARG;
   ctx->cancel = host_flag;
+  return MLORA_OK;
+}
+
+mlora_status_t mlora_set_dropout(mlora_ctx* ctx, double p, uint64_t seed) {
+  if (!ctx || !(p >= 0.0 && p < 1.0)) return MLORA_ERR_INVALID_ARG;
+  ctx->drop.seed = seed;
+  ctx->drop.thr = (uint32_t)std::nearbyint(p * 65536.0);      // ties to even, as the oracle's rounding
+  ctx->drop.keep_scale = (float)(1.0 / (1.0 - p));
   return MLORA_OK;
 }
 

@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "dropout.cuh"
+
 namespace mlora {
 namespace simt {
 
@@ -16,11 +18,12 @@ __device__ __forceinline__ void st(float* p, float v) { *p = v; }
 __device__ __forceinline__ void st(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 
 // Out[t, q] = (scale?) * sum_k In[t, k] P_a(t)[q, k]; one warp per (row, q); rows without an
-// adapter get zeros.  Fine-tuning rows (row_save >= 0) also write u_save (unscaled) and x_save.
+// adapter get zeros.  Fine-tuning rows (row_save >= 0) also write u_save (unscaled) and x_save;
+// with dropout on, their products skip the dropped columns and count 1 / (1 - p).
 template <typename T>
 __global__ void shrink_kernel(const T* In, int64_t ld_in, int D, int R, const T* P_all, const float* scale,
                               const int32_t* row_adapter, const int32_t* row_save, float* Out,
-                              T* x_save, float* u_save, int64_t save_base, int n_rows) {
+                              T* x_save, float* u_save, int64_t save_base, int n_rows, const DropArgs drop) {
   const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (wid >= n_rows * R) return;
@@ -31,9 +34,15 @@ __global__ void shrink_kernel(const T* In, int64_t ld_in, int D, int R, const T*
   if (a >= 0) {
     const T* x = In + (size_t)t * ld_in;
     const T* p = P_all + ((size_t)a * R + q) * D;
-    for (int k = lane; k < D; k += 32) acc = fmaf(ld(x + k), ld(p + k), acc);
+    if (drop.thr != 0 && sv >= 0) {
+      for (int k = lane; k < D; k += 32)
+        if (drop_keep(drop, (uint32_t)sv, (uint32_t)k)) acc = fmaf(ld(x + k), ld(p + k), acc);
+    } else {
+      for (int k = lane; k < D; k += 32) acc = fmaf(ld(x + k), ld(p + k), acc);
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (drop.thr != 0 && sv >= 0) acc *= drop.keep_scale;
   }
   if (lane == 0) {
     Out[(size_t)t * R + q] = (a >= 0 && scale) ? acc * scale[a] : acc;
@@ -48,10 +57,12 @@ __global__ void shrink_kernel(const T* In, int64_t ld_in, int D, int R, const T*
 
 // Out[m, n] = sum_k In[m, k] Wop(k, n) + sum_q P[m, q] sc L_a(m)[q, n], 32 x 32 tiles.
 // W_KMAJOR: Wop(k, n) = W[n * ldw + k]; else Wop(k, n) = W[k * ldw + n].
+// With `drop` on (input gradient only) the low-rank term of element (m, n) is kept or dropped
+// as the branch input (m, n) was in the forward.
 template <typename T, bool W_KMAJOR>
 __global__ void gemm_lora_kernel(const T* In, int64_t ld_in, const T* W, int64_t ldw, const T* L_all,
                                  const float* P, const float* scale, const int32_t* row_adapter,
-                                 T* Out, int64_t ld_out, int M, int N, int K, int R) {
+                                 T* Out, int64_t ld_out, int M, int N, int K, int R, const DropArgs drop) {
   __shared__ float sIn[32][33];
   __shared__ float sW[32][33];
   const int tx = threadIdx.x, ty = threadIdx.y;
@@ -78,6 +89,7 @@ __global__ void gemm_lora_kernel(const T* In, int64_t ld_in, const T* W, int64_t
       const float sc = scale ? scale[a] : 1.0f;
       float lo = 0.f;
       for (int q = 0; q < R; ++q) lo = fmaf(P[(size_t)m * R + q], ld(L_all + ((size_t)a * R + q) * N + n), lo);
+      if (drop.thr != 0) lo = drop_keep(drop, (uint32_t)m, (uint32_t)n) ? lo * drop.keep_scale : 0.f;
       acc = fmaf(sc, lo, acc);
     }
     st(Out + (size_t)m * ld_out + n, acc);
@@ -85,18 +97,22 @@ __global__ void gemm_lora_kernel(const T* In, int64_t ld_in, const T* W, int64_t
 }
 
 // G[slot, q, j] (+)= sum over the slot's rows of sc P[t, q] Q[t, j]; one thread per (q, j).
+// With `drop` on (dA only: Q = the saved branch input) element (t, j) of Q is kept or dropped.
 template <typename T>
 __global__ void grad_kernel(const float* P, int R, const float* scale, const T* Q, int64_t ldq, int D, float* G,
                             const int32_t* slot_chunk_off, const int32_t* chunk_row0, const int32_t* chunk_nrows,
-                            const int32_t* slot_adapter, int accumulate) {
+                            const int32_t* slot_adapter, int accumulate, const DropArgs drop) {
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   const int q = blockIdx.y, slot = blockIdx.z;
   if (j >= D) return;
-  const float sc = scale ? scale[slot_adapter[slot]] : 1.0f;
+  const float sc = (scale ? scale[slot_adapter[slot]] : 1.0f) * (drop.thr != 0 ? drop.keep_scale : 1.0f);
   float acc = 0.f;
   for (int ch = slot_chunk_off[slot]; ch < slot_chunk_off[slot + 1]; ++ch) {
     const int r0 = chunk_row0[ch], nr = chunk_nrows[ch];
-    for (int t = r0; t < r0 + nr; ++t) acc = fmaf(P[(size_t)t * R + q] * sc, ld(Q + (size_t)t * ldq + j), acc);
+    for (int t = r0; t < r0 + nr; ++t) {
+      if (drop.thr != 0 && !drop_keep(drop, (uint32_t)t, (uint32_t)j)) continue;
+      acc = fmaf(P[(size_t)t * R + q] * sc, ld(Q + (size_t)t * ldq + j), acc);
+    }
   }
   float* dst = G + ((size_t)slot * R + q) * D + j;
   *dst = accumulate ? *dst + acc : acc;

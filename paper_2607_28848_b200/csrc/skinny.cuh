@@ -11,6 +11,7 @@
 //  grad_kernel   : G_g[q, j] = sum_{rows t of slot g} P[t, q] * Q[t, j]   (dB = (s U)^T dY, dA = V^T X)
 #pragma once
 
+#include "dropout.cuh"
 #include "plan.h"
 #include "ptx.cuh"
 
@@ -275,6 +276,7 @@ struct StreamArgs {
   int32_t* status;           // device status word
   const int32_t* item_desc;    // [n_items][kItemDescInts] packed item records (see RowSpace::item_desc)
   int32_t tma_save;            // 1: tmSave covers x_save; full contiguous fine-tuning items are saved as blocks
+  DropArgs drop;               // dropout of the fine-tuning rows' branch input (thr == 0: off)
 };
 
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -437,6 +439,7 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
     const int32_t* cur_rows = nullptr;
     const int32_t* cur_saves = nullptr;
     __nv_bfloat16* sp[4] = {nullptr, nullptr, nullptr, nullptr};
+    int msave[4] = {-1, -1, -1, -1};       // save-order place of rows g + 8 j (dropout counter), -1: not a fine-tuning row
     // flush-time values fetched when the item starts: element idx = tid + 256 k of the item's
     // [rows][R] result belongs to row idx / R
     int my_row[RB], my_save[RB];
@@ -474,14 +477,15 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int rl = g + 8 * j;
-          const int sv = (!block_saved && cur_saves && a.x_save && rl < cur_nrows) ? cur_saves[rl] : -1;
-          sp[j] = sv >= 0 ? a.x_save + (size_t)(a.save_base + sv) * a.D + 16 * c : nullptr;
+          msave[j] = (cur_saves && rl < cur_nrows) ? cur_saves[rl] : -1;
+          sp[j] = (!block_saved && a.x_save && msave[j] >= 0)
+                      ? a.x_save + (size_t)(a.save_base + msave[j]) * a.D + 16 * c : nullptr;
         }
 #pragma unroll
         for (int k = 0; k < RB; ++k) {
           const int r = ((int)threadIdx.x + k * STREAM_WARPS * 32) / R;
           my_row[k] = r < cur_nrows ? cur_rows[r] : -1;
-          my_save[k] = (r < cur_nrows && cur_saves && a.u_save) ? cur_saves[r] : -1;
+          my_save[k] = (r < cur_nrows && cur_saves) ? cur_saves[r] : -1;
         }
         my_scale = a.scale ? a.scale[cur_adapter] : 1.0f;
       }
@@ -528,10 +532,25 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
           p[n][0] = lds_v4(rp + sw0);
           p[n][1] = lds_v4(rp + sw1);
         }
+        const int ko = kb * 64;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (sp[j]) {     // activation save of rows that are not block-saved: they pass through here exactly once
+            *reinterpret_cast<uint4*>(sp[j] + ko) = x[j][0];
+            *reinterpret_cast<uint4*>(sp[j] + ko + 8) = x[j][1];
+          }
         // rows past the item's end were not copied: keep their stale bytes out of the MMA
 #pragma unroll
         for (int j = 0; j < 4; ++j)
           if (g + 8 * j >= cur_nrows) { x[j][0] = make_uint4(0, 0, 0, 0); x[j][1] = make_uint4(0, 0, 0, 0); }
+        if (sa.drop.thr != 0) {     // dropout: the saved copy above keeps the row as it is, the product does not
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (msave[j] >= 0) {
+              drop_mask8(sa.drop, (uint32_t)msave[j], (uint32_t)(ko + 16 * c), x[j][0]);
+              drop_mask8(sa.drop, (uint32_t)msave[j], (uint32_t)(ko + 16 * c + 8), x[j][1]);
+            }
+        }
 #pragma unroll
         for (int n = 0; n < RB; ++n) {
           const uint32_t rp[8] = {p[n][0].x, p[n][0].y, p[n][0].z, p[n][0].w, p[n][1].x, p[n][1].y, p[n][1].z, p[n][1].w};
@@ -550,13 +569,6 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
             }
           }
         }
-        const int ko = kb * 64;
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-          if (sp[j]) {     // activation save of rows that are not block-saved: they pass through here exactly once
-            *reinterpret_cast<uint4*>(sp[j] + ko) = x[j][0];
-            *reinterpret_cast<uint4*>(sp[j] + ko + 8) = x[j][1];
-          }
       }
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(bar_empty(st));        // the stage's bytes are in registers now
@@ -622,10 +634,11 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
 #pragma unroll
             for (int w = 0; w < RW; ++w) v += red[w][r][q];
           }
+          if (sa.drop.thr != 0 && my_save[k] >= 0) v *= sa.drop.keep_scale;
           const float vs = v * my_scale;
           a.Out[(size_t)my_row[k] * R + q] = vs;
           fin[r][q] = vs;
-          if (my_save[k] >= 0) a.u_save[(size_t)(a.save_base + my_save[k]) * R + q] = v;
+          if (my_save[k] >= 0 && a.u_save) a.u_save[(size_t)(a.save_base + my_save[k]) * R + q] = v;
         }
         if (c0 != c1 && threadIdx.x == 0) a.counters[this_item] = 0;    // ready for the next launch
         if (a.pbd.pbd) {
@@ -790,6 +803,7 @@ struct GradProblem {
   const float* scale;          // nullable
   float* G;                    // [n_slots, R, D]
   int32_t D, n_strips;         // D / 64
+  DropArgs drop;               // dA with dropout: Q elements kept or dropped, P counts keep_scale (thr == 0: off)
 };
 struct GradStreamArgs {
   GradProblem prob[2];
@@ -885,7 +899,7 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
       const GradProblem& pr = ga.prob[pi];
       const int gl = grp - pi * groups0;
       const int slot = gl / pr.n_strips, strip = gl % pr.n_strips;
-      const float sc = pr.scale ? pr.scale[ga.slot_adapter[slot]] : 1.0f;
+      const float sc = (pr.scale ? pr.scale[ga.slot_adapter[slot]] : 1.0f) * (pr.drop.thr != 0 ? pr.drop.keep_scale : 1.0f);
 #pragma unroll
       for (int m = 0; m < MB; ++m)
 #pragma unroll
@@ -893,6 +907,7 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
       for (int b = ga.slot_blk_off[slot]; b < ga.slot_blk_off[slot + 1]; ++b, ++i) {
         const int st = i % S;
         const int nrows = ga.blk_nrows[b];
+        const int brow0 = ga.blk_row0[b];
 #ifdef MLORA_TIMELINE
         const long long tw0 = tl_clock();
 #endif
@@ -913,6 +928,7 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
             // 16-byte piece g of row r sits at piece (g ^ (r & 7)) of the swizzled 128-byte row
             q[k] = lds_v4(qbase + (uint32_t)r * 128u + (uint32_t)((g ^ (r & 7)) << 4));
             if (r >= nrows) q[k] = make_uint4(0, 0, 0, 0);      // rows of the tile past the block's end
+            else if (pr.drop.thr != 0) drop_mask8(pr.drop, (uint32_t)(brow0 + r), (uint32_t)(strip * 64 + 8 * g), q[k]);
           }
 #pragma unroll
           for (int m = 0; m < MB; ++m) {
@@ -991,6 +1007,60 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
     if (tl_on) { MLORA_TL_SET(9, tl_clock() - tl0); MLORA_TL_SET(15, tl_global()); MLORA_TL_SET(10, tl_nstage); MLORA_TL_SET(8, tl_wait); MLORA_TL_SET(6, tl_flush); MLORA_TL_SET(7, tl_nflush); }
 #endif
   }
+}
+
+// Low-rank part of the input gradient under dropout: dX[m, k] += keep(m, k) / (1 - p) *
+// sum_q V[m, q] A_a(m)[q, k].  grid = (rows, column blocks of 128 x 8); one thread per 8 columns.
+struct ExpandMaskArgs {
+  const float* V;                 // [rows, R] fp32 (already scaled by s)
+  int32_t R;
+  const __nv_bfloat16* A_all;     // [n_adapters, R, D]
+  const int32_t* row_adapter;     // [rows] over the compact fine-tuning rows
+  __nv_bfloat16* dX;              // [rows, D], row stride lddx
+  int64_t lddx;
+  int32_t D, n_rows;
+  DropArgs drop;
+};
+
+__global__ void __launch_bounds__(128)
+expand_mask_kernel(const ExpandMaskArgs a) {
+  __shared__ float v[kMaxRank];
+  const int m = blockIdx.x;
+  const int k = (blockIdx.y * 128 + threadIdx.x) * 8;
+  const int ad = a.row_adapter[m];
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();
+  if (ad < 0) return;
+  for (int q = threadIdx.x; q < a.R; q += 128) v[q] = a.V[(size_t)m * a.R + q];
+  __syncthreads();
+  if (k >= a.D) return;
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  const __nv_bfloat16* Ab = a.A_all + (size_t)ad * a.R * a.D + k;
+  for (int q = 0; q < a.R; ++q) {
+    const uint4 w = ptx::ldg_nc_v4(Ab + (size_t)q * a.D);
+    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      acc[2 * i] = fmaf(v[q], __uint_as_float(ww[i] << 16), acc[2 * i]);
+      acc[2 * i + 1] = fmaf(v[q], __uint_as_float(ww[i] & 0xFFFF0000u), acc[2 * i + 1]);
+    }
+  }
+  const uint64_t z0 = drop_bits(a.drop.seed, (uint32_t)m, (uint32_t)(k >> 2));
+  const uint64_t z1 = drop_bits(a.drop.seed, (uint32_t)m, (uint32_t)(k >> 2) + 1);
+  __nv_bfloat16* dst = a.dX + (size_t)m * a.lddx + k;
+  uint4 o = *reinterpret_cast<const uint4*>(dst);
+  uint32_t ow[4] = {o.x, o.y, o.z, o.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint64_t z = i < 2 ? z0 : z1;
+    const int f = (2 * i) & 3;
+    const bool k0 = (uint32_t)((z >> (16 * f)) & 0xFFFFu) >= a.drop.thr;
+    const bool k1 = (uint32_t)((z >> (16 * (f + 1))) & 0xFFFFu) >= a.drop.thr;
+    const float lo = __uint_as_float(ow[i] << 16) + (k0 ? acc[2 * i] * a.drop.keep_scale : 0.f);
+    const float hi = __uint_as_float(ow[i] & 0xFFFF0000u) + (k1 ? acc[2 * i + 1] * a.drop.keep_scale : 0.f);
+    ow[i] = ptx::pack_bf16(lo, hi);
+  }
+  *reinterpret_cast<uint4*>(dst) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
 }
 
 }  // namespace mlora

@@ -1,0 +1,163 @@
+"""GPU parity of the variants with the oracle: LoRA dropout on the fine-tuning rows (mask checked
+bit for bit with an exact probe, values within the layer's tolerance) and adapters of different
+ranks stored with zero padding."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mlora_oracle as orc
+from paper_2607_28848_b200 import binding as mb
+from paper_2607_28848_b200 import synth
+from paper_2607_28848_b200.runner import LayerRun, Session
+from test_gpu_parity import TOL, assert_close
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sess():
+    s = Session(0)
+    yield s
+    mb.mlora_set_dropout(s.ctx, 0.0, 0)
+    s.close()
+
+
+def check_dropout(sess, w, t, p, seed, path=0, blocked=False, base=0, cap=None):
+    tol = TOL[w.dtype]
+    mb.mlora_set_gemm_path(sess.ctx, path)
+    mb.mlora_set_dropout(sess.ctx, p, seed)
+    run = LayerRun(sess, w.dtype, t, w.segments, w.n_rows, save_row_base=base, save_capacity_rows=cap, guard=True)
+    try:
+        run.forward()
+        assert run.status() == mb.MLORA_OK
+        drop = (p, seed) if p > 0 else None
+        fwd = (orc.forward_blocked if blocked else orc.forward)(t["X"], t["W"], t["A_all"], t["B_all"], t["scale"],
+                                                                 w.segments, dropout=drop)
+        assert_close("Y", run.host(run.Y), fwd["Y"], tol)
+        n = run.ft_rows
+        assert n == fwd["ft_rows"] and n > 0
+        assert np.array_equal(run.host(run.x_save)[base:base + n], fwd["x_save"][:n]), "x_save keeps the undropped rows"
+        assert_close("u_save", run.host(run.u_save)[base:base + n], fwd["u_save"][:n], min(tol, 1e-3))
+        run.backward()
+        assert run.status() == mb.MLORA_OK
+        bwd = (orc.backward_blocked if blocked else orc.backward)(
+            t["dY"], t["W"], t["A_all"], t["B_all"], t["scale"], w.segments, fwd["x_save"], fwd["u_save"],
+            n_rows=w.n_rows, dropout=drop)
+        assert_close("dX", run.host(run.dX)[:n], bwd["dX"], tol)
+        assert_close("dA", run.host(run.dA), bwd["dA"], tol)
+        assert_close("dB", run.host(run.dB), bwd["dB"], tol)
+    finally:
+        mb.mlora_set_dropout(sess.ctx, 0.0, 0)
+        mb.mlora_set_gemm_path(sess.ctx, 0)
+        run.close()
+
+
+@pytest.mark.parametrize("rank", [8, 16, 32])
+def test_dropout_streaming_kernels(sess, rank):
+    # ragged table: gathered single rows, partial items, fine-tuning segments of every length
+    w = synth.random_workload(40 + rank, 512, 384, rank, 5, 700, max_seg=150, p_finetune=0.45)
+    check_dropout(sess, w, synth.make_tensors(w), 0.3, 2 ** 40 + rank)
+
+
+def test_dropout_paper_rate_full_items_and_append(sess):
+    # full 32-row items (block-saved through the tensor-map store) with the paper's p = 0.05,
+    # saved behind rows of an earlier step
+    segs = synth.segments_array([(0, 96, 1, 0), (96, 256, 0, 1), (352, 40, 2, 0), (392, 128, 3, 1)])
+    w = synth.Workload("dropout_full_items", 1024, 512, 16, 4, "bf16", 520, segs, seed=5)
+    check_dropout(sess, w, synth.make_tensors(w), 0.05, 123456789, base=64, cap=64 + 384 + 16)
+
+
+def test_dropout_cuda_core_path_and_fp32(sess):
+    w = synth.random_workload(77, 256, 192, 16, 4, 300, max_seg=90, p_finetune=0.5)
+    check_dropout(sess, w, synth.make_tensors(w), 0.25, 99, path=1)
+    w32 = synth.cfg1_tiny()
+    check_dropout(sess, w32, synth.make_tensors(w32), 0.5, 7)
+
+
+def test_dropout_off_is_the_plain_layer(sess):
+    w = synth.random_workload(78, 256, 256, 16, 4, 200, p_finetune=0.5)
+    check_dropout(sess, w, synth.make_tensors(w), 0.0, 1234)
+
+
+def test_dropout_mask_bit_exact(sess):
+    """Exact probe: with A[q, k] = [k mod r == q], X = 1, W = 0, B[q, j] = [j == q], dY[m, j] = [j < r], s = 1
+    the forward's U[m, q] is (number of kept columns of class q) / (1 - p) and the input gradient is
+    keep[m, k] / (1 - p): every element of the mask shows up exactly."""
+    d_in, d_out, r, n_ad = 512, 256, 16, 2
+    segs = synth.segments_array([(0, 70, 0, 1), (70, 10, 1, 0), (80, 37, 1, 1)])
+    T, n_ft = 117, 107
+    p, seed = 0.4, 0xDEADBEEFCAFE
+    k = np.arange(d_in)
+    A = (k[None, :] % r == np.arange(r)[:, None]).astype(np.float32)
+    B = (np.arange(d_out)[None, :] == np.arange(r)[:, None]).astype(np.float32)
+    t = {"X": np.ones((T, d_in), np.float32), "W": np.zeros((d_in, d_out), np.float32),
+         "A_all": np.stack([A] * n_ad), "B_all": np.stack([B] * n_ad), "scale": np.ones(n_ad, np.float32),
+         "dY": np.concatenate([np.ones((n_ft, r), np.float32), np.zeros((n_ft, d_out - r), np.float32)], axis=1)}
+    keep = orc.dropout_keep_vectorised(seed, n_ft, d_in, p)
+    ks = np.float32(1.0 / (1.0 - p))
+    mb.mlora_set_dropout(sess.ctx, p, seed)
+    run = LayerRun(sess, "bf16", t, segs, T)
+    try:
+        run.forward()
+        run.backward()
+        assert run.status() == mb.MLORA_OK
+        counts = np.stack([keep[:, q::r].sum(axis=1) for q in range(r)], axis=1).astype(np.float32)
+        got_u = run.u_save[:n_ft].cpu().numpy()
+        assert np.array_equal(got_u, counts * ks)
+        got_dx = run.dX[:n_ft].float().cpu().numpy()
+        ks_bf16 = torch.tensor(float(ks)).to(torch.bfloat16).float().item()
+        assert np.array_equal(got_dx, np.where(keep, np.float32(ks_bf16), np.float32(0.0)))
+        # inference rows (70..79) see no dropout: Y = U B with U = d_in / r per class
+        y = run.Y[70:80].float().cpu().numpy()
+        assert np.array_equal(y[:, :r], np.full((10, r), d_in / r, np.float32)) and not y[:, r:].any()
+    finally:
+        mb.mlora_set_dropout(sess.ctx, 0.0, 0)
+        run.close()
+
+
+def test_dropout_large_rank_is_refused(sess):
+    w = synth.random_workload(79, 256, 256, 64, 3, 200, p_finetune=0.5)
+    t = synth.make_tensors(w)
+    mb.mlora_set_dropout(sess.ctx, 0.1, 1)
+    run = LayerRun(sess, w.dtype, t, w.segments, w.n_rows)
+    try:
+        with pytest.raises(mb.MloraError) as e:
+            run.forward()
+        assert e.value.status == mb.MLORA_ERR_UNSUPPORTED
+        with pytest.raises(mb.MloraError):
+            mb.mlora_set_dropout(sess.ctx, 1.0, 1)
+    finally:
+        mb.mlora_set_dropout(sess.ctx, 0.0, 0)
+        run.close()
+
+
+def test_dropout_llama_projection_sampled(sess):
+    """4096 -> 4096, 1600 rows (1024 prefill + 64 decode + 2 x 256 fine-tune), p = 0.05: full check with
+    the blocked oracle."""
+    w = synth.cfg2_single_projection()
+    check_dropout(sess, w, synth.make_tensors(w), 0.05, 2024, blocked=True)
+
+
+def test_different_ranks_through_zero_padding(sess):
+    rng_ranks = [4, 16, 8, 12, 16, 1]
+    w = synth.random_workload(81, 512, 320, 16, len(rng_ranks), 600, max_seg=120, p_finetune=0.4)
+    t = synth.make_tensors(w)
+    A_list, B_list = [], []
+    for a, ra in enumerate(rng_ranks):
+        t["A_all"][a, ra:] = 0.0
+        t["B_all"][a, ra:] = 0.0
+        A_list.append(t["A_all"][a, :ra].copy())
+        B_list.append(t["B_all"][a, :ra].copy())
+        t["scale"][a] = 32.0 / ra                          # alpha / r_a
+    run = LayerRun(sess, w.dtype, t, w.segments, w.n_rows)
+    try:
+        run.forward()
+        run.backward()
+        assert run.status() == mb.MLORA_OK
+        ref = orc.forward_ragged(t["X"], t["W"], A_list, B_list, t["scale"], w.segments)
+        assert_close("Y", run.host(run.Y), ref, TOL["bf16"])
+        dA, dB = run.host(run.dA), run.host(run.dB)
+        for g, a in enumerate(run.slots):                  # gradients of the padding rows are exactly zero
+            assert not dA[g, rng_ranks[a]:].any() and not dB[g, rng_ranks[a]:].any()
+    finally:
+        run.close()
