@@ -146,6 +146,21 @@ def test_gathered_and_contiguous_items(sess):
     run_and_check(sess, w, synth.make_tensors(w))
 
 
+def test_block_save_only_when_save_offsets_run_with_the_rows(sess):
+    """Full 32-row items of fine-tuning rows are saved as one block only when their save offsets are
+    consecutive.  Here adjacent fine-tuning segments of ONE adapter sit in the table out of row order,
+    so 32 adjacent rows map to permuted / interleaved save offsets; next to them a segment whose
+    items can be block-saved, a mixed inference + fine-tune item, and a partial item."""
+    segs = [(0, 8, 0, 1), (16, 8, 0, 1), (8, 8, 0, 1), (24, 8, 0, 1),        # rows 0..31 adjacent, saves 0-7,16-23,8-15,24-31
+            (64, 32, 1, 1), (32, 32, 1, 1),                                   # two full items, second saved first
+            (96, 96, 2, 1),                                                   # three block-saved items
+            (192, 10, 3, 0), (202, 54, 3, 1),                                 # item mixing inference and fine-tune rows
+            (256, 45, 0, 1)]                                                  # full item + partial item, adapter 0 again
+    for path in (0, 2):
+        w = synth.Workload("block_save_order", 768, 256, 16, 4, "bf16", 301, synth.segments_array(segs), seed=path)
+        run_and_check(sess, w, synth.make_tensors(w), path=path, base=5, cap=5 + 291 + 9)
+
+
 def test_base_only_rows_and_no_finetune(sess):
     segs = [(0, 40, -1, 0), (60, 30, 1, 0)]      # rows 40..59 and 90..99 uncovered
     w = synth.Workload("base_only", 192, 256, 16, 2, "bf16", 100, synth.segments_array(segs))
