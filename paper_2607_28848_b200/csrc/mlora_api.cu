@@ -208,8 +208,8 @@ int shrink_ksplit(const mlora_ctx* ctx, int n_items, int D) {
   k = k < kMaxKSplit ? k : kMaxKSplit;
   return k < 1 ? 1 : k;
 }
-template <int RB, int STAGES, int CHUNK>
-mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, const int32_t* item_desc, int n_rows,
+template <int RB, int STAGES, int CHUNK, bool DROP>
+mlora_status_t launch_shrink_stream_d(mlora_ctx* ctx, ShrinkArgs a, int n_items, const int32_t* item_desc, int n_rows,
                                     int n_adapters, cudaStream_t st) {
   constexpr int R = RB * 8;
   constexpr size_t xrow = 32 * (CHUNK * 128 + 16), xtile = (size_t)(CHUNK / 4) * 32 * 512;
@@ -228,7 +228,7 @@ mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, c
     tSave = tIn;
   }
   static bool attr_set = false;
-  auto kern = shrink_stream_kernel<RB, STAGES, CHUNK>;
+  auto kern = shrink_stream_kernel<RB, STAGES, CHUNK, DROP>;
   if (!attr_set) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return MLORA_ERR_CUDA;
     attr_set = true;
@@ -252,6 +252,15 @@ mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, c
   sa.item_desc = item_desc;
   launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(STREAM_THREADS), smem, st, tIn, tP, tSave, sa);
   return scope.done();
+}
+
+// The dropout variant is its own instantiation, so that the usual one carries none of the mask arithmetic.
+template <int RB, int STAGES, int CHUNK>
+mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, const int32_t* item_desc, int n_rows,
+                                    int n_adapters, cudaStream_t st) {
+  if (a.item_save && ctx->drop.thr != 0)
+    return launch_shrink_stream_d<RB, STAGES, CHUNK, true>(ctx, a, n_items, item_desc, n_rows, n_adapters, st);
+  return launch_shrink_stream_d<RB, STAGES, CHUNK, false>(ctx, a, n_items, item_desc, n_rows, n_adapters, st);
 }
 
 mlora_status_t launch_shrink(mlora_ctx* ctx, int R, ShrinkArgs a, int n_items, const int32_t* item_desc, int n_rows,
@@ -280,23 +289,24 @@ mlora_status_t launch_shrink(mlora_ctx* ctx, int R, ShrinkArgs a, int n_items, c
 }
 
 // Both gradients of a backward in one launch of the streaming kernel (dB first, then dA).
-template <int MB>
-mlora_status_t launch_grad_stream2(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& gb, const GradArgs& ga_, int n_slots,
+template <int MB, bool DROP>
+mlora_status_t launch_grad_stream2_d(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& gb, const GradArgs& ga_, int n_slots,
                                    int n_rows, cudaStream_t st) {
-  constexpr size_t smem = (size_t)gstream_stages(MB) * (128 * 128 + 128 * MB * 16 * 4) + (size_t)STREAM_WARPS * MB * 16 * 65 * 4 + 1024;
+  constexpr size_t smem = (size_t)GW_STAGES * (GW_Q_BYTES + GW_ROWS * MB * 16 * 4) + 1024;
   static bool attr_set = false;
-  auto kern = grad_stream_kernel<MB>;
+  auto kern = grad_stream_kernel<MB, DROP>;
   if (!attr_set) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return MLORA_ERR_CUDA;
     attr_set = true;
   }
   CUtensorMap tQ0, tQ1;
   mlora_status_t ms;
-  if ((ms = make_tmap_bf16(ctx, &tQ0, gb.Q, gb.D, n_rows, gb.ldq, 64, 128)) != MLORA_OK) return ms;
-  if ((ms = make_tmap_bf16(ctx, &tQ1, ga_.Q, ga_.D, n_rows, ga_.ldq, 64, 128)) != MLORA_OK) return ms;
+  // (64, rows, D / 64) views: one box = a 64-row tile of a 512-column strip as eight swizzled 64-column blocks
+  if ((ms = make_tmap_bf16_blocked(ctx, &tQ0, gb.Q, n_rows, gb.D, gb.ldq, GW_ROWS, GW_COLS / 64)) != MLORA_OK) return ms;
+  if ((ms = make_tmap_bf16_blocked(ctx, &tQ1, ga_.Q, n_rows, ga_.D, ga_.ldq, GW_ROWS, GW_COLS / 64)) != MLORA_OK) return ms;
   GradStreamArgs g;
-  g.prob[0] = GradProblem{gb.P, gb.scale, gb.G, gb.D, gb.D / 64, DropArgs{0, 0, 1.0f}};
-  g.prob[1] = GradProblem{ga_.P, ga_.scale, ga_.G, ga_.D, ga_.D / 64, ctx->drop};   // dA sees the dropped branch input
+  g.prob[0] = GradProblem{gb.P, gb.scale, gb.G, gb.D, (gb.D + GW_COLS - 1) / GW_COLS, DropArgs{0, 0, 1.0f}};
+  g.prob[1] = GradProblem{ga_.P, ga_.scale, ga_.G, ga_.D, (ga_.D + GW_COLS - 1) / GW_COLS, ctx->drop};   // dA sees the dropped branch input
   g.n_problems = 2; g.R = gb.R; g.accumulate = gb.accumulate;
   g.slot_adapter = p->slot_adapter; g.slot_blk_off = p->slot_blk_off; g.blk_row0 = p->blk_row0; g.blk_nrows = p->blk_nrows;
   g.n_slots = n_slots; g.status = ctx->status_dev;
@@ -306,6 +316,13 @@ mlora_status_t launch_grad_stream2(mlora_ctx* ctx, const mlora_plan* p, const Gr
   LaunchScope scope(ctx, st, KIND_GRAD);
   launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(STREAM_THREADS), smem, st, tQ0, tQ1, g);
   return scope.done();
+}
+
+template <int MB>
+mlora_status_t launch_grad_stream2(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& gb, const GradArgs& ga_, int n_slots,
+                                   int n_rows, cudaStream_t st) {
+  return ctx->drop.thr != 0 ? launch_grad_stream2_d<MB, true>(ctx, p, gb, ga_, n_slots, n_rows, st)
+                            : launch_grad_stream2_d<MB, false>(ctx, p, gb, ga_, n_slots, n_rows, st);
 }
 
 mlora_status_t launch_grad(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& a, int n_slots, int n_rows,
@@ -846,7 +863,8 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (L->dtype == MLORA_F32)
     return backward_simt<float>(ctx, L, p, dY, lddy, x_save, u_save, dA, dB, dX, lddx, accumulate, st);
-  if (lddy % 8 || (dX && lddx % 8) || !aligned16(dY) || !aligned16(x_save) || (dX && !aligned16(dX)))
+  if (lddy % 8 || (dX && lddx % 8) || !aligned16(dY) || !aligned16(x_save) || (dX && !aligned16(dX)) ||
+      !aligned16(dA) || !aligned16(dB) || !aligned16(u_save))
     return MLORA_ERR_UNSUPPORTED;
   if (ctx->gemm_path == 1)
     return backward_simt<__nv_bfloat16>(ctx, L, p, dY, lddy, x_save, u_save, dA, dB, dX, lddx, accumulate, st);

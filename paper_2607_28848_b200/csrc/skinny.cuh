@@ -298,7 +298,7 @@ __device__ __forceinline__ bool stream_wait(uint32_t bar, uint32_t parity, volat
   return false;
 }
 
-template <int RB, int STAGES, int CHUNK>
+template <int RB, int STAGES, int CHUNK, bool DROP>
 __global__ void __launch_bounds__(STREAM_THREADS, 1)
 shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant__ CUtensorMap tmP,
                      const __grid_constant__ CUtensorMap tmSave, const StreamArgs sa) {
@@ -543,7 +543,7 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
 #pragma unroll
         for (int j = 0; j < 4; ++j)
           if (g + 8 * j >= cur_nrows) { x[j][0] = make_uint4(0, 0, 0, 0); x[j][1] = make_uint4(0, 0, 0, 0); }
-        if (sa.drop.thr != 0) {     // dropout: the saved copy above keeps the row as it is, the product does not
+        if (DROP) {     // dropout: the saved copy above keeps the row as it is, the product does not
 #pragma unroll
           for (int j = 0; j < 4; ++j)
             if (msave[j] >= 0) {
@@ -634,7 +634,7 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
 #pragma unroll
             for (int w = 0; w < RW; ++w) v += red[w][r][q];
           }
-          if (sa.drop.thr != 0 && my_save[k] >= 0) v *= sa.drop.keep_scale;
+          if (DROP && my_save[k] >= 0) v *= sa.drop.keep_scale;
           const float vs = v * my_scale;
           a.Out[(size_t)my_row[k] * R + q] = vs;
           fin[r][q] = vs;
@@ -788,13 +788,20 @@ grad_kernel(const GradArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Streaming gradient kernel for ranks up to 32.  A persistent CTA takes whole (slot, 64-column
-// strip) groups in turn; for each it streams the slot's rows as tiles of 128 rows x 64 columns
-// (one tensor-map load into 128B-swizzled shared memory) together with the matching 128 x R block
-// of P (one bulk copy) through a ring of stages, so that the bytes in flight do not depend on
-// registers.  Consumer warp w contracts rows 16w .. 16w+15 of every tile (one MMA K-step, rows as
-// the contraction index); the eight warps are added in a fixed order when the strip is done.
-__host__ __device__ constexpr int gstream_stages(int mb) { return mb == 1 ? 6 : 4; }
+// Streaming gradient kernel for ranks up to 32.  A persistent CTA takes whole (slot, 512-column
+// strip) groups in turn; for each it streams the slot's rows as tiles of 64 rows x 512 columns
+// (ONE tensor-map load: eight 64-column blocks of [64 rows][128 B], 128B-swizzled, i.e. 1 KiB
+// contiguous per row in memory) together with the matching 64 x R block of P (one bulk copy)
+// through a ring of three stages.  Consumer warp w owns column block w of the strip for the whole
+// group: it contracts all rows of every tile (four MMA K-steps, rows as the contraction index)
+// into its own 16 (or 32) x 64 accumulator, so no reduction across warps is needed and the result
+// goes from registers to memory; rows are visited in one fixed order, so the sums are
+// run-to-run bit-reproducible.  The consumers read no table: the producer leaves each tile's row
+// count in shared memory beside the tile.
+constexpr int GW_COLS = 512;          // columns per strip (8 warps x 64)
+constexpr int GW_ROWS = 64;           // rows per staged tile
+constexpr int GW_STAGES = 3;
+constexpr uint32_t GW_Q_BYTES = 8 * GW_ROWS * 128;
 
 // One launch computes both gradients of a backward: problem 0 (dB: P = u_save scaled, Q = dY,
 // D = d_out) and problem 1 (dA: P = V, Q = x_save, D = d_in); groups of problem 0 come first.
@@ -802,7 +809,7 @@ struct GradProblem {
   const float* P;              // [rows, R] fp32
   const float* scale;          // nullable
   float* G;                    // [n_slots, R, D]
-  int32_t D, n_strips;         // D / 64
+  int32_t D, n_strips;         // ceil(D / GW_COLS)
   DropArgs drop;               // dA with dropout: Q elements kept or dropped, P counts keep_scale (thr == 0: off)
 };
 struct GradStreamArgs {
@@ -811,23 +818,23 @@ struct GradStreamArgs {
   int32_t R, accumulate;
   const int32_t* slot_adapter;
   const int32_t* slot_blk_off;
-  const int32_t* blk_row0;
+  const int32_t* blk_row0;     // blocks of <= 128 rows of one slot (compact fine-tuning rows)
   const int32_t* blk_nrows;
   int32_t n_slots;
   int32_t* status;
 };
 
-template <int MB>
+template <int MB, bool DROP>
 __global__ void __launch_bounds__(STREAM_THREADS, 1)
 grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_constant__ CUtensorMap tmQ1,
                    const GradStreamArgs ga) {
-  constexpr int S = gstream_stages(MB);
+  constexpr int S = GW_STAGES;
   constexpr int RMAX = MB * 16;
-  constexpr uint32_t Q_BYTES = 128 * 128;                 // 128 rows x 64 bf16, swizzled
-  constexpr uint32_t P_BYTES = 128 * RMAX * 4;
-  constexpr uint32_t STAGE_BYTES = Q_BYTES + P_BYTES;
+  constexpr uint32_t P_BYTES = GW_ROWS * RMAX * 4;
+  constexpr uint32_t STAGE_BYTES = GW_Q_BYTES + P_BYTES;
   extern __shared__ __align__(1024) uint8_t gs_smem[];
   __shared__ __align__(8) uint64_t bars[2 * S];
+  __shared__ int stage_meta[S][2];     // {first compact row, rows | last-tile-of-group flag << 16} of the staged tile
   __shared__ int abort_word;
   volatile int* abort_flag = &abort_word;
   const int R = ga.R;
@@ -840,8 +847,6 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
   if (tl_on) { for (int i = 0; i < 16; ++i) MLORA_TL_SET(i, 0); MLORA_TL_SET(14, tl_global()); }
 #endif
   const uint32_t ring = (ptx::smem_u32(gs_smem) + 1023u) & ~1023u;      // swizzled tiles need 1 KiB alignment
-  float (*red)[MB * 16][64 + 1] = reinterpret_cast<float (*)[MB * 16][64 + 1]>(
-      gs_smem + (ring - ptx::smem_u32(gs_smem)) + S * STAGE_BYTES);
   const uint32_t bar0 = ptx::smem_u32(bars);
   auto bar_full = [&](int st) { return bar0 + 8u * st; };
   auto bar_empty = [&](int st) { return bar0 + 8u * (S + st); };
@@ -858,6 +863,15 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
 
   if (warp == STREAM_WARPS) {
     // ======================= producer =======================
+    // the plan's tables are not written by the kernel before this one: the first group's entries
+    // are fetched while that kernel may still be running
+    int first_b_begin = 0, first_b_end = 0, first_row0 = 0, first_nrows = 0;
+    if (lane == 0 && (int)blockIdx.x < n_groups) {
+      const int pi = (int)blockIdx.x >= groups0 ? 1 : 0;
+      const int slot = ((int)blockIdx.x - pi * groups0) / ga.prob[pi].n_strips;
+      first_b_begin = ga.slot_blk_off[slot]; first_b_end = ga.slot_blk_off[slot + 1];
+      if (first_b_begin < first_b_end) { first_row0 = ga.blk_row0[first_b_begin]; first_nrows = ga.blk_nrows[first_b_begin]; }
+    }
     ptx::grid_dependency_wait();
     ptx::grid_launch_dependents();
     if (lane == 0) {
@@ -869,15 +883,37 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
         const CUtensorMap* tmQ = pi ? &tmQ1 : &tmQ0;
         const int gl = grp - pi * groups0;
         const int slot = gl / pr.n_strips, strip = gl % pr.n_strips;
-        for (int b = ga.slot_blk_off[slot]; b < ga.slot_blk_off[slot + 1]; ++b, ++i) {
+        const bool first = grp == (int)blockIdx.x;
+        const int b_begin = first ? first_b_begin : ga.slot_blk_off[slot];
+        const int b_end = first ? first_b_end : ga.slot_blk_off[slot + 1];
+        if (b_begin == b_end) {            // a slot without rows: an empty last tile, so that its gradient is still written
           const int st = i % S;
           if (!(ok = stream_wait(bar_empty(st), ((i / S) & 1) ^ 1, abort_flag, ga.status))) break;
-          const int row0 = ga.blk_row0[b], nrows = ga.blk_nrows[b];
-          const uint32_t dst = ring + (uint32_t)st * STAGE_BYTES;
-          const uint32_t pbytes = (uint32_t)nrows * (uint32_t)R * 4u;
-          ptx::mbar_arrive_expect_tx(bar_full(st), Q_BYTES + pbytes);
-          ptx::tma_load_2d(dst, tmQ, strip * 64, row0, bar_full(st));        // rows past the block are masked below
-          bulk_load(dst + Q_BYTES, pr.P + (size_t)row0 * R, pbytes, bar_full(st));
+          stage_meta[st][0] = 0;
+          stage_meta[st][1] = 1 << 16;
+          ptx::mbar_arrive(bar_full(st));
+          ++i;
+          continue;
+        }
+        int row0 = first ? first_row0 : ga.blk_row0[b_begin], nrows = first ? first_nrows : ga.blk_nrows[b_begin];
+        for (int b = b_begin; b < b_end && ok; ++b) {
+          // the next block's table entries are requested before this block's tiles are waited for
+          const int nb1 = b + 1 < b_end ? b + 1 : b;
+          const int next_row0 = ga.blk_row0[nb1], next_nrows = ga.blk_nrows[nb1];
+          for (int off = 0; off < nrows; off += GW_ROWS, ++i) {
+            const int st = i % S;
+            if (!(ok = stream_wait(bar_empty(st), ((i / S) & 1) ^ 1, abort_flag, ga.status))) break;
+            const int nr = min(GW_ROWS, nrows - off);
+            const uint32_t dst = ring + (uint32_t)st * STAGE_BYTES;
+            const uint32_t pbytes = (uint32_t)nr * (uint32_t)R * 4u;
+            stage_meta[st][0] = row0 + off;
+            stage_meta[st][1] = nr | ((b == b_end - 1 && off + GW_ROWS >= nrows) ? (1 << 16) : 0);
+            ptx::mbar_arrive_expect_tx(bar_full(st), GW_Q_BYTES + pbytes);
+            // rows past the tile's count are masked by the consumers; blocks past D arrive as zeros
+            ptx::tma_load_3d(dst, tmQ, 0, row0 + off, strip * (GW_COLS / 64), bar_full(st));
+            bulk_load(dst + GW_Q_BYTES, pr.P + (size_t)(row0 + off) * R, pbytes, bar_full(st));
+          }
+          row0 = next_row0; nrows = next_nrows;
         }
       }
     }
@@ -899,15 +935,15 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
       const GradProblem& pr = ga.prob[pi];
       const int gl = grp - pi * groups0;
       const int slot = gl / pr.n_strips, strip = gl % pr.n_strips;
-      const float sc = (pr.scale ? pr.scale[ga.slot_adapter[slot]] : 1.0f) * (pr.drop.thr != 0 ? pr.drop.keep_scale : 1.0f);
+      const int col0 = strip * GW_COLS + warp * 64;        // this warp's 64 columns
+      const bool active = col0 < pr.D;
+      const float sc = (pr.scale ? pr.scale[ga.slot_adapter[slot]] : 1.0f) * ((DROP && pr.drop.thr != 0) ? pr.drop.keep_scale : 1.0f);
 #pragma unroll
       for (int m = 0; m < MB; ++m)
 #pragma unroll
         for (int n = 0; n < 8; ++n) acc[m][n][0] = acc[m][n][1] = acc[m][n][2] = acc[m][n][3] = 0.f;
-      for (int b = ga.slot_blk_off[slot]; b < ga.slot_blk_off[slot + 1]; ++b, ++i) {
+      for (bool last = false; !last; ++i) {
         const int st = i % S;
-        const int nrows = ga.blk_nrows[b];
-        const int brow0 = ga.blk_row0[b];
 #ifdef MLORA_TIMELINE
         const long long tw0 = tl_clock();
 #endif
@@ -915,54 +951,64 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
 #ifdef MLORA_TIMELINE
         if (tl_on) { tl_wait += tl_clock() - tw0; if (i == 0) MLORA_TL_SET(4, tl_clock() - tl0); ++tl_nstage; }
 #endif
-        const uint32_t qbase = ring + (uint32_t)st * STAGE_BYTES;
-        const uint32_t pbase = qbase + Q_BYTES;
-        if (warp * 16 < nrows) {
-          // rows of this warp's K-step: r = 16 warp + {2c, 2c+1, 2c+8, 2c+9}
-          uint4 q[4];
-          uint32_t ahi[MB][4], alo[MB][4];
-          const int tr[4] = {2 * c, 2 * c + 1, 2 * c + 8, 2 * c + 9};
+        const int trow0 = stage_meta[st][0];
+        const int meta = stage_meta[st][1];
+        const int nrows = meta & 0xFFFF;
+        last = (meta >> 16) != 0;
+        // plain shared-memory loads (no branches around them): what lies past a tile's rows is read
+        // and then replaced by zero
+        const uint8_t* stage_ptr = gs_smem + (ring - ptx::smem_u32(gs_smem)) + (size_t)st * STAGE_BYTES;
+        const uint8_t* qtile = stage_ptr + (size_t)warp * (GW_ROWS * 128u);
+        const float* ptile = reinterpret_cast<const float*>(stage_ptr + GW_Q_BYTES);
+        if (active) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const int r = warp * 16 + tr[k];
-            // 16-byte piece g of row r sits at piece (g ^ (r & 7)) of the swizzled 128-byte row
-            q[k] = lds_v4(qbase + (uint32_t)r * 128u + (uint32_t)((g ^ (r & 7)) << 4));
-            if (r >= nrows) q[k] = make_uint4(0, 0, 0, 0);      // rows of the tile past the block's end
-            else if (pr.drop.thr != 0) drop_mask8(pr.drop, (uint32_t)(brow0 + r), (uint32_t)(strip * 64 + 8 * g), q[k]);
-          }
+          for (int ks = 0; ks < GW_ROWS / 16; ++ks) {
+            if (ks * 16 >= nrows) break;
+            // rows of this K-step: r = 16 ks + {2c, 2c+1, 2c+8, 2c+9}
+            uint4 q[4];
+            uint32_t ahi[MB][4], alo[MB][4];
+            const int tr[4] = {2 * c, 2 * c + 1, 2 * c + 8, 2 * c + 9};
 #pragma unroll
-          for (int m = 0; m < MB; ++m) {
-            float pv[4][2];
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-#pragma unroll
-              for (int h = 0; h < 2; ++h) {
-                const int r = warp * 16 + tr[k], qq = m * 16 + g + 8 * h;
-                float v = 0.f;
-                if (r < nrows && qq < R)
-                  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(pbase + (uint32_t)(r * R + qq) * 4u));
-                pv[k][h] = v * sc;
-              }
-#pragma unroll
-            for (int f = 0; f < 4; ++f) {       // a0 (q=g, rows 2c,2c+1), a1 (q=g+8, same rows), a2, a3: rows 2c+8,2c+9
-              const int h = f & 1, rp = (f >> 1) * 2;
-              const float e0 = pv[rp][h], e1 = pv[rp + 1][h];
-              const __nv_bfloat16 h0 = __float2bfloat16_rn(e0), h1 = __float2bfloat16_rn(e1);
-              ahi[m][f] = ptx::pack_bf16(e0, e1);
-              alo[m][f] = ptx::pack_bf16(e0 - __bfloat162float(h0), e1 - __bfloat162float(h1));
+            for (int k = 0; k < 4; ++k) {
+              const int r = ks * 16 + tr[k];
+              // 16-byte piece g of row r sits at piece (g ^ (r & 7)) of the swizzled 128-byte row
+              const uint4 t = *reinterpret_cast<const uint4*>(qtile + r * 128 + ((g ^ (r & 7)) << 4));
+              const bool in = r < nrows;                           // rows of the tile past the block's end count zero
+              q[k] = make_uint4(in ? t.x : 0u, in ? t.y : 0u, in ? t.z : 0u, in ? t.w : 0u);
+              if (DROP && in && pr.drop.thr != 0) drop_mask8(pr.drop, (uint32_t)(trow0 + r), (uint32_t)(col0 + 8 * g), q[k]);
             }
-          }
-          const uint32_t qr[4][4] = {{q[0].x, q[0].y, q[0].z, q[0].w}, {q[1].x, q[1].y, q[1].z, q[1].w},
-                                     {q[2].x, q[2].y, q[2].z, q[2].w}, {q[3].x, q[3].y, q[3].z, q[3].w}};
-#pragma unroll
-          for (int nb = 0; nb < 8; ++nb) {
-            const uint32_t sel = (nb & 1) ? 0x7632u : 0x5410u;
-            const uint32_t b0 = __byte_perm(qr[0][nb >> 1], qr[1][nb >> 1], sel);
-            const uint32_t b1 = __byte_perm(qr[2][nb >> 1], qr[3][nb >> 1], sel);
 #pragma unroll
             for (int m = 0; m < MB; ++m) {
-              ptx::mma_bf16_16816(acc[m][nb], ahi[m][0], ahi[m][1], ahi[m][2], ahi[m][3], b0, b1);
-              ptx::mma_bf16_16816(acc[m][nb], alo[m][0], alo[m][1], alo[m][2], alo[m][3], b0, b1);
+              float pv[4][2];
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                  const int r = ks * 16 + tr[k], qq = m * 16 + g + 8 * h;
+                  const float v = ptile[r * R + qq];               // inside the stage's P area for every r < 64, qq < 16 MB
+                  pv[k][h] = (r < nrows && qq < R) ? v * sc : 0.f;
+                }
+#pragma unroll
+              for (int f = 0; f < 4; ++f) {       // a0 (q=g, rows 2c,2c+1), a1 (q=g+8, same rows), a2, a3: rows 2c+8,2c+9
+                const int h = f & 1, rp = (f >> 1) * 2;
+                const float e0 = pv[rp][h], e1 = pv[rp + 1][h];
+                const __nv_bfloat16 h0 = __float2bfloat16_rn(e0), h1 = __float2bfloat16_rn(e1);
+                ahi[m][f] = ptx::pack_bf16(e0, e1);
+                alo[m][f] = ptx::pack_bf16(e0 - __bfloat162float(h0), e1 - __bfloat162float(h1));
+              }
+            }
+            const uint32_t qr[4][4] = {{q[0].x, q[0].y, q[0].z, q[0].w}, {q[1].x, q[1].y, q[1].z, q[1].w},
+                                       {q[2].x, q[2].y, q[2].z, q[2].w}, {q[3].x, q[3].y, q[3].z, q[3].w}};
+#pragma unroll
+            for (int nb = 0; nb < 8; ++nb) {
+              const uint32_t sel = (nb & 1) ? 0x7632u : 0x5410u;
+              const uint32_t b0 = __byte_perm(qr[0][nb >> 1], qr[1][nb >> 1], sel);
+              const uint32_t b1 = __byte_perm(qr[2][nb >> 1], qr[3][nb >> 1], sel);
+#pragma unroll
+              for (int m = 0; m < MB; ++m) {
+                ptx::mma_bf16_16816(acc[m][nb], ahi[m][0], ahi[m][1], ahi[m][2], ahi[m][3], b0, b1);
+                ptx::mma_bf16_16816(acc[m][nb], alo[m][0], alo[m][1], alo[m][2], alo[m][3], b0, b1);
+              }
             }
           }
         }
@@ -974,31 +1020,29 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
       const long long tf0 = tl_clock();
       if (tl_on && grp + (int)gridDim.x >= n_groups) MLORA_TL_SET(5, tf0 - tl0);
 #endif
-      // ---- strip done: fixed-order sum over the warps, then write (or add to) the gradient ----
-      {
-        float (*mine)[64 + 1] = red[warp];
+      // ---- group done: this warp's 16 (32) x 64 block goes from registers to the gradient ----
+      // The n index g of the MMA was mapped to piece g of a row, so for thread (g, c) accumulator
+      // element e of column block nb is strip column 8 (2c + (e & 1)) + nb: over nb = 0..7 that is
+      // eight consecutive columns, written as two 16-byte stores (rows g and g + 8 for e >> 1).
+      if (active) {
 #pragma unroll
         for (int m = 0; m < MB; ++m)
 #pragma unroll
-          for (int nb = 0; nb < 8; ++nb) {
-            const int ca = 8 * (2 * c) + nb, cb = 8 * (2 * c + 1) + nb;
-            mine[m * 16 + g][ca] = acc[m][nb][0];
-            mine[m * 16 + g][cb] = acc[m][nb][1];
-            mine[m * 16 + g + 8][ca] = acc[m][nb][2];
-            mine[m * 16 + g + 8][cb] = acc[m][nb][3];
+          for (int e = 0; e < 4; ++e) {
+            const int ql = m * 16 + g + ((e >> 1) ? 8 : 0);
+            if (ql >= R) continue;
+            float4* dst = reinterpret_cast<float4*>(pr.G + ((size_t)slot * R + ql) * pr.D + col0 + 8 * (2 * c + (e & 1)));
+            float4 lo = make_float4(acc[m][0][e], acc[m][1][e], acc[m][2][e], acc[m][3][e]);
+            float4 hi = make_float4(acc[m][4][e], acc[m][5][e], acc[m][6][e], acc[m][7][e]);
+            if (ga.accumulate) {
+              const float4 o0 = dst[0], o1 = dst[1];
+              lo.x += o0.x; lo.y += o0.y; lo.z += o0.z; lo.w += o0.w;
+              hi.x += o1.x; hi.y += o1.y; hi.z += o1.z; hi.w += o1.w;
+            }
+            dst[0] = lo;
+            dst[1] = hi;
           }
       }
-      asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");
-      for (int idx = threadIdx.x; idx < MB * 16 * 64; idx += STREAM_WARPS * 32) {
-        const int ql = idx / 64, j = idx % 64;
-        if (ql >= R) continue;
-        float v = 0.f;
-#pragma unroll
-        for (int w = 0; w < STREAM_WARPS; ++w) v += red[w][ql][j];
-        float* dst = pr.G + ((size_t)slot * R + ql) * pr.D + strip * 64 + j;
-        *dst = ga.accumulate ? (*dst + v) : v;
-      }
-      asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");
 #ifdef MLORA_TIMELINE
       if (tl_on) { tl_flush += tl_clock() - tf0; ++tl_nflush; }
 #endif

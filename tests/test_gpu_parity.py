@@ -121,6 +121,16 @@ def test_segment_lengths_around_a_tile(sess, lens):
     run_and_check(sess, w, synth.make_tensors(w))
 
 
+@pytest.mark.parametrize("path", [0, 1, 2])
+def test_finetune_slot_without_rows(sess, path):
+    """A zero-length fine-tuning segment still opens a gradient slot: its dA / dB are written as zeros."""
+    segs = [(0, 40, 0, 1), (40, 0, 2, 1), (40, 70, 1, 1), (110, 20, 2, 0)]
+    w = synth.Workload("empty_slot", 256, 192, 16, 3, "bf16", 130, synth.segments_array(segs))
+    run = run_and_check(sess, w, synth.make_tensors(w), path=path)
+    assert run.slots == [0, 2, 1]
+    assert not run.host(run.dA)[1].any() and not run.host(run.dB)[1].any()
+
+
 @pytest.mark.parametrize("n_rows", [5, 129, 257])
 def test_small_batches(sess, n_rows):
     """Fewer rows than one tile, and batches that leave the second CTA of a pair tile (almost) empty."""
