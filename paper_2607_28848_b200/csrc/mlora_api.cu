@@ -289,24 +289,25 @@ mlora_status_t launch_shrink(mlora_ctx* ctx, int R, ShrinkArgs a, int n_items, c
 }
 
 // Both gradients of a backward in one launch of the streaming kernel (dB first, then dA).
-template <int MB, bool DROP>
+template <int MB, bool DROP, int CB>
 mlora_status_t launch_grad_stream2_d(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& gb, const GradArgs& ga_, int n_slots,
-                                   int n_rows, cudaStream_t st) {
-  constexpr size_t smem = (size_t)GW_STAGES * (GW_Q_BYTES + GW_ROWS * MB * 16 * 4) + 1024;
+                                     int n_rows, cudaStream_t st) {
+  constexpr size_t smem = gw_smem_bytes(CB, MB);
+  constexpr int cols = CB * 64;
   static bool attr_set = false;
-  auto kern = grad_stream_kernel<MB, DROP>;
+  auto kern = grad_stream_kernel<MB, DROP, CB>;
   if (!attr_set) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return MLORA_ERR_CUDA;
     attr_set = true;
   }
   CUtensorMap tQ0, tQ1;
   mlora_status_t ms;
-  // (64, rows, D / 64) views: one box = a 64-row tile of a 512-column strip as eight swizzled 64-column blocks
-  if ((ms = make_tmap_bf16_blocked(ctx, &tQ0, gb.Q, n_rows, gb.D, gb.ldq, GW_ROWS, GW_COLS / 64)) != MLORA_OK) return ms;
-  if ((ms = make_tmap_bf16_blocked(ctx, &tQ1, ga_.Q, n_rows, ga_.D, ga_.ldq, GW_ROWS, GW_COLS / 64)) != MLORA_OK) return ms;
+  // (64, rows, D / 64) views: one box = a 64-row tile of a strip as CB swizzled 64-column blocks
+  if ((ms = make_tmap_bf16_blocked(ctx, &tQ0, gb.Q, n_rows, gb.D, gb.ldq, GW_ROWS, CB)) != MLORA_OK) return ms;
+  if ((ms = make_tmap_bf16_blocked(ctx, &tQ1, ga_.Q, n_rows, ga_.D, ga_.ldq, GW_ROWS, CB)) != MLORA_OK) return ms;
   GradStreamArgs g;
-  g.prob[0] = GradProblem{gb.P, gb.scale, gb.G, gb.D, (gb.D + GW_COLS - 1) / GW_COLS, DropArgs{0, 0, 1.0f}};
-  g.prob[1] = GradProblem{ga_.P, ga_.scale, ga_.G, ga_.D, (ga_.D + GW_COLS - 1) / GW_COLS, ctx->drop};   // dA sees the dropped branch input
+  g.prob[0] = GradProblem{gb.P, gb.scale, gb.G, gb.D, (gb.D + cols - 1) / cols, DropArgs{0, 0, 1.0f}};
+  g.prob[1] = GradProblem{ga_.P, ga_.scale, ga_.G, ga_.D, (ga_.D + cols - 1) / cols, ctx->drop};   // dA sees the dropped branch input
   g.n_problems = 2; g.R = gb.R; g.accumulate = gb.accumulate;
   g.slot_adapter = p->slot_adapter; g.slot_blk_off = p->slot_blk_off; g.blk_row0 = p->blk_row0; g.blk_nrows = p->blk_nrows;
   g.n_slots = n_slots; g.status = ctx->status_dev;
@@ -318,11 +319,21 @@ mlora_status_t launch_grad_stream2_d(mlora_ctx* ctx, const mlora_plan* p, const 
   return scope.done();
 }
 
+template <int MB, bool DROP>
+mlora_status_t launch_grad_stream2_c(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& gb, const GradArgs& ga_, int n_slots,
+                                     int n_rows, cudaStream_t st) {
+  // 512-column strips unless they leave more than a quarter of the SMs without a group
+  const int groups512 = n_slots * ((gb.D + 511) / 512 + (ga_.D + 511) / 512);
+  if (4 * groups512 < 3 * ctx->sm_count)
+    return launch_grad_stream2_d<MB, DROP, 4>(ctx, p, gb, ga_, n_slots, n_rows, st);
+  return launch_grad_stream2_d<MB, DROP, 8>(ctx, p, gb, ga_, n_slots, n_rows, st);
+}
+
 template <int MB>
 mlora_status_t launch_grad_stream2(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& gb, const GradArgs& ga_, int n_slots,
                                    int n_rows, cudaStream_t st) {
-  return ctx->drop.thr != 0 ? launch_grad_stream2_d<MB, true>(ctx, p, gb, ga_, n_slots, n_rows, st)
-                            : launch_grad_stream2_d<MB, false>(ctx, p, gb, ga_, n_slots, n_rows, st);
+  return ctx->drop.thr != 0 ? launch_grad_stream2_c<MB, true>(ctx, p, gb, ga_, n_slots, n_rows, st)
+                            : launch_grad_stream2_c<MB, false>(ctx, p, gb, ga_, n_slots, n_rows, st);
 }
 
 mlora_status_t launch_grad(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& a, int n_slots, int n_rows,

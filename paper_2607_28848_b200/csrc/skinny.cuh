@@ -798,10 +798,16 @@ grad_kernel(const GradArgs a) {
 // goes from registers to memory; rows are visited in one fixed order, so the sums are
 // run-to-run bit-reproducible.  The consumers read no table: the producer leaves each tile's row
 // count in shared memory beside the tile.
-constexpr int GW_COLS = 512;          // columns per strip (8 warps x 64)
+// Narrow problems (few slots x strips for the SMs there are) use 256-column strips instead: four
+// column blocks, and the two warps of a column block take the upper and the lower half of every
+// tile's rows; the lower-half warps hand their accumulators over through shared memory at the end
+// of the group (one fixed order again).
 constexpr int GW_ROWS = 64;           // rows per staged tile
-constexpr int GW_STAGES = 3;
-constexpr uint32_t GW_Q_BYTES = 8 * GW_ROWS * 128;
+__host__ __device__ constexpr int gw_stages(int cb, int mb) { return cb == 8 ? 3 : (mb == 1 ? 5 : 4); }
+__host__ __device__ constexpr size_t gw_smem_bytes(int cb, int mb) {
+  return (size_t)gw_stages(cb, mb) * ((size_t)cb * GW_ROWS * 128 + (size_t)GW_ROWS * mb * 16 * 4) +
+         (cb == 8 ? 0 : (size_t)cb * mb * 16 * 65 * 4) + 1024;
+}
 
 // One launch computes both gradients of a backward: problem 0 (dB: P = u_save scaled, Q = dY,
 // D = d_out) and problem 1 (dA: P = V, Q = x_save, D = d_in); groups of problem 0 come first.
@@ -809,7 +815,7 @@ struct GradProblem {
   const float* P;              // [rows, R] fp32
   const float* scale;          // nullable
   float* G;                    // [n_slots, R, D]
-  int32_t D, n_strips;         // ceil(D / GW_COLS)
+  int32_t D, n_strips;         // ceil(D / strip width)
   DropArgs drop;               // dA with dropout: Q elements kept or dropped, P counts keep_scale (thr == 0: off)
 };
 struct GradStreamArgs {
@@ -824,12 +830,17 @@ struct GradStreamArgs {
   int32_t* status;
 };
 
-template <int MB, bool DROP>
+template <int MB, bool DROP, int CB>
 __global__ void __launch_bounds__(STREAM_THREADS, 1)
 grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_constant__ CUtensorMap tmQ1,
                    const GradStreamArgs ga) {
-  constexpr int S = GW_STAGES;
+  static_assert(CB == 8 || CB == 4, "column blocks per strip");
+  constexpr int S = gw_stages(CB, MB);
   constexpr int RMAX = MB * 16;
+  constexpr int RH = STREAM_WARPS / CB;                  // warps sharing a column block (row halves of a tile)
+  constexpr int KS_PER_WARP = (GW_ROWS / 16) / RH;
+  constexpr int GW_COLS = CB * 64;
+  constexpr uint32_t GW_Q_BYTES = CB * GW_ROWS * 128;
   constexpr uint32_t P_BYTES = GW_ROWS * RMAX * 4;
   constexpr uint32_t STAGE_BYTES = GW_Q_BYTES + P_BYTES;
   extern __shared__ __align__(1024) uint8_t gs_smem[];
@@ -842,7 +853,11 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 #ifdef MLORA_TIMELINE
   const long long tl0 = tl_clock();
+#ifdef MLORA_TL_NO_GRAD
+  const bool tl_on = false;
+#else
   const bool tl_on = threadIdx.x == 0;
+#endif
   long long tl_wait = 0, tl_flush = 0, tl_nflush = 0, tl_nstage = 0;
   if (tl_on) { for (int i = 0; i < 16; ++i) MLORA_TL_SET(i, 0); MLORA_TL_SET(14, tl_global()); }
 #endif
@@ -850,6 +865,9 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
   const uint32_t bar0 = ptx::smem_u32(bars);
   auto bar_full = [&](int st) { return bar0 + 8u * st; };
   auto bar_empty = [&](int st) { return bar0 + 8u * (S + st); };
+  // hand-over buffer of the lower-half warps (CB == 4 only), after the ring
+  float (*red)[MB * 16][64 + 1] = reinterpret_cast<float (*)[MB * 16][64 + 1]>(
+      gs_smem + (ring - ptx::smem_u32(gs_smem)) + S * STAGE_BYTES);
   if (threadIdx.x == 0) {
     for (int st = 0; st < S; ++st) { ptx::mbar_init(bar_full(st), 1); ptx::mbar_init(bar_empty(st), STREAM_WARPS); }
     abort_word = 0;
@@ -910,7 +928,7 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
             stage_meta[st][1] = nr | ((b == b_end - 1 && off + GW_ROWS >= nrows) ? (1 << 16) : 0);
             ptx::mbar_arrive_expect_tx(bar_full(st), GW_Q_BYTES + pbytes);
             // rows past the tile's count are masked by the consumers; blocks past D arrive as zeros
-            ptx::tma_load_3d(dst, tmQ, 0, row0 + off, strip * (GW_COLS / 64), bar_full(st));
+            ptx::tma_load_3d(dst, tmQ, 0, row0 + off, strip * CB, bar_full(st));
             bulk_load(dst + GW_Q_BYTES, pr.P + (size_t)(row0 + off) * R, pbytes, bar_full(st));
           }
           row0 = next_row0; nrows = next_nrows;
@@ -935,7 +953,8 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
       const GradProblem& pr = ga.prob[pi];
       const int gl = grp - pi * groups0;
       const int slot = gl / pr.n_strips, strip = gl % pr.n_strips;
-      const int col0 = strip * GW_COLS + warp * 64;        // this warp's 64 columns
+      const int cblk = warp % CB, half = warp / CB;
+      const int col0 = strip * GW_COLS + cblk * 64;        // this warp's 64 columns
       const bool active = col0 < pr.D;
       const float sc = (pr.scale ? pr.scale[ga.slot_adapter[slot]] : 1.0f) * ((DROP && pr.drop.thr != 0) ? pr.drop.keep_scale : 1.0f);
 #pragma unroll
@@ -958,11 +977,12 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
         // plain shared-memory loads (no branches around them): what lies past a tile's rows is read
         // and then replaced by zero
         const uint8_t* stage_ptr = gs_smem + (ring - ptx::smem_u32(gs_smem)) + (size_t)st * STAGE_BYTES;
-        const uint8_t* qtile = stage_ptr + (size_t)warp * (GW_ROWS * 128u);
+        const uint8_t* qtile = stage_ptr + (size_t)cblk * (GW_ROWS * 128u);
         const float* ptile = reinterpret_cast<const float*>(stage_ptr + GW_Q_BYTES);
         if (active) {
 #pragma unroll
-          for (int ks = 0; ks < GW_ROWS / 16; ++ks) {
+          for (int kk = 0; kk < KS_PER_WARP; ++kk) {
+            const int ks = half * KS_PER_WARP + kk;
             if (ks * 16 >= nrows) break;
             // rows of this K-step: r = 16 ks + {2c, 2c+1, 2c+8, 2c+9}
             uint4 q[4];
@@ -1024,7 +1044,29 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
       // The n index g of the MMA was mapped to piece g of a row, so for thread (g, c) accumulator
       // element e of column block nb is strip column 8 (2c + (e & 1)) + nb: over nb = 0..7 that is
       // eight consecutive columns, written as two 16-byte stores (rows g and g + 8 for e >> 1).
-      if (active) {
+      if (RH == 2) {       // the lower-half warp of a column block hands its sums to the upper-half warp
+        if (half == 1) {
+#pragma unroll
+          for (int m = 0; m < MB; ++m)
+#pragma unroll
+            for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+              for (int e = 0; e < 4; ++e)
+                red[cblk][m * 16 + g + ((e >> 1) ? 8 : 0)][8 * (2 * c + (e & 1)) + nb] = acc[m][nb][e];
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");
+        if (half == 0) {
+#pragma unroll
+          for (int m = 0; m < MB; ++m)
+#pragma unroll
+            for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+              for (int e = 0; e < 4; ++e)
+                acc[m][nb][e] += red[cblk][m * 16 + g + ((e >> 1) ? 8 : 0)][8 * (2 * c + (e & 1)) + nb];
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");   // red[] is reused by the next group
+      }
+      if (active && half == 0) {
 #pragma unroll
         for (int m = 0; m < MB; ++m)
 #pragma unroll
