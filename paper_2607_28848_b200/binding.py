@@ -123,12 +123,12 @@ def _check(status: int, where: str) -> None:
         raise MloraError(status, where)
 
 
-def _segments_ctypes(segments) -> "ctypes.Array":
+def _segments_ctypes(segments):
+    """A [n, 4] int32 array has the memory layout of mlora_segment_t[n]: pass it as it is."""
     seg = np.ascontiguousarray(np.asarray(segments, dtype=np.int32).reshape(-1, 4))
-    arr = (mlora_segment_t * max(len(seg), 1))()
-    for i, (a, b, c, d) in enumerate(seg.tolist()):
-        arr[i] = mlora_segment_t(a, b, c, d)
-    return arr, len(seg)
+    if len(seg) == 0:
+        return (mlora_segment_t * 1)(), 0
+    return (mlora_segment_t * len(seg)).from_buffer_copy(seg.tobytes()), len(seg)
 
 
 # --------------------------------------------------------------------------------------------
