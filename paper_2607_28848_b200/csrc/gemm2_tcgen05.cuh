@@ -186,6 +186,8 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
 
   const int KB = (args.K + GEMM_BK - 1) / GEMM_BK;
   const int n_units = args.n_units;
+  const int SK = args.split_k;                       // K slices per tile; unit = slice * n_tiles + tile
+  const int n_tiles = args.n_mtiles * args.n_ntiles;
   const int n_pairs = gridDim.x >> 1;
   const int pair = blockIdx.x >> 1;
 
@@ -202,11 +204,13 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
     uint32_t it = 0;
     bool ok = true;
     for (int unit = pair; unit < n_units && ok; unit += n_pairs) {
-      const int mt = unit % args.n_mtiles, nt = unit / args.n_mtiles;
+      const int tile = unit % n_tiles, ks = unit / n_tiles;
+      const int mt = tile % args.n_mtiles, nt = tile / args.n_mtiles;
       const int m0 = mt * GEMM2_BM + (int)rank * 128;
       const int nh = nt * GEMM2_BN + (int)rank * 128;     // this CTA's half of the B columns
-      const int G = tile_groups(mt);
+      const int G = ks == SK - 1 ? tile_groups(mt) : 0;   // the low-rank blocks ride with the last K slice
       const int LC = (G * R + 63) / 64;
+      const int kb_begin = (int)((long long)ks * KB / SK), kb_end = (int)((long long)(ks + 1) * KB / SK);
       const int chunk_base = args.lora_enabled ? args.tile_grp_off[mt] : 0;   // chunk slot = 2 * this + lc
       int32_t ga_reg[8];                                  // G <= 256 adapters of the pair tile
       {
@@ -214,7 +218,7 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
 #pragma unroll
         for (int j = 0; j < 8; ++j) ga_reg[j] = (lane + 32 * j < G) ? ga[lane + 32 * j] : 0;
       }
-      for (int kb = 0; kb < KB; ++kb, ++it) {
+      for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
         const int s = it % S;
         if (lane == 0) {
           ok = gemm2_wait(bar_empty(s), ((it / S) & 1) ^ 1, abort_flag, args.status);
@@ -273,13 +277,15 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
       uint32_t it = 0, lt = 0;
       bool ok = true;
       for (int unit = pair; unit < n_units && ok; unit += n_pairs, ++lt) {
-        const int mt = unit % args.n_mtiles;
+        const int tile = unit % n_tiles, ks = unit / n_tiles;
+        const int mt = tile % args.n_mtiles;
+        const int kb_begin = (int)((long long)ks * KB / SK), kb_end = (int)((long long)(ks + 1) * KB / SK);
         const uint32_t buf = lt & 1;
         if (!(ok = gemm2_wait(bar_tempty(buf), ((lt >> 1) & 1) ^ 1, abort_flag, args.status))) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * GEMM2_BN;
         uint32_t acc = 0;
-        for (int kb = 0; kb < KB; ++kb, ++it) {
+        for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
           const int s = it % S;
           if (!(ok = gemm2_wait(bar_full(s), (it / S) & 1, abort_flag, args.status))) break;
           ptx::tc_fence_after();
@@ -295,7 +301,7 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
           ptx::umma2_commit_both(bar_empty(s));
         }
         if (!ok) break;
-        const int G = tile_groups(mt);
+        const int G = ks == SK - 1 ? tile_groups(mt) : 0;
         const int LC = (G * R + 63) / 64;
         for (int lc = 0; lc < LC; ++lc, ++it) {
           const int s = it % S;
@@ -324,7 +330,8 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
     uint32_t lt = 0;
     bool ok = true;
     for (int unit = pair; unit < n_units && ok; unit += n_pairs, ++lt) {
-      const int mt = unit % args.n_mtiles, nt = unit / args.n_mtiles;
+      const int tile = unit % n_tiles, ks = unit / n_tiles;
+      const int mt = tile % args.n_mtiles, nt = tile / args.n_mtiles;
       const int m0 = mt * GEMM2_BM + (int)rank * 128 + e * 32, n0 = nt * GEMM2_BN;
       const uint32_t buf = lt & 1;
       if (!(ok = gemm2_wait(bar_tfull(buf), (lt >> 1) & 1, abort_flag, args.status))) break;
@@ -340,6 +347,21 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
           ptx::tc_fence_before();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_tempty(buf), 0));
+        }
+        if (SK > 1) {       // a K slice: this lane's row of the fp32 partial, 64 columns, for the reduction kernel
+          const int row = m0 + lane;
+          if (row < args.M) {
+            float* dst = args.ws_splitk + ((size_t)ks * args.M + row) * args.N + n0 + c * 64;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              if (n0 + c * 64 + 4 * j < args.N)
+                *reinterpret_cast<uint4*>(dst + 4 * j) = make_uint4(v0[4 * j], v0[4 * j + 1], v0[4 * j + 2], v0[4 * j + 3]);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              if (n0 + c * 64 + 32 + 4 * j < args.N)
+                *reinterpret_cast<uint4*>(dst + 32 + 4 * j) = make_uint4(v1[4 * j], v1[4 * j + 1], v1[4 * j + 2], v1[4 * j + 3]);
+          }
+          continue;
         }
         const uint32_t sb = stage0 + (uint32_t)(c & 1) * 4096u;
         if (lane == 0) ptx::tma_store_wait_read<1>();
@@ -383,6 +405,28 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
     ptx::tc_fence_after();
     ptx::tmem2_dealloc(tmem_base, GEMM_TMEM_COLS);
   }
+}
+
+// Sum of the K slices of a split product: Out[m, n] = bf16(sum over slices of ws[slice, m, n]),
+// slices added in index order.  One thread per 8 columns (N is a multiple of 64).
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float* ws, int split_k, __nv_bfloat16* Out, int64_t ld_out, int M, int N) {
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();
+  const int64_t n8 = N / 8;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)M * n8) return;
+  const int m = (int)(idx / n8), n = (int)(idx % n8) * 8;
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  for (int s = 0; s < split_k; ++s) {
+    const float4* src = reinterpret_cast<const float4*>(ws + ((size_t)s * M + m) * N + n);
+    const float4 a = src[0], b = src[1];
+    acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
+    acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
+  }
+  *reinterpret_cast<uint4*>(Out + (size_t)m * ld_out + n) =
+      make_uint4(ptx::pack_bf16(acc[0], acc[1]), ptx::pack_bf16(acc[2], acc[3]), ptx::pack_bf16(acc[4], acc[5]),
+                 ptx::pack_bf16(acc[6], acc[7]));
 }
 
 }  // namespace mlora

@@ -37,10 +37,12 @@ struct mlora_ctx {
   int64_t ws_counter_items = 0;
   __nv_bfloat16* ws_pbd = nullptr;   // block-diagonal low-rank operand: [2 * ws_pbd_groups * 256, 64] bf16
   int64_t ws_pbd_groups = 0;
+  float* ws_splitk = nullptr;        // fp32 partial products of a K-split GEMM (fixed size, see kSplitKBytes)
   int64_t launches = 0;
   int32_t gemm_path = 0;
   int32_t shrink_path = 0;           // 0: streaming kernel for rank <= 32; 1: per-item kernel for every rank
   int32_t gemm_pairs = 1;            // 1: two-SM (CTA pair) tensor-core kernel; 0: one-SM kernel
+  int32_t no_split_k = 0;            // 1: the two-SM kernel never splits K (kernel variant 4)
   EncodeTiledFn encode = nullptr;
   const volatile int32_t* cancel = nullptr;   // caller's host flag, read before every launch
   DropArgs drop = {0, 0, 1.0f};               // LoRA dropout of the fine-tuning rows (thr == 0: off)
@@ -99,6 +101,10 @@ struct BlobBuilder {
     return off;
   }
 };
+
+// Workspace for K-split products of small-batch GEMMs: allocated once per context, so that no
+// compute call allocates.  Problems whose partials do not fit run unsplit.
+constexpr size_t kSplitKBytes = 64u << 20;
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -457,11 +463,25 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
     return s;
   if ((s = make_tmap_bf16(ctx, &tOut, Out, N, M, ld_out, 64, 32)) != MLORA_OK) return s;
   GemmArgs g;
-  g.M = M; g.N = N; g.K = K;
+  g.M = M; g.N = N; g.K = K; g.split_k = 1; g.ws_splitk = nullptr;
   if (ctx->gemm_pairs) {            // two-SM kernel: 256-row tiles and their group tables
     g.n_mtiles = (M + GEMM2_BM - 1) / GEMM2_BM;
     g.n_ntiles = (N + GEMM2_BN - 1) / GEMM2_BN;
-    g.n_full = g.n_units = g.n_mtiles * g.n_ntiles;
+    // Few tiles for the CTA pairs there are (small batches, the backward of one 256-token fine-tuning
+    // batch): cut K into slices that run on different pairs; the fp32 partials are summed by a
+    // small kernel afterwards (≈8 µs with its launch, so only contractions of 8192 and more are
+    // split, into slices of at least 32 K-blocks).
+    const int tiles = g.n_mtiles * g.n_ntiles, pairs = ctx->sm_count / 2, kblocks = (K + GEMM_BK - 1) / GEMM_BK;
+    int sk = 1;
+    if (2 * tiles <= pairs && kblocks >= 128 && !ctx->no_split_k) {
+      sk = pairs / tiles;
+      sk = sk < kblocks / 32 ? sk : kblocks / 32;
+      sk = sk < 8 ? sk : 8;
+      while (sk > 1 && (size_t)sk * M * N * sizeof(float) > kSplitKBytes) --sk;
+      sk = sk < 1 ? 1 : sk;
+    }
+    g.split_k = sk; g.ws_splitk = ctx->ws_splitk;
+    g.n_full = g.n_units = tiles * sk;
     g.lora_enabled = (lora && !hs.grp2_adapter.empty()) ? 1 : 0;
     g.row_grp = ds.row_grp2; g.row_adapter = ds.row_adapter;
     g.tile_grp_off = ds.tile2_grp_off; g.grp_adapter = ds.grp2_adapter;
@@ -470,7 +490,13 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
     const uint64_t slots = g.lora_enabled ? 2 * (uint64_t)hs.grp2_adapter.size() : 1;
     if ((s = make_tmap_bf16(ctx, &tPbd, ctx->ws_pbd ? (const void*)ctx->ws_pbd : In, 64, slots * 256, 64, 64, 128)) != MLORA_OK)
       return s;
-    return launch_gemm2<W_KMAJOR>(ctx, R, tIn, tW, tL, tOut, tPbd, g, st);
+    if ((s = launch_gemm2<W_KMAJOR>(ctx, R, tIn, tW, tL, tOut, tPbd, g, st)) != MLORA_OK || sk == 1) return s;
+    if (cancelled(ctx)) return MLORA_CANCELLED;
+    LaunchScope scope(ctx, st, W_KMAJOR ? KIND_GEMM_BWD : KIND_GEMM_FWD);
+    const int64_t threads = (int64_t)M * (N / 8);
+    launch_pdl(scope.slot < 0, splitk_reduce_kernel, dim3((unsigned)((threads + 255) / 256)), dim3(256), 0, st,
+               (const float*)ctx->ws_splitk, sk, (__nv_bfloat16*)Out, ld_out, M, N);
+    return scope.done();
   }
   g.n_mtiles = (M + GEMM_BM - 1) / GEMM_BM;
   g.n_ntiles = (N + GEMM_BN - 1) / GEMM_BN;
@@ -670,6 +696,7 @@ mlora_status_t mlora_create(mlora_ctx** out, int device) {
   }
   c->encode = reinterpret_cast<EncodeTiledFn>(fn);
   if (cudaMalloc(&c->status_dev, sizeof(int32_t)) != cudaSuccess ||
+      cudaMalloc(&c->ws_splitk, kSplitKBytes) != cudaSuccess ||
       cudaMemset(c->status_dev, 0, sizeof(int32_t)) != cudaSuccess) {
     delete c;
     return MLORA_ERR_CUDA;
@@ -718,6 +745,7 @@ void mlora_destroy(mlora_ctx* c) {
   cudaFree(c->ws_partial);
   cudaFree(c->ws_counters);
   cudaFree(c->ws_pbd);
+  cudaFree(c->ws_splitk);
   delete c;
 }
 
@@ -984,10 +1012,11 @@ mlora_status_t mlora_set_dropout(mlora_ctx* ctx, double p, uint64_t seed) {
 int64_t mlora_launch_count(const mlora_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path) {
-  if (!ctx || path < 0 || path > 3) return MLORA_ERR_INVALID_ARG;
+  if (!ctx || path < 0 || path > 4) return MLORA_ERR_INVALID_ARG;
   ctx->gemm_path = path == 1 ? 1 : 0;
   ctx->shrink_path = path == 2 ? 1 : 0;
   ctx->gemm_pairs = path == 3 ? 0 : 1;
+  ctx->no_split_k = path == 4 ? 1 : 0;
   return MLORA_OK;
 }
 

@@ -77,7 +77,7 @@ def test_cfg1_tiny_fp32(sess):
     run_and_check(sess, w, synth.make_tensors(w))
 
 
-@pytest.mark.parametrize("path", [0, 1, 2, 3])
+@pytest.mark.parametrize("path", [0, 1, 2, 3, 4])
 def test_bf16_ragged_multi_tile(sess, path):
     w = synth.random_workload(5, 256, 512, 16, 6, 389, max_seg=150)
     run_and_check(sess, w, synth.make_tensors(w), path=path)
@@ -92,6 +92,23 @@ def test_fp32_ragged(sess):
 def test_rank_sweep(sess, rank):
     w = synth.random_workload(10 + rank, 320, 448, rank, 7, 300, max_seg=90)
     run_and_check(sess, w, synth.make_tensors(w))
+
+
+@pytest.mark.parametrize("rank", [8, 16, 128])
+def test_no_split_k(sess, rank):
+    """The two-SM kernel without K slices on a small problem (kernel variant 4); the default splits it."""
+    w = synth.random_workload(10 + rank, 320, 448, rank, 7, 300, max_seg=90)
+    run_and_check(sess, w, synth.make_tensors(w), path=4)
+
+
+@pytest.mark.parametrize("k", [8192, 8192 + 64 * 37, 16384])
+def test_split_k_slices(sess, k):
+    """Long contractions with few output tiles: 4 to 8 K slices (also a K that the slices do not divide evenly)."""
+    segs = synth.segments_array([(0, 100, 0, 0), (100, 60, 1, 1), (160, 30, 2, 0), (190, 64, 0, 1)])
+    w = synth.Workload("split_k", k, 256, 16, 3, "bf16", 254, segs, seed=k)
+    run_and_check(sess, w, synth.make_tensors(w), blocked=True)
+    w2 = synth.Workload("split_k_bwd", 256, k, 16, 3, "bf16", 254, segs, seed=k + 1)      # long K in the backward GEMM
+    run_and_check(sess, w2, synth.make_tensors(w2), blocked=True)
 
 
 @pytest.mark.parametrize("rank", [8, 128])
