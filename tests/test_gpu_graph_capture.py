@@ -15,9 +15,15 @@ from paper_2607_28848_b200.runner import LayerRun, Session
 pytestmark = pytest.mark.gpu
 
 
-def test_graph_replay_matches_eager_on_new_inputs():
+@pytest.mark.parametrize("case", ["mixed", "long_k_split", "dropout"])
+def test_graph_replay_matches_eager_on_new_inputs(case):
     with Session(0) as sess:
-        w = synth.random_workload(61, 256, 384, 16, 5, 420, max_seg=130, p_finetune=0.4)
+        if case == "long_k_split":      # few output tiles and K = 8192: the K-split GEMM and its reduction kernel
+            w = synth.random_workload(62, 8192, 256, 16, 3, 200, max_seg=80, p_finetune=0.5)
+        else:
+            w = synth.random_workload(61, 256, 384, 16, 5, 420, max_seg=130, p_finetune=0.4)
+        if case == "dropout":           # the seed is part of the captured launch parameters
+            mb.mlora_set_dropout(sess.ctx, 0.1, 4321)
         t = synth.make_tensors(w)
         run = LayerRun(sess, "bf16", t, w.segments, w.n_rows)
         dev = sess.device
