@@ -105,6 +105,7 @@ struct BlobBuilder {
 // Workspace for K-split products of small-batch GEMMs: allocated once per context, so that no
 // compute call allocates.  Problems whose partials do not fit run unsplit.
 constexpr size_t kSplitKBytes = 64u << 20;
+constexpr int kMaxDevices = 64;      // device ordinals a process may create contexts on
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -233,7 +234,8 @@ mlora_status_t launch_shrink_stream_d(mlora_ctx* ctx, ShrinkArgs a, int n_items,
   } else {
     tSave = tIn;
   }
-  static bool attr_set = false;
+  static bool attr_set_dev[kMaxDevices] = {};   // per instantiation and device
+  bool& attr_set = attr_set_dev[ctx->device];
   auto kern = shrink_stream_kernel<RB, STAGES, CHUNK, DROP>;
   if (!attr_set) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return MLORA_ERR_CUDA;
@@ -300,7 +302,8 @@ mlora_status_t launch_grad_stream2_d(mlora_ctx* ctx, const mlora_plan* p, const 
                                      int n_rows, cudaStream_t st) {
   constexpr size_t smem = gw_smem_bytes(CB, MB);
   constexpr int cols = CB * 64;
-  static bool attr_set = false;
+  static bool attr_set_dev[kMaxDevices] = {};   // per instantiation and device
+  bool& attr_set = attr_set_dev[ctx->device];
   auto kern = grad_stream_kernel<MB, DROP, CB>;
   if (!attr_set) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return MLORA_ERR_CUDA;
@@ -347,7 +350,8 @@ mlora_status_t launch_grad(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& 
   if (n_slots <= 0) return MLORA_OK;
   if (cancelled(ctx)) return MLORA_CANCELLED;
   constexpr int smem1 = (GRAD_THREADS / 32) * 16 * 65 * 4, smem2 = 2 * smem1;
-  static bool attr_set = false;
+  static bool attr_set_dev[kMaxDevices] = {};   // per instantiation and device
+  bool& attr_set = attr_set_dev[ctx->device];
   if (!attr_set) {
     if (cudaFuncSetAttribute(grad_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2) != cudaSuccess)
       return MLORA_ERR_CUDA;
@@ -379,7 +383,8 @@ mlora_status_t launch_expand_mask(mlora_ctx* ctx, const mlora_layer_t* L, const 
 template <int R, bool W_KMAJOR>
 mlora_status_t launch_gemm_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUtensorMap& tW, const CUtensorMap& tL,
                              const CUtensorMap& tOut, const GemmArgs& g, cudaStream_t st) {
-  static bool attr_set = false;     // per instantiation; the attribute is per function, per device context
+  static bool attr_set_dev[kMaxDevices] = {};   // per instantiation and device: the attribute belongs to the device's context
+  bool& attr_set = attr_set_dev[ctx->device];
   auto kern = gemm_lora_kernel<R, W_KMAJOR>;
   if (!attr_set) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_BYTES) != cudaSuccess)
@@ -397,7 +402,8 @@ mlora_status_t launch_gemm_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUten
 template <int R, bool W_KMAJOR>
 mlora_status_t launch_gemm2_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUtensorMap& tW, const CUtensorMap& tL,
                               const CUtensorMap& tOut, const CUtensorMap& tPbd, const GemmArgs& g, cudaStream_t st) {
-  static int max_pairs = 0;         // per instantiation
+  static int max_pairs_dev[kMaxDevices] = {};   // per instantiation and device
+  int& max_pairs = max_pairs_dev[ctx->device];
   auto kern = gemm2_lora_kernel<R, W_KMAJOR>;
   if (max_pairs == 0) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM2_SMEM_BYTES) != cudaSuccess)
@@ -598,7 +604,6 @@ mlora_status_t backward_simt(mlora_ctx* ctx, const mlora_layer_t* L, const mlora
 static __device__ __align__(256) float g_noalloc_scratch[MLORA_NOALLOC_MAX_ROWS * mlora::kMaxRank];
 
 namespace {
-constexpr int kMaxDevices = 64;
 float* g_noalloc_addr[kMaxDevices] = {};
 std::mutex g_noalloc_mutex;
 
@@ -678,7 +683,7 @@ mlora_status_t mlora_create(mlora_ctx** out, int device) {
   *out = nullptr;
   int n = 0;
   if (cudaGetDeviceCount(&n) != cudaSuccess || n <= 0) { cudaGetLastError(); return MLORA_ERR_ARCH; }
-  if (device < 0 || device >= n) return MLORA_ERR_INVALID_ARG;
+  if (device < 0 || device >= n || device >= kMaxDevices) return MLORA_ERR_INVALID_ARG;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MLORA_ERR_CUDA;
   if (prop.major != 10) return MLORA_ERR_ARCH;

@@ -458,7 +458,7 @@ def _sampled_check(sess, w, n_sample=24, seed=0):
         run.close()
 
 
-@pytest.mark.parametrize("proj", ["k", "gate", "down"])
+@pytest.mark.parametrize("proj", ["q", "k", "v", "o", "gate", "up", "down"])
 def test_cfg3_projection_sampled(sess, proj):
     _sampled_check(sess, synth.cfg3_layer_set(projections=[proj])[0])
 
