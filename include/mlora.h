@@ -104,6 +104,22 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
                                  int32_t n_rows, int32_t n_adapters, mlora_plan** plan);
 void mlora_plan_destroy(mlora_plan* plan);
 
+/* Stream-ordered variant for serving loops, where every step has a new batch mix (paper,
+ * Section 4.2: the admission decision is taken per scheduling step): the tables go into a buffer
+ * pair (device + pinned host staging) taken from a pool inside the context and are uploaded with
+ * an asynchronous copy on `cuda_stream`; compute calls that use the plan must be queued on that
+ * same stream (or on one ordered after it).  In steady state the call neither allocates nor
+ * synchronises (a pool miss allocates a pair, a batch larger than any before grows the context's
+ * workspace as mlora_plan_create does - neither inside a stream capture).  ctx must not be NULL.
+ * mlora_plan_release gives the pair back: it records an event on `cuda_stream` (the stream the
+ * plan's last compute call was queued on) and the pair is reused once that event has passed; the
+ * plan handle is invalid afterwards.  mlora_plan_destroy also accepts such a plan (it frees the
+ * pair, waiting for the device).  Errors: as mlora_plan_create. */
+mlora_status_t mlora_plan_create_async(mlora_ctx* ctx, const mlora_segment_t* segs, int32_t n_segs,
+                                       int32_t n_rows, int32_t n_adapters, void* cuda_stream,
+                                       mlora_plan** plan);
+mlora_status_t mlora_plan_release(mlora_plan* plan, void* cuda_stream);
+
 int32_t mlora_plan_rows(const mlora_plan* plan);        /* n_rows                              */
 int32_t mlora_plan_ft_rows(const mlora_plan* plan);     /* total fine-tuning rows, T_ft        */
 /* Writes up to `cap` adapter ids, slot g -> adapter id, and returns the number of slots. */

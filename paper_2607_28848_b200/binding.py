@@ -25,7 +25,7 @@ EXPORTS = (
     "mlora_plan_ft_rows", "mlora_plan_ft_adapters", "mlora_plan_describe", "mlora_mixed_forward",
     "mlora_backward", "mlora_poll_status", "mlora_status_string", "mlora_launch_count", "mlora_set_gemm_path",
     "mlora_profile_enable", "mlora_profile_collect", "mlora_forward_noalloc", "mlora_adamw_update",
-    "mlora_set_cancel_flag", "mlora_set_dropout",
+    "mlora_set_cancel_flag", "mlora_set_dropout", "mlora_plan_create_async", "mlora_plan_release",
 )
 MLORA_NOALLOC_MAX_ROWS = 512
 
@@ -78,6 +78,10 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.mlora_plan_create.restype = ctypes.c_int
     lib.mlora_plan_destroy.argtypes = [vp]
     lib.mlora_plan_destroy.restype = None
+    lib.mlora_plan_create_async.argtypes = [vp, P(mlora_segment_t), i32, i32, i32, vp, P(vp)]
+    lib.mlora_plan_create_async.restype = ctypes.c_int
+    lib.mlora_plan_release.argtypes = [vp, vp]
+    lib.mlora_plan_release.restype = ctypes.c_int
     lib.mlora_plan_rows.argtypes = [vp]
     lib.mlora_plan_rows.restype = i32
     lib.mlora_plan_ft_rows.argtypes = [vp]
@@ -154,6 +158,19 @@ def mlora_plan_create(ctx, segments, n_rows: int, n_adapters: int) -> ctypes.c_v
 
 def mlora_plan_destroy(plan) -> None:
     load_library().mlora_plan_destroy(plan)
+
+
+def mlora_plan_create_async(ctx, segments, n_rows: int, n_adapters: int, stream=None) -> ctypes.c_void_p:
+    """Stream-ordered plan from the context's buffer pool (tables uploaded on the current or given stream)."""
+    arr, n = _segments_ctypes(segments)
+    h = ctypes.c_void_p()
+    _check(load_library().mlora_plan_create_async(ctx, arr, n, int(n_rows), int(n_adapters), _stream_ptr(stream),
+                                                  ctypes.byref(h)), "mlora_plan_create_async")
+    return h
+
+
+def mlora_plan_release(plan, stream=None) -> None:
+    _check(load_library().mlora_plan_release(plan, _stream_ptr(stream)), "mlora_plan_release")
 
 
 def mlora_plan_rows(plan) -> int:

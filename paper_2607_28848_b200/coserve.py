@@ -124,19 +124,19 @@ class GpuExecutor:
 
     def forward(self, table, n_rows, save_base, cancel=False) -> bool:
         mb = self.mb
-        plan = mb.mlora_plan_create(self.sess.ctx, table, n_rows, self.n_adapters)
+        plan = mb.mlora_plan_create_async(self.sess.ctx, table, n_rows, self.n_adapters)
         try:
             if cancel:
                 return False
             mb.mlora_mixed_forward(self.sess.ctx, self.layer, plan, self.X, self.Y, self.x_save, self.u_save, save_base,
                                    self.cap)
         finally:
-            mb.mlora_plan_destroy(plan)
+            mb.mlora_plan_release(plan)
         return True
 
     def backward(self, table, n_rows) -> None:
         mb, torch = self.mb, self.torch
-        plan = mb.mlora_plan_create(self.sess.ctx, table, n_rows, self.n_adapters)
+        plan = mb.mlora_plan_create_async(self.sess.ctx, table, n_rows, self.n_adapters)
         try:
             self.slots = mb.mlora_plan_ft_adapters(plan)
             n = max(len(self.slots), 1)
@@ -144,11 +144,11 @@ class GpuExecutor:
             self.dB = torch.empty((n, self.rank, self.d_out), dtype=torch.float32, device=self.sess.device)
             mb.mlora_backward(self.sess.ctx, self.layer, plan, self.dY, self.x_save, self.u_save, self.dA, self.dB, self.dX)
         finally:
-            mb.mlora_plan_destroy(plan)
+            mb.mlora_plan_release(plan)
 
     def update(self, table, n_rows) -> None:
         mb, torch = self.mb, self.torch
-        plan = mb.mlora_plan_create(self.sess.ctx, table, n_rows, self.n_adapters)
+        plan = mb.mlora_plan_create_async(self.sess.ctx, table, n_rows, self.n_adapters)
         try:
             key = tuple(self.slots)
             if key not in self.opt:
@@ -160,7 +160,7 @@ class GpuExecutor:
             mb.mlora_adamw_update(self.sess.ctx, self.layer, plan, self.dA, self.dB, wA, wB, mA, vA, mB, vB, self.step_no,
                                   lr=1e-6)
         finally:
-            mb.mlora_plan_destroy(plan)
+            mb.mlora_plan_release(plan)
 
 
 def synthetic_arrivals(n_steps: int, seed: int, n_adapters: int):

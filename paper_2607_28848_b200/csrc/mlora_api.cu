@@ -25,6 +25,21 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// Device tables + pinned staging of a stream-ordered plan; `free_evt` marks the point on a stream
+// after which the pair may be reused.
+struct PlanBuf {
+  int32_t* dev = nullptr;
+  int32_t* pinned = nullptr;
+  size_t cap = 0;                    // in 32-bit words
+  cudaEvent_t free_evt = nullptr;
+};
+static inline void free_plan_buf(PlanBuf& b) {
+  if (b.dev) cudaFree(b.dev);
+  if (b.pinned) cudaFreeHost(b.pinned);
+  if (b.free_evt) cudaEventDestroy(b.free_evt);
+  b = PlanBuf();
+}
+
 struct mlora_ctx {
   int device = 0;
   int sm_count = 0;
@@ -38,6 +53,7 @@ struct mlora_ctx {
   __nv_bfloat16* ws_pbd = nullptr;   // block-diagonal low-rank operand: [2 * ws_pbd_groups * 256, 64] bf16
   int64_t ws_pbd_groups = 0;
   float* ws_splitk = nullptr;        // fp32 partial products of a K-split GEMM (fixed size, see kSplitKBytes)
+  std::vector<PlanBuf> plan_pool;    // released buffers of stream-ordered plans
   int64_t launches = 0;
   int32_t gemm_path = 0;
   int32_t shrink_path = 0;           // 0: streaming kernel for rank <= 32; 1: per-item kernel for every rank
@@ -79,6 +95,8 @@ struct mlora_plan {
   HostPlan h;
   mlora_ctx* ctx = nullptr;
   int32_t* blob = nullptr;           // all device tables in one allocation
+  PlanBuf buf;                       // pooled plans: the buffer pair the tables live in (blob == buf.dev)
+  bool pooled = false;
   DevRowSpace fwd, bwd;
   const int32_t* slot_chunk_off = nullptr;
   const int32_t* chunk_row0 = nullptr;
@@ -751,8 +769,84 @@ void mlora_destroy(mlora_ctx* c) {
   cudaFree(c->ws_counters);
   cudaFree(c->ws_pbd);
   cudaFree(c->ws_splitk);
+  for (PlanBuf& b : c->plan_pool) free_plan_buf(b);
   delete c;
 }
+
+namespace {
+
+constexpr int kPlanTables = 37;
+
+// All device tables of a plan, packed; o[] receives each table's offset in 32-bit words.
+void pack_plan(const HostPlan& h, BlobBuilder& b, size_t* o) {
+  int n = 0;
+  const RowSpace* rs[2] = {&h.fwd, &h.bwd};
+  for (int i = 0; i < 2; ++i) {
+    o[n++] = b.add(rs[i]->row_adapter); o[n++] = b.add(rs[i]->row_save); o[n++] = b.add(rs[i]->row_grp);
+    o[n++] = b.add(rs[i]->tile_grp_off); o[n++] = b.add(rs[i]->grp_adapter); o[n++] = b.add(rs[i]->item_rows);
+    o[n++] = b.add(rs[i]->row_grp2); o[n++] = b.add(rs[i]->tile2_grp_off); o[n++] = b.add(rs[i]->grp2_adapter);
+    o[n++] = b.add(rs[i]->zero_rows2);
+    o[n++] = b.add(rs[i]->item_save); o[n++] = b.add(rs[i]->item_start); o[n++] = b.add(rs[i]->item_desc);
+    o[n++] = b.add(rs[i]->item_nrows); o[n++] = b.add(rs[i]->item_adapter);
+  }
+  o[n++] = b.add(h.slot_chunk_off); o[n++] = b.add(h.chunk_row0); o[n++] = b.add(h.chunk_nrows);
+  o[n++] = b.add(h.ft_adapters);
+  o[n++] = b.add(h.slot_blk_off); o[n++] = b.add(h.blk_row0); o[n++] = b.add(h.blk_nrows);
+}
+
+// Points the plan's table pointers into p->blob.
+void bind_plan(mlora_plan* p, const size_t* o) {
+  DevRowSpace* ds[2] = {&p->fwd, &p->bwd};
+  int n = 0;
+  for (int i = 0; i < 2; ++i) {
+    ds[i]->row_adapter = p->blob + o[n++]; ds[i]->row_save = p->blob + o[n++]; ds[i]->row_grp = p->blob + o[n++];
+    ds[i]->tile_grp_off = p->blob + o[n++]; ds[i]->grp_adapter = p->blob + o[n++]; ds[i]->item_rows = p->blob + o[n++];
+    ds[i]->row_grp2 = p->blob + o[n++]; ds[i]->tile2_grp_off = p->blob + o[n++]; ds[i]->grp2_adapter = p->blob + o[n++];
+    ds[i]->zero_rows2 = p->blob + o[n++];
+    ds[i]->item_save = p->blob + o[n++]; ds[i]->item_start = p->blob + o[n++]; ds[i]->item_desc = p->blob + o[n++];
+    ds[i]->item_nrows = p->blob + o[n++]; ds[i]->item_adapter = p->blob + o[n++];
+  }
+  p->bwd.row_save = nullptr;       // the compact space has no save offsets
+  p->slot_chunk_off = p->blob + o[n++]; p->chunk_row0 = p->blob + o[n++]; p->chunk_nrows = p->blob + o[n++];
+  p->slot_adapter = p->blob + o[n++];
+  p->slot_blk_off = p->blob + o[n++]; p->blk_row0 = p->blob + o[n++]; p->blk_nrows = p->blob + o[n++];
+}
+
+// Grows the context's workspaces to what this plan needs (synchronises the device when it has to
+// grow one; in steady state nothing happens here).
+mlora_status_t grow_workspaces(mlora_ctx* ctx, const HostPlan& h, int32_t n_rows) {
+  if (n_rows > ctx->ws_rows) {     // the rank-r workspace
+    if (cudaDeviceSynchronize() != cudaSuccess) return MLORA_ERR_CUDA;
+    cudaFree(ctx->ws_p);
+    ctx->ws_p = nullptr; ctx->ws_rows = 0;
+    if (cudaMalloc(&ctx->ws_p, (size_t)n_rows * kMaxRank * sizeof(float)) != cudaSuccess) return MLORA_ERR_CUDA;
+    ctx->ws_rows = n_rows;
+  }
+  const int64_t items = h.fwd.n_items() > h.bwd.n_items() ? h.fwd.n_items() : h.bwd.n_items();
+  const int64_t part_items = items + 4 * ctx->sm_count;      // items * ksplit never exceeds this
+  if (part_items > ctx->ws_partial_items || items > ctx->ws_counter_items) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return MLORA_ERR_CUDA;
+    cudaFree(ctx->ws_partial); cudaFree(ctx->ws_counters);
+    ctx->ws_partial = nullptr; ctx->ws_counters = nullptr; ctx->ws_partial_items = ctx->ws_counter_items = 0;
+    if (cudaMalloc(&ctx->ws_partial, (size_t)part_items * kItemRows * kMaxRank * sizeof(float)) != cudaSuccess ||
+        cudaMalloc(&ctx->ws_counters, (size_t)(2 * items + 1) * sizeof(int32_t)) != cudaSuccess ||
+        cudaMemset(ctx->ws_counters, 0, (size_t)(2 * items + 1) * sizeof(int32_t)) != cudaSuccess)
+      return MLORA_ERR_CUDA;
+    ctx->ws_partial_items = part_items; ctx->ws_counter_items = items;
+  }
+  const int64_t groups = (int64_t)(h.fwd.grp2_adapter.size() > h.bwd.grp2_adapter.size() ? h.fwd.grp2_adapter.size()
+                                                                                        : h.bwd.grp2_adapter.size());
+  if (groups > ctx->ws_pbd_groups) {   // two chunk slots of [256][64] bf16 per adapter group of a tile
+    if (cudaDeviceSynchronize() != cudaSuccess) return MLORA_ERR_CUDA;
+    cudaFree(ctx->ws_pbd);
+    ctx->ws_pbd = nullptr; ctx->ws_pbd_groups = 0;
+    if (cudaMalloc(&ctx->ws_pbd, (size_t)groups * 2 * 256 * 64 * sizeof(__nv_bfloat16)) != cudaSuccess) return MLORA_ERR_CUDA;
+    ctx->ws_pbd_groups = groups;
+  }
+  return MLORA_OK;
+}
+
+}  // namespace
 
 mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, int32_t n_segs, int32_t n_rows,
                                  int32_t n_adapters, mlora_plan** out) {
@@ -766,77 +860,84 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
   if (ctx) {
     if (cudaSetDevice(ctx->device) != cudaSuccess) { delete p; return MLORA_ERR_CUDA; }
     BlobBuilder b;
-    const HostPlan& h = p->h;
-    size_t o[64]; int n = 0;
-    const RowSpace* rs[2] = {&h.fwd, &h.bwd};
-    for (int i = 0; i < 2; ++i) {
-      o[n++] = b.add(rs[i]->row_adapter); o[n++] = b.add(rs[i]->row_save); o[n++] = b.add(rs[i]->row_grp);
-      o[n++] = b.add(rs[i]->tile_grp_off); o[n++] = b.add(rs[i]->grp_adapter); o[n++] = b.add(rs[i]->item_rows);
-      o[n++] = b.add(rs[i]->row_grp2); o[n++] = b.add(rs[i]->tile2_grp_off); o[n++] = b.add(rs[i]->grp2_adapter);
-      o[n++] = b.add(rs[i]->zero_rows2);
-      o[n++] = b.add(rs[i]->item_save); o[n++] = b.add(rs[i]->item_start); o[n++] = b.add(rs[i]->item_desc); o[n++] = b.add(rs[i]->item_nrows); o[n++] = b.add(rs[i]->item_adapter);
-    }
-    o[n++] = b.add(h.slot_chunk_off); o[n++] = b.add(h.chunk_row0); o[n++] = b.add(h.chunk_nrows);
-    o[n++] = b.add(h.ft_adapters);
-    o[n++] = b.add(h.slot_blk_off); o[n++] = b.add(h.blk_row0); o[n++] = b.add(h.blk_nrows);
+    size_t o[kPlanTables];
+    pack_plan(p->h, b, o);
     if (cudaMalloc(&p->blob, b.data.size() * sizeof(int32_t)) != cudaSuccess) { delete p; return MLORA_ERR_CUDA; }
     if (cudaMemcpy(p->blob, b.data.data(), b.data.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
       cudaFree(p->blob); delete p; return MLORA_ERR_CUDA;
     }
-    DevRowSpace* ds[2] = {&p->fwd, &p->bwd};
-    n = 0;
-    for (int i = 0; i < 2; ++i) {
-      ds[i]->row_adapter = p->blob + o[n++]; ds[i]->row_save = p->blob + o[n++]; ds[i]->row_grp = p->blob + o[n++];
-      ds[i]->tile_grp_off = p->blob + o[n++]; ds[i]->grp_adapter = p->blob + o[n++]; ds[i]->item_rows = p->blob + o[n++];
-      ds[i]->row_grp2 = p->blob + o[n++]; ds[i]->tile2_grp_off = p->blob + o[n++]; ds[i]->grp2_adapter = p->blob + o[n++];
-      ds[i]->zero_rows2 = p->blob + o[n++];
-      ds[i]->item_save = p->blob + o[n++]; ds[i]->item_start = p->blob + o[n++]; ds[i]->item_desc = p->blob + o[n++]; ds[i]->item_nrows = p->blob + o[n++]; ds[i]->item_adapter = p->blob + o[n++];
-    }
-    p->bwd.row_save = nullptr;       // the compact space has no save offsets
-    p->slot_chunk_off = p->blob + o[n++]; p->chunk_row0 = p->blob + o[n++]; p->chunk_nrows = p->blob + o[n++];
-    p->slot_adapter = p->blob + o[n++];
-    p->slot_blk_off = p->blob + o[n++]; p->blk_row0 = p->blob + o[n++]; p->blk_nrows = p->blob + o[n++];
-    if (n_rows > ctx->ws_rows) {     // grow the rank-r workspace (the only other device allocation)
-      if (cudaDeviceSynchronize() != cudaSuccess) { cudaFree(p->blob); delete p; return MLORA_ERR_CUDA; }
-      cudaFree(ctx->ws_p);
-      ctx->ws_p = nullptr; ctx->ws_rows = 0;
-      if (cudaMalloc(&ctx->ws_p, (size_t)n_rows * kMaxRank * sizeof(float)) != cudaSuccess) {
-        cudaFree(p->blob); delete p; return MLORA_ERR_CUDA;
-      }
-      ctx->ws_rows = n_rows;
-    }
-    const int64_t items = h.fwd.n_items() > h.bwd.n_items() ? h.fwd.n_items() : h.bwd.n_items();
-    const int64_t part_items = items + 4 * ctx->sm_count;      // items * ksplit never exceeds this
-    if (part_items > ctx->ws_partial_items || items > ctx->ws_counter_items) {
-      if (cudaDeviceSynchronize() != cudaSuccess) { cudaFree(p->blob); delete p; return MLORA_ERR_CUDA; }
-      cudaFree(ctx->ws_partial); cudaFree(ctx->ws_counters);
-      ctx->ws_partial = nullptr; ctx->ws_counters = nullptr; ctx->ws_partial_items = ctx->ws_counter_items = 0;
-      if (cudaMalloc(&ctx->ws_partial, (size_t)part_items * kItemRows * kMaxRank * sizeof(float)) != cudaSuccess ||
-          cudaMalloc(&ctx->ws_counters, (size_t)(2 * items + 1) * sizeof(int32_t)) != cudaSuccess ||
-          cudaMemset(ctx->ws_counters, 0, (size_t)(2 * items + 1) * sizeof(int32_t)) != cudaSuccess) {
-        cudaFree(p->blob); delete p; return MLORA_ERR_CUDA;
-      }
-      ctx->ws_partial_items = part_items; ctx->ws_counter_items = items;
-    }
-    const int64_t groups = (int64_t)(h.fwd.grp2_adapter.size() > h.bwd.grp2_adapter.size() ? h.fwd.grp2_adapter.size()
-                                                                                          : h.bwd.grp2_adapter.size());
-    if (groups > ctx->ws_pbd_groups) {   // two chunk slots of [256][64] bf16 per adapter group of a tile
-      if (cudaDeviceSynchronize() != cudaSuccess) { cudaFree(p->blob); delete p; return MLORA_ERR_CUDA; }
-      cudaFree(ctx->ws_pbd);
-      ctx->ws_pbd = nullptr; ctx->ws_pbd_groups = 0;
-      if (cudaMalloc(&ctx->ws_pbd, (size_t)groups * 2 * 256 * 64 * sizeof(__nv_bfloat16)) != cudaSuccess) {
-        cudaFree(p->blob); delete p; return MLORA_ERR_CUDA;
-      }
-      ctx->ws_pbd_groups = groups;
-    }
+    bind_plan(p, o);
+    if ((s = grow_workspaces(ctx, p->h, n_rows)) != MLORA_OK) { cudaFree(p->blob); delete p; return s; }
   }
   *out = p;
   return MLORA_OK;
 }
 
+mlora_status_t mlora_plan_create_async(mlora_ctx* ctx, const mlora_segment_t* segs, int32_t n_segs, int32_t n_rows,
+                                       int32_t n_adapters, void* cuda_stream, mlora_plan** out) {
+  if (!out || !ctx) return MLORA_ERR_INVALID_ARG;
+  *out = nullptr;
+  mlora_plan* p = new (std::nothrow) mlora_plan();
+  if (!p) return MLORA_ERR_INVALID_ARG;
+  mlora_status_t s = build_plan(segs, n_segs, n_rows, n_adapters, p->h);
+  if (s != MLORA_OK) { delete p; return s; }
+  p->ctx = ctx;
+  if (cudaSetDevice(ctx->device) != cudaSuccess) { delete p; return MLORA_ERR_CUDA; }
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  BlobBuilder b;
+  size_t o[kPlanTables];
+  pack_plan(p->h, b, o);
+  const size_t need = b.data.size();
+  // a released buffer pair that is large enough and whose last user has passed its release point
+  for (size_t i = 0; i < ctx->plan_pool.size(); ++i) {
+    PlanBuf& c = ctx->plan_pool[i];
+    if (c.cap >= need && cudaEventQuery(c.free_evt) == cudaSuccess) {
+      p->buf = c;
+      ctx->plan_pool[i] = ctx->plan_pool.back();
+      ctx->plan_pool.pop_back();
+      break;
+    }
+  }
+  cudaGetLastError();                 // cudaEventQuery reports "not ready" through the error state
+  if (!p->buf.dev) {
+    size_t cap = 4096;
+    while (cap < need) cap *= 2;
+    if (cudaMalloc(&p->buf.dev, cap * sizeof(int32_t)) != cudaSuccess ||
+        cudaMallocHost(&p->buf.pinned, cap * sizeof(int32_t)) != cudaSuccess ||
+        cudaEventCreateWithFlags(&p->buf.free_evt, cudaEventDisableTiming) != cudaSuccess) {
+      free_plan_buf(p->buf); delete p; return MLORA_ERR_CUDA;
+    }
+    p->buf.cap = cap;
+  }
+  p->pooled = true;
+  p->blob = p->buf.dev;
+  std::memcpy(p->buf.pinned, b.data.data(), need * sizeof(int32_t));
+  if (cudaMemcpyAsync(p->blob, p->buf.pinned, need * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    free_plan_buf(p->buf); delete p; return MLORA_ERR_CUDA;
+  }
+  bind_plan(p, o);
+  if ((s = grow_workspaces(ctx, p->h, n_rows)) != MLORA_OK) { free_plan_buf(p->buf); delete p; return s; }
+  *out = p;
+  return MLORA_OK;
+}
+
+mlora_status_t mlora_plan_release(mlora_plan* p, void* cuda_stream) {
+  if (!p) return MLORA_OK;
+  if (!p->pooled || !p->ctx) { mlora_plan_destroy(p); return MLORA_OK; }
+  mlora_ctx* ctx = p->ctx;
+  if (cudaSetDevice(ctx->device) != cudaSuccess) return MLORA_ERR_CUDA;
+  if (cudaEventRecord(p->buf.free_evt, reinterpret_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return MLORA_ERR_CUDA;
+  if (ctx->plan_pool.size() < 64) ctx->plan_pool.push_back(p->buf);
+  else free_plan_buf(p->buf);        // (frees wait for the device: only when far more plans are released than reused)
+  delete p;
+  return MLORA_OK;
+}
+
 void mlora_plan_destroy(mlora_plan* p) {
   if (!p) return;
-  if (p->blob) { if (p->ctx) cudaSetDevice(p->ctx->device); cudaFree(p->blob); }
+  if (p->ctx) cudaSetDevice(p->ctx->device);
+  if (p->pooled) free_plan_buf(p->buf);
+  else if (p->blob) cudaFree(p->blob);
   delete p;
 }
 

@@ -188,6 +188,40 @@ def test_block_save_only_when_save_offsets_run_with_the_rows(sess):
         run_and_check(sess, w, synth.make_tensors(w), path=path, base=5, cap=5 + 291 + 9)
 
 
+def test_stream_ordered_plans_from_the_pool(sess):
+    """Plans created and released on a stream, step after step (buffers come back from the pool while
+    earlier steps may still be running): every step's outputs equal those of an ordinary plan."""
+    w0 = synth.random_workload(90, 256, 320, 16, 5, 600, max_seg=100, p_finetune=0.3)
+    t = synth.make_tensors(w0)
+    run = LayerRun(sess, "bf16", t, w0.segments, w0.n_rows, save_capacity_rows=700)
+    outs, tables = [], []
+    try:
+        for step in range(12):
+            w = synth.random_workload(100 + step, 256, 320, 16, 5, 200 + 31 * step, max_seg=60 + 5 * step, p_finetune=0.3)
+            plan = mb.mlora_plan_create_async(sess.ctx, w.segments, w.n_rows, 5)
+            y = torch.zeros((w.n_rows, 320), dtype=torch.bfloat16, device=sess.device)
+            mb.mlora_mixed_forward(sess.ctx, run.layer, plan, run.X, y, run.x_save, run.u_save, 0, run.capacity)
+            mb.mlora_plan_release(plan)
+            outs.append(y)
+            tables.append(w)
+        torch.cuda.synchronize()
+        assert run.status() == mb.MLORA_OK
+        for y, w in zip(outs, tables):
+            plan = mb.mlora_plan_create(sess.ctx, w.segments, w.n_rows, 5)
+            y2 = torch.zeros_like(y)
+            mb.mlora_mixed_forward(sess.ctx, run.layer, plan, run.X, y2, run.x_save, run.u_save, 0, run.capacity)
+            torch.cuda.synchronize()
+            mb.mlora_plan_destroy(plan)
+            assert torch.equal(y, y2)
+        ref = orc.forward(t["X"][:tables[3].n_rows], t["W"], t["A_all"], t["B_all"], t["scale"], tables[3].segments)
+        assert_close("Y", run.host(outs[3]), ref["Y"], TOL["bf16"])
+        # a pooled plan may also be destroyed the ordinary way
+        plan = mb.mlora_plan_create_async(sess.ctx, w0.segments, w0.n_rows, 5)
+        mb.mlora_plan_destroy(plan)
+    finally:
+        run.close()
+
+
 def test_base_only_rows_and_no_finetune(sess):
     segs = [(0, 40, -1, 0), (60, 30, 1, 0)]      # rows 40..59 and 90..99 uncovered
     w = synth.Workload("base_only", 192, 256, 16, 2, "bf16", 100, synth.segments_array(segs))
