@@ -222,6 +222,14 @@ def test_stream_ordered_plans_from_the_pool(sess):
         run.close()
 
 
+def test_many_rows_many_adapters(sess):
+    """16384 rows (64 pair tiles), 96 adapters, 5000 fine-tuning rows in ragged segments: the workspaces grow,
+    tables and counters stay in range."""
+    w = synth.random_workload(123, 1024, 768, 16, 96, 16384, max_seg=700, p_finetune=0.3)
+    assert w.ft_rows > 3000
+    run_and_check(sess, w, synth.make_tensors(w), blocked=True)
+
+
 def test_base_only_rows_and_no_finetune(sess):
     segs = [(0, 40, -1, 0), (60, 30, 1, 0)]      # rows 40..59 and 90..99 uncovered
     w = synth.Workload("base_only", 192, 256, 16, 2, "bf16", 100, synth.segments_array(segs))
