@@ -123,6 +123,19 @@ __device__ __forceinline__ bool gemm2_wait(uint32_t bar, uint32_t parity, volati
   return false;
 }
 
+// Tile order: m-fastest inside bands of `group_m` row tiles (all row tiles when group_m == 0), so
+// that the tiles in flight at one time cover a near-square block of the output and the operand
+// panels they stream together are as few as possible.
+__device__ __forceinline__ void gemm2_tile(const GemmArgs& args, int tile, int& mt, int& nt) {
+  const int gm_full = args.group_m > 0 ? args.group_m : args.n_mtiles;
+  const int band_tiles = gm_full * args.n_ntiles;
+  const int band = tile / band_tiles, r = tile - band * band_tiles;
+  const int left = args.n_mtiles - band * gm_full;
+  const int gm = left < gm_full ? left : gm_full;
+  mt = band * gm_full + r % gm;
+  nt = r / gm;
+}
+
 // args: n_mtiles counts 256-row pair tiles, n_ntiles 256-column tiles, n_units = their product;
 // row_grp / tile_grp_off / grp_adapter are the tables for 256-row tiles.
 template <int R, bool W_KMAJOR>
@@ -205,7 +218,8 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
     bool ok = true;
     for (int unit = pair; unit < n_units && ok; unit += n_pairs) {
       const int tile = unit % n_tiles, ks = unit / n_tiles;
-      const int mt = tile % args.n_mtiles, nt = tile / args.n_mtiles;
+      int mt, nt;
+      gemm2_tile(args, tile, mt, nt);
       const int m0 = mt * GEMM2_BM + (int)rank * 128;
       const int nh = nt * GEMM2_BN + (int)rank * 128;     // this CTA's half of the B columns
       const int G = ks == SK - 1 ? tile_groups(mt) : 0;   // the low-rank blocks ride with the last K slice
@@ -278,7 +292,8 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
       bool ok = true;
       for (int unit = pair; unit < n_units && ok; unit += n_pairs, ++lt) {
         const int tile = unit % n_tiles, ks = unit / n_tiles;
-        const int mt = tile % args.n_mtiles;
+        int mt, nt_unused;
+        gemm2_tile(args, tile, mt, nt_unused);
         const int kb_begin = (int)((long long)ks * KB / SK), kb_end = (int)((long long)(ks + 1) * KB / SK);
         const uint32_t buf = lt & 1;
         if (!(ok = gemm2_wait(bar_tempty(buf), ((lt >> 1) & 1) ^ 1, abort_flag, args.status))) break;
@@ -331,7 +346,8 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
     bool ok = true;
     for (int unit = pair; unit < n_units && ok; unit += n_pairs, ++lt) {
       const int tile = unit % n_tiles, ks = unit / n_tiles;
-      const int mt = tile % args.n_mtiles, nt = tile / args.n_mtiles;
+      int mt, nt;
+      gemm2_tile(args, tile, mt, nt);
       const int m0 = mt * GEMM2_BM + (int)rank * 128 + e * 32, n0 = nt * GEMM2_BN;
       const uint32_t buf = lt & 1;
       if (!(ok = gemm2_wait(bar_tfull(buf), (lt >> 1) & 1, abort_flag, args.status))) break;

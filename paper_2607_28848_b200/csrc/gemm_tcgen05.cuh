@@ -50,6 +50,7 @@ struct GemmArgs {
   int32_t n_full;                // work units [0, n_full) are whole 128 x 256 tiles; the tiles after
   int32_t n_units;               // them (the last, partly filled wave) are cut into two 128 x 128 halves
   int32_t lora_enabled;
+  int32_t group_m;               // two-SM kernel only: row tiles per band of the tile order (0: one band)
   int32_t split_k;               // two-SM kernel only: K slices per tile (1: none); slice-major unit order
   float* ws_splitk;              // [split_k, M, N] fp32 partial products when split_k > 1
   const int32_t* row_grp;        // [M] group of the row inside its 128-row tile, -1: none
