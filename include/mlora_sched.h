@@ -102,6 +102,19 @@ void mlora_sched_destroy(mlora_sched_t* s);
 mlora_status_t mlora_sched_set_coef(mlora_sched_t* s, const mlora_mixed_coef_t* graph,
                                     const mlora_mixed_coef_t* eager, const mlora_decode_coef_t* decode);
 
+/* Online refinement (Section 4.2, estimator calibration: the estimator keeps refitting each execution
+ * mode from the step times the host reports).  mlora_sched_observe stores one observed step
+ * (composition as in mlora_observation_t, prefill_lens copied) in the ring of its mode - 0 eager,
+ * 1 graph - which keeps the most recent `MLORA_SCHED_RING` (512) observations per mode.
+ * mlora_sched_refit fits Eq. I to the ring of `mode` with mlora_fit_mixed(fit_mask) and, when the fit
+ * succeeds, installs the result as that mode's coefficient set (coefficients outside fit_mask keep
+ * their current values); *out (may be NULL) receives the installed set.  Errors: those of
+ * mlora_fit_mixed (the set is left unchanged), MLORA_ERR_INVALID_ARG for a bad mode. */
+#define MLORA_SCHED_RING 512
+mlora_status_t mlora_sched_observe(mlora_sched_t* s, int32_t mode, const mlora_observation_t* obs);
+int32_t mlora_sched_observations(const mlora_sched_t* s, int32_t mode);
+mlora_status_t mlora_sched_refit(mlora_sched_t* s, int32_t mode, uint32_t fit_mask, mlora_mixed_coef_t* out);
+
 /* Adds a fine-tuning sample of `tokens` (> 0) tokens to the pool Q_ft.  Ids are the caller's;
  * a duplicate id in the pool is MLORA_ERR_INVALID_ARG. */
 mlora_status_t mlora_sched_pool_add(mlora_sched_t* s, int64_t sample_id, int32_t tokens);

@@ -27,8 +27,17 @@ double attn_term(int32_t n, int32_t n_decode) {
 
 }  // namespace
 
+struct StoredObs {
+  std::vector<int32_t> lens;
+  int32_t n_decode;
+  int64_t kv_tokens, ft_tokens;
+  double seconds;
+};
+
 struct mlora_sched {
   mlora_sched_config_t cfg;
+  std::vector<StoredObs> ring[2];       // observed steps per execution mode (0 eager, 1 graph)
+  size_t ring_next[2] = {0, 0};
   std::vector<PoolEntry> pool;
   int64_t reserved = 0;
   uint64_t next_seq = 0;
@@ -138,6 +147,46 @@ mlora_status_t mlora_sched_set_coef(mlora_sched_t* s, const mlora_mixed_coef_t* 
   if (graph) s->cfg.graph = *graph;
   if (eager) s->cfg.eager = *eager;
   if (decode) s->cfg.decode = *decode;
+  return MLORA_OK;
+}
+
+mlora_status_t mlora_sched_observe(mlora_sched_t* s, int32_t mode, const mlora_observation_t* obs) {
+  if (!s || !obs || mode < 0 || mode > 1 || obs->n_prefill < 0 || (obs->n_prefill > 0 && !obs->prefill_lens))
+    return MLORA_ERR_INVALID_ARG;
+  StoredObs o;
+  o.lens.assign(obs->prefill_lens, obs->prefill_lens + obs->n_prefill);
+  o.n_decode = obs->n_decode; o.kv_tokens = obs->kv_tokens; o.ft_tokens = obs->ft_tokens; o.seconds = obs->seconds;
+  std::vector<StoredObs>& r = s->ring[mode];
+  if (r.size() < MLORA_SCHED_RING) {
+    r.push_back(std::move(o));
+  } else {
+    r[s->ring_next[mode]] = std::move(o);
+    s->ring_next[mode] = (s->ring_next[mode] + 1) % MLORA_SCHED_RING;
+  }
+  return MLORA_OK;
+}
+
+int32_t mlora_sched_observations(const mlora_sched_t* s, int32_t mode) {
+  return (s && mode >= 0 && mode <= 1) ? (int32_t)s->ring[mode].size() : -1;
+}
+
+mlora_status_t mlora_sched_refit(mlora_sched_t* s, int32_t mode, uint32_t fit_mask, mlora_mixed_coef_t* out) {
+  if (!s || mode < 0 || mode > 1) return MLORA_ERR_INVALID_ARG;
+  const std::vector<StoredObs>& r = s->ring[mode];
+  std::vector<mlora_observation_t> obs(r.size());
+  for (size_t i = 0; i < r.size(); ++i)
+    obs[i] = mlora_observation_t{r[i].lens.empty() ? nullptr : r[i].lens.data(), (int32_t)r[i].lens.size(), r[i].n_decode,
+                                 r[i].kv_tokens, r[i].ft_tokens, r[i].seconds};
+  mlora_mixed_coef_t fit;
+  const mlora_status_t st = mlora_fit_mixed(obs.empty() ? nullptr : obs.data(), (int32_t)obs.size(), fit_mask, &fit);
+  if (st != MLORA_OK) return st;
+  mlora_mixed_coef_t& cur = mode == 1 ? s->cfg.graph : s->cfg.eager;
+  if (fit_mask & 1u) cur.alpha = fit.alpha;
+  if (fit_mask & 2u) cur.beta = fit.beta;
+  if (fit_mask & 4u) cur.gamma = fit.gamma;
+  if (fit_mask & 8u) cur.eps = fit.eps;
+  if (fit_mask & 16u) cur.c = fit.c;
+  if (out) *out = cur;
   return MLORA_OK;
 }
 

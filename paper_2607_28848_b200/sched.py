@@ -13,8 +13,10 @@ EXPORTS = (
     "mlora_predict_mixed", "mlora_predict_decode", "mlora_ttft_budget", "mlora_fit_mixed",
     "mlora_sched_create", "mlora_sched_destroy", "mlora_sched_set_coef", "mlora_sched_pool_add",
     "mlora_sched_pool_size", "mlora_sched_buffer_left", "mlora_sched_set_backward_running",
-    "mlora_sched_admit", "mlora_sched_requeue", "mlora_sched_buffer_release",
+    "mlora_sched_admit", "mlora_sched_requeue", "mlora_sched_buffer_release", "mlora_sched_observe",
+    "mlora_sched_observations", "mlora_sched_refit",
 )
+MODE_EAGER, MODE_GRAPH = 0, 1
 FIT_ALPHA, FIT_BETA, FIT_GAMMA, FIT_EPS, FIT_C = 1, 2, 4, 8, 16
 
 
@@ -82,6 +84,12 @@ def _lib() -> ctypes.CDLL:
     lib.mlora_sched_requeue.restype = ctypes.c_int
     lib.mlora_sched_buffer_release.argtypes = [vp, i64]
     lib.mlora_sched_buffer_release.restype = ctypes.c_int
+    lib.mlora_sched_observe.argtypes = [vp, i32, P(mlora_observation_t)]
+    lib.mlora_sched_observe.restype = ctypes.c_int
+    lib.mlora_sched_observations.argtypes = [vp, i32]
+    lib.mlora_sched_observations.restype = i32
+    lib.mlora_sched_refit.argtypes = [vp, i32, ctypes.c_uint32, P(mlora_mixed_coef_t)]
+    lib.mlora_sched_refit.restype = ctypes.c_int
     _ready = True
     return lib
 
@@ -188,3 +196,20 @@ def mlora_sched_requeue(s, ids: Sequence[int], tokens: Sequence[int]) -> None:
 
 def mlora_sched_buffer_release(s, tokens: int) -> None:
     _b._check(_lib().mlora_sched_buffer_release(s, int(tokens)), "mlora_sched_buffer_release")
+
+
+def mlora_sched_observe(s, mode: int, prefill_lens: Sequence[int], n_decode: int, kv_tokens: int, ft_tokens: int,
+                        seconds: float) -> None:
+    arr = _i32_array(prefill_lens)
+    obs = mlora_observation_t(arr, len(prefill_lens), int(n_decode), int(kv_tokens), int(ft_tokens), float(seconds))
+    _b._check(_lib().mlora_sched_observe(s, int(mode), ctypes.byref(obs)), "mlora_sched_observe")
+
+
+def mlora_sched_observations(s, mode: int) -> int:
+    return int(_lib().mlora_sched_observations(s, int(mode)))
+
+
+def mlora_sched_refit(s, mode: int, fit_mask: int = 31) -> mlora_mixed_coef_t:
+    out = mlora_mixed_coef_t()
+    _b._check(_lib().mlora_sched_refit(s, int(mode), int(fit_mask), ctypes.byref(out)), "mlora_sched_refit")
+    return out

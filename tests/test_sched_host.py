@@ -155,3 +155,34 @@ def test_predictors_reject_null():
     assert math.isnan(lib.mlora_predict_mixed(None, None, 0, 0, 0, 0))
     assert math.isnan(lib.mlora_predict_decode(None, 1, 1))
     assert ms.mlora_predict_decode(ms.decode_coef(*DEC), 7, 300) == pytest.approx(0.02 * 7 + 1e-4 * 300 + 0.5)
+
+
+def test_online_refit_tracks_a_drift_and_changes_admission():
+    """Observed steps go into a ring per execution mode; a refit installs the new coefficients, and the
+    admission that follows prices batches with them."""
+    s = make(10 ** 6)
+    try:
+        rng = np.random.default_rng(5)
+        slow = so.MixedCoef(0.0, 0.004, 0.001, 0.0, 0.3)           # the eager path got 40% slower per token
+        obs = []
+        for _ in range(700):                                         # more than the ring holds
+            lens = rng.integers(16, 900, rng.integers(1, 4)).tolist()
+            bd, tft = int(rng.integers(0, 64)), int(rng.integers(0, 1024))
+            t = so.predict_mixed(slow, lens, bd, 0, tft)
+            obs.append((lens, bd, 0, tft, t))
+            ms.mlora_sched_observe(s, ms.MODE_EAGER, lens, bd, 0, tft, t)
+        assert ms.mlora_sched_observations(s, ms.MODE_EAGER) == 512 and ms.mlora_sched_observations(s, ms.MODE_GRAPH) == 0
+        with pytest.raises(mb.MloraError):
+            ms.mlora_sched_refit(s, ms.MODE_GRAPH)                   # nothing observed in that mode
+        got = ms.mlora_sched_refit(s, ms.MODE_EAGER, ms.FIT_ALPHA | ms.FIT_BETA | ms.FIT_GAMMA | ms.FIT_C)
+        ref = so.fit_mixed(obs[-512:])                                # the ring keeps the most recent 512
+        assert got.beta == pytest.approx(0.004, rel=1e-9) and got.gamma == pytest.approx(0.001, rel=1e-9)
+        assert got.c == pytest.approx(0.3, rel=1e-9) and got.beta == pytest.approx(ref.beta, rel=1e-6)
+        assert abs(got.alpha) < 1e-12 and got.eps == EAGER[3]        # eps is outside the mask: unchanged
+        for i in range(6):
+            ms.mlora_sched_pool_add(s, i, 100)
+        # budget 2.0: inference 0.3 + 0.004 * 200 = 1.1; a sample costs 100 * (0.004 + 0.001) = 0.5 -> one fits
+        ids, _, _ = ms.mlora_sched_admit(s, [200], 0, 0, t_now=398.0, earliest_arrival=0.0)
+        assert len(ids) == 1
+    finally:
+        ms.mlora_sched_destroy(s)
