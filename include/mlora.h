@@ -23,6 +23,10 @@
  *    given stream, allocate nothing and never synchronise.
  *  - There is no CPU fallback: without an sm_100 device mlora_create fails with
  *    MLORA_ERR_ARCH and no compute entry point can be used.
+ *  - A context owns workspaces (the rank-r intermediate of the running call, the GEMM's low-rank
+ *    operand, partial sums) that serve ONE compute call at a time: the calls on a context must be
+ *    queued on one stream, or on streams ordered after one another.  A context is used from one
+ *    host thread at a time; different contexts (one per GPU, or several on one) are independent.
  *  - The library never aborts the process and throws nothing across this boundary.
  */
 #ifndef MLORA_H_
