@@ -319,13 +319,16 @@ def main():
     if "gemm_fwd" in per_kind:
         kernels["gemm_fwd"] = {**per_kind["gemm_fwd"], "tflops": gemm_fwd_flops / per_kind["gemm_fwd"]["ms_per_step"] / 1e9}
     if "gemm_bwd" in per_kind:
-        kernels["gemm_bwd"] = {**per_kind["gemm_bwd"], "tflops": gemm_bwd_flops / per_kind["gemm_bwd"]["ms_per_step"] / 1e9}
+        kernels["gemm_bwd"] = {**per_kind["gemm_bwd"], "tflops": gemm_bwd_flops / per_kind["gemm_bwd"]["ms_per_step"] / 1e9,
+                               "frac_of_sustained": gemm_bwd_flops / per_kind["gemm_bwd"]["ms_per_step"] / 1e9 / peaks["bf16_tflops_sustained"]}
     if "shrink" in per_kind:
         b = sum(a["shrink_fwd"] + a["shrink_bwd"] for a in ab)
-        kernels["shrink"] = {**per_kind["shrink"], "gbs": b / per_kind["shrink"]["ms_per_step"] / 1e6}
+        kernels["shrink"] = {**per_kind["shrink"], "gbs": b / per_kind["shrink"]["ms_per_step"] / 1e6,
+                             "frac_hbm": b / per_kind["shrink"]["ms_per_step"] / 1e6 / peaks["hbm_gbs"]}
     if "grad" in per_kind:
         b = sum(a["grad_dA"] + a["grad_dB"] for a in ab)
-        kernels["grad"] = {**per_kind["grad"], "gbs": b / per_kind["grad"]["ms_per_step"] / 1e6}
+        kernels["grad"] = {**per_kind["grad"], "gbs": b / per_kind["grad"]["ms_per_step"] / 1e6,
+                           "frac_hbm": b / per_kind["grad"]["ms_per_step"] / 1e6 / peaks["hbm_gbs"]}
     if "adamw" in per_kind:
         b = sum(30.0 * len(r.slots) * w.rank * (w.d_in + w.d_out) for r, w in zip(runs, workloads))
         kernels["adamw"] = {**per_kind["adamw"], "gbs": b / per_kind["adamw"]["ms_per_step"] / 1e6,
