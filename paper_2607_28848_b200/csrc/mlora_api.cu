@@ -6,6 +6,7 @@
 
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -125,6 +126,13 @@ struct BlobBuilder {
 constexpr size_t kSplitKBytes = 64u << 20;
 constexpr int kMaxDevices = 64;      // device ordinals a process may create contexts on
 
+// With MLORA_DEBUG set in the environment, the place and the runtime's message of a failed CUDA call go to stderr.
+mlora_status_t cuda_failure(const char* site, const char* detail) {
+  static const bool verbose = std::getenv("MLORA_DEBUG") != nullptr;
+  if (verbose) std::fprintf(stderr, "mlora: CUDA failure at %s: %s\n", site, detail ? detail : "");
+  return MLORA_ERR_CUDA;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 mlora_status_t make_tmap_bf16(const mlora_ctx* ctx, CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer,
@@ -136,7 +144,14 @@ mlora_status_t make_tmap_bf16(const mlora_ctx* ctx, CUtensorMap* m, const void* 
   CUresult r = ctx->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? MLORA_OK : MLORA_ERR_CUDA;
+  if (r != CUDA_SUCCESS) {
+    char msg[160];
+    std::snprintf(msg, sizeof msg, "code %d, dims %llu x %llu, row stride %llu, box %u x %u, base %p", (int)r,
+                  (unsigned long long)inner, (unsigned long long)outer, (unsigned long long)row_stride_elems, box_inner,
+                  box_outer, base);
+    return cuda_failure("tensor map (2-D)", msg);
+  }
+  return MLORA_OK;
 }
 
 // [rows, cols] (cols contiguous, a multiple of 64) seen as (64, rows, cols / 64): a box of
@@ -151,7 +166,14 @@ mlora_status_t make_tmap_bf16_blocked(const mlora_ctx* ctx, CUtensorMap* m, cons
   CUresult r = ctx->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? MLORA_OK : MLORA_ERR_CUDA;
+  if (r != CUDA_SUCCESS) {
+    char msg[160];
+    std::snprintf(msg, sizeof msg, "code %d, rows %llu, cols %llu, row stride %llu, box rows %u, blocks %u, base %p", (int)r,
+                  (unsigned long long)rows, (unsigned long long)cols, (unsigned long long)row_stride_elems, box_rows,
+                  box_blocks, base);
+    return cuda_failure("tensor map (blocked)", msg);
+  }
+  return MLORA_OK;
 }
 
 bool rank_ok_bf16(int r) { return r == 8 || r == 16 || r == 32 || r == 64 || r == 128; }
@@ -184,7 +206,8 @@ struct LaunchScope {
   mlora_status_t done() {
     if (slot >= 0) cudaEventRecord(ctx->ev_stop[slot], st);
     ctx->launches++;
-    return cudaGetLastError() == cudaSuccess ? MLORA_OK : MLORA_ERR_CUDA;
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? MLORA_OK : cuda_failure("kernel launch", cudaGetErrorString(e));
   }
 };
 
@@ -977,6 +1000,9 @@ mlora_status_t mlora_mixed_forward(mlora_ctx* ctx, const mlora_layer_t* L, const
     if (!u_save) return MLORA_ERR_INVALID_ARG;
   }
   if (h.n_rows > ctx->ws_rows) return MLORA_ERR_INVALID_ARG;
+  // the tensor maps are encoded through the driver API, which needs this device's context current on the
+  // calling thread (a framework's worker threads do not always have one)
+  if (cudaSetDevice(ctx->device) != cudaSuccess) return MLORA_ERR_CUDA;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (L->dtype == MLORA_F32)
     return forward_simt<float>(ctx, L, p, X, ldx, Y, ldy, x_save, u_save, save_row_base, st);
@@ -1010,6 +1036,9 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   if (h.n_adapters > L->n_adapters) return MLORA_ERR_ADAPTER_ID;
   if (h.ft_rows == 0) return MLORA_OK;
   if (!dY || !x_save || !u_save || !dA || !dB || lddy < L->d_out || (dX && lddx < L->d_in)) return MLORA_ERR_INVALID_ARG;
+  // the tensor maps are encoded through the driver API, which needs this device's context current on the
+  // calling thread (a framework's worker threads do not always have one)
+  if (cudaSetDevice(ctx->device) != cudaSuccess) return MLORA_ERR_CUDA;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (L->dtype == MLORA_F32)
     return backward_simt<float>(ctx, L, p, dY, lddy, x_save, u_save, dA, dB, dX, lddx, accumulate, st);
@@ -1083,6 +1112,7 @@ mlora_status_t mlora_adamw_update(mlora_ctx* ctx, const mlora_layer_t* L, const 
   a.inv_bc1 = (float)(1.0 / (1.0 - pow((double)hp->beta1, (double)hp->step)));
   a.inv_bc2 = (float)(1.0 / (1.0 - pow((double)hp->beta2, (double)hp->step)));
   if (cancelled(ctx)) return MLORA_CANCELLED;
+  if (cudaSetDevice(ctx->device) != cudaSuccess) return MLORA_ERR_CUDA;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   const int64_t widest = (int64_t)n_slots * L->rank * (L->d_in > L->d_out ? L->d_in : L->d_out) / 4;
   int blocks = (int)((widest + 255) / 256);

@@ -1,0 +1,167 @@
+"""One decoder layer chained through the library's projections, with the paper's default activation
+policy (Section 3.2): the serving forward keeps only the layer's residual-stream input for the
+fine-tuning rows; the backward recomputes the layer from it, over the fine-tuning rows alone, and
+returns the LoRA gradients of all seven projections and the gradient of the layer input (what the
+layer below needs).
+
+Division of labour: the seven projections (q, k, v, o, gate, up, down) run in this library's kernels
+- `mlora_mixed_forward` in the serving pass, `mlora_mixed_forward` + `mlora_backward` in the
+recompute/backward pass.  Everything between them (RMSNorm, rotary embedding, attention, SiLU gate,
+residual adds) and the chain rule through those pieces are PyTorch library calls: they are glue here,
+not kernels of this library.  A decode row is a one-token sequence (no KV cache in this module).
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, List, Sequence, Tuple
+
+import numpy as np
+import torch
+
+from . import binding as mb
+from . import synth
+
+PROJ = ("q", "k", "v", "o", "gate", "up", "down")
+
+
+class _Projection:
+    def __init__(self, sess, W, A_all, B_all, scale, cap_rows):
+        dev = sess.device
+        self.W, self.A, self.B = (t.to(dev).to(torch.bfloat16).contiguous() for t in (W, A_all, B_all))
+        self.scale = scale.to(dev).to(torch.float32).contiguous()
+        self.layer = mb.make_layer(self.W, self.A, self.B, self.scale)
+        self.d_in, self.d_out, self.rank = self.W.shape[0], self.W.shape[1], self.A.shape[1]
+        self.x_save = torch.empty((cap_rows, self.d_in), dtype=torch.bfloat16, device=dev)
+        self.u_save = torch.empty((cap_rows, self.rank), dtype=torch.float32, device=dev)
+        self.dA = self.dB = None
+
+
+class _ProjFn(torch.autograd.Function):
+    """A multi-LoRA projection over a batch whose rows are all fine-tuning rows (the recompute pass)."""
+
+    @staticmethod
+    def forward(ctx, x, owner, name):
+        pr = owner.proj[name]
+        x = x.contiguous()
+        y = torch.empty((x.shape[0], pr.d_out), dtype=torch.bfloat16, device=x.device)
+        mb.mlora_mixed_forward(owner.sess.ctx, pr.layer, owner.bwd_plan, x, y, pr.x_save, pr.u_save, 0, pr.x_save.shape[0])
+        ctx.owner, ctx.name = owner, name
+        return y
+
+    @staticmethod
+    def backward(ctx, dy):
+        owner, pr = ctx.owner, ctx.owner.proj[ctx.name]
+        dy = dy.to(torch.bfloat16).contiguous()
+        n_slots = len(owner.bwd_slots)
+        pr.dA = torch.empty((n_slots, pr.rank, pr.d_in), dtype=torch.float32, device=dy.device)
+        pr.dB = torch.empty((n_slots, pr.rank, pr.d_out), dtype=torch.float32, device=dy.device)
+        dx = torch.empty((dy.shape[0], pr.d_in), dtype=torch.bfloat16, device=dy.device)
+        mb.mlora_backward(owner.sess.ctx, pr.layer, owner.bwd_plan, dy, pr.x_save, pr.u_save, pr.dA, pr.dB, dx)
+        return dx, None, None
+
+
+def _rmsnorm(x, gain, eps=1e-5):
+    xf = x.float()
+    return (xf * torch.rsqrt((xf * xf).mean(-1, keepdim=True) + eps) * gain).to(torch.bfloat16)
+
+
+def _rope(x, pos, theta=500000.0):
+    d = x.shape[-1]
+    half = d // 2
+    inv = theta ** (-torch.arange(0, half, dtype=torch.float32, device=x.device) * 2.0 / d)
+    ang = pos.float()[:, None] * inv[None, :]
+    cos, sin = torch.cos(ang)[:, None, :], torch.sin(ang)[:, None, :]
+    xf = x.float()
+    x1, x2 = xf[..., :half], xf[..., half:]
+    return torch.cat([x1 * cos - x2 * sin, x2 * cos + x1 * sin], dim=-1).to(torch.bfloat16)
+
+
+class DecoderLayer:
+    def __init__(self, sess, params: Dict[str, torch.Tensor], n_heads: int, n_kv: int, max_ft_rows: int):
+        """params as in the layer oracle: g1, g2, and W_p / A_p / B_p / s_p for the seven projections."""
+        self.sess, self.n_heads, self.n_kv = sess, n_heads, n_kv
+        dev = sess.device
+        self.g1, self.g2 = params["g1"].to(dev).float(), params["g2"].to(dev).float()
+        self.proj = {n: _Projection(sess, params["W_" + n], params["A_" + n], params["B_" + n], params["s_" + n], max_ft_rows)
+                     for n in PROJ}
+        self.n_adapters = params["A_q"].shape[0]
+        self.d = params["W_q"].shape[0]
+        self.saved_x = torch.empty((max_ft_rows, self.d), dtype=torch.bfloat16, device=dev)   # the layer-input buffer
+        self.saved: List[Tuple[int, int]] = []      # (tokens, adapter) of the saved fine-tuning sequences, in save order
+        self.saved_rows = 0
+        self.bwd_plan, self.bwd_slots = None, []
+
+    # -- shared layer body; `lin(name, x)` is the projection call ---------------------------------
+    def _body(self, x, lin, sequences):
+        T = x.shape[0]
+        dh = self.d // self.n_heads
+        pos = torch.zeros(T, dtype=torch.long, device=x.device)
+        for start, n in sequences:
+            pos[start:start + n] = torch.arange(n, device=x.device)
+        h1 = _rmsnorm(x, self.g1)
+        q = _rope(lin("q", h1).reshape(T, self.n_heads, dh), pos)
+        k = _rope(lin("k", h1).reshape(T, self.n_kv, dh), pos)
+        v = lin("v", h1).reshape(T, self.n_kv, dh)
+        rep = self.n_heads // self.n_kv
+        outs = []
+        for start, n in sequences:                  # causal attention inside each sequence (library call)
+            qs = q[start:start + n].transpose(0, 1)[None]
+            ks = k[start:start + n].repeat_interleave(rep, dim=1).transpose(0, 1)[None]
+            vs = v[start:start + n].repeat_interleave(rep, dim=1).transpose(0, 1)[None]
+            o = torch.nn.functional.scaled_dot_product_attention(qs, ks, vs, is_causal=True)
+            outs.append(o[0].transpose(0, 1).reshape(n, self.d))
+        a = torch.cat(outs, dim=0)
+        x2 = x + lin("o", a)
+        h2 = _rmsnorm(x2, self.g2)
+        m = torch.nn.functional.silu(lin("gate", h2).float()).to(torch.bfloat16) * lin("up", h2)
+        return x2 + lin("down", m)
+
+    # -- serving forward: mixed batch, keeps the layer input of the fine-tuning rows --------------
+    @torch.no_grad()
+    def forward(self, x, segments: np.ndarray) -> torch.Tensor:
+        """segments cover the batch contiguously in row order (every segment is one sequence)."""
+        segs = np.asarray(segments, dtype=np.int32).reshape(-1, 4)
+        n_rows = x.shape[0]
+        serving = segs.copy()
+        serving[:, 3] = 0                           # projection-level saves are not kept: the policy saves the layer input
+        plan = mb.mlora_plan_create(self.sess.ctx, serving, n_rows, self.n_adapters)
+        try:
+            def lin(name, inp):
+                pr = self.proj[name]
+                y = torch.empty((n_rows, pr.d_out), dtype=torch.bfloat16, device=x.device)
+                mb.mlora_mixed_forward(self.sess.ctx, pr.layer, plan, inp.contiguous(), y, None, None, 0, 0)
+                return y
+            y = self._body(x, lin, [(int(s), int(n)) for s, n, _, _ in segs if n > 0])
+        finally:
+            torch.cuda.synchronize()
+            mb.mlora_plan_destroy(plan)
+        for s, n, a, ft in segs:                    # activation capture: the residual-stream input of fine-tuning rows
+            if ft and n > 0:
+                self.saved_x[self.saved_rows:self.saved_rows + n] = x[s:s + n]
+                self.saved.append((int(n), int(a)))
+                self.saved_rows += int(n)
+        return y
+
+    # -- backward: recompute from the saved layer input, fine-tuning rows only ---------------------
+    def backward(self, dy_ft: torch.Tensor):
+        """dy_ft [saved rows, d]: gradient of the layer output for the saved rows, in save order.
+        Returns (dx [saved rows, d], {projection: (dA, dB)}, adapters of the gradient slots)."""
+        rows = self.saved_rows
+        table, row = [], 0
+        for n, a in self.saved:
+            table.append((row, n, a, 1)); row += n
+        table = synth.segments_array(table)
+        self.bwd_plan = mb.mlora_plan_create(self.sess.ctx, table, rows, self.n_adapters)
+        self.bwd_slots = mb.mlora_plan_ft_adapters(self.bwd_plan)
+        try:
+            x = self.saved_x[:rows].clone().requires_grad_(True)
+            with torch.enable_grad():
+                y = self._body(x, lambda name, inp: _ProjFn.apply(inp, self, name), [(int(s), int(n)) for s, n, _, _ in table])
+                y.backward(dy_ft.to(torch.bfloat16))
+            torch.cuda.synchronize()
+            grads = {n: (self.proj[n].dA, self.proj[n].dB) for n in PROJ}
+            return x.grad, grads, list(self.bwd_slots)
+        finally:
+            mb.mlora_plan_destroy(self.bwd_plan)
+            self.bwd_plan = None
+            self.saved, self.saved_rows = [], 0

@@ -1,0 +1,73 @@
+"""A decoder layer chained through the library's projections against the fp64 layer oracle: the mixed
+serving forward, then the backward that recomputes the layer from the saved layer input."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import layer_oracle as lo
+from paper_2607_28848_b200 import binding as mb
+from paper_2607_28848_b200 import synth
+from paper_2607_28848_b200.layer import DecoderLayer, PROJ
+from paper_2607_28848_b200.runner import Session
+
+pytestmark = pytest.mark.gpu
+
+
+def bf16(t):
+    return t.to(torch.bfloat16).to(torch.float64)
+
+
+def test_layer_forward_and_recompute_backward_match_the_oracle():
+    d, ffn, r, n_ad, H, Hkv = 512, 1024, 16, 3, 4, 2
+    dh = d // H
+    g = torch.Generator().manual_seed(11)
+    dims = {"q": (d, d), "k": (d, Hkv * dh), "v": (d, Hkv * dh), "o": (d, d), "gate": (d, ffn), "up": (d, ffn), "down": (ffn, d)}
+    p = {"g1": 1.0 + 0.1 * torch.randn(d, generator=g, dtype=torch.float64),
+         "g2": 1.0 + 0.1 * torch.randn(d, generator=g, dtype=torch.float64)}
+    p["g1"], p["g2"] = p["g1"].float().double(), p["g2"].float().double()
+    for name, (di, do) in dims.items():
+        p["W_" + name] = bf16(torch.randn(di, do, generator=g, dtype=torch.float64) / math.sqrt(di))
+        p["A_" + name] = bf16(0.05 * torch.randn(n_ad, r, di, generator=g, dtype=torch.float64))
+        p["B_" + name] = bf16(0.05 * torch.randn(n_ad, r, do, generator=g, dtype=torch.float64))
+        p["s_" + name] = torch.full((n_ad,), 2.0, dtype=torch.float64)
+    # batch: an inference prompt, five decode rows, two fine-tuning sequences, a prompt without adapter
+    segs = [(0, 40, 0, 0)] + [(40 + i, 1, i % 3, 0) for i in range(5)] + [(45, 64, 1, 1), (109, 33, 2, 1), (142, 20, -1, 0)]
+    T = 162
+    x = bf16(torch.randn(T, d, generator=g, dtype=torch.float64))
+    row_adapter = [-1] * T
+    sequences = []
+    for s, n, a, _ in segs:
+        for t in range(s, s + n):
+            row_adapter[t] = a
+        sequences.append(list(range(s, s + n)))
+    y_ref = lo.layer_forward(x, p, row_adapter, sequences, H, Hkv)
+
+    with Session(0) as sess:
+        layer = DecoderLayer(sess, p, H, Hkv, max_ft_rows=128)
+        y = layer.forward(x.to(sess.device).to(torch.bfloat16), synth.segments_array(segs))
+        assert mb.mlora_poll_status(sess.ctx) == mb.MLORA_OK
+        err = (y.double().cpu() - y_ref).abs()
+        assert float((err - 6e-2 * (1 + y_ref.abs())).max()) <= 0, float(err.max())
+        assert layer.saved_rows == 97 and layer.saved == [(64, 1), (33, 2)]
+        assert torch.equal(layer.saved_x[:97].cpu().double(), x[45:142])      # the layer input, bit for bit
+
+        # backward over the fine-tuning rows alone, recomputed from the saved input
+        ft_rows = list(range(45, 142))
+        dy = bf16(torch.randn(97, d, generator=g, dtype=torch.float64))
+        dx, grads, slots = layer.backward(dy.to(sess.device))
+        assert mb.mlora_poll_status(sess.ctx) == mb.MLORA_OK and slots == [1, 2]
+        ref = lo.layer_backward(x[45:142], p, [1] * 64 + [2] * 33, [list(range(0, 64)), list(range(64, 97))], H, Hkv, dy,
+                                adapters=[1, 2])
+
+        def close(name, got, want, tol):
+            got, want = got.double().cpu(), want
+            scale = float(want.abs().max())
+            bad = float(((got - want).abs() - tol * (scale + want.abs())).max())
+            assert bad <= 0, (name, bad, scale)
+        close("dx", dx, ref["dx"], 4e-2)
+        for name in PROJ:
+            close("dA_" + name, grads[name][0], ref["dA_" + name], 4e-2)
+            close("dB_" + name, grads[name][1], ref["dB_" + name], 4e-2)
+        assert layer.saved_rows == 0
