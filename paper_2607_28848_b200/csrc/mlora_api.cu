@@ -19,6 +19,8 @@
 #include "gemm2_tcgen05.cuh"
 #include "simt.cuh"
 #include "skinny.cuh"
+#include "glue.cuh"
+#include "mlora_layer_ops.h"
 
 using namespace mlora;
 
@@ -1172,5 +1174,75 @@ int mlora_debug_timeline_reset() {
   return cudaMemcpyToSymbol(mlora::g_timeline, zeros, sizeof(zeros)) == cudaSuccess ? 0 : -1;
 }
 #endif
+
+// ---- layer pieces around the projections (mlora_layer_ops.h) ----------------------------------
+static inline mlora_status_t launched() {
+  const cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? MLORA_OK : cuda_failure("kernel launch", cudaGetErrorString(e));
+}
+static inline int ew_blocks(int64_t n8) {
+  const int64_t b = (n8 + 255) / 256;
+  return (int)(b < 148 * 8 ? (b < 1 ? 1 : b) : 148 * 8);
+}
+
+mlora_status_t mlora_rmsnorm_forward(const void* x, int64_t ldx, const float* gain, void* y, int64_t ldy,
+                                     int32_t n_rows, int32_t d, float eps, void* cuda_stream) {
+  if (!x || !gain || !y || n_rows < 0 || d <= 0 || ldx < d || ldy < d) return MLORA_ERR_INVALID_ARG;
+  if (d % 8 || ldx % 8 || ldy % 8 || !aligned16(x) || !aligned16(y) || !aligned16(gain)) return MLORA_ERR_UNSUPPORTED;
+  if (n_rows == 0) return MLORA_OK;
+  glue::rmsnorm_fwd_kernel<<<n_rows, 128, 0, reinterpret_cast<cudaStream_t>(cuda_stream)>>>(
+      (const __nv_bfloat16*)x, ldx, gain, (__nv_bfloat16*)y, ldy, d, eps);
+  return launched();
+}
+
+mlora_status_t mlora_rmsnorm_backward(const void* x, int64_t ldx, const float* gain, const void* dy, int64_t lddy,
+                                      void* dx, int64_t lddx, int32_t n_rows, int32_t d, float eps, void* cuda_stream) {
+  if (!x || !gain || !dy || !dx || n_rows < 0 || d <= 0 || ldx < d || lddy < d || lddx < d) return MLORA_ERR_INVALID_ARG;
+  if (d % 8 || ldx % 8 || lddy % 8 || lddx % 8 || !aligned16(x) || !aligned16(dy) || !aligned16(dx) || !aligned16(gain))
+    return MLORA_ERR_UNSUPPORTED;
+  if (n_rows == 0) return MLORA_OK;
+  glue::rmsnorm_bwd_kernel<<<n_rows, 128, 0, reinterpret_cast<cudaStream_t>(cuda_stream)>>>(
+      (const __nv_bfloat16*)x, ldx, gain, (const __nv_bfloat16*)dy, lddy, (__nv_bfloat16*)dx, lddx, d, eps);
+  return launched();
+}
+
+mlora_status_t mlora_rope(const void* x, int64_t ldx, void* y, int64_t ldy, const int32_t* pos, int32_t n_rows,
+                          int32_t n_heads, int32_t d_head, float theta, int32_t transpose, void* cuda_stream) {
+  if (!x || !y || !pos || n_rows < 0 || n_heads <= 0 || d_head <= 0 || !(theta > 0.f)) return MLORA_ERR_INVALID_ARG;
+  if (ldx < (int64_t)n_heads * d_head || ldy < (int64_t)n_heads * d_head) return MLORA_ERR_INVALID_ARG;
+  if (d_head % 16 || ldx % 8 || ldy % 8 || !aligned16(x) || !aligned16(y)) return MLORA_ERR_UNSUPPORTED;
+  if (n_rows == 0) return MLORA_OK;
+  glue::rope_kernel<<<n_rows, 128, 0, reinterpret_cast<cudaStream_t>(cuda_stream)>>>(
+      (const __nv_bfloat16*)x, ldx, (__nv_bfloat16*)y, ldy, pos, n_heads, d_head, log2f(theta), transpose ? -1.0f : 1.0f);
+  return launched();
+}
+
+mlora_status_t mlora_swiglu_forward(const void* g, const void* u, void* m, int64_t n, void* cuda_stream) {
+  if (!g || !u || !m || n < 0) return MLORA_ERR_INVALID_ARG;
+  if (n % 8 || !aligned16(g) || !aligned16(u) || !aligned16(m)) return MLORA_ERR_UNSUPPORTED;
+  if (n == 0) return MLORA_OK;
+  glue::swiglu_fwd_kernel<<<ew_blocks(n / 8), 256, 0, reinterpret_cast<cudaStream_t>(cuda_stream)>>>(
+      (const __nv_bfloat16*)g, (const __nv_bfloat16*)u, (__nv_bfloat16*)m, n / 8);
+  return launched();
+}
+
+mlora_status_t mlora_swiglu_backward(const void* g, const void* u, const void* dm, void* dg, void* du, int64_t n,
+                                     void* cuda_stream) {
+  if (!g || !u || !dm || !dg || !du || n < 0) return MLORA_ERR_INVALID_ARG;
+  if (n % 8 || !aligned16(g) || !aligned16(u) || !aligned16(dm) || !aligned16(dg) || !aligned16(du)) return MLORA_ERR_UNSUPPORTED;
+  if (n == 0) return MLORA_OK;
+  glue::swiglu_bwd_kernel<<<ew_blocks(n / 8), 256, 0, reinterpret_cast<cudaStream_t>(cuda_stream)>>>(
+      (const __nv_bfloat16*)g, (const __nv_bfloat16*)u, (const __nv_bfloat16*)dm, (__nv_bfloat16*)dg, (__nv_bfloat16*)du, n / 8);
+  return launched();
+}
+
+mlora_status_t mlora_add(const void* a, const void* b, void* out, int64_t n, void* cuda_stream) {
+  if (!a || !b || !out || n < 0) return MLORA_ERR_INVALID_ARG;
+  if (n % 8 || !aligned16(a) || !aligned16(b) || !aligned16(out)) return MLORA_ERR_UNSUPPORTED;
+  if (n == 0) return MLORA_OK;
+  glue::add_kernel<<<ew_blocks(n / 8), 256, 0, reinterpret_cast<cudaStream_t>(cuda_stream)>>>(
+      (const __nv_bfloat16*)a, (const __nv_bfloat16*)b, (__nv_bfloat16*)out, n / 8);
+  return launched();
+}
 
 }  // extern "C"

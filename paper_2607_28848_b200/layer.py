@@ -6,9 +6,10 @@ layer below needs).
 
 Division of labour: the seven projections (q, k, v, o, gate, up, down) run in this library's kernels
 - `mlora_mixed_forward` in the serving pass, `mlora_mixed_forward` + `mlora_backward` in the
-recompute/backward pass.  Everything between them (RMSNorm, rotary embedding, attention, SiLU gate,
-residual adds) and the chain rule through those pieces are PyTorch library calls: they are glue here,
-not kernels of this library.  A decode row is a one-token sequence (no KV cache in this module).
+recompute/backward pass - and so do RMSNorm, the rotary embedding, the SiLU gate and the residual adds
+with their input gradients (`mlora_layer_ops.h`).  Attention (softmax(QK^T)V inside each sequence) and
+its gradient are PyTorch library calls: glue here, not a kernel of this library.  PyTorch's autograd
+only strings the pieces together.  A decode row is a one-token sequence (no KV cache in this module).
 """
 from __future__ import annotations
 
@@ -19,6 +20,7 @@ import numpy as np
 import torch
 
 from . import binding as mb
+from . import layer_ops as mo
 from . import synth
 
 PROJ = ("q", "k", "v", "o", "gate", "up", "down")
@@ -60,20 +62,66 @@ class _ProjFn(torch.autograd.Function):
         return dx, None, None
 
 
-def _rmsnorm(x, gain, eps=1e-5):
-    xf = x.float()
-    return (xf * torch.rsqrt((xf * xf).mean(-1, keepdim=True) + eps) * gain).to(torch.bfloat16)
+class _RmsNormFn(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, x, gain):
+        x = x.contiguous()
+        y = torch.empty_like(x)
+        mo.mlora_rmsnorm_forward(x, gain, y)
+        ctx.save_for_backward(x, gain)
+        return y
+
+    @staticmethod
+    def backward(ctx, dy):
+        x, gain = ctx.saved_tensors
+        dx = torch.empty_like(x)
+        mo.mlora_rmsnorm_backward(x, gain, dy.contiguous(), dx)
+        return dx, None
 
 
-def _rope(x, pos, theta=500000.0):
-    d = x.shape[-1]
-    half = d // 2
-    inv = theta ** (-torch.arange(0, half, dtype=torch.float32, device=x.device) * 2.0 / d)
-    ang = pos.float()[:, None] * inv[None, :]
-    cos, sin = torch.cos(ang)[:, None, :], torch.sin(ang)[:, None, :]
-    xf = x.float()
-    x1, x2 = xf[..., :half], xf[..., half:]
-    return torch.cat([x1 * cos - x2 * sin, x2 * cos + x1 * sin], dim=-1).to(torch.bfloat16)
+class _RopeFn(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, x, pos, n_heads, d_head):
+        x = x.contiguous()
+        y = torch.empty_like(x)
+        mo.mlora_rope(x, y, pos, n_heads, d_head)
+        ctx.pos, ctx.shape = pos, (n_heads, d_head)
+        return y
+
+    @staticmethod
+    def backward(ctx, dy):
+        dx = torch.empty_like(dy)
+        mo.mlora_rope(dy.contiguous(), dx, ctx.pos, ctx.shape[0], ctx.shape[1], transpose=True)
+        return dx, None, None, None
+
+
+class _SwigluFn(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, g, u):
+        g, u = g.contiguous(), u.contiguous()
+        m = torch.empty_like(g)
+        mo.mlora_swiglu_forward(g, u, m)
+        ctx.save_for_backward(g, u)
+        return m
+
+    @staticmethod
+    def backward(ctx, dm):
+        g, u = ctx.saved_tensors
+        dg, du = torch.empty_like(g), torch.empty_like(u)
+        mo.mlora_swiglu_backward(g, u, dm.contiguous(), dg, du)
+        return dg, du
+
+
+class _AddFn(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, a, b):
+        out = torch.empty_like(a)
+        mo.mlora_add(a.contiguous(), b.contiguous(), out)
+        return out
+
+    @staticmethod
+    def backward(ctx, d):
+        return d, d
 
 
 class DecoderLayer:
@@ -95,12 +143,12 @@ class DecoderLayer:
     def _body(self, x, lin, sequences):
         T = x.shape[0]
         dh = self.d // self.n_heads
-        pos = torch.zeros(T, dtype=torch.long, device=x.device)
+        pos = torch.zeros(T, dtype=torch.int32, device=x.device)
         for start, n in sequences:
-            pos[start:start + n] = torch.arange(n, device=x.device)
-        h1 = _rmsnorm(x, self.g1)
-        q = _rope(lin("q", h1).reshape(T, self.n_heads, dh), pos)
-        k = _rope(lin("k", h1).reshape(T, self.n_kv, dh), pos)
+            pos[start:start + n] = torch.arange(n, device=x.device, dtype=torch.int32)
+        h1 = _RmsNormFn.apply(x, self.g1)
+        q = _RopeFn.apply(lin("q", h1), pos, self.n_heads, dh).reshape(T, self.n_heads, dh)
+        k = _RopeFn.apply(lin("k", h1), pos, self.n_kv, dh).reshape(T, self.n_kv, dh)
         v = lin("v", h1).reshape(T, self.n_kv, dh)
         rep = self.n_heads // self.n_kv
         outs = []
@@ -111,10 +159,10 @@ class DecoderLayer:
             o = torch.nn.functional.scaled_dot_product_attention(qs, ks, vs, is_causal=True)
             outs.append(o[0].transpose(0, 1).reshape(n, self.d))
         a = torch.cat(outs, dim=0)
-        x2 = x + lin("o", a)
-        h2 = _rmsnorm(x2, self.g2)
-        m = torch.nn.functional.silu(lin("gate", h2).float()).to(torch.bfloat16) * lin("up", h2)
-        return x2 + lin("down", m)
+        x2 = _AddFn.apply(x, lin("o", a))
+        h2 = _RmsNormFn.apply(x2, self.g2)
+        m = _SwigluFn.apply(lin("gate", h2), lin("up", h2))
+        return _AddFn.apply(x2, lin("down", m))
 
     # -- serving forward: mixed batch, keeps the layer input of the fine-tuning rows --------------
     @torch.no_grad()

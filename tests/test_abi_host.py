@@ -17,9 +17,10 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def test_library_exports_every_declared_symbol():
+    from paper_2607_28848_b200 import layer_ops as mo
     from paper_2607_28848_b200 import sched as ms
     lib = mb.load_library()
-    bound = {"mlora.h": set(mb.EXPORTS), "mlora_sched.h": set(ms.EXPORTS)}
+    bound = {"mlora.h": set(mb.EXPORTS), "mlora_sched.h": set(ms.EXPORTS), "mlora_layer_ops.h": set(mo.EXPORTS)}
     inc = os.path.join(ROOT, "include")
     assert sorted(f for f in os.listdir(inc) if f.endswith(".h")) == sorted(bound)
     for fname, names in bound.items():

@@ -1,0 +1,88 @@
+"""The layer pieces around the projections (RMSNorm, rotary embedding, SiLU gate, add) against the
+layer oracle's definitions in fp64; the backward entry points against autograd of those definitions."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import layer_oracle as lo
+from paper_2607_28848_b200 import layer_ops as mo
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def bf(t):
+    return t.to(torch.bfloat16)
+
+
+def close(got, ref, tol=1.2e-2):
+    got, ref = got.double().cpu(), ref.double()
+    assert float(((got - ref).abs() - tol * (1 + ref.abs())).max()) <= 0, float((got - ref).abs().max())
+
+
+@pytest.mark.parametrize("rows,d", [(1, 8), (37, 512), (130, 4096), (5, 14336)])
+def test_rmsnorm_forward_and_backward(rows, d):
+    g = torch.Generator().manual_seed(rows + d)
+    x = bf(torch.randn(rows, d, generator=g) * 1.7).to(DEV)
+    gain = (1 + 0.2 * torch.randn(d, generator=g)).float().to(DEV)
+    dy = bf(torch.randn(rows, d, generator=g)).to(DEV)
+    y, dx = torch.empty_like(x), torch.empty_like(x)
+    mo.mlora_rmsnorm_forward(x, gain, y)
+    mo.mlora_rmsnorm_backward(x, gain, dy, dx)
+    xr = x.double().cpu().requires_grad_(True)
+    yr = lo.rmsnorm(xr, gain.double().cpu())
+    yr.backward(dy.double().cpu())
+    close(y, yr.detach())
+    close(dx, xr.grad)
+
+
+@pytest.mark.parametrize("heads,dh", [(4, 128), (32, 128), (8, 64), (1, 16)])
+def test_rope_forward_and_transpose(heads, dh):
+    g = torch.Generator().manual_seed(heads * dh)
+    T = 77
+    x = bf(torch.randn(T, heads * dh, generator=g)).to(DEV)
+    pos = torch.randint(0, 4000, (T,), generator=g, dtype=torch.int32).to(DEV)
+    y = torch.empty_like(x)
+    mo.mlora_rope(x, y, pos, heads, dh)
+    ref = lo.rope(x.double().cpu().reshape(T, heads, dh), pos.cpu().long()).reshape(T, heads * dh)
+    close(y, ref)
+    # the transposed rotation undoes the forward (up to the two bf16 roundings) and is its input gradient
+    back = torch.empty_like(x)
+    mo.mlora_rope(y, back, pos, heads, dh, transpose=True)
+    close(back, x.double().cpu(), tol=2e-2)
+    xr = x.double().cpu().reshape(T, heads, dh).requires_grad_(True)
+    dy = bf(torch.randn(T, heads * dh, generator=g))
+    lo.rope(xr, pos.cpu().long()).backward(dy.double().reshape(T, heads, dh))
+    dx = torch.empty_like(x)
+    mo.mlora_rope(dy.to(DEV), dx, pos, heads, dh, transpose=True)
+    close(dx, xr.grad.reshape(T, heads * dh))
+    mo.mlora_rope(x, x, pos, heads, dh)                      # in place
+    assert torch.equal(x, y)
+
+
+@pytest.mark.parametrize("n", [8, 4096 * 33, 14336 * 70])
+def test_swiglu_and_add(n):
+    g = torch.Generator().manual_seed(n)
+    a, b, d = (bf(torch.randn(n, generator=g) * 2).to(DEV) for _ in range(3))
+    m, dg, du, s = (torch.empty_like(a) for _ in range(4))
+    mo.mlora_swiglu_forward(a, b, m)
+    mo.mlora_swiglu_backward(a, b, d, dg, du)
+    mo.mlora_add(a, b, s)
+    ar, br = a.double().cpu().requires_grad_(True), b.double().cpu().requires_grad_(True)
+    mr = torch.nn.functional.silu(ar) * br
+    mr.backward(d.double().cpu())
+    close(m, mr.detach())
+    close(dg, ar.grad)
+    close(du, br.grad)
+    close(s, a.double().cpu() + b.double().cpu())
+
+
+def test_argument_errors():
+    x = torch.zeros(4, 12, dtype=torch.bfloat16, device=DEV)           # 12 is not a multiple of 8
+    gain = torch.ones(12, device=DEV)
+    from paper_2607_28848_b200 import binding as mb
+    with pytest.raises(mb.MloraError) as e:
+        mo.mlora_rmsnorm_forward(x, gain, torch.empty_like(x))
+    assert e.value.status == mb.MLORA_ERR_UNSUPPORTED
+    with pytest.raises(mb.MloraError):
+        mo.mlora_rope(x, x, torch.zeros(4, dtype=torch.int32, device=DEV), 1, 12)
