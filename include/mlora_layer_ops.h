@@ -4,7 +4,8 @@
  * residual-stream input of each layer is saved per fine-tuning token and the backward recomputes the
  * layer from it, so these pieces run again there and their input gradients are needed.  The paper
  * describes no kernels for them; the base model is frozen, so no gradient of the norm gain exists.)
- * Attention is not part of this header.
+ * Attention is here too, as a plain CUDA-core statement of the operation for the short sequences of the
+ * fine-tuning path (one warp per row and head, keys visited one by one) - not a tensor-core kernel.
  *
  * All pointers are device pointers on the current device, all buffers borrowed; leading dimensions
  * (ld*) are in elements; rows and element counts must keep 16-byte alignment as stated per call.
@@ -47,6 +48,24 @@ mlora_status_t mlora_swiglu_backward(const void* g, const void* u, const void* d
 
 /* out = a + b over n contiguous bf16 elements (n a multiple of 8); out may alias a or b. */
 mlora_status_t mlora_add(const void* a, const void* b, void* out, int64_t n, void* cuda_stream);
+
+/* Causal softmax attention inside each sequence of a packed batch, grouped-query heads:
+ *   o[i, h] = sum_{j <= i, same sequence} softmax_j(q[i, h] . k[j, h / (n_heads / n_kv)] / sqrt(d_head)) v[j, ...]
+ * q, o bf16 [n_rows, n_heads * d_head] (row strides ldq, ldo), k, v bf16 [n_rows, n_kv * d_head];
+ * seq_start[i] = first row of row i's sequence, seq_end[i] = one past its last row (int32 [n_rows]; the
+ * rows of a sequence are consecutive); lse fp32 [n_rows, n_heads] receives log(sum_j exp(s_ij)), which the
+ * backward needs.  d_head is 64 or 128; n_heads a multiple of n_kv. */
+mlora_status_t mlora_attention_forward(const void* q, int64_t ldq, const void* k, int64_t ldk, const void* v, int64_t ldv,
+                                       void* o, int64_t ldo, float* lse, const int32_t* seq_start, const int32_t* seq_end,
+                                       int32_t n_rows, int32_t n_heads, int32_t n_kv, int32_t d_head, void* cuda_stream);
+
+/* Gradients of the above for a given dO: dq like q, dk and dv like k and v (each element written once; the
+ * sums over the query heads that share a kv head are inside).  o and lse are the forward's outputs. */
+mlora_status_t mlora_attention_backward(const void* q, int64_t ldq, const void* k, int64_t ldk, const void* v, int64_t ldv,
+                                        const void* o, int64_t ldo, const float* lse, const void* dO, int64_t lddo,
+                                        void* dq, int64_t lddq, void* dk, int64_t lddk, void* dv, int64_t lddv,
+                                        const int32_t* seq_start, const int32_t* seq_end, int32_t n_rows,
+                                        int32_t n_heads, int32_t n_kv, int32_t d_head, void* cuda_stream);
 
 #ifdef __cplusplus
 }

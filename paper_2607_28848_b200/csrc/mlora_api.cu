@@ -20,6 +20,7 @@
 #include "simt.cuh"
 #include "skinny.cuh"
 #include "glue.cuh"
+#include "attention.cuh"
 #include "mlora_layer_ops.h"
 
 using namespace mlora;
@@ -1242,6 +1243,50 @@ mlora_status_t mlora_add(const void* a, const void* b, void* out, int64_t n, voi
   if (n == 0) return MLORA_OK;
   glue::add_kernel<<<ew_blocks(n / 8), 256, 0, reinterpret_cast<cudaStream_t>(cuda_stream)>>>(
       (const __nv_bfloat16*)a, (const __nv_bfloat16*)b, (__nv_bfloat16*)out, n / 8);
+  return launched();
+}
+
+mlora_status_t mlora_attention_forward(const void* q, int64_t ldq, const void* k, int64_t ldk, const void* v, int64_t ldv,
+                                       void* o, int64_t ldo, float* lse, const int32_t* seq_start, const int32_t* seq_end,
+                                       int32_t n_rows, int32_t n_heads, int32_t n_kv, int32_t d_head, void* cuda_stream) {
+  if (!q || !k || !v || !o || !lse || !seq_start || !seq_end || n_rows < 0 || n_heads <= 0 || n_kv <= 0)
+    return MLORA_ERR_INVALID_ARG;
+  if ((d_head != 64 && d_head != 128) || n_heads % n_kv) return MLORA_ERR_UNSUPPORTED;
+  if (n_rows == 0) return MLORA_OK;
+  attn::AttnArgs a{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, ldq, ldk, ldv,
+                   seq_start, seq_end, n_rows, n_heads, n_kv, 1.0f / sqrtf((float)d_head)};
+  const int blocks = (int)(((int64_t)n_rows * n_heads + 7) / 8);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (d_head == 128) attn::forward_kernel<4><<<blocks, 256, 0, st>>>(a, (__nv_bfloat16*)o, ldo, lse);
+  else attn::forward_kernel<2><<<blocks, 256, 0, st>>>(a, (__nv_bfloat16*)o, ldo, lse);
+  return launched();
+}
+
+mlora_status_t mlora_attention_backward(const void* q, int64_t ldq, const void* k, int64_t ldk, const void* v, int64_t ldv,
+                                        const void* o, int64_t ldo, const float* lse, const void* dO, int64_t lddo,
+                                        void* dq, int64_t lddq, void* dk, int64_t lddk, void* dv, int64_t lddv,
+                                        const int32_t* seq_start, const int32_t* seq_end, int32_t n_rows,
+                                        int32_t n_heads, int32_t n_kv, int32_t d_head, void* cuda_stream) {
+  if (!q || !k || !v || !o || !lse || !dO || !dq || !dk || !dv || !seq_start || !seq_end || n_rows < 0 || n_heads <= 0 ||
+      n_kv <= 0)
+    return MLORA_ERR_INVALID_ARG;
+  if ((d_head != 64 && d_head != 128) || n_heads % n_kv) return MLORA_ERR_UNSUPPORTED;
+  if (n_rows == 0) return MLORA_OK;
+  attn::AttnArgs a{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, ldq, ldk, ldv,
+                   seq_start, seq_end, n_rows, n_heads, n_kv, 1.0f / sqrtf((float)d_head)};
+  const int bq = (int)(((int64_t)n_rows * n_heads + 7) / 8), bk = (int)(((int64_t)n_rows * n_kv + 7) / 8);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (d_head == 128) {
+    attn::backward_dq_kernel<4><<<bq, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,
+                                                    (__nv_bfloat16*)dq, lddq);
+    attn::backward_dkv_kernel<4><<<bk, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,
+                                                     (__nv_bfloat16*)dk, lddk, (__nv_bfloat16*)dv, lddv);
+  } else {
+    attn::backward_dq_kernel<2><<<bq, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,
+                                                    (__nv_bfloat16*)dq, lddq);
+    attn::backward_dkv_kernel<2><<<bk, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,
+                                                     (__nv_bfloat16*)dk, lddk, (__nv_bfloat16*)dv, lddv);
+  }
   return launched();
 }
 

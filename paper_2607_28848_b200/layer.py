@@ -7,9 +7,9 @@ layer below needs).
 Division of labour: the seven projections (q, k, v, o, gate, up, down) run in this library's kernels
 - `mlora_mixed_forward` in the serving pass, `mlora_mixed_forward` + `mlora_backward` in the
 recompute/backward pass - and so do RMSNorm, the rotary embedding, the SiLU gate and the residual adds
-with their input gradients (`mlora_layer_ops.h`).  Attention (softmax(QK^T)V inside each sequence) and
-its gradient are PyTorch library calls: glue here, not a kernel of this library.  PyTorch's autograd
-only strings the pieces together.  A decode row is a one-token sequence (no KV cache in this module).
+with their input gradients, and attention as a plain CUDA-core kernel pair for short sequences
+(`mlora_layer_ops.h`).  PyTorch's autograd only strings the pieces together; every arithmetic step of
+the layer runs in this library.  A decode row is a one-token sequence (no KV cache in this module).
 """
 from __future__ import annotations
 
@@ -112,6 +112,26 @@ class _SwigluFn(torch.autograd.Function):
         return dg, du
 
 
+class _AttnFn(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, q, k, v, seq_start, seq_end, n_heads, n_kv, d_head):
+        q, k, v = q.contiguous(), k.contiguous(), v.contiguous()
+        o = torch.empty_like(q)
+        lse = torch.empty((q.shape[0], n_heads), dtype=torch.float32, device=q.device)
+        mo.mlora_attention_forward(q, k, v, o, lse, seq_start, seq_end, n_heads, n_kv, d_head)
+        ctx.save_for_backward(q, k, v, o, lse)
+        ctx.meta = (seq_start, seq_end, n_heads, n_kv, d_head)
+        return o
+
+    @staticmethod
+    def backward(ctx, dO):
+        q, k, v, o, lse = ctx.saved_tensors
+        seq_start, seq_end, n_heads, n_kv, d_head = ctx.meta
+        dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+        mo.mlora_attention_backward(q, k, v, o, lse, dO.contiguous(), dq, dk, dv, seq_start, seq_end, n_heads, n_kv, d_head)
+        return dq, dk, dv, None, None, None, None, None
+
+
 class _AddFn(torch.autograd.Function):
     @staticmethod
     def forward(ctx, a, b):
@@ -144,21 +164,17 @@ class DecoderLayer:
         T = x.shape[0]
         dh = self.d // self.n_heads
         pos = torch.zeros(T, dtype=torch.int32, device=x.device)
+        seq_start = torch.arange(T, dtype=torch.int32, device=x.device)          # rows outside every sequence stand alone
+        seq_end = seq_start + 1
         for start, n in sequences:
             pos[start:start + n] = torch.arange(n, device=x.device, dtype=torch.int32)
+            seq_start[start:start + n] = start
+            seq_end[start:start + n] = start + n
         h1 = _RmsNormFn.apply(x, self.g1)
-        q = _RopeFn.apply(lin("q", h1), pos, self.n_heads, dh).reshape(T, self.n_heads, dh)
-        k = _RopeFn.apply(lin("k", h1), pos, self.n_kv, dh).reshape(T, self.n_kv, dh)
-        v = lin("v", h1).reshape(T, self.n_kv, dh)
-        rep = self.n_heads // self.n_kv
-        outs = []
-        for start, n in sequences:                  # causal attention inside each sequence (library call)
-            qs = q[start:start + n].transpose(0, 1)[None]
-            ks = k[start:start + n].repeat_interleave(rep, dim=1).transpose(0, 1)[None]
-            vs = v[start:start + n].repeat_interleave(rep, dim=1).transpose(0, 1)[None]
-            o = torch.nn.functional.scaled_dot_product_attention(qs, ks, vs, is_causal=True)
-            outs.append(o[0].transpose(0, 1).reshape(n, self.d))
-        a = torch.cat(outs, dim=0)
+        q = _RopeFn.apply(lin("q", h1), pos, self.n_heads, dh)
+        k = _RopeFn.apply(lin("k", h1), pos, self.n_kv, dh)
+        v = lin("v", h1)
+        a = _AttnFn.apply(q, k, v, seq_start, seq_end, self.n_heads, self.n_kv, dh)
         x2 = _AddFn.apply(x, lin("o", a))
         h2 = _RmsNormFn.apply(x2, self.g2)
         m = _SwigluFn.apply(lin("gate", h2), lin("up", h2))

@@ -6,7 +6,7 @@ import ctypes
 from . import binding as _b
 
 EXPORTS = ("mlora_rmsnorm_forward", "mlora_rmsnorm_backward", "mlora_rope", "mlora_swiglu_forward",
-           "mlora_swiglu_backward", "mlora_add")
+           "mlora_swiglu_backward", "mlora_add", "mlora_attention_forward", "mlora_attention_backward")
 _ready = False
 
 
@@ -22,6 +22,9 @@ def _lib():
     lib.mlora_swiglu_forward.argtypes = [vp, vp, vp, i64, vp]
     lib.mlora_swiglu_backward.argtypes = [vp, vp, vp, vp, vp, i64, vp]
     lib.mlora_add.argtypes = [vp, vp, vp, i64, vp]
+    lib.mlora_attention_forward.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, vp, vp, i32, i32, i32, i32, vp]
+    lib.mlora_attention_backward.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64, vp, i64, vp, i64,
+                                             vp, vp, i32, i32, i32, i32, vp]
     for name in EXPORTS:
         getattr(lib, name).restype = ctypes.c_int
     _ready = True
@@ -60,3 +63,18 @@ def mlora_swiglu_backward(g, u, dm, dg, du, stream=None) -> None:
 
 def mlora_add(a, b, out, stream=None) -> None:
     _b._check(_lib().mlora_add(_p(a), _p(b), _p(out), a.numel(), _b._stream_ptr(stream)), "mlora_add")
+
+
+def mlora_attention_forward(q, k, v, o, lse, seq_start, seq_end, n_heads: int, n_kv: int, d_head: int, stream=None) -> None:
+    """q, o [T, n_heads * d_head], k, v [T, n_kv * d_head] bf16; lse fp32 [T, n_heads]; seq_start / seq_end int32 [T]."""
+    _b._check(_lib().mlora_attention_forward(_p(q), q.stride(0), _p(k), k.stride(0), _p(v), v.stride(0), _p(o), o.stride(0),
+                                             _p(lse), _p(seq_start), _p(seq_end), q.shape[0], int(n_heads), int(n_kv),
+                                             int(d_head), _b._stream_ptr(stream)), "mlora_attention_forward")
+
+
+def mlora_attention_backward(q, k, v, o, lse, dO, dq, dk, dv, seq_start, seq_end, n_heads: int, n_kv: int, d_head: int,
+                             stream=None) -> None:
+    _b._check(_lib().mlora_attention_backward(_p(q), q.stride(0), _p(k), k.stride(0), _p(v), v.stride(0), _p(o), o.stride(0),
+                                              _p(lse), _p(dO), dO.stride(0), _p(dq), dq.stride(0), _p(dk), dk.stride(0),
+                                              _p(dv), dv.stride(0), _p(seq_start), _p(seq_end), q.shape[0], int(n_heads),
+                                              int(n_kv), int(d_head), _b._stream_ptr(stream)), "mlora_attention_backward")

@@ -77,6 +77,35 @@ def test_swiglu_and_add(n):
     close(s, a.double().cpu() + b.double().cpu())
 
 
+@pytest.mark.parametrize("heads,kv,dh", [(4, 2, 128), (8, 8, 64), (6, 1, 128)])
+def test_attention_forward_and_backward(heads, kv, dh):
+    g = torch.Generator().manual_seed(heads * 100 + kv)
+    lens = [1, 37, 5, 130, 1, 64]                                  # packed sequences, decode-like single rows among them
+    T = sum(lens)
+    q = bf(torch.randn(T, heads * dh, generator=g)).to(DEV)
+    k = bf(torch.randn(T, kv * dh, generator=g)).to(DEV)
+    v = bf(torch.randn(T, kv * dh, generator=g)).to(DEV)
+    dO = bf(torch.randn(T, heads * dh, generator=g)).to(DEV)
+    start, end, seqs, r = [], [], [], 0
+    for n in lens:
+        start += [r] * n; end += [r + n] * n; seqs.append(list(range(r, r + n))); r += n
+    ss, se = torch.tensor(start, dtype=torch.int32, device=DEV), torch.tensor(end, dtype=torch.int32, device=DEV)
+    o, dq = torch.empty_like(q), torch.empty_like(q)
+    dk, dv = torch.empty_like(k), torch.empty_like(v)
+    lse = torch.empty((T, heads), dtype=torch.float32, device=DEV)
+    mo.mlora_attention_forward(q, k, v, o, lse, ss, se, heads, kv, dh)
+    mo.mlora_attention_backward(q, k, v, o, lse, dO, dq, dk, dv, ss, se, heads, kv, dh)
+    qr = q.double().cpu().reshape(T, heads, dh).requires_grad_(True)
+    kr = k.double().cpu().reshape(T, kv, dh).requires_grad_(True)
+    vr = v.double().cpu().reshape(T, kv, dh).requires_grad_(True)
+    orf = lo.attention(qr, kr, vr, seqs)
+    orf.backward(dO.double().cpu().reshape(T, heads, dh))
+    close(o, orf.detach().reshape(T, heads * dh))
+    close(dq, qr.grad.reshape(T, heads * dh), tol=2e-2)
+    close(dk, kr.grad.reshape(T, kv * dh), tol=2e-2)
+    close(dv, vr.grad.reshape(T, kv * dh), tol=2e-2)
+
+
 def test_argument_errors():
     x = torch.zeros(4, 12, dtype=torch.bfloat16, device=DEV)           # 12 is not a multiple of 8
     gain = torch.ones(12, device=DEV)
