@@ -1,14 +1,18 @@
-// Rank-r ("skinny") kernels of the multi-LoRA layer for bf16 storage.  Both are bound by the
-// bytes of the wide operand they stream once from HBM; the rank-r contraction itself runs on the
-// warp-level tensor-core instruction (mma.sync m16n8k16, fp32 accumulate) because at rank 16 and
-// above the CUDA cores could not keep up with the memory system.
+// Rank-r ("skinny") kernels of the multi-LoRA layer for bf16 storage.  They are bound by the bytes of
+// the wide operand they stream once from HBM; the rank-r contraction itself runs on the warp-level
+// tensor-core instruction (mma.sync m16n8k16, fp32 accumulate) because at rank 16 and above the CUDA
+// cores could not keep up with the memory system.
 //
-//  shrink_kernel : Out[t, q] = sum_k In[t, k] * P_a(t)[q, k]      (U = X A^T  and  V = s dY B^T)
-//                  work item = up to 32 rows that share one adapter, GATHERED by adapter id (they
-//                  need not be adjacent: decode rows of one adapter form one item, prefill and
-//                  fine-tune segments are runs of items); optionally copies the rows of In and the
-//                  result into the fine-tuning activation buffers on the way.
-//  grad_kernel   : G_g[q, j] = sum_{rows t of slot g} P[t, q] * Q[t, j]   (dB = (s U)^T dY, dA = V^T X)
+//  shrink : Out[t, q] = sum_k In[t, k] * P_a(t)[q, k]      (U = X A^T  and  V = s dY B^T)
+//           work item = up to 32 rows that share one adapter, GATHERED by adapter id (they need not be
+//           adjacent: decode rows of one adapter form one item, prefill and fine-tune segments are
+//           runs of items); optionally copies the rows of In and the result into the fine-tuning
+//           activation buffers on the way.
+//           shrink_stream_kernel (rank <= 32, the default): persistent, stages filled by the copy engine;
+//           shrink_kernel (rank 64 / 128): one CTA per item, operands straight from global memory.
+//  grad   : G_g[q, j] = sum_{rows t of slot g} P[t, q] * Q[t, j]   (dB = (s U)^T dY, dA = V^T X)
+//           grad_stream_kernel (rank <= 32: both gradients in one launch); grad_kernel (rank 64 / 128).
+//  expand_mask_kernel : the low-rank part of the input gradient under dropout.
 #pragma once
 
 #include "dropout.cuh"
