@@ -100,22 +100,28 @@ __global__ void __launch_bounds__(128)
 rope_kernel(const __nv_bfloat16* x, int64_t ldx, __nv_bfloat16* y, int64_t ldy, const int32_t* pos, int heads, int dh,
             float log2_theta, float sign) {
   const int t = blockIdx.x;
-  const int half = dh / 2, per_head = half / 8;
+  const int half = dh / 2, per_head = half / 8;     // 8-pair chunks per head
   const float p = (float)pos[t];
-  for (int w = threadIdx.x; w < heads * per_head; w += 128) {
-    const int h = w / per_head, i0 = (w % per_head) * 8;
+  // a thread owns one chunk of frequencies: their sines and cosines are computed once and used for
+  // every head it visits (heads hg, hg + 128 / per_head, ...)
+  const int chunk = threadIdx.x % per_head, hg = threadIdx.x / per_head, n_hg = 128 / per_head;
+  const int i0 = chunk * 8;
+  float sn[8], cs[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float inv = exp2f(-log2_theta * 2.0f * (float)(i0 + i) / (float)dh);
+    sincosf(p * inv, &sn[i], &cs[i]);
+    sn[i] *= sign;
+  }
+  for (int h = hg; h < heads; h += n_hg) {
     const __nv_bfloat16* src = x + (size_t)t * ldx + h * dh + i0;
     float a[8], b[8], oa[8], ob[8];
     unpack8(*reinterpret_cast<const uint4*>(src), a);
     unpack8(*reinterpret_cast<const uint4*>(src + half), b);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const float inv = exp2f(-log2_theta * 2.0f * (float)(i0 + i) / (float)dh);
-      float s, c;
-      sincosf(p * inv, &s, &c);
-      s *= sign;
-      oa[i] = a[i] * c - b[i] * s;
-      ob[i] = b[i] * c + a[i] * s;
+      oa[i] = a[i] * cs[i] - b[i] * sn[i];
+      ob[i] = b[i] * cs[i] + a[i] * sn[i];
     }
     __nv_bfloat16* dst = y + (size_t)t * ldy + h * dh + i0;
     *reinterpret_cast<uint4*>(dst) = pack8(oa);
@@ -131,7 +137,7 @@ swiglu_fwd_kernel(const __nv_bfloat16* g, const __nv_bfloat16* u, __nv_bfloat16*
     unpack8(reinterpret_cast<const uint4*>(g)[i], a);
     unpack8(reinterpret_cast<const uint4*>(u)[i], b);
 #pragma unroll
-    for (int k = 0; k < 8; ++k) o[k] = a[k] / (1.0f + __expf(-a[k])) * b[k];
+    for (int k = 0; k < 8; ++k) o[k] = __fdividef(a[k], 1.0f + __expf(-a[k])) * b[k];
     reinterpret_cast<uint4*>(m)[i] = pack8(o);
   }
 }
@@ -147,7 +153,7 @@ swiglu_bwd_kernel(const __nv_bfloat16* g, const __nv_bfloat16* u, const __nv_bfl
     unpack8(reinterpret_cast<const uint4*>(dm)[i], d);
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-      const float sg = 1.0f / (1.0f + __expf(-a[k]));
+      const float sg = __fdividef(1.0f, 1.0f + __expf(-a[k]));
       og[k] = d[k] * b[k] * sg * (1.0f + a[k] * (1.0f - sg));
       ou[k] = d[k] * a[k] * sg;
     }
