@@ -1252,13 +1252,15 @@ mlora_status_t mlora_attention_forward(const void* q, int64_t ldq, const void* k
   if (!q || !k || !v || !o || !lse || !seq_start || !seq_end || n_rows < 0 || n_heads <= 0 || n_kv <= 0)
     return MLORA_ERR_INVALID_ARG;
   if ((d_head != 64 && d_head != 128) || n_heads % n_kv) return MLORA_ERR_UNSUPPORTED;
+  if (ldq % 8 || ldk % 8 || ldv % 8 || ldo % 8 || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o))
+    return MLORA_ERR_UNSUPPORTED;
   if (n_rows == 0) return MLORA_OK;
   attn::AttnArgs a{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, ldq, ldk, ldv,
                    seq_start, seq_end, n_rows, n_heads, n_kv, 1.0f / sqrtf((float)d_head)};
   const int blocks = (int)(((int64_t)n_rows * n_heads + 7) / 8);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-  if (d_head == 128) attn::forward_kernel<4><<<blocks, 256, 0, st>>>(a, (__nv_bfloat16*)o, ldo, lse);
-  else attn::forward_kernel<2><<<blocks, 256, 0, st>>>(a, (__nv_bfloat16*)o, ldo, lse);
+  if (d_head == 128) attn::forward_kernel<32><<<blocks, 256, 0, st>>>(a, (__nv_bfloat16*)o, ldo, lse);
+  else attn::forward_kernel<16><<<blocks, 256, 0, st>>>(a, (__nv_bfloat16*)o, ldo, lse);
   return launched();
 }
 
@@ -1271,20 +1273,23 @@ mlora_status_t mlora_attention_backward(const void* q, int64_t ldq, const void* 
       n_kv <= 0)
     return MLORA_ERR_INVALID_ARG;
   if ((d_head != 64 && d_head != 128) || n_heads % n_kv) return MLORA_ERR_UNSUPPORTED;
+  if (ldq % 8 || ldk % 8 || ldv % 8 || ldo % 8 || lddo % 8 || lddq % 8 || lddk % 8 || lddv % 8 || !aligned16(q) ||
+      !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(dO) || !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
+    return MLORA_ERR_UNSUPPORTED;
   if (n_rows == 0) return MLORA_OK;
   attn::AttnArgs a{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, ldq, ldk, ldv,
                    seq_start, seq_end, n_rows, n_heads, n_kv, 1.0f / sqrtf((float)d_head)};
   const int bq = (int)(((int64_t)n_rows * n_heads + 7) / 8), bk = (int)(((int64_t)n_rows * n_kv + 7) / 8);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (d_head == 128) {
-    attn::backward_dq_kernel<4><<<bq, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,
+    attn::backward_dq_kernel<32><<<bq, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,
                                                     (__nv_bfloat16*)dq, lddq);
-    attn::backward_dkv_kernel<4><<<bk, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,
+    attn::backward_dkv_kernel<32><<<bk, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,
                                                      (__nv_bfloat16*)dk, lddk, (__nv_bfloat16*)dv, lddv);
   } else {
-    attn::backward_dq_kernel<2><<<bq, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,
+    attn::backward_dq_kernel<16><<<bq, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,
                                                     (__nv_bfloat16*)dq, lddq);
-    attn::backward_dkv_kernel<2><<<bk, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,
+    attn::backward_dkv_kernel<16><<<bk, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,
                                                      (__nv_bfloat16*)dk, lddk, (__nv_bfloat16*)dv, lddv);
   }
   return launched();
