@@ -323,8 +323,11 @@ gemm_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constant
         }
         ptx::fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0 && m0 < args.M && n0 + c * 64 < args.N) {
-          ptx::tma_store_2d(&tmOut, sb, n0 + c * 64, m0);     // rows / columns past the edge are clipped
+        // One group per chunk, empty for a chunk past the edge: the wait above counts groups, so a
+        // skipped commit would let the chunk after next reuse a buffer whose store is still reading.
+        if (lane == 0) {
+          if (m0 < args.M && n0 + c * 64 < args.N)
+            ptx::tma_store_2d(&tmOut, sb, n0 + c * 64, m0);   // rows / columns past the edge are clipped
           ptx::tma_store_commit();
         }
       }
