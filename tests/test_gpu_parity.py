@@ -124,6 +124,23 @@ def test_output_width_not_a_multiple_of_the_column_tile(sess, path, d_in, d_out)
         run_and_check(sess, w, t, path=path, blocked=True)
 
 
+@pytest.mark.parametrize("seed", range(4))
+def test_random_shapes_tables_and_kernel_variants(sess, seed):
+    """Seeded random layer shapes, ranks, adapter counts, segment tables, save offsets and kernel
+    variants on one warm context, each checked element by element (forward, saves, backward)."""
+    rng = np.random.default_rng(7000 + seed)
+    for it in range(10):
+        d_in = int(rng.choice([64, 128, 192, 256, 320, 512, 576, 1024, 2048]))
+        d_out = int(rng.choice([64, 128, 192, 256, 448, 512, 704, 1024, 4096]))
+        rank = int(rng.choice([8, 16, 32, 64, 128]))
+        w = synth.random_workload(7000 + 100 * seed + it, d_in, d_out, rank, int(rng.integers(1, 40)),
+                                  int(rng.integers(1, 1200)), max_seg=int(rng.integers(1, 400)),
+                                  p_decode=float(rng.uniform(0, 0.9)), p_finetune=float(rng.uniform(0, 0.7)))
+        cap = None if rng.random() < 0.5 else int(w.ft_rows + 30)
+        run_and_check(sess, w, synth.make_tensors(w), path=int(rng.choice([0, 0, 0, 2, 3, 4])), blocked=True,
+                      base=int(rng.integers(0, 3)) * 7, cap=cap)
+
+
 @pytest.mark.parametrize("rank", [8, 128])
 def test_one_sm_gemm_kernel(sess, rank):
     """The one-SM tensor-core kernel (kernel variant 3) on ranks at both ends."""
