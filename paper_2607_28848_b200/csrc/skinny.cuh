@@ -540,8 +540,10 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
 #pragma unroll
         for (int j = 0; j < 4; ++j)
           if (sp[j]) {     // activation save of rows that are not block-saved: they pass through here exactly once
-            *reinterpret_cast<uint4*>(sp[j] + ko) = x[j][0];
-            *reinterpret_cast<uint4*>(sp[j] + ko + 8) = x[j][1];
+            // this thread's 32 contiguous bytes of the row as one 256-bit store (a whole sector)
+            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(sp[j] + ko),
+                         "r"(x[j][0].x), "r"(x[j][0].y), "r"(x[j][0].z), "r"(x[j][0].w),
+                         "r"(x[j][1].x), "r"(x[j][1].y), "r"(x[j][1].z), "r"(x[j][1].w) : "memory");
           }
         // rows past the item's end were not copied: keep their stale bytes out of the MMA
 #pragma unroll
