@@ -38,13 +38,13 @@ struct PbdArgs {
 };
 
 // One warp writes all chunks of one row: `vals` = the row's R fp32 values (nullptr: all zero).
+// The table entries of the row (first group slot of its tile, groups of the tile, the row's own
+// group or -1) are passed in, so that a caller can fetch them long before the values exist.
 template <int R>
-__device__ __forceinline__ void pbd_write_row(const PbdArgs& pa, int row, const float* vals, float sc, int lane) {
-  const int tile = row >> 8, rl = row & 255;
-  const int goff = pa.tile2_grp_off[tile];
-  const int G = pa.tile2_grp_off[tile + 1] - goff;
+__device__ __forceinline__ void pbd_write_row_at(const PbdArgs& pa, int row, int goff, int G, int g, const float* vals,
+                                                 float sc, int lane) {
+  const int rl = row & 255;
   const int LC = (G * R + 63) / 64;
-  const int g = vals ? pa.row_grp2[row] : -1;
   for (int piece = lane; piece < LC * 8; piece += 32) {
     const int c = piece >> 3, kcol = piece * 8;          // chunk, first low-rank column of the piece
     uint4 v = make_uint4(0, 0, 0, 0);
@@ -57,6 +57,13 @@ __device__ __forceinline__ void pbd_write_row(const PbdArgs& pa, int row, const 
     __nv_bfloat16* dst = pa.pbd + ((size_t)(2 * goff + c) * 256 + rl) * 64 + (piece & 7) * 8;
     *reinterpret_cast<uint4*>(dst) = v;
   }
+}
+
+template <int R>
+__device__ __forceinline__ void pbd_write_row(const PbdArgs& pa, int row, const float* vals, float sc, int lane) {
+  const int tile = row >> 8;
+  const int goff = pa.tile2_grp_off[tile];
+  pbd_write_row_at<R>(pa, row, goff, pa.tile2_grp_off[tile + 1] - goff, vals ? pa.row_grp2[row] : -1, vals, sc, lane);
 }
 
 struct ShrinkArgs {
@@ -447,7 +454,8 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
     // flush-time values fetched when the item starts: element idx = tid + 256 k of the item's
     // [rows][R] result belongs to row idx / R
     int my_row[RB], my_save[RB];
-    float my_scale = 1.0f;
+    float my_scale = 1.0f, pb_scale = 1.0f;
+    int pb_row[32 / STREAM_WARPS], pb_goff[32 / STREAM_WARPS], pb_G[32 / STREAM_WARPS], pb_g[32 / STREAM_WARPS];
     // this thread's pieces of a K-block: elements 16c .. 16c+15 of the block
 #ifdef MLORA_TIMELINE
     if (tl_on) MLORA_TL_SET(1, tl_clock() - tl0);
@@ -492,6 +500,20 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
           my_save[k] = (r < cur_nrows && cur_saves) ? cur_saves[r] : -1;
         }
         my_scale = a.scale ? a.scale[cur_adapter] : 1.0f;
+        if (a.pbd.pbd) {     // table entries of the rows whose operand chunks this warp writes at the flush
+          pb_scale = a.pbd.scale ? a.pbd.scale[cur_adapter] : 1.0f;
+#pragma unroll
+          for (int j = 0; j < 32 / STREAM_WARPS; ++j) {
+            const int r = warp + STREAM_WARPS * j;
+            pb_row[j] = r < cur_nrows ? cur_rows[r] : -1;
+            if (pb_row[j] >= 0) {
+              const int tile = pb_row[j] >> 8;
+              pb_goff[j] = a.pbd.tile2_grp_off[tile];
+              pb_G[j] = a.pbd.tile2_grp_off[tile + 1] - pb_goff[j];
+              pb_g[j] = a.pbd.row_grp2[pb_row[j]];
+            }
+          }
+        }
       }
 #ifdef MLORA_TIMELINE
       const long long tw0 = tl_clock();
@@ -649,8 +671,10 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
         if (c0 != c1 && threadIdx.x == 0) a.counters[this_item] = 0;    // ready for the next launch
         if (a.pbd.pbd) {
           asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");  // fin[] complete
-          for (int r = warp; r < cur_nrows; r += STREAM_WARPS)
-            pbd_write_row<R>(a.pbd, cur_rows[r], fin[r], a.pbd.scale ? a.pbd.scale[cur_adapter] : 1.0f, lane);
+#pragma unroll
+          for (int j = 0; j < 32 / STREAM_WARPS; ++j)
+            if (pb_row[j] >= 0)
+              pbd_write_row_at<R>(a.pbd, pb_row[j], pb_goff[j], pb_G[j], pb_g[j], fin[warp + STREAM_WARPS * j], pb_scale, lane);
         }
       }
       asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");      // red[] and fin[] are reused by the next item
