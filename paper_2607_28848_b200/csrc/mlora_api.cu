@@ -57,6 +57,8 @@ struct mlora_ctx {
   __nv_bfloat16* ws_pbd = nullptr;   // block-diagonal low-rank operand: [2 * ws_pbd_groups * 256, 64] bf16
   int64_t ws_pbd_groups = 0;
   float* ws_splitk = nullptr;        // fp32 partial products of a K-split GEMM (fixed size, see kSplitKBytes)
+  float* ws_gpart = nullptr;         // row-split gradient groups: [sm_count][32][512] fp32 partial sums
+  int32_t* ws_gcounters = nullptr;   // [sm_count] arrival counters of those groups, zero between launches
   std::vector<PlanBuf> plan_pool;    // released buffers of stream-ordered plans
   int64_t launches = 0;
   int32_t gemm_path = 0;
@@ -365,7 +367,22 @@ mlora_status_t launch_grad_stream2_d(mlora_ctx* ctx, const mlora_plan* p, const 
   g.slot_adapter = p->slot_adapter; g.slot_blk_off = p->slot_blk_off; g.blk_row0 = p->blk_row0; g.blk_nrows = p->blk_nrows;
   g.n_slots = n_slots; g.status = ctx->status_dev;
   const int groups = n_slots * (g.prob[0].n_strips + g.prob[1].n_strips);
-  const int grid = groups < ctx->sm_count ? groups : ctx->sm_count;
+  // One or two fine-tuning adapters leave most SMs without a group: the row blocks of each slot are
+  // then dealt out over several CTAs per group (at most one CTA per SM in all, so the partial sums
+  // fit the context's workspace), and the last CTA of a group adds the parts in index order.
+  int parts = 1;
+  if (2 * groups <= ctx->sm_count) {
+    int max_blocks = 1;
+    for (int sl = 0; sl < n_slots; ++sl) {
+      const int nb = p->h.slot_blk_off[sl + 1] - p->h.slot_blk_off[sl];
+      max_blocks = nb > max_blocks ? nb : max_blocks;
+    }
+    parts = ctx->sm_count / groups;
+    parts = parts < max_blocks ? parts : max_blocks;
+  }
+  g.n_parts = parts; g.part_ws = ctx->ws_gpart; g.part_counters = ctx->ws_gcounters;
+  const int units = groups * parts;
+  const int grid = units < ctx->sm_count ? units : ctx->sm_count;
   if (cancelled(ctx)) return MLORA_CANCELLED;
   LaunchScope scope(ctx, st, KIND_GRAD);
   launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(STREAM_THREADS), smem, st, tQ0, tQ1, g);
@@ -751,8 +768,12 @@ mlora_status_t mlora_create(mlora_ctx** out, int device) {
   c->encode = reinterpret_cast<EncodeTiledFn>(fn);
   if (cudaMalloc(&c->status_dev, sizeof(int32_t)) != cudaSuccess ||
       cudaMalloc(&c->ws_splitk, kSplitKBytes) != cudaSuccess ||
+      cudaMalloc(&c->ws_gpart, (size_t)c->sm_count * 32 * 512 * sizeof(float)) != cudaSuccess ||
+      cudaMalloc(&c->ws_gcounters, (size_t)c->sm_count * sizeof(int32_t)) != cudaSuccess ||
+      cudaMemset(c->ws_gcounters, 0, (size_t)c->sm_count * sizeof(int32_t)) != cudaSuccess ||
       cudaMemset(c->status_dev, 0, sizeof(int32_t)) != cudaSuccess) {
-    delete c;
+    cudaGetLastError();
+    mlora_destroy(c);       // frees whatever was allocated
     return MLORA_ERR_CUDA;
   }
   *out = c;
@@ -800,6 +821,8 @@ void mlora_destroy(mlora_ctx* c) {
   cudaFree(c->ws_counters);
   cudaFree(c->ws_pbd);
   cudaFree(c->ws_splitk);
+  cudaFree(c->ws_gpart);
+  cudaFree(c->ws_gcounters);
   for (PlanBuf& b : c->plan_pool) free_plan_buf(b);
   delete c;
 }

@@ -858,6 +858,13 @@ struct GradStreamArgs {
   const int32_t* blk_nrows;
   int32_t n_slots;
   int32_t* status;
+  // Few groups for the SMs there are (one or two fine-tuning adapters): the row blocks of a slot are
+  // dealt out over n_parts CTAs per group; each leaves its fp32 sums in part_ws[group * n_parts +
+  // part][16 MB][strip width], and the CTA that arrives last at part_counters[group] adds the parts
+  // in index order (so the result does not depend on who was last) and writes the gradient.
+  int32_t n_parts;             // >= 1
+  float* part_ws;
+  int32_t* part_counters;      // [groups], zero between launches
 };
 
 template <int MB, bool DROP, int CB>
@@ -877,6 +884,7 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
   __shared__ __align__(8) uint64_t bars[2 * S];
   __shared__ int stage_meta[S][2];     // {first compact row, rows | last-tile-of-group flag << 16} of the staged tile
   __shared__ int abort_word;
+  __shared__ int part_is_last;
   volatile int* abort_flag = &abort_word;
   const int R = ga.R;
 
@@ -908,16 +916,25 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
   __syncthreads();
   const int groups0 = ga.n_slots * ga.prob[0].n_strips;
   const int n_groups = groups0 + (ga.n_problems > 1 ? ga.n_slots * ga.prob[1].n_strips : 0);
+  const int NP = ga.n_parts;
+  const int n_units = n_groups * NP;       // unit = group * NP + part
 
   if (warp == STREAM_WARPS) {
     // ======================= producer =======================
     // the plan's tables are not written by the kernel before this one: the first group's entries
     // are fetched while that kernel may still be running
+    // the blocks [b0, b1) of a slot's blocks [s_begin, s_end) that part `part` of NP takes
+    auto part_range = [&](int s_begin, int s_end, int part, int& b0, int& b1) {
+      const int per = (s_end - s_begin + NP - 1) / NP;
+      b0 = min(s_end, s_begin + part * per);
+      b1 = min(s_end, b0 + per);
+    };
     int first_b_begin = 0, first_b_end = 0, first_row0 = 0, first_nrows = 0;
-    if (lane == 0 && (int)blockIdx.x < n_groups) {
-      const int pi = (int)blockIdx.x >= groups0 ? 1 : 0;
-      const int slot = ((int)blockIdx.x - pi * groups0) / ga.prob[pi].n_strips;
-      first_b_begin = ga.slot_blk_off[slot]; first_b_end = ga.slot_blk_off[slot + 1];
+    if (lane == 0 && (int)blockIdx.x < n_units) {
+      const int grp0 = (int)blockIdx.x / NP;
+      const int pi = grp0 >= groups0 ? 1 : 0;
+      const int slot = (grp0 - pi * groups0) / ga.prob[pi].n_strips;
+      part_range(ga.slot_blk_off[slot], ga.slot_blk_off[slot + 1], (int)blockIdx.x % NP, first_b_begin, first_b_end);
       if (first_b_begin < first_b_end) { first_row0 = ga.blk_row0[first_b_begin]; first_nrows = ga.blk_nrows[first_b_begin]; }
     }
     ptx::grid_dependency_wait();
@@ -925,16 +942,17 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
     if (lane == 0) {
       uint32_t i = 0;
       bool ok = true;
-      for (int grp = blockIdx.x; grp < n_groups && ok; grp += gridDim.x) {
+      for (int un = blockIdx.x; un < n_units && ok; un += gridDim.x) {
+        const int grp = un / NP;
         const int pi = grp >= groups0 ? 1 : 0;
         const GradProblem& pr = ga.prob[pi];
         const CUtensorMap* tmQ = pi ? &tmQ1 : &tmQ0;
         const int gl = grp - pi * groups0;
         const int slot = gl / pr.n_strips, strip = gl % pr.n_strips;
-        const bool first = grp == (int)blockIdx.x;
-        const int b_begin = first ? first_b_begin : ga.slot_blk_off[slot];
-        const int b_end = first ? first_b_end : ga.slot_blk_off[slot + 1];
-        if (b_begin == b_end) {            // a slot without rows: an empty last tile, so that its gradient is still written
+        const bool first = un == (int)blockIdx.x;
+        int b_begin = first_b_begin, b_end = first_b_end;
+        if (!first) part_range(ga.slot_blk_off[slot], ga.slot_blk_off[slot + 1], un % NP, b_begin, b_end);
+        if (b_begin == b_end) {            // no rows (an empty slot, or a part past the slot's blocks): an empty last tile, so that the sums are still written
           const int st = i % S;
           if (!(ok = stream_wait(bar_empty(st), ((i / S) & 1) ^ 1, abort_flag, ga.status))) break;
           stage_meta[st][0] = 0;
@@ -978,7 +996,8 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
     float acc[MB][8][4];
     uint32_t i = 0;
     bool ok = true;
-    for (int grp = blockIdx.x; grp < n_groups && ok; grp += gridDim.x) {
+    for (int un = blockIdx.x; un < n_units && ok; un += gridDim.x) {
+      const int grp = un / NP;
       const int pi = grp >= groups0 ? 1 : 0;
       const GradProblem& pr = ga.prob[pi];
       const int gl = grp - pi * groups0;
@@ -1068,7 +1087,7 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
       if (!ok) break;
 #ifdef MLORA_TIMELINE
       const long long tf0 = tl_clock();
-      if (tl_on && grp + (int)gridDim.x >= n_groups) MLORA_TL_SET(5, tf0 - tl0);
+      if (tl_on && un + (int)gridDim.x >= n_units) MLORA_TL_SET(5, tf0 - tl0);
 #endif
       // ---- group done: this warp's 16 (32) x 64 block goes from registers to the gradient ----
       // The n index g of the MMA was mapped to piece g of a row, so for thread (g, c) accumulator
@@ -1096,7 +1115,50 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
         }
         asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");   // red[] is reused by the next group
       }
-      if (active && half == 0) {
+      bool write_out = true;
+      if (NP > 1) {        // row-split group: leave this part's sums, the last arrival adds all parts in index order
+        if (active && half == 0) {
+          float* mine = ga.part_ws + (size_t)un * (RMAX * GW_COLS);
+#pragma unroll
+          for (int m = 0; m < MB; ++m)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int ql = m * 16 + g + ((e >> 1) ? 8 : 0);
+              float4* dst = reinterpret_cast<float4*>(mine + (size_t)ql * GW_COLS + cblk * 64 + 8 * (2 * c + (e & 1)));
+              dst[0] = make_float4(acc[m][0][e], acc[m][1][e], acc[m][2][e], acc[m][3][e]);
+              dst[1] = make_float4(acc[m][4][e], acc[m][5][e], acc[m][6][e], acc[m][7][e]);
+            }
+        }
+        __threadfence();
+        asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");
+        if (threadIdx.x == 0) part_is_last = (atomicAdd(ga.part_counters + grp, 1) == NP - 1);
+        asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");
+        write_out = part_is_last != 0;
+        if (write_out) {
+          __threadfence();
+          if (active && half == 0) {
+#pragma unroll
+            for (int m = 0; m < MB; ++m)
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int ql = m * 16 + g + ((e >> 1) ? 8 : 0);
+                float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
+                for (int pp = 0; pp < NP; ++pp) {
+                  const float4* src = reinterpret_cast<const float4*>(
+                      ga.part_ws + ((size_t)grp * NP + pp) * (RMAX * GW_COLS) + (size_t)ql * GW_COLS + cblk * 64 + 8 * (2 * c + (e & 1)));
+                  const float4 a0 = __ldcg(src), a1 = __ldcg(src + 1);
+                  lo.x += a0.x; lo.y += a0.y; lo.z += a0.z; lo.w += a0.w;
+                  hi.x += a1.x; hi.y += a1.y; hi.z += a1.z; hi.w += a1.w;
+                }
+                acc[m][0][e] = lo.x; acc[m][1][e] = lo.y; acc[m][2][e] = lo.z; acc[m][3][e] = lo.w;
+                acc[m][4][e] = hi.x; acc[m][5][e] = hi.y; acc[m][6][e] = hi.z; acc[m][7][e] = hi.w;
+              }
+          }
+          if (threadIdx.x == 0) ga.part_counters[grp] = 0;       // ready for the next launch
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");   // part_is_last is reused by the next group
+      }
+      if (write_out && active && half == 0) {
 #pragma unroll
         for (int m = 0; m < MB; ++m)
 #pragma unroll

@@ -396,6 +396,37 @@ def test_accumulate_and_optional_outputs(sess):
     run2.close()
 
 
+@pytest.mark.parametrize("rank", [8, 16, 32])
+@pytest.mark.parametrize("lens", [(1100, 40), (2048,), (256,), (70, 700, 3)])
+def test_gradient_groups_split_over_rows(sess, rank, lens):
+    """One to three fine-tuning adapters leave the gradient kernel fewer (slot, strip) groups than
+    half the SMs: the row blocks of a slot are then dealt out over several CTAs per group and the
+    last one to arrive adds the partial sums in index order.  Slots of very different sizes (parts
+    without any block), overwrite and accumulate, and bit-identical results from run to run."""
+    segs, row = [(0, 37, 3, 0)], 37
+    for a, n in enumerate(lens):
+        segs.append((row, n, a, 1))
+        row += n
+    segs.append((row, 20, 0, 0))
+    row += 20
+    w = synth.Workload("few_slots", 512, 1024, rank, 4, "bf16", row, synth.segments_array(segs), seed=300 + rank)
+    t = synth.make_tensors(w)
+    run = run_and_check(sess, w, t, blocked=True)
+    run = LayerRun(sess, "bf16", t, w.segments, w.n_rows)
+    run.forward()
+    outs = []
+    for _ in range(3):
+        run.backward(accumulate=False)
+        outs.append((run.dA.clone(), run.dB.clone()))
+    for dA, dB in outs[1:]:
+        assert torch.equal(dA, outs[0][0]) and torch.equal(dB, outs[0][1])
+    run.backward(accumulate=True, want_dx=False)
+    assert_close("dA x2", run.host(run.dA), 2 * run.host(outs[0][0]), 1e-5)
+    assert_close("dB x2", run.host(run.dB), 2 * run.host(outs[0][1]), 1e-5)
+    assert run.status() == mb.MLORA_OK
+    run.close()
+
+
 def test_strided_inputs_and_outputs(sess):
     w = synth.random_workload(22, 128, 256, 16, 3, 200, max_seg=70)
     t = synth.make_tensors(w)
