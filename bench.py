@@ -288,6 +288,17 @@ def main():
         sampler.mark_stop()
     gpu_launches = mb.mlora_launch_count(sess.ctx) - l0
     ms_total = replicas.max_over_ranks(ev0.elapsed_time(ev1), sess.device)     # slowest rank
+    # Spread of single steps (median and best of up to 50 more steps, one event between steps):
+    # reported beside the headline mean, never instead of it.
+    stat_n = max(1, min(args.steps, 50))
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(stat_n + 1)]
+    marks[0].record()
+    for i in range(stat_n):
+        step()
+        marks[i + 1].record()
+    torch.cuda.synchronize()
+    step_ms = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(stat_n))
+    step_stats = {"steps": stat_n, "median_ms": step_ms[stat_n // 2], "best_ms": step_ms[0]}
     # Per-kernel durations: the same steps once more, now with the library recording a CUDA event
     # pair around every launch (which also switches off the overlap of a kernel's set-up with its
     # predecessor's tail, so each pair times one whole kernel).  Kept out of the region above so
@@ -450,6 +461,7 @@ def main():
                                 "frac_of_burst_peak": tot_flops / (peaks["bf16_tflops"] * 1e12) * 1e3 / ms_per_step,
                                 "frac_of_sustained_peak": tot_flops / (peaks["bf16_tflops_sustained"] * 1e12) * 1e3 / ms_per_step},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches), "device_status": int(status),
+        "step_stats": step_stats,
         "roofline": roofline, "kernels": kernels,
     }
     if not args.no_cpu_baseline and world == 1:

@@ -589,11 +589,7 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
             const uint32_t rb[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
 #pragma unroll
             for (int s = 0; s < 4; ++s) {
-#ifdef MLORA_EXP_NOMMA
-              acc[m][n][0] += __uint_as_float(ra[2 * s] ^ rb[2 * s] ^ ra[2 * s + 1] ^ rb[2 * s + 1] ^ rp[2 * s] ^ rp[2 * s + 1]);
-#else
               ptx::mma_bf16_16816(acc[m][n], ra[2 * s], rb[2 * s], ra[2 * s + 1], rb[2 * s + 1], rp[2 * s], rp[2 * s + 1]);
-#endif
             }
           }
         }
