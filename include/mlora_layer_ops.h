@@ -54,10 +54,17 @@ mlora_status_t mlora_add(const void* a, const void* b, void* out, int64_t n, voi
  * q, o bf16 [n_rows, n_heads * d_head] (row strides ldq, ldo), k, v bf16 [n_rows, n_kv * d_head];
  * seq_start[i] = first row of row i's sequence, seq_end[i] = one past its last row (int32 [n_rows]; the
  * rows of a sequence are consecutive); lse fp32 [n_rows, n_heads] receives log(sum_j exp(s_ij)), which the
- * backward needs.  d_head is 64 or 128; n_heads a multiple of n_kv. */
+ * backward needs.  d_head is 64 or 128 (128: tcgen05 tensor-core kernel, 64: CUDA cores); n_heads a multiple
+ * of n_kv; seq_start must not decrease from row to row (sequences are stored one after the other). */
 mlora_status_t mlora_attention_forward(const void* q, int64_t ldq, const void* k, int64_t ldk, const void* v, int64_t ldv,
                                        void* o, int64_t ldo, float* lse, const int32_t* seq_start, const int32_t* seq_end,
                                        int32_t n_rows, int32_t n_heads, int32_t n_kv, int32_t d_head, void* cuda_stream);
+
+/* The forward for d_head = 128 runs on the tensor cores with bounded waits inside the kernel; a wait
+ * that runs out makes the kernel return early and leaves MLORA_ERR_DEVICE_TIMEOUT in a device status
+ * word.  This call synchronises the stream, returns that word (MLORA_OK when nothing happened) and
+ * clears it.  The outputs of a call that timed out are undefined. */
+mlora_status_t mlora_layer_ops_poll_status(void* cuda_stream);
 
 /* Gradients of the above for a given dO: dq like q, dk and dv like k and v (each element written once; the
  * sums over the query heads that share a kv head are inside).  o and lse are the forward's outputs. */

@@ -21,6 +21,7 @@
 #include "skinny.cuh"
 #include "glue.cuh"
 #include "attention.cuh"
+#include "attention_tc.cuh"
 #include "mlora_layer_ops.h"
 
 using namespace mlora;
@@ -1269,6 +1270,41 @@ mlora_status_t mlora_add(const void* a, const void* b, void* out, int64_t n, voi
   return launched();
 }
 
+// Head size 128: the tcgen05 kernel.  The layer pieces have no context object, so the tensor-map
+// encoder is looked up once per process here.
+static mlora_status_t attention_forward_tc(const void* q, int64_t ldq, const void* k, int64_t ldk, const void* v,
+                                           int64_t ldv, void* o, int64_t ldo, float* lse, const int32_t* seq_start,
+                                           int32_t n_rows, int32_t n_heads, int32_t n_kv, cudaStream_t st) {
+  static mlora_ctx enc;            // only its encoder entry is used
+  static bool enc_ok = [] {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) != cudaSuccess ||
+        qr != cudaDriverEntryPointSuccess || !fn)
+      return false;
+    enc.encode = reinterpret_cast<EncodeTiledFn>(fn);
+    return true;
+  }();
+  if (!enc_ok) return MLORA_ERR_CUDA;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MLORA_ERR_CUDA;
+  static bool attr_set_dev[kMaxDevices] = {};
+  if (!attr_set_dev[dev]) {
+    if (cudaFuncSetAttribute(attn_tc::forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)attn_tc::SMEM_BYTES) != cudaSuccess)
+      return MLORA_ERR_CUDA;
+    attr_set_dev[dev] = true;
+  }
+  CUtensorMap tQ, tK, tV;
+  mlora_status_t s;
+  if ((s = make_tmap_bf16(&enc, &tQ, q, (uint64_t)n_heads * 128, n_rows, ldq, 64, 128)) != MLORA_OK) return s;
+  if ((s = make_tmap_bf16(&enc, &tK, k, (uint64_t)n_kv * 128, n_rows, ldk, 64, 128)) != MLORA_OK) return s;
+  if ((s = make_tmap_bf16_blocked(&enc, &tV, v, n_rows, (uint64_t)n_kv * 128, ldv, 64, 2)) != MLORA_OK) return s;
+  attn_tc::Args a{(__nv_bfloat16*)o, ldo, lse, seq_start, n_rows, n_heads, n_kv, 1.4426950408889634f / sqrtf(128.0f)};
+  attn_tc::forward_kernel<<<dim3((n_rows + 127) / 128, n_heads), attn_tc::THREADS, attn_tc::SMEM_BYTES, st>>>(tQ, tK, tV, a);
+  return launched();
+}
+
 mlora_status_t mlora_attention_forward(const void* q, int64_t ldq, const void* k, int64_t ldk, const void* v, int64_t ldv,
                                        void* o, int64_t ldo, float* lse, const int32_t* seq_start, const int32_t* seq_end,
                                        int32_t n_rows, int32_t n_heads, int32_t n_kv, int32_t d_head, void* cuda_stream) {
@@ -1278,13 +1314,24 @@ mlora_status_t mlora_attention_forward(const void* q, int64_t ldq, const void* k
   if (ldq % 8 || ldk % 8 || ldv % 8 || ldo % 8 || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o))
     return MLORA_ERR_UNSUPPORTED;
   if (n_rows == 0) return MLORA_OK;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (d_head == 128) return attention_forward_tc(q, ldq, k, ldk, v, ldv, o, ldo, lse, seq_start, n_rows, n_heads, n_kv, st);
   attn::AttnArgs a{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, ldq, ldk, ldv,
                    seq_start, seq_end, n_rows, n_heads, n_kv, 1.0f / sqrtf((float)d_head)};
   const int blocks = (int)(((int64_t)n_rows * n_heads + 7) / 8);
-  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-  if (d_head == 128) attn::forward_kernel<32><<<blocks, 256, 0, st>>>(a, (__nv_bfloat16*)o, ldo, lse);
-  else attn::forward_kernel<16><<<blocks, 256, 0, st>>>(a, (__nv_bfloat16*)o, ldo, lse);
+  attn::forward_kernel<16><<<blocks, 256, 0, st>>>(a, (__nv_bfloat16*)o, ldo, lse);
   return launched();
+}
+
+mlora_status_t mlora_layer_ops_poll_status(void* cuda_stream) {
+  if (cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return MLORA_ERR_CUDA;
+  int32_t v = 0;
+  if (cudaMemcpyFromSymbol(&v, attn_tc::g_status, sizeof v) != cudaSuccess) return MLORA_ERR_CUDA;
+  if (v != 0) {
+    const int32_t zero = 0;
+    if (cudaMemcpyToSymbol(attn_tc::g_status, &zero, sizeof zero) != cudaSuccess) return MLORA_ERR_CUDA;
+  }
+  return (mlora_status_t)v;
 }
 
 mlora_status_t mlora_attention_backward(const void* q, int64_t ldq, const void* k, int64_t ldk, const void* v, int64_t ldv,

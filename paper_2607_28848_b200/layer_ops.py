@@ -6,7 +6,8 @@ import ctypes
 from . import binding as _b
 
 EXPORTS = ("mlora_rmsnorm_forward", "mlora_rmsnorm_backward", "mlora_rope", "mlora_swiglu_forward",
-           "mlora_swiglu_backward", "mlora_add", "mlora_attention_forward", "mlora_attention_backward")
+           "mlora_swiglu_backward", "mlora_add", "mlora_attention_forward", "mlora_attention_backward",
+           "mlora_layer_ops_poll_status")
 _ready = False
 
 
@@ -25,6 +26,7 @@ def _lib():
     lib.mlora_attention_forward.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, vp, vp, i32, i32, i32, i32, vp]
     lib.mlora_attention_backward.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64, vp, i64, vp, i64,
                                              vp, vp, i32, i32, i32, i32, vp]
+    lib.mlora_layer_ops_poll_status.argtypes = [vp]
     for name in EXPORTS:
         getattr(lib, name).restype = ctypes.c_int
     _ready = True
@@ -78,3 +80,8 @@ def mlora_attention_backward(q, k, v, o, lse, dO, dq, dk, dv, seq_start, seq_end
                                               _p(lse), _p(dO), dO.stride(0), _p(dq), dq.stride(0), _p(dk), dk.stride(0),
                                               _p(dv), dv.stride(0), _p(seq_start), _p(seq_end), q.shape[0], int(n_heads),
                                               int(n_kv), int(d_head), _b._stream_ptr(stream)), "mlora_attention_backward")
+
+
+def mlora_layer_ops_poll_status(stream=None) -> int:
+    """Synchronises the stream; returns and clears the status word of the layer pieces' bounded waits."""
+    return int(_lib().mlora_layer_ops_poll_status(_b._stream_ptr(stream)))

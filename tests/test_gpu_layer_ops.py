@@ -106,6 +106,40 @@ def test_attention_forward_and_backward(heads, kv, dh):
     close(dv, vr.grad.reshape(T, kv * dh), tol=2e-2)
 
 
+@pytest.mark.parametrize("lens", [[1], [127], [128], [129], [300, 5, 1, 1, 200], [64] * 9, [1] * 140, [700]])
+@pytest.mark.parametrize("heads,kv", [(4, 2), (3, 1)])
+def test_attention_forward_tensor_core_kernel(lens, heads, kv):
+    """Head size 128 (the tcgen05 kernel): query tiles that hold one sequence, several sequences or a
+    ragged last tile; sequences longer than one key block (online softmax over several blocks);
+    outputs and log-sum-exp against the fp64 definition."""
+    dh = 128
+    g = torch.Generator().manual_seed(sum(lens) * 10 + heads)
+    T = sum(lens)
+    q = bf(torch.randn(T, heads * dh, generator=g) * 2.0).to(DEV)     # a wider score range than unit inputs give
+    k = bf(torch.randn(T, kv * dh, generator=g)).to(DEV)
+    v = bf(torch.randn(T, kv * dh, generator=g)).to(DEV)
+    start, end, seqs, r = [], [], [], 0
+    for n in lens:
+        start += [r] * n; end += [r + n] * n; seqs.append(list(range(r, r + n))); r += n
+    ss, se = torch.tensor(start, dtype=torch.int32, device=DEV), torch.tensor(end, dtype=torch.int32, device=DEV)
+    o = torch.full_like(q, float("nan"))
+    lse = torch.full((T, heads), float("nan"), dtype=torch.float32, device=DEV)
+    mo.mlora_attention_forward(q, k, v, o, lse, ss, se, heads, kv, dh)
+    assert mo.mlora_layer_ops_poll_status() == 0
+    qr, kr, vr = (x.double().cpu() for x in (q, k, v))
+    ref = lo.attention(qr.reshape(T, heads, dh), kr.reshape(T, kv, dh), vr.reshape(T, kv, dh), seqs)
+    close(o, ref.reshape(T, heads * dh))
+    # log-sum-exp of the scaled scores of every row, from the definition
+    rep = heads // kv
+    lse_ref = torch.empty(T, heads, dtype=torch.float64)
+    for rows in seqs:
+        for h in range(heads):
+            sc = qr.reshape(T, heads, dh)[rows, h] @ kr.reshape(T, kv, dh)[rows, h // rep].T / dh ** 0.5
+            sc = sc.masked_fill(torch.triu(torch.ones(len(rows), len(rows), dtype=torch.bool), 1), float("-inf"))
+            lse_ref[rows, h] = torch.logsumexp(sc, dim=1)
+    assert torch.allclose(lse.double().cpu(), lse_ref, rtol=0, atol=2e-3), float((lse.double().cpu() - lse_ref).abs().max())
+
+
 def test_argument_errors():
     x = torch.zeros(4, 12, dtype=torch.bfloat16, device=DEV)           # 12 is not a multiple of 8
     gain = torch.ones(12, device=DEV)
