@@ -1,7 +1,8 @@
 // Causal softmax attention inside the sequences of a packed batch, head size 128, on the
-// tcgen05 tensor cores (forward only; the gradients use the CUDA-core kernels of attention.cuh).
+// tcgen05 tensor cores: the forward kernel first, the two gradient kernels after it (head size 64
+// uses the CUDA-core kernels of attention.cuh).
 //
-// One CTA = one tile of 128 query rows of one head.  It walks the key rows from the first row of
+// Forward: one CTA = one tile of 128 query rows of one head.  It walks the key rows from the first row of
 // the tile's first sequence to the tile's last row in blocks of 128:
 //   warp 0 (one lane)  TMA producer: Q once; K and V blocks through a ring of two stages
 //   warp 1 (one lane)  MMA issuer:   S = Q K^T into tensor memory (columns 0..127), then, once the
@@ -247,6 +248,433 @@ forward_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   if (warp == 1) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+
+// =============================================================================================
+// Gradients, head size 128.  P is recomputed from the saved log-sum-exp (no running maximum is
+// needed), D[i] = sum_d dO[i, d] O[i, d], dS = P o (dP - D):
+//   dq kernel : CTA = (128 query rows, head).   Per key block: S = Q K^T and dP = dO V^T into tensor
+//               memory, the softmax threads (one query row each) write dS as a bf16 operand, and
+//               dQ += dS K accumulates in tensor memory over all key blocks.
+//   dkv kernel: CTA = (128 key rows, key-value head).  Per (query head of the group, query block):
+//               S^T = K Q^T and dP^T = V dO^T, the threads (one key row each) write P^T and dS^T,
+//               dV += P^T dO and dK += dS^T Q accumulate in tensor memory over all heads and blocks,
+//               so every element of dk and dv is written once.
+// A [rows][64] K-major tile (rows of 128 bytes, 128-byte swizzle) is byte for byte also the
+// MN-major operand whose K index is the row, so K, Q and dO are loaded once and used in both roles
+// (as an MN-major operand: descriptor start + 8 KiB per 64 rows, 16 KiB between the two 64-column
+// blocks).
+// =============================================================================================
+struct BwdArgs {
+  const __nv_bfloat16* o;  int64_t ldo;
+  const __nv_bfloat16* dO; int64_t lddo;
+  const float* lse;                         // [n_rows, n_heads]
+  const int32_t* seq_start;
+  const int32_t* seq_end;
+  __nv_bfloat16* dq; int64_t lddq;
+  __nv_bfloat16* dk; int64_t lddk;
+  __nv_bfloat16* dv; int64_t lddv;
+  int32_t n_rows, n_heads, n_kv;
+  float scale, scale_log2;
+};
+
+constexpr uint32_t DQ_SMEM_BYTES = 1024 + 2 * Q_BYTES + P_BYTES + STAGES * (K_BYTES + V_BYTES) + 256;
+constexpr uint32_t DKV_SMEM_BYTES = 1024 + 6 * Q_BYTES + 3 * 512 + 256;
+constexpr uint32_t BWD_TMEM_COLS = 512;
+
+// 32 columns of a row of a bf16 operand tile: pieces 4 (cc % 2) .. + 3 of K-block cc / 2
+__device__ __forceinline__ void store_row_chunk(uint32_t tile, int row, int cc, const uint32_t (&pk)[16]) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const uint32_t pc = (uint32_t)((cc & 1) * 4 + q);
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(tile + (uint32_t)row * 128u + (uint32_t)(cc >> 1) * 16384u + ((pc ^ (uint32_t)(row & 7)) << 4)),
+                 "r"(pk[4 * q]), "r"(pk[4 * q + 1]), "r"(pk[4 * q + 2]), "r"(pk[4 * q + 3]) : "memory");
+  }
+}
+
+// 128 x 128 x 128 product of two K-major tiles (two 64-wide K-blocks each) into d_tmem.
+__device__ __forceinline__ void mma_kk(uint32_t d_tmem, uint32_t a_tile, uint32_t b_tile, uint32_t first_acc) {
+  constexpr uint32_t idesc = ptx::make_idesc_bf16(BM, BN, false, false);
+  uint32_t acc = first_acc;
+#pragma unroll
+  for (int kb = 0; kb < 2; ++kb) {
+    const uint64_t ad = ptx::make_smem_desc(a_tile + kb * 16384, 16, 1024);
+    const uint64_t bd = ptx::make_smem_desc(b_tile + kb * 16384, 16, 1024);
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) {
+      ptx::umma_f16(d_tmem, ad + (uint64_t)(ks * 2), bd + (uint64_t)(ks * 2), idesc, acc);
+      acc = 1;
+    }
+  }
+}
+// d_tmem (+)= A B with A a K-major tile [128][128] (K = its 128 columns) and B a [128 rows][128
+// columns] tile read as the MN-major operand whose K index is the row.
+__device__ __forceinline__ void mma_kn(uint32_t d_tmem, uint32_t a_tile, uint32_t b_tile, uint32_t first_acc) {
+  constexpr uint32_t idesc = ptx::make_idesc_bf16(BM, DH, false, true);
+  uint32_t acc = first_acc;
+#pragma unroll
+  for (int kb = 0; kb < 2; ++kb) {
+    const uint64_t ad = ptx::make_smem_desc(a_tile + kb * 16384, 16, 1024);
+    const uint64_t bd = ptx::make_smem_desc(b_tile + kb * 8192, 16384, 1024);
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) {
+      ptx::umma_f16(d_tmem, ad + (uint64_t)(ks * 2), bd + (uint64_t)(ks * 128), idesc, acc);
+      acc = 1;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+backward_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmdO,
+                   const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const BwdArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - ptx::smem_u32(smem_raw));
+  const uint32_t sQ = base, sdO = base + Q_BYTES, sDS = base + 2 * Q_BYTES;
+  auto sK = [&](int s) { return base + 2 * Q_BYTES + P_BYTES + (uint32_t)s * (K_BYTES + V_BYTES); };
+  auto sV = [&](int s) { return sK(s) + K_BYTES; };
+  const uint32_t sBar = base + 2 * Q_BYTES + P_BYTES + STAGES * (K_BYTES + V_BYTES);
+  const uint32_t bar_q = sBar, bar_s = sBar + 8, bar_ds = sBar + 16, bar_done = sBar + 24;
+  auto bar_kv_full = [&](int s) { return sBar + 32u + 8u * s; };
+  auto bar_kv_empty = [&](int s) { return sBar + 48u + 8u * s; };
+  uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(gen + (sBar - base) + 64);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (sBar - base) + 72);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.x * BM, h = blockIdx.y;
+  const int hk = h / (a.n_heads / a.n_kv);
+  const int row_last = min(m0 + BM, a.n_rows) - 1;
+  const int kmin = a.seq_start[m0];
+  const int nblk = (row_last - kmin) / BN + 1;
+
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(bar_q, 1);
+    ptx::mbar_init(bar_s, 1);
+    ptx::mbar_init(bar_ds, BM);
+    ptx::mbar_init(bar_done, 1);
+    for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(bar_kv_full(s), 1); ptx::mbar_init(bar_kv_empty(s), 1); }
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmdO); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_u32(tmem_ptr_smem), BWD_TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_ptr_smem;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      ptx::mbar_arrive_expect_tx(bar_q, 2 * Q_BYTES);
+      ptx::tma_load_2d(sQ, &tmQ, h * DH, m0, bar_q);
+      ptx::tma_load_2d(sQ + 16384, &tmQ, h * DH + 64, m0, bar_q);
+      ptx::tma_load_2d(sdO, &tmdO, h * DH, m0, bar_q);
+      ptx::tma_load_2d(sdO + 16384, &tmdO, h * DH + 64, m0, bar_q);
+      for (int j = 0; j < nblk; ++j) {
+        const int s = j % STAGES;
+        if (!gemm_wait(bar_kv_empty(s), ((j / STAGES) & 1) ^ 1, abort_flag, &g_status)) break;
+        const int key0 = kmin + j * BN;
+        ptx::mbar_arrive_expect_tx(bar_kv_full(s), K_BYTES + V_BYTES);
+        ptx::tma_load_2d(sK(s), &tmK, hk * DH, key0, bar_kv_full(s));
+        ptx::tma_load_2d(sK(s) + 16384, &tmK, hk * DH + 64, key0, bar_kv_full(s));
+        ptx::tma_load_2d(sV(s), &tmV, hk * DH, key0, bar_kv_full(s));
+        ptx::tma_load_2d(sV(s) + 16384, &tmV, hk * DH + 64, key0, bar_kv_full(s));
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t tS = tmem_base, tP = tmem_base + 128, tDQ = tmem_base + 256;
+      bool ok = gemm_wait(bar_q, 0, abort_flag, &g_status);
+      for (int j = 0; j < nblk && ok; ++j) {
+        const int s = j % STAGES;
+        if (!(ok = gemm_wait(bar_kv_full(s), (j / STAGES) & 1, abort_flag, &g_status))) break;
+        ptx::tc_fence_after();
+        mma_kk(tS, sQ, sK(s), 0);             // S = Q K^T
+        mma_kk(tP, sdO, sV(s), 0);            // dP = dO V^T
+        ptx::umma_commit(bar_s);
+        if (!(ok = gemm_wait(bar_ds, j & 1, abort_flag, &g_status))) break;
+        ptx::tc_fence_after();
+        mma_kn(tDQ, sDS, sK(s), j > 0 ? 1u : 0u);    // dQ += dS K
+        ptx::umma_commit(bar_kv_empty(s));
+        if (j == nblk - 1) ptx::umma_commit(bar_done);
+      }
+    }
+    __syncwarp();
+  } else {
+    const int e = warp & 3;
+    const int row = e * 32 + lane;
+    const int i_abs = m0 + row;
+    const bool row_ok = i_abs < a.n_rows;
+    const int my_start = row_ok ? a.seq_start[i_abs] : 0x7fffffff;
+    const uint32_t tS = tmem_base + ((uint32_t)(e * 32) << 16), tP = tS + 128, tDQ = tS + 256;
+    float lse2 = 0.f, D = 0.f;
+    if (row_ok) {
+      lse2 = a.lse[(size_t)i_abs * a.n_heads + h] * 1.4426950408889634f;
+      const uint4* po = reinterpret_cast<const uint4*>(a.o + (size_t)i_abs * a.ldo + (size_t)h * DH);
+      const uint4* pd = reinterpret_cast<const uint4*>(a.dO + (size_t)i_abs * a.lddo + (size_t)h * DH);
+#pragma unroll 4
+      for (int k = 0; k < DH / 8; ++k) {
+        const uint4 x = po[k], y = pd[k];
+        const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          D = fmaf(__uint_as_float(xs[t] << 16), __uint_as_float(ys[t] << 16), D);
+          D = fmaf(__uint_as_float(xs[t] & 0xFFFF0000u), __uint_as_float(ys[t] & 0xFFFF0000u), D);
+        }
+      }
+    }
+    bool ok = true;
+    for (int j = 0; j < nblk; ++j) {
+      const int key0 = kmin + j * BN;
+      ok = __all_sync(0xffffffffu, gemm_wait(bar_s, j & 1, abort_flag, &g_status));
+      if (!ok) break;
+      ptx::tc_fence_after();
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t vs[32], vp[32];
+        ptx::tmem_ld_32x32b_x32(tS + cc * 32, vs);
+        ptx::tmem_ld_32x32b_x32(tP + cc * 32, vp);
+        ptx::tmem_ld_wait();
+        uint32_t pk[16];
+#pragma unroll
+        for (int k = 0; k < 32; k += 2) {
+          const int col = key0 + cc * 32 + k;
+          const float p0 = (col >= my_start && col <= i_abs) ? exp2f(__uint_as_float(vs[k]) * a.scale_log2 - lse2) : 0.f;
+          const float p1 = (col + 1 >= my_start && col + 1 <= i_abs) ? exp2f(__uint_as_float(vs[k + 1]) * a.scale_log2 - lse2) : 0.f;
+          pk[k >> 1] = ptx::pack_bf16(p0 * (__uint_as_float(vp[k]) - D), p1 * (__uint_as_float(vp[k + 1]) - D));
+        }
+        store_row_chunk(sDS, row, cc, pk);
+      }
+      ptx::fence_proxy_async_smem();
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(bar_ds);
+    }
+    if (ok) ok = __all_sync(0xffffffffu, gemm_wait(bar_done, 0, abort_flag, &g_status));
+    if (ok) {
+      ptx::tc_fence_after();
+      __nv_bfloat16* dst = a.dq + (size_t)i_abs * a.lddq + (size_t)h * DH;
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t v[32];
+        ptx::tmem_ld_32x32b_x32(tDQ + cc * 32, v);
+        ptx::tmem_ld_wait();
+        if (row_ok) {
+#pragma unroll
+          for (int k = 0; k < 32; k += 8) {
+            uint4 w;
+            w.x = ptx::pack_bf16(__uint_as_float(v[k]) * a.scale, __uint_as_float(v[k + 1]) * a.scale);
+            w.y = ptx::pack_bf16(__uint_as_float(v[k + 2]) * a.scale, __uint_as_float(v[k + 3]) * a.scale);
+            w.z = ptx::pack_bf16(__uint_as_float(v[k + 4]) * a.scale, __uint_as_float(v[k + 5]) * a.scale);
+            w.w = ptx::pack_bf16(__uint_as_float(v[k + 6]) * a.scale, __uint_as_float(v[k + 7]) * a.scale);
+            *reinterpret_cast<uint4*>(dst + cc * 32 + k) = w;
+          }
+        }
+      }
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, BWD_TMEM_COLS);
+  }
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+backward_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmdO,
+                    const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmK,
+                    const __grid_constant__ CUtensorMap tmV, const BwdArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - ptx::smem_u32(smem_raw));
+  const uint32_t sKt = base, sVt = base + Q_BYTES, sQ = base + 2 * Q_BYTES, sdO = base + 3 * Q_BYTES;
+  const uint32_t sOP = base + 4 * Q_BYTES;      // the O block, then P^T
+  const uint32_t sDS = base + 5 * Q_BYTES;
+  float* sL = reinterpret_cast<float*>(gen + 6 * Q_BYTES);            // per query of the block: lse * log2 e
+  float* sD = sL + 128;                                               // D
+  int* sQS = reinterpret_cast<int*>(sD + 128);                        // first row of the query's sequence
+  const uint32_t sBar = base + 6 * Q_BYTES + 3 * 512;
+  const uint32_t bar_kv = sBar, bar_s = sBar + 8, bar_p = sBar + 16, bar_done = sBar + 24;
+  const uint32_t bar_ld_full = sBar + 32, bar_ld_empty = sBar + 40, bar_tab = sBar + 48;
+  uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(gen + (sBar - base) + 64);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (sBar - base) + 72);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int k0 = blockIdx.x * BM, hk = blockIdx.y;
+  const int rep = a.n_heads / a.n_kv;
+  const int key_last = min(k0 + BM, a.n_rows) - 1;
+  const int qend = a.seq_end[key_last];                    // queries past the last key's sequence see none of these keys
+  const int nqb = (qend - k0 + BM - 1) / BM;               // query blocks start at the key tile's first row (causality)
+  const int n_it = rep * nqb;
+
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(bar_kv, 1);
+    ptx::mbar_init(bar_s, 1);
+    ptx::mbar_init(bar_p, BM);
+    ptx::mbar_init(bar_done, 1);
+    ptx::mbar_init(bar_ld_full, 1);
+    ptx::mbar_init(bar_ld_empty, 1);
+    ptx::mbar_init(bar_tab, BM);
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmQ); ptx::prefetch_tmap(&tmdO); ptx::prefetch_tmap(&tmO); ptx::prefetch_tmap(&tmK); ptx::prefetch_tmap(&tmV);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_u32(tmem_ptr_smem), BWD_TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_ptr_smem;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      ptx::mbar_arrive_expect_tx(bar_kv, 2 * Q_BYTES);
+      ptx::tma_load_2d(sKt, &tmK, hk * DH, k0, bar_kv);
+      ptx::tma_load_2d(sKt + 16384, &tmK, hk * DH + 64, k0, bar_kv);
+      ptx::tma_load_2d(sVt, &tmV, hk * DH, k0, bar_kv);
+      ptx::tma_load_2d(sVt + 16384, &tmV, hk * DH + 64, k0, bar_kv);
+      for (int it = 0; it < n_it; ++it) {
+        const int h = hk * rep + it / nqb, q0 = k0 + (it % nqb) * BM;
+        if (!gemm_wait(bar_ld_empty, (it & 1) ^ 1, abort_flag, &g_status)) break;
+        ptx::mbar_arrive_expect_tx(bar_ld_full, 3 * Q_BYTES);
+        ptx::tma_load_2d(sQ, &tmQ, h * DH, q0, bar_ld_full);
+        ptx::tma_load_2d(sQ + 16384, &tmQ, h * DH + 64, q0, bar_ld_full);
+        ptx::tma_load_2d(sdO, &tmdO, h * DH, q0, bar_ld_full);
+        ptx::tma_load_2d(sdO + 16384, &tmdO, h * DH + 64, q0, bar_ld_full);
+        ptx::tma_load_2d(sOP, &tmO, h * DH, q0, bar_ld_full);
+        ptx::tma_load_2d(sOP + 16384, &tmO, h * DH + 64, q0, bar_ld_full);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t tS = tmem_base, tP = tmem_base + 128, tDV = tmem_base + 256, tDK = tmem_base + 384;
+      bool ok = gemm_wait(bar_kv, 0, abort_flag, &g_status);
+      for (int it = 0; it < n_it && ok; ++it) {
+        if (!(ok = gemm_wait(bar_ld_full, it & 1, abort_flag, &g_status))) break;
+        ptx::tc_fence_after();
+        mma_kk(tS, sKt, sQ, 0);               // S^T = K Q^T
+        mma_kk(tP, sVt, sdO, 0);              // dP^T = V dO^T
+        ptx::umma_commit(bar_s);
+        if (!(ok = gemm_wait(bar_p, it & 1, abort_flag, &g_status))) break;
+        ptx::tc_fence_after();
+        mma_kn(tDV, sOP, sdO, it > 0 ? 1u : 0u);     // dV += P^T dO
+        mma_kn(tDK, sDS, sQ, it > 0 ? 1u : 0u);      // dK += dS^T Q
+        ptx::umma_commit(bar_ld_empty);
+        if (it == n_it - 1) ptx::umma_commit(bar_done);
+      }
+    }
+    __syncwarp();
+  } else {
+    const int e = warp & 3;
+    const int row = e * 32 + lane;                      // key row of the tile, and the query this thread prepares
+    const int j_abs = k0 + row;
+    const uint32_t tS = tmem_base + ((uint32_t)(e * 32) << 16), tP = tS + 128, tDV = tS + 256, tDK = tS + 384;
+    bool ok = true;
+    for (int it = 0; it < n_it; ++it) {
+      const int h = hk * rep + it / nqb, q0 = k0 + (it % nqb) * BM;
+      ok = __all_sync(0xffffffffu, gemm_wait(bar_ld_full, it & 1, abort_flag, &g_status));
+      if (!ok) break;
+      {   // query q0 + row: D from the staged dO and O rows (same swizzle, so piece by piece), lse, sequence start
+        const int i = q0 + row;
+        float D = 0.f;
+#pragma unroll
+        for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+          for (int pz = 0; pz < 8; ++pz) {
+            const uint32_t off = (uint32_t)kb * 16384u + (uint32_t)row * 128u + (uint32_t)pz * 16u;
+            uint4 x, y;
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(x.x), "=r"(x.y), "=r"(x.z), "=r"(x.w) : "r"(sOP + off));
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(y.x), "=r"(y.y), "=r"(y.z), "=r"(y.w) : "r"(sdO + off));
+            const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+              D = fmaf(__uint_as_float(xs[t] << 16), __uint_as_float(ys[t] << 16), D);
+              D = fmaf(__uint_as_float(xs[t] & 0xFFFF0000u), __uint_as_float(ys[t] & 0xFFFF0000u), D);
+            }
+          }
+        const bool q_ok = i < a.n_rows;
+        sD[row] = D;
+        sL[row] = q_ok ? a.lse[(size_t)i * a.n_heads + h] * 1.4426950408889634f : 0.f;
+        sQS[row] = q_ok ? a.seq_start[i] : 0x7fffffff;
+      }
+      // the block's tables are complete and every O row has been read once all 128 threads have
+      // arrived (an mbarrier with a bounded wait rather than bar.sync: a warp that gave up never arrives)
+      ptx::mbar_arrive(bar_tab);
+      ok = __all_sync(0xffffffffu, gemm_wait(bar_tab, it & 1, abort_flag, &g_status));
+      if (!ok) break;
+      ok = __all_sync(0xffffffffu, gemm_wait(bar_s, it & 1, abort_flag, &g_status));
+      if (!ok) break;
+      ptx::tc_fence_after();
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t vs[32], vp[32];
+        ptx::tmem_ld_32x32b_x32(tS + cc * 32, vs);
+        ptx::tmem_ld_32x32b_x32(tP + cc * 32, vp);
+        ptx::tmem_ld_wait();
+        uint32_t pp[16], pd[16];
+#pragma unroll
+        for (int k = 0; k < 32; k += 2) {
+          const int c0 = cc * 32 + k;
+          const int i0 = q0 + c0;
+          const float p0 = (j_abs <= i0 && j_abs >= sQS[c0]) ? exp2f(__uint_as_float(vs[k]) * a.scale_log2 - sL[c0]) : 0.f;
+          const float p1 = (j_abs <= i0 + 1 && j_abs >= sQS[c0 + 1]) ? exp2f(__uint_as_float(vs[k + 1]) * a.scale_log2 - sL[c0 + 1]) : 0.f;
+          pp[k >> 1] = ptx::pack_bf16(p0, p1);
+          pd[k >> 1] = ptx::pack_bf16(p0 * (__uint_as_float(vp[k]) - sD[c0]), p1 * (__uint_as_float(vp[k + 1]) - sD[c0 + 1]));
+        }
+        store_row_chunk(sOP, row, cc, pp);
+        store_row_chunk(sDS, row, cc, pd);
+      }
+      ptx::fence_proxy_async_smem();
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(bar_p);
+    }
+    if (ok) ok = __all_sync(0xffffffffu, gemm_wait(bar_done, 0, abort_flag, &g_status));
+    if (ok) {
+      ptx::tc_fence_after();
+      const bool key_ok = j_abs < a.n_rows;
+      __nv_bfloat16* dvp = a.dv + (size_t)j_abs * a.lddv + (size_t)hk * DH;
+      __nv_bfloat16* dkp = a.dk + (size_t)j_abs * a.lddk + (size_t)hk * DH;
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t v[32], w[32];
+        ptx::tmem_ld_32x32b_x32(tDV + cc * 32, v);
+        ptx::tmem_ld_32x32b_x32(tDK + cc * 32, w);
+        ptx::tmem_ld_wait();
+        if (key_ok) {
+#pragma unroll
+          for (int k = 0; k < 32; k += 8) {
+            uint4 x, y;
+            x.x = ptx::pack_bf16(__uint_as_float(v[k]), __uint_as_float(v[k + 1]));
+            x.y = ptx::pack_bf16(__uint_as_float(v[k + 2]), __uint_as_float(v[k + 3]));
+            x.z = ptx::pack_bf16(__uint_as_float(v[k + 4]), __uint_as_float(v[k + 5]));
+            x.w = ptx::pack_bf16(__uint_as_float(v[k + 6]), __uint_as_float(v[k + 7]));
+            y.x = ptx::pack_bf16(__uint_as_float(w[k]) * a.scale, __uint_as_float(w[k + 1]) * a.scale);
+            y.y = ptx::pack_bf16(__uint_as_float(w[k + 2]) * a.scale, __uint_as_float(w[k + 3]) * a.scale);
+            y.z = ptx::pack_bf16(__uint_as_float(w[k + 4]) * a.scale, __uint_as_float(w[k + 5]) * a.scale);
+            y.w = ptx::pack_bf16(__uint_as_float(w[k + 6]) * a.scale, __uint_as_float(w[k + 7]) * a.scale);
+            *reinterpret_cast<uint4*>(dvp + cc * 32 + k) = x;
+            *reinterpret_cast<uint4*>(dkp + cc * 32 + k) = y;
+          }
+        }
+      }
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, BWD_TMEM_COLS);
   }
 }
 

@@ -1270,13 +1270,13 @@ mlora_status_t mlora_add(const void* a, const void* b, void* out, int64_t n, voi
   return launched();
 }
 
-// Head size 128: the tcgen05 kernel.  The layer pieces have no context object, so the tensor-map
-// encoder is looked up once per process here.
-static mlora_status_t attention_forward_tc(const void* q, int64_t ldq, const void* k, int64_t ldk, const void* v,
-                                           int64_t ldv, void* o, int64_t ldo, float* lse, const int32_t* seq_start,
-                                           int32_t n_rows, int32_t n_heads, int32_t n_kv, cudaStream_t st) {
-  static mlora_ctx enc;            // only its encoder entry is used
-  static bool enc_ok = [] {
+}  // extern "C"
+
+// Head size 128: the tcgen05 kernels.  The layer pieces have no context object, so the tensor-map
+// encoder is looked up once per process here (only that entry of the object is used).
+static mlora_ctx* layer_ops_encoder() {
+  static mlora_ctx enc;
+  static bool ok = [] {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qr;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) != cudaSuccess ||
@@ -1285,25 +1285,66 @@ static mlora_status_t attention_forward_tc(const void* q, int64_t ldq, const voi
     enc.encode = reinterpret_cast<EncodeTiledFn>(fn);
     return true;
   }();
-  if (!enc_ok) return MLORA_ERR_CUDA;
+  return ok ? &enc : nullptr;
+}
+
+template <typename Kern>
+static mlora_status_t attn_tc_smem(Kern kern, uint32_t bytes, bool* done_dev) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MLORA_ERR_CUDA;
-  static bool attr_set_dev[kMaxDevices] = {};
-  if (!attr_set_dev[dev]) {
-    if (cudaFuncSetAttribute(attn_tc::forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)attn_tc::SMEM_BYTES) != cudaSuccess)
-      return MLORA_ERR_CUDA;
-    attr_set_dev[dev] = true;
+  if (!done_dev[dev]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) return MLORA_ERR_CUDA;
+    done_dev[dev] = true;
   }
-  CUtensorMap tQ, tK, tV;
+  return MLORA_OK;
+}
+
+static mlora_status_t attention_forward_tc(const void* q, int64_t ldq, const void* k, int64_t ldk, const void* v,
+                                           int64_t ldv, void* o, int64_t ldo, float* lse, const int32_t* seq_start,
+                                           int32_t n_rows, int32_t n_heads, int32_t n_kv, cudaStream_t st) {
+  mlora_ctx* enc = layer_ops_encoder();
+  if (!enc) return MLORA_ERR_CUDA;
+  static bool attr_dev[kMaxDevices] = {};
   mlora_status_t s;
-  if ((s = make_tmap_bf16(&enc, &tQ, q, (uint64_t)n_heads * 128, n_rows, ldq, 64, 128)) != MLORA_OK) return s;
-  if ((s = make_tmap_bf16(&enc, &tK, k, (uint64_t)n_kv * 128, n_rows, ldk, 64, 128)) != MLORA_OK) return s;
-  if ((s = make_tmap_bf16_blocked(&enc, &tV, v, n_rows, (uint64_t)n_kv * 128, ldv, 64, 2)) != MLORA_OK) return s;
+  if ((s = attn_tc_smem(attn_tc::forward_kernel, attn_tc::SMEM_BYTES, attr_dev)) != MLORA_OK) return s;
+  CUtensorMap tQ, tK, tV;
+  if ((s = make_tmap_bf16(enc, &tQ, q, (uint64_t)n_heads * 128, n_rows, ldq, 64, 128)) != MLORA_OK) return s;
+  if ((s = make_tmap_bf16(enc, &tK, k, (uint64_t)n_kv * 128, n_rows, ldk, 64, 128)) != MLORA_OK) return s;
+  if ((s = make_tmap_bf16_blocked(enc, &tV, v, n_rows, (uint64_t)n_kv * 128, ldv, 64, 2)) != MLORA_OK) return s;
   attn_tc::Args a{(__nv_bfloat16*)o, ldo, lse, seq_start, n_rows, n_heads, n_kv, 1.4426950408889634f / sqrtf(128.0f)};
   attn_tc::forward_kernel<<<dim3((n_rows + 127) / 128, n_heads), attn_tc::THREADS, attn_tc::SMEM_BYTES, st>>>(tQ, tK, tV, a);
   return launched();
 }
+
+static mlora_status_t attention_backward_tc(const void* q, int64_t ldq, const void* k, int64_t ldk, const void* v, int64_t ldv,
+                                            const void* o, int64_t ldo, const float* lse, const void* dO, int64_t lddo,
+                                            void* dq, int64_t lddq, void* dk, int64_t lddk, void* dv, int64_t lddv,
+                                            const int32_t* seq_start, const int32_t* seq_end, int32_t n_rows,
+                                            int32_t n_heads, int32_t n_kv, cudaStream_t st) {
+  mlora_ctx* enc = layer_ops_encoder();
+  if (!enc) return MLORA_ERR_CUDA;
+  static bool attr_dq[kMaxDevices] = {}, attr_dkv[kMaxDevices] = {};
+  mlora_status_t s;
+  if ((s = attn_tc_smem(attn_tc::backward_dq_kernel, attn_tc::DQ_SMEM_BYTES, attr_dq)) != MLORA_OK) return s;
+  if ((s = attn_tc_smem(attn_tc::backward_dkv_kernel, attn_tc::DKV_SMEM_BYTES, attr_dkv)) != MLORA_OK) return s;
+  CUtensorMap tQ, tdO, tO, tK, tV;       // all [rows][64-column] boxes of 128 rows
+  if ((s = make_tmap_bf16(enc, &tQ, q, (uint64_t)n_heads * 128, n_rows, ldq, 64, 128)) != MLORA_OK) return s;
+  if ((s = make_tmap_bf16(enc, &tdO, dO, (uint64_t)n_heads * 128, n_rows, lddo, 64, 128)) != MLORA_OK) return s;
+  if ((s = make_tmap_bf16(enc, &tO, o, (uint64_t)n_heads * 128, n_rows, ldo, 64, 128)) != MLORA_OK) return s;
+  if ((s = make_tmap_bf16(enc, &tK, k, (uint64_t)n_kv * 128, n_rows, ldk, 64, 128)) != MLORA_OK) return s;
+  if ((s = make_tmap_bf16(enc, &tV, v, (uint64_t)n_kv * 128, n_rows, ldv, 64, 128)) != MLORA_OK) return s;
+  const float scale = 1.0f / sqrtf(128.0f);
+  attn_tc::BwdArgs a{(const __nv_bfloat16*)o, ldo, (const __nv_bfloat16*)dO, lddo, lse, seq_start, seq_end,
+                     (__nv_bfloat16*)dq, lddq, (__nv_bfloat16*)dk, lddk, (__nv_bfloat16*)dv, lddv,
+                     n_rows, n_heads, n_kv, scale, scale * 1.4426950408889634f};
+  const int tiles = (n_rows + 127) / 128;
+  attn_tc::backward_dq_kernel<<<dim3(tiles, n_heads), attn_tc::THREADS, attn_tc::DQ_SMEM_BYTES, st>>>(tQ, tdO, tK, tV, a);
+  if ((s = launched()) != MLORA_OK) return s;
+  attn_tc::backward_dkv_kernel<<<dim3(tiles, n_kv), attn_tc::THREADS, attn_tc::DKV_SMEM_BYTES, st>>>(tQ, tdO, tO, tK, tV, a);
+  return launched();
+}
+
+extern "C" {
 
 mlora_status_t mlora_attention_forward(const void* q, int64_t ldq, const void* k, int64_t ldk, const void* v, int64_t ldv,
                                        void* o, int64_t ldo, float* lse, const int32_t* seq_start, const int32_t* seq_end,
@@ -1347,16 +1388,14 @@ mlora_status_t mlora_attention_backward(const void* q, int64_t ldq, const void* 
       !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(dO) || !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
     return MLORA_ERR_UNSUPPORTED;
   if (n_rows == 0) return MLORA_OK;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (d_head == 128)
+    return attention_backward_tc(q, ldq, k, ldk, v, ldv, o, ldo, lse, dO, lddo, dq, lddq, dk, lddk, dv, lddv, seq_start,
+                                 seq_end, n_rows, n_heads, n_kv, st);
   attn::AttnArgs a{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, ldq, ldk, ldv,
                    seq_start, seq_end, n_rows, n_heads, n_kv, 1.0f / sqrtf((float)d_head)};
   const int bq = (int)(((int64_t)n_rows * n_heads + 7) / 8), bk = (int)(((int64_t)n_rows * n_kv + 7) / 8);
-  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-  if (d_head == 128) {
-    attn::backward_dq_kernel<32><<<bq, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,
-                                                    (__nv_bfloat16*)dq, lddq);
-    attn::backward_dkv_kernel<32><<<bk, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,
-                                                     (__nv_bfloat16*)dk, lddk, (__nv_bfloat16*)dv, lddv);
-  } else {
+  {
     attn::backward_dq_kernel<16><<<bq, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,
                                                     (__nv_bfloat16*)dq, lddq);
     attn::backward_dkv_kernel<16><<<bk, 256, 0, st>>>(a, (const __nv_bfloat16*)o, ldo, lse, (const __nv_bfloat16*)dO, lddo,

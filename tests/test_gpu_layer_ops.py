@@ -108,7 +108,7 @@ def test_attention_forward_and_backward(heads, kv, dh):
 
 @pytest.mark.parametrize("lens", [[1], [127], [128], [129], [300, 5, 1, 1, 200], [64] * 9, [1] * 140, [700]])
 @pytest.mark.parametrize("heads,kv", [(4, 2), (3, 1)])
-def test_attention_forward_tensor_core_kernel(lens, heads, kv):
+def test_attention_tensor_core_kernels(lens, heads, kv):
     """Head size 128 (the tcgen05 kernel): query tiles that hold one sequence, several sequences or a
     ragged last tile; sequences longer than one key block (online softmax over several blocks);
     outputs and log-sum-exp against the fp64 definition."""
@@ -138,6 +138,21 @@ def test_attention_forward_tensor_core_kernel(lens, heads, kv):
             sc = sc.masked_fill(torch.triu(torch.ones(len(rows), len(rows), dtype=torch.bool), 1), float("-inf"))
             lse_ref[rows, h] = torch.logsumexp(sc, dim=1)
     assert torch.allclose(lse.double().cpu(), lse_ref, rtol=0, atol=2e-3), float((lse.double().cpu() - lse_ref).abs().max())
+    # the gradients (tcgen05 kernels as well): dq per query tile, dk and dv per key tile over the heads of the group
+    dO = bf(torch.randn(T, heads * dh, generator=g)).to(DEV)
+    dq = torch.full_like(q, float("nan"))
+    dk, dv = torch.full_like(k, float("nan")), torch.full_like(v, float("nan"))
+    mo.mlora_attention_backward(q, k, v, o, lse, dO, dq, dk, dv, ss, se, heads, kv, dh)
+    assert mo.mlora_layer_ops_poll_status() == 0
+    qg = qr.reshape(T, heads, dh).clone().requires_grad_(True)
+    kg = kr.reshape(T, kv, dh).clone().requires_grad_(True)
+    vg = vr.reshape(T, kv, dh).clone().requires_grad_(True)
+    lo.attention(qg, kg, vg, seqs).backward(dO.double().cpu().reshape(T, heads, dh))
+    # P and dS enter the tensor cores rounded to bf16 (relative 2^-9 per term, up to 128 terms per block):
+    # with the doubled queries of this test dS reaches ~10, so the bound is 3e-2 here (2e-2 at unit scale above)
+    close(dq, qg.grad.reshape(T, heads * dh), tol=3e-2)
+    close(dk, kg.grad.reshape(T, kv * dh), tol=3e-2)
+    close(dv, vg.grad.reshape(T, kv * dh), tol=3e-2)
 
 
 def test_argument_errors():
