@@ -163,13 +163,14 @@ class DecoderLayer:
     def _body(self, x, lin, sequences):
         T = x.shape[0]
         dh = self.d // self.n_heads
-        pos = torch.zeros(T, dtype=torch.int32, device=x.device)
-        seq_start = torch.arange(T, dtype=torch.int32, device=x.device)          # rows outside every sequence stand alone
-        seq_end = seq_start + 1
+        pos_h = np.zeros(T, dtype=np.int32)                                     # tables built on the host, one copy each
+        start_h = np.arange(T, dtype=np.int32)                                  # rows outside every sequence stand alone
+        end_h = start_h + 1
         for start, n in sequences:
-            pos[start:start + n] = torch.arange(n, device=x.device, dtype=torch.int32)
-            seq_start[start:start + n] = start
-            seq_end[start:start + n] = start + n
+            pos_h[start:start + n] = np.arange(n, dtype=np.int32)
+            start_h[start:start + n] = start
+            end_h[start:start + n] = start + n
+        pos, seq_start, seq_end = (torch.from_numpy(t).to(x.device) for t in (pos_h, start_h, end_h))
         h1 = _RmsNormFn.apply(x, self.g1)
         q = _RopeFn.apply(lin("q", h1), pos, self.n_heads, dh)
         k = _RopeFn.apply(lin("k", h1), pos, self.n_kv, dh)

@@ -27,6 +27,48 @@ def timeit(fn, n=50):
     return e0.elapsed_time(e1) / n * 1e-3
 
 
+def whole_layer(dev) -> str:
+    """One Llama-3-8B-sized decoder layer through DecoderLayer: the mixed serving forward of the cfg3 batch
+    (4096 rows: 12 prompts, 1024 decode rows, four 512-token fine-tuning sequences) and the backward that
+    recomputes the layer for the 2048 fine-tuning rows from the saved layer input."""
+    import math
+    import numpy as np
+    from . import synth
+    from .layer import DecoderLayer
+    from .runner import Session
+    d, ffn, r, n_ad, H, Hkv = 4096, 14336, 16, 32, 32, 8
+    dh = d // H
+    g = torch.Generator().manual_seed(5)
+    dims = {"q": (d, d), "k": (d, Hkv * dh), "v": (d, Hkv * dh), "o": (d, d), "gate": (d, ffn), "up": (d, ffn), "down": (ffn, d)}
+    p = {"g1": torch.ones(d), "g2": torch.ones(d)}
+    for name, (di, do) in dims.items():
+        p["W_" + name] = (torch.randn(di, do, generator=g) / math.sqrt(di)).to(torch.bfloat16)
+        p["A_" + name] = (0.02 * torch.randn(n_ad, r, di, generator=g)).to(torch.bfloat16)
+        p["B_" + name] = (0.02 * torch.randn(n_ad, r, do, generator=g)).to(torch.bfloat16)
+        p["s_" + name] = torch.full((n_ad,), 2.0)
+    segs, T = synth.cfg3_segments(0)
+    ft_rows = int(segs[segs[:, 3] != 0, 1].sum())
+    x = torch.randn(T, d, generator=g).to(torch.bfloat16).to(dev)
+    dy = torch.randn(ft_rows, d, generator=g).to(torch.bfloat16).to(dev)
+    with Session(0) as sess:
+        layer = DecoderLayer(sess, p, H, Hkv, max_ft_rows=ft_rows)
+        tf, tb = [], []
+        for it in range(6):
+            torch.cuda.synchronize()
+            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            e0.record()
+            layer.forward(x, segs)
+            e1.record()
+            layer.backward(dy)
+            e2.record()
+            torch.cuda.synchronize()
+            if it >= 2:
+                tf.append(e0.elapsed_time(e1)); tb.append(e1.elapsed_time(e2))
+    return (f"whole decoder layer (Llama-3-8B sizes, cfg3 batch: {T} rows, {ft_rows} fine-tuning), through DecoderLayer with "
+            f"PyTorch autograd stringing the kernels together (host overheads included): serving forward "
+            f"{np.median(tf):.2f} ms, recompute + backward over the fine-tuning rows {np.median(tb):.2f} ms")
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--out", default="")
@@ -69,6 +111,7 @@ def main(argv=None):
     lines.append(f"attention, 4 sequences x 512 tokens, 32 query / 8 key-value heads of 128: forward (tcgen05 kernel) "
                  f"{tf * 1e3:.3f} ms ({fl / tf / 1e12:.1f} TFLOP/s over the causal half), backward {tb * 1e3:.2f} ms "
                  f"({2.5 * fl / tb / 1e12:.1f} TFLOP/s)")
+    lines += ["", whole_layer(dev)]
     text = "\n".join(lines) + "\n"
     sys.stdout.write(text)
     if args.out:
