@@ -15,11 +15,14 @@ from paper_2607_28848_b200.runner import LayerRun, Session
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("case", ["mixed", "long_k_split", "dropout"])
+@pytest.mark.parametrize("case", ["mixed", "long_k_split", "dropout", "one_finetune_adapter"])
 def test_graph_replay_matches_eager_on_new_inputs(case):
     with Session(0) as sess:
         if case == "long_k_split":      # few output tiles and K = 8192: the K-split GEMM and its reduction kernel
             w = synth.random_workload(62, 8192, 256, 16, 3, 200, max_seg=80, p_finetune=0.5)
+        elif case == "one_finetune_adapter":   # gradient groups split over rows: partial sums and arrival counters inside the graph
+            segs = synth.segments_array([(0, 60, 2, 0), (60, 900, 0, 1), (960, 40, 1, 0)])
+            w = synth.Workload("one_slot", 512, 768, 16, 3, "bf16", 1000, segs, seed=63)
         else:
             w = synth.random_workload(61, 256, 384, 16, 5, 420, max_seg=130, p_finetune=0.4)
         if case == "dropout":           # the seed is part of the captured launch parameters
