@@ -299,6 +299,26 @@ def main():
     torch.cuda.synchronize()
     step_ms = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(stat_n))
     step_stats = {"steps": stat_n, "median_ms": step_ms[stat_n // 2], "best_ms": step_ms[0]}
+    # Plan build (host validation, routing tables, upload) for this workload's segment table: outside the
+    # timed step, as the plans are prebuilt there; one table serves all projections of a layer.
+    import time as _time
+    w0 = workloads[0]
+    plan_ms = {}
+    for kind in ("blocking", "stream_ordered"):
+        ts = []
+        for _ in range(20):
+            t0 = _time.perf_counter()
+            if kind == "blocking":
+                pl = mb.mlora_plan_create(sess.ctx, w0.segments, w0.n_rows, w0.n_adapters)
+                mb.mlora_plan_destroy(pl)
+            else:
+                pl = mb.mlora_plan_create_async(sess.ctx, w0.segments, w0.n_rows, w0.n_adapters)
+                mb.mlora_plan_release(pl)
+            ts.append((_time.perf_counter() - t0) * 1e3)
+        torch.cuda.synchronize()
+        plan_ms[kind] = sorted(ts)[len(ts) // 2]
+    step_stats["plan_build_host_ms"] = plan_ms
+    step_stats["segments"] = int(len(w0.segments))
     # Per-kernel durations: the same steps once more, now with the library recording a CUDA event
     # pair around every launch (which also switches off the overlap of a kernel's set-up with its
     # predecessor's tail, so each pair times one whole kernel).  Kept out of the region above so
