@@ -72,6 +72,7 @@ def whole_layer(dev) -> str:
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--out", default="")
+    ap.add_argument("--attention-only", action="store_true", help="only the attention timings (a small case for profiling)")
     args = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise RuntimeError("needs the CUDA path: no GPU visible")
@@ -92,7 +93,7 @@ def main(argv=None):
         ("add", lambda: mo.mlora_add(x, dy, y), 3 * T * d * 2),
     ]
     lines = ["| kernel | bytes | µs | GB/s | of the measured copy bandwidth |", "|---|---|---|---|---|"]
-    for name, fn, nbytes in rows:
+    for name, fn, nbytes in ([] if args.attention_only else rows):
         t = timeit(fn)
         lines.append(f"| {name} | {nbytes / 1e6:.0f} MB | {t * 1e6:.1f} | {nbytes / t / 1e9:.0f} | {nbytes / t / 1e9 / hbm:.2f} |")
     # attention: 4 sequences of 512 tokens, 32 query heads over 8 kv heads
@@ -111,7 +112,8 @@ def main(argv=None):
     lines.append(f"attention, 4 sequences x 512 tokens, 32 query / 8 key-value heads of 128: forward (tcgen05 kernel) "
                  f"{tf * 1e3:.3f} ms ({fl / tf / 1e12:.1f} TFLOP/s over the causal half), backward {tb * 1e3:.2f} ms "
                  f"({2.5 * fl / tb / 1e12:.1f} TFLOP/s)")
-    lines += ["", whole_layer(dev)]
+    if not args.attention_only:
+        lines += ["", whole_layer(dev)]
     text = "\n".join(lines) + "\n"
     sys.stdout.write(text)
     if args.out:
