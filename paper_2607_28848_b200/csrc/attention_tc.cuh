@@ -37,6 +37,14 @@ constexpr uint32_t P_BYTES = BM * BN * 2;     // two 64-key K-blocks of [128 row
 constexpr uint32_t SMEM_BYTES = 1024 + Q_BYTES + STAGES * (K_BYTES + V_BYTES) + P_BYTES + 256;
 constexpr uint32_t TMEM_COLS = 256;
 
+// 2^x by the special-function unit (the arguments here are differences from a row maximum or a
+// log-sum-exp, so nothing overflows; large negative arguments give 0)
+__device__ __forceinline__ float fast_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 __device__ int32_t g_status;                  // MLORA_ERR_DEVICE_TIMEOUT once a bounded wait ran out
 
 struct Args {
@@ -184,7 +192,7 @@ forward_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           mx = fmaxf(mx, sc);
         }
       }
-      const float alpha = exp2f(m - mx);
+      const float alpha = fast_ex2(m - mx);
       float rowsum = 0.f;
 #pragma unroll
       for (int cc = 0; cc < 4; ++cc) {
@@ -195,8 +203,8 @@ forward_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 #pragma unroll
         for (int k = 0; k < 32; k += 2) {
           const int col = key0 + cc * 32 + k;
-          const float p0 = (col >= my_start && col <= i_abs) ? exp2f(__uint_as_float(v[k]) * a.scale_log2 - mx) : 0.f;
-          const float p1 = (col + 1 >= my_start && col + 1 <= i_abs) ? exp2f(__uint_as_float(v[k + 1]) * a.scale_log2 - mx) : 0.f;
+          const float p0 = (col >= my_start && col <= i_abs) ? fast_ex2(__uint_as_float(v[k]) * a.scale_log2 - mx) : 0.f;
+          const float p1 = (col + 1 >= my_start && col + 1 <= i_abs) ? fast_ex2(__uint_as_float(v[k + 1]) * a.scale_log2 - mx) : 0.f;
           rowsum += p0 + p1;
           pk[k >> 1] = ptx::pack_bf16(p0, p1);
         }
@@ -445,8 +453,8 @@ backward_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
         for (int k = 0; k < 32; k += 2) {
           const int col = key0 + cc * 32 + k;
-          const float p0 = (col >= my_start && col <= i_abs) ? exp2f(__uint_as_float(vs[k]) * a.scale_log2 - lse2) : 0.f;
-          const float p1 = (col + 1 >= my_start && col + 1 <= i_abs) ? exp2f(__uint_as_float(vs[k + 1]) * a.scale_log2 - lse2) : 0.f;
+          const float p0 = (col >= my_start && col <= i_abs) ? fast_ex2(__uint_as_float(vs[k]) * a.scale_log2 - lse2) : 0.f;
+          const float p1 = (col + 1 >= my_start && col + 1 <= i_abs) ? fast_ex2(__uint_as_float(vs[k + 1]) * a.scale_log2 - lse2) : 0.f;
           pk[k >> 1] = ptx::pack_bf16(p0 * (__uint_as_float(vp[k]) - D), p1 * (__uint_as_float(vp[k + 1]) - D));
         }
         store_row_chunk(sDS, row, cc, pk);
@@ -623,13 +631,23 @@ backward_dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         ptx::tmem_ld_wait();
         uint32_t pp[16], pd[16];
 #pragma unroll
-        for (int k = 0; k < 32; k += 2) {
-          const int c0 = cc * 32 + k;
-          const int i0 = q0 + c0;
-          const float p0 = (j_abs <= i0 && j_abs >= sQS[c0]) ? exp2f(__uint_as_float(vs[k]) * a.scale_log2 - sL[c0]) : 0.f;
-          const float p1 = (j_abs <= i0 + 1 && j_abs >= sQS[c0 + 1]) ? exp2f(__uint_as_float(vs[k + 1]) * a.scale_log2 - sL[c0 + 1]) : 0.f;
-          pp[k >> 1] = ptx::pack_bf16(p0, p1);
-          pd[k >> 1] = ptx::pack_bf16(p0 * (__uint_as_float(vp[k]) - sD[c0]), p1 * (__uint_as_float(vp[k + 1]) - sD[c0 + 1]));
+        for (int k4 = 0; k4 < 32; k4 += 4) {       // the per-query tables come in as vectors, four columns at a time
+          const int c0 = cc * 32 + k4;
+          const float4 l4 = *reinterpret_cast<const float4*>(sL + c0);
+          const float4 d4 = *reinterpret_cast<const float4*>(sD + c0);
+          const int4 s4 = *reinterpret_cast<const int4*>(sQS + c0);
+          const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dv4[4] = {d4.x, d4.y, d4.z, d4.w};
+          const int sv[4] = {s4.x, s4.y, s4.z, s4.w};
+          float p[4];
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            const int i = q0 + c0 + t;
+            p[t] = (j_abs <= i && j_abs >= sv[t]) ? fast_ex2(__uint_as_float(vs[k4 + t]) * a.scale_log2 - lv[t]) : 0.f;
+          }
+          pp[k4 >> 1] = ptx::pack_bf16(p[0], p[1]);
+          pp[(k4 >> 1) + 1] = ptx::pack_bf16(p[2], p[3]);
+          pd[k4 >> 1] = ptx::pack_bf16(p[0] * (__uint_as_float(vp[k4]) - dv4[0]), p[1] * (__uint_as_float(vp[k4 + 1]) - dv4[1]));
+          pd[(k4 >> 1) + 1] = ptx::pack_bf16(p[2] * (__uint_as_float(vp[k4 + 2]) - dv4[2]), p[3] * (__uint_as_float(vp[k4 + 3]) - dv4[3]));
         }
         store_row_chunk(sOP, row, cc, pp);
         store_row_chunk(sDS, row, cc, pd);
