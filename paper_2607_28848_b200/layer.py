@@ -163,13 +163,15 @@ class DecoderLayer:
     def _body(self, x, lin, sequences):
         T = x.shape[0]
         dh = self.d // self.n_heads
-        pos_h = np.zeros(T, dtype=np.int32)                                     # tables built on the host, one copy each
+        # tables built on the host without a Python loop over the sequences, one copy each
         start_h = np.arange(T, dtype=np.int32)                                  # rows outside every sequence stand alone
         end_h = start_h + 1
-        for start, n in sequences:
-            pos_h[start:start + n] = np.arange(n, dtype=np.int32)
-            start_h[start:start + n] = start
-            end_h[start:start + n] = start + n
+        sq = np.asarray(sequences, dtype=np.int64).reshape(-1, 2)
+        if len(sq):
+            rows = np.repeat(sq[:, 0], sq[:, 1]) + (np.arange(int(sq[:, 1].sum())) - np.repeat(np.cumsum(sq[:, 1]) - sq[:, 1], sq[:, 1]))
+            start_h[rows] = np.repeat(sq[:, 0], sq[:, 1])
+            end_h[rows] = np.repeat(sq[:, 0] + sq[:, 1], sq[:, 1])
+        pos_h = (np.arange(T, dtype=np.int32) - start_h).astype(np.int32)
         pos, seq_start, seq_end = (torch.from_numpy(t).to(x.device) for t in (pos_h, start_h, end_h))
         h1 = _RmsNormFn.apply(x, self.g1)
         q = _RopeFn.apply(lin("q", h1), pos, self.n_heads, dh)
@@ -196,15 +198,15 @@ class DecoderLayer:
                 y = torch.empty((n_rows, pr.d_out), dtype=torch.bfloat16, device=x.device)
                 mb.mlora_mixed_forward(self.sess.ctx, pr.layer, plan, inp.contiguous(), y, None, None, 0, 0)
                 return y
-            y = self._body(x, lin, [(int(s), int(n)) for s, n, _, _ in segs if n > 0])
+            y = self._body(x, lin, segs[segs[:, 1] > 0][:, :2])
         finally:
             torch.cuda.synchronize()
             mb.mlora_plan_destroy(plan)
-        for s, n, a, ft in segs:                    # activation capture: the residual-stream input of fine-tuning rows
-            if ft and n > 0:
-                self.saved_x[self.saved_rows:self.saved_rows + n] = x[s:s + n]
-                self.saved.append((int(n), int(a)))
-                self.saved_rows += int(n)
+        # activation capture: the residual-stream input of the fine-tuning rows
+        for s, n, a, _ in segs[(segs[:, 3] != 0) & (segs[:, 1] > 0)]:
+            self.saved_x[self.saved_rows:self.saved_rows + n] = x[s:s + n]
+            self.saved.append((int(n), int(a)))
+            self.saved_rows += int(n)
         return y
 
     # -- backward: recompute from the saved layer input, fine-tuning rows only ---------------------
