@@ -438,7 +438,7 @@ mlora_status_t launch_expand_mask(mlora_ctx* ctx, const mlora_layer_t* L, const 
   a.V = ctx->ws_p; a.R = L->rank; a.A_all = (const __nv_bfloat16*)L->A_all; a.row_adapter = ds.row_adapter;
   a.dX = (__nv_bfloat16*)dX; a.lddx = lddx; a.D = L->d_in; a.n_rows = n_rows; a.drop = ctx->drop;
   LaunchScope scope(ctx, st, KIND_SHRINK);
-  launch_pdl(scope.slot < 0, expand_mask_kernel, dim3(n_rows, (L->d_in / 8 + 127) / 128), dim3(128), 0, st, a);
+  launch_pdl(scope.slot < 0, expand_mask_kernel, dim3((n_rows + EM_ROWS - 1) / EM_ROWS, (L->d_in / 8 + 127) / 128), dim3(128), 0, st, a);
   return scope.done();
 }
 

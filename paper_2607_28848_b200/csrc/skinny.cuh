@@ -1184,7 +1184,7 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
 }
 
 // Low-rank part of the input gradient under dropout: dX[m, k] += keep(m, k) / (1 - p) *
-// sum_q V[m, q] A_a(m)[q, k].  grid = (rows, column blocks of 128 x 8); one thread per 8 columns.
+// sum_q V[m, q] A_a(m)[q, k].
 struct ExpandMaskArgs {
   const float* V;                 // [rows, R] fp32 (already scaled by s)
   int32_t R;
@@ -1196,45 +1196,87 @@ struct ExpandMaskArgs {
   DropArgs drop;
 };
 
+constexpr int EM_ROWS = 8;       // rows per block of the masked expand
+
+// grid = (ceil(rows / EM_ROWS), column blocks of 128 x 8); one thread per 8 columns and EM_ROWS rows.
+// Rows of a block that share their adapter (the usual case: fine-tuning rows of one sequence) read each
+// piece of A once for all of them; a block with mixed adapters takes its rows one by one.
 __global__ void __launch_bounds__(128)
 expand_mask_kernel(const ExpandMaskArgs a) {
-  __shared__ float v[kMaxRank];
-  const int m = blockIdx.x;
+  __shared__ float v[EM_ROWS][kMaxRank];
+  __shared__ int ads[EM_ROWS];
+  const int m0 = blockIdx.x * EM_ROWS;
   const int k = (blockIdx.y * 128 + threadIdx.x) * 8;
-  const int ad = a.row_adapter[m];
+  if (threadIdx.x < EM_ROWS) ads[threadIdx.x] = (m0 + (int)threadIdx.x < a.n_rows) ? a.row_adapter[m0 + threadIdx.x] : -1;
   ptx::grid_dependency_wait();
   ptx::grid_launch_dependents();
-  if (ad < 0) return;
-  for (int q = threadIdx.x; q < a.R; q += 128) v[q] = a.V[(size_t)m * a.R + q];
+  for (int idx = threadIdx.x; idx < EM_ROWS * a.R; idx += 128) {
+    const int r = idx / a.R, q = idx % a.R;
+    v[r][q] = (m0 + r < a.n_rows) ? a.V[(size_t)(m0 + r) * a.R + q] : 0.f;
+  }
   __syncthreads();
   if (k >= a.D) return;
-  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-  const __nv_bfloat16* Ab = a.A_all + (size_t)ad * a.R * a.D + k;
-  for (int q = 0; q < a.R; ++q) {
-    const uint4 w = ptx::ldg_nc_v4(Ab + (size_t)q * a.D);
-    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+  bool same = true;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      acc[2 * i] = fmaf(v[q], __uint_as_float(ww[i] << 16), acc[2 * i]);
-      acc[2 * i + 1] = fmaf(v[q], __uint_as_float(ww[i] & 0xFFFF0000u), acc[2 * i + 1]);
+  for (int r = 1; r < EM_ROWS; ++r) same = same && (ads[r] == ads[0] || ads[r] < 0);
+  float acc[EM_ROWS][8];
+#pragma unroll
+  for (int r = 0; r < EM_ROWS; ++r)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[r][i] = 0.f;
+  if (same && ads[0] >= 0) {
+    const __nv_bfloat16* Ab = a.A_all + (size_t)ads[0] * a.R * a.D + k;
+    for (int q = 0; q < a.R; ++q) {
+      const uint4 w = ptx::ldg_nc_v4(Ab + (size_t)q * a.D);
+      const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+      for (int r = 0; r < EM_ROWS; ++r) {
+        const float vq = v[r][q];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          acc[r][2 * i] = fmaf(vq, __uint_as_float(ww[i] << 16), acc[r][2 * i]);
+          acc[r][2 * i + 1] = fmaf(vq, __uint_as_float(ww[i] & 0xFFFF0000u), acc[r][2 * i + 1]);
+        }
+      }
+    }
+  } else {
+#pragma unroll
+    for (int r = 0; r < EM_ROWS; ++r) {
+      if (ads[r] < 0) continue;
+      const __nv_bfloat16* Ab = a.A_all + (size_t)ads[r] * a.R * a.D + k;
+      for (int q = 0; q < a.R; ++q) {
+        const uint4 w = ptx::ldg_nc_v4(Ab + (size_t)q * a.D);
+        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+        const float vq = v[r][q];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          acc[r][2 * i] = fmaf(vq, __uint_as_float(ww[i] << 16), acc[r][2 * i]);
+          acc[r][2 * i + 1] = fmaf(vq, __uint_as_float(ww[i] & 0xFFFF0000u), acc[r][2 * i + 1]);
+        }
+      }
     }
   }
-  const uint64_t z0 = drop_bits(a.drop.seed, (uint32_t)m, (uint32_t)(k >> 2));
-  const uint64_t z1 = drop_bits(a.drop.seed, (uint32_t)m, (uint32_t)(k >> 2) + 1);
-  __nv_bfloat16* dst = a.dX + (size_t)m * a.lddx + k;
-  uint4 o = *reinterpret_cast<const uint4*>(dst);
-  uint32_t ow[4] = {o.x, o.y, o.z, o.w};
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const uint64_t z = i < 2 ? z0 : z1;
-    const int f = (2 * i) & 3;
-    const bool k0 = (uint32_t)((z >> (16 * f)) & 0xFFFFu) >= a.drop.thr;
-    const bool k1 = (uint32_t)((z >> (16 * (f + 1))) & 0xFFFFu) >= a.drop.thr;
-    const float lo = __uint_as_float(ow[i] << 16) + (k0 ? acc[2 * i] * a.drop.keep_scale : 0.f);
-    const float hi = __uint_as_float(ow[i] & 0xFFFF0000u) + (k1 ? acc[2 * i + 1] * a.drop.keep_scale : 0.f);
-    ow[i] = ptx::pack_bf16(lo, hi);
+  for (int r = 0; r < EM_ROWS; ++r) {
+    const int m = m0 + r;
+    if (ads[r] < 0) continue;               // also rows past the end
+    const uint64_t z0 = drop_bits(a.drop.seed, (uint32_t)m, (uint32_t)(k >> 2));
+    const uint64_t z1 = drop_bits(a.drop.seed, (uint32_t)m, (uint32_t)(k >> 2) + 1);
+    __nv_bfloat16* dst = a.dX + (size_t)m * a.lddx + k;
+    const uint4 o = *reinterpret_cast<const uint4*>(dst);
+    uint32_t ow[4] = {o.x, o.y, o.z, o.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint64_t z = i < 2 ? z0 : z1;
+      const int f = (2 * i) & 3;
+      const bool k0 = (uint32_t)((z >> (16 * f)) & 0xFFFFu) >= a.drop.thr;
+      const bool k1 = (uint32_t)((z >> (16 * (f + 1))) & 0xFFFFu) >= a.drop.thr;
+      const float lo = __uint_as_float(ow[i] << 16) + (k0 ? acc[r][2 * i] * a.drop.keep_scale : 0.f);
+      const float hi = __uint_as_float(ow[i] & 0xFFFF0000u) + (k1 ? acc[r][2 * i + 1] * a.drop.keep_scale : 0.f);
+      ow[i] = ptx::pack_bf16(lo, hi);
+    }
+    *reinterpret_cast<uint4*>(dst) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
   }
-  *reinterpret_cast<uint4*>(dst) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
 }
 
 }  // namespace mlora
