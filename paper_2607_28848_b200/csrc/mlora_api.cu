@@ -63,7 +63,7 @@ struct mlora_ctx {
   std::vector<PlanBuf> plan_pool;    // released buffers of stream-ordered plans
   int64_t launches = 0;
   int32_t gemm_path = 0;
-  int32_t shrink_path = 0;           // 0: streaming kernel for rank <= 32; 1: per-item kernel for every rank
+  int32_t shrink_path = 0;           // 0: streaming shrink for rank <= 64 (gradients: <= 32); 1: per-item kernels for every rank
   int32_t gemm_pairs = 1;            // 1: two-SM (CTA pair) tensor-core kernel; 0: one-SM kernel
   int32_t no_split_k = 0;            // 1: the two-SM kernel never splits K (kernel variant 4)
   EncodeTiledFn encode = nullptr;
@@ -268,7 +268,8 @@ mlora_status_t launch_shrink_stream_d(mlora_ctx* ctx, ShrinkArgs a, int n_items,
   constexpr int R = RB * 8;
   constexpr size_t xrow = 32 * (CHUNK * 128 + 16), xtile = (size_t)(CHUNK / 4) * 32 * 512;
   constexpr size_t xbytes = ((xrow > xtile ? xrow : xtile) + 1023) / 1024 * 1024;
-  constexpr size_t smem = 1024 + (size_t)STAGES * (xbytes + (size_t)(CHUNK / 4) * R * 512) + (size_t)(RB >= 4 ? 4 : 8) * 32 * (R + 1) * 4;
+  constexpr size_t smem = 1024 + (size_t)STAGES * (xbytes + (size_t)(CHUNK / 4) * R * 512) +
+                          (size_t)(RB >= 8 ? 2 : (RB >= 4 ? 4 : 8)) * 32 * (R + 1) * 4;
   CUtensorMap tIn, tP, tSave;
   mlora_status_t ms;
   // (64, rows, D / 64) views: one box = 4 K-blocks x rows x 128 bytes, 128-byte swizzle
@@ -313,8 +314,10 @@ mlora_status_t launch_shrink_stream_d(mlora_ctx* ctx, ShrinkArgs a, int n_items,
 template <int RB, int STAGES, int CHUNK>
 mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, const int32_t* item_desc, int n_rows,
                                     int n_adapters, cudaStream_t st) {
-  if (a.item_save && ctx->drop.thr != 0)
-    return launch_shrink_stream_d<RB, STAGES, CHUNK, true>(ctx, a, n_items, item_desc, n_rows, n_adapters, st);
+  if constexpr (RB <= 4) {           // dropout is offered up to rank 32
+    if (a.item_save && ctx->drop.thr != 0)
+      return launch_shrink_stream_d<RB, STAGES, CHUNK, true>(ctx, a, n_items, item_desc, n_rows, n_adapters, st);
+  }
   return launch_shrink_stream_d<RB, STAGES, CHUNK, false>(ctx, a, n_items, item_desc, n_rows, n_adapters, st);
 }
 
@@ -325,6 +328,7 @@ mlora_status_t launch_shrink(mlora_ctx* ctx, int R, ShrinkArgs a, int n_items, c
     if (R == 8) return launch_shrink_stream<1, 2, 16>(ctx, a, n_items, item_desc, n_rows, n_adapters, st);
     if (R == 16) return launch_shrink_stream<2, 2, 16>(ctx, a, n_items, item_desc, n_rows, n_adapters, st);
     if (R == 32) return launch_shrink_stream<4, 3, 8>(ctx, a, n_items, item_desc, n_rows, n_adapters, st);
+    if (R == 64) return launch_shrink_stream<8, 2, 8>(ctx, a, n_items, item_desc, n_rows, n_adapters, st);
   }
   if (cancelled(ctx)) return MLORA_CANCELLED;
   const int ksplit = shrink_ksplit(ctx, n_items, a.D);

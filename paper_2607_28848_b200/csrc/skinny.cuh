@@ -324,7 +324,7 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
   constexpr uint32_t PBOX_BYTES = 4 * R * 128;            // adapter rows: [4 K-blocks][R rows][128 B], swizzled
   constexpr uint32_t STAGE_BYTES = X_BYTES + NBOX * PBOX_BYTES;
   static_assert(CHUNK % STREAM_WARPS == 0, "each consumer warp takes CHUNK / 8 K-blocks of a unit");
-  constexpr int RW = RB >= 4 ? 4 : 8;                     // reduction buffers (rank 32: two rounds of 4 warps)
+  constexpr int RW = RB >= 8 ? 2 : (RB >= 4 ? 4 : 8);     // reduction buffers (rank 32: two rounds of 4 warps, rank 64: four of 2)
   extern __shared__ __align__(128) uint8_t stream_smem[];
   __shared__ __align__(16) float fin[32][R];             // an item's final rows, read back for the operand chunks
   __shared__ __align__(8) uint64_t bars[2 * STAGES];     // full[STAGES] | empty[STAGES]
