@@ -58,7 +58,7 @@ struct mlora_ctx {
   __nv_bfloat16* ws_pbd = nullptr;   // block-diagonal low-rank operand: [2 * ws_pbd_groups * 256, 64] bf16
   int64_t ws_pbd_groups = 0;
   float* ws_splitk = nullptr;        // fp32 partial products of a K-split GEMM (fixed size, see kSplitKBytes)
-  float* ws_gpart = nullptr;         // row-split gradient groups: [sm_count][32][512] fp32 partial sums
+  float* ws_gpart = nullptr;         // row-split gradient groups: [sm_count][64][512] fp32 partial sums
   int32_t* ws_gcounters = nullptr;   // [sm_count] arrival counters of those groups, zero between launches
   std::vector<PlanBuf> plan_pool;    // released buffers of stream-ordered plans
   int64_t launches = 0;
@@ -407,8 +407,10 @@ mlora_status_t launch_grad_stream2_c(mlora_ctx* ctx, const mlora_plan* p, const 
 template <int MB>
 mlora_status_t launch_grad_stream2(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& gb, const GradArgs& ga_, int n_slots,
                                    int n_rows, cudaStream_t st) {
-  return ctx->drop.thr != 0 ? launch_grad_stream2_c<MB, true>(ctx, p, gb, ga_, n_slots, n_rows, st)
-                            : launch_grad_stream2_c<MB, false>(ctx, p, gb, ga_, n_slots, n_rows, st);
+  if constexpr (MB <= 2) {           // dropout is offered up to rank 32
+    if (ctx->drop.thr != 0) return launch_grad_stream2_c<MB, true>(ctx, p, gb, ga_, n_slots, n_rows, st);
+  }
+  return launch_grad_stream2_c<MB, false>(ctx, p, gb, ga_, n_slots, n_rows, st);
 }
 
 mlora_status_t launch_grad(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& a, int n_slots, int n_rows,
@@ -773,7 +775,7 @@ mlora_status_t mlora_create(mlora_ctx** out, int device) {
   c->encode = reinterpret_cast<EncodeTiledFn>(fn);
   if (cudaMalloc(&c->status_dev, sizeof(int32_t)) != cudaSuccess ||
       cudaMalloc(&c->ws_splitk, kSplitKBytes) != cudaSuccess ||
-      cudaMalloc(&c->ws_gpart, (size_t)c->sm_count * 32 * 512 * sizeof(float)) != cudaSuccess ||
+      cudaMalloc(&c->ws_gpart, (size_t)c->sm_count * 64 * 512 * sizeof(float)) != cudaSuccess ||
       cudaMalloc(&c->ws_gcounters, (size_t)c->sm_count * sizeof(int32_t)) != cudaSuccess ||
       cudaMemset(c->ws_gcounters, 0, (size_t)c->sm_count * sizeof(int32_t)) != cudaSuccess ||
       cudaMemset(c->status_dev, 0, sizeof(int32_t)) != cudaSuccess) {
@@ -1098,9 +1100,10 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   ga.slot_adapter = p->slot_adapter; ga.accumulate = accumulate;
   GradArgs gA = ga;                  // dA = V^T X
   gA.P = ctx->ws_p; gA.scale = nullptr; gA.Q = (const __nv_bfloat16*)x_save; gA.ldq = L->d_in; gA.D = L->d_in; gA.G = dA;
-  if (ctx->shrink_path == 0 && L->rank <= 32) {      // both gradients in one launch of the streaming kernel
+  if (ctx->shrink_path == 0 && L->rank <= 64) {      // both gradients in one launch of the streaming kernel
     s = L->rank <= 16 ? launch_grad_stream2<1>(ctx, p, ga, gA, n_slots, h.ft_rows, st)
-                      : launch_grad_stream2<2>(ctx, p, ga, gA, n_slots, h.ft_rows, st);
+        : L->rank <= 32 ? launch_grad_stream2<2>(ctx, p, ga, gA, n_slots, h.ft_rows, st)
+                        : launch_grad_stream2<4>(ctx, p, ga, gA, n_slots, h.ft_rows, st);
     if (s != MLORA_OK) return s;
     if (!dX) return MLORA_OK;
     if (dropping) {   // the mask acts on the low-rank term per element: base product first, then the masked expand

@@ -829,7 +829,9 @@ grad_kernel(const GradArgs a) {
 // tile's rows; the lower-half warps hand their accumulators over through shared memory at the end
 // of the group (one fixed order again).
 constexpr int GW_ROWS = 64;           // rows per staged tile
-__host__ __device__ constexpr int gw_stages(int cb, int mb) { return cb == 8 ? 3 : (mb == 1 ? 5 : 4); }
+__host__ __device__ constexpr int gw_stages(int cb, int mb) {
+  return mb >= 4 ? (cb == 8 ? 2 : 3) : (cb == 8 ? 3 : (mb == 1 ? 5 : 4));     // what fits 227 KiB of shared memory
+}
 __host__ __device__ constexpr size_t gw_smem_bytes(int cb, int mb) {
   return (size_t)gw_stages(cb, mb) * ((size_t)cb * GW_ROWS * 128 + (size_t)GW_ROWS * mb * 16 * 4) +
          (cb == 8 ? 0 : (size_t)cb * mb * 16 * 65 * 4) + 1024;

@@ -396,7 +396,7 @@ def test_accumulate_and_optional_outputs(sess):
     run2.close()
 
 
-@pytest.mark.parametrize("rank", [8, 16, 32])
+@pytest.mark.parametrize("rank", [8, 16, 32, 64])
 @pytest.mark.parametrize("lens", [(1100, 40), (2048,), (256,), (70, 700, 3)])
 def test_gradient_groups_split_over_rows(sess, rank, lens):
     """One to three fine-tuning adapters leave the gradient kernel fewer (slot, strip) groups than
