@@ -269,9 +269,9 @@ mlora_status_t mlora_profile_enable(mlora_ctx* ctx, int32_t max_records);
 int32_t mlora_profile_collect(mlora_ctx* ctx, int32_t* kinds, float* ms, int32_t cap);
 
 /* Selects kernel variants for MLORA_BF16 layers: 0 = defaults (two-SM tcgen05 tensor-core GEMM,
- * streaming shrink kernel for rank <= 32); 1 = the plain CUDA-core kernels for every step (a slow
+ * streaming shrink and gradient kernels for rank <= 64); 1 = the plain CUDA-core kernels for every step (a slow
  * cross-check used by the tests); 2 = defaults, but the per-item shrink kernel for every rank
- * (the variant ranks 64 and 128 always use); 3 = defaults, but the one-SM tensor-core GEMM;
+ * (the variant rank 128 always uses); 3 = defaults, but the one-SM tensor-core GEMM;
  * 4 = defaults, but the two-SM GEMM never splits K (by default a product with too few output
  * tiles for the SMs is cut into K slices whose fp32 partials a small kernel adds up). */
 mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path);

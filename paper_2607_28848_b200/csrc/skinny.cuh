@@ -8,10 +8,10 @@
 //           adjacent: decode rows of one adapter form one item, prefill and fine-tune segments are
 //           runs of items); optionally copies the rows of In and the result into the fine-tuning
 //           activation buffers on the way.
-//           shrink_stream_kernel (rank <= 32, the default): persistent, stages filled by the copy engine;
-//           shrink_kernel (rank 64 / 128): one CTA per item, operands straight from global memory.
+//           shrink_stream_kernel (rank <= 64, the default): persistent, stages filled by the copy engine;
+//           shrink_kernel (rank 128): one CTA per item, operands straight from global memory.
 //  grad   : G_g[q, j] = sum_{rows t of slot g} P[t, q] * Q[t, j]   (dB = (s U)^T dY, dA = V^T X)
-//           grad_stream_kernel (rank <= 32: both gradients in one launch); grad_kernel (rank 64 / 128).
+//           grad_stream_kernel (rank <= 64: both gradients in one launch); grad_kernel (rank 128).
 //  expand_mask_kernel : the low-rank part of the input gradient under dropout.
 #pragma once
 
