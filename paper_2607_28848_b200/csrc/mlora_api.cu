@@ -314,7 +314,7 @@ mlora_status_t launch_shrink_stream_d(mlora_ctx* ctx, ShrinkArgs a, int n_items,
 template <int RB, int STAGES, int CHUNK>
 mlora_status_t launch_shrink_stream(mlora_ctx* ctx, ShrinkArgs a, int n_items, const int32_t* item_desc, int n_rows,
                                     int n_adapters, cudaStream_t st) {
-  if constexpr (RB <= 4) {           // dropout is offered up to rank 32
+  if constexpr (RB <= 8) {           // dropout is offered up to rank 64 (the streaming kernels' range)
     if (a.item_save && ctx->drop.thr != 0)
       return launch_shrink_stream_d<RB, STAGES, CHUNK, true>(ctx, a, n_items, item_desc, n_rows, n_adapters, st);
   }
@@ -407,7 +407,7 @@ mlora_status_t launch_grad_stream2_c(mlora_ctx* ctx, const mlora_plan* p, const 
 template <int MB>
 mlora_status_t launch_grad_stream2(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& gb, const GradArgs& ga_, int n_slots,
                                    int n_rows, cudaStream_t st) {
-  if constexpr (MB <= 2) {           // dropout is offered up to rank 32
+  if constexpr (MB <= 4) {           // dropout is offered up to rank 64 (the streaming kernels' range)
     if (ctx->drop.thr != 0) return launch_grad_stream2_c<MB, true>(ctx, p, gb, ga_, n_slots, n_rows, st);
   }
   return launch_grad_stream2_c<MB, false>(ctx, p, gb, ga_, n_slots, n_rows, st);
@@ -1043,7 +1043,7 @@ mlora_status_t mlora_mixed_forward(mlora_ctx* ctx, const mlora_layer_t* L, const
   if (ctx->gemm_path == 1)
     return forward_simt<__nv_bfloat16>(ctx, L, p, X, ldx, Y, ldy, x_save, u_save, save_row_base, st);
 
-  if (ctx->drop.thr != 0 && h.ft_rows > 0 && (ctx->shrink_path != 0 || L->rank > 32)) return MLORA_ERR_UNSUPPORTED;
+  if (ctx->drop.thr != 0 && h.ft_rows > 0 && (ctx->shrink_path != 0 || L->rank > 64)) return MLORA_ERR_UNSUPPORTED;
   ShrinkArgs sa;
   sa.In = (const __nv_bfloat16*)X; sa.ld_in = ldx; sa.D = L->d_in;
   sa.P_all = (const __nv_bfloat16*)L->A_all; sa.scale = nullptr; sa.Out = ctx->ws_p;
@@ -1083,7 +1083,7 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
 
   const int n_slots = (int)h.ft_adapters.size();
   const bool dropping = ctx->drop.thr != 0;
-  if (dropping && (ctx->shrink_path != 0 || L->rank > 32)) return MLORA_ERR_UNSUPPORTED;
+  if (dropping && (ctx->shrink_path != 0 || L->rank > 64)) return MLORA_ERR_UNSUPPORTED;
   ShrinkArgs sa;                     // V = s dY B^T
   sa.In = (const __nv_bfloat16*)dY; sa.ld_in = lddy; sa.D = L->d_out;
   sa.P_all = (const __nv_bfloat16*)L->B_all; sa.scale = L->scale; sa.Out = ctx->ws_p;

@@ -52,7 +52,7 @@ def check_dropout(sess, w, t, p, seed, path=0, blocked=False, base=0, cap=None):
         run.close()
 
 
-@pytest.mark.parametrize("rank", [8, 16, 32])
+@pytest.mark.parametrize("rank", [8, 16, 32, 64])
 def test_dropout_streaming_kernels(sess, rank):
     # ragged table: gathered single rows, partial items, fine-tuning segments of every length
     w = synth.random_workload(40 + rank, 512, 384, rank, 5, 700, max_seg=150, p_finetune=0.45)
@@ -116,7 +116,7 @@ def test_dropout_mask_bit_exact(sess):
 
 
 def test_dropout_large_rank_is_refused(sess):
-    w = synth.random_workload(79, 256, 256, 64, 3, 200, p_finetune=0.5)
+    w = synth.random_workload(79, 256, 256, 128, 3, 200, p_finetune=0.5)
     t = synth.make_tensors(w)
     mb.mlora_set_dropout(sess.ctx, 0.1, 1)
     run = LayerRun(sess, w.dtype, t, w.segments, w.n_rows)
