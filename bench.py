@@ -197,6 +197,7 @@ def main():
     ap.add_argument("--with-update", action="store_true",
                     help="also run the AdamW update of the fine-tuned adapters after each backward (not part of the "
                          "headline step; reported under kernels.adamw)")
+    ap.add_argument("--graph", action="store_true", help="also time the step replayed from a CUDA graph (step_stats)")
     ap.add_argument("--dropout", type=float, default=0.0,
                     help="LoRA dropout rate on the fine-tuning rows (the paper trains with 0.05; the headline step "
                          "runs without it); a new seed every step")
@@ -298,6 +299,29 @@ def main():
         marks[i + 1].record()
     torch.cuda.synchronize()
     step_ms = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(stat_n))
+    # The same step captured once in a CUDA graph and replayed (the calls allocate nothing and never
+    # synchronise, so forward + activation save + backward capture as they are); reported beside the
+    # headline, which stays the eagerly launched step.
+    graph_ms = None
+    if args.graph and not args.with_update and args.dropout == 0:
+        gstream = torch.cuda.Stream(device=sess.device)
+        with torch.cuda.stream(gstream):
+            step()
+            gstream.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=gstream):
+                step()
+            for _ in range(3):
+                g.replay()
+            gstream.synchronize()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record(gstream)
+            for _ in range(args.steps):
+                g.replay()
+            g1.record(gstream)
+            gstream.synchronize()
+            graph_ms = g0.elapsed_time(g1) / args.steps
+        del g
     step_stats = {"steps": stat_n, "median_ms": step_ms[stat_n // 2], "best_ms": step_ms[0]}
     # Plan build (host validation, routing tables, upload) for this workload's segment table: outside the
     # timed step, as the plans are prebuilt there; one table serves all projections of a layer.
@@ -318,6 +342,8 @@ def main():
         torch.cuda.synchronize()
         plan_ms[kind] = sorted(ts)[len(ts) // 2]
     step_stats["plan_build_host_ms"] = plan_ms
+    if graph_ms is not None:
+        step_stats["graph_replay_ms_per_step"] = graph_ms
     step_stats["segments"] = int(len(w0.segments))
     # Per-kernel durations: the same steps once more, now with the library recording a CUDA event
     # pair around every launch (which also switches off the overlap of a kernel's set-up with its
