@@ -155,6 +155,39 @@ def test_attention_tensor_core_kernels(lens, heads, kv):
     close(dv, vg.grad.reshape(T, kv * dh), tol=3e-2)
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_attention_random_sequence_mixes(seed):
+    """Seeded random packed batches (one to eleven sequences of 1 to 600 rows, several head groupings),
+    forward and gradients of the head-size-128 kernels against the fp64 definition and its autograd."""
+    import numpy as np
+    rng = np.random.default_rng(900 + seed)
+    n_seq = int(rng.integers(1, 12))
+    lens = [int(x) for x in (rng.integers(1, 40, n_seq) if seed % 3 == 0 else rng.integers(1, 600, n_seq))]
+    heads, kv = [(4, 2), (8, 1), (2, 2), (6, 3)][int(rng.integers(0, 4))]
+    dh, T = 128, sum(lens)
+    g = torch.Generator().manual_seed(seed)
+    q, k, v, dO = (bf(torch.randn(T, n * dh, generator=g)).to(DEV) for n in (heads, kv, kv, heads))
+    start, end, seqs, r = [], [], [], 0
+    for n in lens:
+        start += [r] * n; end += [r + n] * n; seqs.append(list(range(r, r + n))); r += n
+    ss, se = torch.tensor(start, dtype=torch.int32, device=DEV), torch.tensor(end, dtype=torch.int32, device=DEV)
+    o, dq = torch.full_like(q, float("nan")), torch.full_like(q, float("nan"))
+    dk, dv = torch.full_like(k, float("nan")), torch.full_like(v, float("nan"))
+    lse = torch.empty((T, heads), dtype=torch.float32, device=DEV)
+    mo.mlora_attention_forward(q, k, v, o, lse, ss, se, heads, kv, dh)
+    mo.mlora_attention_backward(q, k, v, o, lse, dO, dq, dk, dv, ss, se, heads, kv, dh)
+    assert mo.mlora_layer_ops_poll_status() == 0
+    qr = q.double().cpu().reshape(T, heads, dh).requires_grad_(True)
+    kr = k.double().cpu().reshape(T, kv, dh).requires_grad_(True)
+    vr = v.double().cpu().reshape(T, kv, dh).requires_grad_(True)
+    ref = lo.attention(qr, kr, vr, seqs)
+    ref.backward(dO.double().cpu().reshape(T, heads, dh))
+    close(o, ref.detach().reshape(T, heads * dh))
+    close(dq, qr.grad.reshape(T, heads * dh), tol=2e-2)
+    close(dk, kr.grad.reshape(T, kv * dh), tol=2e-2)
+    close(dv, vr.grad.reshape(T, kv * dh), tol=2e-2)
+
+
 def test_argument_errors():
     x = torch.zeros(4, 12, dtype=torch.bfloat16, device=DEV)           # 12 is not a multiple of 8
     gain = torch.ones(12, device=DEV)
