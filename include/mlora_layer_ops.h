@@ -67,7 +67,9 @@ mlora_status_t mlora_attention_forward(const void* q, int64_t ldq, const void* k
 mlora_status_t mlora_layer_ops_poll_status(void* cuda_stream);
 
 /* Gradients of the above for a given dO: dq like q, dk and dv like k and v (each element written once; the
- * sums over the query heads that share a kv head are inside).  o and lse are the forward's outputs. */
+ * sums over the query heads that share a kv head are inside).  o and lse are the forward's outputs.
+ * d_head = 128 runs on the tensor cores like the forward (the probabilities, recomputed from lse, and dS
+ * enter the products rounded to bf16; accumulation is fp32); d_head = 64 on the CUDA cores in fp32. */
 mlora_status_t mlora_attention_backward(const void* q, int64_t ldq, const void* k, int64_t ldk, const void* v, int64_t ldv,
                                         const void* o, int64_t ldo, const float* lse, const void* dO, int64_t lddo,
                                         void* dq, int64_t lddq, void* dk, int64_t lddk, void* dv, int64_t lddv,
