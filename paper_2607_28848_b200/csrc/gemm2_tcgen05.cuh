@@ -136,7 +136,16 @@ __device__ __forceinline__ void gemm2_tile(const GemmArgs& args, int tile, int& 
   nt = r / gm;
 }
 
-// args: n_mtiles counts 256-row pair tiles, n_ntiles 256-column tiles, n_units = their product;
+// Work unit -> (tile, K slice, slices of that tile).
+__device__ __forceinline__ void gemm2_unit(const GemmArgs& args, int unit, int& tile, int& ks, int& sk) {
+  if (unit < args.n_whole) { tile = unit; ks = 0; sk = 1; return; }
+  const int u = unit - args.n_whole;
+  ks = u / args.n_tail;
+  tile = args.n_whole + u - ks * args.n_tail;
+  sk = args.split_k;
+}
+
+// args: n_mtiles counts 256-row pair tiles, n_ntiles 256-column tiles, n_units = n_whole + n_tail * split_k;
 // row_grp / tile_grp_off / grp_adapter are the tables for 256-row tiles.
 template <int R, bool W_KMAJOR>
 __global__ void __launch_bounds__(GEMM2_THREADS, 1)
@@ -199,8 +208,6 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
 
   const int KB = (args.K + GEMM_BK - 1) / GEMM_BK;
   const int n_units = args.n_units;
-  const int SK = args.split_k;                       // K slices per tile; unit = slice * n_tiles + tile
-  const int n_tiles = args.n_mtiles * args.n_ntiles;
   const int n_pairs = gridDim.x >> 1;
   const int pair = blockIdx.x >> 1;
 
@@ -217,7 +224,8 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
     uint32_t it = 0;
     bool ok = true;
     for (int unit = pair; unit < n_units && ok; unit += n_pairs) {
-      const int tile = unit % n_tiles, ks = unit / n_tiles;
+      int tile, ks, SK;
+      gemm2_unit(args, unit, tile, ks, SK);
       int mt, nt;
       gemm2_tile(args, tile, mt, nt);
       const int m0 = mt * GEMM2_BM + (int)rank * 128;
@@ -291,7 +299,8 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
       uint32_t it = 0, lt = 0;
       bool ok = true;
       for (int unit = pair; unit < n_units && ok; unit += n_pairs, ++lt) {
-        const int tile = unit % n_tiles, ks = unit / n_tiles;
+        int tile, ks, SK;
+        gemm2_unit(args, unit, tile, ks, SK);
         int mt, nt_unused;
         gemm2_tile(args, tile, mt, nt_unused);
         const int kb_begin = (int)((long long)ks * KB / SK), kb_end = (int)((long long)(ks + 1) * KB / SK);
@@ -345,7 +354,8 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
     uint32_t lt = 0;
     bool ok = true;
     for (int unit = pair; unit < n_units && ok; unit += n_pairs, ++lt) {
-      const int tile = unit % n_tiles, ks = unit / n_tiles;
+      int tile, ks, SK;
+      gemm2_unit(args, unit, tile, ks, SK);
       int mt, nt;
       gemm2_tile(args, tile, mt, nt);
       const int m0 = mt * GEMM2_BM + (int)rank * 128 + e * 32, n0 = nt * GEMM2_BN;
@@ -367,15 +377,21 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
         if (SK > 1) {       // a K slice: this lane's row of the fp32 partial, 64 columns, for the reduction kernel
           const int row = m0 + lane;
           if (row < args.M) {
-            float* dst = args.ws_splitk + ((size_t)ks * args.M + row) * args.N + n0 + c * 64;
+            float* dst = args.ws_splitk + (((size_t)ks * args.n_tail + (tile - args.n_whole)) * GEMM2_BM +
+                                           ((int)rank * 128 + e * 32 + lane)) * GEMM2_BN + c * 64;
+            // 256-bit stores: every store fills whole 32-byte sectors of this lane's row
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-              if (n0 + c * 64 + 4 * j < args.N)
-                *reinterpret_cast<uint4*>(dst + 4 * j) = make_uint4(v0[4 * j], v0[4 * j + 1], v0[4 * j + 2], v0[4 * j + 3]);
+            for (int j = 0; j < 4; ++j)
+              if (n0 + c * 64 + 8 * j < args.N)
+                asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + 8 * j),
+                             "r"(v0[8 * j]), "r"(v0[8 * j + 1]), "r"(v0[8 * j + 2]), "r"(v0[8 * j + 3]),
+                             "r"(v0[8 * j + 4]), "r"(v0[8 * j + 5]), "r"(v0[8 * j + 6]), "r"(v0[8 * j + 7]) : "memory");
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-              if (n0 + c * 64 + 32 + 4 * j < args.N)
-                *reinterpret_cast<uint4*>(dst + 32 + 4 * j) = make_uint4(v1[4 * j], v1[4 * j + 1], v1[4 * j + 2], v1[4 * j + 3]);
+            for (int j = 0; j < 4; ++j)
+              if (n0 + c * 64 + 32 + 8 * j < args.N)
+                asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + 32 + 8 * j),
+                             "r"(v1[8 * j]), "r"(v1[8 * j + 1]), "r"(v1[8 * j + 2]), "r"(v1[8 * j + 3]),
+                             "r"(v1[8 * j + 4]), "r"(v1[8 * j + 5]), "r"(v1[8 * j + 6]), "r"(v1[8 * j + 7]) : "memory");
           }
           continue;
         }
@@ -425,19 +441,24 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
   }
 }
 
-// Sum of the K slices of a split product: Out[m, n] = bf16(sum over slices of ws[slice, m, n]),
-// slices added in index order.  One thread per 8 columns (N is a multiple of 64).
+// Sum of the K slices of the split tiles: Out[m, n] = bf16(sum over slices of the tile's fp32
+// partials), slices added in index order.  One thread per 8 columns of a row of a split tile
+// (256 x 32 threads per tile); rows and columns past the output's edge are skipped.
 __global__ void __launch_bounds__(256)
-splitk_reduce_kernel(const float* ws, int split_k, __nv_bfloat16* Out, int64_t ld_out, int M, int N) {
+splitk_reduce_kernel(const GemmArgs args, __nv_bfloat16* Out, int64_t ld_out) {
   ptx::grid_dependency_wait();
   ptx::grid_launch_dependents();
-  const int64_t n8 = N / 8;
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= (int64_t)M * n8) return;
-  const int m = (int)(idx / n8), n = (int)(idx % n8) * 8;
+  const int t = blockIdx.x / 32;                                       // split tile
+  const int idx = (blockIdx.x % 32) * 256 + threadIdx.x;               // 0 .. 8191
+  const int r = idx >> 5, c8 = (idx & 31) * 8;
+  int mt, nt;
+  gemm2_tile(args, args.n_whole + t, mt, nt);
+  const int m = mt * GEMM2_BM + r, n = nt * GEMM2_BN + c8;
+  if (m >= args.M || n >= args.N) return;
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-  for (int s = 0; s < split_k; ++s) {
-    const float4* src = reinterpret_cast<const float4*>(ws + ((size_t)s * M + m) * N + n);
+  for (int s = 0; s < args.split_k; ++s) {
+    const float4* src = reinterpret_cast<const float4*>(
+        args.ws_splitk + (((size_t)s * args.n_tail + t) * GEMM2_BM + r) * GEMM2_BN + c8);
     const float4 a = src[0], b = src[1];
     acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
     acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;

@@ -51,8 +51,13 @@ struct GemmArgs {
   int32_t n_units;               // them (the last, partly filled wave) are cut into two 128 x 128 halves
   int32_t lora_enabled;
   int32_t group_m;               // two-SM kernel only: row tiles per band of the tile order (0: one band)
-  int32_t split_k;               // two-SM kernel only: K slices per tile (1: none); slice-major unit order
-  float* ws_splitk;              // [split_k, M, N] fp32 partial products when split_k > 1
+  // Two-SM kernel only: tiles [0, n_whole) are whole work units; each of the n_tail tiles after them is
+  // cut into split_k K slices (units after the whole ones, slice-major), whose fp32 partial tiles go
+  // to ws_splitk[slice][tail tile][256][256] and are added up by splitk_reduce_kernel.  n_tail = 0:
+  // no split; n_whole = 0: every tile is split (few tiles for the SMs); otherwise only the tiles of
+  // the last, partly filled wave are.
+  int32_t split_k, n_whole, n_tail;
+  float* ws_splitk;
   const int32_t* row_grp;        // [M] group of the row inside its 128-row tile, -1: none
   const int32_t* row_adapter;    // [M]
   const int32_t* tile_grp_off;   // [n_mtiles + 1]

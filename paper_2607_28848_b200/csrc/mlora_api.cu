@@ -551,16 +551,34 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
     // small kernel afterwards (≈8 µs with its launch, so only contractions of 8192 and more are
     // split, into slices of at least 32 K-blocks).
     const int tiles = g.n_mtiles * g.n_ntiles, pairs = ctx->sm_count / 2, kblocks = (K + GEMM_BK - 1) / GEMM_BK;
-    int sk = 1;
-    if (2 * tiles <= pairs && kblocks >= 128 && !ctx->no_split_k) {
+    const size_t tile_ws = (size_t)GEMM2_BM * GEMM2_BN * sizeof(float);
+    int sk = 1, n_tail = 0;
+    if (2 * tiles <= pairs && kblocks >= 128 && !ctx->no_split_k) {          // every tile is split
       sk = pairs / tiles;
       sk = sk < kblocks / 32 ? sk : kblocks / 32;
       sk = sk < 8 ? sk : 8;
-      while (sk > 1 && (size_t)sk * M * N * sizeof(float) > kSplitKBytes) --sk;
-      sk = sk < 1 ? 1 : sk;
+      n_tail = tiles;
+    } else if (tiles > pairs && !ctx->no_split_k) {
+      // More tiles than CTA pairs, and the last wave fills at most half of them: only its tiles are
+      // cut along K (slices of at least 16 K-blocks), so that the wave takes 1 / slices of a tile's
+      // time.  E.g. 160 tiles on 74 pairs: 12 tail tiles in 6 slices, 2.17 instead of 3 tile times.
+      const int rem = tiles % pairs;
+      if (rem > 0 && 2 * rem <= pairs && kblocks >= 32) {
+        sk = pairs / rem;
+        sk = sk < kblocks / 16 ? sk : kblocks / 16;
+        sk = sk < 8 ? sk : 8;
+        n_tail = rem;
+        // Worth it only on long contractions: the K-blocks the last wave no longer waits for (≈0.4 µs
+        // each) have to outweigh the reduction kernel and the fp32 partial traffic.  Measured: 4096-deep
+        // products did not gain (103 -> 101 + 8.6 µs; 5120-deep with adapter-heavy tail tiles lost),
+        // 14336-deep ones did (343 -> 305 + 8.6 µs; 13824-deep with 12 tail tiles 255 -> 177 + 8.7 µs).
+        if (sk < 2 || (int64_t)kblocks * (sk - 1) < 100 * (int64_t)sk) { sk = 1; n_tail = 0; }
+      }
     }
-    g.split_k = sk; g.ws_splitk = ctx->ws_splitk;
-    g.n_full = g.n_units = tiles * sk;
+    while (sk > 1 && (size_t)sk * n_tail * tile_ws > kSplitKBytes) --sk;
+    if (sk <= 1) { sk = 1; n_tail = 0; }
+    g.split_k = sk; g.n_tail = n_tail; g.n_whole = tiles - n_tail; g.ws_splitk = ctx->ws_splitk;
+    g.n_full = g.n_units = g.n_whole + n_tail * sk;
     g.lora_enabled = (lora && !hs.grp2_adapter.empty()) ? 1 : 0;
     g.row_grp = ds.row_grp2; g.row_adapter = ds.row_adapter;
     g.tile_grp_off = ds.tile2_grp_off; g.grp_adapter = ds.grp2_adapter;
@@ -572,9 +590,8 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
     if ((s = launch_gemm2<W_KMAJOR>(ctx, R, tIn, tW, tL, tOut, tPbd, g, st)) != MLORA_OK || sk == 1) return s;
     if (cancelled(ctx)) return MLORA_CANCELLED;
     LaunchScope scope(ctx, st, W_KMAJOR ? KIND_GEMM_BWD : KIND_GEMM_FWD);
-    const int64_t threads = (int64_t)M * (N / 8);
-    launch_pdl(scope.slot < 0, splitk_reduce_kernel, dim3((unsigned)((threads + 255) / 256)), dim3(256), 0, st,
-               (const float*)ctx->ws_splitk, sk, (__nv_bfloat16*)Out, ld_out, M, N);
+    launch_pdl(scope.slot < 0, splitk_reduce_kernel, dim3((unsigned)(n_tail * 32)), dim3(256), 0, st, g,
+               (__nv_bfloat16*)Out, ld_out);
     return scope.done();
   }
   g.n_mtiles = (M + GEMM_BM - 1) / GEMM_BM;
