@@ -111,6 +111,19 @@ def test_split_k_slices(sess, k):
     run_and_check(sess, w2, synth.make_tensors(w2), blocked=True)
 
 
+@pytest.mark.parametrize("d_in,d_out", [(8192, 4096), (4096, 8192)])
+def test_k_split_of_the_last_wave_only(sess, d_in, d_out):
+    """More output tiles than CTA pairs with a small last wave on a long contraction: 5 x 16 tiles of
+    the forward (d_in = 8192) or of the input-gradient product (d_out = 8192) leave 6 tiles for the last
+    wave, which are cut into 8 K slices while the other 74 run whole.  Checked against the blocked oracle;
+    the variant without any K split must give the same numbers up to the rounding of the partial sums."""
+    segs = synth.segments_array([(0, 1130, 0, 1), (1130, 70, 1, 0)])
+    w = synth.Workload("tail_split", d_in, d_out, 16, 2, "bf16", 1200, segs, seed=d_in + 1)
+    t = synth.make_tensors(w)
+    run_and_check(sess, w, t, blocked=True)
+    run_and_check(sess, w, t, path=4, blocked=True)
+
+
 @pytest.mark.parametrize("path", [0, 3])
 @pytest.mark.parametrize("d_in,d_out", [(64, 128), (128, 64), (320, 448), (192, 320)])
 def test_output_width_not_a_multiple_of_the_column_tile(sess, path, d_in, d_out):
