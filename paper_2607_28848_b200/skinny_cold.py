@@ -48,12 +48,12 @@ def cold_skinny(sess, w, reps, copies):
         for i in range(reps):
             c = i % copies
             mb.mlora_mixed_forward(sess.ctx, run.layer, run.plan, Xs[c], run.Y, xss[c], uss[c], 0, run.capacity)
-            kinds, ms = mb.mlora_profile_collect(sess.ctx, 16)
-            assert kinds.tolist() == [KIND_SHRINK, KIND_GEMM_FWD], kinds
+            kinds, ms = mb.mlora_profile_collect(sess.ctx, 16)      # shrink, GEMM (and its K-split reduction, if any)
+            assert kinds[0] == KIND_SHRINK and set(kinds[1:].tolist()) == {KIND_GEMM_FWD}, kinds
             out["shrink_fwd"].append(ms[0] * 1e3)
             mb.mlora_backward(sess.ctx, run.layer, run.plan, dYs[c], xss[c], uss[c], run.dA, run.dB, run.dX)
-            kinds, ms = mb.mlora_profile_collect(sess.ctx, 16)
-            assert kinds.tolist() == [KIND_SHRINK, KIND_GRAD, KIND_GEMM_BWD], kinds
+            kinds, ms = mb.mlora_profile_collect(sess.ctx, 16)      # shrink, gradients, GEMM (and its reduction)
+            assert kinds[0] == KIND_SHRINK and kinds[1] == KIND_GRAD and set(kinds[2:].tolist()) == {KIND_GEMM_BWD}, kinds
             out["shrink_bwd"].append(ms[0] * 1e3)
             out["grad"].append(ms[1] * 1e3)
     finally:
