@@ -85,8 +85,11 @@ typedef struct {
 
 /* ---- context ---------------------------------------------------------------------------*/
 
-/* Creates the per-device state on CUDA device `device`.  Fails with MLORA_ERR_ARCH when the
- * device is not compute capability 10.x, MLORA_ERR_CUDA when the runtime cannot be used. */
+/* Creates the per-device state on CUDA device `device`, including two workspaces of fixed size
+ * that are allocated here so that no compute call allocates: 64 MiB for the fp32 partial products
+ * of K-split GEMMs and SMs x 128 KiB for the partial sums of row-split gradient groups.  Fails
+ * with MLORA_ERR_ARCH when the device is not compute capability 10.x, MLORA_ERR_CUDA when the
+ * runtime cannot be used or the workspaces cannot be allocated. */
 mlora_status_t mlora_create(mlora_ctx** ctx, int device);
 void mlora_destroy(mlora_ctx* ctx);
 
