@@ -144,6 +144,23 @@ class _AddFn(torch.autograd.Function):
         return d, d
 
 
+def sequence_tables(n_rows: int, sequences) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """Per-row position inside its sequence, first row and one-past-last row of its sequence (int32 [n_rows])
+    for sequences given as (first row, length) pairs; rows outside every sequence stand alone.  Built on the
+    host without a Python loop over the sequences."""
+    start = np.arange(n_rows, dtype=np.int32)
+    end = start + 1
+    sq = np.asarray(sequences, dtype=np.int64).reshape(-1, 2)
+    sq = sq[sq[:, 1] > 0]
+    if len(sq):
+        first = np.repeat(sq[:, 0], sq[:, 1])
+        rows = first + (np.arange(int(sq[:, 1].sum())) - np.repeat(np.cumsum(sq[:, 1]) - sq[:, 1], sq[:, 1]))
+        start[rows] = first
+        end[rows] = np.repeat(sq[:, 0] + sq[:, 1], sq[:, 1])
+    pos = (np.arange(n_rows, dtype=np.int32) - start).astype(np.int32)
+    return pos, start, end
+
+
 class DecoderLayer:
     def __init__(self, sess, params: Dict[str, torch.Tensor], n_heads: int, n_kv: int, max_ft_rows: int):
         """params as in the layer oracle: g1, g2, and W_p / A_p / B_p / s_p for the seven projections."""
@@ -163,16 +180,7 @@ class DecoderLayer:
     def _body(self, x, lin, sequences):
         T = x.shape[0]
         dh = self.d // self.n_heads
-        # tables built on the host without a Python loop over the sequences, one copy each
-        start_h = np.arange(T, dtype=np.int32)                                  # rows outside every sequence stand alone
-        end_h = start_h + 1
-        sq = np.asarray(sequences, dtype=np.int64).reshape(-1, 2)
-        if len(sq):
-            rows = np.repeat(sq[:, 0], sq[:, 1]) + (np.arange(int(sq[:, 1].sum())) - np.repeat(np.cumsum(sq[:, 1]) - sq[:, 1], sq[:, 1]))
-            start_h[rows] = np.repeat(sq[:, 0], sq[:, 1])
-            end_h[rows] = np.repeat(sq[:, 0] + sq[:, 1], sq[:, 1])
-        pos_h = (np.arange(T, dtype=np.int32) - start_h).astype(np.int32)
-        pos, seq_start, seq_end = (torch.from_numpy(t).to(x.device) for t in (pos_h, start_h, end_h))
+        pos, seq_start, seq_end = (torch.from_numpy(t).to(x.device) for t in sequence_tables(T, sequences))
         h1 = _RmsNormFn.apply(x, self.g1)
         q = _RopeFn.apply(lin("q", h1), pos, self.n_heads, dh)
         k = _RopeFn.apply(lin("k", h1), pos, self.n_kv, dh)

@@ -100,3 +100,28 @@ def test_interrupted_forward_returns_its_samples():
         assert sorted(out["admitted"]) == [0, 1, 2, 3] and out["backward"]
     finally:
         ms.mlora_sched_destroy(s)
+
+
+def test_sequence_tables_of_the_layer_module_match_a_plain_loop():
+    """Host-side tables of the decoder-layer module (position, first and one-past-last row of each row's
+    sequence) against the obvious loop, on random sequence layouts with gaps and single-row sequences."""
+    import numpy as np
+    from paper_2607_28848_b200.layer import sequence_tables
+    rng = np.random.default_rng(3)
+    for _ in range(20):
+        seqs, row = [], 0
+        for _ in range(int(rng.integers(0, 30))):
+            row += int(rng.integers(0, 3))                    # rows that belong to no sequence
+            n = int(rng.integers(0, 50)) if rng.random() < 0.7 else 1
+            seqs.append((row, n))
+            row += n
+        T = row + int(rng.integers(0, 4))
+        pos, start, end = sequence_tables(T, seqs)
+        p_ref, s_ref = np.zeros(T, np.int32), np.arange(T, dtype=np.int32)
+        e_ref = s_ref + 1
+        for s0, n in seqs:
+            p_ref[s0:s0 + n] = np.arange(n)
+            s_ref[s0:s0 + n] = s0
+            e_ref[s0:s0 + n] = s0 + n
+        assert np.array_equal(pos, p_ref) and np.array_equal(start, s_ref) and np.array_equal(end, e_ref)
+        assert pos.dtype == start.dtype == end.dtype == np.int32
