@@ -230,8 +230,10 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
       gemm2_tile(args, tile, mt, nt);
       const int m0 = mt * GEMM2_BM + (int)rank * 128;
       const int nh = nt * GEMM2_BN + (int)rank * 128;     // this CTA's half of the B columns
-      const int G = ks == SK - 1 ? tile_groups(mt) : 0;   // the low-rank blocks ride with the last K slice
+      const int G = tile_groups(mt);
       const int LC = (G * R + 63) / 64;
+      // a K slice takes its share of the low-rank blocks as well (an adapter-heavy tile has more of them than K-blocks)
+      const int lc_begin = (int)((long long)ks * LC / SK), lc_end = (int)((long long)(ks + 1) * LC / SK);
       const int kb_begin = (int)((long long)ks * KB / SK), kb_end = (int)((long long)(ks + 1) * KB / SK);
       const int chunk_base = args.lora_enabled ? args.tile_grp_off[mt] : 0;   // chunk slot = 2 * this + lc
       int32_t ga_reg[8];                                  // G <= 256 adapters of the pair tile
@@ -257,13 +259,13 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
         if (!ok) break;
       }
       if (!ok) break;
-      if (LC > 0) {
+      if (lc_end > lc_begin) {
 #pragma unroll
         for (int j = 0; j < 8; ++j)
           if (lane + 32 * j < G) ga_smem[lane + 32 * j] = ga_reg[j];
         __syncwarp();
       }
-      for (int lc = 0; lc < LC; ++lc, ++it) {
+      for (int lc = lc_begin; lc < lc_end; ++lc, ++it) {
         const int s = it % S;
         if (lane == 0) ok = gemm2_wait(bar_empty(s), ((it / S) & 1) ^ 1, abort_flag, args.status);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -325,9 +327,10 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
           ptx::umma2_commit_both(bar_empty(s));
         }
         if (!ok) break;
-        const int G = ks == SK - 1 ? tile_groups(mt) : 0;
+        const int G = tile_groups(mt);
         const int LC = (G * R + 63) / 64;
-        for (int lc = 0; lc < LC; ++lc, ++it) {
+        const int lc_begin = (int)((long long)ks * LC / SK), lc_end = (int)((long long)(ks + 1) * LC / SK);
+        for (int lc = lc_begin; lc < lc_end; ++lc, ++it) {
           const int s = it % S;
           if (!(ok = gemm2_wait(bar_full(s), (it / S) & 1, abort_flag, args.status))) break;
           ptx::tc_fence_after();

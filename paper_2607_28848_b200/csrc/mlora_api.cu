@@ -568,11 +568,12 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
         sk = sk < kblocks / 16 ? sk : kblocks / 16;
         sk = sk < 8 ? sk : 8;
         n_tail = rem;
-        // Worth it only on long contractions: the K-blocks the last wave no longer waits for (≈0.4 µs
-        // each) have to outweigh the reduction kernel and the fp32 partial traffic.  Measured: 4096-deep
-        // products did not gain (103 -> 101 + 8.6 µs; 5120-deep with adapter-heavy tail tiles lost),
-        // 14336-deep ones did (343 -> 305 + 8.6 µs; 13824-deep with 12 tail tiles 255 -> 177 + 8.7 µs).
-        if (sk < 2 || (int64_t)kblocks * (sk - 1) < 100 * (int64_t)sk) { sk = 1; n_tail = 0; }
+        // Worth it only if the K-blocks the last wave no longer waits for (≈0.4 µs each) outweigh the
+        // reduction kernel and the fp32 partial traffic (≈8 µs): the bound below keeps out e.g. a
+        // 4096-deep product with a half-full last wave (two slices: 103 -> 101 + 8.6 µs) and lets in
+        // a 4096-deep one with 8 tail tiles in four slices (330 -> 314 + 7.7 µs) and the 14336-deep
+        // ones (343 -> 305 + 8.6 µs; 13824-deep with 12 tail tiles 255 -> 177 + 8.7 µs).
+        if (sk < 2 || (int64_t)kblocks * (sk - 1) < 40 * (int64_t)sk) { sk = 1; n_tail = 0; }
       }
     }
     while (sk > 1 && (size_t)sk * n_tail * tile_ws > kSplitKBytes) --sk;
