@@ -547,17 +547,20 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
     g.n_mtiles = (M + GEMM2_BM - 1) / GEMM2_BM;
     g.n_ntiles = (N + GEMM2_BN - 1) / GEMM2_BN;
     // Few tiles for the CTA pairs there are (small batches, the backward of one 256-token fine-tuning
-    // batch): cut K into slices that run on different pairs; the fp32 partials are summed by a
-    // small kernel afterwards (≈8 µs with its launch, so only contractions of 8192 and more are
-    // split, into slices of at least 32 K-blocks).
+    // batch): cut K into slices of at least 16 K-blocks that run on different pairs; the fp32 partials
+    // are summed by a small kernel afterwards (≈8 µs with its launch, hence the bound on what the split
+    // has to save).
     const int tiles = g.n_mtiles * g.n_ntiles, pairs = ctx->sm_count / 2, kblocks = (K + GEMM_BK - 1) / GEMM_BK;
     const size_t tile_ws = (size_t)GEMM2_BM * GEMM2_BN * sizeof(float);
     int sk = 1, n_tail = 0;
-    if (2 * tiles <= pairs && kblocks >= 128 && !ctx->no_split_k) {          // every tile is split
+    if (2 * tiles <= pairs && kblocks >= 64 && !ctx->no_split_k) {          // every tile is split
       sk = pairs / tiles;
-      sk = sk < kblocks / 32 ? sk : kblocks / 32;
+      sk = sk < kblocks / 16 ? sk : kblocks / 16;
       sk = sk < 8 ? sk : 8;
       n_tail = tiles;
+      // the same bound as for the last wave below (4096 -> 4096 backward of 256 rows, 16 tiles in
+      // four slices: 42.6 -> 36.3 µs for the whole call; two slices of such a product do not pay)
+      if (sk < 2 || (int64_t)kblocks * (sk - 1) < 40 * (int64_t)sk) { sk = 1; n_tail = 0; }
     } else if (tiles > pairs && !ctx->no_split_k) {
       // More tiles than CTA pairs, and the last wave fills at most half of them: only its tiles are
       // cut along K (slices of at least 16 K-blocks), so that the wave takes 1 / slices of a tile's
