@@ -392,7 +392,11 @@ def main():
                             "note": "30 bytes per adapter element: grad, weight, two moments read; weight, moments, stored weight written"}
     # per-launch view of the memory-bound kernels: which launch is which follows from the fixed order
     # shrink(fwd), GEMM fwd, shrink(bwd), gradients (dB and dA in one launch), GEMM bwd [, update] per projection
-    per_step = len(kms) // prof_steps if prof_steps else 0
+    if "splitk_reduce" in per_kind:     # the small kernels that add up the K slices of split GEMM tiles
+        kernels["splitk_reduce"] = per_kind["splitk_reduce"]
+    reduce_kind = mb.PROFILE_KINDS.index("splitk_reduce")
+    kms_main = kms[kinds != reduce_kind]              # the fixed per-projection order below has no reduction launches
+    per_step = len(kms_main) // prof_steps if prof_steps else 0
     labels = []
     for w, a_ in zip(workloads, ab):
         labels += [(w.name, "shrink_fwd", a_["shrink_fwd"]), (w.name, "gemm_fwd", None), (w.name, "shrink_bwd", a_["shrink_bwd"]),
@@ -401,7 +405,7 @@ def main():
             labels.append((w.name, "adamw", None))
     skinny = []
     if per_step == len(labels) and per_step > 0:
-        mean_ms = kms[:per_step * prof_steps].reshape(prof_steps, per_step).mean(0)
+        mean_ms = kms_main[:per_step * prof_steps].reshape(prof_steps, per_step).mean(0)
         for (proj, kern, nbytes), t in zip(labels, mean_ms):
             if nbytes:
                 skinny.append({"launch": f"{proj}:{kern}", "mbytes": nbytes / 1e6, "us": float(t * 1e3),

@@ -266,7 +266,8 @@ int64_t mlora_launch_count(const mlora_ctx* ctx);
  * of this context record one pair around itself on the launching stream, until the pairs run
  * out; n = 0 switches recording off and frees the events.  mlora_profile_collect synchronises
  * the device, writes for each recorded launch its kind (0 shrink, 1 forward GEMM, 2 input-gradient
- * GEMM, 3 gradient kernel, 4 CUDA-core kernels, 5 optimizer update) and its duration in milliseconds into the host
+ * GEMM, 3 gradient kernel, 4 CUDA-core kernels, 5 optimizer update, 6 reduction kernel of a K-split GEMM) and its
+ * duration in milliseconds into the host
  * arrays (up to cap entries), forgets the records and returns how many there were. */
 mlora_status_t mlora_profile_enable(mlora_ctx* ctx, int32_t max_records);
 int32_t mlora_profile_collect(mlora_ctx* ctx, int32_t* kinds, float* ms, int32_t cap);

@@ -255,7 +255,7 @@ def mlora_set_gemm_path(ctx, path: int) -> None:
     _check(load_library().mlora_set_gemm_path(ctx, int(path)), "mlora_set_gemm_path")
 
 
-PROFILE_KINDS = ("shrink", "gemm_fwd", "gemm_bwd", "grad", "simt", "adamw")
+PROFILE_KINDS = ("shrink", "gemm_fwd", "gemm_bwd", "grad", "simt", "adamw", "splitk_reduce")
 
 
 def mlora_adamw_update(ctx, layer: mlora_layer_t, plan, dA, dB, wA, wB, mA, vA, mB, vB, step: int, lr: float = 1e-3,

@@ -77,7 +77,7 @@ struct mlora_ctx {
 
 constexpr int kMaxKSplit = 16;
 
-enum { KIND_SHRINK = 0, KIND_GEMM_FWD = 1, KIND_GEMM_BWD = 2, KIND_GRAD = 3, KIND_SIMT = 4, KIND_ADAMW = 5 };
+enum { KIND_SHRINK = 0, KIND_GEMM_FWD = 1, KIND_GEMM_BWD = 2, KIND_GRAD = 3, KIND_SIMT = 4, KIND_ADAMW = 5, KIND_REDUCE = 6 };
 
 // Device copy of one RowSpace.
 struct DevRowSpace {
@@ -593,7 +593,7 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
       return s;
     if ((s = launch_gemm2<W_KMAJOR>(ctx, R, tIn, tW, tL, tOut, tPbd, g, st)) != MLORA_OK || sk == 1) return s;
     if (cancelled(ctx)) return MLORA_CANCELLED;
-    LaunchScope scope(ctx, st, W_KMAJOR ? KIND_GEMM_BWD : KIND_GEMM_FWD);
+    LaunchScope scope(ctx, st, KIND_REDUCE);
     launch_pdl(scope.slot < 0, splitk_reduce_kernel, dim3((unsigned)(n_tail * 32)), dim3(256), 0, st, g,
                (__nv_bfloat16*)Out, ld_out);
     return scope.done();
