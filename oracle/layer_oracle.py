@@ -17,8 +17,12 @@ no biases - the Llama-3 conventions; the paper names the model, not these detail
 
 Pins (tests/test_layer_pins.py): RMSNorm and rotary embedding against hand-computed values and their
 defining properties (unit RMS; norm preservation and dependence on relative position only), causality
-and independence of sequences, B = 0 gives the base layer, and central finite differences for the
-adapter and input gradients.
+and independence of sequences, B = 0 gives the base layer, central finite differences for the
+adapter and input gradients, and the wiring written out as literals: the SiLU gate against a hand value
+that tells gate from up, both residual connections (all projections zero returns the input; the attention
+branch alone gives 2 x), the 1 / sqrt(d_head) softmax scale on a two-token example with weights (1/4, 3/4),
+the grouped-query head mapping on constant key-value heads, and lora_linear against the hot path's own
+oracle (mlora_oracle.forward) on a mixed table.
 """
 from __future__ import annotations
 

@@ -102,3 +102,94 @@ def test_gradients_by_finite_differences():
     for t, c in ((0, 0), (3, 5), (6, 15)):
         xp, xm = x.clone(), x.clone(); xp[t, c] += h; xm[t, c] -= h
         assert float(g["dx"][t, c]) == pytest.approx((loss(xp, p) - loss(xm, p)) / (2 * h), rel=1e-5, abs=1e-8)
+
+
+# ---- wiring pins: each is written out as literals, so that a swapped operand, a dropped residual, a
+# ---- missing softmax scale or a wrong head mapping in the oracle changes the expected numbers -----------
+def _tiny_params(d, ffn, n_kv_cols):
+    """One adapter slot with B = 0 (base layer only); every weight zero until a test fills it in."""
+    z = lambda r, c: torch.zeros(r, c, dtype=F64)
+    dims = {"q": (d, d), "k": (d, n_kv_cols), "v": (d, n_kv_cols), "o": (d, d), "gate": (d, ffn), "up": (d, ffn),
+            "down": (ffn, d)}
+    p = {"g1": torch.ones(d, dtype=F64), "g2": torch.ones(d, dtype=F64)}
+    for name, (di, do) in dims.items():
+        p["W_" + name] = z(di, do)
+        p["A_" + name] = torch.zeros(1, 1, di, dtype=F64)
+        p["B_" + name] = torch.zeros(1, 1, do, dtype=F64)
+        p["s_" + name] = torch.ones(1, dtype=F64)
+    return p
+
+
+def test_all_projections_zero_returns_the_input():
+    """Both residual connections: with every projection zero the layer is the identity."""
+    p = _tiny_params(4, 6, 2)
+    x = torch.randn(5, 4, dtype=F64)
+    assert torch.equal(lo.layer_forward(x, p, [-1] * 5, [[0, 1, 2], [3, 4]], 2, 1), x)
+
+
+def test_silu_gate_hand_value_tells_gate_from_up():
+    """x = [1, -1] has unit RMS, so h2 = x (up to eps); gate gives g = [1, 2], up gives u = [3, -1], the down
+    projection is the identity and the attention branch is zero:  y = x + [silu(1) 3, silu(2) (-1)].
+    silu(1) = 0.7310585786300049, silu(2) = 1.7615941559557646.  (With gate and up swapped the second
+    term would be [silu(3) 1, silu(-1) 2] = [2.8577, -0.5379].)"""
+    p = _tiny_params(2, 2, 2)
+    p["W_gate"] = torch.tensor([[1.0, 2.0], [0.0, 0.0]], dtype=F64)
+    p["W_up"] = torch.tensor([[3.0, -1.0], [0.0, 0.0]], dtype=F64)
+    p["W_down"] = torch.eye(2, dtype=F64)
+    y = lo.layer_forward(torch.tensor([[1.0, -1.0]], dtype=F64), p, [-1], [[0]], 1, 1)
+    want = torch.tensor([[1.0 + 3 * 0.7310585786300049, -1.0 - 1.7615941559557646]], dtype=F64)
+    assert torch.allclose(y, want, atol=1e-4, rtol=0)
+
+
+def test_attention_residual_hand_value():
+    """One-token sequence, W_v = W_o = identity, no feed-forward:  y = x + RMSNorm(x) = 2 x for unit-RMS x."""
+    p = _tiny_params(2, 2, 2)
+    p["W_v"] = torch.eye(2, dtype=F64)
+    p["W_o"] = torch.eye(2, dtype=F64)
+    y = lo.layer_forward(torch.tensor([[1.0, -1.0]], dtype=F64), p, [-1], [[0]], 1, 1)
+    assert torch.allclose(y, torch.tensor([[2.0, -2.0]], dtype=F64), atol=1e-4, rtol=0)
+
+
+def test_attention_softmax_scale_hand_value():
+    """Two tokens, one head of size 4: q1 . k1 = 2 ln 3 and q1 . k0 = 0, so with the 1 / sqrt(4) scale the scores
+    of token 1 are (0, ln 3) and its weights (1/4, 3/4); without the scale they would be (1/10, 9/10)."""
+    q = torch.tensor([[[0.0, 0, 0, 0]], [[2.0, 0, 0, 0]]], dtype=F64)
+    k = torch.tensor([[[0.0, 0, 0, 0]], [[math.log(3.0), 0, 0, 0]]], dtype=F64)
+    v = torch.tensor([[[1.0, 0, 0, 0]], [[0.0, 1, 0, 0]]], dtype=F64)
+    out = lo.attention(q, k, v, [[0, 1]])
+    assert torch.allclose(out[0, 0], torch.tensor([1.0, 0, 0, 0], dtype=F64))            # token 0 sees only itself
+    assert torch.allclose(out[1, 0], torch.tensor([0.25, 0.75, 0, 0], dtype=F64), atol=1e-12)
+
+
+def test_grouped_query_heads_read_their_own_kv_head():
+    """Four query heads over two key-value heads: heads 0, 1 read kv head 0 and heads 2, 3 read kv head 1."""
+    q = torch.randn(1, 4, 2, dtype=F64)
+    k = torch.randn(1, 2, 2, dtype=F64)
+    v = torch.tensor([[[1.0, 1.0], [2.0, 2.0]]], dtype=F64)          # kv head 0 is all ones, kv head 1 all twos
+    out = lo.attention(q, k, v, [[0]])
+    want = torch.tensor([[[1.0, 1.0], [1.0, 1.0], [2.0, 2.0], [2.0, 2.0]]], dtype=F64)
+    assert torch.equal(out, want)
+    # and the scores use the same mapping: two tokens, the key of kv head 1 at token 1 is large along the
+    # query of head 2 only, so only heads 2 and 3 can prefer token 1 ... head 3's query is orthogonal to it
+    q2 = torch.zeros(2, 4, 2, dtype=F64); q2[1, 2, 0] = 50.0
+    k2 = torch.zeros(2, 2, 2, dtype=F64); k2[1, 1, 0] = 50.0
+    v2 = torch.zeros(2, 2, 2, dtype=F64); v2[1, :, 1] = 1.0          # token 1 carries the marker in both kv heads
+    out2 = lo.attention(q2, k2, v2, [[0, 1]])
+    assert out2[1, 2, 1] > 0.999                                      # head 2 attends to token 1
+    assert torch.allclose(out2[1, [0, 1, 3], 1], torch.full((3,), 0.5, dtype=F64))   # the others split evenly
+
+
+def test_lora_linear_is_the_hot_path_oracle():
+    """The layer oracle's projection equals the layer-free oracle of the hot path on a mixed table."""
+    from oracle import mlora_oracle as orc
+    rng = np.random.default_rng(5)
+    T, d_in, d_out, r, n = 11, 6, 5, 2, 3
+    X, W = rng.standard_normal((T, d_in)), rng.standard_normal((d_in, d_out))
+    A, B = rng.standard_normal((n, r, d_in)), rng.standard_normal((n, r, d_out))
+    s = np.array([2.0, 0.5, 1.25])
+    segs = np.array([[0, 3, 1, 0], [3, 2, -1, 0], [5, 4, 0, 1], [10, 1, 2, 0]], dtype=np.int32)   # row 9 uncovered
+    ref = orc.forward(X, W, A, B, s, segs)["Y"]
+    ra = [1, 1, 1, -1, -1, 0, 0, 0, 0, -1, 2]
+    t = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float64))
+    got = lo.lora_linear(t(X), t(W), t(A), t(B), t(s), ra)
+    assert np.allclose(got.numpy(), ref, rtol=1e-12, atol=1e-12)
