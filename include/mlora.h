@@ -103,8 +103,11 @@ void mlora_destroy(mlora_ctx* ctx);
  * schedules of the kernels.  Segments may come in any order; zero-length segments are legal;
  * rows covered by no segment use the base weight only.
  * With ctx == NULL the plan is host-only (for inspection; it cannot be executed).  With a
- * context the tables are uploaded and the context's workspace is grown if needed, so this
- * call may allocate device memory and synchronise; the compute calls never do.
+ * context the tables are uploaded and the context's workspaces are enlarged if this batch is larger
+ * than any before, so this call may allocate device memory and synchronise; the compute calls never
+ * do.  An enlarged workspace is a NEW block; the block it replaces stays allocated until
+ * mlora_destroy, so kernels already queued and CUDA graphs captured earlier keep working on memory
+ * that is still theirs - creating a larger plan never invalidates an earlier plan or graph.
  * Errors: MLORA_ERR_SEGMENT_RANGE, MLORA_ERR_SEGMENT_OVERLAP, MLORA_ERR_ADAPTER_ID,
  * MLORA_ERR_INVALID_ARG, MLORA_ERR_CUDA. */
 mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, int32_t n_segs,
@@ -254,9 +257,21 @@ mlora_status_t mlora_adamw_update(mlora_ctx* ctx, const mlora_layer_t* layer, co
 
 /* Synchronises the stream and returns the device status word: MLORA_OK, or
  * MLORA_ERR_DEVICE_TIMEOUT when a bounded wait inside a kernel gave up (the kernel then
- * released its resources and returned; its outputs are invalid).  Clears the word. */
+ * released its resources and returned; its outputs are invalid).  Clears the word, and after a
+ * timeout also the arrival counters of work items that several CTAs share (a kernel that gave up may
+ * have left them partly counted), so that the next compute call starts from a clean state. */
 mlora_status_t mlora_poll_status(mlora_ctx* ctx, void* cuda_stream);
 const char* mlora_status_string(mlora_status_t s);
+
+/* Self-test of that report path (the paper has no counterpart; it belongs to this library's rule that no
+ * wait inside a kernel is unbounded).  Queues one tiny kernel whose only work is to wait, with the wait
+ * helper of the streaming kernels, on a barrier that nothing ever arrives at, for `polls` polls
+ * (1 .. 2^20; a thousand take microseconds).  The wait runs out, the kernel records
+ * MLORA_ERR_DEVICE_TIMEOUT in the status word and returns normally: nothing faults or hangs and the
+ * context stays usable.  The next mlora_poll_status therefore returns MLORA_ERR_DEVICE_TIMEOUT, clears the
+ * word together with the arrival counters of split work items, and the poll after that returns MLORA_OK.
+ * Errors: MLORA_ERR_INVALID_ARG (NULL context, polls out of range), MLORA_ERR_CUDA. */
+mlora_status_t mlora_selftest_timeout(mlora_ctx* ctx, uint32_t polls, void* cuda_stream);
 
 /* Number of kernels the library has launched on this context since it was created. */
 int64_t mlora_launch_count(const mlora_ctx* ctx);
@@ -295,7 +310,9 @@ mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path);
  * (MLORA_NOALLOC_MAX_ROWS x 128 floats = 256 KiB, held by every GPU that loads the library until
  * the process exits).  It calls no cudaMalloc, cudaFree or allocating library routine.
  *   layer        as for mlora_mixed_forward (either dtype; no 64-multiple requirement here)
- *   row_adapter  device [n_rows] int32, each in [-1, layer->n_adapters); NOT checked on the host
+ *   row_adapter  device [n_rows] int32, each in [-1, layer->n_adapters).  The table lives on the device, so
+ *                the host cannot check it; the kernels treat an id outside that range as -1 (the row
+ *                gets the base product only) and never index the adapter tables with it
  *   X, Y         device [n_rows, d_in] / [n_rows, d_out], row strides ldx / ldy
  * Runs on the CURRENT device, asynchronously on the given stream.  Nothing is saved for
  * fine-tuning; use the planned path for that.

@@ -26,6 +26,7 @@ EXPORTS = (
     "mlora_backward", "mlora_poll_status", "mlora_status_string", "mlora_launch_count", "mlora_set_gemm_path",
     "mlora_profile_enable", "mlora_profile_collect", "mlora_forward_noalloc", "mlora_adamw_update",
     "mlora_set_cancel_flag", "mlora_set_dropout", "mlora_plan_create_async", "mlora_plan_release",
+    "mlora_selftest_timeout",
 )
 MLORA_NOALLOC_MAX_ROWS = 512
 
@@ -112,6 +113,8 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.mlora_set_cancel_flag.restype = ctypes.c_int
     lib.mlora_set_dropout.argtypes = [vp, ctypes.c_double, ctypes.c_uint64]
     lib.mlora_set_dropout.restype = ctypes.c_int
+    lib.mlora_selftest_timeout.argtypes = [vp, ctypes.c_uint32, vp]
+    lib.mlora_selftest_timeout.restype = ctypes.c_int
     lib.mlora_forward_noalloc.argtypes = [P(mlora_layer_t), vp, i32, vp, i64, vp, i64, vp]
     lib.mlora_forward_noalloc.restype = ctypes.c_int
     _lib = lib
@@ -245,6 +248,11 @@ def mlora_backward(ctx, layer: mlora_layer_t, plan, dY, x_save, u_save, dA, dB, 
 
 def mlora_poll_status(ctx, stream=None) -> int:
     return int(load_library().mlora_poll_status(ctx, _stream_ptr(stream)))
+
+
+def mlora_selftest_timeout(ctx, polls: int = 1024, stream=None) -> None:
+    """Queue the kernel whose bounded wait runs out on purpose (the next poll reports the timeout)."""
+    _check(load_library().mlora_selftest_timeout(ctx, int(polls), _stream_ptr(stream)), "mlora_selftest_timeout")
 
 
 def mlora_launch_count(ctx) -> int:

@@ -60,6 +60,8 @@ struct mlora_ctx {
   float* ws_splitk = nullptr;        // fp32 partial products of a K-split GEMM (fixed size, see kSplitKBytes)
   float* ws_gpart = nullptr;         // row-split gradient groups: [sm_count][64][512] fp32 partial sums
   int32_t* ws_gcounters = nullptr;   // [sm_count] arrival counters of those groups, zero between launches
+  std::vector<void*> retired;        // workspaces replaced by larger ones: kept until the context is destroyed,
+                                     // because a captured graph may still hold their addresses
   std::vector<PlanBuf> plan_pool;    // released buffers of stream-ordered plans
   int64_t launches = 0;
   int32_t gemm_path = 0;
@@ -131,6 +133,10 @@ struct BlobBuilder {
 // compute call allocates.  Problems whose partials do not fit run unsplit.
 constexpr size_t kSplitKBytes = 64u << 20;
 constexpr int kMaxDevices = 64;      // device ordinals a process may create contexts on
+// One-time kernel attributes (opt-in shared-memory size, resident cluster count) are cached per kernel
+// instantiation and device in function-local arrays; contexts are independent across host threads, so
+// two threads may reach the same cache at once: every read-check-set of such a cache holds this lock.
+std::mutex g_attr_mutex;
 
 // With MLORA_DEBUG set in the environment, the place and the runtime's message of a failed CUDA call go to stderr.
 mlora_status_t cuda_failure(const char* site, const char* detail) {
@@ -285,9 +291,12 @@ mlora_status_t launch_shrink_stream_d(mlora_ctx* ctx, ShrinkArgs a, int n_items,
   static bool attr_set_dev[kMaxDevices] = {};   // per instantiation and device
   bool& attr_set = attr_set_dev[ctx->device];
   auto kern = shrink_stream_kernel<RB, STAGES, CHUNK, DROP>;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return MLORA_ERR_CUDA;
-    attr_set = true;
+  {
+    std::lock_guard<std::mutex> lock(g_attr_mutex);
+    if (!attr_set) {
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return MLORA_ERR_CUDA;
+      attr_set = true;
+    }
   }
   StreamArgs sa;
   sa.s = a;
@@ -356,9 +365,12 @@ mlora_status_t launch_grad_stream2_d(mlora_ctx* ctx, const mlora_plan* p, const 
   static bool attr_set_dev[kMaxDevices] = {};   // per instantiation and device
   bool& attr_set = attr_set_dev[ctx->device];
   auto kern = grad_stream_kernel<MB, DROP, CB>;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return MLORA_ERR_CUDA;
-    attr_set = true;
+  {
+    std::lock_guard<std::mutex> lock(g_attr_mutex);
+    if (!attr_set) {
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return MLORA_ERR_CUDA;
+      attr_set = true;
+    }
   }
   CUtensorMap tQ0, tQ1;
   mlora_status_t ms;
@@ -420,10 +432,13 @@ mlora_status_t launch_grad(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& 
   constexpr int smem1 = (GRAD_THREADS / 32) * 16 * 65 * 4, smem2 = 2 * smem1;
   static bool attr_set_dev[kMaxDevices] = {};   // per instantiation and device
   bool& attr_set = attr_set_dev[ctx->device];
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(grad_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2) != cudaSuccess)
-      return MLORA_ERR_CUDA;
-    attr_set = true;
+  {
+    std::lock_guard<std::mutex> lock(g_attr_mutex);
+    if (!attr_set) {
+      if (cudaFuncSetAttribute(grad_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2) != cudaSuccess)
+        return MLORA_ERR_CUDA;
+      attr_set = true;
+    }
   }
   LaunchScope scope(ctx, st, KIND_GRAD);
   if (a.R <= 16) {
@@ -454,10 +469,13 @@ mlora_status_t launch_gemm_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUten
   static bool attr_set_dev[kMaxDevices] = {};   // per instantiation and device: the attribute belongs to the device's context
   bool& attr_set = attr_set_dev[ctx->device];
   auto kern = gemm_lora_kernel<R, W_KMAJOR>;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_BYTES) != cudaSuccess)
-      return MLORA_ERR_CUDA;
-    attr_set = true;
+  {
+    std::lock_guard<std::mutex> lock(g_attr_mutex);
+    if (!attr_set) {
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_BYTES) != cudaSuccess)
+        return MLORA_ERR_CUDA;
+      attr_set = true;
+    }
   }
   if (cancelled(ctx)) return MLORA_CANCELLED;
   const int grid = g.n_units < ctx->sm_count ? g.n_units : ctx->sm_count;
@@ -473,6 +491,7 @@ mlora_status_t launch_gemm2_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUte
   static int max_pairs_dev[kMaxDevices] = {};   // per instantiation and device
   int& max_pairs = max_pairs_dev[ctx->device];
   auto kern = gemm2_lora_kernel<R, W_KMAJOR>;
+  std::unique_lock<std::mutex> attr_lock(g_attr_mutex);
   if (max_pairs == 0) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM2_SMEM_BYTES) != cudaSuccess)
       return MLORA_ERR_CUDA;
@@ -486,8 +505,9 @@ mlora_status_t launch_gemm2_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUte
     if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) { cudaGetLastError(); return MLORA_ERR_CUDA; }
     max_pairs = n;
   }
-  if (cancelled(ctx)) return MLORA_CANCELLED;
   const int pairs = g.n_units < max_pairs ? g.n_units : max_pairs;
+  attr_lock.unlock();
+  if (cancelled(ctx)) return MLORA_CANCELLED;
   LaunchScope scope(ctx, st, W_KMAJOR ? KIND_GEMM_BWD : KIND_GEMM_FWD);
   launch_pdl_pairs(scope.slot < 0, kern, dim3(2 * pairs), dim3(GEMM2_THREADS), GEMM2_SMEM_BYTES, st, tIn, tW, tL, tOut, tPbd, g);
   return scope.done();
@@ -621,27 +641,27 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
 template <typename T>
 mlora_status_t simt_shrink(mlora_ctx* ctx, const T* In, int64_t ld_in, int D, int R, const T* P_all,
                            const float* scale, const DevRowSpace& ds, float* Out, T* x_save, float* u_save,
-                           int64_t save_base, int n_rows, const DropArgs& drop, cudaStream_t st) {
+                           int64_t save_base, int n_rows, int n_adapters, const DropArgs& drop, cudaStream_t st) {
   if (n_rows <= 0) return MLORA_OK;
   if (cancelled(ctx)) return MLORA_CANCELLED;
   const int64_t warps = (int64_t)n_rows * R;
   const int blocks = (int)((warps * 32 + 255) / 256);
   LaunchScope scope(ctx, st, KIND_SIMT);
   simt::shrink_kernel<T><<<blocks, 256, 0, st>>>(In, ld_in, D, R, P_all, scale, ds.row_adapter, ds.row_save, Out,
-                                                 x_save, u_save, save_base, n_rows, drop);
+                                                 x_save, u_save, save_base, n_rows, n_adapters, drop);
   return scope.done();
 }
 
 template <typename T, bool W_KMAJOR>
 mlora_status_t simt_gemm(mlora_ctx* ctx, const T* In, int64_t ld_in, const T* W, int64_t ldw, const T* L_all,
                          const float* P, const float* scale, const DevRowSpace& ds, T* Out, int64_t ld_out, int M,
-                         int N, int K, int R, const DropArgs& drop, cudaStream_t st) {
+                         int N, int K, int R, int n_adapters, const DropArgs& drop, cudaStream_t st) {
   if (M <= 0) return MLORA_OK;
   if (cancelled(ctx)) return MLORA_CANCELLED;
   dim3 grid((N + 31) / 32, (M + 31) / 32), block(32, 32);
   LaunchScope scope(ctx, st, KIND_SIMT);
   simt::gemm_lora_kernel<T, W_KMAJOR><<<grid, block, 0, st>>>(In, ld_in, W, ldw, L_all, P, scale, ds.row_adapter, Out,
-                                                              ld_out, M, N, K, R, drop);
+                                                              ld_out, M, N, K, R, n_adapters, drop);
   return scope.done();
 }
 
@@ -663,10 +683,10 @@ mlora_status_t forward_simt(mlora_ctx* ctx, const mlora_layer_t* L, const mlora_
                             void* Y, int64_t ldy, void* x_save, float* u_save, int64_t save_base, cudaStream_t st) {
   const DropArgs off = {0, 0, 1.0f};
   mlora_status_t s = simt_shrink<T>(ctx, (const T*)X, ldx, L->d_in, L->rank, (const T*)L->A_all, nullptr, p->fwd,
-                                    ctx->ws_p, (T*)x_save, u_save, save_base, p->h.n_rows, ctx->drop, st);
+                                    ctx->ws_p, (T*)x_save, u_save, save_base, p->h.n_rows, L->n_adapters, ctx->drop, st);
   if (s != MLORA_OK) return s;
   return simt_gemm<T, false>(ctx, (const T*)X, ldx, (const T*)L->W, L->ldw, (const T*)L->B_all, ctx->ws_p, L->scale,
-                             p->fwd, (T*)Y, ldy, p->h.n_rows, L->d_out, L->d_in, L->rank, off, st);
+                             p->fwd, (T*)Y, ldy, p->h.n_rows, L->d_out, L->d_in, L->rank, L->n_adapters, off, st);
 }
 
 template <typename T>
@@ -676,7 +696,7 @@ mlora_status_t backward_simt(mlora_ctx* ctx, const mlora_layer_t* L, const mlora
   const int Tft = p->h.ft_rows;
   const DropArgs off = {0, 0, 1.0f};
   mlora_status_t s = simt_shrink<T>(ctx, (const T*)dY, lddy, L->d_out, L->rank, (const T*)L->B_all, L->scale, p->bwd,
-                                    ctx->ws_p, (T*)nullptr, nullptr, 0, Tft, off, st);
+                                    ctx->ws_p, (T*)nullptr, nullptr, 0, Tft, L->n_adapters, off, st);
   if (s != MLORA_OK) return s;
   if ((s = simt_grad<T>(ctx, p, u_save, L->rank, L->scale, (const T*)dY, lddy, L->d_out, dB, accumulate, off, st)) != MLORA_OK)
     return s;
@@ -685,7 +705,7 @@ mlora_status_t backward_simt(mlora_ctx* ctx, const mlora_layer_t* L, const mlora
     return s;
   if (dX)
     s = simt_gemm<T, true>(ctx, (const T*)dY, lddy, (const T*)L->W, L->ldw, (const T*)L->A_all, ctx->ws_p, nullptr,
-                           p->bwd, (T*)dX, lddx, Tft, L->d_in, L->d_out, L->rank, ctx->drop, st);
+                           p->bwd, (T*)dX, lddx, Tft, L->d_in, L->d_out, L->rank, L->n_adapters, ctx->drop, st);
   return s;
 }
 
@@ -723,15 +743,17 @@ mlora_status_t forward_noalloc_t(const mlora_layer_t* L, const int32_t* row_adap
                                  int64_t ldx, void* Y, int64_t ldy, float* scratch, cudaStream_t st) {
   const int64_t warps = (int64_t)n_rows * L->rank;
   const int blocks = (int)((warps * 32 + 255) / 256);
-  // rank-r intermediate of every row (zeros for rows without an adapter) -> scratch
+  // rank-r intermediate of every row (zeros for rows without an adapter, or with an id outside the layer's
+  // adapter tables: the caller's device table has not been validated by anyone) -> scratch
   simt::shrink_kernel<T><<<blocks, 256, 0, st>>>((const T*)X, ldx, L->d_in, L->rank, (const T*)L->A_all, nullptr,
                                                  row_adapter, nullptr, scratch, (T*)nullptr, nullptr, 0, n_rows,
-                                                 DropArgs{0, 0, 1.0f});
+                                                 L->n_adapters, DropArgs{0, 0, 1.0f});
   if (cudaGetLastError() != cudaSuccess) return MLORA_ERR_CUDA;
   dim3 grid((L->d_out + 31) / 32, (n_rows + 31) / 32), block(32, 32);
   simt::gemm_lora_kernel<T, false><<<grid, block, 0, st>>>((const T*)X, ldx, (const T*)L->W, L->ldw,
                                                            (const T*)L->B_all, scratch, L->scale, row_adapter, (T*)Y,
-                                                           ldy, n_rows, L->d_out, L->d_in, L->rank, DropArgs{0, 0, 1.0f});
+                                                           ldy, n_rows, L->d_out, L->d_in, L->rank, L->n_adapters,
+                                                           DropArgs{0, 0, 1.0f});
   return cudaGetLastError() == cudaSuccess ? MLORA_OK : MLORA_ERR_CUDA;
 }
 }  // namespace
@@ -851,6 +873,7 @@ void mlora_destroy(mlora_ctx* c) {
   cudaFree(c->ws_splitk);
   cudaFree(c->ws_gpart);
   cudaFree(c->ws_gcounters);
+  for (void* r : c->retired) cudaFree(r);
   for (PlanBuf& b : c->plan_pool) free_plan_buf(b);
   delete c;
 }
@@ -894,36 +917,43 @@ void bind_plan(mlora_plan* p, const size_t* o) {
   p->slot_blk_off = p->blob + o[n++]; p->blk_row0 = p->blob + o[n++]; p->blk_nrows = p->blob + o[n++];
 }
 
-// Grows the context's workspaces to what this plan needs (synchronises the device when it has to
-// grow one; in steady state nothing happens here).
+// Grows the context's workspaces to what this plan needs.  A workspace that is too small is REPLACED
+// by a larger one (at least half as large again), never freed or moved: the old block stays allocated
+// until mlora_destroy, so launches that already carry its address - kernels still queued, and above
+// all kernels inside a captured CUDA graph - keep working on memory that is theirs.  In steady state
+// nothing happens here.
+mlora_status_t replace_workspace(mlora_ctx* ctx, void** ptr, size_t bytes, bool zero) {
+  void* fresh = nullptr;
+  if (cudaMalloc(&fresh, bytes) != cudaSuccess) { cudaGetLastError(); return MLORA_ERR_CUDA; }
+  if (zero && cudaMemset(fresh, 0, bytes) != cudaSuccess) { cudaFree(fresh); return MLORA_ERR_CUDA; }
+  if (*ptr) ctx->retired.push_back(*ptr);
+  *ptr = fresh;
+  return MLORA_OK;
+}
+
 mlora_status_t grow_workspaces(mlora_ctx* ctx, const HostPlan& h, int32_t n_rows) {
+  mlora_status_t s;
+  auto grown = [](int64_t need, int64_t have) { return need > have + have / 2 ? need : have + have / 2; };
   if (n_rows > ctx->ws_rows) {     // the rank-r workspace
-    if (cudaDeviceSynchronize() != cudaSuccess) return MLORA_ERR_CUDA;
-    cudaFree(ctx->ws_p);
-    ctx->ws_p = nullptr; ctx->ws_rows = 0;
-    if (cudaMalloc(&ctx->ws_p, (size_t)n_rows * kMaxRank * sizeof(float)) != cudaSuccess) return MLORA_ERR_CUDA;
-    ctx->ws_rows = n_rows;
+    const int64_t rows = grown(n_rows, ctx->ws_rows);
+    if ((s = replace_workspace(ctx, (void**)&ctx->ws_p, (size_t)rows * kMaxRank * sizeof(float), false)) != MLORA_OK) return s;
+    ctx->ws_rows = rows;
   }
   const int64_t items = h.fwd.n_items() > h.bwd.n_items() ? h.fwd.n_items() : h.bwd.n_items();
-  const int64_t part_items = items + 4 * ctx->sm_count;      // items * ksplit never exceeds this
-  if (part_items > ctx->ws_partial_items || items > ctx->ws_counter_items) {
-    if (cudaDeviceSynchronize() != cudaSuccess) return MLORA_ERR_CUDA;
-    cudaFree(ctx->ws_partial); cudaFree(ctx->ws_counters);
-    ctx->ws_partial = nullptr; ctx->ws_counters = nullptr; ctx->ws_partial_items = ctx->ws_counter_items = 0;
-    if (cudaMalloc(&ctx->ws_partial, (size_t)part_items * kItemRows * kMaxRank * sizeof(float)) != cudaSuccess ||
-        cudaMalloc(&ctx->ws_counters, (size_t)(2 * items + 1) * sizeof(int32_t)) != cudaSuccess ||
-        cudaMemset(ctx->ws_counters, 0, (size_t)(2 * items + 1) * sizeof(int32_t)) != cudaSuccess)
-      return MLORA_ERR_CUDA;
-    ctx->ws_partial_items = part_items; ctx->ws_counter_items = items;
+  if (items + 4 * ctx->sm_count > ctx->ws_partial_items || items > ctx->ws_counter_items) {
+    const int64_t it = grown(items, ctx->ws_counter_items);
+    const int64_t part_items = it + 4 * ctx->sm_count;      // items * ksplit never exceeds this
+    if ((s = replace_workspace(ctx, (void**)&ctx->ws_partial, (size_t)part_items * kItemRows * kMaxRank * sizeof(float), false)) != MLORA_OK ||
+        (s = replace_workspace(ctx, (void**)&ctx->ws_counters, (size_t)(2 * it + 1) * sizeof(int32_t), true)) != MLORA_OK)
+      return s;
+    ctx->ws_partial_items = part_items; ctx->ws_counter_items = it;
   }
   const int64_t groups = (int64_t)(h.fwd.grp2_adapter.size() > h.bwd.grp2_adapter.size() ? h.fwd.grp2_adapter.size()
                                                                                         : h.bwd.grp2_adapter.size());
   if (groups > ctx->ws_pbd_groups) {   // two chunk slots of [256][64] bf16 per adapter group of a tile
-    if (cudaDeviceSynchronize() != cudaSuccess) return MLORA_ERR_CUDA;
-    cudaFree(ctx->ws_pbd);
-    ctx->ws_pbd = nullptr; ctx->ws_pbd_groups = 0;
-    if (cudaMalloc(&ctx->ws_pbd, (size_t)groups * 2 * 256 * 64 * sizeof(__nv_bfloat16)) != cudaSuccess) return MLORA_ERR_CUDA;
-    ctx->ws_pbd_groups = groups;
+    const int64_t g = grown(groups, ctx->ws_pbd_groups);
+    if ((s = replace_workspace(ctx, (void**)&ctx->ws_pbd, (size_t)g * 2 * 256 * 64 * sizeof(__nv_bfloat16), false)) != MLORA_OK) return s;
+    ctx->ws_pbd_groups = g;
   }
   return MLORA_OK;
 }
@@ -1185,10 +1215,23 @@ mlora_status_t mlora_poll_status(mlora_ctx* ctx, void* cuda_stream) {
   if (cudaMemcpyAsync(&v, ctx->status_dev, sizeof(v), cudaMemcpyDeviceToHost, st) != cudaSuccess) return MLORA_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return MLORA_ERR_CUDA;
   if (v != 0) {
+    // A kernel that gave up may have left the arrival counters of split work items partly counted (only a
+    // launch that runs to its end puts them back to zero), so they are cleared together with the word.
     cudaMemsetAsync(ctx->status_dev, 0, sizeof(v), st);
+    if (ctx->ws_counters) cudaMemsetAsync(ctx->ws_counters, 0, (size_t)(2 * ctx->ws_counter_items + 1) * sizeof(int32_t), st);
+    cudaMemsetAsync(ctx->ws_gcounters, 0, (size_t)ctx->sm_count * sizeof(int32_t), st);
     cudaStreamSynchronize(st);
   }
   return (mlora_status_t)v;
+}
+
+mlora_status_t mlora_selftest_timeout(mlora_ctx* ctx, uint32_t polls, void* cuda_stream) {
+  if (!ctx || polls == 0 || polls > (1u << 20)) return MLORA_ERR_INVALID_ARG;
+  if (cudaSetDevice(ctx->device) != cudaSuccess) return MLORA_ERR_CUDA;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  LaunchScope scope(ctx, st, KIND_SIMT);
+  wait_selftest_kernel<<<1, 64, 0, st>>>(ctx->status_dev, polls);
+  return scope.done();
 }
 
 mlora_status_t mlora_set_cancel_flag(mlora_ctx* ctx, const volatile int32_t* host_flag) {
@@ -1215,18 +1258,6 @@ mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path) {
   ctx->no_split_k = path == 4 ? 1 : 0;
   return MLORA_OK;
 }
-
-#ifdef MLORA_TIMELINE
-// Development aid, not part of the ABI: copies the per-CTA clock stamps of the last streaming launch.
-int mlora_debug_timeline(long long* host, int n) {
-  if (cudaDeviceSynchronize() != cudaSuccess) return -1;
-  return cudaMemcpyFromSymbol(host, mlora::g_timeline, sizeof(long long) * (size_t)n) == cudaSuccess ? 0 : -1;
-}
-int mlora_debug_timeline_reset() {
-  static long long zeros[160 * 16];
-  return cudaMemcpyToSymbol(mlora::g_timeline, zeros, sizeof(zeros)) == cudaSuccess ? 0 : -1;
-}
-#endif
 
 // ---- layer pieces around the projections (mlora_layer_ops.h) ----------------------------------
 static inline mlora_status_t launched() {
@@ -1303,6 +1334,7 @@ mlora_status_t mlora_add(const void* a, const void* b, void* out, int64_t n, voi
 // Head size 128: the tcgen05 kernels.  The layer pieces have no context object, so the tensor-map
 // encoder is looked up once per process here (only that entry of the object is used).
 static mlora_ctx* layer_ops_encoder() {
+  // function-local statics: the language runs this initialisation once, under its own lock
   static mlora_ctx enc;
   static bool ok = [] {
     void* fn = nullptr;
@@ -1320,6 +1352,7 @@ template <typename Kern>
 static mlora_status_t attn_tc_smem(Kern kern, uint32_t bytes, bool* done_dev) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MLORA_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_attr_mutex);
   if (!done_dev[dev]) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) return MLORA_ERR_CUDA;
     done_dev[dev] = true;

@@ -18,17 +18,20 @@ __device__ __forceinline__ void st(float* p, float v) { *p = v; }
 __device__ __forceinline__ void st(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 
 // Out[t, q] = (scale?) * sum_k In[t, k] P_a(t)[q, k]; one warp per (row, q); rows without an
-// adapter get zeros.  Fine-tuning rows (row_save >= 0) also write u_save (unscaled) and x_save;
+// adapter get zeros, and so do rows whose id lies outside [-1, n_adapters) (the planned path has
+// validated its ids on the host; a caller-supplied device table has not been looked at by anyone).  Fine-tuning rows (row_save >= 0) also write u_save (unscaled) and x_save;
 // with dropout on, their products skip the dropped columns and count 1 / (1 - p).
 template <typename T>
 __global__ void shrink_kernel(const T* In, int64_t ld_in, int D, int R, const T* P_all, const float* scale,
                               const int32_t* row_adapter, const int32_t* row_save, float* Out,
-                              T* x_save, float* u_save, int64_t save_base, int n_rows, const DropArgs drop) {
+                              T* x_save, float* u_save, int64_t save_base, int n_rows, int n_adapters,
+                              const DropArgs drop) {
   const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (wid >= n_rows * R) return;
   const int t = wid / R, q = wid % R;
-  const int a = row_adapter[t];
+  int a = row_adapter[t];
+  if (a >= n_adapters) a = -1;
   const int sv = row_save ? row_save[t] : -1;
   float acc = 0.f;
   if (a >= 0) {
@@ -62,7 +65,8 @@ __global__ void shrink_kernel(const T* In, int64_t ld_in, int D, int R, const T*
 template <typename T, bool W_KMAJOR>
 __global__ void gemm_lora_kernel(const T* In, int64_t ld_in, const T* W, int64_t ldw, const T* L_all,
                                  const float* P, const float* scale, const int32_t* row_adapter,
-                                 T* Out, int64_t ld_out, int M, int N, int K, int R, const DropArgs drop) {
+                                 T* Out, int64_t ld_out, int M, int N, int K, int R, int n_adapters,
+                                 const DropArgs drop) {
   __shared__ float sIn[32][33];
   __shared__ float sW[32][33];
   const int tx = threadIdx.x, ty = threadIdx.y;
@@ -85,7 +89,7 @@ __global__ void gemm_lora_kernel(const T* In, int64_t ld_in, const T* W, int64_t
   }
   if (m < M && n < N) {
     const int a = row_adapter ? row_adapter[m] : -1;
-    if (a >= 0) {
+    if (a >= 0 && a < n_adapters) {        // an id outside the adapter tables counts as no adapter
       const float sc = scale ? scale[a] : 1.0f;
       float lo = 0.f;
       for (int q = 0; q < R; ++q) lo = fmaf(P[(size_t)m * R + q], ld(L_all + ((size_t)a * R + q) * N + n), lo);

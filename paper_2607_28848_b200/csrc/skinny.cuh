@@ -266,17 +266,6 @@ constexpr int STREAM_THREADS = (STREAM_WARPS + 1) * 32;
 // bytes apart, so that fragment loads hit distinct banks.
 constexpr uint32_t STREAM_SPIN_LIMIT = 1u << 22;
 
-#ifdef MLORA_TIMELINE
-// Development aid (off in the product build): per-CTA clock stamps of the streaming kernels.
-__device__ long long g_timeline[160 * 16];
-__device__ __forceinline__ long long tl_clock() { return clock64(); }
-__device__ __forceinline__ long long tl_global() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define MLORA_TL_SET(slot, v) do { g_timeline[blockIdx.x * 16 + (slot)] = (v); } while (0)
-#define MLORA_TL_ADD(slot, v) do { g_timeline[blockIdx.x * 16 + (slot)] += (v); } while (0)
-#else
-#define MLORA_TL_SET(slot, v) do {} while (0)
-#define MLORA_TL_ADD(slot, v) do {} while (0)
-#endif
 
 struct StreamArgs {
   ShrinkArgs s;
@@ -299,14 +288,36 @@ __device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
   asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
   return v;
 }
-__device__ __forceinline__ bool stream_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  for (uint32_t i = 0; i < STREAM_SPIN_LIMIT; ++i) {
+__device__ __forceinline__ bool stream_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                            uint32_t limit = STREAM_SPIN_LIMIT) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 255u && *abort_flag) return false;
   }
   *abort_flag = 1;
   atomicExch(status, (int32_t)MLORA_ERR_DEVICE_TIMEOUT);
   return false;
+}
+
+// Self-test of the give-up path shared by every bounded wait: one thread waits, with the helper the
+// streaming kernels use, on a barrier that nothing will ever arrive at, for `polls` polls.  The wait
+// then runs out, raises the CTA's abort flag, leaves MLORA_ERR_DEVICE_TIMEOUT in the status word and
+// the kernel returns normally - no copy is in flight and no tensor memory is held, so nothing has to
+// be drained.  A second thread then waits on the same barrier: it finds the abort flag at its first
+// look at it and leaves at once, as the other warps of a streaming CTA do.
+__global__ void __launch_bounds__(64)
+wait_selftest_kernel(int32_t* status, uint32_t polls) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_word;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(ptx::smem_u32(&bar), 1);
+    abort_word = 0;
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) stream_wait(ptx::smem_u32(&bar), 0, &abort_word, status, polls);
+  __syncthreads();
+  if (threadIdx.x == 32) stream_wait(ptx::smem_u32(&bar), 0, &abort_word, status, 512u);
 }
 
 template <int RB, int STAGES, int CHUNK, bool DROP>
@@ -347,12 +358,6 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
   float (*red)[32][R + 1] = reinterpret_cast<float (*)[32][R + 1]>(
       stream_smem + (ring - ptx::smem_u32(stream_smem)) + STAGES * STAGE_BYTES);
 
-#ifdef MLORA_TIMELINE
-  const long long tl0 = tl_clock();
-  const bool tl_on = threadIdx.x == 0;
-  long long tl_wait = 0, tl_flush = 0, tl_nflush = 0;
-  if (tl_on) { for (int i = 0; i < 16; ++i) MLORA_TL_SET(i, 0); MLORA_TL_SET(14, tl_global()); }
-#endif
   if (threadIdx.x == 0) {
     for (int st = 0; st < STAGES; ++st) {
       ptx::mbar_init(bar_full(st), 1);
@@ -457,21 +462,12 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
     float my_scale = 1.0f, pb_scale = 1.0f;
     int pb_row[32 / STREAM_WARPS], pb_goff[32 / STREAM_WARPS], pb_G[32 / STREAM_WARPS], pb_g[32 / STREAM_WARPS];
     // this thread's pieces of a K-block: elements 16c .. 16c+15 of the block
-#ifdef MLORA_TIMELINE
-    if (tl_on) MLORA_TL_SET(1, tl_clock() - tl0);
-#endif
     ptx::grid_dependency_wait();
-#ifdef MLORA_TIMELINE
-    if (tl_on) MLORA_TL_SET(2, tl_clock() - tl0);
-#endif
     bool ok = true;
     if (a.pbd.pbd)                                            // rows nobody else owns: all-zero chunks
       for (int i = cta * STREAM_WARPS + warp; i < a.pbd.n_zero_rows; i += gridDim.x * STREAM_WARPS)
         pbd_write_row<R>(a.pbd, a.pbd.zero_rows[i], nullptr, 0.f, lane);
 
-#ifdef MLORA_TIMELINE
-    if (tl_on) MLORA_TL_SET(3, tl_clock() - tl0);
-#endif
     for (int u = u_begin; u < u_end; ++u) {
       const int i = u - u_begin, st = i % STAGES;
       if (item != cur_item) {
@@ -481,9 +477,6 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
         cur_adapter = d0.z;
         cur_contig = d0.w & 1;
         const bool block_saved = sa.tma_save && (d0.w & 2);   // the producer stores this item's rows
-#ifdef MLORA_TIMELINE
-        if (tl_on) MLORA_TL_SET(11, 8 + d0.w + (block_saved ? 4 : 0) + ((cur_saves && cur_saves[0] >= 0) ? 16 : 0));
-#endif
         cur_rows = a.item_rows + d0.x;
         cur_saves = a.item_save ? a.item_save + d0.x : nullptr;
 #pragma unroll
@@ -515,14 +508,8 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
           }
         }
       }
-#ifdef MLORA_TIMELINE
-      const long long tw0 = tl_clock();
-#endif
       ok = stream_wait(bar_full(st), (i / STAGES) & 1, abort_flag, sa.status);
       if (!ok) break;
-#ifdef MLORA_TIMELINE
-      if (tl_on) { tl_wait += tl_clock() - tw0; if (i == 0) MLORA_TL_SET(4, tl_clock() - tl0); }
-#endif
 #pragma unroll
       for (int kk = 0; kk < CHUNK / STREAM_WARPS; ++kk) {
         const int kb = kc * CHUNK + kk * STREAM_WARPS + warp;
@@ -602,10 +589,6 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
       const int this_item = item;
       if (++kc == KC) { kc = 0; ++item; }
       if (!item_ends) continue;
-#ifdef MLORA_TIMELINE
-      const long long tf0 = tl_clock();
-      if (tl_on && u == u_end - 1) MLORA_TL_SET(5, tf0 - tl0);
-#endif
 #pragma unroll
       for (int round = 0; round < STREAM_WARPS / RW; ++round) {
         if (warp / RW == round) {
@@ -674,13 +657,7 @@ shrink_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_cons
         }
       }
       asm volatile("bar.sync 1, %0;" ::"n"(STREAM_WARPS * 32) : "memory");      // red[] and fin[] are reused by the next item
-#ifdef MLORA_TIMELINE
-      if (tl_on) { tl_flush += tl_clock() - tf0; ++tl_nflush; }
-#endif
     }
-#ifdef MLORA_TIMELINE
-    if (tl_on) { MLORA_TL_SET(9, tl_clock() - tl0); MLORA_TL_SET(15, tl_global()); MLORA_TL_SET(10, u_end - u_begin); MLORA_TL_SET(8, tl_wait); MLORA_TL_SET(6, tl_flush); MLORA_TL_SET(7, tl_nflush); }
-#endif
   }
 }
 
@@ -887,16 +864,6 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
   const int R = ga.R;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-#ifdef MLORA_TIMELINE
-  const long long tl0 = tl_clock();
-#ifdef MLORA_TL_NO_GRAD
-  const bool tl_on = false;
-#else
-  const bool tl_on = threadIdx.x == 0;
-#endif
-  long long tl_wait = 0, tl_flush = 0, tl_nflush = 0, tl_nstage = 0;
-  if (tl_on) { for (int i = 0; i < 16; ++i) MLORA_TL_SET(i, 0); MLORA_TL_SET(14, tl_global()); }
-#endif
   const uint32_t ring = (ptx::smem_u32(gs_smem) + 1023u) & ~1023u;      // swizzled tiles need 1 KiB alignment
   const uint32_t bar0 = ptx::smem_u32(bars);
   auto bar_full = [&](int st) { return bar0 + 8u * st; };
@@ -984,13 +951,7 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
   } else {
     // ======================= consumers =======================
     const int g = lane >> 2, c = lane & 3;
-#ifdef MLORA_TIMELINE
-    if (tl_on) MLORA_TL_SET(1, tl_clock() - tl0);
-#endif
     ptx::grid_dependency_wait();
-#ifdef MLORA_TIMELINE
-    if (tl_on) { MLORA_TL_SET(2, tl_clock() - tl0); MLORA_TL_SET(3, tl_clock() - tl0); }
-#endif
     float acc[MB][8][4];
     uint32_t i = 0;
     bool ok = true;
@@ -1010,13 +971,7 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
         for (int n = 0; n < 8; ++n) acc[m][n][0] = acc[m][n][1] = acc[m][n][2] = acc[m][n][3] = 0.f;
       for (bool last = false; !last; ++i) {
         const int st = i % S;
-#ifdef MLORA_TIMELINE
-        const long long tw0 = tl_clock();
-#endif
         if (!(ok = stream_wait(bar_full(st), (i / S) & 1, abort_flag, ga.status))) break;
-#ifdef MLORA_TIMELINE
-        if (tl_on) { tl_wait += tl_clock() - tw0; if (i == 0) MLORA_TL_SET(4, tl_clock() - tl0); ++tl_nstage; }
-#endif
         const int trow0 = stage_meta[st][0];
         const int meta = stage_meta[st][1];
         const int nrows = meta & 0xFFFF;
@@ -1083,10 +1038,6 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
         if (lane == 0) ptx::mbar_arrive(bar_empty(st));
       }
       if (!ok) break;
-#ifdef MLORA_TIMELINE
-      const long long tf0 = tl_clock();
-      if (tl_on && un + (int)gridDim.x >= n_units) MLORA_TL_SET(5, tf0 - tl0);
-#endif
       // ---- group done: this warp's 16 (32) x 64 block goes from registers to the gradient ----
       // The n index g of the MMA was mapped to piece g of a row, so for thread (g, c) accumulator
       // element e of column block nb is strip column 8 (2c + (e & 1)) + nb: over nb = 0..7 that is
@@ -1175,13 +1126,7 @@ grad_stream_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_consta
             dst[1] = hi;
           }
       }
-#ifdef MLORA_TIMELINE
-      if (tl_on) { tl_flush += tl_clock() - tf0; ++tl_nflush; }
-#endif
     }
-#ifdef MLORA_TIMELINE
-    if (tl_on) { MLORA_TL_SET(9, tl_clock() - tl0); MLORA_TL_SET(15, tl_global()); MLORA_TL_SET(10, tl_nstage); MLORA_TL_SET(8, tl_wait); MLORA_TL_SET(6, tl_flush); MLORA_TL_SET(7, tl_nflush); }
-#endif
   }
 }
 

@@ -59,16 +59,31 @@ def uniform01(seed: int, tag: int, start: int, count: int) -> np.ndarray:
 
 
 def normal(seed: int, tag: int, count: int, std: float = 1.0, chunk: int = 1 << 22) -> np.ndarray:
-    """``count`` independent N(0, std^2) float64 draws (Box-Muller on counter pairs)."""
+    """``count`` independent N(0, std^2) float64 draws (Box-Muller on counter pairs).
+
+    Every element is a function of (seed, tag, index) alone, so the chunks are independent; large
+    draws spread them over the host's cores (numpy releases the interpreter lock inside its loops).
+    """
     out = np.empty(count, dtype=np.float64)
-    for lo in range(0, count, chunk):
+
+    def fill(lo: int) -> None:
         n = min(chunk, count - lo)
         u1 = uniform01(seed, tag, 2 * lo, 2 * n)
         u2 = u1[1::2]
         u1 = u1[0::2]
         out[lo:lo + n] = np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2)
-    if std != 1.0:
-        out *= std
+        if std != 1.0:
+            out[lo:lo + n] *= std
+
+    starts = range(0, count, chunk)
+    if len(starts) > 1:
+        import os
+        from concurrent.futures import ThreadPoolExecutor
+        with ThreadPoolExecutor(max_workers=min(len(starts), os.cpu_count() or 1)) as pool:
+            list(pool.map(fill, starts))
+    else:
+        for lo in starts:
+            fill(lo)
     return out
 
 

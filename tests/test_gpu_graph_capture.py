@@ -60,3 +60,40 @@ def test_graph_replay_matches_eager_on_new_inputs(case):
             assert torch.equal(a, b)
         assert float(run.Y.float().abs().max()) > 0
         run.close()
+
+
+def test_a_larger_plan_after_capture_leaves_the_graph_valid():
+    """A plan for a larger batch makes the context replace its workspaces by larger ones.  The blocks they
+    replace stay allocated, so a graph captured before still runs on memory of its own: its replay gives
+    the eager result, and so does the large batch."""
+    with Session(0) as sess:
+        w = synth.random_workload(64, 256, 384, 16, 5, 300, max_seg=90, p_finetune=0.4)
+        t = synth.make_tensors(w)
+        run = LayerRun(sess, "bf16", t, w.segments, w.n_rows)
+        stream = torch.cuda.Stream(device=sess.device)
+        with torch.cuda.stream(stream):
+            for _ in range(2):
+                run.forward(); run.backward()
+            stream.synchronize()
+            eager = [b.clone() for b in (run.Y, run.u_save, run.dA, run.dB, run.dX)]
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                run.forward(); run.backward()
+            # many more rows, items and adapter groups than anything this context has seen
+            big = synth.random_workload(65, 256, 384, 16, 40, 9000, max_seg=60, p_decode=0.6, p_finetune=0.3)
+            tb = synth.make_tensors(big)
+            run_big = LayerRun(sess, "bf16", tb, big.segments, big.n_rows)
+            run_big.forward(); run_big.backward()
+            stream.synchronize()
+            for b in (run.Y, run.u_save, run.dA, run.dB, run.dX):
+                b.zero_()
+            graph.replay()
+            stream.synchronize()
+        assert mb.mlora_poll_status(sess.ctx) == mb.MLORA_OK
+        for a, b in zip(eager, (run.Y, run.u_save, run.dA, run.dB, run.dX)):
+            assert torch.equal(a, b)
+        from oracle import mlora_oracle as orc
+        ref = orc.forward_blocked(tb["X"], tb["W"], tb["A_all"], tb["B_all"], tb["scale"], big.segments)["Y"]
+        got = run_big.host(run_big.Y)
+        assert (np.abs(got - ref) <= 2e-2 * (1 + np.abs(ref))).all()
+        run.close(); run_big.close()

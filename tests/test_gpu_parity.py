@@ -526,64 +526,89 @@ def test_cancel_flag_stops_between_kernels(sess):
     run.close()
 
 
-# ---- full-size configurations --------------------------------------------------------------
+def test_bounded_wait_runs_out_and_is_reported(sess):
+    """A wait inside a kernel that can never be satisfied gives up after its poll limit, the kernel returns,
+    and the status word carries MLORA_ERR_DEVICE_TIMEOUT until it is polled; the poll clears it (and the
+    arrival counters), and the same forward + backward before and after are bit-identical.  Nothing faults
+    or hangs: the kernel is the library's own self-test, one warp waiting 1024 polls on a barrier nobody
+    arrives at."""
+    segs = synth.segments_array([(0, 37, 3, 0), (37, 2048, 0, 1), (2085, 20, 1, 0)])     # one slot: row-split gradient groups
+    w = synth.Workload("timeout_probe", 2048, 512, 16, 4, "bf16", 2105, segs, seed=77)
+    t = synth.make_tensors(w)
+    run = LayerRun(sess, "bf16", t, w.segments, w.n_rows)
+    run.forward(); run.backward()
+    before = [x.clone() for x in (run.Y, run.u_save, run.dA, run.dB, run.dX)]
+    assert run.status() == mb.MLORA_OK
+    mb.mlora_selftest_timeout(sess.ctx, 1024)
+    assert mb.mlora_poll_status(sess.ctx) == mb.MLORA_ERR_DEVICE_TIMEOUT
+    assert mb.mlora_poll_status(sess.ctx) == mb.MLORA_OK
+    for b in (run.Y, run.u_save, run.dA, run.dB, run.dX):
+        b.zero_()
+    run.forward(); run.backward()
+    assert run.status() == mb.MLORA_OK
+    for a, b in zip(before, (run.Y, run.u_save, run.dA, run.dB, run.dX)):
+        assert torch.equal(a, b)
+    run.close()
+
+
+# ---- full-size configurations: every element of every output against the oracle --------------------
 def test_cfg2_full_size(sess):
     w = synth.cfg2_single_projection()
     run_and_check(sess, w, synth.make_tensors(w), blocked=True)
 
 
-def _sampled_check(sess, w, n_sample=24, seed=0):
-    """Full-size run in the benchmark's launch configuration; the oracle recomputes sampled rows of Y
-    and dX one by one and sampled columns of dA / dB."""
-    t = synth.make_tensors(w)
-    run = LayerRun(sess, w.dtype, t, w.segments, w.n_rows)
-    try:
-        run.forward()
-        assert run.status() == mb.MLORA_OK
-        rng = np.random.default_rng(seed)
-        rows = np.unique(np.concatenate([[0, w.n_rows - 1], rng.integers(0, w.n_rows, n_sample)]))
-        y_ref = orc.forward_rows(t["X"], t["W"], t["A_all"], t["B_all"], t["scale"], w.segments, rows)
-        assert_close("Y[sample]", run.host(run.Y[torch.from_numpy(rows).to(sess.device)]), y_ref, 2e-2)
-        _ra, ft, n, slots = orc.route(w.segments, w.n_rows, w.n_adapters)
-        if not n:
-            return
-        # saved rows: bit-exact against X for every fine-tuning row
-        src = np.concatenate([np.arange(s, s + ln) for s, ln, _a, _o in ft])
-        assert torch.equal(run.x_save[:n], run.X[torch.from_numpy(src).to(sess.device)])
-        run.backward()
-        assert run.status() == mb.MLORA_OK
-        A, B, W, sc = (t[k].astype(np.float64) for k in ("A_all", "B_all", "W", "scale"))
-        Xs = t["X"].astype(np.float64)[src]
-        dY = t["dY"].astype(np.float64)
-        m_ad = np.concatenate([np.full(ln, a) for _s, ln, a, _o in ft])
-        # V and U for all fine-tuning rows (cheap), then sampled rows / columns of the big outputs
-        V = np.stack([sc[a] * (B[a] @ dY[m]) for m, a in enumerate(m_ad)])
-        U = np.stack([A[a] @ Xs[m] for m, a in enumerate(m_ad)])
-        assert_close("u_save", run.host(run.u_save[:n]), U, 1e-3)
-        ms = np.unique(np.concatenate([[0, n - 1], rng.integers(0, n, n_sample)]))
-        dx_ref = np.stack([W @ dY[m] + V[m] @ A[m_ad[m]] for m in ms])
-        assert_close("dX[sample]", run.host(run.dX[torch.from_numpy(ms).to(sess.device)]), dx_ref, 2e-2)
-        cols_o = rng.integers(0, w.d_out, 16)
-        cols_i = rng.integers(0, w.d_in, 16)
-        dA, dB = run.host(run.dA), run.host(run.dB)
-        for g, a in enumerate(slots):
-            sel = m_ad == a
-            assert_close("dB[cols]", dB[g][:, cols_o], sc[a] * (U[sel].T @ dY[sel][:, cols_o]), 2e-2)
-            assert_close("dA[cols]", dA[g][:, cols_i], V[sel].T @ Xs[sel][:, cols_i], 2e-2)
-    finally:
-        run.close()
-
-
 @pytest.mark.parametrize("proj", ["q", "k", "v", "o", "gate", "up", "down"])
-def test_cfg3_projection_sampled(sess, proj):
-    _sampled_check(sess, synth.cfg3_layer_set(projections=[proj])[0])
+def test_cfg3_projection_full_size(sess, proj):
+    """The benchmark's launch configuration (banded tile order and the K split of the last wave included):
+    Y, the saved rows, u_save, dX, dA and dB element by element against oracle.forward_blocked /
+    oracle.backward_blocked."""
+    w = synth.cfg3_layer_set(projections=[proj])[0]
+    run_and_check(sess, w, synth.make_tensors(w), blocked=True)
 
 
-def test_cfg5_decode_heavy_sampled(sess):
-    _sampled_check(sess, synth.cfg5_decode_heavy())
+@pytest.mark.parametrize("mode", ["decode", "finetune", "mixed"])
+def test_cfg5_decode_heavy_full_size(sess, mode):
+    """The three runs the decode-heavy configuration reports: decode rows only, the fine-tuning segment
+    only, and both in one batch."""
+    w = synth.cfg5_decode_heavy(mode=mode)
+    run_and_check(sess, w, synth.make_tensors(w), blocked=True)
 
 
-@pytest.mark.parametrize("rank,n_adapters,f,sorted_rows", [(8, 256, 0.25, True), (128, 64, 0.5, True),
-                                                           (16, 64, 0.0, False)])
-def test_cfg4_points_sampled(sess, rank, n_adapters, f, sorted_rows):
-    _sampled_check(sess, synth.cfg4_sweep_point(rank, n_adapters, f, sorted_rows=sorted_rows), n_sample=12)
+_CFG4_CACHE = {}
+
+
+def _cfg4_tensors(w):
+    """synth.make_tensors for a sweep point, keeping the tensors that do not change from point to point
+    (X and W always, the adapters per (rank, adapter count)): every tensor is a pure function of
+    (seed, tag, shape), so the cached arrays are exactly what make_tensors would draw again."""
+    def draw(key, tag, shape, std):
+        if key not in _CFG4_CACHE:
+            n = int(np.prod(shape))
+            _CFG4_CACHE[key] = synth.round_to_storage(synth.normal(w.seed, w.tag_base + tag, n, std=std).reshape(shape), w.dtype)
+        return _CFG4_CACHE[key]
+    for k in [k for k in _CFG4_CACHE if k[0] in ("A", "B") and k[1:] != (w.rank, w.n_adapters)]:
+        del _CFG4_CACHE[k]                           # one adapter set at a time (the largest is 2.4 GB)
+    t = {"X": draw(("X",), 1, (w.n_rows, w.d_in), 1.0), "W": draw(("W",), 2, (w.d_in, w.d_out), w.d_in ** -0.5),
+         "A_all": draw(("A", w.rank, w.n_adapters), 3, (w.n_adapters, w.rank, w.d_in), 0.02),
+         "B_all": draw(("B", w.rank, w.n_adapters), 4, (w.n_adapters, w.rank, w.d_out), 0.02),
+         "scale": np.full(w.n_adapters, w.lora_scale, dtype=np.float32)}
+    n = w.ft_rows
+    t["dY"] = synth.round_to_storage(synth.normal(w.seed, w.tag_base + 5, n * w.d_out).reshape(n, w.d_out), w.dtype)
+    return t
+
+
+def test_cfg4_cached_tensors_are_the_generator_s(sess):
+    w = synth.cfg4_sweep_point(8, 1, 0.5)
+    a, b = _cfg4_tensors(w), synth.make_tensors(w)
+    assert all(np.array_equal(a[k], b[k]) for k in b)
+
+
+CFG4_GRID = [(r, n, f, True) for r in (8, 16, 32, 64, 128) for n in (1, 256) for f in (0.0, 0.5)] + [(16, 64, 0.25, False)]
+
+
+@pytest.mark.parametrize("rank,n_adapters,f,sorted_rows", CFG4_GRID)
+def test_cfg4_sweep_grid_full_size(sess, rank, n_adapters, f, sorted_rows):
+    """Every rank x {1, 256} adapters x fine-tune fraction {0, 0.5} of the sweep on 4096 -> 14336, plus one
+    point with unsorted rows (every row its own segment), each compared element by element."""
+    w = synth.cfg4_sweep_point(rank, n_adapters, f, sorted_rows=sorted_rows)
+    run_and_check(sess, w, _cfg4_tensors(w), blocked=True)
