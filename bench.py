@@ -8,8 +8,11 @@ projection set (q, k, v, o, gate, up, down; 32 adapters of rank 16; 4096 rows of
 decode rows and 2048 fine-tuning rows).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3|cfg2|cfg5] [--impl reference]
+                    [--no-extra-configs]
 
-Prints ONE JSON line.  With N > 1 (under torchrun) every rank runs the same workload on its own
+Prints ONE JSON line.  Beside the headline workload the line carries a `configs` block with the other
+seeded configurations (cfg2, the three cfg5 runs and their fill ratio, three cfg4 sweep points) and a
+`skinny_cold` block (the rank-r kernels on rotating inputs), measured after the headline.  With N > 1 (under torchrun) every rank runs the same workload on its own
 GPU (rows are independent, the path needs no collective): weak scaling, value = all ranks' tokens
 divided by the slowest rank's time.  `--impl reference` times the CPU oracle instead.
 """
@@ -57,61 +60,100 @@ from paper_2607_28848_b200.accounting import algorithmic_bytes, flops, load_peak
 # ---------------------------------------------------------------------------------------------
 # clocks
 # ---------------------------------------------------------------------------------------------
-class ClockSampler:
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+def _sampler_child(path: str, uuid: str, index: int, period_s: float = 0.004) -> None:
+    """Child process: reads SM clock, power and clock-event reasons through NVML every few milliseconds
+    (queries only; nothing is set) and appends `time sm_mhz power_w reasons_bitmask` lines to `path`."""
+    import pynvml
+    pynvml.nvmlInit()
+    h = None
+    if uuid:
+        for cand in (uuid, "GPU-" + uuid):
+            try:
+                h = pynvml.nvmlDeviceGetHandleByUUID(cand.encode() if hasattr(cand, "encode") else cand)
+                break
+            except Exception:
+                h = None
+    if h is None:
+        h = pynvml.nvmlDeviceGetHandleByIndex(index)
+    try:
+        mx = pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM)
+    except Exception:
+        mx = 0
+    reasons_fn = getattr(pynvml, "nvmlDeviceGetCurrentClocksEventReasons", None) or pynvml.nvmlDeviceGetCurrentClocksThrottleReasons
+    with open(path, "w", buffering=1) as fh:
+        fh.write(f"# max {mx}\n")
+        while True:
+            t = time.time()
+            try:
+                fh.write(f"{t:.6f} {pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)} "
+                         f"{pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0:.1f} {int(reasons_fn(h))}\n")
+            except Exception:
+                pass
+            dt = period_s - (time.time() - t)
+            if dt > 0:
+                time.sleep(dt)
 
-    def __init__(self, gpu_index: int):
-        self.path = tempfile.NamedTemporaryFile(prefix="clocks_", suffix=".csv", delete=False).name
-        self.proc = None
+
+class ClockSampler:
+    """SM clock, power and clock-event reasons DURING named regions, sampled every ~4 ms by a child
+    process through NVML (read-only queries), so that a 50 ms timed region still holds a dozen samples."""
+    # NVML clock-event reason bits
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown"}
+
+    def __init__(self, gpu_index: int, uuid: str = ""):
+        self.path = tempfile.NamedTemporaryFile(prefix="clocks_", suffix=".txt", delete=False).name
+        self.regions = {}
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(gpu_index), f"--query-gpu=timestamp,{self.Q}", "--format=csv,noheader,nounits",
-                 "-lms", "100", "-f", self.path], stdout=subprocess.DEVNULL, stderr=subprocess.DEVNULL)
+            self.proc = subprocess.Popen([sys.executable, os.path.abspath(__file__), "--clock-sampler", self.path,
+                                          "--sampler-uuid", uuid, "--sampler-index", str(gpu_index)],
+                                         stdout=subprocess.DEVNULL, stderr=subprocess.DEVNULL)
+            time.sleep(0.5)              # NVML is up before the first region starts
         except OSError:
             self.proc = None
-        self.t0 = self.t1 = None
 
-    def mark_start(self):
-        self.t0 = time.time()
+    def start(self, name: str):
+        self.regions[name] = [time.time(), None]
 
-    def mark_stop(self):
-        self.t1 = time.time()
+    def stop(self, name: str):
+        self.regions[name][1] = time.time()
 
     def finish(self) -> dict:
+        """Per region: median / min SM MHz, sample count, max power, reasons seen."""
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+            return {}
+        time.sleep(0.02)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        rows = []
+        rows, mx = [], None
         try:
-            import datetime
             with open(self.path) as fh:
                 for ln in fh:
-                    f = [x.strip() for x in ln.split(",")]
-                    if len(f) < 8:
+                    if ln.startswith("# max"):
+                        mx = float(ln.split()[2])
                         continue
-                    try:
-                        ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
-                        rows.append((ts, float(f[1]), float(f[2]), float(f[3]), f[4:8]))
-                    except ValueError:
-                        continue
+                    f = ln.split()
+                    if len(f) == 4:
+                        rows.append((float(f[0]), float(f[1]), float(f[2]), int(f[3])))
             os.unlink(self.path)
-        except OSError:
+        except (OSError, ValueError):
             pass
-        if not rows:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
-        inside = [r for r in rows if self.t0 is not None and self.t0 <= r[0] <= self.t1] or rows
-        sm = float(np.median([r[1] for r in inside]))
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = sorted({names[i] for r in inside for i in range(4) if r[4][i].lower().startswith("active")})
-        return {"sm_mhz": sm, "sm_max_mhz": rows[0][2], "reasons": reasons, "samples": len(inside),
-                "power_w_max": max(r[3] for r in inside)}
+        out = {}
+        for name, (t0, t1) in self.regions.items():
+            inside = [r for r in rows if t1 is not None and t0 <= r[0] <= t1]
+            if not inside:
+                out[name] = {"sm_mhz": None, "sm_max_mhz": mx, "reasons": ["no samples"], "samples": 0}
+                continue
+            bits = 0
+            for r in inside:
+                bits |= r[3]
+            out[name] = {"sm_mhz": float(np.median([r[1] for r in inside])), "sm_mhz_min": min(r[1] for r in inside),
+                         "sm_max_mhz": mx, "reasons": sorted(v for k, v in self.REASONS.items() if bits & k),
+                         "samples": len(inside), "power_w_max": max(r[2] for r in inside),
+                         "seconds": round(t1 - t0, 4)}
+        return out
 
 
 # ---------------------------------------------------------------------------------------------
@@ -135,47 +177,48 @@ def host_threads() -> int:
     return os.cpu_count() or 1
 
 
-def cpu_baseline(workloads, sample_names) -> dict:
-    """Times the oracle as it stands on a bounded sample and scales by algorithmic FLOPs."""
+def oracle_sample_text(workloads, secs) -> str:
     total = sum(flops(w)["fwd"] + flops(w)["bwd"] for w in workloads)
-    sample = [w for w in workloads if w.name.split("_", 1)[1] in sample_names] or workloads[:1]
-    sflops, secs = 0.0, 0.0
-    for w in sample:
-        t = synth.make_tensors(w)
-        t0 = time.perf_counter()
+    return (f"fp64 numpy oracle (forward_blocked + backward_blocked), one pass over every projection of the workload "
+            f"{[w.name for w in workloads]} = {total / 1e9:.0f} GFLOP, the whole step, nothing scaled: {secs:.1f} s")
+
+
+def oracle_step_seconds(workloads, tensors) -> float:
+    t0 = time.perf_counter()
+    for w, t in zip(workloads, tensors):
         oracle_pass(w, t)
-        secs += time.perf_counter() - t0
-        sflops += flops(w)["fwd"] + flops(w)["bwd"]
-    est = secs * total / sflops
-    return {"value": workloads[0].n_rows / est, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
-            "sample": f"fp64 numpy oracle, forward+backward of projection(s) {[w.name for w in sample]} "
-                      f"({sflops / 1e9:.0f} of {total / 1e9:.0f} GFLOP) in {secs:.1f} s, scaled to the whole step by FLOPs"}
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(workloads) -> dict:
+    """The oracle as it stands, timed once on the whole step (every projection of the workload): the same
+    sample the reference arm times per step."""
+    tensors = [synth.make_tensors(w) for w in workloads]
+    secs = oracle_step_seconds(workloads, tensors)
+    return {"value": workloads[0].n_rows / secs, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+            "sample": oracle_sample_text(workloads, secs)}
 
 
 def run_reference(args, workloads, label):
-    """The reference arm: the CPU oracle timed on the host cores, one bounded sample per step."""
+    """The reference arm: the CPU oracle timed on the host cores; a step is one pass over every projection of
+    the workload (the same sample as the GPU arm's cpu_baseline leg), so nothing is extrapolated."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    total = sum(flops(w)["fwd"] + flops(w)["bwd"] for w in workloads)
-    w = min(workloads, key=lambda x: flops(x)["fwd"] + flops(x)["bwd"])
-    t = synth.make_tensors(w)
+    tensors = [synth.make_tensors(w) for w in workloads]
     for _ in range(args.warmup):
-        oracle_pass(w, t)
+        oracle_step_seconds(workloads, tensors)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle_pass(w, t)
+        oracle_step_seconds(workloads, tensors)
     secs = (time.perf_counter() - t0) / max(args.steps, 1)
-    sf = flops(w)["fwd"] + flops(w)["bwd"]
-    est = secs * total / sf
-    value = workloads[0].n_rows / est
-    sample = (f"each step = fp64 numpy oracle forward+backward of {w.name} ({sf / 1e9:.0f} of {total / 1e9:.0f} GFLOP "
-              f"per full step), scaled to the whole step by FLOPs")
+    value = workloads[0].n_rows / secs
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": label},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": host_threads(), "kind": "oracle", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+                             "sample": oracle_sample_text(workloads, secs)},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
@@ -198,10 +241,18 @@ def main():
                     help="also run the AdamW update of the fine-tuned adapters after each backward (not part of the "
                          "headline step; reported under kernels.adamw)")
     ap.add_argument("--graph", action="store_true", help="also time the step replayed from a CUDA graph (step_stats)")
+    ap.add_argument("--no-extra-configs", action="store_true",
+                    help="skip the `configs` and `skinny_cold` blocks (the other seeded configurations measured after the headline)")
+    ap.add_argument("--clock-sampler", default="", help=argparse.SUPPRESS)       # child-process mode of ClockSampler
+    ap.add_argument("--sampler-uuid", default="", help=argparse.SUPPRESS)
+    ap.add_argument("--sampler-index", type=int, default=0, help=argparse.SUPPRESS)
     ap.add_argument("--dropout", type=float, default=0.0,
                     help="LoRA dropout rate on the fine-tuning rows (the paper trains with 0.05; the headline step "
                          "runs without it); a new seed every step")
     args = ap.parse_args()
+    if args.clock_sampler:
+        _sampler_child(args.clock_sampler, args.sampler_uuid, args.sampler_index)
+        return
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -274,11 +325,17 @@ def main():
     step()
     launches_per_step = mb.mlora_launch_count(sess.ctx) - launches_per_step_probe
 
-    sampler = ClockSampler(local_rank) if rank == 0 else None
+    sampler = None
+    if rank == 0:
+        try:
+            uuid = str(torch.cuda.get_device_properties(local_rank).uuid)
+        except Exception:
+            uuid = ""
+        sampler = ClockSampler(local_rank, uuid)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     if sampler:
-        sampler.mark_start()
+        sampler.start("timed")
     l0 = mb.mlora_launch_count(sess.ctx)
     ev0.record()
     for _ in range(args.steps):
@@ -286,18 +343,22 @@ def main():
     ev1.record()
     barrier()
     if sampler:
-        sampler.mark_stop()
+        sampler.stop("timed")
     gpu_launches = mb.mlora_launch_count(sess.ctx) - l0
     ms_total = replicas.max_over_ranks(ev0.elapsed_time(ev1), sess.device)     # slowest rank
     # Spread of single steps (median and best of up to 50 more steps, one event between steps):
     # reported beside the headline mean, never instead of it.
     stat_n = max(1, min(args.steps, 50))
     marks = [torch.cuda.Event(enable_timing=True) for _ in range(stat_n + 1)]
+    if sampler:
+        sampler.start("single_steps")
     marks[0].record()
     for i in range(stat_n):
         step()
         marks[i + 1].record()
     torch.cuda.synchronize()
+    if sampler:
+        sampler.stop("single_steps")
     step_ms = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(stat_n))
     # The same step captured once in a CUDA graph and replayed (the calls allocate nothing and never
     # synchronise, so forward + activation save + backward capture as they are); reported beside the
@@ -351,10 +412,13 @@ def main():
     # that the headline number carries no event overhead.
     prof_steps = max(1, min(args.steps, 20))
     mb.mlora_profile_enable(sess.ctx, launches_per_step * prof_steps)
+    if sampler:
+        sampler.start("per_kernel")
     for _ in range(prof_steps):
         step()
     barrier()
-    clocks = sampler.finish() if sampler else None
+    if sampler:
+        sampler.stop("per_kernel")
     kinds, kms = mb.mlora_profile_collect(sess.ctx)
     mb.mlora_profile_enable(sess.ctx, 0)
 
@@ -416,11 +480,10 @@ def main():
     if "gemm_fwd" in kernels:
         n_launch = per_kind["gemm_fwd"]["launches_per_step"]
         achieved = kernels["gemm_fwd"]["tflops"]
-        peak = peaks["bf16_tflops_sustained"]
         roofline = {"kernel": "gemm2_lora_kernel<R, false> (forward: base GEMM + LoRA expand, two-SM tcgen05)", "bound": "tensor",
-                    "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                    "peak_source": f"{peaks['source']} sustained bf16 ({peak}); burst {peaks['bf16_tflops']}",
+                    "achieved": achieved, "unit": "TFLOP/s",
                     "frac_of_burst": achieved / peaks["bf16_tflops"],
+                    "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
                     "flops_per_launch": gemm_fwd_flops / n_launch,
                     "avg_launch_ms": per_kind["gemm_fwd"]["ms_per_step"] / n_launch,
                     "traffic": None}
@@ -428,10 +491,12 @@ def main():
         if os.path.exists(prof):
             try:
                 with open(prof) as fh:
-                    roofline["traffic"] = json.load(fh).get(args.workload, {}).get("gemm_fwd_bytes_per_launch")
+                    rec = json.load(fh).get(args.workload, {})
+                roofline["traffic"] = rec.get("gemm_fwd_bytes_per_launch")
+                roofline["traffic_source"] = ("ncu capture of this kernel recorded in profiles/traffic.json (not measured in this run): "
+                                              + str(rec.get("source", "")) + ", build " + str(rec.get("build", "unrecorded")))
             except Exception:
                 pass
-
     # ---- end to end through the public API with host buffers ----
     e2e = None
     if args.e2e_steps > 0 and (rank == 0 or world > 1):
@@ -492,11 +557,43 @@ def main():
         e2e = {"value": world * T * args.e2e_steps / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.e2e_steps, "steps": args.e2e_steps}
 
+    # ---- the other seeded configurations and the skinny kernels cold (rank 0, one GPU) ----
+    configs_block, cold_block = None, None
+    if rank == 0 and world == 1 and not args.no_extra_configs and not args.projections:
+        for r in runs:
+            r.close()
+        del runs[:]
+        torch.cuda.empty_cache()
+        configs_block, cold_block = extra_configs(sess, peaks, args.workload)
+
+    clock_regions = sampler.finish() if sampler else {}
+    clocks = clock_regions.get("timed")
     status = mb.mlora_poll_status(sess.ctx)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
+
+    if roofline is not None:
+        # Which measured peak the kernel is held against follows from the clocks of the pass in which its launches
+        # were timed (the per-kernel pass): at (nearly) the full boost clock the comparator is the burst figure, a
+        # pass that ran clocked down under the power cap is held against the sustained one.  Both fractions are printed.
+        ck = clock_regions.get("per_kernel") or {}
+        mhz, mx = ck.get("sm_mhz"), ck.get("sm_max_mhz")
+        capped = bool(mhz and mx and mhz < 0.9 * mx and "sw_power_cap" in ck.get("reasons", []))
+        roofline["peak"] = peaks["bf16_tflops_sustained"] if capped else peaks["bf16_tflops"]
+        roofline["frac"] = roofline["achieved"] / roofline["peak"]
+        roofline["peak_source"] = (f"{peaks['source']} {'sustained' if capped else 'burst'} bf16 peak: the per-kernel pass ran at a median "
+                                   f"{mhz} MHz of {mx} ({ck.get('seconds')} s, {ck.get('samples')} clock samples, reasons {ck.get('reasons')})")
+    step_stats["clocks"] = clock_regions.get("single_steps")
+    if clocks and clocks.get("sm_mhz"):
+        step_stats["ms_per_step_x_sm_mhz"] = ms_per_step * clocks["sm_mhz"]
+        ss = step_stats["clocks"] or {}
+        if ss.get("sm_mhz"):
+            step_stats["median_ms_x_sm_mhz"] = step_stats["median_ms"] * ss["sm_mhz"]
+        step_stats["note"] = ("the timed region comes first and is short; the single steps behind median_ms / best_ms run after it, "
+                              "when the board's power controller may have lowered the SM clock (see both clock records: time x MHz "
+                              "compares runs at different clocks)")
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
@@ -514,12 +611,55 @@ def main():
         "step_stats": step_stats,
         "roofline": roofline, "kernels": kernels,
     }
+    if configs_block is not None:
+        line["configs"] = configs_block
+        line["skinny_cold"] = cold_block
     if not args.no_cpu_baseline and world == 1:
-        names = {"cfg3": ["q", "k", "v", "o", "gate", "up", "down"], "cfg2": ["proj4096"], "cfg5": ["mixed"]}[args.workload]
-        line["cpu_baseline"] = cpu_baseline(workloads, names)
+        line["cpu_baseline"] = cpu_baseline(workloads)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def extra_configs(sess, peaks, headline: str):
+    """cfg2, the three cfg5 runs (+ fill ratio) and three cfg4 sweep points: forward + LoRA backward per
+    repetition with an L2 flush between repetitions (their inputs are smaller than the L2), median and best
+    of 30; then the rank-r kernels cold on their largest instances (rotating copies of the inputs)."""
+    import bench_tables as bt
+
+    def entry(w, reps=30):
+        med, best = bt.step_time(sess, w, reps)
+        fl = flops(w)
+        tot = fl["fwd"] + (fl["bwd"] if w.ft_rows else 0.0)
+        ab = algorithmic_bytes(w)
+        nbytes = ab["gemm_fwd"] + (ab["gemm_bwd"] if w.ft_rows else 0.0)
+        t_roof_us = max(tot / (peaks["bf16_tflops"] * 1e12), nbytes / (peaks["hbm_gbs"] * 1e9)) * 1e6
+        return {"workload": w.name, "rows": w.n_rows, "ft_rows": w.ft_rows, "median_us": med, "best_us": best,
+                "tokens_per_s": w.n_rows / (med * 1e-6), "tflops": tot / (med * 1e-6) / 1e12,
+                "t_roof_us": t_roof_us, "frac_of_roofline": t_roof_us / med,
+                "roofline_bound": "tensor" if tot / (peaks["bf16_tflops"] * 1e12) >= nbytes / (peaks["hbm_gbs"] * 1e9) else "hbm"}
+
+    out = {"protocol": "forward + LoRA backward per repetition, 256 MB L2 flush between repetitions, CUDA events per repetition, "
+                       "median of 30 (best beside it); roofline = slower of FLOPs at the measured burst bf16 peak and each "
+                       "tensor once at the measured copy bandwidth"}
+    if headline != "cfg2":
+        out["cfg2"] = entry(synth.cfg2_single_projection(0))
+    if headline != "cfg5":
+        c5 = {m: entry(synth.cfg5_decode_heavy(0, m)) for m in ("decode", "finetune", "mixed")}
+        c5["fill_ratio_mixed_over_decode_plus_finetune"] = c5["mixed"]["median_us"] / (c5["decode"]["median_us"] + c5["finetune"]["median_us"])
+        out["cfg5"] = c5
+    out["cfg4"] = [entry(synth.cfg4_sweep_point(r, n, f), reps=20) for r, n, f in ((16, 8, 0.5), (64, 64, 0.25), (128, 256, 0.5))]
+    cold = {"protocol": "every repetition on another copy of X, dY and the activation buffers (6 copies), one CUDA event pair per launch, "
+                        "40 repetitions; bytes = every operand once; fraction of the measured copy bandwidth (median / best)"}
+    rows = []
+    for w in synth.cfg3_layer_set(0, projections=["gate", "down"]) + [synth.cfg5_decode_heavy(0)]:
+        times, nbytes, _rot = bt.cold_skinny(sess, w, 40, 6)
+        for k, ts in times.items():
+            med, best = float(np.median(ts)), float(np.min(ts))
+            rows.append({"launch": f"{w.name}:{k}", "mbytes": nbytes[k] / 1e6, "median_us": med, "best_us": best,
+                         "frac_hbm_median": nbytes[k] / med / 1e3 / peaks["hbm_gbs"], "frac_hbm_best": nbytes[k] / best / 1e3 / peaks["hbm_gbs"]})
+    cold["launches"] = rows
+    return out, cold
 
 
 if __name__ == "__main__":
