@@ -288,11 +288,14 @@ mlora_status_t mlora_profile_enable(mlora_ctx* ctx, int32_t max_records);
 int32_t mlora_profile_collect(mlora_ctx* ctx, int32_t* kinds, float* ms, int32_t cap);
 
 /* Selects kernel variants for MLORA_BF16 layers: 0 = defaults (two-SM tcgen05 tensor-core GEMM,
- * streaming shrink and gradient kernels for rank <= 64); 1 = the plain CUDA-core kernels for every step (a slow
+ * streaming shrink and gradient kernels for rank <= 64, tcgen05 gradient kernel for rank 128); 1 = the plain CUDA-core kernels for every step (a slow
  * cross-check used by the tests); 2 = defaults, but the per-item shrink kernel for every rank
  * (the variant rank 128 always uses); 3 = defaults, but the one-SM tensor-core GEMM;
  * 4 = defaults, but the two-SM GEMM never splits K (by default a product with too few output
- * tiles for the SMs is cut into K slices whose fp32 partials a small kernel adds up). */
+ * tiles for the SMs is cut into K slices whose fp32 partials a small kernel adds up);
+ * 5 = defaults, but both gradients on the mma.sync kernels for every rank (by default rank 128 uses the
+ * tcgen05 gradient kernel); 6 = defaults, but both gradients on the tcgen05 gradient kernel for every
+ * rank (with dropout on, the mma.sync kernels always run). */
 mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path);
 
 /* ---- forward without any allocation -----------------------------------------------------*/

@@ -19,6 +19,7 @@
 #include "gemm2_tcgen05.cuh"
 #include "simt.cuh"
 #include "skinny.cuh"
+#include "grad_tc.cuh"
 #include "glue.cuh"
 #include "attention.cuh"
 #include "attention_tc.cuh"
@@ -58,8 +59,10 @@ struct mlora_ctx {
   __nv_bfloat16* ws_pbd = nullptr;   // block-diagonal low-rank operand: [2 * ws_pbd_groups * 256, 64] bf16
   int64_t ws_pbd_groups = 0;
   float* ws_splitk = nullptr;        // fp32 partial products of a K-split GEMM (fixed size, see kSplitKBytes)
-  float* ws_gpart = nullptr;         // row-split gradient groups: [sm_count][64][512] fp32 partial sums
+  float* ws_gpart = nullptr;         // partial gradient sums that several CTAs share: [sm_count][4][64 KiB] (the streaming kernel's
+                                     // row-split groups use the first 128 KiB per SM, the tensor-core kernel's split strips all of it)
   int32_t* ws_gcounters = nullptr;   // [sm_count] arrival counters of those groups, zero between launches
+  int32_t* ws_tc_counters = nullptr; // [kTcCounters] counters of the tensor-core gradient kernel, zero between launches
   std::vector<void*> retired;        // workspaces replaced by larger ones: kept until the context is destroyed,
                                      // because a captured graph may still hold their addresses
   std::vector<PlanBuf> plan_pool;    // released buffers of stream-ordered plans
@@ -68,6 +71,8 @@ struct mlora_ctx {
   int32_t shrink_path = 0;           // 0: streaming shrink for rank <= 64 (gradients: <= 32); 1: per-item kernels for every rank
   int32_t gemm_pairs = 1;            // 1: two-SM (CTA pair) tensor-core kernel; 0: one-SM kernel
   int32_t no_split_k = 0;            // 1: the two-SM kernel never splits K (kernel variant 4)
+  int32_t grad_mode = 0;             // 0: default choice by rank; 1: mma.sync kernels for every rank (kernel variant 5);
+                                     // 2: the tcgen05 gradient kernel for every rank (kernel variant 6)
   EncodeTiledFn encode = nullptr;
   const volatile int32_t* cancel = nullptr;   // caller's host flag, read before every launch
   DropArgs drop = {0, 0, 1.0f};               // LoRA dropout of the fine-tuning rows (thr == 0: off)
@@ -78,6 +83,10 @@ struct mlora_ctx {
 };
 
 constexpr int kMaxKSplit = 16;
+// Ranks from which the tcgen05 gradient kernel is the default.  Measured on B200 (one launch, 4096 -> 14336, 1024-2048
+// fine-tuning rows): rank 8 20.9 vs 14.7 us for the mma.sync streaming kernel, rank 16 27.0 vs 20.8, rank 32 39.3 vs 39.3,
+// rank 64 43.4 vs 33.1, rank 128 70 vs 144 (two launches of the per-item kernel).
+constexpr int kTcGradMinRank = 128;
 
 enum { KIND_SHRINK = 0, KIND_GEMM_FWD = 1, KIND_GEMM_BWD = 2, KIND_GRAD = 3, KIND_SIMT = 4, KIND_ADAMW = 5, KIND_REDUCE = 6 };
 
@@ -132,6 +141,7 @@ struct BlobBuilder {
 // Workspace for K-split products of small-batch GEMMs: allocated once per context, so that no
 // compute call allocates.  Problems whose partials do not fit run unsplit.
 constexpr size_t kSplitKBytes = 64u << 20;
+constexpr int kTcCounters = 1 << 18;    // counter words of the tensor-core gradient kernel (1 MiB, allocated with the context)
 constexpr int kMaxDevices = 64;      // device ordinals a process may create contexts on
 // One-time kernel attributes (opt-in shared-memory size, resident cluster count) are cached per kernel
 // instantiation and device in function-local arrays; contexts are independent across host threads, so
@@ -423,6 +433,80 @@ mlora_status_t launch_grad_stream2(mlora_ctx* ctx, const mlora_plan* p, const Gr
     if (ctx->drop.thr != 0) return launch_grad_stream2_c<MB, true>(ctx, p, gb, ga_, n_slots, n_rows, st);
   }
   return launch_grad_stream2_c<MB, false>(ctx, p, gb, ga_, n_slots, n_rows, st);
+}
+
+// Both gradients on the tcgen05 kernel: can this call use it?  (A slot without rows gets its zeros from the
+// other kernels; the counters have a fixed size.)
+template <int R>
+bool grad_tc_fits(const mlora_layer_t* L, const mlora_plan* p) {
+  using C = gtc::Cfg<R>;
+  const HostPlan& h = p->h;
+  const int n_slots = (int)h.ft_adapters.size();
+  if (n_slots < 1) return false;
+  for (int sl = 0; sl < n_slots; ++sl)
+    if (h.slot_blk_off[sl + 1] == h.slot_blk_off[sl]) return false;
+  const int64_t NB = (int64_t)h.blk_row0.size();
+  const int64_t NS0 = (L->d_out + C::COLS - 1) / C::COLS, NS1 = (L->d_in + C::COLS - 1) / C::COLS;
+  if (1 + n_slots * (NS0 + NS1) > kTcCounters) return false;
+  return NB * (NS0 + NS1) < (1 << 30);
+}
+
+// First tile of CTA c's range in the combined list, with the ends moved down to strip boundaries (what the
+// kernel does when `snap` is set): used to decide whether snapping keeps the ranges even.
+int64_t grad_tc_snapped_begin(const HostPlan& h, int64_t NS0, int64_t NS1, int c, int G) {
+  const int64_t NB = (int64_t)h.blk_row0.size(), N0 = NB * NS0, N = NB * (NS0 + NS1);
+  int64_t g = (int64_t)c * N / G;
+  if (g >= N) return N;
+  const int64_t NS = g >= N0 ? NS1 : NS0, t = g >= N0 ? g - N0 : g;
+  size_t slot = 0;
+  while ((int64_t)h.slot_blk_off[slot + 1] * NS <= t) ++slot;
+  const int64_t nb = h.slot_blk_off[slot + 1] - h.slot_blk_off[slot];
+  return g - (t - (int64_t)h.slot_blk_off[slot] * NS) % nb;
+}
+
+template <int R>
+mlora_status_t launch_grad_tc(mlora_ctx* ctx, const mlora_layer_t* L, const mlora_plan* p, const void* dY, int64_t lddy,
+                              const void* x_save, const float* u_save, float* dA, float* dB, int accumulate, cudaStream_t st) {
+  using C = gtc::Cfg<R>;
+  const HostPlan& h = p->h;
+  static bool attr_set_dev[kMaxDevices] = {};   // per instantiation and device
+  bool& attr_set = attr_set_dev[ctx->device];
+  auto kern = gtc::grad_tc_kernel<R>;
+  {
+    std::lock_guard<std::mutex> lock(g_attr_mutex);
+    if (!attr_set) {
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES) != cudaSuccess) return MLORA_ERR_CUDA;
+      attr_set = true;
+    }
+  }
+  CUtensorMap tQ0, tQ1;
+  mlora_status_t ms;
+  // (64, rows, D / 64) views: one box = a 128-row tile as CB swizzled 64-column blocks
+  if ((ms = make_tmap_bf16_blocked(ctx, &tQ0, dY, h.ft_rows, L->d_out, lddy, gtc::ROWS, C::CB)) != MLORA_OK) return ms;
+  if ((ms = make_tmap_bf16_blocked(ctx, &tQ1, x_save, h.ft_rows, L->d_in, L->d_in, gtc::ROWS, C::CB)) != MLORA_OK) return ms;
+  gtc::Args a;
+  const int NS0 = (L->d_out + C::COLS - 1) / C::COLS, NS1 = (L->d_in + C::COLS - 1) / C::COLS;
+  a.prob[0] = gtc::Problem{u_save, L->scale, dB, L->d_out, NS0};       // dB = (s u)^T dY
+  a.prob[1] = gtc::Problem{ctx->ws_p, nullptr, dA, L->d_in, NS1};      // dA = V^T x, V already carries s
+  a.slot_adapter = p->slot_adapter; a.slot_blk_off = p->slot_blk_off; a.blk_row0 = p->blk_row0; a.blk_nrows = p->blk_nrows;
+  a.n_slots = (int)h.ft_adapters.size(); a.NB = (int)h.blk_row0.size();
+  a.part_ws = ctx->ws_gpart; a.counters = ctx->ws_tc_counters; a.n_counters = 1 + a.n_slots * (NS0 + NS1);
+  a.accumulate = accumulate; a.status = ctx->status_dev;
+  const int64_t tiles = (int64_t)a.NB * (NS0 + NS1);
+  const int grid = tiles < ctx->sm_count ? (int)tiles : ctx->sm_count;
+  // Ranges that end at strip boundaries need no partial sums; taken when they stay nearly as even as plain ranges.
+  int64_t most_plain = 0, most_snapped = 0;
+  for (int c = 0; c < grid; ++c) {
+    const int64_t plain = (int64_t)(c + 1) * tiles / grid - (int64_t)c * tiles / grid;
+    const int64_t snapped = grad_tc_snapped_begin(h, NS0, NS1, c + 1, grid) - grad_tc_snapped_begin(h, NS0, NS1, c, grid);
+    most_plain = plain > most_plain ? plain : most_plain;
+    most_snapped = snapped > most_snapped ? snapped : most_snapped;
+  }
+  a.snap = (8 * most_snapped <= 9 * most_plain) ? 1 : 0;
+  if (cancelled(ctx)) return MLORA_CANCELLED;
+  LaunchScope scope(ctx, st, KIND_GRAD);
+  launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(gtc::THREADS), C::SMEM_BYTES, st, tQ0, tQ1, a);
+  return scope.done();
 }
 
 mlora_status_t launch_grad(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& a, int n_slots, int n_rows,
@@ -818,9 +902,11 @@ mlora_status_t mlora_create(mlora_ctx** out, int device) {
   c->encode = reinterpret_cast<EncodeTiledFn>(fn);
   if (cudaMalloc(&c->status_dev, sizeof(int32_t)) != cudaSuccess ||
       cudaMalloc(&c->ws_splitk, kSplitKBytes) != cudaSuccess ||
-      cudaMalloc(&c->ws_gpart, (size_t)c->sm_count * 64 * 512 * sizeof(float)) != cudaSuccess ||
+      cudaMalloc(&c->ws_gpart, (size_t)c->sm_count * 4 * 65536) != cudaSuccess ||
       cudaMalloc(&c->ws_gcounters, (size_t)c->sm_count * sizeof(int32_t)) != cudaSuccess ||
       cudaMemset(c->ws_gcounters, 0, (size_t)c->sm_count * sizeof(int32_t)) != cudaSuccess ||
+      cudaMalloc(&c->ws_tc_counters, (size_t)kTcCounters * sizeof(int32_t)) != cudaSuccess ||
+      cudaMemset(c->ws_tc_counters, 0, (size_t)kTcCounters * sizeof(int32_t)) != cudaSuccess ||
       cudaMemset(c->status_dev, 0, sizeof(int32_t)) != cudaSuccess) {
     cudaGetLastError();
     mlora_destroy(c);       // frees whatever was allocated
@@ -873,6 +959,7 @@ void mlora_destroy(mlora_ctx* c) {
   cudaFree(c->ws_splitk);
   cudaFree(c->ws_gpart);
   cudaFree(c->ws_gcounters);
+  cudaFree(c->ws_tc_counters);
   for (void* r : c->retired) cudaFree(r);
   for (PlanBuf& b : c->plan_pool) free_plan_buf(b);
   delete c;
@@ -1151,6 +1238,29 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   ga.slot_adapter = p->slot_adapter; ga.accumulate = accumulate;
   GradArgs gA = ga;                  // dA = V^T X
   gA.P = ctx->ws_p; gA.scale = nullptr; gA.Q = (const __nv_bfloat16*)x_save; gA.ldq = L->d_in; gA.D = L->d_in; gA.G = dA;
+  // both gradients on the tensor-core kernel where it is the faster one (V is in the workspace by now)
+  bool tc_grad = false;
+  if (ctx->grad_mode != 1 && ctx->shrink_path == 0 && !dropping && (ctx->grad_mode == 2 || L->rank >= kTcGradMinRank)) {
+    switch (L->rank) {
+      case 8: tc_grad = grad_tc_fits<8>(L, p); break;
+      case 16: tc_grad = grad_tc_fits<16>(L, p); break;
+      case 32: tc_grad = grad_tc_fits<32>(L, p); break;
+      case 64: tc_grad = grad_tc_fits<64>(L, p); break;
+      case 128: tc_grad = grad_tc_fits<128>(L, p); break;
+    }
+  }
+  if (tc_grad) {
+    switch (L->rank) {
+      case 8: s = launch_grad_tc<8>(ctx, L, p, dY, lddy, x_save, u_save, dA, dB, accumulate, st); break;
+      case 16: s = launch_grad_tc<16>(ctx, L, p, dY, lddy, x_save, u_save, dA, dB, accumulate, st); break;
+      case 32: s = launch_grad_tc<32>(ctx, L, p, dY, lddy, x_save, u_save, dA, dB, accumulate, st); break;
+      case 64: s = launch_grad_tc<64>(ctx, L, p, dY, lddy, x_save, u_save, dA, dB, accumulate, st); break;
+      default: s = launch_grad_tc<128>(ctx, L, p, dY, lddy, x_save, u_save, dA, dB, accumulate, st); break;
+    }
+    if (s != MLORA_OK || !dX) return s;
+    return gemm_bf16<true>(ctx, L, h.bwd, p->bwd, dY, lddy, dX, lddx, L->A_all, ctx->ws_p, nullptr, h.ft_rows, L->d_in,
+                           L->d_out, st);
+  }
   if (ctx->shrink_path == 0 && L->rank <= 64) {      // both gradients in one launch of the streaming kernel
     s = L->rank <= 16 ? launch_grad_stream2<1>(ctx, p, ga, gA, n_slots, h.ft_rows, st)
         : L->rank <= 32 ? launch_grad_stream2<2>(ctx, p, ga, gA, n_slots, h.ft_rows, st)
@@ -1220,6 +1330,7 @@ mlora_status_t mlora_poll_status(mlora_ctx* ctx, void* cuda_stream) {
     cudaMemsetAsync(ctx->status_dev, 0, sizeof(v), st);
     if (ctx->ws_counters) cudaMemsetAsync(ctx->ws_counters, 0, (size_t)(2 * ctx->ws_counter_items + 1) * sizeof(int32_t), st);
     cudaMemsetAsync(ctx->ws_gcounters, 0, (size_t)ctx->sm_count * sizeof(int32_t), st);
+    cudaMemsetAsync(ctx->ws_tc_counters, 0, (size_t)kTcCounters * sizeof(int32_t), st);
     cudaStreamSynchronize(st);
   }
   return (mlora_status_t)v;
@@ -1251,11 +1362,12 @@ mlora_status_t mlora_set_dropout(mlora_ctx* ctx, double p, uint64_t seed) {
 int64_t mlora_launch_count(const mlora_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path) {
-  if (!ctx || path < 0 || path > 4) return MLORA_ERR_INVALID_ARG;
+  if (!ctx || path < 0 || path > 6) return MLORA_ERR_INVALID_ARG;
   ctx->gemm_path = path == 1 ? 1 : 0;
   ctx->shrink_path = path == 2 ? 1 : 0;
   ctx->gemm_pairs = path == 3 ? 0 : 1;
   ctx->no_split_k = path == 4 ? 1 : 0;
+  ctx->grad_mode = path == 5 ? 1 : (path == 6 ? 2 : 0);
   return MLORA_OK;
 }
 

@@ -77,7 +77,7 @@ def test_cfg1_tiny_fp32(sess):
     run_and_check(sess, w, synth.make_tensors(w))
 
 
-@pytest.mark.parametrize("path", [0, 1, 2, 3, 4])
+@pytest.mark.parametrize("path", [0, 1, 2, 3, 4, 5, 6])
 def test_bf16_ragged_multi_tile(sess, path):
     w = synth.random_workload(5, 256, 512, 16, 6, 389, max_seg=150)
     run_and_check(sess, w, synth.make_tensors(w), path=path)
@@ -152,6 +152,54 @@ def test_random_shapes_tables_and_kernel_variants(sess, seed):
         cap = None if rng.random() < 0.5 else int(w.ft_rows + 30)
         run_and_check(sess, w, synth.make_tensors(w), path=int(rng.choice([0, 0, 0, 2, 3, 4])), blocked=True,
                       base=int(rng.integers(0, 3)) * 7, cap=cap)
+
+
+@pytest.mark.parametrize("path", [5, 6])
+@pytest.mark.parametrize("rank", [8, 16, 32, 64, 128])
+def test_gradient_kernel_variants_rank_sweep(sess, rank, path):
+    """Both gradient kernels on every rank: variant 5 = the mma.sync kernels (per-item kernel at rank 128), variant 6 =
+    the tcgen05 gradient kernel (the default only at rank 128)."""
+    w = synth.random_workload(60 + rank, 320, 448, rank, 7, 420, max_seg=150, p_finetune=0.5)
+    run_and_check(sess, w, synth.make_tensors(w), path=path)
+
+
+@pytest.mark.parametrize("lens", [(1100, 40), (2048,), (256,), (70, 700, 3)])
+def test_tensor_core_gradient_kernel_on_split_strips(sess, lens):
+    """The tcgen05 gradient kernel (kernel variant 6) where a slot's strips are shared by several CTAs: pieces summed by the
+    last arrival in CTA order, slots of very different sizes, short last blocks, overwrite and accumulate, and the
+    same bits from run to run."""
+    segs, row = [(0, 37, 3, 0)], 37
+    for a, n in enumerate(lens):
+        segs.append((row, n, a, 1))
+        row += n
+    segs.append((row, 20, 0, 0))
+    row += 20
+    w = synth.Workload("few_slots_tc", 512, 1024, 16, 4, "bf16", row, synth.segments_array(segs), seed=400 + len(lens))
+    t = synth.make_tensors(w)
+    run_and_check(sess, w, t, blocked=True, path=6)
+    mb.mlora_set_gemm_path(sess.ctx, 6)
+    try:
+        run = LayerRun(sess, "bf16", t, w.segments, w.n_rows)
+        run.forward()
+        outs = []
+        for _ in range(3):
+            run.backward(accumulate=False)
+            outs.append((run.dA.clone(), run.dB.clone()))
+        for dA, dB in outs[1:]:
+            assert torch.equal(dA, outs[0][0]) and torch.equal(dB, outs[0][1])
+        run.backward(accumulate=True, want_dx=False)
+        assert_close("dA x2", run.host(run.dA), 2 * run.host(outs[0][0]), 1e-5)
+        assert_close("dB x2", run.host(run.dB), 2 * run.host(outs[0][1]), 1e-5)
+        assert run.status() == mb.MLORA_OK
+        run.close()
+    finally:
+        mb.mlora_set_gemm_path(sess.ctx, 0)
+
+
+def test_tensor_core_gradient_kernel_full_size(sess):
+    """Kernel variant 6 on the widest projection of the layer set (plain ranges with shared strips at this size)."""
+    w = synth.cfg3_layer_set(projections=["gate"])[0]
+    run_and_check(sess, w, synth.make_tensors(w), blocked=True, path=6)
 
 
 @pytest.mark.parametrize("rank", [8, 128])
