@@ -294,8 +294,8 @@ int32_t mlora_profile_collect(mlora_ctx* ctx, int32_t* kinds, float* ms, int32_t
  * 4 = defaults, but the two-SM GEMM never splits K (by default a product with too few output
  * tiles for the SMs is cut into K slices whose fp32 partials a small kernel adds up);
  * 5 = defaults, but both gradients on the mma.sync kernels for every rank (by default rank 128 uses the
- * tcgen05 gradient kernel); 6 = defaults, but both gradients on the tcgen05 gradient kernel for every
- * rank (with dropout on, the mma.sync kernels always run). */
+ * tcgen05 gradient kernel); 6 = defaults, but the whole rank-r part of the backward on tcgen05 kernels for every
+ * rank: V = s dY B^T and both gradients (with dropout on, the gradients stay on the mma.sync kernels). */
 mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path);
 
 /* ---- forward without any allocation -----------------------------------------------------*/

@@ -20,6 +20,7 @@
 #include "simt.cuh"
 #include "skinny.cuh"
 #include "grad_tc.cuh"
+#include "vshrink_tc.cuh"
 #include "glue.cuh"
 #include "attention.cuh"
 #include "attention_tc.cuh"
@@ -433,6 +434,40 @@ mlora_status_t launch_grad_stream2(mlora_ctx* ctx, const mlora_plan* p, const Gr
     if (ctx->drop.thr != 0) return launch_grad_stream2_c<MB, true>(ctx, p, gb, ga_, n_slots, n_rows, st);
   }
   return launch_grad_stream2_c<MB, false>(ctx, p, gb, ga_, n_slots, n_rows, st);
+}
+
+// V = s dY B^T on the tcgen05 kernel (the fine-tuning rows come as 128-row blocks of one adapter each).
+template <int R>
+mlora_status_t launch_vshrink_tc(mlora_ctx* ctx, const mlora_layer_t* L, const mlora_plan* p, const void* dY, int64_t lddy,
+                                 bool want_pbd, cudaStream_t st) {
+  using C = vtc::Cfg<R>;
+  const HostPlan& h = p->h;
+  static bool attr_set_dev[kMaxDevices] = {};   // per instantiation and device
+  bool& attr_set = attr_set_dev[ctx->device];
+  auto kern = vtc::vshrink_tc_kernel<R>;
+  {
+    std::lock_guard<std::mutex> lock(g_attr_mutex);
+    if (!attr_set) {
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES) != cudaSuccess) return MLORA_ERR_CUDA;
+      attr_set = true;
+    }
+  }
+  CUtensorMap tQ, tB;
+  mlora_status_t ms;
+  if ((ms = make_tmap_bf16_blocked(ctx, &tQ, dY, h.ft_rows, L->d_out, lddy, vtc::ROWS, C::CB)) != MLORA_OK) return ms;
+  if ((ms = make_tmap_bf16_blocked(ctx, &tB, L->B_all, (uint64_t)L->n_adapters * R, L->d_out, L->d_out, C::RP, C::CB)) != MLORA_OK) return ms;
+  vtc::Args a;
+  a.scale = L->scale; a.blk_row0 = p->blk_row0; a.blk_nrows = p->blk_nrows; a.row_adapter = p->bwd.row_adapter;
+  a.NB = (int)h.blk_row0.size(); a.NS = (L->d_out + C::COLS - 1) / C::COLS; a.D = L->d_out;
+  a.V_out = ctx->ws_p;
+  a.pbd = PbdArgs{want_pbd ? ctx->ws_pbd : nullptr, p->bwd.row_grp2, p->bwd.tile2_grp_off, nullptr, p->bwd.zero_rows2, 0};
+  a.part_ws = ctx->ws_gpart; a.counters = ctx->ws_tc_counters; a.status = ctx->status_dev;
+  const int64_t tiles = (int64_t)a.NB * a.NS;
+  const int grid = tiles < ctx->sm_count ? (int)tiles : ctx->sm_count;
+  if (cancelled(ctx)) return MLORA_CANCELLED;
+  LaunchScope scope(ctx, st, KIND_SHRINK);
+  launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(vtc::THREADS), C::SMEM_BYTES, st, tQ, tB, a);
+  return scope.done();
 }
 
 // Both gradients on the tcgen05 kernel: can this call use it?  (A slot without rows gets its zeros from the
@@ -1229,8 +1264,23 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   sa.pbd = PbdArgs{(ctx->gemm_pairs && dX && !dropping) ? ctx->ws_pbd : nullptr, p->bwd.row_grp2, p->bwd.tile2_grp_off, nullptr,
                    p->bwd.zero_rows2, (int32_t)h.bwd.zero_rows2.size()};
   sa.item_adapter = p->bwd.item_adapter; sa.item_save = nullptr; sa.x_save = nullptr; sa.u_save = nullptr; sa.save_base = 0; sa.save_cap = 0;
-  if ((s = launch_shrink(ctx, L->rank, sa, h.bwd.n_items(), p->bwd.item_desc, h.ft_rows, L->n_adapters, st)) != MLORA_OK)
-    return s;
+  // V from the streaming shrink kernel; the tcgen05 V kernel under kernel variant 6 (measured on B200, one launch with
+  // its events: 31.1 vs 28.9 us on 2048 x 14336 rows of dY at rank 16, 22.9 vs 16.8 us on 2048 x 4096, 37.2 vs 30 us at
+  // rank 32 on 2048 x 13824 - the mma.sync kernel is the faster one at every size tried)
+  const bool tc_v = ctx->shrink_path == 0 && ctx->grad_mode == 2 && h.bwd.zero_rows2.empty() &&
+                    (int64_t)h.blk_row0.size() + 1 <= kTcCounters && h.ft_rows > 0;
+  if (tc_v) {
+    switch (L->rank) {
+      case 8: s = launch_vshrink_tc<8>(ctx, L, p, dY, lddy, sa.pbd.pbd != nullptr, st); break;
+      case 16: s = launch_vshrink_tc<16>(ctx, L, p, dY, lddy, sa.pbd.pbd != nullptr, st); break;
+      case 32: s = launch_vshrink_tc<32>(ctx, L, p, dY, lddy, sa.pbd.pbd != nullptr, st); break;
+      case 64: s = launch_vshrink_tc<64>(ctx, L, p, dY, lddy, sa.pbd.pbd != nullptr, st); break;
+      default: s = launch_vshrink_tc<128>(ctx, L, p, dY, lddy, sa.pbd.pbd != nullptr, st); break;
+    }
+  } else {
+    s = launch_shrink(ctx, L->rank, sa, h.bwd.n_items(), p->bwd.item_desc, h.ft_rows, L->n_adapters, st);
+  }
+  if (s != MLORA_OK) return s;
 
   GradArgs ga;                       // dB = (s U)^T dY
   ga.P = u_save; ga.R = L->rank; ga.scale = L->scale; ga.Q = (const __nv_bfloat16*)dY; ga.ldq = lddy; ga.D = L->d_out;
