@@ -4,8 +4,9 @@
  * residual-stream input of each layer is saved per fine-tuning token and the backward recomputes the
  * layer from it, so these pieces run again there and their input gradients are needed.  The paper
  * describes no kernels for them; the base model is frozen, so no gradient of the norm gain exists.)
- * Attention is here too, as a plain CUDA-core statement of the operation for the short sequences of the
- * fine-tuning path (one warp per row and head, keys visited one by one) - not a tensor-core kernel.
+ * Attention is here too: for head size 128 three tcgen05 kernels (forward, dq, dk/dv: scores and
+ * products in tensor memory, operands by TMA, every wait bounded with its status read by
+ * mlora_layer_ops_poll_status), for head size 64 plain CUDA-core kernels (one warp per row and head).
  *
  * All pointers are device pointers on the current device, all buffers borrowed; leading dimensions
  * (ld*) are in elements; rows and element counts must keep 16-byte alignment as stated per call.
@@ -46,7 +47,9 @@ mlora_status_t mlora_swiglu_forward(const void* g, const void* u, void* m, int64
 mlora_status_t mlora_swiglu_backward(const void* g, const void* u, const void* dm, void* dg, void* du, int64_t n,
                                      void* cuda_stream);
 
-/* out = a + b over n contiguous bf16 elements (n a multiple of 8); out may alias a or b. */
+/* out = a + b over n contiguous bf16 elements (n a multiple of 8); out may alias a or b.  The residual
+ * connections of the forward, and in the backward the sum of the gradients of a tensor that feeds several
+ * consumers (layer input -> norm and residual, normed input -> q, k and v or gate and up). */
 mlora_status_t mlora_add(const void* a, const void* b, void* out, int64_t n, void* cuda_stream);
 
 /* Causal softmax attention inside each sequence of a packed batch, grouped-query heads:

@@ -4,12 +4,14 @@ fine-tuning rows; the backward recomputes the layer from it, over the fine-tunin
 returns the LoRA gradients of all seven projections and the gradient of the layer input (what the
 layer below needs).
 
-Division of labour: the seven projections (q, k, v, o, gate, up, down) run in this library's kernels
-- `mlora_mixed_forward` in the serving pass, `mlora_mixed_forward` + `mlora_backward` in the
-recompute/backward pass - and so do RMSNorm, the rotary embedding, the SiLU gate and the residual adds
-with their input gradients, and attention as a plain CUDA-core kernel pair for short sequences
-(`mlora_layer_ops.h`).  PyTorch's autograd only strings the pieces together; every arithmetic step of
-the layer runs in this library.  A decode row is a one-token sequence (no KV cache in this module).
+Division of labour: every arithmetic step of the layer is a kernel of this library - the seven projections
+(q, k, v, o, gate, up, down) through `mlora_mixed_forward` (serving pass, recompute pass) and
+`mlora_backward`; RMSNorm, the rotary embedding, the SiLU gate, the residual adds and attention with
+their input gradients through the entry points of `mlora_layer_ops.h` (attention on the tcgen05 kernels
+for head size 128, CUDA-core kernels for head size 64).  The backward is written out call by call: where
+a tensor feeds several consumers (the layer input feeds the norm and the residual, the normed input feeds
+q, k and v, the second normed input feeds gate and up) the gradients are summed by `mlora_add`.  PyTorch
+only owns the buffers.  A decode row is a one-token sequence (no KV cache in this module).
 """
 from __future__ import annotations
 
@@ -36,112 +38,6 @@ class _Projection:
         self.x_save = torch.empty((cap_rows, self.d_in), dtype=torch.bfloat16, device=dev)
         self.u_save = torch.empty((cap_rows, self.rank), dtype=torch.float32, device=dev)
         self.dA = self.dB = None
-
-
-class _ProjFn(torch.autograd.Function):
-    """A multi-LoRA projection over a batch whose rows are all fine-tuning rows (the recompute pass)."""
-
-    @staticmethod
-    def forward(ctx, x, owner, name):
-        pr = owner.proj[name]
-        x = x.contiguous()
-        y = torch.empty((x.shape[0], pr.d_out), dtype=torch.bfloat16, device=x.device)
-        mb.mlora_mixed_forward(owner.sess.ctx, pr.layer, owner.bwd_plan, x, y, pr.x_save, pr.u_save, 0, pr.x_save.shape[0])
-        ctx.owner, ctx.name = owner, name
-        return y
-
-    @staticmethod
-    def backward(ctx, dy):
-        owner, pr = ctx.owner, ctx.owner.proj[ctx.name]
-        dy = dy.to(torch.bfloat16).contiguous()
-        n_slots = len(owner.bwd_slots)
-        pr.dA = torch.empty((n_slots, pr.rank, pr.d_in), dtype=torch.float32, device=dy.device)
-        pr.dB = torch.empty((n_slots, pr.rank, pr.d_out), dtype=torch.float32, device=dy.device)
-        dx = torch.empty((dy.shape[0], pr.d_in), dtype=torch.bfloat16, device=dy.device)
-        mb.mlora_backward(owner.sess.ctx, pr.layer, owner.bwd_plan, dy, pr.x_save, pr.u_save, pr.dA, pr.dB, dx)
-        return dx, None, None
-
-
-class _RmsNormFn(torch.autograd.Function):
-    @staticmethod
-    def forward(ctx, x, gain):
-        x = x.contiguous()
-        y = torch.empty_like(x)
-        mo.mlora_rmsnorm_forward(x, gain, y)
-        ctx.save_for_backward(x, gain)
-        return y
-
-    @staticmethod
-    def backward(ctx, dy):
-        x, gain = ctx.saved_tensors
-        dx = torch.empty_like(x)
-        mo.mlora_rmsnorm_backward(x, gain, dy.contiguous(), dx)
-        return dx, None
-
-
-class _RopeFn(torch.autograd.Function):
-    @staticmethod
-    def forward(ctx, x, pos, n_heads, d_head):
-        x = x.contiguous()
-        y = torch.empty_like(x)
-        mo.mlora_rope(x, y, pos, n_heads, d_head)
-        ctx.pos, ctx.shape = pos, (n_heads, d_head)
-        return y
-
-    @staticmethod
-    def backward(ctx, dy):
-        dx = torch.empty_like(dy)
-        mo.mlora_rope(dy.contiguous(), dx, ctx.pos, ctx.shape[0], ctx.shape[1], transpose=True)
-        return dx, None, None, None
-
-
-class _SwigluFn(torch.autograd.Function):
-    @staticmethod
-    def forward(ctx, g, u):
-        g, u = g.contiguous(), u.contiguous()
-        m = torch.empty_like(g)
-        mo.mlora_swiglu_forward(g, u, m)
-        ctx.save_for_backward(g, u)
-        return m
-
-    @staticmethod
-    def backward(ctx, dm):
-        g, u = ctx.saved_tensors
-        dg, du = torch.empty_like(g), torch.empty_like(u)
-        mo.mlora_swiglu_backward(g, u, dm.contiguous(), dg, du)
-        return dg, du
-
-
-class _AttnFn(torch.autograd.Function):
-    @staticmethod
-    def forward(ctx, q, k, v, seq_start, seq_end, n_heads, n_kv, d_head):
-        q, k, v = q.contiguous(), k.contiguous(), v.contiguous()
-        o = torch.empty_like(q)
-        lse = torch.empty((q.shape[0], n_heads), dtype=torch.float32, device=q.device)
-        mo.mlora_attention_forward(q, k, v, o, lse, seq_start, seq_end, n_heads, n_kv, d_head)
-        ctx.save_for_backward(q, k, v, o, lse)
-        ctx.meta = (seq_start, seq_end, n_heads, n_kv, d_head)
-        return o
-
-    @staticmethod
-    def backward(ctx, dO):
-        q, k, v, o, lse = ctx.saved_tensors
-        seq_start, seq_end, n_heads, n_kv, d_head = ctx.meta
-        dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
-        mo.mlora_attention_backward(q, k, v, o, lse, dO.contiguous(), dq, dk, dv, seq_start, seq_end, n_heads, n_kv, d_head)
-        return dq, dk, dv, None, None, None, None, None
-
-
-class _AddFn(torch.autograd.Function):
-    @staticmethod
-    def forward(ctx, a, b):
-        out = torch.empty_like(a)
-        mo.mlora_add(a.contiguous(), b.contiguous(), out)
-        return out
-
-    @staticmethod
-    def backward(ctx, d):
-        return d, d
 
 
 def sequence_tables(n_rows: int, sequences) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
@@ -176,20 +72,28 @@ class DecoderLayer:
         self.saved_rows = 0
         self.bwd_plan, self.bwd_slots = None, []
 
-    # -- shared layer body; `lin(name, x)` is the projection call ---------------------------------
+    # -- layer body; `lin(name, x)` is the projection call; returns the output and every intermediate ---
     def _body(self, x, lin, sequences):
         T = x.shape[0]
         dh = self.d // self.n_heads
-        pos, seq_start, seq_end = (torch.from_numpy(t).to(x.device) for t in sequence_tables(T, sequences))
-        h1 = _RmsNormFn.apply(x, self.g1)
-        q = _RopeFn.apply(lin("q", h1), pos, self.n_heads, dh)
-        k = _RopeFn.apply(lin("k", h1), pos, self.n_kv, dh)
-        v = lin("v", h1)
-        a = _AttnFn.apply(q, k, v, seq_start, seq_end, self.n_heads, self.n_kv, dh)
-        x2 = _AddFn.apply(x, lin("o", a))
-        h2 = _RmsNormFn.apply(x2, self.g2)
-        m = _SwigluFn.apply(lin("gate", h2), lin("up", h2))
-        return _AddFn.apply(x2, lin("down", m))
+        dev = x.device
+        pos, seq_start, seq_end = (torch.from_numpy(t).to(dev) for t in sequence_tables(T, sequences))
+        new = torch.empty_like
+        t = {"x": x, "pos": pos, "seq_start": seq_start, "seq_end": seq_end}
+        t["h1"] = new(x); mo.mlora_rmsnorm_forward(x, self.g1, t["h1"])
+        q0, k0, t["v"] = lin("q", t["h1"]), lin("k", t["h1"]), lin("v", t["h1"])
+        t["q"], t["k"] = new(q0), new(k0)
+        mo.mlora_rope(q0, t["q"], pos, self.n_heads, dh)
+        mo.mlora_rope(k0, t["k"], pos, self.n_kv, dh)
+        t["a"] = new(t["q"])
+        t["lse"] = torch.empty((T, self.n_heads), dtype=torch.float32, device=dev)
+        mo.mlora_attention_forward(t["q"], t["k"], t["v"], t["a"], t["lse"], seq_start, seq_end, self.n_heads, self.n_kv, dh)
+        t["x2"] = new(x); mo.mlora_add(x, lin("o", t["a"]), t["x2"])
+        t["h2"] = new(x); mo.mlora_rmsnorm_forward(t["x2"], self.g2, t["h2"])
+        t["g"], t["u"] = lin("gate", t["h2"]), lin("up", t["h2"])
+        t["m"] = new(t["g"]); mo.mlora_swiglu_forward(t["g"], t["u"], t["m"])
+        y = new(x); mo.mlora_add(t["x2"], lin("down", t["m"]), y)
+        return y, t
 
     # -- serving forward: mixed batch, keeps the layer input of the fine-tuning rows --------------
     @torch.no_grad()
@@ -206,7 +110,7 @@ class DecoderLayer:
                 y = torch.empty((n_rows, pr.d_out), dtype=torch.bfloat16, device=x.device)
                 mb.mlora_mixed_forward(self.sess.ctx, pr.layer, plan, inp.contiguous(), y, None, None, 0, 0)
                 return y
-            y = self._body(x, lin, segs[segs[:, 1] > 0][:, :2])
+            y, _ = self._body(x, lin, segs[segs[:, 1] > 0][:, :2])
         finally:
             torch.cuda.synchronize()
             mb.mlora_plan_destroy(plan)
@@ -229,13 +133,53 @@ class DecoderLayer:
         self.bwd_plan = mb.mlora_plan_create(self.sess.ctx, table, rows, self.n_adapters)
         self.bwd_slots = mb.mlora_plan_ft_adapters(self.bwd_plan)
         try:
-            x = self.saved_x[:rows].clone().requires_grad_(True)
-            with torch.enable_grad():
-                y = self._body(x, lambda name, inp: _ProjFn.apply(inp, self, name), [(int(s), int(n)) for s, n, _, _ in table])
-                y.backward(dy_ft.to(torch.bfloat16))
+            dev, ctx = self.saved_x.device, self.sess.ctx
+            n_slots = len(self.bwd_slots)
+            x = self.saved_x[:rows]
+            dh = self.d // self.n_heads
+
+            def lin(name, inp):          # recompute pass: every row is a fine-tuning row, each projection saves its own input and x A^T
+                pr = self.proj[name]
+                y = torch.empty((rows, pr.d_out), dtype=torch.bfloat16, device=dev)
+                mb.mlora_mixed_forward(ctx, pr.layer, self.bwd_plan, inp, y, pr.x_save, pr.u_save, 0, pr.x_save.shape[0])
+                return y
+
+            def lin_bwd(name, dy):       # LoRA gradients of one projection and the gradient of its input
+                pr = self.proj[name]
+                pr.dA = torch.empty((n_slots, pr.rank, pr.d_in), dtype=torch.float32, device=dev)
+                pr.dB = torch.empty((n_slots, pr.rank, pr.d_out), dtype=torch.float32, device=dev)
+                dx = torch.empty((rows, pr.d_in), dtype=torch.bfloat16, device=dev)
+                mb.mlora_backward(ctx, pr.layer, self.bwd_plan, dy, pr.x_save, pr.u_save, pr.dA, pr.dB, dx)
+                return dx
+
+            _y, t = self._body(x, lin, [(int(s), int(n)) for s, n, _, _ in table])
+            dy = dy_ft.to(torch.bfloat16).contiguous()
+            # y = x2 + down(m): dy reaches x2 directly and through the feed-forward branch
+            dm = lin_bwd("down", dy)
+            dg, du = torch.empty_like(t["g"]), torch.empty_like(t["u"])
+            mo.mlora_swiglu_backward(t["g"], t["u"], dm, dg, du)
+            dh2 = lin_bwd("gate", dg)
+            mo.mlora_add(dh2, lin_bwd("up", du), dh2)                   # h2 feeds gate and up
+            dx2 = torch.empty_like(x)
+            mo.mlora_rmsnorm_backward(t["x2"], self.g2, dh2, dx2)
+            mo.mlora_add(dx2, dy, dx2)                                  # x2 feeds the norm and the residual
+            # x2 = x + o(a)
+            da = lin_bwd("o", dx2)
+            dq, dk, dv = torch.empty_like(t["q"]), torch.empty_like(t["k"]), torch.empty_like(t["v"])
+            mo.mlora_attention_backward(t["q"], t["k"], t["v"], t["a"], t["lse"], da, dq, dk, dv, t["seq_start"], t["seq_end"],
+                                        self.n_heads, self.n_kv, dh)
+            dq0, dk0 = torch.empty_like(dq), torch.empty_like(dk)
+            mo.mlora_rope(dq, dq0, t["pos"], self.n_heads, dh, transpose=True)
+            mo.mlora_rope(dk, dk0, t["pos"], self.n_kv, dh, transpose=True)
+            dh1 = lin_bwd("q", dq0)
+            mo.mlora_add(dh1, lin_bwd("k", dk0), dh1)                   # h1 feeds q, k and v
+            mo.mlora_add(dh1, lin_bwd("v", dv), dh1)
+            dx = torch.empty_like(x)
+            mo.mlora_rmsnorm_backward(x, self.g1, dh1, dx)
+            mo.mlora_add(dx, dx2, dx)                                   # x feeds the norm and the residual
             torch.cuda.synchronize()
             grads = {n: (self.proj[n].dA, self.proj[n].dB) for n in PROJ}
-            return x.grad, grads, list(self.bwd_slots)
+            return dx, grads, list(self.bwd_slots)
         finally:
             mb.mlora_plan_destroy(self.bwd_plan)
             self.bwd_plan = None
