@@ -49,7 +49,7 @@ def test_layer_forward_and_recompute_backward_match_the_oracle():
         y = layer.forward(x.to(sess.device).to(torch.bfloat16), synth.segments_array(segs))
         assert mb.mlora_poll_status(sess.ctx) == mb.MLORA_OK
         err = (y.double().cpu() - y_ref).abs()
-        assert float((err - 6e-2 * (1 + y_ref.abs())).max()) <= 0, float(err.max())
+        assert float((err - 3e-2 * (1 + y_ref.abs())).max()) <= 0, float(err.max())   # measured 2.2e-2: a dozen bf16 roundings in series (norms, rotary, scores, three residual adds), one more than the hot path's 2e-2 allows
         assert layer.saved_rows == 97 and layer.saved == [(64, 1), (33, 2)]
         assert torch.equal(layer.saved_x[:97].cpu().double(), x[45:142])      # the layer input, bit for bit
 
@@ -66,8 +66,8 @@ def test_layer_forward_and_recompute_backward_match_the_oracle():
             scale = float(want.abs().max())
             bad = float(((got - want).abs() - tol * (scale + want.abs())).max())
             assert bad <= 0, (name, bad, scale)
-        close("dx", dx, ref["dx"], 4e-2)
+        close("dx", dx, ref["dx"], 2e-2)
         for name in PROJ:
-            close("dA_" + name, grads[name][0], ref["dA_" + name], 4e-2)
-            close("dB_" + name, grads[name][1], ref["dB_" + name], 4e-2)
+            close("dA_" + name, grads[name][0], ref["dA_" + name], 2e-2)
+            close("dB_" + name, grads[name][1], ref["dB_" + name], 2e-2)
         assert layer.saved_rows == 0
