@@ -295,7 +295,11 @@ int32_t mlora_profile_collect(mlora_ctx* ctx, int32_t* kinds, float* ms, int32_t
  * tiles for the SMs is cut into K slices whose fp32 partials a small kernel adds up);
  * 5 = defaults, but both gradients on the mma.sync kernels for every rank (by default rank 128 uses the
  * tcgen05 gradient kernel); 6 = defaults, but the whole rank-r part of the backward on tcgen05 kernels for every
- * rank: V = s dY B^T and both gradients (with dropout on, the gradients stay on the mma.sync kernels). */
+ * rank: V = s dY B^T and both gradients (with dropout on, the gradients stay on the mma.sync kernels);
+ * 7 = defaults, but the two-SM GEMM always deals its tiles out round robin (by default a batch whose
+ * 256-row tiles differ much in their number of adapter groups gets, per shape it is used with, a list
+ * that spreads the tiles over the CTA pairs by cost; the list is built on the host at the first such
+ * call, kept with the plan, and never built while the stream is being captured). */
 mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path);
 
 /* ---- forward without any allocation -----------------------------------------------------*/

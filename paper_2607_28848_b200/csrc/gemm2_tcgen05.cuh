@@ -126,7 +126,7 @@ __device__ __forceinline__ bool gemm2_wait(uint32_t bar, uint32_t parity, volati
 // Tile order: m-fastest inside bands of `group_m` row tiles (all row tiles when group_m == 0), so
 // that the tiles in flight at one time cover a near-square block of the output and the operand
 // panels they stream together are as few as possible.
-__device__ __forceinline__ void gemm2_tile(const GemmArgs& args, int tile, int& mt, int& nt) {
+__host__ __device__ __forceinline__ void gemm2_tile(const GemmArgs& args, int tile, int& mt, int& nt) {
   const int gm_full = args.group_m > 0 ? args.group_m : args.n_mtiles;
   const int band_tiles = gm_full * args.n_ntiles;
   const int band = tile / band_tiles, r = tile - band * band_tiles;
@@ -137,7 +137,7 @@ __device__ __forceinline__ void gemm2_tile(const GemmArgs& args, int tile, int& 
 }
 
 // Work unit -> (tile, K slice, slices of that tile).
-__device__ __forceinline__ void gemm2_unit(const GemmArgs& args, int unit, int& tile, int& ks, int& sk) {
+__host__ __device__ __forceinline__ void gemm2_unit(const GemmArgs& args, int unit, int& tile, int& ks, int& sk) {
   if (unit < args.n_whole) { tile = unit; ks = 0; sk = 1; return; }
   const int u = unit - args.n_whole;
   ks = u / args.n_tail;
@@ -210,6 +210,12 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
   const int n_units = args.n_units;
   const int n_pairs = gridDim.x >> 1;
   const int pair = blockIdx.x >> 1;
+  // Units of this pair: every n_pairs-th one, or - when the tiles differ in cost (adapter-heavy row tiles) -
+  // entries [unit_list[pair], unit_list[pair + 1]) of a list the host balanced by cost.
+  const int32_t* ulist = args.unit_list;
+  const int u_begin = ulist ? ulist[pair] : pair;
+  const int u_end = ulist ? ulist[pair + 1] : n_units;
+  const int u_step = ulist ? 1 : n_pairs;
 
   auto tile_groups = [&](int mt) -> int {
     return args.lora_enabled ? (args.tile_grp_off[mt + 1] - args.tile_grp_off[mt]) : 0;
@@ -223,7 +229,8 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
     int32_t* ga_smem = reinterpret_cast<int32_t*>(smem_gen + (sMisc - smem_base) + 64);   // 256 entries
     uint32_t it = 0;
     bool ok = true;
-    for (int unit = pair; unit < n_units && ok; unit += n_pairs) {
+    for (int ui = u_begin; ui < u_end && ok; ui += u_step) {
+      const int unit = ulist ? ulist[ui] : ui;
       int tile, ks, SK;
       gemm2_unit(args, unit, tile, ks, SK);
       int mt, nt;
@@ -300,7 +307,8 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
       constexpr uint32_t idesc_lora = ptx::make_idesc_bf16(GEMM2_BM, GEMM2_BN, false, true);
       uint32_t it = 0, lt = 0;
       bool ok = true;
-      for (int unit = pair; unit < n_units && ok; unit += n_pairs, ++lt) {
+      for (int ui = u_begin; ui < u_end && ok; ui += u_step, ++lt) {
+        const int unit = ulist ? ulist[ui] : ui;
         int tile, ks, SK;
         gemm2_unit(args, unit, tile, ks, SK);
         int mt, nt_unused;
@@ -356,7 +364,8 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
     const uint32_t stage0 = sEpi + (uint32_t)(warp - 2) * 8192u;
     uint32_t lt = 0;
     bool ok = true;
-    for (int unit = pair; unit < n_units && ok; unit += n_pairs, ++lt) {
+    for (int ui = u_begin; ui < u_end && ok; ui += u_step, ++lt) {
+      const int unit = ulist ? ulist[ui] : ui;
       int tile, ks, SK;
       gemm2_unit(args, unit, tile, ks, SK);
       int mt, nt;

@@ -58,6 +58,11 @@ struct GemmArgs {
   // the last, partly filled wave are.
   int32_t split_k, n_whole, n_tail;
   float* ws_splitk;
+  // Two-SM kernel only: nullptr (pair p takes units p, p + pairs, ...) or a list balanced by cost:
+  // [0, pairs] offsets into this same array, then the units of each pair (sched_pairs = the pair count
+  // the list was made for).
+  const int32_t* unit_list;
+  int32_t sched_pairs;
   const int32_t* row_grp;        // [M] group of the row inside its 128-row tile, -1: none
   const int32_t* row_adapter;    // [M]
   const int32_t* tile_grp_off;   // [n_mtiles + 1]

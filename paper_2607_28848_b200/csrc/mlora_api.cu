@@ -8,7 +8,9 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <algorithm>
 #include <mutex>
+#include <queue>
 #include <new>
 #include <utility>
 #include <vector>
@@ -72,6 +74,7 @@ struct mlora_ctx {
   int32_t shrink_path = 0;           // 0: streaming shrink for rank <= 64 (gradients: <= 32); 1: per-item kernels for every rank
   int32_t gemm_pairs = 1;            // 1: two-SM (CTA pair) tensor-core kernel; 0: one-SM kernel
   int32_t no_split_k = 0;            // 1: the two-SM kernel never splits K (kernel variant 4)
+  int32_t no_unit_lists = 0;         // 1: the two-SM kernel always deals its units out round robin (kernel variant 7)
   int32_t grad_mode = 0;             // 0: default choice by rank; 1: mma.sync kernels for every rank (kernel variant 5);
                                      // 2: the tcgen05 gradient kernel for every rank (kernel variant 6)
   EncodeTiledFn encode = nullptr;
@@ -91,8 +94,30 @@ constexpr int kTcGradMinRank = 128;
 
 enum { KIND_SHRINK = 0, KIND_GEMM_FWD = 1, KIND_GEMM_BWD = 2, KIND_GRAD = 3, KIND_SIMT = 4, KIND_ADAMW = 5, KIND_REDUCE = 6 };
 
+// Cost-balanced unit lists of the two-SM GEMM (see balanced_units), cached per plan and row space: a
+// batch whose row tiles differ much in their number of adapter groups gets, per (columns, depth, rank)
+// it is used with, one list in device memory reserved with the plan's tables.
+constexpr int kSchedSlots = 4;          // shapes per row space; further shapes run round robin
+constexpr int kSchedCap = 8192;         // 32-bit words per list (pairs + 1 offsets, then the units)
+struct SchedEntry {
+  int32_t n_ntiles = 0, kblocks = 0, rank = 0, pairs = 0, n_whole = 0, n_tail = 0, split_k = 0, group_m = 0;
+  bool use = false;                     // false: round robin is as good for this shape
+  cudaEvent_t filled = nullptr;         // recorded behind the copy that fills the device list
+  cudaStream_t stream = nullptr;        // the stream of that copy
+  std::vector<int32_t> host;            // source of that copy
+};
+struct SchedCache {
+  std::mutex mu;
+  int32_t* dev = nullptr;               // [kSchedSlots][kSchedCap], nullptr: nothing reserved (even row space)
+  int32_t n = 0;
+  int32_t lc_spread = 0;                // most minus fewest adapter groups of a 256-row tile
+  SchedEntry e[kSchedSlots];
+  ~SchedCache() { for (SchedEntry& x : e) if (x.filled) cudaEventDestroy(x.filled); }
+};
+
 // Device copy of one RowSpace.
 struct DevRowSpace {
+  SchedCache* sched = nullptr;
   const int32_t* row_adapter = nullptr;
   const int32_t* row_save = nullptr;
   const int32_t* row_grp = nullptr;
@@ -117,6 +142,7 @@ struct mlora_plan {
   PlanBuf buf;                       // pooled plans: the buffer pair the tables live in (blob == buf.dev)
   bool pooled = false;
   DevRowSpace fwd, bwd;
+  SchedCache sched[2];               // unit lists of the forward and the compact row space
   const int32_t* slot_chunk_off = nullptr;
   const int32_t* chunk_row0 = nullptr;
   const int32_t* chunk_nrows = nullptr;
@@ -627,8 +653,10 @@ mlora_status_t launch_gemm2_r(mlora_ctx* ctx, const CUtensorMap& tIn, const CUte
   const int pairs = g.n_units < max_pairs ? g.n_units : max_pairs;
   attr_lock.unlock();
   if (cancelled(ctx)) return MLORA_CANCELLED;
+  GemmArgs ga = g;
+  if (ga.unit_list && ga.sched_pairs != pairs) ga.unit_list = nullptr;   // the list was made for another grid
   LaunchScope scope(ctx, st, W_KMAJOR ? KIND_GEMM_BWD : KIND_GEMM_FWD);
-  launch_pdl_pairs(scope.slot < 0, kern, dim3(2 * pairs), dim3(GEMM2_THREADS), GEMM2_SMEM_BYTES, st, tIn, tW, tL, tOut, tPbd, g);
+  launch_pdl_pairs(scope.slot < 0, kern, dim3(2 * pairs), dim3(GEMM2_THREADS), GEMM2_SMEM_BYTES, st, tIn, tW, tL, tOut, tPbd, ga);
   return scope.done();
 }
 
@@ -658,6 +686,99 @@ mlora_status_t launch_gemm(mlora_ctx* ctx, int R, const CUtensorMap& tIn, const 
   }
 }
 
+// Units of the two-SM GEMM dealt out by cost.  The kernel's default - pair p takes units p, p + pairs, ... -
+// assumes tiles of equal cost; a 256-row tile with G adapter groups carries ceil(G r / 64) low-rank
+// K-blocks on top of its K / 64 main ones, so a batch with one tile of 135 single-row adapters next to
+// tiles of one group (rank 128: 334 against 66 blocks) leaves the pairs that meet the heavy tiles with
+// 1.5 times the mean load.  Here the units go, heaviest first, to the pair with the least load so far
+// (each pair's units then in tile order).  The list is made once per plan and shape on the host and
+// copied behind the plan's tables; g.unit_list stays null when round robin is within 3% of it, when the
+// plan reserved no room (even row spaces), or when the stream is being captured before the list exists.
+void balanced_units(mlora_ctx* ctx, const RowSpace& hs, const DevRowSpace& ds, int R, int kblocks, GemmArgs& g,
+                    cudaStream_t st) {
+  g.unit_list = nullptr; g.sched_pairs = 0;
+  SchedCache* sc = ds.sched;
+  if (!sc || !sc->dev || ctx->no_unit_lists || !g.lora_enabled) return;
+  if ((int64_t)sc->lc_spread * R < 2 * 64) return;          // tiles differ by less than two K-blocks
+  const int pairs = g.n_units < ctx->sm_count / 2 ? g.n_units : ctx->sm_count / 2;
+  if (pairs < 2 || g.n_units + pairs + 1 > kSchedCap) return;
+  std::lock_guard<std::mutex> lock(sc->mu);
+  SchedEntry* e = nullptr;
+  int slot = 0;
+  for (; slot < sc->n; ++slot) {
+    SchedEntry& x = sc->e[slot];
+    if (x.n_ntiles == g.n_ntiles && x.kblocks == kblocks && x.rank == R && x.pairs == pairs && x.n_whole == g.n_whole &&
+        x.n_tail == g.n_tail && x.split_k == g.split_k && x.group_m == g.group_m) { e = &x; break; }
+  }
+  if (!e) {
+    if (sc->n >= kSchedSlots) return;
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) { cudaGetLastError(); return; }
+    // cost of every unit in K-blocks (+2: accumulator hand-over and the first loads of a tile)
+    std::vector<int32_t> cost(g.n_units);
+    for (int u = 0; u < g.n_units; ++u) {
+      int tile, ks, sk, mt, nt;
+      gemm2_unit(g, u, tile, ks, sk);
+      gemm2_tile(g, tile, mt, nt);
+      const int G = hs.tile2_grp_off[mt + 1] - hs.tile2_grp_off[mt];
+      const int LC = (G * R + 63) / 64;
+      const int kb = (int)((int64_t)(ks + 1) * kblocks / sk) - (int)((int64_t)ks * kblocks / sk);
+      const int lc = (int)((int64_t)(ks + 1) * LC / sk) - (int)((int64_t)ks * LC / sk);
+      cost[u] = kb + lc + 2;
+    }
+    std::vector<int64_t> rr(pairs, 0);
+    for (int u = 0; u < g.n_units; ++u) rr[u % pairs] += cost[u];
+    const int64_t rr_max = *std::max_element(rr.begin(), rr.end());
+    std::vector<int32_t> order(g.n_units);
+    for (int u = 0; u < g.n_units; ++u) order[u] = u;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return cost[a] > cost[b]; });
+    typedef std::pair<int64_t, int> Load;                     // (load, pair): the least loaded pair, lowest index first
+    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+    for (int p = 0; p < pairs; ++p) heap.push(Load(0, p));
+    std::vector<std::vector<int32_t>> mine(pairs);
+    int64_t lpt_max = 0;
+    for (int u : order) {
+      Load l = heap.top(); heap.pop();
+      l.first += cost[u];
+      mine[l.second].push_back(u);
+      lpt_max = l.first > lpt_max ? l.first : lpt_max;
+      heap.push(l);
+    }
+    e = &sc->e[sc->n];
+    e->n_ntiles = g.n_ntiles; e->kblocks = kblocks; e->rank = R; e->pairs = pairs; e->n_whole = g.n_whole;
+    e->n_tail = g.n_tail; e->split_k = g.split_k; e->group_m = g.group_m;
+    e->use = 100 * lpt_max < 97 * rr_max;
+    slot = sc->n;
+    if (e->use) {
+      e->host.assign(pairs + 1, 0);            // offsets (into this same array), then each pair's units in tile order
+      for (int p = 0; p < pairs; ++p) {
+        std::sort(mine[p].begin(), mine[p].end());
+        e->host[p] = (int32_t)e->host.size();
+        e->host.insert(e->host.end(), mine[p].begin(), mine[p].end());
+      }
+      e->host[pairs] = (int32_t)e->host.size();
+      if (cudaEventCreateWithFlags(&e->filled, cudaEventDisableTiming) != cudaSuccess ||
+          cudaMemcpyAsync(sc->dev + (size_t)slot * kSchedCap, e->host.data(), e->host.size() * sizeof(int32_t),
+                          cudaMemcpyHostToDevice, st) != cudaSuccess ||
+          cudaEventRecord(e->filled, st) != cudaSuccess) {
+        cudaGetLastError();
+        e->use = false;
+      }
+      e->stream = st;
+    }
+    sc->n++;
+  }
+  if (!e->use) return;
+  if (e->stream != st && e->filled) {        // another stream than the one that filled the list: order behind the copy
+    if (cudaEventQuery(e->filled) != cudaSuccess) {
+      cudaGetLastError();
+      if (cudaStreamWaitEvent(st, e->filled, 0) != cudaSuccess) { cudaGetLastError(); return; }
+    }
+  }
+  g.unit_list = sc->dev + (size_t)slot * kSchedCap;
+  g.sched_pairs = e->pairs;
+}
+
 // Out = In Wop + (scale) P L over one row space, tensor-core path.
 template <bool W_KMAJOR>
 mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace& hs, const DevRowSpace& ds,
@@ -676,7 +797,7 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
     return s;
   if ((s = make_tmap_bf16(ctx, &tOut, Out, N, M, ld_out, 64, 32)) != MLORA_OK) return s;
   GemmArgs g;
-  g.M = M; g.N = N; g.K = K; g.split_k = 1; g.ws_splitk = nullptr;
+  g.M = M; g.N = N; g.K = K; g.split_k = 1; g.ws_splitk = nullptr; g.unit_list = nullptr; g.sched_pairs = 0;
   // Long contractions with many row tiles: the operand panels of one wave of tiles no longer fit the
   // L2 together with their neighbours', so the tiles are walked in bands of 8 row tiles (a wave then
   // covers about 8 x 9 tiles and streams 17 panels instead of 16 + 5 per 74 tiles; measured +2% on
@@ -726,6 +847,7 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
     g.row_grp = ds.row_grp2; g.row_adapter = ds.row_adapter;
     g.tile_grp_off = ds.tile2_grp_off; g.grp_adapter = ds.grp2_adapter;
     g.P = P; g.scale = scale; g.status = ctx->status_dev;
+    balanced_units(ctx, hs, ds, R, kblocks, g, st);
     CUtensorMap tPbd;
     const uint64_t slots = g.lora_enabled ? 2 * (uint64_t)hs.grp2_adapter.size() : 1;
     if ((s = make_tmap_bf16(ctx, &tPbd, ctx->ws_pbd ? (const void*)ctx->ws_pbd : In, 64, slots * 256, 64, 64, 128)) != MLORA_OK)
@@ -1021,6 +1143,36 @@ void pack_plan(const HostPlan& h, BlobBuilder& b, size_t* o) {
   o[n++] = b.add(h.slot_blk_off); o[n++] = b.add(h.blk_row0); o[n++] = b.add(h.blk_nrows);
 }
 
+// Words to reserve behind the plan's tables for unit lists: only row spaces whose 256-row tiles differ in
+// their number of adapter groups can need one.
+size_t sched_reserve(mlora_plan* p) {
+  const RowSpace* rs[2] = {&p->h.fwd, &p->h.bwd};
+  size_t words = 0;
+  for (int i = 0; i < 2; ++i) {
+    int32_t lo = 1 << 30, hi = 0;
+    const std::vector<int32_t>& off = rs[i]->tile2_grp_off;
+    for (size_t t = 0; t + 1 < off.size(); ++t) {
+      const int32_t g = off[t + 1] - off[t];
+      lo = g < lo ? g : lo; hi = g > hi ? g : hi;
+    }
+    p->sched[i].lc_spread = hi > lo ? hi - lo : 0;
+    if (off.size() > 2 && hi - lo >= 2) words += (size_t)kSchedSlots * kSchedCap;
+  }
+  return words;
+}
+// Points the unit-list areas at the reserved words that start at word `at` of the blob.
+void bind_sched(mlora_plan* p, size_t at) {
+  const RowSpace* rs[2] = {&p->h.fwd, &p->h.bwd};
+  DevRowSpace* ds[2] = {&p->fwd, &p->bwd};
+  for (int i = 0; i < 2; ++i) {
+    ds[i]->sched = &p->sched[i];
+    if (rs[i]->tile2_grp_off.size() > 2 && p->sched[i].lc_spread >= 2) {
+      p->sched[i].dev = p->blob + at;
+      at += (size_t)kSchedSlots * kSchedCap;
+    }
+  }
+}
+
 // Points the plan's table pointers into p->blob.
 void bind_plan(mlora_plan* p, const size_t* o) {
   DevRowSpace* ds[2] = {&p->fwd, &p->bwd};
@@ -1096,11 +1248,13 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
     BlobBuilder b;
     size_t o[kPlanTables];
     pack_plan(p->h, b, o);
-    if (cudaMalloc(&p->blob, b.data.size() * sizeof(int32_t)) != cudaSuccess) { delete p; return MLORA_ERR_CUDA; }
+    const size_t reserve = sched_reserve(p);
+    if (cudaMalloc(&p->blob, (b.data.size() + reserve) * sizeof(int32_t)) != cudaSuccess) { delete p; return MLORA_ERR_CUDA; }
     if (cudaMemcpy(p->blob, b.data.data(), b.data.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
       cudaFree(p->blob); delete p; return MLORA_ERR_CUDA;
     }
     bind_plan(p, o);
+    bind_sched(p, b.data.size());
     if ((s = grow_workspaces(ctx, p->h, n_rows)) != MLORA_OK) { cudaFree(p->blob); delete p; return s; }
   }
   *out = p;
@@ -1121,7 +1275,8 @@ mlora_status_t mlora_plan_create_async(mlora_ctx* ctx, const mlora_segment_t* se
   BlobBuilder b;
   size_t o[kPlanTables];
   pack_plan(p->h, b, o);
-  const size_t need = b.data.size();
+  const size_t tables = b.data.size();
+  const size_t need = tables + sched_reserve(p);
   // a released buffer pair that is large enough and whose last user has passed its release point
   for (size_t i = 0; i < ctx->plan_pool.size(); ++i) {
     PlanBuf& c = ctx->plan_pool[i];
@@ -1145,11 +1300,12 @@ mlora_status_t mlora_plan_create_async(mlora_ctx* ctx, const mlora_segment_t* se
   }
   p->pooled = true;
   p->blob = p->buf.dev;
-  std::memcpy(p->buf.pinned, b.data.data(), need * sizeof(int32_t));
-  if (cudaMemcpyAsync(p->blob, p->buf.pinned, need * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+  std::memcpy(p->buf.pinned, b.data.data(), tables * sizeof(int32_t));
+  if (cudaMemcpyAsync(p->blob, p->buf.pinned, tables * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess) {
     free_plan_buf(p->buf); delete p; return MLORA_ERR_CUDA;
   }
   bind_plan(p, o);
+  bind_sched(p, tables);
   if ((s = grow_workspaces(ctx, p->h, n_rows)) != MLORA_OK) { free_plan_buf(p->buf); delete p; return s; }
   *out = p;
   return MLORA_OK;
@@ -1412,11 +1568,12 @@ mlora_status_t mlora_set_dropout(mlora_ctx* ctx, double p, uint64_t seed) {
 int64_t mlora_launch_count(const mlora_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 mlora_status_t mlora_set_gemm_path(mlora_ctx* ctx, int32_t path) {
-  if (!ctx || path < 0 || path > 6) return MLORA_ERR_INVALID_ARG;
+  if (!ctx || path < 0 || path > 7) return MLORA_ERR_INVALID_ARG;
   ctx->gemm_path = path == 1 ? 1 : 0;
   ctx->shrink_path = path == 2 ? 1 : 0;
   ctx->gemm_pairs = path == 3 ? 0 : 1;
   ctx->no_split_k = path == 4 ? 1 : 0;
+  ctx->no_unit_lists = path == 7 ? 1 : 0;
   ctx->grad_mode = path == 5 ? 1 : (path == 6 ? 2 : 0);
   return MLORA_OK;
 }

@@ -124,6 +124,37 @@ def test_k_split_of_the_last_wave_only(sess, d_in, d_out):
     run_and_check(sess, w, t, path=4, blocked=True)
 
 
+@pytest.mark.parametrize("rank", [32, 128])
+def test_row_tiles_of_unequal_cost_get_balanced_unit_lists(sess, rank):
+    """One 256-row tile of 200 single-row adapters between tiles of one group each: the heavy tile carries
+    100 (rank 32) or 400 (rank 128) low-rank K-blocks against 8 main ones, so the units of the two-SM
+    kernel are dealt out by cost from a list kept with the plan instead of round robin (5 x 20 tiles on
+    74 pairs).  Same numbers as the oracle's, and bit for bit those of the round-robin variant (7): which
+    pair computes a tile does not enter its arithmetic.  The second pass finds the list cached."""
+    segs = [(0, 256, 0, 0)] + [(256 + i, 1, 1 + i, 0) for i in range(200)] + [(456, 56, 201, 0), (512, 300, 202, 1),
+                                                                               (812, 212, 203, 1), (1024, 90, 3, 0)]
+    w = synth.Workload("uneven_tiles", 512, 5120, rank, 204, "bf16", 1114, synth.segments_array(segs), seed=70 + rank)
+    t = synth.make_tensors(w)
+    outs = []
+    for path in (0, 0, 7):
+        run = None
+        mb.mlora_set_gemm_path(sess.ctx, path)
+        run = LayerRun(sess, w.dtype, t, w.segments, w.n_rows)
+        try:
+            for _ in range(2):
+                run.forward(); run.backward()
+            assert run.status() == mb.MLORA_OK
+            outs.append([b.clone() for b in (run.Y, run.dX, run.dA, run.dB)])
+        finally:
+            mb.mlora_set_gemm_path(sess.ctx, 0)
+            run.close()
+    for a, b in zip(outs[0], outs[1]):
+        assert torch.equal(a, b)
+    for a, b in zip(outs[0], outs[2]):
+        assert torch.equal(a, b)
+    run_and_check(sess, w, t, blocked=True)
+
+
 @pytest.mark.parametrize("path", [0, 3])
 @pytest.mark.parametrize("d_in,d_out", [(64, 128), (128, 64), (320, 448), (192, 320)])
 def test_output_width_not_a_multiple_of_the_column_tile(sess, path, d_in, d_out):
