@@ -287,15 +287,17 @@ int64_t mlora_launch_count(const mlora_ctx* ctx);
 mlora_status_t mlora_profile_enable(mlora_ctx* ctx, int32_t max_records);
 int32_t mlora_profile_collect(mlora_ctx* ctx, int32_t* kinds, float* ms, int32_t cap);
 
-/* Selects kernel variants for MLORA_BF16 layers: 0 = defaults (two-SM tcgen05 tensor-core GEMM,
- * streaming shrink and gradient kernels for rank <= 64, tcgen05 gradient kernel for rank 128); 1 = the plain CUDA-core kernels for every step (a slow
- * cross-check used by the tests); 2 = defaults, but the per-item shrink kernel for every rank
- * (the variant rank 128 always uses); 3 = defaults, but the one-SM tensor-core GEMM;
+/* Selects kernel variants for MLORA_BF16 layers: 0 = defaults (two-SM tcgen05 tensor-core GEMM; rank <= 32:
+ * streaming mma.sync shrink and gradient kernels; rank 64 and 128: the tcgen05 shrink with its finish
+ * kernel for U = X A^T and V = s dY B^T wherever the rows come in runs of four or more per adapter on
+ * average, and the tcgen05 gradient kernel); 1 = the plain CUDA-core kernels for every step (a slow
+ * cross-check used by the tests); 2 = defaults, but the per-item mma.sync shrink and gradient kernels
+ * for every rank; 3 = defaults, but the one-SM tensor-core GEMM;
  * 4 = defaults, but the two-SM GEMM never splits K (by default a product with too few output
  * tiles for the SMs is cut into K slices whose fp32 partials a small kernel adds up);
- * 5 = defaults, but both gradients on the mma.sync kernels for every rank (by default rank 128 uses the
- * tcgen05 gradient kernel); 6 = defaults, but the whole rank-r part of the backward on tcgen05 kernels for every
- * rank: V = s dY B^T and both gradients (with dropout on, the gradients stay on the mma.sync kernels);
+ * 5 = defaults, but both gradients on the mma.sync kernels for every rank;
+ * 6 = defaults, but every rank-r product on the tcgen05 kernels for every rank: U, V and both gradients
+ * (with dropout on, everything stays on the mma.sync kernels);
  * 7 = defaults, but the two-SM GEMM always deals its tiles out round robin (by default a batch whose
  * 256-row tiles differ much in their number of adapter groups gets, per shape it is used with, a list
  * that spreads the tiles over the CTA pairs by cost; the list is built on the host at the first such

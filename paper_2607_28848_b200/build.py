@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG_DIR)
 LIB_PATH = os.path.join(PKG_DIR, "libmlora.so")
 SOURCES = [os.path.join(PKG_DIR, "csrc", "mlora_api.cu"), os.path.join(PKG_DIR, "csrc", "sched.cpp")]
 HEADERS = [os.path.join(PKG_DIR, "csrc", f) for f in
-           ("plan.h", "ptx.cuh", "dropout.cuh", "gemm_tcgen05.cuh", "gemm2_tcgen05.cuh", "skinny.cuh", "grad_tc.cuh", "vshrink_tc.cuh", "simt.cuh", "glue.cuh", "attention.cuh", "attention_tc.cuh")] + \
+           ("plan.h", "ptx.cuh", "dropout.cuh", "gemm_tcgen05.cuh", "gemm2_tcgen05.cuh", "skinny.cuh", "grad_tc.cuh", "shrink_tc.cuh", "simt.cuh", "glue.cuh", "attention.cuh", "attention_tc.cuh")] + \
           [os.path.join(ROOT, "include", f) for f in ("mlora.h", "mlora_sched.h", "mlora_layer_ops.h")]
 
 

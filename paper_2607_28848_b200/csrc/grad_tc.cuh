@@ -86,6 +86,7 @@ struct Args {
   int32_t accumulate;
   int32_t snap;                  // ranges end at strip boundaries (no partial pieces)
   int32_t* status;
+  const uint8_t* pop;            // nullable: the P operands made ahead by psplit_kernel, [2 problems][NB][P_BYTES]
 };
 
 // Position in one problem's tile list (slot > strip > block).
@@ -142,6 +143,57 @@ struct Ranges {
     return (int)(((g + 1) * G + N - 1) / N) - 1;
   }
 };
+
+// The P operands of both problems, made once per block instead of once per tile: grid = (NB, 2, R / QC), 128
+// threads, thread = row of the block, a CTA takes QC = 32 (rank 8, 16: all) of the low-rank columns.  Image of a block = what the kernel's operand buffer holds: (scaled) P[row, :] as
+// bf16 head | remainder, [2 K-blocks of 64 rows][N2 columns][128 B] with the 16-byte pieces swizzled by the
+// column index, rows past the block's end zero.  The gradient kernel then fetches an operand with one bulk copy.
+__host__ __device__ constexpr int psplit_cols(int r) { return r < 32 ? r : 32; }
+
+template <int R>
+__global__ void __launch_bounds__(128)
+psplit_kernel(const Args a, uint8_t* pop) {
+  using C = Cfg<R>;
+  constexpr int N2 = C::N2;
+  const int blk = blockIdx.x, p = blockIdx.y, trow = threadIdx.x;
+  const Problem& pr = a.prob[p];
+  int slot = 0;
+  while (slot + 1 < a.n_slots && a.slot_blk_off[slot + 1] <= blk) ++slot;
+  const int nrows = a.blk_nrows[blk], row0 = a.blk_row0[blk];
+  const bool live = trow < nrows;
+  const float sc = pr.scale ? pr.scale[a.slot_adapter[slot]] : 1.0f;
+  ptx::grid_dependency_wait();               // V comes from the launch before
+  ptx::grid_launch_dependents();
+  uint8_t* img = pop + ((size_t)p * a.NB + blk) * C::P_BYTES + (size_t)(trow >> 6) * (N2 * 128u);
+  const uint32_t kk = (uint32_t)(trow & 63);
+  const float4* src = reinterpret_cast<const float4*>(pr.P + (size_t)(row0 + (live ? trow : 0)) * R);
+  constexpr int QC = psplit_cols(R);
+  {
+    const int q0 = (int)blockIdx.z * QC;
+    float pv[QC];
+#pragma unroll
+    for (int c0 = 0; c0 < QC; c0 += 4) {
+      const float4 x = __ldg(src + ((q0 + c0) >> 2));
+      pv[c0] = live ? x.x * sc : 0.f; pv[c0 + 1] = live ? x.y * sc : 0.f;
+      pv[c0 + 2] = live ? x.z * sc : 0.f; pv[c0 + 3] = live ? x.w * sc : 0.f;
+    }
+#pragma unroll
+    for (int c = 0; c < QC; ++c) {
+      const int qq = q0 + c;
+      const __nv_bfloat16 hi = __float2bfloat16_rn(pv[c]);
+      const uint32_t off_hi = (uint32_t)qq * 128u + ((((kk >> 3) ^ (uint32_t)(qq & 7)) << 4) | ((kk & 7u) << 1));
+      *reinterpret_cast<__nv_bfloat16*>(img + off_hi) = hi;
+      const __nv_bfloat16 lo = __float2bfloat16_rn(pv[c] - __bfloat162float(hi));
+      const uint32_t off_lo = (uint32_t)(R + qq) * 128u + ((((kk >> 3) ^ (uint32_t)((R + qq) & 7)) << 4) | ((kk & 7u) << 1));
+      *reinterpret_cast<__nv_bfloat16*>(img + off_lo) = lo;
+    }
+  }
+  if (2 * R < N2 && blockIdx.z == 0) {       // (N2 = 2 R for every rank offered; kept for the layout's sake)
+    for (int qq = 2 * R; qq < N2; ++qq)
+      *reinterpret_cast<__nv_bfloat16*>(img + (uint32_t)qq * 128u + ((((kk >> 3) ^ (uint32_t)(qq & 7)) << 4) | ((kk & 7u) << 1))) =
+          __float2bfloat16_rn(0.f);
+  }
+}
 
 template <int R>
 __global__ void __launch_bounds__(THREADS, 1)
@@ -299,6 +351,18 @@ grad_tc_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_constant__
       // ---- a tile's P operand: (scaled) P[row, :] as bf16 (head | remainder), K-major, 128-byte swizzle ----
       auto convert = [&](const TileIt& it) -> bool {
         const int blk_abs = it.b0 + it.blk;
+        if (a.pop) {       // the operand image exists in memory: one bulk copy instead of a conversion per tile
+          const int pb = ic % NPB;
+          if (!__all_sync(0xffffffffu, gemm_wait(bar_pempty(pb), ((ic / NPB) & 1) ^ 1, abort_flag, a.status))) return false;
+          if (tid == 0) {
+            ptx::mbar_arrive_expect_tx(bar_pfull(pb), C::P_BYTES);
+            bulk_load(s_pbuf(pb), a.pop + ((size_t)p * a.NB + blk_abs) * C::P_BYTES, C::P_BYTES, bar_pfull(pb));
+          } else {
+            ptx::mbar_arrive(bar_pfull(pb));
+          }
+          ++ic;
+          return true;
+        }
         const int nrows = a.blk_nrows[blk_abs], row0 = a.blk_row0[blk_abs];
         float pv[R];
         const bool live = trow < nrows;

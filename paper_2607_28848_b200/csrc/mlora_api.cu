@@ -22,7 +22,7 @@
 #include "simt.cuh"
 #include "skinny.cuh"
 #include "grad_tc.cuh"
-#include "vshrink_tc.cuh"
+#include "shrink_tc.cuh"
 #include "glue.cuh"
 #include "attention.cuh"
 #include "attention_tc.cuh"
@@ -65,6 +65,9 @@ struct mlora_ctx {
   float* ws_gpart = nullptr;         // partial gradient sums that several CTAs share: [sm_count][4][64 KiB] (the streaming kernel's
                                      // row-split groups use the first 128 KiB per SM, the tensor-core kernel's split strips all of it)
   int32_t* ws_gcounters = nullptr;   // [sm_count] arrival counters of those groups, zero between launches
+  uint8_t* ws_pop = nullptr;         // P operands of the tensor-core gradient kernel: [2][ws_pop_blocks][64 KiB]
+  int64_t ws_pop_blocks = 0;
+  float* ws_tc_part = nullptr;       // run sums of the tensor-core shrink: [ws_rows + 128 * sm_count][kMaxRank]
   int32_t* ws_tc_counters = nullptr; // [kTcCounters] counters of the tensor-core gradient kernel, zero between launches
   std::vector<void*> retired;        // workspaces replaced by larger ones: kept until the context is destroyed,
                                      // because a captured graph may still hold their addresses
@@ -87,10 +90,17 @@ struct mlora_ctx {
 };
 
 constexpr int kMaxKSplit = 16;
-// Ranks from which the tcgen05 gradient kernel is the default.  Measured on B200 (one launch, 4096 -> 14336, 1024-2048
-// fine-tuning rows): rank 8 20.9 vs 14.7 us for the mma.sync streaming kernel, rank 16 27.0 vs 20.8, rank 32 39.3 vs 39.3,
-// rank 64 43.4 vs 33.1, rank 128 70 vs 144 (two launches of the per-item kernel).
-constexpr int kTcGradMinRank = 128;
+// Ranks from which the tcgen05 gradient kernel (with its P operands made ahead by psplit_kernel) is the default.
+// Measured on B200 (both launches with their event pairs, 4096 -> 14336, 1024 fine-tuning rows), against the mma.sync
+// streaming kernel: rank 16 7 + 27 vs 21 us, rank 32 8 + 23 vs 29, rank 64 9 + 25 vs 33-50 (whole step 295 vs 315 us with
+// one adapter, 404 vs 410 with 256), rank 128 9 + 25 vs 144 (two launches of the per-item kernel).  Before the operands
+// were made ahead, every tile converted its own (rank 128: 7 us per tile, 56-70 us per launch).
+constexpr int kTcGradMinRank = 64;
+// Ranks from which the tcgen05 shrink (U = X A^T with the activation save, V = s dY B^T) is the default.  Measured on
+// B200 (main + finish launch with their event pairs, 2048 x 4096 forward / 1024 x 14336 backward): rank 128 19 + 12 and
+// 20 + 10 us vs 43 and 74 for the per-item kernel; rank 64 15 + 13 and 17 + 9 vs 31 and 37 for the streaming kernel;
+// rank 32 14 + 15 and 17 + 9 vs 20 and 25 (hence not the default there).
+constexpr int kTcShrinkMinRank = 64;
 
 enum { KIND_SHRINK = 0, KIND_GEMM_FWD = 1, KIND_GEMM_BWD = 2, KIND_GRAD = 3, KIND_SIMT = 4, KIND_ADAMW = 5, KIND_REDUCE = 6 };
 
@@ -133,6 +143,9 @@ struct DevRowSpace {
   const int32_t* item_nrows = nullptr;
   const int32_t* item_adapter = nullptr;
   const int32_t* item_desc = nullptr;
+  const int32_t* tcb_row0 = nullptr;
+  const int32_t* tcb_nrows = nullptr;
+  const int32_t* tcb_adapter = nullptr;
 };
 
 struct mlora_plan {
@@ -168,6 +181,7 @@ struct BlobBuilder {
 // Workspace for K-split products of small-batch GEMMs: allocated once per context, so that no
 // compute call allocates.  Problems whose partials do not fit run unsplit.
 constexpr size_t kSplitKBytes = 64u << 20;
+constexpr int64_t kPopMaxBlocks = 512;  // most 128-row blocks whose gradient operands are made ahead (64 MiB)
 constexpr int kTcCounters = 1 << 18;    // counter words of the tensor-core gradient kernel (1 MiB, allocated with the context)
 constexpr int kMaxDevices = 64;      // device ordinals a process may create contexts on
 // One-time kernel attributes (opt-in shared-memory size, resident cluster count) are cached per kernel
@@ -462,15 +476,15 @@ mlora_status_t launch_grad_stream2(mlora_ctx* ctx, const mlora_plan* p, const Gr
   return launch_grad_stream2_c<MB, false>(ctx, p, gb, ga_, n_slots, n_rows, st);
 }
 
-// V = s dY B^T on the tcgen05 kernel (the fine-tuning rows come as 128-row blocks of one adapter each).
+// U = X A^T (forward, with the activation save) or V = s dY B^T (backward) on the tcgen05 kernels: the rows come
+// as blocks of <= 128 consecutive rows of one adapter.  `fa` carries what the finish kernel writes.
 template <int R>
-mlora_status_t launch_vshrink_tc(mlora_ctx* ctx, const mlora_layer_t* L, const mlora_plan* p, const void* dY, int64_t lddy,
-                                 bool want_pbd, cudaStream_t st) {
-  using C = vtc::Cfg<R>;
-  const HostPlan& h = p->h;
+mlora_status_t launch_shrink_tc(mlora_ctx* ctx, const RowSpace& hs, const DevRowSpace& ds, const void* In, int64_t ld_in,
+                                int n_rows, int D, const void* P_all, int n_adapters, stc::FinArgs fa, cudaStream_t st) {
+  using C = stc::Cfg<R>;
   static bool attr_set_dev[kMaxDevices] = {};   // per instantiation and device
   bool& attr_set = attr_set_dev[ctx->device];
-  auto kern = vtc::vshrink_tc_kernel<R>;
+  auto kern = stc::shrink_tc_kernel<R>;
   {
     std::lock_guard<std::mutex> lock(g_attr_mutex);
     if (!attr_set) {
@@ -480,20 +494,50 @@ mlora_status_t launch_vshrink_tc(mlora_ctx* ctx, const mlora_layer_t* L, const m
   }
   CUtensorMap tQ, tB;
   mlora_status_t ms;
-  if ((ms = make_tmap_bf16_blocked(ctx, &tQ, dY, h.ft_rows, L->d_out, lddy, vtc::ROWS, C::CB)) != MLORA_OK) return ms;
-  if ((ms = make_tmap_bf16_blocked(ctx, &tB, L->B_all, (uint64_t)L->n_adapters * R, L->d_out, L->d_out, C::RP, C::CB)) != MLORA_OK) return ms;
-  vtc::Args a;
-  a.scale = L->scale; a.blk_row0 = p->blk_row0; a.blk_nrows = p->blk_nrows; a.row_adapter = p->bwd.row_adapter;
-  a.NB = (int)h.blk_row0.size(); a.NS = (L->d_out + C::COLS - 1) / C::COLS; a.D = L->d_out;
-  a.V_out = ctx->ws_p;
-  a.pbd = PbdArgs{want_pbd ? ctx->ws_pbd : nullptr, p->bwd.row_grp2, p->bwd.tile2_grp_off, nullptr, p->bwd.zero_rows2, 0};
-  a.part_ws = ctx->ws_gpart; a.counters = ctx->ws_tc_counters; a.status = ctx->status_dev;
+  if ((ms = make_tmap_bf16_blocked(ctx, &tQ, In, n_rows, D, ld_in, stc::ROWS, C::CB)) != MLORA_OK) return ms;
+  if ((ms = make_tmap_bf16_blocked(ctx, &tB, P_all, (uint64_t)n_adapters * R, D, D, C::RP, C::CB)) != MLORA_OK) return ms;
+  stc::Args a;
+  a.blk_row0 = ds.tcb_row0; a.blk_nrows = ds.tcb_nrows; a.blk_adapter = ds.tcb_adapter;
+  a.NB = (int)hs.tcb_row0.size(); a.NS = (D + C::COLS - 1) / C::COLS;
+  a.part_ws = ctx->ws_tc_part; a.status = ctx->status_dev;
   const int64_t tiles = (int64_t)a.NB * a.NS;
   const int grid = tiles < ctx->sm_count ? (int)tiles : ctx->sm_count;
   if (cancelled(ctx)) return MLORA_CANCELLED;
+  {
+    LaunchScope scope(ctx, st, KIND_SHRINK);
+    launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(stc::THREADS), C::SMEM_BYTES, st, tQ, tB, a);
+    if ((ms = scope.done()) != MLORA_OK) return ms;
+  }
+  fa.blk_row0 = a.blk_row0; fa.blk_nrows = a.blk_nrows; fa.blk_adapter = a.blk_adapter;
+  fa.NB = a.NB; fa.NS = a.NS; fa.G = grid; fa.part_ws = ctx->ws_tc_part;
+  const int zero_ctas = fa.pbd.pbd ? (fa.pbd.n_zero_rows + C::FIN_ROWS - 1) / C::FIN_ROWS : 0;
+  if (cancelled(ctx)) return MLORA_CANCELLED;
   LaunchScope scope(ctx, st, KIND_SHRINK);
-  launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(vtc::THREADS), C::SMEM_BYTES, st, tQ, tB, a);
+  launch_pdl(scope.slot < 0, stc::shrink_tc_finish_kernel<R>, dim3(a.NB + zero_ctas, stc::ROWS / C::FIN_ROWS), dim3(C::FIN_THREADS), 0,
+             st, fa);
   return scope.done();
+}
+
+// Can this row space run on the tensor-core shrink?  Blocks that are nearly empty waste the 128-row MMA: with
+// fewer than four rows per block on average the kernels that gather rows by adapter are the better choice.
+inline bool shrink_tc_fits(const mlora_ctx* ctx, const RowSpace& hs, int n_rows, int D) {
+  const int64_t NB = (int64_t)hs.tcb_row0.size();
+  if (NB < 1 || D % 64 != 0 || n_rows > ctx->ws_rows || !ctx->ws_tc_part) return false;
+  if (4 * NB > (int64_t)hs.item_rows.size()) return false;
+  return NB * ((D + 127) / 128) < (1 << 30) && NB + (int64_t)hs.zero_rows2.size() / 8 + 1 < (1 << 30);
+}
+
+inline mlora_status_t launch_shrink_tc_any(mlora_ctx* ctx, int rank, const RowSpace& hs, const DevRowSpace& ds, const void* In,
+                                           int64_t ld_in, int n_rows, int D, const void* P_all, int n_adapters,
+                                           const stc::FinArgs& fa, cudaStream_t st) {
+  switch (rank) {
+    case 8: return launch_shrink_tc<8>(ctx, hs, ds, In, ld_in, n_rows, D, P_all, n_adapters, fa, st);
+    case 16: return launch_shrink_tc<16>(ctx, hs, ds, In, ld_in, n_rows, D, P_all, n_adapters, fa, st);
+    case 32: return launch_shrink_tc<32>(ctx, hs, ds, In, ld_in, n_rows, D, P_all, n_adapters, fa, st);
+    case 64: return launch_shrink_tc<64>(ctx, hs, ds, In, ld_in, n_rows, D, P_all, n_adapters, fa, st);
+    case 128: return launch_shrink_tc<128>(ctx, hs, ds, In, ld_in, n_rows, D, P_all, n_adapters, fa, st);
+    default: return MLORA_ERR_UNSUPPORTED;
+  }
 }
 
 // Both gradients on the tcgen05 kernel: can this call use it?  (A slot without rows gets its zeros from the
@@ -564,6 +608,14 @@ mlora_status_t launch_grad_tc(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
     most_snapped = snapped > most_snapped ? snapped : most_snapped;
   }
   a.snap = (8 * most_snapped <= 9 * most_plain) ? 1 : 0;
+  a.pop = nullptr;
+  if (a.NB <= ctx->ws_pop_blocks && ctx->ws_pop) {     // both problems' operands once per block, ahead of the kernel
+    if (cancelled(ctx)) return MLORA_CANCELLED;
+    LaunchScope scope(ctx, st, KIND_GRAD);
+    launch_pdl(scope.slot < 0, gtc::psplit_kernel<R>, dim3(a.NB, 2, R / gtc::psplit_cols(R)), dim3(128), 0, st, a, ctx->ws_pop);
+    if ((ms = scope.done()) != MLORA_OK) return ms;
+    a.pop = ctx->ws_pop;
+  }
   if (cancelled(ctx)) return MLORA_CANCELLED;
   LaunchScope scope(ctx, st, KIND_GRAD);
   launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(gtc::THREADS), C::SMEM_BYTES, st, tQ0, tQ1, a);
@@ -748,6 +800,9 @@ void balanced_units(mlora_ctx* ctx, const RowSpace& hs, const DevRowSpace& ds, i
     e->n_ntiles = g.n_ntiles; e->kblocks = kblocks; e->rank = R; e->pairs = pairs; e->n_whole = g.n_whole;
     e->n_tail = g.n_tail; e->split_k = g.split_k; e->group_m = g.group_m;
     e->use = 100 * lpt_max < 97 * rr_max;
+    if (std::getenv("MLORA_DEBUG"))
+      std::fprintf(stderr, "mlora: unit list for %d x %d tiles, %d K-blocks, rank %d: round robin %lld, by cost %lld blocks -> %s\n",
+                   g.n_mtiles, g.n_ntiles, kblocks, R, (long long)rr_max, (long long)lpt_max, e->use ? "list" : "round robin");
     slot = sc->n;
     if (e->use) {
       e->host.assign(pairs + 1, 0);            // offsets (into this same array), then each pair's units in tile order
@@ -1124,7 +1179,7 @@ void mlora_destroy(mlora_ctx* c) {
 
 namespace {
 
-constexpr int kPlanTables = 37;
+constexpr int kPlanTables = 43;
 
 // All device tables of a plan, packed; o[] receives each table's offset in 32-bit words.
 void pack_plan(const HostPlan& h, BlobBuilder& b, size_t* o) {
@@ -1137,6 +1192,7 @@ void pack_plan(const HostPlan& h, BlobBuilder& b, size_t* o) {
     o[n++] = b.add(rs[i]->zero_rows2);
     o[n++] = b.add(rs[i]->item_save); o[n++] = b.add(rs[i]->item_start); o[n++] = b.add(rs[i]->item_desc);
     o[n++] = b.add(rs[i]->item_nrows); o[n++] = b.add(rs[i]->item_adapter);
+    o[n++] = b.add(rs[i]->tcb_row0); o[n++] = b.add(rs[i]->tcb_nrows); o[n++] = b.add(rs[i]->tcb_adapter);
   }
   o[n++] = b.add(h.slot_chunk_off); o[n++] = b.add(h.chunk_row0); o[n++] = b.add(h.chunk_nrows);
   o[n++] = b.add(h.ft_adapters);
@@ -1184,6 +1240,7 @@ void bind_plan(mlora_plan* p, const size_t* o) {
     ds[i]->zero_rows2 = p->blob + o[n++];
     ds[i]->item_save = p->blob + o[n++]; ds[i]->item_start = p->blob + o[n++]; ds[i]->item_desc = p->blob + o[n++];
     ds[i]->item_nrows = p->blob + o[n++]; ds[i]->item_adapter = p->blob + o[n++];
+    ds[i]->tcb_row0 = p->blob + o[n++]; ds[i]->tcb_nrows = p->blob + o[n++]; ds[i]->tcb_adapter = p->blob + o[n++];
   }
   p->bwd.row_save = nullptr;       // the compact space has no save offsets
   p->slot_chunk_off = p->blob + o[n++]; p->chunk_row0 = p->blob + o[n++]; p->chunk_nrows = p->blob + o[n++];
@@ -1211,6 +1268,8 @@ mlora_status_t grow_workspaces(mlora_ctx* ctx, const HostPlan& h, int32_t n_rows
   if (n_rows > ctx->ws_rows) {     // the rank-r workspace
     const int64_t rows = grown(n_rows, ctx->ws_rows);
     if ((s = replace_workspace(ctx, (void**)&ctx->ws_p, (size_t)rows * kMaxRank * sizeof(float), false)) != MLORA_OK) return s;
+    if ((s = replace_workspace(ctx, (void**)&ctx->ws_tc_part, (size_t)(rows + 128 * ctx->sm_count) * kMaxRank * sizeof(float),
+                               false)) != MLORA_OK) return s;
     ctx->ws_rows = rows;
   }
   const int64_t items = h.fwd.n_items() > h.bwd.n_items() ? h.fwd.n_items() : h.bwd.n_items();
@@ -1221,6 +1280,12 @@ mlora_status_t grow_workspaces(mlora_ctx* ctx, const HostPlan& h, int32_t n_rows
         (s = replace_workspace(ctx, (void**)&ctx->ws_counters, (size_t)(2 * it + 1) * sizeof(int32_t), true)) != MLORA_OK)
       return s;
     ctx->ws_partial_items = part_items; ctx->ws_counter_items = it;
+  }
+  const int64_t blocks = (int64_t)h.blk_row0.size();
+  if (blocks > ctx->ws_pop_blocks && blocks <= kPopMaxBlocks) {      // beyond that the gradient kernel converts per tile
+    const int64_t nb = grown(blocks, ctx->ws_pop_blocks) < kPopMaxBlocks ? grown(blocks, ctx->ws_pop_blocks) : kPopMaxBlocks;
+    if ((s = replace_workspace(ctx, (void**)&ctx->ws_pop, (size_t)nb * 2 * 65536, false)) != MLORA_OK) return s;
+    ctx->ws_pop_blocks = nb;
   }
   const int64_t groups = (int64_t)(h.fwd.grp2_adapter.size() > h.bwd.grp2_adapter.size() ? h.fwd.grp2_adapter.size()
                                                                                         : h.bwd.grp2_adapter.size());
@@ -1382,8 +1447,19 @@ mlora_status_t mlora_mixed_forward(mlora_ctx* ctx, const mlora_layer_t* L, const
                    p->fwd.zero_rows2, (int32_t)h.fwd.zero_rows2.size()};
   sa.x_save = (__nv_bfloat16*)x_save; sa.u_save = u_save; sa.save_base = save_row_base;
   sa.save_cap = save_capacity_rows;
-  if ((s = launch_shrink(ctx, L->rank, sa, h.fwd.n_items(), p->fwd.item_desc, h.n_rows, L->n_adapters, st)) != MLORA_OK)
-    return s;
+  // rank >= kTcShrinkMinRank (every rank under kernel variant 6): the tcgen05 shrink and its finish kernel
+  const bool tc_shrink = ctx->shrink_path == 0 && ctx->drop.thr == 0 && !h.fwd.tcb_row0.empty() &&
+                         (L->rank >= kTcShrinkMinRank || ctx->grad_mode == 2) && shrink_tc_fits(ctx, h.fwd, h.n_rows, L->d_in);
+  if (tc_shrink) {
+    stc::FinArgs fa = {};
+    fa.scale = nullptr; fa.Out = ctx->ws_p; fa.pbd = sa.pbd;
+    fa.row_save = h.ft_rows > 0 ? p->fwd.row_save : nullptr; fa.u_save = u_save;
+    fa.X = (const __nv_bfloat16*)X; fa.ldx = ldx; fa.x_save = (__nv_bfloat16*)x_save; fa.save_base = save_row_base; fa.D = L->d_in;
+    s = launch_shrink_tc_any(ctx, L->rank, h.fwd, p->fwd, X, ldx, h.n_rows, L->d_in, L->A_all, L->n_adapters, fa, st);
+  } else {
+    s = launch_shrink(ctx, L->rank, sa, h.fwd.n_items(), p->fwd.item_desc, h.n_rows, L->n_adapters, st);
+  }
+  if (s != MLORA_OK) return s;
   return gemm_bf16<false>(ctx, L, h.fwd, p->fwd, X, ldx, Y, ldy, L->B_all, ctx->ws_p, L->scale, h.n_rows, L->d_out,
                           L->d_in, st);
 }
@@ -1420,19 +1496,13 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   sa.pbd = PbdArgs{(ctx->gemm_pairs && dX && !dropping) ? ctx->ws_pbd : nullptr, p->bwd.row_grp2, p->bwd.tile2_grp_off, nullptr,
                    p->bwd.zero_rows2, (int32_t)h.bwd.zero_rows2.size()};
   sa.item_adapter = p->bwd.item_adapter; sa.item_save = nullptr; sa.x_save = nullptr; sa.u_save = nullptr; sa.save_base = 0; sa.save_cap = 0;
-  // V from the streaming shrink kernel; the tcgen05 V kernel under kernel variant 6 (measured on B200, one launch with
-  // its events: 31.1 vs 28.9 us on 2048 x 14336 rows of dY at rank 16, 22.9 vs 16.8 us on 2048 x 4096, 37.2 vs 30 us at
-  // rank 32 on 2048 x 13824 - the mma.sync kernel is the faster one at every size tried)
-  const bool tc_v = ctx->shrink_path == 0 && ctx->grad_mode == 2 && h.bwd.zero_rows2.empty() &&
-                    (int64_t)h.blk_row0.size() + 1 <= kTcCounters && h.ft_rows > 0;
+  // V on the tcgen05 shrink from rank kTcShrinkMinRank (every rank under kernel variant 6), else on the mma.sync kernels
+  const bool tc_v = ctx->shrink_path == 0 && !dropping && (L->rank >= kTcShrinkMinRank || ctx->grad_mode == 2) &&
+                    shrink_tc_fits(ctx, h.bwd, h.ft_rows, L->d_out);
   if (tc_v) {
-    switch (L->rank) {
-      case 8: s = launch_vshrink_tc<8>(ctx, L, p, dY, lddy, sa.pbd.pbd != nullptr, st); break;
-      case 16: s = launch_vshrink_tc<16>(ctx, L, p, dY, lddy, sa.pbd.pbd != nullptr, st); break;
-      case 32: s = launch_vshrink_tc<32>(ctx, L, p, dY, lddy, sa.pbd.pbd != nullptr, st); break;
-      case 64: s = launch_vshrink_tc<64>(ctx, L, p, dY, lddy, sa.pbd.pbd != nullptr, st); break;
-      default: s = launch_vshrink_tc<128>(ctx, L, p, dY, lddy, sa.pbd.pbd != nullptr, st); break;
-    }
+    stc::FinArgs fa = {};
+    fa.scale = L->scale; fa.Out = ctx->ws_p; fa.pbd = sa.pbd;
+    s = launch_shrink_tc_any(ctx, L->rank, h.bwd, p->bwd, dY, lddy, h.ft_rows, L->d_out, L->B_all, L->n_adapters, fa, st);
   } else {
     s = launch_shrink(ctx, L->rank, sa, h.bwd.n_items(), p->bwd.item_desc, h.ft_rows, L->n_adapters, st);
   }

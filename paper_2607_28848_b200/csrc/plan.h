@@ -42,6 +42,8 @@ struct RowSpace {
   // item's rows are consecutive rows of the batch; bit 1: additionally the item is full
   // (kItemRows rows) and its save offsets are consecutive, so its rows can be saved as one block.
   std::vector<int32_t> item_desc;
+  // Blocks for the tensor-core shrink: runs of <= kTileRows consecutive rows that share one adapter.
+  std::vector<int32_t> tcb_row0, tcb_nrows, tcb_adapter;
   int32_t n_tiles() const { return (n_rows + kTileRows - 1) / kTileRows; }
   int32_t n_items() const { return (int32_t)item_start.size(); }
 };
@@ -92,6 +94,17 @@ inline void build_tiles_and_items(RowSpace& rs) {
   for (int32_t t = 0; t < n; ++t) {
     const int32_t tile = t / kPairTileRows;
     if (rs.row_adapter[t] < 0 && rs.tile2_grp_off[tile + 1] > rs.tile2_grp_off[tile]) rs.zero_rows2.push_back(t);
+  }
+  rs.tcb_row0.clear(); rs.tcb_nrows.clear(); rs.tcb_adapter.clear();
+  for (int32_t t = 0; t < n; ++t) {
+    const int32_t a = rs.row_adapter[t];
+    if (a < 0) continue;
+    if (!rs.tcb_row0.empty() && rs.tcb_adapter.back() == a && rs.tcb_row0.back() + rs.tcb_nrows.back() == t &&
+        rs.tcb_nrows.back() < kTileRows) {
+      rs.tcb_nrows.back()++;
+    } else {
+      rs.tcb_row0.push_back(t); rs.tcb_nrows.push_back(1); rs.tcb_adapter.push_back(a);
+    }
   }
   rs.item_rows.clear(); rs.item_start.clear(); rs.item_nrows.clear(); rs.item_adapter.clear(); rs.item_desc.clear();
   int32_t max_adapter = -1;
