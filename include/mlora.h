@@ -216,9 +216,11 @@ mlora_status_t mlora_set_cancel_flag(mlora_ctx* ctx, const volatile int32_t* hos
  * keep their form.  The forward and the backward of one batch must run under the same (p, seed);
  * the caller changes the seed from step to step and from layer to layer.  A captured graph keeps
  * the values it was captured with.
- * Supported for fp32 layers and for bf16 layers of rank <= 64 on the default kernel path;
- * otherwise the compute call returns MLORA_ERR_UNSUPPORTED.  With dropout on, the low-rank part
- * of dX is added by one extra elementwise kernel after the base product.
+ * Supported for fp32 layers and for bf16 layers of every rank on the default kernel path (the
+ * mma.sync kernels mask the rows as they read them: the streaming kernels up to rank 64, the
+ * per-item kernels at rank 128); under kernel variant 2 only at rank 128, otherwise the compute
+ * call returns MLORA_ERR_UNSUPPORTED.  With dropout on, the low-rank part of dX is added by one
+ * extra elementwise kernel after the base product.
  * Errors: MLORA_ERR_INVALID_ARG (NULL context, p outside [0, 1)). */
 mlora_status_t mlora_set_dropout(mlora_ctx* ctx, double p, uint64_t seed);
 

@@ -50,8 +50,9 @@ Python on tiny shapes, a hand-computed worked example, the B = 0 and s-linearity
 invariants, the merged-weight identity W_eff of Section 2.2 per segment, invariance
 under table reordering / segment splitting / the is_finetune flag, and central finite
 differences for every gradient; for the variants, the published SplitMix64 test vector, the
-p = 0 and keep-frequency checks, finite differences through the masked forward, and the
-zero-padding identity against per-adapter matrices of their own ranks.  No function here is
+p = 0 and keep-frequency checks, finite differences through the masked forward, the
+zero-padding identity against per-adapter matrices of their own ranks, and central finite
+differences of ``forward_ragged`` for every output of ``backward_ragged``.  No function here is
 "parity unpinned".
 """
 from __future__ import annotations
@@ -300,6 +301,31 @@ def backward(dY, W, A_all, B_all, scale, segments, x_save, u_save, n_rows: Optio
                 dA[g] += np.outer(V[m], x_save[m] * k)     # the branch saw x * k
                 dX[m] = W @ dY[m] + (V[m] @ A_all[a]) * k
     return {"dA": dA, "dB": dB, "dX": dX, "V": V, "ft_adapters": ft_adapters}
+
+
+def backward_ragged(dY, W, A_list, B_list, scale, segments, x_save, n_rows: int):
+    """Gradients when adapter a has its own rank r_a (Section 5 trains adapters of different ranks side by side):
+    the same chain rule as ``backward`` with each adapter's own matrices, nothing padded.  ``u`` is recomputed
+    from the saved input (u = A_a x), since saved rows of different adapters would have different widths.
+    Returns ``dA`` and ``dB`` as lists (slot g: [r_a, d_in] and [r_a, d_out]), ``dX`` [ft_rows, d_in] and
+    ``ft_adapters``."""
+    dY, W, scale, x_save = _f64(dY), _f64(W), _f64(scale), _f64(x_save)
+    _, ft_segments, ft_rows, ft_adapters = route(segments, n_rows, len(A_list))
+    if dY.shape[0] != ft_rows:
+        raise SegmentError("dY must have one row per fine-tuning row")
+    dA = [np.zeros_like(_f64(A_list[a])) for a in ft_adapters]
+    dB = [np.zeros_like(_f64(B_list[a])) for a in ft_adapters]
+    dX = np.zeros((ft_rows, W.shape[0]))
+    for _start, length, a, off in ft_segments:
+        g = ft_adapters.index(a)
+        A, B, s = _f64(A_list[a]), _f64(B_list[a]), scale[a]
+        for m in range(off, off + length):
+            u = A @ x_save[m]                              # u = x A_a^T
+            v = s * (B @ dY[m])                            # v = s dy B_a^T
+            dB[g] += s * np.outer(u, dY[m])
+            dA[g] += np.outer(v, x_save[m])
+            dX[m] = W @ dY[m] + v @ A
+    return {"dA": dA, "dB": dB, "dX": dX, "ft_adapters": ft_adapters}
 
 
 def backward_blocked(dY, W, A_all, B_all, scale, segments, x_save, u_save,

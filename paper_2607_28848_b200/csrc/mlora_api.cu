@@ -401,7 +401,14 @@ mlora_status_t launch_shrink(mlora_ctx* ctx, int R, ShrinkArgs a, int n_items, c
     case 16: launch_shrink_rb<2, 2, 8, 2>(scope.slot < 0, a, n_items, ksplit, st); break;
     case 32: launch_shrink_rb<4, 2, 8, 2>(scope.slot < 0, a, n_items, ksplit, st); break;
     case 64: launch_shrink_rb<8, 2, 4, 2>(scope.slot < 0, a, n_items, ksplit, st); break;
-    case 128: launch_shrink_rb<16, 1, 4, 2>(scope.slot < 0, a, n_items, ksplit, st); break;
+    case 128:
+      if (ctx->drop.thr != 0 && a.item_save) {      // forward with dropout: the mask acts on the rows as they are read
+        a.drop = ctx->drop;
+        launch_pdl(scope.slot < 0, shrink_kernel<16, 1, 4, 2, true>, dim3(n_items, ksplit, kItemRows / 16), dim3(4 * 32), 0, st, a);
+      } else {
+        launch_shrink_rb<16, 1, 4, 2>(scope.slot < 0, a, n_items, ksplit, st);
+      }
+      break;
     default: return MLORA_ERR_UNSUPPORTED;
   }
   return scope.done();
@@ -632,7 +639,8 @@ mlora_status_t launch_grad(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& 
   {
     std::lock_guard<std::mutex> lock(g_attr_mutex);
     if (!attr_set) {
-      if (cudaFuncSetAttribute(grad_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2) != cudaSuccess)
+      if (cudaFuncSetAttribute(grad_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2) != cudaSuccess ||
+          cudaFuncSetAttribute(grad_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2) != cudaSuccess)
         return MLORA_ERR_CUDA;
       attr_set = true;
     }
@@ -641,7 +649,10 @@ mlora_status_t launch_grad(mlora_ctx* ctx, const mlora_plan* p, const GradArgs& 
   if (a.R <= 16) {
     launch_pdl(scope.slot < 0, grad_kernel<1>, dim3(a.D / 64, n_slots, 1), dim3(GRAD_THREADS), smem1, st, a);
   } else {
-    launch_pdl(scope.slot < 0, grad_kernel<2>, dim3(a.D / 64, n_slots, (a.R + 31) / 32), dim3(GRAD_THREADS), smem2, st, a);
+    if (a.drop.thr != 0)
+      launch_pdl(scope.slot < 0, grad_kernel<2, true>, dim3(a.D / 64, n_slots, (a.R + 31) / 32), dim3(GRAD_THREADS), smem2, st, a);
+    else
+      launch_pdl(scope.slot < 0, grad_kernel<2>, dim3(a.D / 64, n_slots, (a.R + 31) / 32), dim3(GRAD_THREADS), smem2, st, a);
   }
   return scope.done();
 }
@@ -1437,7 +1448,7 @@ mlora_status_t mlora_mixed_forward(mlora_ctx* ctx, const mlora_layer_t* L, const
   if (ctx->gemm_path == 1)
     return forward_simt<__nv_bfloat16>(ctx, L, p, X, ldx, Y, ldy, x_save, u_save, save_row_base, st);
 
-  if (ctx->drop.thr != 0 && h.ft_rows > 0 && (ctx->shrink_path != 0 || L->rank > 64)) return MLORA_ERR_UNSUPPORTED;
+  if (ctx->drop.thr != 0 && h.ft_rows > 0 && ctx->shrink_path != 0 && L->rank <= 64) return MLORA_ERR_UNSUPPORTED;
   ShrinkArgs sa;
   sa.In = (const __nv_bfloat16*)X; sa.ld_in = ldx; sa.D = L->d_in;
   sa.P_all = (const __nv_bfloat16*)L->A_all; sa.scale = nullptr; sa.Out = ctx->ws_p;
@@ -1488,7 +1499,7 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
 
   const int n_slots = (int)h.ft_adapters.size();
   const bool dropping = ctx->drop.thr != 0;
-  if (dropping && (ctx->shrink_path != 0 || L->rank > 64)) return MLORA_ERR_UNSUPPORTED;
+  if (dropping && ctx->shrink_path != 0 && L->rank <= 64) return MLORA_ERR_UNSUPPORTED;
   ShrinkArgs sa;                     // V = s dY B^T
   sa.In = (const __nv_bfloat16*)dY; sa.ld_in = lddy; sa.D = L->d_out;
   sa.P_all = (const __nv_bfloat16*)L->B_all; sa.scale = L->scale; sa.Out = ctx->ws_p;
@@ -1497,7 +1508,7 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
                    p->bwd.zero_rows2, (int32_t)h.bwd.zero_rows2.size()};
   sa.item_adapter = p->bwd.item_adapter; sa.item_save = nullptr; sa.x_save = nullptr; sa.u_save = nullptr; sa.save_base = 0; sa.save_cap = 0;
   // V on the tcgen05 shrink from rank kTcShrinkMinRank (every rank under kernel variant 6), else on the mma.sync kernels
-  const bool tc_v = ctx->shrink_path == 0 && !dropping && (L->rank >= kTcShrinkMinRank || ctx->grad_mode == 2) &&
+  const bool tc_v = ctx->shrink_path == 0 && (L->rank >= kTcShrinkMinRank || ctx->grad_mode == 2) &&
                     shrink_tc_fits(ctx, h.bwd, h.ft_rows, L->d_out);
   if (tc_v) {
     stc::FinArgs fa = {};
@@ -1554,9 +1565,16 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   }
   if ((s = launch_grad(ctx, p, ga, n_slots, h.ft_rows, st)) != MLORA_OK) return s;
   ga.P = ctx->ws_p; ga.scale = nullptr; ga.Q = (const __nv_bfloat16*)x_save; ga.ldq = L->d_in; ga.D = L->d_in;
-  ga.G = dA;                         // dA = V^T X
+  ga.G = dA;                         // dA = V^T X (with dropout: the kept elements of X, V counted 1 / (1 - p) times)
+  if (dropping) ga.drop = ctx->drop;
   if ((s = launch_grad(ctx, p, ga, n_slots, h.ft_rows, st)) != MLORA_OK) return s;
   if (!dX) return MLORA_OK;
+  if (dropping) {   // the mask acts on the low-rank term per element: base product first, then the masked expand
+    if ((s = gemm_bf16<true>(ctx, L, h.bwd, p->bwd, dY, lddy, dX, lddx, L->A_all, ctx->ws_p, nullptr, h.ft_rows, L->d_in,
+                             L->d_out, st, false)) != MLORA_OK)
+      return s;
+    return launch_expand_mask(ctx, L, p->bwd, dX, lddx, h.ft_rows, st);
+  }
   return gemm_bf16<true>(ctx, L, h.bwd, p->bwd, dY, lddy, dX, lddx, L->A_all, ctx->ws_p, nullptr, h.ft_rows, L->d_in,
                          L->d_out, st);
 }

@@ -86,6 +86,7 @@ struct ShrinkArgs {
   float* partial;              // [n_items * gridDim.z * gridDim.y, MT * 16, R] scratch
   int32_t* counters;           // [n_items * gridDim.z], zero between launches
   PbdArgs pbd;                 // optional block-diagonal copy of the result for the two-SM GEMM
+  DropArgs drop = {0, 0, 1.0f}; // per-item kernel with DROP: dropout of the fine-tuning rows' branch input
 };
 
 // One CTA per item; its warps take the 64-wide K blocks round-robin and reduce through shared
@@ -97,7 +98,7 @@ struct ShrinkArgs {
 // With gridDim.y > 1 the K range of an item is split over that many CTAs; each leaves its partial
 // result in scratch and the CTA that finishes last adds them up in a fixed order, so the result
 // does not depend on which CTA that was.
-template <int RB, int MT, int WARPS, int MIN_CTAS>
+template <int RB, int MT, int WARPS, int MIN_CTAS, bool DROP = false>
 __global__ void __launch_bounds__(WARPS * 32, MIN_CTAS)
 shrink_kernel(const ShrinkArgs a) {
   constexpr int R = RB * 8;
@@ -119,15 +120,17 @@ shrink_kernel(const ShrinkArgs a) {
   // this thread's rows: local index g + 8 j, j < 2 MT
   const __nv_bfloat16* xp[2 * MT];
   __nv_bfloat16* sp[2 * MT];
+  int msave[2 * MT];             // DROP: save-order place of the row (the mask's row counter), -1: not a fine-tuning row
 #pragma unroll
   for (int j = 0; j < 2 * MT; ++j) {
     const int rl = g + 8 * j;
-    xp[j] = nullptr; sp[j] = nullptr;
+    xp[j] = nullptr; sp[j] = nullptr; msave[j] = -1;
     if (rl < nrows) {
       const int row = rows[rl];
       xp[j] = a.In + (size_t)row * a.ld_in + 16 * c;
       const int sv = (saves && a.x_save) ? saves[rl] : -1;
       if (sv >= 0) sp[j] = a.x_save + (size_t)(a.save_base + sv) * a.D + 16 * c;
+      if (DROP && saves) msave[j] = saves[rl];
     }
   }
   const __nv_bfloat16* p0 = a.P_all + ((size_t)adapter * R + g) * a.D + 16 * c;
@@ -157,6 +160,19 @@ shrink_kernel(const ShrinkArgs a) {
       x[j][0] = zero4; x[j][1] = zero4;
       if (xp[j]) { x[j][0] = ptx::ldg_nc_v4(xp[j] + ko); x[j][1] = ptx::ldg_nc_v4(xp[j] + ko + 8); }
     }
+    if (DROP) {      // the saved copy keeps the row as it is, the product does not
+#pragma unroll
+      for (int j = 0; j < 2 * MT; ++j) {
+        if (sp[j]) {
+          *reinterpret_cast<uint4*>(sp[j] + ko) = x[j][0];
+          *reinterpret_cast<uint4*>(sp[j] + ko + 8) = x[j][1];
+        }
+        if (msave[j] >= 0) {
+          drop_mask8(a.drop, (uint32_t)msave[j], (uint32_t)(ko + 16 * c), x[j][0]);
+          drop_mask8(a.drop, (uint32_t)msave[j], (uint32_t)(ko + 16 * c + 8), x[j][1]);
+        }
+      }
+    }
 #pragma unroll
     for (int nb0 = 0; nb0 < RB; nb0 += NBG) {
       uint4 pa[NBG], pb[NBG];
@@ -184,7 +200,7 @@ shrink_kernel(const ShrinkArgs a) {
     // activation save: the rows of In pass through registers exactly once
 #pragma unroll
     for (int j = 0; j < 2 * MT; ++j)
-      if (sp[j]) {
+      if (!DROP && sp[j]) {
         *reinterpret_cast<uint4*>(sp[j] + ko) = x[j][0];
         *reinterpret_cast<uint4*>(sp[j] + ko + 8) = x[j][1];
       }
@@ -229,11 +245,10 @@ shrink_kernel(const ShrinkArgs a) {
       for (int w = 0; w < WARPS; ++w) u += red[w][r][q];     // fixed order
     }
     const int row = rows[r];
+    const int sv = saves ? saves[r] : -1;
+    if (DROP && sv >= 0) u *= a.drop.keep_scale;
     a.Out[(size_t)row * R + q] = u * sc;
-    if (a.u_save && saves) {
-      const int sv = saves[r];
-      if (sv >= 0) a.u_save[(size_t)(a.save_base + sv) * R + q] = u;
-    }
+    if (a.u_save && sv >= 0) a.u_save[(size_t)(a.save_base + sv) * R + q] = u;
   }
   if (ksplit > 1 && threadIdx.x == 0) a.counters[item] = 0;     // ready for the next launch
   if (a.pbd.pbd) {
@@ -674,6 +689,7 @@ struct GradArgs {
   const int32_t* chunk_nrows;
   const int32_t* slot_adapter;
   int32_t accumulate;
+  DropArgs drop = {0, 0, 1.0f}; // per-item kernel with DROP (dA): elements of Q kept or dropped, P counts keep_scale
 };
 
 // grid = (D / 64, n_slots, ceil(R / (16 MB))).  A CTA owns a 64-column strip of one slot's
@@ -681,7 +697,7 @@ struct GradArgs {
 // accumulating G^T-style with the rows as the MMA's contraction index, and are summed in a fixed
 // order, so the result does not depend on scheduling.  P is split into a bf16 head and a bf16
 // remainder (two MMAs) to keep ~16 bits of its mantissa.
-template <int MB>
+template <int MB, bool DROP = false>
 __global__ void __launch_bounds__(GRAD_THREADS, MB == 1 ? 2 : 1)
 grad_kernel(const GradArgs a) {
   extern __shared__ float grad_smem[];
@@ -703,7 +719,7 @@ grad_kernel(const GradArgs a) {
   const int ch0 = a.slot_chunk_off[slot], ch1 = a.slot_chunk_off[slot + 1];
   ptx::grid_dependency_wait();       // only plan tables were read so far
   ptx::grid_launch_dependents();
-  const float sc = a.scale ? a.scale[slot_ad] : 1.0f;
+  const float sc = (a.scale ? a.scale[slot_ad] : 1.0f) * (DROP ? a.drop.keep_scale : 1.0f);
   const uint4 zero4 = make_uint4(0, 0, 0, 0);
   const int tr[4] = {2 * c, 2 * c + 1, 2 * c + 8, 2 * c + 9};
   // Two-deep register pipeline: the loads of chunk i+1 (4 rows of Q, 8 values of P per rank
@@ -712,8 +728,10 @@ grad_kernel(const GradArgs a) {
   auto load_chunk = [&](int ch, ChunkRegs& r) {
     const int row0 = a.chunk_row0[ch], nrows = a.chunk_nrows[ch];
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < 4; ++i) {
       r.q[i] = tr[i] < nrows ? ptx::ldg_nc_v4(a.Q + (size_t)(row0 + tr[i]) * a.ldq + j0 + 8 * g) : zero4;
+      if (DROP && tr[i] < nrows) drop_mask8(a.drop, (uint32_t)(row0 + tr[i]), (uint32_t)(j0 + 8 * g), r.q[i]);   // compact row = place in save order
+    }
 #pragma unroll
     for (int m = 0; m < MB; ++m)
 #pragma unroll

@@ -52,8 +52,10 @@ def check_dropout(sess, w, t, p, seed, path=0, blocked=False, base=0, cap=None):
         run.close()
 
 
-@pytest.mark.parametrize("rank", [8, 16, 32, 64])
-def test_dropout_streaming_kernels(sess, rank):
+@pytest.mark.parametrize("rank", [8, 16, 32, 64, 128])
+def test_dropout_every_rank(sess, rank):
+    """Ranks up to 64: the streaming kernels mask the rows as they pass; rank 128: the per-item kernels do, V comes
+    from the tcgen05 shrink (no mask enters it), and the input gradient is the base product plus the masked expand."""
     # ragged table: gathered single rows, partial items, fine-tuning segments of every length
     w = synth.random_workload(40 + rank, 512, 384, rank, 5, 700, max_seg=150, p_finetune=0.45)
     check_dropout(sess, w, synth.make_tensors(w), 0.3, 2 ** 40 + rank)
@@ -115,10 +117,12 @@ def test_dropout_mask_bit_exact(sess):
         run.close()
 
 
-def test_dropout_large_rank_is_refused(sess):
-    w = synth.random_workload(79, 256, 256, 128, 3, 200, p_finetune=0.5)
+def test_dropout_refusals(sess):
+    """The per-item kernels of kernel variant 2 carry the mask only at rank 128; a rate of 1 is no rate."""
+    w = synth.random_workload(79, 256, 256, 16, 3, 200, p_finetune=0.5)
     t = synth.make_tensors(w)
     mb.mlora_set_dropout(sess.ctx, 0.1, 1)
+    mb.mlora_set_gemm_path(sess.ctx, 2)
     run = LayerRun(sess, w.dtype, t, w.segments, w.n_rows)
     try:
         with pytest.raises(mb.MloraError) as e:
@@ -128,7 +132,15 @@ def test_dropout_large_rank_is_refused(sess):
             mb.mlora_set_dropout(sess.ctx, 1.0, 1)
     finally:
         mb.mlora_set_dropout(sess.ctx, 0.0, 0)
+        mb.mlora_set_gemm_path(sess.ctx, 0)
         run.close()
+
+
+def test_dropout_rank_128_llama_projection(sess):
+    """4096 -> 4096 at rank 128, 1600 rows with 2 x 256 fine-tuning rows, p = 0.05, against the blocked oracle."""
+    w0 = synth.cfg2_single_projection()
+    w = synth.Workload("cfg2_rank128", w0.d_in, w0.d_out, 128, w0.n_adapters, "bf16", w0.n_rows, w0.segments, seed=31)
+    check_dropout(sess, w, synth.make_tensors(w), 0.05, 777, blocked=True)
 
 
 def test_dropout_llama_projection_sampled(sess):
@@ -157,7 +169,14 @@ def test_different_ranks_through_zero_padding(sess):
         ref = orc.forward_ragged(t["X"], t["W"], A_list, B_list, t["scale"], w.segments)
         assert_close("Y", run.host(run.Y), ref, TOL["bf16"])
         dA, dB = run.host(run.dA), run.host(run.dB)
-        for g, a in enumerate(run.slots):                  # gradients of the padding rows are exactly zero
-            assert not dA[g, rng_ranks[a]:].any() and not dB[g, rng_ranks[a]:].any()
+        fwd = orc.forward(t["X"], t["W"], t["A_all"], t["B_all"], t["scale"], w.segments)
+        rag = orc.backward_ragged(t["dY"], t["W"], A_list, B_list, t["scale"], w.segments, fwd["x_save"], n_rows=w.n_rows)
+        assert rag["ft_adapters"] == run.slots
+        for g, a in enumerate(run.slots):
+            ra = rng_ranks[a]                              # gradients of the padding rows are exactly zero,
+            assert not dA[g, ra:].any() and not dB[g, ra:].any()
+            assert_close(f"dA[{g}]", dA[g, :ra], rag["dA"][g], TOL["bf16"])      # the others those of the adapter's own rank
+            assert_close(f"dB[{g}]", dB[g, :ra], rag["dB"][g], TOL["bf16"])
+        assert_close("dX", run.host(run.dX)[:run.ft_rows], rag["dX"], TOL["bf16"])
     finally:
         run.close()

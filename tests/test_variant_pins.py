@@ -147,3 +147,54 @@ def test_ragged_ranks_equal_zero_padding():
     g_rows = slice(0, 3)
     u = X[0:3] @ A_list[0].T
     np.testing.assert_allclose(bwd["dB"][0, :1], scale[0] * (u.T @ dY[g_rows]), rtol=1e-12)
+
+
+def test_backward_ragged_is_the_gradient_of_forward_ragged():
+    """L = sum(Y * dY_full) over the fine-tuning rows: every entry of dA, dB (own ranks, nothing padded) and dX
+    against central finite differences of ``forward_ragged``; and the padded layer's gradients agree on the
+    rows that exist."""
+    rng = np.random.default_rng(14)
+    T, d_in, d_out = 10, 7, 5
+    ranks = [2, 5, 1, 3]
+    A_list = [rng.standard_normal((r, d_in)) for r in ranks]
+    B_list = [rng.standard_normal((r, d_out)) for r in ranks]
+    X, W = rng.standard_normal((T, d_in)), rng.standard_normal((d_in, d_out))
+    scale = np.array([4.0 / r for r in ranks])
+    segs = np.array([(0, 2, 3, 1), (2, 3, 1, 0), (5, 2, 0, 1), (7, 3, 3, 1)])      # adapter 3 trains on two segments
+    ft_rows = [0, 1, 5, 6, 7, 8, 9]                                               # save order = table order
+    dY = rng.standard_normal((len(ft_rows), d_out))
+    x_save = X[ft_rows]
+    got = orc.backward_ragged(dY, W, A_list, B_list, scale, segs, x_save, n_rows=T)
+    assert got["ft_adapters"] == [3, 0]
+
+    def loss(Xv, Al, Bl):
+        Y = orc.forward_ragged(Xv, W, Al, Bl, scale, segs)
+        return float((Y[ft_rows] * dY).sum())
+
+    eps = 1e-6
+    for g, a in enumerate(got["ft_adapters"]):
+        for name, lst, grad in (("A", A_list, got["dA"][g]), ("B", B_list, got["dB"][g])):
+            num = np.zeros_like(grad)
+            for idx in np.ndindex(*grad.shape):
+                hi = [m.copy() for m in lst]; lo = [m.copy() for m in lst]
+                hi[a][idx] += eps; lo[a][idx] -= eps
+                args_hi = (hi, B_list) if name == "A" else (A_list, hi)
+                args_lo = (lo, B_list) if name == "A" else (A_list, lo)
+                num[idx] = (loss(X, *args_hi) - loss(X, *args_lo)) / (2 * eps)
+            np.testing.assert_allclose(grad, num, rtol=1e-6, atol=1e-7)
+    num = np.zeros((len(ft_rows), d_in))
+    for m, t in enumerate(ft_rows):
+        for k in range(d_in):
+            hi, lo = X.copy(), X.copy()
+            hi[t, k] += eps; lo[t, k] -= eps
+            num[m, k] = (loss(hi, A_list, B_list) - loss(lo, A_list, B_list)) / (2 * eps)
+    np.testing.assert_allclose(got["dX"], num, rtol=1e-6, atol=1e-7)
+    # the zero-padded layer gives the same numbers where the rows exist
+    A_all, B_all = orc.pad_adapters(A_list, B_list, 5)
+    fwd = orc.forward(X, W, A_all, B_all, scale, segs)
+    pad = orc.backward(dY, W, A_all, B_all, scale, segs, fwd["x_save"], fwd["u_save"], n_rows=T)
+    assert pad["ft_adapters"] == got["ft_adapters"]
+    for g, a in enumerate(got["ft_adapters"]):
+        np.testing.assert_allclose(pad["dA"][g, :ranks[a]], got["dA"][g], rtol=1e-12, atol=1e-12)
+        np.testing.assert_allclose(pad["dB"][g, :ranks[a]], got["dB"][g], rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(pad["dX"], got["dX"], rtol=1e-12, atol=1e-12)
