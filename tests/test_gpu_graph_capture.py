@@ -15,7 +15,7 @@ from paper_2607_28848_b200.runner import LayerRun, Session
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("case", ["mixed", "long_k_split", "dropout", "one_finetune_adapter"])
+@pytest.mark.parametrize("case", ["mixed", "long_k_split", "dropout", "one_finetune_adapter", "rank_128", "uneven_tiles"])
 def test_graph_replay_matches_eager_on_new_inputs(case):
     with Session(0) as sess:
         if case == "long_k_split":      # few output tiles and K = 8192: the K-split GEMM and its reduction kernel
@@ -23,6 +23,11 @@ def test_graph_replay_matches_eager_on_new_inputs(case):
         elif case == "one_finetune_adapter":   # gradient groups split over rows: partial sums and arrival counters inside the graph
             segs = synth.segments_array([(0, 60, 2, 0), (60, 900, 0, 1), (960, 40, 1, 0)])
             w = synth.Workload("one_slot", 512, 768, 16, 3, "bf16", 1000, segs, seed=63)
+        elif case == "rank_128":          # tcgen05 shrink + finish kernel, operand split + tcgen05 gradient kernel
+            w = synth.random_workload(66, 512, 640, 128, 4, 700, max_seg=200, p_decode=0.05, p_finetune=0.5)
+        elif case == "uneven_tiles":      # the cost-balanced unit list of the GEMM is made in the warm-up and found by the capture
+            segs = [(0, 256, 0, 0)] + [(256 + i, 1, 1 + i, 0) for i in range(200)] + [(456, 312, 201, 1), (768, 256, 202, 1)]
+            w = synth.Workload("uneven", 512, 5120, 32, 203, "bf16", 1024, synth.segments_array(segs), seed=67)
         else:
             w = synth.random_workload(61, 256, 384, 16, 5, 420, max_seg=130, p_finetune=0.4)
         if case == "dropout":           # the seed is part of the captured launch parameters
