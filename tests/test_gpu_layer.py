@@ -53,6 +53,21 @@ def test_layer_forward_and_recompute_backward_match_the_oracle():
         assert layer.saved_rows == 97 and layer.saved == [(64, 1), (33, 2)]
         assert torch.equal(layer.saved_x[:97].cpu().double(), x[45:142])      # the layer input, bit for bit
 
+        # the same forward captured in a CUDA graph and replayed on a new batch of the same layout
+        cap = layer.capture_forward(x.to(sess.device).to(torch.bfloat16), synth.segments_array(segs))
+        cap.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(cap.y, y)
+        x2 = bf16(torch.randn(T, d, generator=g, dtype=torch.float64))
+        cap.x.copy_(x2.to(sess.device).to(torch.bfloat16))
+        cap.replay()
+        torch.cuda.synchronize()
+        y2_ref = lo.layer_forward(x2, p, row_adapter, sequences, H, Hkv)
+        err2 = (cap.y.double().cpu() - y2_ref).abs()
+        assert float((err2 - 3e-2 * (1 + y2_ref.abs())).max()) <= 0, float(err2.max())
+        cap.close()
+        assert mb.mlora_poll_status(sess.ctx) == mb.MLORA_OK
+
         # backward over the fine-tuning rows alone, recomputed from the saved input
         ft_rows = list(range(45, 142))
         dy = bf16(torch.randn(97, d, generator=g, dtype=torch.float64))
