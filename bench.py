@@ -60,7 +60,7 @@ from paper_2607_28848_b200.accounting import algorithmic_bytes, flops, load_peak
 # ---------------------------------------------------------------------------------------------
 # clocks
 # ---------------------------------------------------------------------------------------------
-def _sampler_child(path: str, uuid: str, index: int, period_s: float = 0.004) -> None:
+def _sampler_child(path: str, uuid: str, index: int, period_s: float = 0.003) -> None:
     """Child process: reads SM clock, power and clock-event reasons through NVML every few milliseconds
     (queries only; nothing is set) and appends `time sm_mhz power_w reasons_bitmask` lines to `path`."""
     import pynvml
@@ -82,13 +82,16 @@ def _sampler_child(path: str, uuid: str, index: int, period_s: float = 0.004) ->
     reasons_fn = getattr(pynvml, "nvmlDeviceGetCurrentClocksEventReasons", None) or pynvml.nvmlDeviceGetCurrentClocksThrottleReasons
     with open(path, "w", buffering=1) as fh:
         fh.write(f"# max {mx}\n")
+        n, power = 0, 0.0
         while True:
             t = time.time()
             try:
-                fh.write(f"{t:.6f} {pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)} "
-                         f"{pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0:.1f} {int(reasons_fn(h))}\n")
+                if n % 4 == 0:           # power changes slowly and its query is the slow one
+                    power = pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0
+                fh.write(f"{t:.6f} {pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)} {power:.1f} {int(reasons_fn(h))}\n")
             except Exception:
                 pass
+            n += 1
             dt = period_s - (time.time() - t)
             if dt > 0:
                 time.sleep(dt)
@@ -143,6 +146,12 @@ class ClockSampler:
         out = {}
         for name, (t0, t1) in self.regions.items():
             inside = [r for r in rows if t1 is not None and t0 <= r[0] <= t1]
+            nearest = False
+            if not inside and t1 is not None and rows:
+                # An NVML query can stall for tens of milliseconds while the process queues hundreds of launches: a
+                # short region may then hold no sample of its own.  Take the samples just around it and say so.
+                inside = [r for r in rows if t0 - 0.05 <= r[0] <= t1 + 0.05]
+                nearest = True
             if not inside:
                 out[name] = {"sm_mhz": None, "sm_max_mhz": mx, "reasons": ["no samples"], "samples": 0}
                 continue
@@ -153,6 +162,8 @@ class ClockSampler:
                          "sm_max_mhz": mx, "reasons": sorted(v for k, v in self.REASONS.items() if bits & k),
                          "samples": len(inside), "power_w_max": max(r[2] for r in inside),
                          "seconds": round(t1 - t0, 4)}
+            if nearest:
+                out[name]["note"] = "no sample fell inside the region: these are the samples within 50 ms around it"
         return out
 
 

@@ -525,12 +525,15 @@ mlora_status_t launch_shrink_tc(mlora_ctx* ctx, const RowSpace& hs, const DevRow
   return scope.done();
 }
 
-// Can this row space run on the tensor-core shrink?  Blocks that are nearly empty waste the 128-row MMA: with
-// fewer than four rows per block on average the kernels that gather rows by adapter are the better choice.
-inline bool shrink_tc_fits(const mlora_ctx* ctx, const RowSpace& hs, int n_rows, int D) {
+// Can this row space run on the tensor-core shrink?  Blocks that are nearly empty waste the 128-row MMA: below four
+// rows per block on average at rank 128 (where the alternative is the per-item kernel: 256 adapters on 2048 rows,
+// 11 rows per block, 45 + 15 us against 85), eight at the lower ranks (where it is the streaming kernel that gathers
+// rows by adapter: 512 single-row blocks beside 2048 fine-tuning rows at rank 32, 83 + 23 us against 41), the
+// mma.sync kernels are the better choice.
+inline bool shrink_tc_fits(const mlora_ctx* ctx, const RowSpace& hs, int n_rows, int D, int rank) {
   const int64_t NB = (int64_t)hs.tcb_row0.size();
   if (NB < 1 || D % 64 != 0 || n_rows > ctx->ws_rows || !ctx->ws_tc_part) return false;
-  if (4 * NB > (int64_t)hs.item_rows.size()) return false;
+  if ((rank >= 128 ? 4 : 8) * NB > (int64_t)hs.item_rows.size()) return false;
   return NB * ((D + 127) / 128) < (1 << 30) && NB + (int64_t)hs.zero_rows2.size() / 8 + 1 < (1 << 30);
 }
 
@@ -1460,7 +1463,7 @@ mlora_status_t mlora_mixed_forward(mlora_ctx* ctx, const mlora_layer_t* L, const
   sa.save_cap = save_capacity_rows;
   // rank >= kTcShrinkMinRank (every rank under kernel variant 6): the tcgen05 shrink and its finish kernel
   const bool tc_shrink = ctx->shrink_path == 0 && ctx->drop.thr == 0 && !h.fwd.tcb_row0.empty() &&
-                         (L->rank >= kTcShrinkMinRank || ctx->grad_mode == 2) && shrink_tc_fits(ctx, h.fwd, h.n_rows, L->d_in);
+                         (L->rank >= kTcShrinkMinRank || ctx->grad_mode == 2) && shrink_tc_fits(ctx, h.fwd, h.n_rows, L->d_in, L->rank);
   if (tc_shrink) {
     stc::FinArgs fa = {};
     fa.scale = nullptr; fa.Out = ctx->ws_p; fa.pbd = sa.pbd;
@@ -1509,7 +1512,7 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   sa.item_adapter = p->bwd.item_adapter; sa.item_save = nullptr; sa.x_save = nullptr; sa.u_save = nullptr; sa.save_base = 0; sa.save_cap = 0;
   // V on the tcgen05 shrink from rank kTcShrinkMinRank (every rank under kernel variant 6), else on the mma.sync kernels
   const bool tc_v = ctx->shrink_path == 0 && (L->rank >= kTcShrinkMinRank || ctx->grad_mode == 2) &&
-                    shrink_tc_fits(ctx, h.bwd, h.ft_rows, L->d_out);
+                    shrink_tc_fits(ctx, h.bwd, h.ft_rows, L->d_out, L->rank);
   if (tc_v) {
     stc::FinArgs fa = {};
     fa.scale = L->scale; fa.Out = ctx->ws_p; fa.pbd = sa.pbd;
