@@ -181,7 +181,7 @@ def test_random_shapes_tables_and_kernel_variants(sess, seed):
                                   int(rng.integers(1, 1200)), max_seg=int(rng.integers(1, 400)),
                                   p_decode=float(rng.uniform(0, 0.9)), p_finetune=float(rng.uniform(0, 0.7)))
         cap = None if rng.random() < 0.5 else int(w.ft_rows + 30)
-        run_and_check(sess, w, synth.make_tensors(w), path=int(rng.choice([0, 0, 0, 2, 3, 4])), blocked=True,
+        run_and_check(sess, w, synth.make_tensors(w), path=int(rng.choice([0, 0, 0, 2, 3, 4, 5, 6, 7])), blocked=True,
                       base=int(rng.integers(0, 3)) * 7, cap=cap)
 
 
@@ -396,19 +396,22 @@ def test_integer_probe_bit_exact(sess, dtype):
         run.close()
 
 
+@pytest.mark.parametrize("path", [0, 6])
 @pytest.mark.parametrize("seed", range(8))
-def test_random_tables_route_bit_exactly(sess, seed):
+def test_random_tables_route_bit_exactly(sess, seed, path):
     """Random valid segment tables (ragged lengths, single rows, gaps, adapter -1, shuffled order,
     several fine-tune segments per adapter) on the exact-integer probe: every output must equal the
-    oracle bit for bit, so any mis-routed row, wrong scale or mis-indexed save row shows."""
+    oracle bit for bit, so any mis-routed row, wrong scale or mis-indexed save row shows.  Under kernel
+    variant 6 every rank-r product runs on the tcgen05 kernels (blocks, run sums, operand images)."""
     rng = np.random.default_rng(seed)
     n_rows = int(rng.integers(1, 700))
     n_adapters = int(rng.integers(1, 40))
-    rank = int(rng.choice([8, 16, 32]))
+    rank = int(rng.choice([8, 16, 32, 64, 128]))
     d_in, d_out = int(rng.choice([64, 128, 192])), int(rng.choice([64, 256, 320]))
     p = integer_probe(n_rows=n_rows, d_in=d_in, d_out=d_out, rank=rank, n_adapters=n_adapters, seed=100 + seed,
                       max_seg=int(rng.integers(2, 300)))
     fwd = orc.forward(p["X"], p["W"], p["A_all"], p["B_all"], p["scale"], p["segments"])
+    mb.mlora_set_gemm_path(sess.ctx, path)
     run = LayerRun(sess, "bf16", p, p["segments"], n_rows, guard=True)
     try:
         run.forward()
@@ -426,6 +429,7 @@ def test_random_tables_route_bit_exactly(sess, seed):
             assert np.array_equal(run.host(run.dA), bwd["dA"])
             assert np.array_equal(run.host(run.dB), bwd["dB"])
     finally:
+        mb.mlora_set_gemm_path(sess.ctx, 0)
         run.close()
 
 
