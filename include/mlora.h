@@ -112,6 +112,20 @@ void mlora_destroy(mlora_ctx* ctx);
  * MLORA_ERR_INVALID_ARG, MLORA_ERR_CUDA. */
 mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, int32_t n_segs,
                                  int32_t n_rows, int32_t n_adapters, mlora_plan** plan);
+/* The same plan for adapters that have ranks of their own (Section 5 serves and trains adapters of
+ * different ranks side by side).  adapter_rank: HOST array [n_adapters], 1 <= r_a <= 128; NULL makes
+ * this call mlora_plan_create.  Storage does not change: every adapter still occupies `rank` rows of
+ * A_all and B_all in each layer, rows r_a .. rank - 1 zero, and gradients come back in that shape with
+ * those rows zero.  What changes is the work: in the base product's fused expand a group of rows is
+ * as wide as its adapter's rank rounded up to 16, not as wide as the layer's padded rank, so the
+ * extra K-blocks of a 256-row tile number ceil(sum of those widths / 64) instead of
+ * ceil(groups * rank / 64).  (The shrink and the gradients still run over all `rank` rows.)
+ * A plan made this way serves layers with rank % 16 == 0 and rank >= every r_a; other layers are
+ * refused by the compute calls with MLORA_ERR_INVALID_ARG.  Errors as mlora_plan_create, plus
+ * MLORA_ERR_INVALID_ARG for a rank outside [1, 128]. */
+mlora_status_t mlora_plan_create_ranked(mlora_ctx* ctx, const mlora_segment_t* segs, int32_t n_segs,
+                                        int32_t n_rows, int32_t n_adapters, const int32_t* adapter_rank,
+                                        mlora_plan** plan);
 void mlora_plan_destroy(mlora_plan* plan);
 
 /* Stream-ordered variant for serving loops, where every step has a new batch mix (paper,

@@ -238,7 +238,9 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
       const int m0 = mt * GEMM2_BM + (int)rank * 128;
       const int nh = nt * GEMM2_BN + (int)rank * 128;     // this CTA's half of the B columns
       const int G = tile_groups(mt);
-      const int LC = (G * R + 63) / 64;
+      const bool ranked = args.piece_src != nullptr && args.lora_enabled;
+      const int LC = ((ranked ? args.tile_cols[mt] : G * R) + 63) / 64;
+      const int pc_base = ranked ? args.tile_piece_off[mt] : 0, pc_end = ranked ? args.tile_piece_off[mt + 1] : 0;
       // a K slice takes its share of the low-rank blocks as well (an adapter-heavy tile has more of them than K-blocks)
       const int lc_begin = (int)((long long)ks * LC / SK), lc_end = (int)((long long)(ks + 1) * LC / SK);
       const int kb_begin = (int)((long long)ks * KB / SK), kb_end = (int)((long long)(ks + 1) * KB / SK);
@@ -266,22 +268,44 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
         if (!ok) break;
       }
       if (!ok) break;
-      if (lc_end > lc_begin) {
+      if (lc_end > lc_begin && !ranked) {
 #pragma unroll
         for (int j = 0; j < 8; ++j)
           if (lane + 32 * j < G) ga_smem[lane + 32 * j] = ga_reg[j];
         __syncwarp();
       }
+      // ranked plans: the pieces of eight chunks at a time, one per lane (one memory latency per eight chunks, the next
+      // eight already on their way)
+      auto piece_batch = [&](int first_chunk) -> int {
+        const int idx = pc_base + 4 * first_chunk + lane;
+        return (ranked && idx < pc_end) ? args.piece_src[idx] : 0;
+      };
+      int pb_chunk0 = lc_begin & ~7;
+      int pb_cur = piece_batch(pb_chunk0), pb_next = piece_batch(pb_chunk0 + 8);
       for (int lc = lc_begin; lc < lc_end; ++lc, ++it) {
         const int s = it % S;
         if (lane == 0) ok = gemm2_wait(bar_empty(s), ((it / S) & 1) ^ 1, abort_flag, args.status);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) break;
+        if (ranked && (lc & ~7) != pb_chunk0) { pb_chunk0 += 8; pb_cur = pb_next; pb_next = piece_batch(pb_chunk0 + 8); }
+        const int piece_of_lane = __shfl_sync(0xffffffffu, pb_cur, 4 * (lc & 7) + (lane & 3));
         const uint32_t a = sA0 + s * GEMM2_STAGE_BYTES, b = a + GEMM2_A_BYTES;
         const uint32_t full = ptx::map_to_cta(bar_full(s), 0);
         // A operand: this CTA's 128 rows of chunk lc of the tile's block-diagonal low-rank matrix
         if (lane == 0) ptx::tma2_load_2d(a, &tmPbd, 0, (2 * chunk_base + lc) * 256 + (int)rank * 128, full);
-        if (R <= 64) {
+        if (ranked) {
+          // B operand: up to four 16-row pieces of the adapters' matrices, one per lane (tmL has 16-row boxes here)
+          const int left = pc_end - (pc_base + 4 * lc);
+          const int np = left < 4 ? left : 4;
+          if (leader && lane == 0) ptx::mbar_arrive_expect_tx(bar_full(s), 2u * (GEMM2_A_BYTES + (uint32_t)np * 16u * 128u * 2u));
+          if (lane < np) {
+            const int src = piece_of_lane;
+            const int brow = (src >> 8) * R + (src & 255) * 16;
+#pragma unroll
+            for (int nb = 0; nb < 2; ++nb)
+              ptx::tma2_load_3d(b + nb * 8192 + lane * 16 * 128, &tmL, 0, brow, (nh >> 6) + nb, full);
+          }
+        } else if (R <= 64) {
           const int g0 = lc * GPC;
           const int ng = G - g0 < GPC ? G - g0 : GPC;
           const int ngl = (R == 8 && (ng & 1)) ? ng + 1 : ng;   // rank 8: pad a half-filled MMA step
@@ -314,6 +338,8 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
         int mt, nt_unused;
         gemm2_tile(args, tile, mt, nt_unused);
         const int kb_begin = (int)((long long)ks * KB / SK), kb_end = (int)((long long)(ks + 1) * KB / SK);
+        // columns of the tile's low-rank operand (read here, so that the main loop hides the latency)
+        const int lcols = (args.piece_src != nullptr && args.lora_enabled) ? args.tile_cols[mt] : tile_groups(mt) * R;
         const uint32_t buf = lt & 1;
         if (!(ok = gemm2_wait(bar_tempty(buf), ((lt >> 1) & 1) ^ 1, abort_flag, args.status))) break;
         ptx::tc_fence_after();
@@ -335,8 +361,7 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
           ptx::umma2_commit_both(bar_empty(s));
         }
         if (!ok) break;
-        const int G = tile_groups(mt);
-        const int LC = (G * R + 63) / 64;
+        const int LC = (lcols + 63) / 64;
         const int lc_begin = (int)((long long)ks * LC / SK), lc_end = (int)((long long)(ks + 1) * LC / SK);
         for (int lc = lc_begin; lc < lc_end; ++lc, ++it) {
           const int s = it % S;
@@ -345,7 +370,7 @@ gemm2_lora_kernel(const __grid_constant__ CUtensorMap tmIn, const __grid_constan
           const uint32_t a = sA0 + s * GEMM2_STAGE_BYTES, b = a + GEMM2_A_BYTES;
           const uint64_t adesc = ptx::make_smem_desc(a, 16, 1024);
           const uint64_t bdesc = ptx::make_smem_desc(b, 8192, 1024);
-          int ksteps = (G * R - lc * 64 + 15) / 16;
+          int ksteps = (lcols - lc * 64 + 15) / 16;
           ksteps = ksteps < 4 ? ksteps : 4;
           for (int ks = 0; ks < ksteps; ++ks) {
             ptx::umma2_f16(d_tmem, adesc + (uint64_t)(ks * 2), bdesc + (uint64_t)(ks * 128), idesc_lora, acc);

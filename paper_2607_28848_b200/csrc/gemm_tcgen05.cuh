@@ -63,6 +63,12 @@ struct GemmArgs {
   // the list was made for).
   const int32_t* unit_list;
   int32_t sched_pairs;
+  // Two-SM kernel, plans made with per-adapter ranks (all null otherwise): columns of each 256-row tile's low-rank
+  // operand, and its B-side rows as 16-row pieces of the adapters' matrices (piece_src = adapter << 8 | row / 16)
+  // in column order; the low-rank tensor map then has 16-row boxes.
+  const int32_t* tile_cols;
+  const int32_t* tile_piece_off;
+  const int32_t* piece_src;
   const int32_t* row_grp;        // [M] group of the row inside its 128-row tile, -1: none
   const int32_t* row_adapter;    // [M]
   const int32_t* tile_grp_off;   // [n_mtiles + 1]

@@ -146,6 +146,12 @@ struct DevRowSpace {
   const int32_t* tcb_row0 = nullptr;
   const int32_t* tcb_nrows = nullptr;
   const int32_t* tcb_adapter = nullptr;
+  // plans made with per-adapter ranks (null otherwise)
+  const int32_t* grp2_col = nullptr;
+  const int32_t* grp2_width = nullptr;
+  const int32_t* tile2_cols = nullptr;
+  const int32_t* tile2_piece_off = nullptr;
+  const int32_t* piece_src = nullptr;
 };
 
 struct mlora_plan {
@@ -787,7 +793,7 @@ void balanced_units(mlora_ctx* ctx, const RowSpace& hs, const DevRowSpace& ds, i
       gemm2_unit(g, u, tile, ks, sk);
       gemm2_tile(g, tile, mt, nt);
       const int G = hs.tile2_grp_off[mt + 1] - hs.tile2_grp_off[mt];
-      const int LC = (G * R + 63) / 64;
+      const int LC = ((g.piece_src ? hs.tile2_cols[mt] : G * R) + 63) / 64;
       const int kb = (int)((int64_t)(ks + 1) * kblocks / sk) - (int)((int64_t)ks * kblocks / sk);
       const int lc = (int)((int64_t)(ks + 1) * LC / sk) - (int)((int64_t)ks * LC / sk);
       cost[u] = kb + lc + 2;
@@ -848,6 +854,18 @@ void balanced_units(mlora_ctx* ctx, const RowSpace& hs, const DevRowSpace& ds, i
   g.sched_pairs = e->pairs;
 }
 
+// A plan made with per-adapter ranks serves layers whose padded rank is a multiple of 16 and at least every adapter's own.
+inline bool ranked_plan_fits(const HostPlan& h, const mlora_layer_t* L) {
+  if (h.adapter_rank.empty()) return true;
+  if (L->rank % 16 != 0) return false;
+  for (int32_t r : h.adapter_rank)
+    if (r > L->rank) return false;
+  return true;
+}
+inline void set_ranked(PbdArgs& pa, const DevRowSpace& ds) {
+  pa.grp2_col = ds.grp2_col; pa.grp2_width = ds.grp2_width; pa.tile2_cols = ds.tile2_cols;
+}
+
 // Out = In Wop + (scale) P L over one row space, tensor-core path.
 template <bool W_KMAJOR>
 mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace& hs, const DevRowSpace& ds,
@@ -862,11 +880,14 @@ mlora_status_t gemm_bf16(mlora_ctx* ctx, const mlora_layer_t* L, const RowSpace&
     if ((s = make_tmap_bf16_blocked(ctx, &tW, L->W, K, N, L->ldw, GEMM_BK, 2)) != MLORA_OK) return s;
   }
   const int R = L->rank;
-  if ((s = make_tmap_bf16_blocked(ctx, &tL, L_all, (uint64_t)L->n_adapters * R, N, N, R < 64 ? R : 64, 1)) != MLORA_OK)
+  const bool ranked = ds.piece_src != nullptr && ctx->gemm_pairs;    // B-side rows of the low-rank blocks come as 16-row pieces
+  if ((s = make_tmap_bf16_blocked(ctx, &tL, L_all, (uint64_t)L->n_adapters * R, N, N, ranked ? 16 : (R < 64 ? R : 64), 1)) != MLORA_OK)
     return s;
   if ((s = make_tmap_bf16(ctx, &tOut, Out, N, M, ld_out, 64, 32)) != MLORA_OK) return s;
   GemmArgs g;
   g.M = M; g.N = N; g.K = K; g.split_k = 1; g.ws_splitk = nullptr; g.unit_list = nullptr; g.sched_pairs = 0;
+  g.tile_cols = ranked ? ds.tile2_cols : nullptr; g.tile_piece_off = ranked ? ds.tile2_piece_off : nullptr;
+  g.piece_src = ranked ? ds.piece_src : nullptr;
   // Long contractions with many row tiles: the operand panels of one wave of tiles no longer fit the
   // L2 together with their neighbours', so the tiles are walked in bands of 8 row tiles (a wave then
   // covers about 8 x 9 tiles and streams 17 panels instead of 16 + 5 per 74 tiles; measured +2% on
@@ -1193,7 +1214,7 @@ void mlora_destroy(mlora_ctx* c) {
 
 namespace {
 
-constexpr int kPlanTables = 43;
+constexpr int kPlanTables = 53;
 
 // All device tables of a plan, packed; o[] receives each table's offset in 32-bit words.
 void pack_plan(const HostPlan& h, BlobBuilder& b, size_t* o) {
@@ -1207,6 +1228,8 @@ void pack_plan(const HostPlan& h, BlobBuilder& b, size_t* o) {
     o[n++] = b.add(rs[i]->item_save); o[n++] = b.add(rs[i]->item_start); o[n++] = b.add(rs[i]->item_desc);
     o[n++] = b.add(rs[i]->item_nrows); o[n++] = b.add(rs[i]->item_adapter);
     o[n++] = b.add(rs[i]->tcb_row0); o[n++] = b.add(rs[i]->tcb_nrows); o[n++] = b.add(rs[i]->tcb_adapter);
+    o[n++] = b.add(rs[i]->grp2_col); o[n++] = b.add(rs[i]->grp2_width); o[n++] = b.add(rs[i]->tile2_cols);
+    o[n++] = b.add(rs[i]->tile2_piece_off); o[n++] = b.add(rs[i]->piece_src);
   }
   o[n++] = b.add(h.slot_chunk_off); o[n++] = b.add(h.chunk_row0); o[n++] = b.add(h.chunk_nrows);
   o[n++] = b.add(h.ft_adapters);
@@ -1255,6 +1278,12 @@ void bind_plan(mlora_plan* p, const size_t* o) {
     ds[i]->item_save = p->blob + o[n++]; ds[i]->item_start = p->blob + o[n++]; ds[i]->item_desc = p->blob + o[n++];
     ds[i]->item_nrows = p->blob + o[n++]; ds[i]->item_adapter = p->blob + o[n++];
     ds[i]->tcb_row0 = p->blob + o[n++]; ds[i]->tcb_nrows = p->blob + o[n++]; ds[i]->tcb_adapter = p->blob + o[n++];
+    const bool ranked = !p->h.adapter_rank.empty();
+    ds[i]->grp2_col = ranked ? p->blob + o[n] : nullptr; ++n;
+    ds[i]->grp2_width = ranked ? p->blob + o[n] : nullptr; ++n;
+    ds[i]->tile2_cols = ranked ? p->blob + o[n] : nullptr; ++n;
+    ds[i]->tile2_piece_off = ranked ? p->blob + o[n] : nullptr; ++n;
+    ds[i]->piece_src = ranked ? p->blob + o[n] : nullptr; ++n;
   }
   p->bwd.row_save = nullptr;       // the compact space has no save offsets
   p->slot_chunk_off = p->blob + o[n++]; p->chunk_row0 = p->blob + o[n++]; p->chunk_nrows = p->blob + o[n++];
@@ -1315,11 +1344,16 @@ mlora_status_t grow_workspaces(mlora_ctx* ctx, const HostPlan& h, int32_t n_rows
 
 mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, int32_t n_segs, int32_t n_rows,
                                  int32_t n_adapters, mlora_plan** out) {
+  return mlora_plan_create_ranked(ctx, segs, n_segs, n_rows, n_adapters, nullptr, out);
+}
+
+mlora_status_t mlora_plan_create_ranked(mlora_ctx* ctx, const mlora_segment_t* segs, int32_t n_segs, int32_t n_rows,
+                                        int32_t n_adapters, const int32_t* adapter_rank, mlora_plan** out) {
   if (!out) return MLORA_ERR_INVALID_ARG;
   *out = nullptr;
   mlora_plan* p = new (std::nothrow) mlora_plan();
   if (!p) return MLORA_ERR_INVALID_ARG;
-  mlora_status_t s = build_plan(segs, n_segs, n_rows, n_adapters, p->h);
+  mlora_status_t s = build_plan(segs, n_segs, n_rows, n_adapters, p->h, adapter_rank);
   if (s != MLORA_OK) { delete p; return s; }
   p->ctx = ctx;
   if (ctx) {
@@ -1440,7 +1474,7 @@ mlora_status_t mlora_mixed_forward(mlora_ctx* ctx, const mlora_layer_t* L, const
     if (save_row_base + h.ft_rows > save_capacity_rows) return MLORA_ERR_SAVE_CAPACITY;
     if (!u_save) return MLORA_ERR_INVALID_ARG;
   }
-  if (h.n_rows > ctx->ws_rows) return MLORA_ERR_INVALID_ARG;
+  if (h.n_rows > ctx->ws_rows || !ranked_plan_fits(h, L)) return MLORA_ERR_INVALID_ARG;
   // the tensor maps are encoded through the driver API, which needs this device's context current on the
   // calling thread (a framework's worker threads do not always have one)
   if (cudaSetDevice(ctx->device) != cudaSuccess) return MLORA_ERR_CUDA;
@@ -1459,6 +1493,7 @@ mlora_status_t mlora_mixed_forward(mlora_ctx* ctx, const mlora_layer_t* L, const
   sa.item_adapter = p->fwd.item_adapter; sa.item_save = p->fwd.item_save;
   sa.pbd = PbdArgs{ctx->gemm_pairs ? ctx->ws_pbd : nullptr, p->fwd.row_grp2, p->fwd.tile2_grp_off, L->scale,
                    p->fwd.zero_rows2, (int32_t)h.fwd.zero_rows2.size()};
+  set_ranked(sa.pbd, p->fwd);
   sa.x_save = (__nv_bfloat16*)x_save; sa.u_save = u_save; sa.save_base = save_row_base;
   sa.save_cap = save_capacity_rows;
   // rank >= kTcShrinkMinRank (every rank under kernel variant 6): the tcgen05 shrink and its finish kernel
@@ -1488,6 +1523,7 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   if (h.n_adapters > L->n_adapters) return MLORA_ERR_ADAPTER_ID;
   if (h.ft_rows == 0) return MLORA_OK;
   if (!dY || !x_save || !u_save || !dA || !dB || lddy < L->d_out || (dX && lddx < L->d_in)) return MLORA_ERR_INVALID_ARG;
+  if (!ranked_plan_fits(h, L)) return MLORA_ERR_INVALID_ARG;
   // the tensor maps are encoded through the driver API, which needs this device's context current on the
   // calling thread (a framework's worker threads do not always have one)
   if (cudaSetDevice(ctx->device) != cudaSuccess) return MLORA_ERR_CUDA;
@@ -1509,6 +1545,7 @@ mlora_status_t mlora_backward(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   sa.item_rows = p->bwd.item_rows; sa.item_start = p->bwd.item_start; sa.item_nrows = p->bwd.item_nrows;
   sa.pbd = PbdArgs{(ctx->gemm_pairs && dX && !dropping) ? ctx->ws_pbd : nullptr, p->bwd.row_grp2, p->bwd.tile2_grp_off, nullptr,
                    p->bwd.zero_rows2, (int32_t)h.bwd.zero_rows2.size()};
+  set_ranked(sa.pbd, p->bwd);
   sa.item_adapter = p->bwd.item_adapter; sa.item_save = nullptr; sa.x_save = nullptr; sa.u_save = nullptr; sa.save_base = 0; sa.save_cap = 0;
   // V on the tcgen05 shrink from rank kTcShrinkMinRank (every rank under kernel variant 6), else on the mma.sync kernels
   const bool tc_v = ctx->shrink_path == 0 && (L->rank >= kTcShrinkMinRank || ctx->grad_mode == 2) &&

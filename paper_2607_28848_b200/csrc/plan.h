@@ -44,12 +44,19 @@ struct RowSpace {
   std::vector<int32_t> item_desc;
   // Blocks for the tensor-core shrink: runs of <= kTileRows consecutive rows that share one adapter.
   std::vector<int32_t> tcb_row0, tcb_nrows, tcb_adapter;
+  // Plans made with per-adapter ranks only (empty otherwise): in the block-diagonal low-rank operand of a
+  // 256-row tile a group is as wide as its adapter's rank rounded up to 16 columns, not as wide as the layer's
+  // padded rank.  grp2_col / grp2_width: first column and width of each group; tile2_cols: columns of each
+  // tile's operand; the operand's rows on the B side are 16-row PIECES of the adapters' matrices, listed per
+  // tile in column order: piece_src = adapter << 8 | (first row of the piece inside the adapter / 16).
+  std::vector<int32_t> grp2_col, grp2_width, tile2_cols, tile2_piece_off, piece_src;
   int32_t n_tiles() const { return (n_rows + kTileRows - 1) / kTileRows; }
   int32_t n_items() const { return (int32_t)item_start.size(); }
 };
 
 struct HostPlan {
   int32_t n_rows = 0, n_adapters = 0, n_segs = 0;
+  std::vector<int32_t> adapter_rank;   // [n_adapters] own rank of each adapter, or empty: every adapter has the layer's rank
   int32_t ft_rows = 0;
   std::vector<int32_t> seg_save_off;   // [n_segs] save offset or -1
   std::vector<int32_t> ft_adapters;    // slot -> adapter id
@@ -83,6 +90,25 @@ inline void build_tile_groups(const std::vector<int32_t>& row_adapter, int32_t t
       row_grp[t] = g;
     }
     tile_grp_off.push_back((int32_t)grp_adapter.size());
+  }
+}
+
+// Group widths and B-side pieces of a ranked plan (see RowSpace).
+inline void build_ranked(RowSpace& rs, const std::vector<int32_t>& adapter_rank) {
+  rs.grp2_col.clear(); rs.grp2_width.clear(); rs.tile2_cols.clear(); rs.piece_src.clear();
+  rs.tile2_piece_off.assign(1, 0);
+  for (size_t t = 0; t + 1 < rs.tile2_grp_off.size(); ++t) {
+    int32_t col = 0;
+    for (int32_t i = rs.tile2_grp_off[t]; i < rs.tile2_grp_off[t + 1]; ++i) {
+      const int32_t a = rs.grp2_adapter[i];
+      const int32_t w = (adapter_rank[a] + 15) / 16 * 16;
+      rs.grp2_col.push_back(col);
+      rs.grp2_width.push_back(w);
+      for (int32_t j = 0; j < w / 16; ++j) rs.piece_src.push_back((a << 8) | j);
+      col += w;
+    }
+    rs.tile2_cols.push_back(col);
+    rs.tile2_piece_off.push_back((int32_t)rs.piece_src.size());
   }
 }
 
@@ -144,11 +170,15 @@ inline void build_tiles_and_items(RowSpace& rs) {
 
 // Validates the table and fills `p`.  Returns MLORA_OK or the error the header documents.
 inline mlora_status_t build_plan(const mlora_segment_t* segs, int32_t n_segs, int32_t n_rows,
-                                 int32_t n_adapters, HostPlan& p) {
+                                 int32_t n_adapters, HostPlan& p, const int32_t* adapter_rank = nullptr) {
   if (n_segs < 0 || n_rows < 0 || n_adapters < 0 || (n_segs > 0 && segs == nullptr))
     return MLORA_ERR_INVALID_ARG;
+  if (adapter_rank)
+    for (int32_t a = 0; a < n_adapters; ++a)
+      if (adapter_rank[a] < 1 || adapter_rank[a] > kMaxRank) return MLORA_ERR_INVALID_ARG;
   p = HostPlan();
   p.n_rows = n_rows; p.n_adapters = n_adapters; p.n_segs = n_segs;
+  if (adapter_rank) p.adapter_rank.assign(adapter_rank, adapter_rank + n_adapters);
   p.fwd.n_rows = n_rows;
   p.fwd.row_adapter.assign(n_rows, -1);
   p.fwd.row_save.assign(n_rows, -1);
@@ -182,6 +212,7 @@ inline mlora_status_t build_plan(const mlora_segment_t* segs, int32_t n_segs, in
   }
   p.ft_rows = off;
   build_tiles_and_items(p.fwd);
+  if (!p.adapter_rank.empty()) build_ranked(p.fwd, p.adapter_rank);
 
   // compact fine-tuning row space (save order) and the gradient chunk lists
   p.bwd.n_rows = p.ft_rows;
@@ -191,6 +222,7 @@ inline mlora_status_t build_plan(const mlora_segment_t* segs, int32_t n_segs, in
     for (int32_t i = 0; i < segs[k].row_len; ++i) p.bwd.row_adapter[p.seg_save_off[k] + i] = segs[k].adapter_id;
   }
   build_tiles_and_items(p.bwd);
+  if (!p.adapter_rank.empty()) build_ranked(p.bwd, p.adapter_rank);
   p.slot_chunk_off.assign(1, 0);
   for (int32_t a : p.ft_adapters) {
     for (int32_t k = 0; k < n_segs; ++k) {

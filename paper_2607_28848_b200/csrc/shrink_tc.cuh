@@ -239,7 +239,7 @@ shrink_tc_finish_kernel(const FinArgs a) {
     const int row = a.pbd.zero_rows[zi];
     const int tile = row >> 8, rl = row & 255;
     const int goff = a.pbd.tile2_grp_off[tile], Gt = a.pbd.tile2_grp_off[tile + 1] - goff;
-    const int LC = (Gt * R + 63) / 64;
+    const int LC = ((a.pbd.tile2_cols ? a.pbd.tile2_cols[tile] : Gt * R) + 63) / 64;
     __nv_bfloat16* base = a.pbd.pbd + ((size_t)(2 * goff) * 256 + rl) * 64;
     for (int pi = j; pi < LC * 8; pi += TPR)
       *reinterpret_cast<uint4*>(base + (size_t)(pi >> 3) * (256 * 64) + (pi & 7) * 8) = make_uint4(0, 0, 0, 0);
@@ -255,12 +255,16 @@ shrink_tc_finish_kernel(const FinArgs a) {
   const float sc = a.scale ? a.scale[ad] : 1.0f;
   const float psc = a.pbd.scale ? a.pbd.scale[ad] : 1.0f;
   const int sv = (live && a.row_save) ? a.row_save[row] : -1;
-  int goff = 0, Gt = 0, g = -1;
+  int goff = 0, g = -1, cols = 0, c0 = 0, cw = 0;     // the tile's operand columns; the row's own: [c0, c0 + cw)
   if (a.pbd.pbd) {
     const int tile = row >> 8;
     goff = a.pbd.tile2_grp_off[tile];
-    Gt = a.pbd.tile2_grp_off[tile + 1] - goff;
     g = a.pbd.row_grp2[row];
+    cols = a.pbd.tile2_cols ? a.pbd.tile2_cols[tile] : (a.pbd.tile2_grp_off[tile + 1] - goff) * R;
+    if (g >= 0) {
+      c0 = a.pbd.grp2_col ? a.pbd.grp2_col[goff + g] : g * R;
+      cw = a.pbd.grp2_width ? a.pbd.grp2_width[goff + g] : R;
+    }
   }
   const int N = a.NB * a.NS, gbase = blk * a.NS;
   const int c_first = owner(gbase, a.G, N), c_last = owner(gbase + a.NS - 1, a.G, N);
@@ -299,15 +303,15 @@ shrink_tc_finish_kernel(const FinArgs a) {
     uint32_t w0 = ptx::pack_bf16(vs.x * psc, vs.y * psc), w1 = ptx::pack_bf16(vs.z * psc, vs.w * psc);
     const uint32_t n0 = __shfl_down_sync(0xffffffffu, w0, 1), n1 = __shfl_down_sync(0xffffffffu, w1, 1);
     if (live) {
-      const int LC = (Gt * R + 63) / 64;
+      const int LC = (cols + 63) / 64;
       __nv_bfloat16* base = a.pbd.pbd + ((size_t)(2 * goff) * 256 + (row & 255)) * 64;
-      const int p0 = g >= 0 ? g * (R / 8) : LC * 8;
-      if (g >= 0 && (j & 1) == 0) {
+      const int p0 = g >= 0 ? c0 / 8 : LC * 8, pw = cw / 8;     // the row's own 16-byte pieces: [p0, p0 + pw)
+      if (g >= 0 && (j & 1) == 0 && (j >> 1) < pw) {
         const int pi = p0 + (j >> 1);
         *reinterpret_cast<uint4*>(base + (size_t)(pi >> 3) * (256 * 64) + (pi & 7) * 8) = make_uint4(w0, w1, n0, n1);
       }
       for (int pi = j; pi < LC * 8; pi += TPR)
-        if (pi < p0 || pi >= p0 + R / 8)
+        if (pi < p0 || pi >= p0 + pw)
           *reinterpret_cast<uint4*>(base + (size_t)(pi >> 3) * (256 * 64) + (pi & 7) * 8) = make_uint4(0, 0, 0, 0);
     }
   }

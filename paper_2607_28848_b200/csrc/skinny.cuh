@@ -35,6 +35,10 @@ struct PbdArgs {
   const float* scale;            // nullable: values multiplied by scale[adapter]
   const int32_t* zero_rows;      // rows without an adapter inside tiles that have groups
   int32_t n_zero_rows;
+  // plans made with per-adapter ranks (all three null otherwise: group g of a tile starts at column g R and is R wide)
+  const int32_t* grp2_col = nullptr;     // [groups] first column of the group in its tile's operand
+  const int32_t* grp2_width = nullptr;   // [groups] its width (the adapter's rank rounded up to 16)
+  const int32_t* tile2_cols = nullptr;   // [tiles] columns of the tile's operand
 };
 
 // One warp writes all chunks of one row: `vals` = the row's R fp32 values (nullptr: all zero).
@@ -44,13 +48,16 @@ template <int R>
 __device__ __forceinline__ void pbd_write_row_at(const PbdArgs& pa, int row, int goff, int G, int g, const float* vals,
                                                  float sc, int lane) {
   const int rl = row & 255;
-  const int LC = (G * R + 63) / 64;
+  const int cols = pa.tile2_cols ? pa.tile2_cols[row >> 8] : G * R;
+  const int LC = (cols + 63) / 64;
+  const int c0 = g < 0 ? 0 : (pa.grp2_col ? pa.grp2_col[goff + g] : g * R);        // the row's own columns: [c0, c0 + w)
+  const int w = g < 0 ? 0 : (pa.grp2_width ? pa.grp2_width[goff + g] : R);
   for (int piece = lane; piece < LC * 8; piece += 32) {
     const int c = piece >> 3, kcol = piece * 8;          // chunk, first low-rank column of the piece
     uint4 v = make_uint4(0, 0, 0, 0);
-    if (g >= 0 && kcol >= g * R && kcol < (g + 1) * R) {
-      const float4 f0 = *reinterpret_cast<const float4*>(vals + (kcol - g * R));
-      const float4 f1 = *reinterpret_cast<const float4*>(vals + (kcol - g * R) + 4);
+    if (kcol >= c0 && kcol < c0 + w) {
+      const float4 f0 = *reinterpret_cast<const float4*>(vals + (kcol - c0));
+      const float4 f1 = *reinterpret_cast<const float4*>(vals + (kcol - c0) + 4);
       v.x = ptx::pack_bf16(f0.x * sc, f0.y * sc); v.y = ptx::pack_bf16(f0.z * sc, f0.w * sc);
       v.z = ptx::pack_bf16(f1.x * sc, f1.y * sc); v.w = ptx::pack_bf16(f1.z * sc, f1.w * sc);
     }

@@ -46,7 +46,7 @@ class LayerRun:
 
     def __init__(self, sess: Session, dtype: str, tensors: Dict[str, np.ndarray], segments: np.ndarray,
                  n_rows: int, save_row_base: int = 0, save_capacity_rows: Optional[int] = None,
-                 save_x: bool = True, guard: bool = False):
+                 save_x: bool = True, guard: bool = False, adapter_rank=None):
         self.sess, self.dtype = sess, dtype
         td = torch_dtype(dtype)
         dev = sess.device
@@ -59,7 +59,10 @@ class LayerRun:
         self.d_out = self.B_all.shape[2]
         self.n_rows = n_rows
         self.segments = np.asarray(segments, dtype=np.int32).reshape(-1, 4)
-        self.plan = mb.mlora_plan_create(sess.ctx, self.segments, n_rows, self.n_adapters)
+        if adapter_rank is None:
+            self.plan = mb.mlora_plan_create(sess.ctx, self.segments, n_rows, self.n_adapters)
+        else:               # adapters with ranks of their own (stored padded to the layer's rank)
+            self.plan = mb.mlora_plan_create_ranked(sess.ctx, self.segments, n_rows, self.n_adapters, adapter_rank)
         self.ft_rows = mb.mlora_plan_ft_rows(self.plan)
         self.slots = mb.mlora_plan_ft_adapters(self.plan)
         self.layer = mb.make_layer(self.W, self.A_all, self.B_all, self.scale)

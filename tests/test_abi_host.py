@@ -71,6 +71,25 @@ def test_plan_refuses_bad_tables(bad, code):
     assert e.value.status == code
 
 
+def test_ranked_plan_on_the_host():
+    """Per-adapter ranks do not touch routing: same offsets, slots and row table; ranks outside [1, 128] are refused;
+    no rank array is the plain plan."""
+    segs = [(10, 4, 2, 1), (0, 3, 1, 0), (20, 5, 0, 1), (4, 2, 2, 1)]
+    plain = host_plan(segs, 30, 3)
+    ranked = mb.mlora_plan_create_ranked(None, segs, 30, 3, [4, 128, 17])
+    try:
+        assert mb.mlora_plan_ft_adapters(ranked) == mb.mlora_plan_ft_adapters(plain) == [2, 0]
+        a, b = mb.mlora_plan_describe(plain, len(segs)), mb.mlora_plan_describe(ranked, len(segs))
+        assert a[0].tolist() == b[0].tolist() and a[1].tolist() == b[1].tolist()
+    finally:
+        mb.mlora_plan_destroy(plain)
+        mb.mlora_plan_destroy(ranked)
+    for bad in ([4, 0, 8], [4, 129, 8], [-1, 8, 8]):
+        with pytest.raises(mb.MloraError) as e:
+            mb.mlora_plan_create_ranked(None, segs, 30, 3, bad)
+        assert e.value.status == mb.MLORA_ERR_INVALID_ARG
+
+
 def test_empty_table_and_empty_batch():
     p = host_plan(np.zeros((0, 4), np.int32), 5, 2)
     assert mb.mlora_plan_ft_rows(p) == 0 and mb.mlora_plan_ft_adapters(p) == []

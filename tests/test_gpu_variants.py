@@ -180,3 +180,93 @@ def test_different_ranks_through_zero_padding(sess):
         assert_close("dX", run.host(run.dX)[:run.ft_rows], rag["dX"], TOL["bf16"])
     finally:
         run.close()
+
+
+def _ragged_case(seed, d_in, d_out, R, ranks, n_rows, **kw):
+    w = synth.random_workload(seed, d_in, d_out, R, len(ranks), n_rows, **kw)
+    t = synth.make_tensors(w)
+    A_list, B_list = [], []
+    for a, ra in enumerate(ranks):
+        t["A_all"][a, ra:] = 0.0
+        t["B_all"][a, ra:] = 0.0
+        A_list.append(t["A_all"][a, :ra].copy())
+        B_list.append(t["B_all"][a, :ra].copy())
+        t["scale"][a] = 32.0 / ra
+    return w, t, A_list, B_list
+
+
+def _check_ragged(run, w, t, A_list, B_list, ranks):
+    run.forward()
+    run.backward()
+    assert run.status() == mb.MLORA_OK
+    ref = orc.forward_ragged(t["X"], t["W"], A_list, B_list, t["scale"], w.segments)
+    assert_close("Y", run.host(run.Y), ref, TOL["bf16"])
+    fwd = orc.forward(t["X"], t["W"], t["A_all"], t["B_all"], t["scale"], w.segments)
+    rag = orc.backward_ragged(t["dY"], t["W"], A_list, B_list, t["scale"], w.segments, fwd["x_save"], n_rows=w.n_rows)
+    assert rag["ft_adapters"] == run.slots
+    dA, dB = run.host(run.dA), run.host(run.dB)
+    for g, a in enumerate(run.slots):
+        ra = ranks[a]
+        assert not dA[g, ra:].any() and not dB[g, ra:].any()
+        assert_close(f"dA[{g}]", dA[g, :ra], rag["dA"][g], TOL["bf16"])
+        assert_close(f"dB[{g}]", dB[g, :ra], rag["dB"][g], TOL["bf16"])
+    assert_close("dX", run.host(run.dX)[:run.ft_rows], rag["dX"], TOL["bf16"])
+
+
+@pytest.mark.parametrize("R,path", [(16, 0), (32, 0), (64, 0), (128, 0), (64, 2), (32, 6), (64, 7)])
+def test_plans_with_per_adapter_ranks(sess, R, path):
+    """mlora_plan_create_ranked: the fused expand packs every group of a tile by its own rank (rounded up to 16)
+    instead of the layer's padded rank.  Same numbers as the per-rank oracle, forward and backward, on ragged tables
+    with single-row groups, on every kernel that writes the GEMM's low-rank operand (streaming shrink, per-item
+    shrink = kernel variant 2, tcgen05 finish kernel = ranks 64 / 128 and kernel variant 6)."""
+    ranks = [r for r in (1, 4, 8, 12, 16, 24, 32, 48, 64, 100, 128) if r <= R]
+    ranks = (ranks * 3)[:max(6, len(ranks))]
+    w, t, A_list, B_list = _ragged_case(300 + R + path, 384, 768, R, ranks, 900, max_seg=140, p_decode=0.4, p_finetune=0.35)
+    mb.mlora_set_gemm_path(sess.ctx, path)
+    run = LayerRun(sess, w.dtype, t, w.segments, w.n_rows, adapter_rank=ranks)
+    try:
+        _check_ragged(run, w, t, A_list, B_list, ranks)
+    finally:
+        mb.mlora_set_gemm_path(sess.ctx, 0)
+        run.close()
+
+
+def test_ranked_plan_gives_the_padded_plan_s_numbers_bit_for_bit(sess):
+    """Packing the groups changes which zero columns the tensor cores multiply, not a single product that counts:
+    a ranked plan and a plain plan over the same zero-padded adapters give identical bits."""
+    ranks = [16, 64, 32, 16, 48, 8, 16, 64]
+    w, t, _, _ = _ragged_case(77, 512, 1024, 64, ranks, 1100, max_seg=60, p_decode=0.5, p_finetune=0.3)
+    outs = []
+    for ar in (None, ranks):
+        run = LayerRun(sess, w.dtype, t, w.segments, w.n_rows, adapter_rank=ar)
+        try:
+            run.forward(); run.backward()
+            assert run.status() == mb.MLORA_OK
+            outs.append([b.clone() for b in (run.Y, run.dX, run.dA, run.dB)])
+        finally:
+            run.close()
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
+def test_ranked_plan_refusals(sess):
+    w = synth.random_workload(78, 128, 128, 8, 3, 100, p_finetune=0.4)
+    t = synth.make_tensors(w)
+    with pytest.raises(mb.MloraError) as e:                 # rank outside [1, 128]
+        mb.mlora_plan_create_ranked(sess.ctx, w.segments, w.n_rows, 3, [4, 0, 8])
+    assert e.value.status == mb.MLORA_ERR_INVALID_ARG
+    run = LayerRun(sess, w.dtype, t, w.segments, w.n_rows, adapter_rank=[4, 8, 8])      # layer rank 8: not a multiple of 16
+    try:
+        with pytest.raises(mb.MloraError) as e:
+            run.forward()
+        assert e.value.status == mb.MLORA_ERR_INVALID_ARG
+    finally:
+        run.close()
+    w16 = synth.random_workload(79, 128, 128, 16, 3, 100, p_finetune=0.4)
+    run = LayerRun(sess, w16.dtype, synth.make_tensors(w16), w16.segments, w16.n_rows, adapter_rank=[4, 32, 8])   # an adapter wider than the layer
+    try:
+        with pytest.raises(mb.MloraError) as e:
+            run.forward()
+        assert e.value.status == mb.MLORA_ERR_INVALID_ARG
+    finally:
+        run.close()
