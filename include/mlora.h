@@ -142,6 +142,10 @@ void mlora_plan_destroy(mlora_plan* plan);
 mlora_status_t mlora_plan_create_async(mlora_ctx* ctx, const mlora_segment_t* segs, int32_t n_segs,
                                        int32_t n_rows, int32_t n_adapters, void* cuda_stream,
                                        mlora_plan** plan);
+/* mlora_plan_create_async for adapters with ranks of their own (see mlora_plan_create_ranked). */
+mlora_status_t mlora_plan_create_ranked_async(mlora_ctx* ctx, const mlora_segment_t* segs, int32_t n_segs,
+                                              int32_t n_rows, int32_t n_adapters, const int32_t* adapter_rank,
+                                              void* cuda_stream, mlora_plan** plan);
 mlora_status_t mlora_plan_release(mlora_plan* plan, void* cuda_stream);
 
 int32_t mlora_plan_rows(const mlora_plan* plan);        /* n_rows                              */

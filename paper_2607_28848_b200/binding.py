@@ -24,7 +24,7 @@ EXPORTS = (
     "mlora_create", "mlora_destroy", "mlora_plan_create", "mlora_plan_destroy", "mlora_plan_rows",
     "mlora_plan_ft_rows", "mlora_plan_ft_adapters", "mlora_plan_describe", "mlora_mixed_forward",
     "mlora_backward", "mlora_poll_status", "mlora_status_string", "mlora_launch_count", "mlora_set_gemm_path",
-    "mlora_plan_create_ranked", "mlora_profile_enable", "mlora_profile_collect", "mlora_forward_noalloc", "mlora_adamw_update",
+    "mlora_plan_create_ranked", "mlora_plan_create_ranked_async", "mlora_profile_enable", "mlora_profile_collect", "mlora_forward_noalloc", "mlora_adamw_update",
     "mlora_set_cancel_flag", "mlora_set_dropout", "mlora_plan_create_async", "mlora_plan_release",
     "mlora_selftest_timeout",
 )
@@ -79,6 +79,8 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.mlora_plan_create.restype = ctypes.c_int
     lib.mlora_plan_create_ranked.argtypes = [vp, P(mlora_segment_t), i32, i32, i32, P(i32), P(vp)]
     lib.mlora_plan_create_ranked.restype = ctypes.c_int
+    lib.mlora_plan_create_ranked_async.argtypes = [vp, P(mlora_segment_t), i32, i32, i32, P(i32), vp, P(vp)]
+    lib.mlora_plan_create_ranked_async.restype = ctypes.c_int
     lib.mlora_plan_destroy.argtypes = [vp]
     lib.mlora_plan_destroy.restype = None
     lib.mlora_plan_create_async.argtypes = [vp, P(mlora_segment_t), i32, i32, i32, vp, P(vp)]
@@ -181,6 +183,16 @@ def mlora_plan_create_async(ctx, segments, n_rows: int, n_adapters: int, stream=
     h = ctypes.c_void_p()
     _check(load_library().mlora_plan_create_async(ctx, arr, n, int(n_rows), int(n_adapters), _stream_ptr(stream),
                                                   ctypes.byref(h)), "mlora_plan_create_async")
+    return h
+
+
+def mlora_plan_create_ranked_async(ctx, segments, n_rows: int, n_adapters: int, adapter_rank, stream=None) -> ctypes.c_void_p:
+    """Stream-ordered plan for adapters with ranks of their own."""
+    arr, n = _segments_ctypes(segments)
+    ranks = (ctypes.c_int32 * int(n_adapters))(*[int(r) for r in adapter_rank])
+    h = ctypes.c_void_p()
+    _check(load_library().mlora_plan_create_ranked_async(ctx, arr, n, int(n_rows), int(n_adapters), ranks, _stream_ptr(stream),
+                                                         ctypes.byref(h)), "mlora_plan_create_ranked_async")
     return h
 
 

@@ -1376,11 +1376,17 @@ mlora_status_t mlora_plan_create_ranked(mlora_ctx* ctx, const mlora_segment_t* s
 
 mlora_status_t mlora_plan_create_async(mlora_ctx* ctx, const mlora_segment_t* segs, int32_t n_segs, int32_t n_rows,
                                        int32_t n_adapters, void* cuda_stream, mlora_plan** out) {
+  return mlora_plan_create_ranked_async(ctx, segs, n_segs, n_rows, n_adapters, nullptr, cuda_stream, out);
+}
+
+mlora_status_t mlora_plan_create_ranked_async(mlora_ctx* ctx, const mlora_segment_t* segs, int32_t n_segs, int32_t n_rows,
+                                              int32_t n_adapters, const int32_t* adapter_rank, void* cuda_stream,
+                                              mlora_plan** out) {
   if (!out || !ctx) return MLORA_ERR_INVALID_ARG;
   *out = nullptr;
   mlora_plan* p = new (std::nothrow) mlora_plan();
   if (!p) return MLORA_ERR_INVALID_ARG;
-  mlora_status_t s = build_plan(segs, n_segs, n_rows, n_adapters, p->h);
+  mlora_status_t s = build_plan(segs, n_segs, n_rows, n_adapters, p->h, adapter_rank);
   if (s != MLORA_OK) { delete p; return s; }
   p->ctx = ctx;
   if (cudaSetDevice(ctx->device) != cudaSuccess) { delete p; return MLORA_ERR_CUDA; }

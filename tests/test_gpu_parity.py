@@ -340,6 +340,14 @@ def test_stream_ordered_plans_from_the_pool(sess):
         # a pooled plan may also be destroyed the ordinary way
         plan = mb.mlora_plan_create_async(sess.ctx, w0.segments, w0.n_rows, 5)
         mb.mlora_plan_destroy(plan)
+        # stream-ordered plans with per-adapter ranks (all 16 here, the layer's own): the same bits as the plain plan's
+        w = tables[5]
+        plan = mb.mlora_plan_create_ranked_async(sess.ctx, w.segments, w.n_rows, 5, [16] * 5)
+        y3 = torch.zeros_like(outs[5])
+        mb.mlora_mixed_forward(sess.ctx, run.layer, plan, run.X, y3, run.x_save, run.u_save, 0, run.capacity)
+        mb.mlora_plan_release(plan)
+        torch.cuda.synchronize()
+        assert torch.equal(y3, outs[5])
     finally:
         run.close()
 
