@@ -114,11 +114,12 @@ struct SchedEntry {
   bool use = false;                     // false: round robin is as good for this shape
   cudaEvent_t filled = nullptr;         // recorded behind the copy that fills the device list
   cudaStream_t stream = nullptr;        // the stream of that copy
-  std::vector<int32_t> host;            // source of that copy
 };
 struct SchedCache {
   std::mutex mu;
   int32_t* dev = nullptr;               // [kSchedSlots][kSchedCap], nullptr: nothing reserved (even row space)
+  int32_t* mirror = nullptr;            // the same area in pinned host memory: source of the copies (a copy from
+                                        // pageable memory would make the runtime wait for the stream first)
   int32_t n = 0;
   int32_t lc_spread = 0;                // most minus fewest adapter groups of a 256-row tile
   SchedEntry e[kSchedSlots];
@@ -162,6 +163,7 @@ struct mlora_plan {
   bool pooled = false;
   DevRowSpace fwd, bwd;
   SchedCache sched[2];               // unit lists of the forward and the compact row space
+  int32_t* sched_pinned = nullptr;   // plans that are not pooled: pinned mirror of the unit-list areas (pooled plans use buf.pinned)
   const int32_t* slot_chunk_off = nullptr;
   const int32_t* chunk_row0 = nullptr;
   const int32_t* chunk_nrows = nullptr;
@@ -770,7 +772,7 @@ void balanced_units(mlora_ctx* ctx, const RowSpace& hs, const DevRowSpace& ds, i
                     cudaStream_t st) {
   g.unit_list = nullptr; g.sched_pairs = 0;
   SchedCache* sc = ds.sched;
-  if (!sc || !sc->dev || ctx->no_unit_lists || !g.lora_enabled) return;
+  if (!sc || !sc->dev || !sc->mirror || ctx->no_unit_lists || !g.lora_enabled) return;
   if ((int64_t)sc->lc_spread * R < 2 * 64) return;          // tiles differ by less than two K-blocks
   const int pairs = g.n_units < ctx->sm_count / 2 ? g.n_units : ctx->sm_count / 2;
   if (pairs < 2 || g.n_units + pairs + 1 > kSchedCap) return;
@@ -825,16 +827,16 @@ void balanced_units(mlora_ctx* ctx, const RowSpace& hs, const DevRowSpace& ds, i
                    g.n_mtiles, g.n_ntiles, kblocks, R, (long long)rr_max, (long long)lpt_max, e->use ? "list" : "round robin");
     slot = sc->n;
     if (e->use) {
-      e->host.assign(pairs + 1, 0);            // offsets (into this same array), then each pair's units in tile order
+      int32_t* list = sc->mirror + (size_t)slot * kSchedCap;      // offsets (into this same array), then each pair's units in tile order
+      int32_t at = pairs + 1;
       for (int p = 0; p < pairs; ++p) {
         std::sort(mine[p].begin(), mine[p].end());
-        e->host[p] = (int32_t)e->host.size();
-        e->host.insert(e->host.end(), mine[p].begin(), mine[p].end());
+        list[p] = at;
+        for (int32_t u : mine[p]) list[at++] = u;
       }
-      e->host[pairs] = (int32_t)e->host.size();
+      list[pairs] = at;
       if (cudaEventCreateWithFlags(&e->filled, cudaEventDisableTiming) != cudaSuccess ||
-          cudaMemcpyAsync(sc->dev + (size_t)slot * kSchedCap, e->host.data(), e->host.size() * sizeof(int32_t),
-                          cudaMemcpyHostToDevice, st) != cudaSuccess ||
+          cudaMemcpyAsync(sc->dev + (size_t)slot * kSchedCap, list, (size_t)at * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess ||
           cudaEventRecord(e->filled, st) != cudaSuccess) {
         cudaGetLastError();
         e->use = false;
@@ -1253,15 +1255,18 @@ size_t sched_reserve(mlora_plan* p) {
   }
   return words;
 }
-// Points the unit-list areas at the reserved words that start at word `at` of the blob.
-void bind_sched(mlora_plan* p, size_t at) {
+// Points the unit-list areas at the reserved words that start at word `at` of the blob, and their pinned mirrors at
+// `mirror` (which holds the reserved words only; nullptr: no lists for this plan).
+void bind_sched(mlora_plan* p, size_t at, int32_t* mirror) {
   const RowSpace* rs[2] = {&p->h.fwd, &p->h.bwd};
   DevRowSpace* ds[2] = {&p->fwd, &p->bwd};
+  size_t m = 0;
   for (int i = 0; i < 2; ++i) {
     ds[i]->sched = &p->sched[i];
-    if (rs[i]->tile2_grp_off.size() > 2 && p->sched[i].lc_spread >= 2) {
-      p->sched[i].dev = p->blob + at;
-      at += (size_t)kSchedSlots * kSchedCap;
+    if (mirror && rs[i]->tile2_grp_off.size() > 2 && p->sched[i].lc_spread >= 2) {
+      p->sched[i].dev = p->blob + at + m;
+      p->sched[i].mirror = mirror + m;
+      m += (size_t)kSchedSlots * kSchedCap;
     }
   }
 }
@@ -1367,8 +1372,12 @@ mlora_status_t mlora_plan_create_ranked(mlora_ctx* ctx, const mlora_segment_t* s
       cudaFree(p->blob); delete p; return MLORA_ERR_CUDA;
     }
     bind_plan(p, o);
-    bind_sched(p, b.data.size());
-    if ((s = grow_workspaces(ctx, p->h, n_rows)) != MLORA_OK) { cudaFree(p->blob); delete p; return s; }
+    if (reserve && cudaMallocHost(&p->sched_pinned, reserve * sizeof(int32_t)) != cudaSuccess) {
+      cudaGetLastError();
+      p->sched_pinned = nullptr;          // no pinned memory: this plan's tiles are dealt out round robin
+    }
+    bind_sched(p, b.data.size(), p->sched_pinned);
+    if ((s = grow_workspaces(ctx, p->h, n_rows)) != MLORA_OK) { mlora_plan_destroy(p); return s; }
   }
   *out = p;
   return MLORA_OK;
@@ -1424,7 +1433,7 @@ mlora_status_t mlora_plan_create_ranked_async(mlora_ctx* ctx, const mlora_segmen
     free_plan_buf(p->buf); delete p; return MLORA_ERR_CUDA;
   }
   bind_plan(p, o);
-  bind_sched(p, tables);
+  bind_sched(p, tables, p->buf.pinned + tables);
   if ((s = grow_workspaces(ctx, p->h, n_rows)) != MLORA_OK) { free_plan_buf(p->buf); delete p; return s; }
   *out = p;
   return MLORA_OK;
@@ -1447,6 +1456,7 @@ void mlora_plan_destroy(mlora_plan* p) {
   if (p->ctx) cudaSetDevice(p->ctx->device);
   if (p->pooled) free_plan_buf(p->buf);
   else if (p->blob) cudaFree(p->blob);
+  if (p->sched_pinned) cudaFreeHost(p->sched_pinned);
   delete p;
 }
 
