@@ -74,12 +74,12 @@ struct mlora_ctx {
   std::vector<PlanBuf> plan_pool;    // released buffers of stream-ordered plans
   int64_t launches = 0;
   int32_t gemm_path = 0;
-  int32_t shrink_path = 0;           // 0: streaming shrink for rank <= 64 (gradients: <= 32); 1: per-item kernels for every rank
+  int32_t shrink_path = 0;           // 0: default choice by rank (streaming mma.sync kernels, tcgen05 kernels from rank 64); 1: per-item kernels for every rank
   int32_t gemm_pairs = 1;            // 1: two-SM (CTA pair) tensor-core kernel; 0: one-SM kernel
   int32_t no_split_k = 0;            // 1: the two-SM kernel never splits K (kernel variant 4)
   int32_t no_unit_lists = 0;         // 1: the two-SM kernel always deals its units out round robin (kernel variant 7)
   int32_t grad_mode = 0;             // 0: default choice by rank; 1: mma.sync kernels for every rank (kernel variant 5);
-                                     // 2: the tcgen05 gradient kernel for every rank (kernel variant 6)
+                                     // 2: the tcgen05 shrink and gradient kernels for every rank (kernel variant 6)
   EncodeTiledFn encode = nullptr;
   const volatile int32_t* cancel = nullptr;   // caller's host flag, read before every launch
   DropArgs drop = {0, 0, 1.0f};               // LoRA dropout of the fine-tuning rows (thr == 0: off)

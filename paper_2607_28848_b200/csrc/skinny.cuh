@@ -1,17 +1,20 @@
-// Rank-r ("skinny") kernels of the multi-LoRA layer for bf16 storage.  They are bound by the bytes of
-// the wide operand they stream once from HBM; the rank-r contraction itself runs on the warp-level
-// tensor-core instruction (mma.sync m16n8k16, fp32 accumulate) because at rank 16 and above the CUDA
-// cores could not keep up with the memory system.
+// Rank-r ("skinny") kernels of the multi-LoRA layer for bf16 storage, mma.sync family.  They are bound by
+// the bytes of the wide operand they stream once from HBM; the rank-r contraction itself runs on the
+// warp-level tensor-core instruction (mma.sync m16n8k16, fp32 accumulate) because at rank 16 and above the
+// CUDA cores could not keep up with the memory system.  These are the defaults up to rank 32 and, at every
+// rank, wherever the rows pass through registers for a reason: gathered decode rows, the dropout mask.
+// Ranks 64 and 128 otherwise run on the tcgen05 kernels of shrink_tc.cuh and grad_tc.cuh.
 //
 //  shrink : Out[t, q] = sum_k In[t, k] * P_a(t)[q, k]      (U = X A^T  and  V = s dY B^T)
 //           work item = up to 32 rows that share one adapter, GATHERED by adapter id (they need not be
 //           adjacent: decode rows of one adapter form one item, prefill and fine-tune segments are
 //           runs of items); optionally copies the rows of In and the result into the fine-tuning
 //           activation buffers on the way.
-//           shrink_stream_kernel (rank <= 64, the default): persistent, stages filled by the copy engine;
-//           shrink_kernel (rank 128): one CTA per item, operands straight from global memory.
+//           shrink_stream_kernel (rank <= 64): persistent, stages filled by the copy engine;
+//           shrink_kernel (every rank; the only mma.sync shrink at rank 128): one CTA per item, operands
+//           straight from global memory.
 //  grad   : G_g[q, j] = sum_{rows t of slot g} P[t, q] * Q[t, j]   (dB = (s U)^T dY, dA = V^T X)
-//           grad_stream_kernel (rank <= 64: both gradients in one launch); grad_kernel (rank 128).
+//           grad_stream_kernel (rank <= 64: both gradients in one launch); grad_kernel (every rank, per strip).
 //  expand_mask_kernel : the low-rank part of the input gradient under dropout.
 #pragma once
 
