@@ -112,8 +112,8 @@ void mlora_destroy(mlora_ctx* ctx);
  * MLORA_ERR_INVALID_ARG, MLORA_ERR_CUDA. */
 mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, int32_t n_segs,
                                  int32_t n_rows, int32_t n_adapters, mlora_plan** plan);
-/* The same plan for adapters that have ranks of their own (Section 5 serves and trains adapters of
- * different ranks side by side).  adapter_rank: HOST array [n_adapters], 1 <= r_a <= 128; NULL makes
+/* The same plan for adapters that have ranks of their own (Section 2.2: a serving system hosts many
+ * adapters over one frozen base model; nothing makes them share a rank).  adapter_rank: HOST array [n_adapters], 1 <= r_a <= 128; NULL makes
  * this call mlora_plan_create.  Storage does not change: every adapter still occupies `rank` rows of
  * A_all and B_all in each layer, rows r_a .. rank - 1 zero, and gradients come back in that shape with
  * those rows zero.  What changes is the work: in the base product's fused expand a group of rows is

@@ -304,7 +304,8 @@ def backward(dY, W, A_all, B_all, scale, segments, x_save, u_save, n_rows: Optio
 
 
 def backward_ragged(dY, W, A_list, B_list, scale, segments, x_save, n_rows: int):
-    """Gradients when adapter a has its own rank r_a (Section 5 trains adapters of different ranks side by side):
+    """Gradients when adapter a has its own rank r_a (Section 2.2: many adapters share one base model; nothing makes
+    them share a rank):
     the same chain rule as ``backward`` with each adapter's own matrices, nothing padded.  ``u`` is recomputed
     from the saved input (u = A_a x), since saved rows of different adapters would have different widths.
     Returns ``dA`` and ``dB`` as lists (slot g: [r_a, d_in] and [r_a, d_out]), ``dX`` [ft_rows, d_in] and
