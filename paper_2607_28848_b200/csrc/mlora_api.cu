@@ -147,6 +147,7 @@ struct DevRowSpace {
   const int32_t* tcb_row0 = nullptr;
   const int32_t* tcb_nrows = nullptr;
   const int32_t* tcb_adapter = nullptr;
+  const int32_t* tcb_width = nullptr;      // plans made with per-adapter ranks (null otherwise)
   // plans made with per-adapter ranks (null otherwise)
   const int32_t* grp2_col = nullptr;
   const int32_t* grp2_width = nullptr;
@@ -507,12 +508,18 @@ mlora_status_t launch_shrink_tc(mlora_ctx* ctx, const RowSpace& hs, const DevRow
       attr_set = true;
     }
   }
-  CUtensorMap tQ, tB;
+  CUtensorMap tQ, tB, tB16, tB32, tB64;
   mlora_status_t ms;
   if ((ms = make_tmap_bf16_blocked(ctx, &tQ, In, n_rows, D, ld_in, stc::ROWS, C::CB)) != MLORA_OK) return ms;
   if ((ms = make_tmap_bf16_blocked(ctx, &tB, P_all, (uint64_t)n_adapters * R, D, D, C::RP, C::CB)) != MLORA_OK) return ms;
+  tB16 = tB; tB32 = tB; tB64 = tB;
+  if (ds.tcb_width) {      // plans with per-adapter ranks: a block reads only as many rows of its adapter's matrix as the rank needs
+    if ((ms = make_tmap_bf16_blocked(ctx, &tB16, P_all, (uint64_t)n_adapters * R, D, D, 16, C::CB)) != MLORA_OK) return ms;
+    if (C::RP > 32 && (ms = make_tmap_bf16_blocked(ctx, &tB32, P_all, (uint64_t)n_adapters * R, D, D, 32, C::CB)) != MLORA_OK) return ms;
+    if (C::RP > 64 && (ms = make_tmap_bf16_blocked(ctx, &tB64, P_all, (uint64_t)n_adapters * R, D, D, 64, C::CB)) != MLORA_OK) return ms;
+  }
   stc::Args a;
-  a.blk_row0 = ds.tcb_row0; a.blk_nrows = ds.tcb_nrows; a.blk_adapter = ds.tcb_adapter;
+  a.blk_row0 = ds.tcb_row0; a.blk_nrows = ds.tcb_nrows; a.blk_adapter = ds.tcb_adapter; a.blk_width = ds.tcb_width;
   a.NB = (int)hs.tcb_row0.size(); a.NS = (D + C::COLS - 1) / C::COLS;
   a.part_ws = ctx->ws_tc_part; a.status = ctx->status_dev;
   const int64_t tiles = (int64_t)a.NB * a.NS;
@@ -520,10 +527,10 @@ mlora_status_t launch_shrink_tc(mlora_ctx* ctx, const RowSpace& hs, const DevRow
   if (cancelled(ctx)) return MLORA_CANCELLED;
   {
     LaunchScope scope(ctx, st, KIND_SHRINK);
-    launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(stc::THREADS), C::SMEM_BYTES, st, tQ, tB, a);
+    launch_pdl(scope.slot < 0, kern, dim3(grid), dim3(stc::THREADS), C::SMEM_BYTES, st, tQ, tB, tB16, tB32, tB64, a);
     if ((ms = scope.done()) != MLORA_OK) return ms;
   }
-  fa.blk_row0 = a.blk_row0; fa.blk_nrows = a.blk_nrows; fa.blk_adapter = a.blk_adapter;
+  fa.blk_row0 = a.blk_row0; fa.blk_nrows = a.blk_nrows; fa.blk_adapter = a.blk_adapter; fa.blk_width = a.blk_width;
   fa.NB = a.NB; fa.NS = a.NS; fa.G = grid; fa.part_ws = ctx->ws_tc_part;
   const int zero_ctas = fa.pbd.pbd ? (fa.pbd.n_zero_rows + C::FIN_ROWS - 1) / C::FIN_ROWS : 0;
   if (cancelled(ctx)) return MLORA_CANCELLED;
@@ -1216,7 +1223,7 @@ void mlora_destroy(mlora_ctx* c) {
 
 namespace {
 
-constexpr int kPlanTables = 53;
+constexpr int kPlanTables = 55;
 
 // All device tables of a plan, packed; o[] receives each table's offset in 32-bit words.
 void pack_plan(const HostPlan& h, BlobBuilder& b, size_t* o) {
@@ -1232,6 +1239,7 @@ void pack_plan(const HostPlan& h, BlobBuilder& b, size_t* o) {
     o[n++] = b.add(rs[i]->tcb_row0); o[n++] = b.add(rs[i]->tcb_nrows); o[n++] = b.add(rs[i]->tcb_adapter);
     o[n++] = b.add(rs[i]->grp2_col); o[n++] = b.add(rs[i]->grp2_width); o[n++] = b.add(rs[i]->tile2_cols);
     o[n++] = b.add(rs[i]->tile2_piece_off); o[n++] = b.add(rs[i]->piece_src);
+    o[n++] = b.add(rs[i]->tcb_width);
   }
   o[n++] = b.add(h.slot_chunk_off); o[n++] = b.add(h.chunk_row0); o[n++] = b.add(h.chunk_nrows);
   o[n++] = b.add(h.ft_adapters);
@@ -1289,6 +1297,7 @@ void bind_plan(mlora_plan* p, const size_t* o) {
     ds[i]->tile2_cols = ranked ? p->blob + o[n] : nullptr; ++n;
     ds[i]->tile2_piece_off = ranked ? p->blob + o[n] : nullptr; ++n;
     ds[i]->piece_src = ranked ? p->blob + o[n] : nullptr; ++n;
+    ds[i]->tcb_width = ranked ? p->blob + o[n] : nullptr; ++n;
   }
   p->bwd.row_save = nullptr;       // the compact space has no save offsets
   p->slot_chunk_off = p->blob + o[n++]; p->chunk_row0 = p->blob + o[n++]; p->chunk_nrows = p->blob + o[n++];

@@ -50,6 +50,7 @@ struct RowSpace {
   // tile's operand; the operand's rows on the B side are 16-row PIECES of the adapters' matrices, listed per
   // tile in column order: piece_src = adapter << 8 | (first row of the piece inside the adapter / 16).
   std::vector<int32_t> grp2_col, grp2_width, tile2_cols, tile2_piece_off, piece_src;
+  std::vector<int32_t> tcb_width;      // [blocks] rows of the adapter's matrix a block of the tensor-core shrink reads: its rank rounded up to 16, 32, 64 or 128
   int32_t n_tiles() const { return (n_rows + kTileRows - 1) / kTileRows; }
   int32_t n_items() const { return (int32_t)item_start.size(); }
 };
@@ -97,6 +98,12 @@ inline void build_tile_groups(const std::vector<int32_t>& row_adapter, int32_t t
 inline void build_ranked(RowSpace& rs, const std::vector<int32_t>& adapter_rank) {
   rs.grp2_col.clear(); rs.grp2_width.clear(); rs.tile2_cols.clear(); rs.piece_src.clear();
   rs.tile2_piece_off.assign(1, 0);
+  rs.tcb_width.clear();
+  for (int32_t a : rs.tcb_adapter) {
+    int32_t w = 16;
+    while (w < adapter_rank[a]) w *= 2;
+    rs.tcb_width.push_back(w);
+  }
   for (size_t t = 0; t + 1 < rs.tile2_grp_off.size(); ++t) {
     int32_t col = 0;
     for (int32_t i = rs.tile2_grp_off[t]; i < rs.tile2_grp_off[t + 1]; ++i) {

@@ -57,6 +57,7 @@ struct Args {
   const int32_t* blk_row0;       // [NB] first row of the block
   const int32_t* blk_nrows;      // [NB] 1 .. 128
   const int32_t* blk_adapter;    // [NB]
+  const int32_t* blk_width;      // nullable (plans with per-adapter ranks): [NB] rows of the adapter's matrix the block needs, 16 / 32 / 64 / 128
   int32_t NB, NS;                // blocks, column strips per block
   float* part_ws;                // [rows + 128 * grid][R] fp32 sums of the runs
   int32_t* status;
@@ -66,6 +67,7 @@ struct FinArgs {
   const int32_t* blk_row0;
   const int32_t* blk_nrows;
   const int32_t* blk_adapter;
+  const int32_t* blk_width;      // nullable: columns of the result that exist (the rest is written as zero)
   int32_t NB, NS, G;             // G: grid of the main kernel
   const float* part_ws;
   const float* scale;            // nullable: Out (and the operand chunks) multiplied by scale[adapter]
@@ -86,7 +88,11 @@ __host__ __device__ __forceinline__ int owner(int t, int G, int N) { return (int
 
 template <int R>
 __global__ void __launch_bounds__(THREADS, 1)
-shrink_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmB, const Args a) {
+shrink_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmB,
+                 const __grid_constant__ CUtensorMap tmB16, const __grid_constant__ CUtensorMap tmB32,
+                 const __grid_constant__ CUtensorMap tmB64, const Args a) {
+  // tmB has boxes of RP rows (the whole padded adapter); tmB16 / 32 / 64 boxes of that many rows, for blocks whose
+  // adapter has a smaller rank of its own (a.blk_width)
   using C = Cfg<R>;
   constexpr int RP = C::RP, CB = C::CB, S = C::S;
   extern __shared__ uint8_t smem_raw[];
@@ -114,6 +120,7 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmQ);
     ptx::prefetch_tmap(&tmB);
+    if (a.blk_width) { ptx::prefetch_tmap(&tmB16); ptx::prefetch_tmap(&tmB32); ptx::prefetch_tmap(&tmB64); }
   }
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_u32(tmem_ptr_smem), C::TMEM_COLS);
@@ -128,8 +135,9 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   if (warp == 0) {
     // ================================ TMA producer ================================
     int blk = t0 < t1 ? t0 / a.NS : 0, strip = t0 - blk * a.NS;
-    int row0 = 0, brow = 0;
-    if (t0 < t1) { row0 = a.blk_row0[blk]; brow = a.blk_adapter[blk] * R; }     // plan tables: readable before the wait
+    int row0 = 0, brow = 0, bw = RP;
+    auto width_of = [&](int b) { const int w = a.blk_width ? a.blk_width[b] : RP; return w < RP ? w : RP; };
+    if (t0 < t1) { row0 = a.blk_row0[blk]; brow = a.blk_adapter[blk] * R; bw = width_of(blk); }   // plan tables: readable before the wait
     ptx::grid_dependency_wait();             // the workspace may still be read by the launch before the last
     ptx::grid_launch_dependents();
     if (lane == 0) {
@@ -137,12 +145,14 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       for (int t = t0, i = 0; t < t1 && ok; ++t, ++i) {
         const int s = i % S;
         if (!(ok = gemm_wait(bar_empty(s), ((i / S) & 1) ^ 1, abort_flag, a.status))) break;
-        ptx::mbar_arrive_expect_tx(bar_full(s), C::STAGE_BYTES);
+        ptx::mbar_arrive_expect_tx(bar_full(s), C::Q_BYTES + (uint32_t)(CB * bw * 128));
         ptx::tma_load_3d(s_stage(s), &tmQ, 0, row0, strip * CB, bar_full(s));
-        ptx::tma_load_3d(s_stage(s) + C::Q_BYTES, &tmB, 0, brow, strip * CB, bar_full(s));
+        // the adapter's rows over the tile's columns: [CB][bw rows][128 B]
+        const CUtensorMap* mb = bw >= RP ? &tmB : (bw == 16 ? &tmB16 : (bw == 32 ? &tmB32 : &tmB64));
+        ptx::tma_load_3d(s_stage(s) + C::Q_BYTES, mb, 0, brow, strip * CB, bar_full(s));
         if (++strip == a.NS && t + 1 < t1) {
           strip = 0; ++blk;
-          row0 = a.blk_row0[blk]; brow = a.blk_adapter[blk] * R;
+          row0 = a.blk_row0[blk]; brow = a.blk_adapter[blk] * R; bw = width_of(blk);
         }
       }
     }
@@ -150,11 +160,18 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   } else if (warp == 1) {
     // ================================ MMA issuer ================================
     if (lane == 0) {
-      constexpr uint32_t idesc = ptx::make_idesc_bf16(128, RP, false, false);
       uint32_t n_run = 0;
       bool ok = true;
+      int cur_blk = -1, bw = RP;
+      uint32_t idesc = ptx::make_idesc_bf16(128, RP, false, false);
       for (int t = t0, i = 0; t < t1 && ok; ++t, ++i) {
         const int s = i % S, blk = t / a.NS, strip = t - blk * a.NS;
+        if (blk != cur_blk) {                  // N = the rows of the adapter's matrix this block reads
+          cur_blk = blk;
+          const int w = a.blk_width ? a.blk_width[blk] : RP;
+          bw = w < RP ? w : RP;
+          idesc = ptx::make_idesc_bf16(128, (uint32_t)bw, false, false);
+        }
         const bool first = t == t0 || strip == 0, last = t == t1 - 1 || strip == a.NS - 1;
         const int v = n_run & 1;
         if (first && !(ok = gemm_wait(bar_vempty(v), ((n_run >> 1) & 1) ^ 1, abort_flag, a.status))) break;
@@ -165,7 +182,7 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
         for (int cb = 0; cb < CB; ++cb) {
           const uint64_t ad = ptx::make_smem_desc(q + (uint32_t)cb * C::BLK, 16, 1024);
-          const uint64_t bd = ptx::make_smem_desc(q + C::Q_BYTES + (uint32_t)cb * (RP * 128u), 16, 1024);
+          const uint64_t bd = ptx::make_smem_desc(q + C::Q_BYTES + (uint32_t)cb * ((uint32_t)bw * 128u), 16, 1024);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) {
             ptx::umma_f16(d, ad + (uint64_t)(ks * 2), bd + (uint64_t)(ks * 2), idesc, acc);
@@ -188,6 +205,7 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const int blk = t / a.NS, strip0 = t - blk * a.NS;
       const int len = min(a.NS - strip0, t1 - t);           // this run: strips strip0 .. strip0 + len of the block
       const int nrows = a.blk_nrows[blk];
+      const int bwid = a.blk_width ? min(a.blk_width[blk], RP) : RP;       // columns that exist (the same for the whole warp)
       float* dst = a.part_ws + ((size_t)a.blk_row0[blk] + (size_t)128 * cta + trow) * R;
       const int v = n_run & 1;
       if (!(ok = __all_sync(0xffffffffu, gemm_wait(bar_vfull(v), (n_run >> 1) & 1, abort_flag, a.status)))) break;
@@ -196,6 +214,7 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       constexpr int QC = R < 64 ? (R < 16 ? 16 : R) : 64;   // columns per round of loads
 #pragma unroll
       for (int q0 = 0; q0 < RP; q0 += QC) {
+        if (q0 >= bwid) break;
         uint32_t vv[QC];
 #pragma unroll
         for (int c0 = 0; c0 < QC; c0 += 16) ptx::tmem_ld_32x32b_x16(tmem_base + tlane + (uint32_t)(v * RP + q0 + c0), vv + c0);
@@ -203,7 +222,7 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (trow < nrows) {
 #pragma unroll
           for (int c0 = 0; c0 < QC; c0 += 4)
-            if (q0 + c0 < R)
+            if (q0 + c0 < R && q0 + c0 < bwid)
               *reinterpret_cast<float4*>(dst + q0 + c0) = make_float4(__uint_as_float(vv[c0]), __uint_as_float(vv[c0 + 1]),
                                                                       __uint_as_float(vv[c0 + 2]), __uint_as_float(vv[c0 + 3]));
         }
@@ -250,6 +269,7 @@ shrink_tc_finish_kernel(const FinArgs a) {
   if ((int)blockIdx.y * FIN_ROWS >= nrows) return;
   const int r = (int)blockIdx.y * FIN_ROWS + r_in;
   const bool live = r < nrows;
+  const bool exists = !a.blk_width || 4 * j < a.blk_width[blk];     // columns past the adapter's own rank: zero, nothing to add
   const int row0 = a.blk_row0[blk], row = row0 + (live ? r : 0);
   const int ad = a.blk_adapter[blk];
   const float sc = a.scale ? a.scale[ad] : 1.0f;
@@ -286,7 +306,7 @@ shrink_tc_finish_kernel(const FinArgs a) {
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
         const int cc = c0 + k;
-        x[k] = (live && cc <= c_last) ? __ldcg(reinterpret_cast<const float4*>(src + (size_t)128 * cc * R))
+        x[k] = (live && exists && cc <= c_last) ? __ldcg(reinterpret_cast<const float4*>(src + (size_t)128 * cc * R))
                                       : make_float4(0.f, 0.f, 0.f, 0.f);
       }
 #pragma unroll
