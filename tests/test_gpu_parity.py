@@ -124,6 +124,14 @@ def test_k_split_of_the_last_wave_only(sess, d_in, d_out):
     run_and_check(sess, w, t, path=4, blocked=True)
 
 
+@pytest.mark.parametrize("rank", [64, 128])
+def test_high_rank_large_batch(sess, rank):
+    """8192 rows over 40 adapters at rank 64 / 128 (2048 -> 4096): the tcgen05 shrink with a few hundred blocks and runs
+    shared by several CTAs, its finish kernel's zero rows, the operand images of ~30 gradient blocks, unit lists."""
+    w = synth.random_workload(500 + rank, 2048, 4096, rank, 40, 8192, max_seg=300, p_decode=0.35, p_finetune=0.4)
+    run_and_check(sess, w, synth.make_tensors(w), blocked=True)
+
+
 @pytest.mark.parametrize("rank", [32, 128])
 def test_row_tiles_of_unequal_cost_get_balanced_unit_lists(sess, rank):
     """One 256-row tile of 200 single-row adapters between tiles of one group each: the heavy tile carries
