@@ -120,8 +120,9 @@ mlora_status_t mlora_plan_create(mlora_ctx* ctx, const mlora_segment_t* segs, in
  * as wide as its adapter's rank rounded up to 16, not as wide as the layer's padded rank, so the
  * extra K-blocks of a 256-row tile number ceil(sum of those widths / 64) instead of
  * ceil(groups * rank / 64); and the tcgen05 shrink (layer ranks 64 and 128) reads, per block of rows,
- * only the first 16 / 32 / 64 / 128 rows of the adapter's matrices that its rank needs.  (The
- * mma.sync shrink and the gradient kernels still run over all `rank` rows.)
+ * only the first 16 / 32 / 64 / 128 rows of the adapter's matrices that its rank needs, and the
+ * tcgen05 gradient kernel contracts only those rows of a slot's gradient (the rest is written as
+ * zero).  (The mma.sync kernels of the lower layer ranks still run over all `rank` rows.)
  * A plan made this way serves layers with rank % 16 == 0 and rank >= every r_a; other layers are
  * refused by the compute calls with MLORA_ERR_INVALID_ARG.  Errors as mlora_plan_create, plus
  * MLORA_ERR_INVALID_ARG for a rank outside [1, 128]. */

@@ -87,6 +87,9 @@ struct Args {
   int32_t snap;                  // ranges end at strip boundaries (no partial pieces)
   int32_t* status;
   const uint8_t* pop;            // nullable: the P operands made ahead by psplit_kernel, [2 problems][NB][P_BYTES]
+  const int32_t* slot_width;     // nullable (plans with per-adapter ranks, and only with pop): rank rows of a slot's gradient
+                                 // that exist, w = 16 / 32 / 64 / 128; its operand image is then [2][2 w rows][128 B] (head | remainder
+                                 // of w columns each), the MMAs have N = 2 w, and rows w .. R - 1 of the gradient are zero
 };
 
 // Position in one problem's tile list (slot > strip > block).
@@ -162,9 +165,12 @@ psplit_kernel(const Args a, uint8_t* pop) {
   const int nrows = a.blk_nrows[blk], row0 = a.blk_row0[blk];
   const bool live = trow < nrows;
   const float sc = pr.scale ? pr.scale[a.slot_adapter[slot]] : 1.0f;
+  const int w = a.slot_width ? (a.slot_width[slot] < R ? a.slot_width[slot] : R) : R;     // columns that exist
+  if ((int)blockIdx.z * psplit_cols(R) >= w) return;
+  const int n2 = a.slot_width ? 2 * w : N2;                                                 // rows of a K-block of the image
   ptx::grid_dependency_wait();               // V comes from the launch before
   ptx::grid_launch_dependents();
-  uint8_t* img = pop + ((size_t)p * a.NB + blk) * C::P_BYTES + (size_t)(trow >> 6) * (N2 * 128u);
+  uint8_t* img = pop + ((size_t)p * a.NB + blk) * C::P_BYTES + (size_t)(trow >> 6) * ((uint32_t)n2 * 128u);
   const uint32_t kk = (uint32_t)(trow & 63);
   const float4* src = reinterpret_cast<const float4*>(pr.P + (size_t)(row0 + (live ? trow : 0)) * R);
   constexpr int QC = psplit_cols(R);
@@ -180,15 +186,16 @@ psplit_kernel(const Args a, uint8_t* pop) {
 #pragma unroll
     for (int c = 0; c < QC; ++c) {
       const int qq = q0 + c;
+      if (qq >= w) break;                    // a narrower image ends here (its remainder rows start at w)
       const __nv_bfloat16 hi = __float2bfloat16_rn(pv[c]);
       const uint32_t off_hi = (uint32_t)qq * 128u + ((((kk >> 3) ^ (uint32_t)(qq & 7)) << 4) | ((kk & 7u) << 1));
       *reinterpret_cast<__nv_bfloat16*>(img + off_hi) = hi;
       const __nv_bfloat16 lo = __float2bfloat16_rn(pv[c] - __bfloat162float(hi));
-      const uint32_t off_lo = (uint32_t)(R + qq) * 128u + ((((kk >> 3) ^ (uint32_t)((R + qq) & 7)) << 4) | ((kk & 7u) << 1));
+      const uint32_t off_lo = (uint32_t)(w + qq) * 128u + ((((kk >> 3) ^ (uint32_t)((w + qq) & 7)) << 4) | ((kk & 7u) << 1));
       *reinterpret_cast<__nv_bfloat16*>(img + off_lo) = lo;
     }
   }
-  if (2 * R < N2 && blockIdx.z == 0) {       // (N2 = 2 R for every rank offered; kept for the layout's sake)
+  if (2 * R < N2 && blockIdx.z == 0 && !a.slot_width) {       // (N2 = 2 R for every rank offered; kept for the layout's sake)
     for (int qq = 2 * R; qq < N2; ++qq)
       *reinterpret_cast<__nv_bfloat16*>(img + (uint32_t)qq * 128u + ((((kk >> 3) ^ (uint32_t)(qq & 7)) << 4) | ((kk & 7u) << 1))) =
           __float2bfloat16_rn(0.f);
@@ -274,7 +281,6 @@ grad_tc_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_constant__
     __syncwarp();
   } else if (warp == 1) {
     // ================================ MMA issuer ================================
-    constexpr uint32_t idesc = ptx::make_idesc_bf16(128, N2, true, false);
     uint32_t i = 0, n_piece = 0;
     bool ok = true;
     // the whole warp waits (one decision for all lanes); lane 0 issues
@@ -290,6 +296,8 @@ grad_tc_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_constant__
         const int s = i % S, pb = i % NPB, ab = n_piece & 1;
         const bool first_piece = t == t0 || it.blk == 0, last_piece = t == t1 - 1 || it.blk == it.nb - 1;
         const int nrows = a.blk_nrows[it.b0 + it.blk];
+        const int n2 = a.slot_width ? 2 * min(a.slot_width[it.slot], R) : N2;      // operand rows per K-block = the MMAs' N
+        const uint32_t idesc = ptx::make_idesc_bf16(128, (uint32_t)n2, true, false);
         if (!(ok = wait_all(bar_pfull(pb), (i / NPB) & 1))) break;
         if (!(ok = wait_all(bar_full(s), (i / S) & 1))) break;
         const uint32_t q = s_stage(s);
@@ -314,7 +322,7 @@ grad_tc_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_constant__
             const uint32_t d = tmem_base + (uint32_t)(ab * C::ACC_COLS + mb * N2);
             const uint64_t ad = ptx::make_smem_desc(q + (uint32_t)(2 * mb) * C::BLK, C::BLK, 1024);
             for (int ks = 0; ks < ksteps; ++ks)      // K-step ks: rows 16 ks .. of the tile; P's K-block ks / 4, 32 bytes per step inside it
-              ptx::umma_f16(d, ad + (uint64_t)(ks * 128), bd0 + (uint64_t)((ks >> 2) * (N2 * 8) + (ks & 3) * 2), idesc,
+              ptx::umma_f16(d, ad + (uint64_t)(ks * 128), bd0 + (uint64_t)((ks >> 2) * (n2 * 8) + (ks & 3) * 2), idesc,
                             (ks == 0 && first_piece) ? 0u : 1u);
           }
           ptx::umma_commit(bar_empty(s));
@@ -355,8 +363,9 @@ grad_tc_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_constant__
           const int pb = ic % NPB;
           if (!__all_sync(0xffffffffu, gemm_wait(bar_pempty(pb), ((ic / NPB) & 1) ^ 1, abort_flag, a.status))) return false;
           if (tid == 0) {
-            ptx::mbar_arrive_expect_tx(bar_pfull(pb), C::P_BYTES);
-            bulk_load(s_pbuf(pb), a.pop + ((size_t)p * a.NB + blk_abs) * C::P_BYTES, C::P_BYTES, bar_pfull(pb));
+            const uint32_t bytes = a.slot_width ? 512u * (uint32_t)min(a.slot_width[it.slot], R) : C::P_BYTES;   // [2][2 w][128 B]
+            ptx::mbar_arrive_expect_tx(bar_pfull(pb), bytes);
+            bulk_load(s_pbuf(pb), a.pop + ((size_t)p * a.NB + blk_abs) * C::P_BYTES, bytes, bar_pfull(pb));
           } else {
             ptx::mbar_arrive(bar_pfull(pb));
           }
@@ -417,6 +426,7 @@ grad_tc_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_constant__
           ptx::tc_fence_after();
           ++n_piece;
           const bool complete = piece_blk0 == 0 && it.blk == it.nb - 1;
+          const int w = a.slot_width ? min(a.slot_width[it.slot], R) : R;  // rank rows that exist: head columns [0, w), remainder [w, 2 w)
           const int gbase = it.b0 * pr.NS + it.strip * it.nb;            // first tile of the (slot, strip)
           float* mine = a.part_ws + ((size_t)cta * 4 + p * 2 + (t0 >= gbase ? 0 : 1)) * C::PIECE_FLOATS;
 #pragma unroll
@@ -429,8 +439,13 @@ grad_tc_kernel(const __grid_constant__ CUtensorMap tmQ0, const __grid_constant__
               uint32_t wh[C::QC < 16 ? 16 : C::QC], wl[C::QC < 16 ? 16 : C::QC];
 #pragma unroll
               for (int c0 = 0; c0 < C::QC; c0 += 16) {
-                ptx::tmem_ld_32x32b_x16(tacc + (uint32_t)(q0 + c0), wh + c0);
-                if (R >= 16) ptx::tmem_ld_32x32b_x16(tacc + (uint32_t)(R + q0 + c0), wl + c0);
+                if (q0 + c0 < w) {
+                  ptx::tmem_ld_32x32b_x16(tacc + (uint32_t)(q0 + c0), wh + c0);
+                  if (R >= 16) ptx::tmem_ld_32x32b_x16(tacc + (uint32_t)(w + q0 + c0), wl + c0);
+                } else {                                                  // rows past the adapter's own rank: zero
+#pragma unroll
+                  for (int z = 0; z < 16; ++z) { wh[c0 + z] = 0u; wl[c0 + z] = 0u; }
+                }
               }
               ptx::tmem_ld_wait();
               // rank 8: one load of 16 columns holds both halves

@@ -172,6 +172,7 @@ struct mlora_plan {
   const int32_t* slot_blk_off = nullptr;
   const int32_t* blk_row0 = nullptr;
   const int32_t* blk_nrows = nullptr;
+  const int32_t* slot_width = nullptr;   // plans made with per-adapter ranks (null otherwise)
 };
 
 namespace {
@@ -634,7 +635,9 @@ mlora_status_t launch_grad_tc(mlora_ctx* ctx, const mlora_layer_t* L, const mlor
   }
   a.snap = (8 * most_snapped <= 9 * most_plain) ? 1 : 0;
   a.pop = nullptr;
+  a.slot_width = nullptr;
   if (a.NB <= ctx->ws_pop_blocks && ctx->ws_pop) {     // both problems' operands once per block, ahead of the kernel
+    a.slot_width = p->slot_width;                      // (ranked plans: only the rows of a gradient that exist)
     if (cancelled(ctx)) return MLORA_CANCELLED;
     LaunchScope scope(ctx, st, KIND_GRAD);
     launch_pdl(scope.slot < 0, gtc::psplit_kernel<R>, dim3(a.NB, 2, R / gtc::psplit_cols(R)), dim3(128), 0, st, a, ctx->ws_pop);
@@ -1223,7 +1226,7 @@ void mlora_destroy(mlora_ctx* c) {
 
 namespace {
 
-constexpr int kPlanTables = 55;
+constexpr int kPlanTables = 56;
 
 // All device tables of a plan, packed; o[] receives each table's offset in 32-bit words.
 void pack_plan(const HostPlan& h, BlobBuilder& b, size_t* o) {
@@ -1244,6 +1247,7 @@ void pack_plan(const HostPlan& h, BlobBuilder& b, size_t* o) {
   o[n++] = b.add(h.slot_chunk_off); o[n++] = b.add(h.chunk_row0); o[n++] = b.add(h.chunk_nrows);
   o[n++] = b.add(h.ft_adapters);
   o[n++] = b.add(h.slot_blk_off); o[n++] = b.add(h.blk_row0); o[n++] = b.add(h.blk_nrows);
+  o[n++] = b.add(h.slot_width);
 }
 
 // Words to reserve behind the plan's tables for unit lists: only row spaces whose 256-row tiles differ in
@@ -1303,6 +1307,7 @@ void bind_plan(mlora_plan* p, const size_t* o) {
   p->slot_chunk_off = p->blob + o[n++]; p->chunk_row0 = p->blob + o[n++]; p->chunk_nrows = p->blob + o[n++];
   p->slot_adapter = p->blob + o[n++];
   p->slot_blk_off = p->blob + o[n++]; p->blk_row0 = p->blob + o[n++]; p->blk_nrows = p->blob + o[n++];
+  p->slot_width = p->h.slot_width.empty() ? nullptr : p->blob + o[n]; ++n;
 }
 
 // Grows the context's workspaces to what this plan needs.  A workspace that is too small is REPLACED

@@ -69,6 +69,7 @@ struct HostPlan {
   // The same rows as blocks of <= kTileRows consecutive compact rows (tiles of the streaming kernel).
   std::vector<int32_t> slot_blk_off;   // [n_slots + 1]
   std::vector<int32_t> blk_row0, blk_nrows;
+  std::vector<int32_t> slot_width;     // ranked plans only: rows of the slot's gradient that exist (its adapter's rank rounded up to 16, 32, 64 or 128)
 };
 
 inline void build_tile_groups(const std::vector<int32_t>& row_adapter, int32_t tile_rows,
@@ -252,6 +253,12 @@ inline mlora_status_t build_plan(const mlora_segment_t* segs, int32_t n_segs, in
     }
     p.slot_blk_off.push_back((int32_t)p.blk_row0.size());
   }
+  if (!p.adapter_rank.empty())
+    for (int32_t a : p.ft_adapters) {
+      int32_t w = 16;
+      while (w < p.adapter_rank[a]) w *= 2;
+      p.slot_width.push_back(w);
+    }
   return MLORA_OK;
 }
 
