@@ -310,10 +310,10 @@ int64_t mlora_launch_count(const mlora_ctx* ctx);
 mlora_status_t mlora_profile_enable(mlora_ctx* ctx, int32_t max_records);
 int32_t mlora_profile_collect(mlora_ctx* ctx, int32_t* kinds, float* ms, int32_t cap);
 
-/* Selects kernel variants for MLORA_BF16 layers: 0 = defaults (two-SM tcgen05 tensor-core GEMM; rank <= 32:
- * streaming mma.sync shrink and gradient kernels; rank 64 and 128: the tcgen05 shrink with its finish
- * kernel for U = X A^T and V = s dY B^T wherever the rows come in runs of four or more per adapter on
- * average, and the tcgen05 gradient kernel); 1 = the plain CUDA-core kernels for every step (a slow
+/* Selects kernel variants for MLORA_BF16 layers: 0 = defaults (two-SM tcgen05 tensor-core GEMM; rank <= 16:
+ * streaming mma.sync shrink and gradient kernels; rank 32, 64 and 128: the tcgen05 shrink with its finish
+ * kernel for U = X A^T and V = s dY B^T wherever the rows come in runs of eight (rank 128: four) or more
+ * per adapter on average, and the tcgen05 gradient kernel); 1 = the plain CUDA-core kernels for every step (a slow
  * cross-check used by the tests); 2 = defaults, but the per-item mma.sync shrink and gradient kernels
  * for every rank; 3 = defaults, but the one-SM tensor-core GEMM;
  * 4 = defaults, but the two-SM GEMM never splits K (by default a product with too few output

@@ -94,13 +94,16 @@ constexpr int kMaxKSplit = 16;
 // Measured on B200 (both launches with their event pairs, 4096 -> 14336, 1024 fine-tuning rows), against the mma.sync
 // streaming kernel: rank 16 7 + 27 vs 21 us, rank 32 8 + 23 vs 29, rank 64 9 + 25 vs 33-50 (whole step 295 vs 315 us with
 // one adapter, 404 vs 410 with 256), rank 128 9 + 25 vs 144 (two launches of the per-item kernel).  Before the operands
-// were made ahead, every tile converted its own (rank 128: 7 us per tile, 56-70 us per launch).
-constexpr int kTcGradMinRank = 64;
+// were made ahead, every tile converted its own (rank 128: 7 us per tile, 56-70 us per launch).  Rank 32 is a draw launch by
+// launch and 2% ahead in the step where the fine-tuning rows come in long runs (5120 -> 13824, 2048 fine-tuning rows of one
+// adapter, forward + backward with both tcgen05 families: 448 vs 458 us; with 512 decode rows beside them 575 vs 587).
+constexpr int kTcGradMinRank = 32;
 // Ranks from which the tcgen05 shrink (U = X A^T with the activation save, V = s dY B^T) is the default.  Measured on
 // B200 (main + finish launch with their event pairs, 2048 x 4096 forward / 1024 x 14336 backward): rank 128 19 + 12 and
 // 20 + 10 us vs 43 and 74 for the per-item kernel; rank 64 15 + 13 and 17 + 9 vs 31 and 37 for the streaming kernel;
-// rank 32 14 + 15 and 17 + 9 vs 20 and 25 (hence not the default there).
-constexpr int kTcShrinkMinRank = 64;
+// rank 32 14 + 15 and 17 + 9 vs 20 and 25 one by one, but inside the step (launch overlap on) the pair is the faster one
+// (see above), hence the default from rank 32.
+constexpr int kTcShrinkMinRank = 32;
 
 enum { KIND_SHRINK = 0, KIND_GEMM_FWD = 1, KIND_GEMM_BWD = 2, KIND_GRAD = 3, KIND_SIMT = 4, KIND_ADAMW = 5, KIND_REDUCE = 6 };
 

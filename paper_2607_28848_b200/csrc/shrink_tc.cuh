@@ -1,5 +1,6 @@
 // The rank-r products U = X A_a^T (forward shrink) and V = s dY B_a^T (backward) on the tcgen05 tensor
-// cores, for the higher ranks (64, 128), where the mma.sync kernels run out of registers and shared memory.
+// cores, for the higher ranks (the default from 32; at 64 and 128 the mma.sync kernels run out of registers and shared
+// memory).
 //
 // Rows come as BLOCKS: runs of <= 128 consecutive rows that share one adapter (the plan's block tables).
 // A block is one MMA operand: a tile of 128 rows x COLS columns of the input (TMA, 128-byte swizzle) is

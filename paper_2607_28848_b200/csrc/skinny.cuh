@@ -1,9 +1,9 @@
 // Rank-r ("skinny") kernels of the multi-LoRA layer for bf16 storage, mma.sync family.  They are bound by
 // the bytes of the wide operand they stream once from HBM; the rank-r contraction itself runs on the
 // warp-level tensor-core instruction (mma.sync m16n8k16, fp32 accumulate) because at rank 16 and above the
-// CUDA cores could not keep up with the memory system.  These are the defaults up to rank 32 and, at every
+// CUDA cores could not keep up with the memory system.  These are the defaults up to rank 16 and, at every
 // rank, wherever the rows pass through registers for a reason: gathered decode rows, the dropout mask.
-// Ranks 64 and 128 otherwise run on the tcgen05 kernels of shrink_tc.cuh and grad_tc.cuh.
+// Ranks 32 to 128 otherwise run on the tcgen05 kernels of shrink_tc.cuh and grad_tc.cuh.
 //
 //  shrink : Out[t, q] = sum_k In[t, k] * P_a(t)[q, k]      (U = X A^T  and  V = s dY B^T)
 //           work item = up to 32 rows that share one adapter, GATHERED by adapter id (they need not be
