@@ -124,6 +124,32 @@ def test_k_split_of_the_last_wave_only(sess, d_in, d_out):
     run_and_check(sess, w, t, path=4, blocked=True)
 
 
+@pytest.mark.parametrize("rank", [32, 128])
+def test_tensor_core_rank_r_kernels_are_bit_reproducible(sess, rank):
+    """The tcgen05 shrink adds its runs in CTA order and the gradient kernel its pieces likewise: ten forward + backward
+    passes over a batch whose blocks are shared by many CTAs (one adapter, long contraction) give the same bits."""
+    segs = synth.segments_array([(0, 700, 0, 1), (700, 300, 1, 0), (1000, 500, 0, 1)])
+    w = synth.Workload("repro_tc", 4096, 1024, rank, 2, "bf16", 1500, segs, seed=600 + rank)
+    t = synth.make_tensors(w)
+    run = LayerRun(sess, w.dtype, t, w.segments, w.n_rows)
+    try:
+        first = None
+        for it in range(10):
+            for b in (run.Y, run.u_save, run.dA, run.dB, run.dX):
+                b.zero_()
+            run.forward(); run.backward()
+            torch.cuda.synchronize()
+            got = [b.clone() for b in (run.Y, run.u_save, run.dA, run.dB, run.dX)]
+            if first is None:
+                first = got
+            else:
+                for a, b in zip(first, got):
+                    assert torch.equal(a, b), it
+        assert run.status() == mb.MLORA_OK
+    finally:
+        run.close()
+
+
 @pytest.mark.parametrize("rank", [64, 128])
 def test_high_rank_large_batch(sess, rank):
     """8192 rows over 40 adapters at rank 64 / 128 (2048 -> 4096): the tcgen05 shrink with a few hundred blocks and runs
