@@ -39,8 +39,8 @@ constexpr int THREADS = 192;
 template <int R>
 struct Cfg {
   static constexpr int RP = R < 16 ? 16 : R;            // rank padded to the smallest N of a 128-row MMA
-  static constexpr int CB = R <= 16 ? 4 : 2;            // 64-column blocks per tile
-  static constexpr int S = R <= 16 ? 3 : (R == 32 ? 5 : (R == 64 ? 4 : 3));   // stages
+  static constexpr int CB = R <= 64 ? 4 : 2;            // 64-column blocks per tile
+  static constexpr int S = R <= 16 ? 3 : (R <= 64 ? 2 : 3);   // stages (what fits 227 KiB)
   static constexpr int COLS = CB * 64;
   static constexpr uint32_t BLK = ROWS * 128;           // one 64-column block of a tile: [128 rows][128 B]
   static constexpr uint32_t Q_BYTES = CB * BLK;
