@@ -158,6 +158,13 @@ int32_t mlora_plan_ft_adapters(const mlora_plan* plan, int32_t* ids, int32_t cap
 /* Inspection: out[k] = save offset of segment k, or -1 when it is not a fine-tuning segment
  * (n_segs entries); row_adapter[t] = adapter of row t or -1 (n_rows entries). Either may be NULL. */
 mlora_status_t mlora_plan_describe(const mlora_plan* plan, int32_t* seg_save_offset, int32_t* row_adapter);
+/* Cost view of the fused expand: for every 256-row tile of the batch, how many columns its low-rank
+ * operand has = the contraction depth the tile adds to the base product (in steps of 64 it is the
+ * tile's count of extra K-blocks).  Without per-adapter ranks that is (distinct adapters in the
+ * tile) * rank; a plan made by mlora_plan_create_ranked counts each adapter with its own rank
+ * rounded up to 16, and `rank` is ignored.  Writes up to cap entries into cols and returns the number
+ * of tiles, ceil(n_rows / 256).  Works without a context (host-only plans). */
+int32_t mlora_plan_lowrank_columns(const mlora_plan* plan, int32_t rank, int32_t* cols, int32_t cap);
 
 /* ---- forward ---------------------------------------------------------------------------*/
 

@@ -24,7 +24,7 @@ EXPORTS = (
     "mlora_create", "mlora_destroy", "mlora_plan_create", "mlora_plan_destroy", "mlora_plan_rows",
     "mlora_plan_ft_rows", "mlora_plan_ft_adapters", "mlora_plan_describe", "mlora_mixed_forward",
     "mlora_backward", "mlora_poll_status", "mlora_status_string", "mlora_launch_count", "mlora_set_gemm_path",
-    "mlora_plan_create_ranked", "mlora_plan_create_ranked_async", "mlora_profile_enable", "mlora_profile_collect", "mlora_forward_noalloc", "mlora_adamw_update",
+    "mlora_plan_create_ranked", "mlora_plan_create_ranked_async", "mlora_plan_lowrank_columns", "mlora_profile_enable", "mlora_profile_collect", "mlora_forward_noalloc", "mlora_adamw_update",
     "mlora_set_cancel_flag", "mlora_set_dropout", "mlora_plan_create_async", "mlora_plan_release",
     "mlora_selftest_timeout",
 )
@@ -81,6 +81,8 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.mlora_plan_create_ranked.restype = ctypes.c_int
     lib.mlora_plan_create_ranked_async.argtypes = [vp, P(mlora_segment_t), i32, i32, i32, P(i32), vp, P(vp)]
     lib.mlora_plan_create_ranked_async.restype = ctypes.c_int
+    lib.mlora_plan_lowrank_columns.argtypes = [vp, i32, P(i32), i32]
+    lib.mlora_plan_lowrank_columns.restype = i32
     lib.mlora_plan_destroy.argtypes = [vp]
     lib.mlora_plan_destroy.restype = None
     lib.mlora_plan_create_async.argtypes = [vp, P(mlora_segment_t), i32, i32, i32, vp, P(vp)]
@@ -194,6 +196,15 @@ def mlora_plan_create_ranked_async(ctx, segments, n_rows: int, n_adapters: int, 
     _check(load_library().mlora_plan_create_ranked_async(ctx, arr, n, int(n_rows), int(n_adapters), ranks, _stream_ptr(stream),
                                                          ctypes.byref(h)), "mlora_plan_create_ranked_async")
     return h
+
+
+def mlora_plan_lowrank_columns(plan, rank: int) -> List[int]:
+    """Columns of the low-rank operand of every 256-row tile (the extra contraction depth of the fused expand)."""
+    lib = load_library()
+    n = int(lib.mlora_plan_lowrank_columns(plan, int(rank), None, 0))
+    buf = (ctypes.c_int32 * max(n, 1))()
+    lib.mlora_plan_lowrank_columns(plan, int(rank), buf, n)
+    return [int(buf[i]) for i in range(n)]
 
 
 def mlora_plan_release(plan, stream=None) -> None:

@@ -1485,6 +1485,15 @@ int32_t mlora_plan_ft_adapters(const mlora_plan* p, int32_t* ids, int32_t cap) {
   for (int32_t i = 0; ids && i < n && i < cap; ++i) ids[i] = p->h.ft_adapters[i];
   return n;
 }
+int32_t mlora_plan_lowrank_columns(const mlora_plan* p, int32_t rank, int32_t* cols, int32_t cap) {
+  if (!p) return 0;
+  const RowSpace& rs = p->h.fwd;
+  const int32_t tiles = (int32_t)rs.tile2_grp_off.size() - 1;
+  for (int32_t t = 0; t < tiles && t < cap && cols; ++t)
+    cols[t] = rs.tile2_cols.empty() ? (rs.tile2_grp_off[t + 1] - rs.tile2_grp_off[t]) * rank : rs.tile2_cols[t];
+  return tiles < 0 ? 0 : tiles;
+}
+
 mlora_status_t mlora_plan_describe(const mlora_plan* p, int32_t* seg_save_offset, int32_t* row_adapter) {
   if (!p) return MLORA_ERR_INVALID_ARG;
   if (seg_save_offset) for (int32_t k = 0; k < p->h.n_segs; ++k) seg_save_offset[k] = p->h.seg_save_off[k];

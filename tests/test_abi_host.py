@@ -90,6 +90,21 @@ def test_ranked_plan_on_the_host():
         assert e.value.status == mb.MLORA_ERR_INVALID_ARG
 
 
+def test_lowrank_columns_hand_listed():
+    """600 rows = three 256-row tiles.  Tile 0: adapters 0 and 2; tile 1: adapters 2 (continued), 1 and 3, and a
+    stretch without adapter; tile 2: adapter 3 (continued) and a fine-tuning segment of adapter 0."""
+    segs = [(0, 100, 0, 0), (100, 200, 2, 0), (300, 50, 1, 0), (350, 60, -1, 0), (410, 140, 3, 0), (550, 50, 0, 1)]
+    plain = host_plan(segs, 600, 4)
+    ranked = mb.mlora_plan_create_ranked(None, segs, 600, 4, [8, 40, 64, 17])      # widths 16, 48, 64, 32
+    try:
+        assert mb.mlora_plan_lowrank_columns(plain, 64) == [2 * 64, 3 * 64, 2 * 64]
+        assert mb.mlora_plan_lowrank_columns(plain, 16) == [32, 48, 32]
+        assert mb.mlora_plan_lowrank_columns(ranked, 64) == [16 + 64, 64 + 48 + 32, 32 + 16]
+    finally:
+        mb.mlora_plan_destroy(plain)
+        mb.mlora_plan_destroy(ranked)
+
+
 def test_empty_table_and_empty_batch():
     p = host_plan(np.zeros((0, 4), np.int32), 5, 2)
     assert mb.mlora_plan_ft_rows(p) == 0 and mb.mlora_plan_ft_adapters(p) == []
