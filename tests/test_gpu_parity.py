@@ -737,3 +737,29 @@ def test_cfg4_sweep_grid_full_size(sess, rank, n_adapters, f, sorted_rows):
     point with unsorted rows (every row its own segment), each compared element by element."""
     w = synth.cfg4_sweep_point(rank, n_adapters, f, sorted_rows=sorted_rows)
     run_and_check(sess, w, _cfg4_tensors(w), blocked=True)
+
+
+def test_two_contexts_on_two_host_threads():
+    """Contexts are independent across host threads (the per-device caches of one-time kernel attributes are shared and
+    locked): two threads, each with its own context, stream and plans, run different ranks at the same time on the same
+    device; each checks its own results against the oracle."""
+    import threading
+    errors = []
+
+    def worker(seed, rank):
+        try:
+            stream = torch.cuda.Stream(device=torch.device("cuda", 0))
+            with torch.cuda.stream(stream):
+                with Session(0) as s2:
+                    for it in range(3):
+                        w = synth.random_workload(seed + it, 256, 384, rank, 5, 500, max_seg=120, p_finetune=0.4)
+                        run_and_check(s2, w, synth.make_tensors(w))
+        except Exception as e:          # noqa: BLE001 - reported below, in the main thread
+            errors.append((seed, rank, repr(e)))
+
+    threads = [threading.Thread(target=worker, args=(910, 16)), threading.Thread(target=worker, args=(920, 64))]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    assert not errors, errors
