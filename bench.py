@@ -660,6 +660,19 @@ def extra_configs(sess, peaks, headline: str):
         c5["fill_ratio_mixed_over_decode_plus_finetune"] = c5["mixed"]["median_us"] / (c5["decode"]["median_us"] + c5["finetune"]["median_us"])
         out["cfg5"] = c5
     out["cfg4"] = [entry(synth.cfg4_sweep_point(r, n, f), reps=20) for r, n, f in ((16, 8, 0.5), (64, 64, 0.25), (128, 256, 0.5))]
+    # the same rank-128 point when the 256 adapters have ranks of their own (8 ... 128, stored zero-padded): a plan that
+    # knows them packs the fused expand by rank and reads only the rows a rank needs
+    w = synth.cfg4_sweep_point(128, 256, 0.5)
+    t = synth.make_tensors(w)
+    ranks = [(8, 16, 16, 32, 64, 128)[a % 6] for a in range(w.n_adapters)]
+    for a, ra in enumerate(ranks):
+        t["A_all"][a, ra:] = 0.0
+        t["B_all"][a, ra:] = 0.0
+    padded = bt.step_time(sess, w, 20, tensors=t)
+    ranked = bt.step_time(sess, w, 20, tensors=t, adapter_rank=ranks)
+    out["cfg4_mixed_ranks"] = {"workload": w.name + " with adapter ranks cycling through 8, 16, 16, 32, 64, 128 (stored padded to 128)",
+                               "plain_plan_median_us": padded[0], "ranked_plan_median_us": ranked[0],
+                               "note": "mlora_plan_create_ranked; not one of the five seeded configurations"}
     cold = {"protocol": "every repetition on another copy of X, dY and the activation buffers (6 copies), one CUDA event pair per launch, "
                         "40 repetitions; bytes = every operand once; fraction of the measured copy bandwidth (median / best)"}
     rows = []

@@ -105,9 +105,12 @@ def cold_skinny(sess, w, reps, copies):
     return out, nbytes, moved * copies
 
 
-def step_time(sess, w, reps):
-    """Median and best time (µs) of forward + backward (forward only without fine-tuning rows)."""
-    run = LayerRun(sess, w.dtype, synth.make_tensors(w, with_grad=w.ft_rows > 0), w.segments, w.n_rows)
+def step_time(sess, w, reps, tensors=None, adapter_rank=None):
+    """Median and best time (µs) of forward + backward (forward only without fine-tuning rows); `adapter_rank`
+    makes the plan with the adapters' own ranks."""
+    if tensors is None:
+        tensors = synth.make_tensors(w, with_grad=w.ft_rows > 0)
+    run = LayerRun(sess, w.dtype, tensors, w.segments, w.n_rows, adapter_rank=adapter_rank)
 
     def step():
         run.forward()
