@@ -305,10 +305,25 @@ def whole_layer(dev) -> str:
         y_eager = layer.forward(x, segs)
         same = bool(torch.equal(cap.y, y_eager))
         cap.close()
+        saved = list(layer.saved)
+        capb = layer.capture_backward(saved)
+        capb.dy.copy_(dy)
+        tgb = []
+        for it in range(8):
+            torch.cuda.synchronize()
+            e0, e1 = (torch.cuda.Event(enable_timing=True) for _ in range(2))
+            e0.record()
+            capb.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            if it >= 2:
+                tgb.append(e0.elapsed_time(e1))
+        capb.close()
     return (f"whole decoder layer (Llama-3-8B sizes, cfg3 batch: {T} rows, {ft_rows} fine-tuning), through DecoderLayer (one "
             f"library call after the other from Python, host overheads included): serving forward "
             f"{np.median(tf):.2f} ms, recompute + backward over the fine-tuning rows {np.median(tb):.2f} ms; the same serving "
-            f"forward replayed from a CUDA graph: {np.median(tg):.2f} ms (output bit-identical to the eager one: {same})")
+            f"forward replayed from a CUDA graph: {np.median(tg):.2f} ms (output bit-identical to the eager one: {same}); the recompute + "
+            f"backward replayed from a CUDA graph: {np.median(tgb):.2f} ms")
 
 
 def table_layer_ops(args):

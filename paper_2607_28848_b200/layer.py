@@ -147,6 +147,7 @@ class DecoderLayer:
         class Captured:
             pass
         cap = Captured()
+        cap.tables = tables                      # the graph's kernels read them on every replay
         cap.x = x.clone()
         stream = torch.cuda.Stream(device=dev)
         with torch.cuda.stream(stream):
@@ -165,65 +166,111 @@ class DecoderLayer:
         return cap
 
     # -- backward: recompute from the saved layer input, fine-tuning rows only ---------------------
+    def _backward_body(self, x, dy, plan, n_slots, sequences, tables=None):
+        """Recompute the layer over the saved rows `x` and backpropagate `dy`; every call is a library kernel."""
+        rows = x.shape[0]
+        dev, ctx = x.device, self.sess.ctx
+        dh = self.d // self.n_heads
+
+        def lin(name, inp):          # recompute pass: every row is a fine-tuning row, each projection saves its own input and x A^T
+            pr = self.proj[name]
+            y = torch.empty((rows, pr.d_out), dtype=torch.bfloat16, device=dev)
+            mb.mlora_mixed_forward(ctx, pr.layer, plan, inp, y, pr.x_save, pr.u_save, 0, pr.x_save.shape[0])
+            return y
+
+        def lin_bwd(name, g):        # LoRA gradients of one projection and the gradient of its input
+            pr = self.proj[name]
+            pr.dA = torch.empty((n_slots, pr.rank, pr.d_in), dtype=torch.float32, device=dev)
+            pr.dB = torch.empty((n_slots, pr.rank, pr.d_out), dtype=torch.float32, device=dev)
+            dx = torch.empty((rows, pr.d_in), dtype=torch.bfloat16, device=dev)
+            mb.mlora_backward(ctx, pr.layer, plan, g, pr.x_save, pr.u_save, pr.dA, pr.dB, dx)
+            return dx
+
+        _y, t = self._body(x, lin, sequences, tables)
+        # y = x2 + down(m): dy reaches x2 directly and through the feed-forward branch
+        dm = lin_bwd("down", dy)
+        dg, du = torch.empty_like(t["g"]), torch.empty_like(t["u"])
+        mo.mlora_swiglu_backward(t["g"], t["u"], dm, dg, du)
+        dh2 = lin_bwd("gate", dg)
+        mo.mlora_add(dh2, lin_bwd("up", du), dh2)                   # h2 feeds gate and up
+        dx2 = torch.empty_like(x)
+        mo.mlora_rmsnorm_backward(t["x2"], self.g2, dh2, dx2)
+        mo.mlora_add(dx2, dy, dx2)                                  # x2 feeds the norm and the residual
+        # x2 = x + o(a)
+        da = lin_bwd("o", dx2)
+        dq, dk, dv = torch.empty_like(t["q"]), torch.empty_like(t["k"]), torch.empty_like(t["v"])
+        mo.mlora_attention_backward(t["q"], t["k"], t["v"], t["a"], t["lse"], da, dq, dk, dv, t["seq_start"], t["seq_end"],
+                                    self.n_heads, self.n_kv, dh)
+        dq0, dk0 = torch.empty_like(dq), torch.empty_like(dk)
+        mo.mlora_rope(dq, dq0, t["pos"], self.n_heads, dh, transpose=True)
+        mo.mlora_rope(dk, dk0, t["pos"], self.n_kv, dh, transpose=True)
+        dh1 = lin_bwd("q", dq0)
+        mo.mlora_add(dh1, lin_bwd("k", dk0), dh1)                   # h1 feeds q, k and v
+        mo.mlora_add(dh1, lin_bwd("v", dv), dh1)
+        dx = torch.empty_like(x)
+        mo.mlora_rmsnorm_backward(x, self.g1, dh1, dx)
+        mo.mlora_add(dx, dx2, dx)                                   # x feeds the norm and the residual
+        grads = {n: (self.proj[n].dA, self.proj[n].dB) for n in PROJ}
+        return dx, grads
+
+    @staticmethod
+    def _saved_table(saved):
+        table, row = [], 0
+        for n, a in saved:
+            table.append((row, n, a, 1)); row += n
+        return synth.segments_array(table), row
+
     def backward(self, dy_ft: torch.Tensor):
         """dy_ft [saved rows, d]: gradient of the layer output for the saved rows, in save order.
         Returns (dx [saved rows, d], {projection: (dA, dB)}, adapters of the gradient slots)."""
         rows = self.saved_rows
-        table, row = [], 0
-        for n, a in self.saved:
-            table.append((row, n, a, 1)); row += n
-        table = synth.segments_array(table)
+        table, _ = self._saved_table(self.saved)
         self.bwd_plan = mb.mlora_plan_create(self.sess.ctx, table, rows, self.n_adapters)
         self.bwd_slots = mb.mlora_plan_ft_adapters(self.bwd_plan)
         try:
-            dev, ctx = self.saved_x.device, self.sess.ctx
-            n_slots = len(self.bwd_slots)
             x = self.saved_x[:rows]
-            dh = self.d // self.n_heads
-
-            def lin(name, inp):          # recompute pass: every row is a fine-tuning row, each projection saves its own input and x A^T
-                pr = self.proj[name]
-                y = torch.empty((rows, pr.d_out), dtype=torch.bfloat16, device=dev)
-                mb.mlora_mixed_forward(ctx, pr.layer, self.bwd_plan, inp, y, pr.x_save, pr.u_save, 0, pr.x_save.shape[0])
-                return y
-
-            def lin_bwd(name, dy):       # LoRA gradients of one projection and the gradient of its input
-                pr = self.proj[name]
-                pr.dA = torch.empty((n_slots, pr.rank, pr.d_in), dtype=torch.float32, device=dev)
-                pr.dB = torch.empty((n_slots, pr.rank, pr.d_out), dtype=torch.float32, device=dev)
-                dx = torch.empty((rows, pr.d_in), dtype=torch.bfloat16, device=dev)
-                mb.mlora_backward(ctx, pr.layer, self.bwd_plan, dy, pr.x_save, pr.u_save, pr.dA, pr.dB, dx)
-                return dx
-
-            _y, t = self._body(x, lin, [(int(s), int(n)) for s, n, _, _ in table])
             dy = dy_ft.to(torch.bfloat16).contiguous()
-            # y = x2 + down(m): dy reaches x2 directly and through the feed-forward branch
-            dm = lin_bwd("down", dy)
-            dg, du = torch.empty_like(t["g"]), torch.empty_like(t["u"])
-            mo.mlora_swiglu_backward(t["g"], t["u"], dm, dg, du)
-            dh2 = lin_bwd("gate", dg)
-            mo.mlora_add(dh2, lin_bwd("up", du), dh2)                   # h2 feeds gate and up
-            dx2 = torch.empty_like(x)
-            mo.mlora_rmsnorm_backward(t["x2"], self.g2, dh2, dx2)
-            mo.mlora_add(dx2, dy, dx2)                                  # x2 feeds the norm and the residual
-            # x2 = x + o(a)
-            da = lin_bwd("o", dx2)
-            dq, dk, dv = torch.empty_like(t["q"]), torch.empty_like(t["k"]), torch.empty_like(t["v"])
-            mo.mlora_attention_backward(t["q"], t["k"], t["v"], t["a"], t["lse"], da, dq, dk, dv, t["seq_start"], t["seq_end"],
-                                        self.n_heads, self.n_kv, dh)
-            dq0, dk0 = torch.empty_like(dq), torch.empty_like(dk)
-            mo.mlora_rope(dq, dq0, t["pos"], self.n_heads, dh, transpose=True)
-            mo.mlora_rope(dk, dk0, t["pos"], self.n_kv, dh, transpose=True)
-            dh1 = lin_bwd("q", dq0)
-            mo.mlora_add(dh1, lin_bwd("k", dk0), dh1)                   # h1 feeds q, k and v
-            mo.mlora_add(dh1, lin_bwd("v", dv), dh1)
-            dx = torch.empty_like(x)
-            mo.mlora_rmsnorm_backward(x, self.g1, dh1, dx)
-            mo.mlora_add(dx, dx2, dx)                                   # x feeds the norm and the residual
+            dx, grads = self._backward_body(x, dy, self.bwd_plan, len(self.bwd_slots), [(int(s), int(n)) for s, n, _, _ in table])
             torch.cuda.synchronize()
-            grads = {n: (self.proj[n].dA, self.proj[n].dB) for n in PROJ}
             return dx, grads, list(self.bwd_slots)
         finally:
             mb.mlora_plan_destroy(self.bwd_plan)
             self.bwd_plan = None
             self.saved, self.saved_rows = [], 0
+
+    @torch.no_grad()
+    def capture_backward(self, saved):
+        """The recompute + backward over a fixed layout of saved fine-tuning sequences (`saved`: (tokens, adapter) in
+        save order, e.g. the paper's backward batches of 256 tokens) captured once in a CUDA graph.  The layer input
+        of those rows is read from the layer's own save buffer (where the serving forwards put it), `dy` is a static
+        buffer to copy the output gradient into.  Returns an object with ``dy``, ``dx``, ``grads`` (static outputs),
+        ``slots``, ``replay()`` and ``close()``."""
+        table, rows = self._saved_table(saved)
+        plan = mb.mlora_plan_create(self.sess.ctx, table, rows, self.n_adapters)
+        slots = mb.mlora_plan_ft_adapters(plan)
+        dev = self.saved_x.device
+        seqs = [(int(s), int(n)) for s, n, _, _ in table]
+        tables = tuple(torch.from_numpy(t).to(dev) for t in sequence_tables(rows, seqs))
+        x = self.saved_x[:rows]
+
+        class Captured:
+            pass
+        cap = Captured()
+        cap.tables = tables                      # the graph's kernels read them on every replay
+        cap.dy = torch.zeros((rows, self.d), dtype=torch.bfloat16, device=dev)
+        cap.slots = list(slots)
+        stream = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(stream):
+            for _ in range(2):
+                self._backward_body(x, cap.dy, plan, len(slots), None, tables)
+            stream.synchronize()
+            cap.graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(cap.graph, stream=stream):
+                cap.dx, cap.grads = self._backward_body(x, cap.dy, plan, len(slots), None, tables)
+        cap.replay = cap.graph.replay
+
+        def close():
+            torch.cuda.synchronize()
+            mb.mlora_plan_destroy(plan)
+        cap.close = close
+        return cap

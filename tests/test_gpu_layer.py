@@ -86,3 +86,24 @@ def test_layer_forward_and_recompute_backward_match_the_oracle():
             close("dA_" + name, grads[name][0], ref["dA_" + name], 2e-2)
             close("dB_" + name, grads[name][1], ref["dB_" + name], 2e-2)
         assert layer.saved_rows == 0
+
+        # the same recompute + backward captured in a CUDA graph (the save buffer still holds the layer input)
+        capb = layer.capture_backward([(64, 1), (33, 2)])
+        capb.dy.copy_(dy.to(sess.device).to(torch.bfloat16))
+        capb.replay()
+        torch.cuda.synchronize()
+        assert capb.slots == [1, 2] and torch.equal(capb.dx, dx)
+        for name in PROJ:
+            assert torch.equal(capb.grads[name][0], grads[name][0]) and torch.equal(capb.grads[name][1], grads[name][1])
+        dy2 = bf16(torch.randn(97, d, generator=g, dtype=torch.float64))
+        capb.dy.copy_(dy2.to(sess.device).to(torch.bfloat16))
+        capb.replay()
+        torch.cuda.synchronize()
+        ref2 = lo.layer_backward(x[45:142], p, [1] * 64 + [2] * 33, [list(range(0, 64)), list(range(64, 97))], H, Hkv, dy2,
+                                 adapters=[1, 2])
+        close("dx (graph)", capb.dx, ref2["dx"], 2e-2)
+        for name in PROJ:
+            close("dA_" + name + " (graph)", capb.grads[name][0], ref2["dA_" + name], 2e-2)
+            close("dB_" + name + " (graph)", capb.grads[name][1], ref2["dB_" + name], 2e-2)
+        capb.close()
+        assert mb.mlora_poll_status(sess.ctx) == mb.MLORA_OK
