@@ -55,6 +55,8 @@ def test_layer_forward_and_recompute_backward_match_the_oracle():
 
         # the same forward captured in a CUDA graph and replayed on a new batch of the same layout
         cap = layer.capture_forward(x.to(sess.device).to(torch.bfloat16), synth.segments_array(segs))
+        # whatever the capture freed is handed out again and overwritten: the graph must own all it reads
+        junk = [torch.full((n,), -7, dtype=torch.int32, device=sess.device) for n in (T, T, T, 16, 16, 512, 512) * 4]
         cap.replay()
         torch.cuda.synchronize()
         assert torch.equal(cap.y, y)
@@ -89,6 +91,7 @@ def test_layer_forward_and_recompute_backward_match_the_oracle():
 
         # the same recompute + backward captured in a CUDA graph (the save buffer still holds the layer input)
         capb = layer.capture_backward([(64, 1), (33, 2)])
+        junk += [torch.full((n,), -7, dtype=torch.int32, device=sess.device) for n in (97, 97, 97, 16, 16, 512, 512) * 4]
         capb.dy.copy_(dy.to(sess.device).to(torch.bfloat16))
         capb.replay()
         torch.cuda.synchronize()
