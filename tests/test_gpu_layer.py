@@ -19,8 +19,11 @@ def bf16(t):
     return t.to(torch.bfloat16).to(torch.float64)
 
 
-def test_layer_forward_and_recompute_backward_match_the_oracle():
-    d, ffn, r, n_ad, H, Hkv = 512, 1024, 16, 3, 4, 2
+@pytest.mark.parametrize("d,ffn,r,H,Hkv,ft1,ft2", [(512, 1024, 16, 4, 2, 64, 33), (1024, 1536, 32, 8, 2, 200, 141)])
+def test_layer_forward_and_recompute_backward_match_the_oracle(d, ffn, r, H, Hkv, ft1, ft2):
+    """Second case: rank 32 (the tcgen05 shrink and gradient kernels inside the chain), fine-tuning sequences that
+    cross the 128-row tiles of the attention kernels, 341 saved rows."""
+    n_ad = 3
     dh = d // H
     g = torch.Generator().manual_seed(11)
     dims = {"q": (d, d), "k": (d, Hkv * dh), "v": (d, Hkv * dh), "o": (d, d), "gate": (d, ffn), "up": (d, ffn), "down": (ffn, d)}
@@ -33,8 +36,9 @@ def test_layer_forward_and_recompute_backward_match_the_oracle():
         p["B_" + name] = bf16(0.05 * torch.randn(n_ad, r, do, generator=g, dtype=torch.float64))
         p["s_" + name] = torch.full((n_ad,), 2.0, dtype=torch.float64)
     # batch: an inference prompt, five decode rows, two fine-tuning sequences, a prompt without adapter
-    segs = [(0, 40, 0, 0)] + [(40 + i, 1, i % 3, 0) for i in range(5)] + [(45, 64, 1, 1), (109, 33, 2, 1), (142, 20, -1, 0)]
-    T = 162
+    ft = ft1 + ft2
+    segs = [(0, 40, 0, 0)] + [(40 + i, 1, i % 3, 0) for i in range(5)] + [(45, ft1, 1, 1), (45 + ft1, ft2, 2, 1), (45 + ft, 20, -1, 0)]
+    T = 65 + ft
     x = bf16(torch.randn(T, d, generator=g, dtype=torch.float64))
     row_adapter = [-1] * T
     sequences = []
@@ -45,13 +49,21 @@ def test_layer_forward_and_recompute_backward_match_the_oracle():
     y_ref = lo.layer_forward(x, p, row_adapter, sequences, H, Hkv)
 
     with Session(0) as sess:
-        layer = DecoderLayer(sess, p, H, Hkv, max_ft_rows=128)
+        layer = DecoderLayer(sess, p, H, Hkv, max_ft_rows=(ft + 127) // 128 * 128)
         y = layer.forward(x.to(sess.device).to(torch.bfloat16), synth.segments_array(segs))
         assert mb.mlora_poll_status(sess.ctx) == mb.MLORA_OK
-        err = (y.double().cpu() - y_ref).abs()
-        assert float((err - 3e-2 * (1 + y_ref.abs())).max()) <= 0, float(err.max())   # measured 2.2e-2: a dozen bf16 roundings in series (norms, rotary, scores, three residual adds), one more than the hot path's 2e-2 allows
-        assert layer.saved_rows == 97 and layer.saved == [(64, 1), (33, 2)]
-        assert torch.equal(layer.saved_x[:97].cpu().double(), x[45:142])      # the layer input, bit for bit
+        def check_y(got, want):
+            # y = x2 + down(m) is a sum that cancels: the residual stream reaches |x2| ~ 11 in the larger case, where bf16
+            # steps are 0.0625, so an element's error follows its row's scale rather than its own value (measured: at most
+            # 1.2e-2 of the row maximum, rms error 0.3-0.7% of the rms output)
+            err = (got.double().cpu() - want).abs()
+            row_scale = want.abs().max(1, keepdim=True).values
+            assert float((err - 1.5e-2 * (row_scale + want.abs())).max()) <= 0, float(err.max())
+            if d == 512:      # measured 2.2e-2: a dozen bf16 roundings in series (norms, rotary, scores, three residual adds), one more than the hot path's 2e-2 allows
+                assert float((err - 3e-2 * (1 + want.abs())).max()) <= 0, float(err.max())
+        check_y(y, y_ref)
+        assert layer.saved_rows == ft and layer.saved == [(ft1, 1), (ft2, 2)]
+        assert torch.equal(layer.saved_x[:ft].cpu().double(), x[45:45 + ft])      # the layer input, bit for bit
 
         # the same forward captured in a CUDA graph and replayed on a new batch of the same layout
         cap = layer.capture_forward(x.to(sess.device).to(torch.bfloat16), synth.segments_array(segs))
@@ -65,17 +77,15 @@ def test_layer_forward_and_recompute_backward_match_the_oracle():
         cap.replay()
         torch.cuda.synchronize()
         y2_ref = lo.layer_forward(x2, p, row_adapter, sequences, H, Hkv)
-        err2 = (cap.y.double().cpu() - y2_ref).abs()
-        assert float((err2 - 3e-2 * (1 + y2_ref.abs())).max()) <= 0, float(err2.max())
+        check_y(cap.y, y2_ref)
         cap.close()
         assert mb.mlora_poll_status(sess.ctx) == mb.MLORA_OK
 
         # backward over the fine-tuning rows alone, recomputed from the saved input
-        ft_rows = list(range(45, 142))
-        dy = bf16(torch.randn(97, d, generator=g, dtype=torch.float64))
+        dy = bf16(torch.randn(ft, d, generator=g, dtype=torch.float64))
         dx, grads, slots = layer.backward(dy.to(sess.device))
         assert mb.mlora_poll_status(sess.ctx) == mb.MLORA_OK and slots == [1, 2]
-        ref = lo.layer_backward(x[45:142], p, [1] * 64 + [2] * 33, [list(range(0, 64)), list(range(64, 97))], H, Hkv, dy,
+        ref = lo.layer_backward(x[45:45 + ft], p, [1] * ft1 + [2] * ft2, [list(range(0, ft1)), list(range(ft1, ft))], H, Hkv, dy,
                                 adapters=[1, 2])
 
         def close(name, got, want, tol):
@@ -90,19 +100,19 @@ def test_layer_forward_and_recompute_backward_match_the_oracle():
         assert layer.saved_rows == 0
 
         # the same recompute + backward captured in a CUDA graph (the save buffer still holds the layer input)
-        capb = layer.capture_backward([(64, 1), (33, 2)])
-        junk += [torch.full((n,), -7, dtype=torch.int32, device=sess.device) for n in (97, 97, 97, 16, 16, 512, 512) * 4]
+        capb = layer.capture_backward([(ft1, 1), (ft2, 2)])
+        junk += [torch.full((n,), -7, dtype=torch.int32, device=sess.device) for n in (ft, ft, ft, 16, 16, 512, 512) * 4]
         capb.dy.copy_(dy.to(sess.device).to(torch.bfloat16))
         capb.replay()
         torch.cuda.synchronize()
         assert capb.slots == [1, 2] and torch.equal(capb.dx, dx)
         for name in PROJ:
             assert torch.equal(capb.grads[name][0], grads[name][0]) and torch.equal(capb.grads[name][1], grads[name][1])
-        dy2 = bf16(torch.randn(97, d, generator=g, dtype=torch.float64))
+        dy2 = bf16(torch.randn(ft, d, generator=g, dtype=torch.float64))
         capb.dy.copy_(dy2.to(sess.device).to(torch.bfloat16))
         capb.replay()
         torch.cuda.synchronize()
-        ref2 = lo.layer_backward(x[45:142], p, [1] * 64 + [2] * 33, [list(range(0, 64)), list(range(64, 97))], H, Hkv, dy2,
+        ref2 = lo.layer_backward(x[45:45 + ft], p, [1] * ft1 + [2] * ft2, [list(range(0, ft1)), list(range(ft1, ft))], H, Hkv, dy2,
                                  adapters=[1, 2])
         close("dx (graph)", capb.dx, ref2["dx"], 2e-2)
         for name in PROJ:
