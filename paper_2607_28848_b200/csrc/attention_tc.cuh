@@ -5,15 +5,21 @@
 // Forward: one CTA = one tile of 128 query rows of one head.  It walks the key rows from the first row of
 // the tile's first sequence to the tile's last row in blocks of 128:
 //   warp 0 (one lane)  TMA producer: Q once; K and V blocks through a ring of two stages
-//   warp 1 (one lane)  MMA issuer:   S = Q K^T into tensor memory (columns 0..127), then, once the
-//                                    softmax warps have left P in shared memory, O_blk = P V into
-//                                    columns 128..255
-//   warps 2..5         softmax:      thread = query row.  Reads S twice from tensor memory (row
-//                                    maximum, then exponentials), masks (same sequence, key <= query),
-//                                    writes P as bf16 in the K-major swizzled operand layout, then
-//                                    adds O_blk into its 128 fp32 output registers, rescaled by
-//                                    exp2(m_old - m_new) (online softmax; nothing is rescaled in
-//                                    tensor memory).
+//   warp 1 (one lane)  MMA issuer:   S_j = Q K_j^T into one of two score buffers in tensor memory
+//                                    (columns 0..127 / 128..255), issued one block ahead: S_{j+1} is
+//                                    on the tensor pipe before P_j is waited for; then O_blk = P_j V_j
+//                                    into columns 256..383
+//   warps 2..9         softmax:      two threads per query row (warps w and w + 4 own the same 32 lanes of
+//                                    tensor memory), each with 64 of the block's 128 keys and 64 of the 128
+//                                    output columns.  A thread reads its half of S_j twice from tensor memory
+//                                    (row maximum - exchanged with its partner through shared memory behind an
+//                                    mbarrier of the warp pair - then exponentials), masks (same sequence,
+//                                    key <= query) and keeps P_j as packed bf16 in 32 registers; only then it
+//                                    takes the previous block's O_blk into its 64 fp32 output registers,
+//                                    rescaled by exp2(m_old - m_new) (online softmax; nothing is rescaled in
+//                                    tensor memory), and writes P_j in the K-major swizzled operand layout -
+//                                    so the product P_{j-1} V_{j-1} and the scores S_{j+1} run on the tensor
+//                                    pipe while the threads work on block j.
 // Scores are kept in the log2 domain (scale * log2 e folded into one factor).  A row's sequence is
 // given per row (seq_start), so a tile may span several sequences: keys before the row's own
 // sequence are masked like keys after the row.  Every mbarrier wait is bounded; a wait that runs
@@ -34,8 +40,10 @@ constexpr uint32_t Q_BYTES = BM * DH * 2;     // two 64-wide K-blocks of [128 ro
 constexpr uint32_t K_BYTES = BN * DH * 2;     // the same for 128 keys
 constexpr uint32_t V_BYTES = BN * DH * 2;     // two blocks of 64 keys, each 2 x [64 keys][64 columns] (MN-major operand)
 constexpr uint32_t P_BYTES = BM * BN * 2;     // two 64-key K-blocks of [128 rows][128 B]
-constexpr uint32_t SMEM_BYTES = 1024 + Q_BYTES + STAGES * (K_BYTES + V_BYTES) + P_BYTES + 256;
-constexpr uint32_t TMEM_COLS = 256;
+constexpr int FWD_THREADS = 64 + 256;         // forward: producer warp, MMA warp, eight softmax warps
+constexpr uint32_t X_BYTES = 3 * 1024;        // forward: row maxima of the two halves (two blocks in flight) and the final row sums
+constexpr uint32_t SMEM_BYTES = 1024 + Q_BYTES + STAGES * (K_BYTES + V_BYTES) + P_BYTES + 256 + X_BYTES;
+constexpr uint32_t TMEM_COLS = 512;           // forward: S (two buffers of 128 columns), O_blk (128), 128 unused
 
 // 2^x by the special-function unit (the arguments here are differences from a row maximum or a
 // log-sum-exp, so nothing overflows; large negative arguments give 0)
@@ -56,7 +64,7 @@ struct Args {
   float scale_log2;              // log2(e) / sqrt(d_head)
 };
 
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __launch_bounds__(FWD_THREADS, 1)
 forward_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                const __grid_constant__ CUtensorMap tmV, const Args a) {
   extern __shared__ uint8_t smem_raw[];
@@ -67,11 +75,14 @@ forward_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   auto sV = [&](int s) { return sK(s) + K_BYTES; };
   const uint32_t sP = base + Q_BYTES + STAGES * (K_BYTES + V_BYTES);
   const uint32_t sBar = sP + P_BYTES;
-  const uint32_t bar_q = sBar, bar_s = sBar + 8, bar_p = sBar + 16, bar_o = sBar + 24;
-  auto bar_kv_full = [&](int s) { return sBar + 32u + 8u * s; };
-  auto bar_kv_empty = [&](int s) { return sBar + 48u + 8u * s; };
-  uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(gen + (sBar - base) + 64);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (sBar - base) + 72);
+  const uint32_t bar_q = sBar, bar_p = sBar + 8, bar_o = sBar + 16;
+  auto bar_s = [&](int j) { return sBar + 24u + 8u * (j & 1); };
+  auto bar_kv_full = [&](int s) { return sBar + 40u + 8u * s; };
+  auto bar_kv_empty = [&](int s) { return sBar + 56u + 8u * s; };
+  auto bar_x = [&](int e) { return sBar + 72u + 8u * e; };      // one per pair of softmax warps (same 32 rows)
+  uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(gen + (sBar - base) + 104);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (sBar - base) + 112);
+  float* xch = reinterpret_cast<float*>(gen + (sBar - base) + 256);   // [3][2 halves][128 rows]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * BM, h = blockIdx.y;
@@ -82,10 +93,12 @@ forward_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     ptx::mbar_init(bar_q, 1);
-    ptx::mbar_init(bar_s, 1);
-    ptx::mbar_init(bar_p, BM);
+    ptx::mbar_init(bar_s(0), 1);
+    ptx::mbar_init(bar_s(1), 1);
+    ptx::mbar_init(bar_p, 2 * BM);
     ptx::mbar_init(bar_o, 1);
     for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(bar_kv_full(s), 1); ptx::mbar_init(bar_kv_empty(s), 1); }
+    for (int e = 0; e < 4; ++e) ptx::mbar_init(bar_x(e), 64);
     *abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmQ);
@@ -124,12 +137,15 @@ forward_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     if (lane == 0) {
       constexpr uint32_t idesc_s = ptx::make_idesc_bf16(BM, BN, false, false);   // Q and K both K-major
       constexpr uint32_t idesc_o = ptx::make_idesc_bf16(BM, DH, false, true);    // V: keys are its K-rows
-      const uint32_t tS = tmem_base, tO = tmem_base + BN;
+      const uint32_t tO = tmem_base + 2 * BN;
       bool ok = gemm_wait(bar_q, 0, abort_flag, &g_status);
-      for (int j = 0; j < nblk && ok; ++j) {
+      // S_j = Q K_j^T into score buffer j & 1 (its previous reader, the softmax of block j - 2, was done
+      // before P_{j-2} arrived, which this thread has waited for)
+      auto issue_s = [&](int j) -> bool {
         const int s = j % STAGES;
-        if (!(ok = gemm_wait(bar_kv_full(s), (j / STAGES) & 1, abort_flag, &g_status))) break;
+        if (!gemm_wait(bar_kv_full(s), (j / STAGES) & 1, abort_flag, &g_status)) return false;
         ptx::tc_fence_after();
+        const uint32_t tS = tmem_base + (uint32_t)(j & 1) * BN;
         uint32_t acc = 0;
 #pragma unroll
         for (int kb = 0; kb < 2; ++kb) {
@@ -141,10 +157,16 @@ forward_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             acc = 1;
           }
         }
-        ptx::umma_commit(bar_s);
-        if (!(ok = gemm_wait(bar_p, j & 1, abort_flag, &g_status))) break;     // P in shared memory, S and O_blk read
+        ptx::umma_commit(bar_s(j));
+        return true;
+      };
+      if (ok) ok = issue_s(0);
+      for (int j = 0; j < nblk && ok; ++j) {
+        const int s = j % STAGES;
+        if (j + 1 < nblk && !(ok = issue_s(j + 1))) break;                     // one block ahead of the softmax
+        if (!(ok = gemm_wait(bar_p, j & 1, abort_flag, &g_status))) break;     // P_j in shared memory, S_j and O_blk of block j - 1 read
         ptx::tc_fence_after();
-        acc = 0;
+        uint32_t acc = 0;
 #pragma unroll
         for (int kb = 0; kb < 2; ++kb) {
           const uint64_t ad = ptx::make_smem_desc(sP + kb * 16384, 16, 1024);
@@ -161,27 +183,52 @@ forward_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     }
     __syncwarp();
   } else {
-    // ============================ softmax, one query row per thread ============================
+    // ============================ softmax, two threads per query row ============================
     const int e = warp & 3;                         // the quarter of tensor memory this warp may read
+    const int half = (warp - 2) >> 2;               // which 64 keys of a block and which 64 output columns
     const int row = e * 32 + lane;
     const int i_abs = m0 + row;
     const bool row_ok = i_abs < a.n_rows;
     const int my_start = row_ok ? a.seq_start[i_abs] : 0x7fffffff;
-    const uint32_t tS = tmem_base + ((uint32_t)(e * 32) << 16), tO = tS + BN;
-    const uint32_t prow = sP + (uint32_t)row * 128u;
-    float O[DH];
+    const uint32_t tS0 = tmem_base + ((uint32_t)(e * 32) << 16) + (uint32_t)half * 64u;
+    const uint32_t tO = tmem_base + ((uint32_t)(e * 32) << 16) + 2 * BN + (uint32_t)half * 64u;
+    const uint32_t prow = sP + (uint32_t)half * 16384u + (uint32_t)row * 128u;       // K-block `half` of P
+    float* x_mine = xch + half * BM + row;          // + 256 per slot
+    const float* x_peer = xch + (half ^ 1) * BM + row;
+    float O[DH / 2];
 #pragma unroll
-    for (int k = 0; k < DH; ++k) O[k] = 0.f;
-    float m = -1e30f, l = 0.f;
+    for (int k = 0; k < DH / 2; ++k) O[k] = 0.f;
+    float m = -1e30f, l = 0.f, alpha_prev = 1.f;    // l: the sum over this thread's keys only
     bool ok = true;
+    // O += O_blk of one block, the sum so far rescaled to that block's running maximum
+    auto take_o = [&](float alpha) {
+#pragma unroll
+      for (int cc = 0; cc < 2; ++cc) {
+        uint32_t v[32];
+        ptx::tmem_ld_32x32b_x32(tO + cc * 32, v);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int k = 0; k < 32; ++k) O[cc * 32 + k] = fmaf(O[cc * 32 + k], alpha, __uint_as_float(v[k]));
+      }
+    };
+    // value exchange between the two threads of a row: slot picks one of three buffers, phase counts the
+    // uses of the pair's barrier
+    auto exchange = [&](float mine, int slot, int phase, float& peer) -> bool {
+      x_mine[slot * 2 * BM] = mine;
+      ptx::mbar_arrive(bar_x(e));
+      const bool got = __all_sync(0xffffffffu, gemm_wait(bar_x(e), phase & 1, abort_flag, &g_status));
+      if (got) peer = x_peer[slot * 2 * BM];
+      return got;
+    };
     for (int j = 0; j < nblk; ++j) {
-      const int key0 = kmin + j * BN;
-      ok = __all_sync(0xffffffffu, gemm_wait(bar_s, j & 1, abort_flag, &g_status));   // one decision per warp:
-      if (!ok) break;                                                                  // the loads below are warp-wide
+      const int key0 = kmin + j * BN + half * 64;
+      const uint32_t tS = tS0 + (uint32_t)(j & 1) * BN;
+      ok = __all_sync(0xffffffffu, gemm_wait(bar_s(j), (j >> 1) & 1, abort_flag, &g_status));   // one decision per warp:
+      if (!ok) break;                                                                            // the loads below are warp-wide
       ptx::tc_fence_after();
       float mx = m;
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
+      for (int cc = 0; cc < 2; ++cc) {
         uint32_t v[32];
         ptx::tmem_ld_32x32b_x32(tS + cc * 32, v);
         ptx::tmem_ld_wait();
@@ -192,53 +239,60 @@ forward_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           mx = fmaxf(mx, sc);
         }
       }
+      float peer_mx;
+      if (!(ok = exchange(mx, j & 1, j, peer_mx))) break;
+      mx = fmaxf(mx, peer_mx);
       const float alpha = fast_ex2(m - mx);
       float rowsum = 0.f;
+      uint32_t pk[32];
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
+      for (int cc = 0; cc < 2; ++cc) {
         uint32_t v[32];
         ptx::tmem_ld_32x32b_x32(tS + cc * 32, v);
         ptx::tmem_ld_wait();
-        uint32_t pk[16];
 #pragma unroll
         for (int k = 0; k < 32; k += 2) {
           const int col = key0 + cc * 32 + k;
           const float p0 = (col >= my_start && col <= i_abs) ? fast_ex2(__uint_as_float(v[k]) * a.scale_log2 - mx) : 0.f;
           const float p1 = (col + 1 >= my_start && col + 1 <= i_abs) ? fast_ex2(__uint_as_float(v[k + 1]) * a.scale_log2 - mx) : 0.f;
           rowsum += p0 + p1;
-          pk[k >> 1] = ptx::pack_bf16(p0, p1);
-        }
-        // columns 32 cc .. 32 cc + 31 of P: K-block cc / 2, 16-byte pieces 4 (cc % 2) .. + 3 of the row,
-        // piece i stored at i ^ (row & 7) (the operand's 128-byte swizzle)
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const uint32_t pc = (uint32_t)((cc & 1) * 4 + q);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(prow + (uint32_t)(cc >> 1) * 16384u + ((pc ^ (uint32_t)(row & 7)) << 4)),
-                       "r"(pk[4 * q]), "r"(pk[4 * q + 1]), "r"(pk[4 * q + 2]), "r"(pk[4 * q + 3]) : "memory");
+          pk[cc * 16 + (k >> 1)] = ptx::pack_bf16(p0, p1);
         }
       }
+      if (j > 0) {      // the previous block's P V ran while this block's scores were worked on
+        ok = __all_sync(0xffffffffu, gemm_wait(bar_o, (j - 1) & 1, abort_flag, &g_status));
+        if (!ok) break;
+        ptx::tc_fence_after();
+        take_o(alpha_prev);
+      }
+      // this thread's 64 keys are K-block `half` of P: eight 16-byte pieces of the row, piece i stored at
+      // i ^ (row & 7) (the operand's 128-byte swizzle); the previous product has finished reading the buffer
+#pragma unroll
+      for (int pc = 0; pc < 8; ++pc)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(prow + (((uint32_t)pc ^ (uint32_t)(row & 7)) << 4)),
+                     "r"(pk[4 * pc]), "r"(pk[4 * pc + 1]), "r"(pk[4 * pc + 2]), "r"(pk[4 * pc + 3]) : "memory");
       ptx::fence_proxy_async_smem();
       ptx::tc_fence_before();
-      ptx::mbar_arrive(bar_p);
-      ok = __all_sync(0xffffffffu, gemm_wait(bar_o, j & 1, abort_flag, &g_status));
-      if (!ok) break;
-      ptx::tc_fence_after();
-#pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        uint32_t v[32];
-        ptx::tmem_ld_32x32b_x32(tO + cc * 32, v);
-        ptx::tmem_ld_wait();
-#pragma unroll
-        for (int k = 0; k < 32; ++k) O[cc * 32 + k] = fmaf(O[cc * 32 + k], alpha, __uint_as_float(v[k]));
-      }
+      ptx::mbar_arrive(bar_p);          // P_j is in place, S_j and the previous O_blk have been read
       l = fmaf(l, alpha, rowsum);
       m = mx;
+      alpha_prev = alpha;
+    }
+    float peer_l = 0.f;
+    if (ok) {
+      ok = __all_sync(0xffffffffu, gemm_wait(bar_o, (nblk - 1) & 1, abort_flag, &g_status));
+      if (ok) {
+        ptx::tc_fence_after();
+        take_o(alpha_prev);
+        ok = exchange(l, 2, nblk, peer_l);
+      }
     }
     if (ok && row_ok) {
+      l += peer_l;
       const float inv = 1.0f / l;
-      __nv_bfloat16* dst = a.o + (size_t)i_abs * a.ldo + (size_t)h * DH;
+      __nv_bfloat16* dst = a.o + (size_t)i_abs * a.ldo + (size_t)h * DH + half * (DH / 2);
 #pragma unroll
-      for (int k = 0; k < DH; k += 8) {
+      for (int k = 0; k < DH / 2; k += 8) {
         uint4 w;
         w.x = ptx::pack_bf16(O[k] * inv, O[k + 1] * inv);
         w.y = ptx::pack_bf16(O[k + 2] * inv, O[k + 3] * inv);
@@ -246,7 +300,7 @@ forward_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         w.w = ptx::pack_bf16(O[k + 6] * inv, O[k + 7] * inv);
         *reinterpret_cast<uint4*>(dst + k) = w;
       }
-      a.lse[(size_t)i_abs * a.n_heads + h] = (m + log2f(l)) * 0.6931471805599453f;
+      if (half == 0) a.lse[(size_t)i_abs * a.n_heads + h] = (m + log2f(l)) * 0.6931471805599453f;
     }
   }
 

@@ -1862,7 +1862,7 @@ static mlora_status_t attention_forward_tc(const void* q, int64_t ldq, const voi
   if ((s = make_tmap_bf16(enc, &tK, k, (uint64_t)n_kv * 128, n_rows, ldk, 64, 128)) != MLORA_OK) return s;
   if ((s = make_tmap_bf16_blocked(enc, &tV, v, n_rows, (uint64_t)n_kv * 128, ldv, 64, 2)) != MLORA_OK) return s;
   attn_tc::Args a{(__nv_bfloat16*)o, ldo, lse, seq_start, n_rows, n_heads, n_kv, 1.4426950408889634f / sqrtf(128.0f)};
-  attn_tc::forward_kernel<<<dim3((n_rows + 127) / 128, n_heads), attn_tc::THREADS, attn_tc::SMEM_BYTES, st>>>(tQ, tK, tV, a);
+  attn_tc::forward_kernel<<<dim3((n_rows + 127) / 128, n_heads), attn_tc::FWD_THREADS, attn_tc::SMEM_BYTES, st>>>(tQ, tK, tV, a);
   return launched();
 }
 
