@@ -495,6 +495,7 @@ def main():
                     "achieved": achieved, "unit": "TFLOP/s",
                     "frac_of_burst": achieved / peaks["bf16_tflops"],
                     "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+                    "frac_of_nominal": achieved / 2250.0,      # datasheet dense bf16 figure, context only
                     "flops_per_launch": gemm_fwd_flops / n_launch,
                     "avg_launch_ms": per_kind["gemm_fwd"]["ms_per_step"] / n_launch,
                     "traffic": None}
