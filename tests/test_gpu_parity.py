@@ -394,6 +394,18 @@ def test_many_rows_many_adapters(sess):
     run_and_check(sess, w, synth.make_tensors(w), blocked=True)
 
 
+@pytest.mark.parametrize("rows,d_in,d_out,rank,n_ad,kw", [
+    (70000, 512, 1024, 128, 32, dict(max_seg=5000, p_decode=0.1, p_finetune=0.6)),
+    (50000, 1024, 512, 32, 500, dict(max_seg=40, p_decode=0.8, p_finetune=0.3)),
+])
+def test_batches_beyond_the_tensor_core_rank_r_kernels_limits(sess, rows, d_in, d_out, rank, n_ad, kw):
+    """Tens of thousands of rows: 39616 fine-tuning rows at rank 128 (more 128-row blocks than the operand
+    workspace of the tcgen05 gradient kernel holds), and 8762 segments over 500 adapters (unit lists, item tables
+    and partial-sum workspaces at their largest).  Every element against the oracle."""
+    w = synth.random_workload(7, d_in, d_out, rank, n_ad, rows, **kw)
+    run_and_check(sess, w, synth.make_tensors(w), blocked=True)
+
+
 def test_base_only_rows_and_no_finetune(sess):
     segs = [(0, 40, -1, 0), (60, 30, 1, 0)]      # rows 40..59 and 90..99 uncovered
     w = synth.Workload("base_only", 192, 256, 16, 2, "bf16", 100, synth.segments_array(segs))
