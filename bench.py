@@ -659,6 +659,10 @@ def extra_configs(sess, peaks, headline: str):
     if headline != "cfg5":
         c5 = {m: entry(synth.cfg5_decode_heavy(0, m)) for m in ("decode", "finetune", "mixed")}
         c5["fill_ratio_mixed_over_decode_plus_finetune"] = c5["mixed"]["median_us"] / (c5["decode"]["median_us"] + c5["finetune"]["median_us"])
+        # the same decode rows ordered by adapter (a layout choice of the caller): a 256-row tile then meets 64 adapters
+        # instead of about 110, so the fused expand is 32 instead of 55 extra K-blocks per tile
+        c5["decode_sorted_by_adapter"] = entry(synth.cfg5_decode_heavy(0, "decode", sorted_rows=True))
+        c5["mixed_sorted_by_adapter"] = entry(synth.cfg5_decode_heavy(0, "mixed", sorted_rows=True))
         out["cfg5"] = c5
     out["cfg4"] = [entry(synth.cfg4_sweep_point(r, n, f), reps=20) for r, n, f in ((16, 8, 0.5), (64, 64, 0.25), (128, 256, 0.5))]
     # the same rank-128 point when the 256 adapters have ranks of their own (8 ... 128, stored zero-padded): a plan that

@@ -287,12 +287,17 @@ def cfg4_sweep_point(rank: int, n_adapters: int, ft_fraction: float, seed: int =
     return Workload(nm, 4096, 14336, rank, n_adapters, "bf16", rows, segs, seed=seed)
 
 
-def cfg5_decode_heavy(seed: int = 0, mode: str = "mixed") -> Workload:
-    """5120 -> 13824 bf16, 128 adapters of rank 32; 512 decode rows and/or one 2048-row fine-tune segment."""
+def cfg5_decode_heavy(seed: int = 0, mode: str = "mixed", sorted_rows: bool = False) -> Workload:
+    """5120 -> 13824 bf16, 128 adapters of rank 32; 512 decode rows and/or one 2048-row fine-tune segment.
+
+    The decode rows come in arrival order (a random adapter per row); with ``sorted_rows`` the same rows are
+    ordered by adapter, the layout a serving engine that sorts its decode batch hands over."""
     dec = randint(seed, 501, 512, 128).tolist() if mode in ("mixed", "decode") else []
+    if sorted_rows:
+        dec = sorted(dec)
     ft = [(2048, 127)] if mode in ("mixed", "finetune") else []
     segs, rows = layout_segments([], dec, ft)
-    return Workload(f"cfg5_{mode}", 5120, 13824, 32, 128, "bf16", rows, segs, seed=seed)
+    return Workload(f"cfg5_{mode}" + ("_sorted" if sorted_rows and dec else ""), 5120, 13824, 32, 128, "bf16", rows, segs, seed=seed)
 
 
 def random_workload(seed: int, d_in: int, d_out: int, rank: int, n_adapters: int, n_rows: int,
