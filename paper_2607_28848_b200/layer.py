@@ -103,7 +103,8 @@ class DecoderLayer:
         n_rows = x.shape[0]
         serving = segs.copy()
         serving[:, 3] = 0                           # projection-level saves are not kept: the policy saves the layer input
-        plan = mb.mlora_plan_create(self.sess.ctx, serving, n_rows, self.n_adapters)
+        # a plan per batch, from the context's pool and ordered on the stream: no allocation, no synchronisation
+        plan = mb.mlora_plan_create_async(self.sess.ctx, serving, n_rows, self.n_adapters)
         try:
             def lin(name, inp):
                 pr = self.proj[name]
@@ -112,8 +113,7 @@ class DecoderLayer:
                 return y
             y, _ = self._body(x, lin, segs[segs[:, 1] > 0][:, :2])
         finally:
-            torch.cuda.synchronize()
-            mb.mlora_plan_destroy(plan)
+            mb.mlora_plan_release(plan)
         # activation capture: the residual-stream input of the fine-tuning rows
         for s, n, a, _ in segs[(segs[:, 3] != 0) & (segs[:, 1] > 0)]:
             self.saved_x[self.saved_rows:self.saved_rows + n] = x[s:s + n]
@@ -225,7 +225,7 @@ class DecoderLayer:
         Returns (dx [saved rows, d], {projection: (dA, dB)}, adapters of the gradient slots)."""
         rows = self.saved_rows
         table, _ = self._saved_table(self.saved)
-        self.bwd_plan = mb.mlora_plan_create(self.sess.ctx, table, rows, self.n_adapters)
+        self.bwd_plan = mb.mlora_plan_create_async(self.sess.ctx, table, rows, self.n_adapters)
         self.bwd_slots = mb.mlora_plan_ft_adapters(self.bwd_plan)
         try:
             x = self.saved_x[:rows]
@@ -234,7 +234,7 @@ class DecoderLayer:
             torch.cuda.synchronize()
             return dx, grads, list(self.bwd_slots)
         finally:
-            mb.mlora_plan_destroy(self.bwd_plan)
+            mb.mlora_plan_release(self.bwd_plan)
             self.bwd_plan = None
             self.saved, self.saved_rows = [], 0
 
