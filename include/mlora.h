@@ -104,8 +104,10 @@ void mlora_destroy(mlora_ctx* ctx);
  * rows covered by no segment use the base weight only.
  * With ctx == NULL the plan is host-only (for inspection; it cannot be executed).  With a
  * context the tables are uploaded and the context's workspaces are enlarged if this batch is larger
- * than any before, so this call may allocate device memory and synchronise; the compute calls never
- * do.  An enlarged workspace is a NEW block; the block it replaces stays allocated until
+ * than any before, so this call allocates device (and, for batches whose row tiles differ in cost,
+ * pinned host) memory and synchronises - about two milliseconds for a table of a thousand segments; a
+ * plan that lives for one step is what mlora_plan_create_async below is for.  The compute calls never
+ * allocate or synchronise.  An enlarged workspace is a NEW block; the block it replaces stays allocated until
  * mlora_destroy, so kernels already queued and CUDA graphs captured earlier keep working on memory
  * that is still theirs - creating a larger plan never invalidates an earlier plan or graph.
  * Errors: MLORA_ERR_SEGMENT_RANGE, MLORA_ERR_SEGMENT_OVERLAP, MLORA_ERR_ADAPTER_ID,
