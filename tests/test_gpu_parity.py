@@ -593,6 +593,35 @@ def test_strided_inputs_and_outputs(sess):
     run.close()
 
 
+@pytest.mark.parametrize("rank,path", [(8, 0), (16, 2), (32, 0), (64, 0), (128, 0), (16, 6)])
+def test_row_strides_on_every_operand(sess, rank, path):
+    """X, Y, dY and dX as column slices of wider buffers (row strides 8 to 200 elements beyond the width): the same bits
+    as with packed operands on every kernel family (streaming, per-item, tcgen05 rank-r kernels), nothing written outside."""
+    w = synth.random_workload(500 + rank, 512, 448, rank, 6, 700, max_seg=150, p_decode=0.3, p_finetune=0.5)
+    t = synth.make_tensors(w)
+    mb.mlora_set_gemm_path(sess.ctx, path)
+    run = LayerRun(sess, "bf16", t, w.segments, w.n_rows)
+    try:
+        run.forward(); run.backward()
+        ref = [x.clone() for x in (run.Y, run.u_save, run.x_save, run.dA, run.dB, run.dX)]
+        dev, n = sess.device, run.ft_rows
+        bx = torch.full((w.n_rows, 512 + 24), 3.0, dtype=torch.bfloat16, device=dev); bx[:, 24:] = run.X
+        by = torch.full((w.n_rows, 448 + 200), 7.0, dtype=torch.bfloat16, device=dev)
+        bdy = torch.full((run.dY.shape[0], 448 + 8), 5.0, dtype=torch.bfloat16, device=dev); bdy[:, :448] = run.dY
+        bdx = torch.full((run.dX.shape[0], 512 + 64), 9.0, dtype=torch.bfloat16, device=dev)
+        run.X, run.Y, run.dY, run.dX = bx[:, 24:], by[:, :448], bdy[:, :448], bdx[:, 64:]
+        run.u_save.fill_(float("nan")); run.x_save.fill_(float("nan")); run.dA.fill_(float("nan")); run.dB.fill_(float("nan"))
+        run.forward(); run.backward()
+        assert run.status() == mb.MLORA_OK
+        got = (run.Y, run.u_save, run.x_save, run.dA, run.dB, run.dX)
+        for i, (g, r) in enumerate(zip(got, ref)):
+            assert torch.equal(g[:n], r[:n]) if i in (1, 2, 5) else torch.equal(g, r), i
+        assert (by[:, 448:] == 7.0).all() and (bdx[:, :64] == 9.0).all()
+    finally:
+        mb.mlora_set_gemm_path(sess.ctx, 0)
+        run.close()
+
+
 def test_run_to_run_determinism(sess):
     w = synth.random_workload(23, 256, 320, 32, 5, 500, max_seg=120, p_finetune=0.5)
     t = synth.make_tensors(w)
