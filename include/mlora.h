@@ -103,12 +103,13 @@ void mlora_destroy(mlora_ctx* ctx);
  * schedules of the kernels.  Segments may come in any order; zero-length segments are legal;
  * rows covered by no segment use the base weight only.
  * With ctx == NULL the plan is host-only (for inspection; it cannot be executed).  With a
- * context the tables are uploaded and the context's workspaces are enlarged if this batch is larger
- * than any before, so this call allocates device (and, for batches whose row tiles differ in cost,
- * pinned host) memory and frees it in mlora_plan_destroy: 0.14 ms for a table of a thousand segments when
- * the driver's allocator has pages at hand, 2 to 5 ms when it has to map and unmap them (measured both) or
- * when work is in flight that the freeing call waits for; a plan that lives for one step is what
- * mlora_plan_create_async below is for.  The compute calls never
+ * context the tables are uploaded (through a buffer pair - device tables and pinned staging - taken
+ * from a pool inside the context, on the default stream, and the upload is waited for) and the
+ * context's workspaces are enlarged if this batch is larger than any before.  mlora_plan_destroy
+ * waits for the device and gives the pair back to the pool, so in steady state the two calls make no
+ * cudaMalloc / cudaMallocHost / cudaFree (0.14 ms for a table of a thousand segments; each of those
+ * calls costs milliseconds when the driver has to map or unmap pages).  They still synchronise: a
+ * plan that lives for one step is what mlora_plan_create_async below is for.  The compute calls never
  * allocate or synchronise.  An enlarged workspace is a NEW block; the block it replaces stays allocated until
  * mlora_destroy, so kernels already queued and CUDA graphs captured earlier keep working on memory
  * that is still theirs - creating a larger plan never invalidates an earlier plan or graph.

@@ -167,7 +167,7 @@ struct mlora_plan {
   bool pooled = false;
   DevRowSpace fwd, bwd;
   SchedCache sched[2];               // unit lists of the forward and the compact row space
-  int32_t* sched_pinned = nullptr;   // plans that are not pooled: pinned mirror of the unit-list areas (pooled plans use buf.pinned)
+  int32_t* sched_pinned = nullptr;   // pinned mirror of the unit-list areas of a plan that is not pooled (every plan with a context is pooled now)
   const int32_t* slot_chunk_off = nullptr;
   const int32_t* chunk_row0 = nullptr;
   const int32_t* chunk_nrows = nullptr;
@@ -1373,30 +1373,25 @@ mlora_status_t mlora_plan_create_ranked(mlora_ctx* ctx, const mlora_segment_t* s
                                         int32_t n_adapters, const int32_t* adapter_rank, mlora_plan** out) {
   if (!out) return MLORA_ERR_INVALID_ARG;
   *out = nullptr;
-  mlora_plan* p = new (std::nothrow) mlora_plan();
-  if (!p) return MLORA_ERR_INVALID_ARG;
-  mlora_status_t s = build_plan(segs, n_segs, n_rows, n_adapters, p->h, adapter_rank);
-  if (s != MLORA_OK) { delete p; return s; }
-  p->ctx = ctx;
-  if (ctx) {
-    if (cudaSetDevice(ctx->device) != cudaSuccess) { delete p; return MLORA_ERR_CUDA; }
-    BlobBuilder b;
-    size_t o[kPlanTables];
-    pack_plan(p->h, b, o);
-    const size_t reserve = sched_reserve(p);
-    if (cudaMalloc(&p->blob, (b.data.size() + reserve) * sizeof(int32_t)) != cudaSuccess) { delete p; return MLORA_ERR_CUDA; }
-    if (cudaMemcpy(p->blob, b.data.data(), b.data.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
-      cudaFree(p->blob); delete p; return MLORA_ERR_CUDA;
-    }
-    bind_plan(p, o);
-    if (reserve && cudaMallocHost(&p->sched_pinned, reserve * sizeof(int32_t)) != cudaSuccess) {
-      cudaGetLastError();
-      p->sched_pinned = nullptr;          // no pinned memory: this plan's tiles are dealt out round robin
-    }
-    bind_sched(p, b.data.size(), p->sched_pinned);
-    if ((s = grow_workspaces(ctx, p->h, n_rows)) != MLORA_OK) { mlora_plan_destroy(p); return s; }
+  if (!ctx) {                          // host-only plan: tables for inspection, nothing on a device
+    mlora_plan* p = new (std::nothrow) mlora_plan();
+    if (!p) return MLORA_ERR_INVALID_ARG;
+    const mlora_status_t s = build_plan(segs, n_segs, n_rows, n_adapters, p->h, adapter_rank);
+    if (s != MLORA_OK) { delete p; return s; }
+    *out = p;
+    return MLORA_OK;
   }
-  *out = p;
+  // With a context: the stream-ordered plan on the default stream, and the upload waited for.  The buffer pair
+  // comes from (and mlora_plan_destroy returns it to) the context's pool, so that in steady state this call
+  // makes no cudaMalloc / cudaMallocHost / cudaFree - each of them milliseconds when the driver has to map pages.
+  mlora_status_t s = mlora_plan_create_ranked_async(ctx, segs, n_segs, n_rows, n_adapters, adapter_rank, nullptr, out);
+  if (s != MLORA_OK) return s;
+  if (cudaStreamSynchronize(nullptr) != cudaSuccess) {
+    cudaGetLastError();
+    mlora_plan_destroy(*out);
+    *out = nullptr;
+    return MLORA_ERR_CUDA;
+  }
   return MLORA_OK;
 }
 
@@ -1471,8 +1466,17 @@ mlora_status_t mlora_plan_release(mlora_plan* p, void* cuda_stream) {
 void mlora_plan_destroy(mlora_plan* p) {
   if (!p) return;
   if (p->ctx) cudaSetDevice(p->ctx->device);
-  if (p->pooled) free_plan_buf(p->buf);
-  else if (p->blob) cudaFree(p->blob);
+  if (p->pooled && p->ctx) {
+    // wait for the device (whatever stream used the plan last), then the pair is free for the next plan
+    const bool idle = cudaDeviceSynchronize() == cudaSuccess;
+    if (!idle) cudaGetLastError();
+    if (idle && p->ctx->plan_pool.size() < 64) p->ctx->plan_pool.push_back(p->buf);
+    else free_plan_buf(p->buf);
+  } else if (p->pooled) {
+    free_plan_buf(p->buf);
+  } else if (p->blob) {
+    cudaFree(p->blob);
+  }
   if (p->sched_pinned) cudaFreeHost(p->sched_pinned);
   delete p;
 }
