@@ -240,10 +240,20 @@ def _ptr(t) -> Optional[int]:
     return None if t is None else int(t.data_ptr())
 
 
+_raw_stream = None      # torch's accessor for the current stream's handle (None: not looked up yet, False: absent)
+
+
 def _stream_ptr(stream=None) -> int:
+    """Handle of the given torch stream, or of the current stream of the current device."""
+    global _raw_stream
     import torch
-    s = torch.cuda.current_stream() if stream is None else stream
-    return int(s.cuda_stream)
+    if stream is not None:
+        return int(stream.cuda_stream)
+    if _raw_stream is None:
+        _raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", False)
+    if _raw_stream:         # the handle straight from the runtime: the Stream object costs ten times the call
+        return int(_raw_stream(torch.cuda.current_device()))
+    return int(torch.cuda.current_stream().cuda_stream)
 
 
 def make_layer(W, A_all, B_all, scale) -> mlora_layer_t:
