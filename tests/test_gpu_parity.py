@@ -386,6 +386,24 @@ def test_stream_ordered_plans_from_the_pool(sess):
         run.close()
 
 
+def test_blocking_plans_reuse_the_pool(sess):
+    """mlora_plan_create / mlora_plan_destroy take their buffer pair from the context's pool and give it back: three
+    hundred plans of mixed sizes later the device holds no more memory than after the first few, and a plan made
+    this way computes what the oracle says."""
+    tables = [synth.random_workload(90 + i, 128, 128, 16, 6, 100 + 700 * i, max_seg=50 + 40 * i) for i in range(4)]
+    for w in tables:
+        mb.mlora_plan_destroy(mb.mlora_plan_create(sess.ctx, w.segments, w.n_rows, w.n_adapters))
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for i in range(300):
+        w = tables[i % 4]
+        mb.mlora_plan_destroy(mb.mlora_plan_create(sess.ctx, w.segments, w.n_rows, w.n_adapters))
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free0 - free1 < (8 << 20), (free0, free1)
+    run_and_check(sess, tables[1], synth.make_tensors(tables[1]))
+
+
 def test_many_rows_many_adapters(sess):
     """16384 rows (64 pair tiles), 96 adapters, 5000 fine-tuning rows in ragged segments: the workspaces grow,
     tables and counters stay in range."""
