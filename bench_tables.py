@@ -250,6 +250,27 @@ def table_smallbatch(args):
                     raise RuntimeError("device status non-zero")
                 run.close()
                 lines.append(f"| {d_in} → {d_out} | 256 + {t_ft} | {res[4][0]:.1f} / {res[0][0]:.1f} | {res[4][1]:.1f} / {res[0][1]:.1f} |")
+        # decode-sized forward calls: back to back (launch overlap on), and each kernel with its own event pair
+        lines += ["", "| projection | decode rows | µs per forward call back to back | weight read once at the measured copy bandwidth | shrink / GEMM / reduction (event pairs) |",
+                  "|---|---|---|---|---|"]
+        hbm = load_peaks()["hbm_gbs"]
+        names = {KIND_SHRINK: "shrink", KIND_GEMM_FWD: "gemm", KIND_REDUCE: "reduce"}
+        for rows, d_in, d_out, n_ad in ((16, 4096, 4096, 4), (64, 4096, 4096, 8), (256, 4096, 4096, 32), (64, 4096, 14336, 8), (64, 14336, 4096, 8)):
+            w = synth.random_workload(3, d_in, d_out, 16, n_ad, rows, max_seg=8, p_decode=0.9, p_finetune=0.0)
+            run = LayerRun(sess, w.dtype, synth.make_tensors(w), w.segments, w.n_rows)
+            t_call = timeit(run.forward, n=200)
+            mb.mlora_profile_enable(sess.ctx, 64)
+            acc = {}
+            for _ in range(10):
+                run.forward()
+                torch.cuda.synchronize()
+                kinds, ms = mb.mlora_profile_collect(sess.ctx, 32)
+                for k, m in zip(kinds, ms):
+                    acc.setdefault(int(k), []).append(float(m) * 1e3)
+            mb.mlora_profile_enable(sess.ctx, 0)
+            parts = " / ".join(f"{np.median(acc[k]):.1f}" if k in acc else "—" for k in (KIND_SHRINK, KIND_GEMM_FWD, KIND_REDUCE))
+            run.close()
+            lines.append(f"| {d_in} → {d_out} | {rows} | {t_call:.1f} | {d_in * d_out * 2 / hbm / 1e3:.1f} | {parts} |")
     _emit(lines, args.out)
 
 
