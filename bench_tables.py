@@ -371,22 +371,25 @@ def table_layer_ops(args):
     for name, fn, nbytes in ([] if args.attention_only else rows):
         t = timeit(fn) * 1e-6
         lines.append(f"| {name} | {nbytes / 1e6:.0f} MB | {t * 1e6:.1f} | {nbytes / t / 1e9:.0f} | {nbytes / t / 1e9 / hbm:.2f} |")
-    # attention: 4 sequences of 512 tokens, 32 query heads over 8 kv heads
-    Ta = 2048
-    q = torch.randn(Ta, H * dh, device=dev).to(bf)
-    k, v = (torch.randn(Ta, Hkv * dh, device=dev).to(bf) for _ in range(2))
-    o, dq = torch.empty_like(q), torch.empty_like(q)
-    dk, dv = torch.empty_like(k), torch.empty_like(v)
-    lse = torch.empty(Ta, H, device=dev)
-    ss = (torch.arange(Ta, device=dev, dtype=torch.int32) // 512) * 512
-    se = ss + 512
-    tf = timeit(lambda: mo.mlora_attention_forward(q, k, v, o, lse, ss, se, H, Hkv, dh), n=20) * 1e-6
-    tb = timeit(lambda: mo.mlora_attention_backward(q, k, v, o, lse, q, dq, dk, dv, ss, se, H, Hkv, dh), n=5) * 1e-6
-    fl = 4 * 512 * 513 / 2 * dh * 2 * 2 * H               # QK^T and PV over the causal half, 4 sequences
+    # attention: 32 query heads over 8 kv heads; the first case (4 sequences of 512 tokens) is the one the layer runs
     lines.append("")
-    lines.append(f"attention, 4 sequences x 512 tokens, 32 query / 8 key-value heads of 128: forward (tcgen05 kernel) "
-                 f"{tf * 1e3:.3f} ms ({fl / tf / 1e12:.1f} TFLOP/s over the causal half), backward {tb * 1e3:.2f} ms "
-                 f"({2.5 * fl / tb / 1e12:.1f} TFLOP/s)")
+    for n_seq, L in ((4, 512), (4, 2048), (1, 8192), (16, 128)):
+        Ta = n_seq * L
+        q = torch.randn(Ta, H * dh, device=dev).to(bf)
+        k, v = (torch.randn(Ta, Hkv * dh, device=dev).to(bf) for _ in range(2))
+        o, dq = torch.empty_like(q), torch.empty_like(q)
+        dk, dv = torch.empty_like(k), torch.empty_like(v)
+        lse = torch.empty(Ta, H, device=dev)
+        ss = (torch.arange(Ta, device=dev, dtype=torch.int32) // L) * L
+        se = ss + L
+        tf = timeit(lambda: mo.mlora_attention_forward(q, k, v, o, lse, ss, se, H, Hkv, dh), n=20) * 1e-6
+        tb = timeit(lambda: mo.mlora_attention_backward(q, k, v, o, lse, q, dq, dk, dv, ss, se, H, Hkv, dh), n=5) * 1e-6
+        fl = n_seq * L * (L + 1) / 2 * dh * 2 * 2 * H         # QK^T and PV over the causal half
+        lines.append(f"attention, {n_seq} sequences x {L} tokens, 32 query / 8 key-value heads of 128: forward (tcgen05 kernel) "
+                     f"{tf * 1e3:.3f} ms ({fl / tf / 1e12:.1f} TFLOP/s over the causal half), backward {tb * 1e3:.2f} ms "
+                     f"({2.5 * fl / tb / 1e12:.1f} TFLOP/s)")
+        if mo.mlora_layer_ops_poll_status() != 0:
+            raise RuntimeError("device status non-zero")
     if not args.attention_only:
         lines += ["", whole_layer(dev)]
     _emit(lines, args.out)
